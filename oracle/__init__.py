@@ -1,0 +1,174 @@
+"""Python face of the CPU oracle (oracle/emo_oracle.c).
+
+TEST INFRASTRUCTURE ONLY: imported by tests/, by the smoke check and by the bench's
+CPU-baseline leg.  It imports nothing from the CUDA package and the CUDA package imports nothing
+from here.  The arithmetic lives in the C file; this module only builds it with gcc, loads it
+with ctypes and marshals numpy arrays.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+from concurrent.futures import ThreadPoolExecutor
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "emo_oracle.c")
+_LIB = os.path.join(_HERE, "libemo_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (no fast-math, no contraction)."""
+    with _lock:
+        if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+            tmp = _LIB + f".tmp{os.getpid()}"
+            subprocess.check_call(["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-ffp-contract=off",
+                                   "-Wall", "-Wextra", "-o", tmp, _SRC, "-lm"])
+            os.replace(tmp, _LIB)
+    return _LIB
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        build()
+        L = ctypes.CDLL(_LIB)
+        p = ctypes.c_void_p
+        i32, i64 = ctypes.c_int32, ctypes.c_int64
+        L.emo_oracle_topo.argtypes = [i32, p, p, p]
+        L.emo_oracle_topo.restype = ctypes.c_int
+        L.emo_oracle_durations.argtypes = [i32, i32, p, p, p, p, i64, p, p]
+        L.emo_oracle_durations.restype = ctypes.c_int
+        L.emo_oracle_forward.argtypes = [i32, p, p, p, p, p, p]
+        L.emo_oracle_forward.restype = i64
+        L.emo_oracle_backward.argtypes = [i32, p, p, p, p, i64, p]
+        L.emo_oracle_backward.restype = ctypes.c_int
+        L.emo_oracle_energy.argtypes = [i32, p]
+        L.emo_oracle_energy.restype = ctypes.c_double
+        L.emo_oracle_batch.argtypes = [i32, p, p, i32, p, p, p, p, i64, i64, i64, p, p, p, p, p, i64, i64, p, p]
+        L.emo_oracle_batch.restype = ctypes.c_int
+        L.emo_oracle_target.argtypes = [i64, i64]
+        L.emo_oracle_target.restype = i64
+        L.emo_oracle_select.argtypes = [i64, p, p, i64]
+        L.emo_oracle_select.restype = i64
+        _lib = L
+    return _lib
+
+
+def _ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _c(a, dtype):
+    return np.ascontiguousarray(a, dtype=dtype)
+
+
+class OracleError(RuntimeError):
+    pass
+
+
+def topo_order(n, row_ptr, col) -> np.ndarray:
+    row_ptr = _c(row_ptr, np.int64)
+    col = _c(col, np.int32)
+    order = np.empty(max(n, 1), dtype=np.int32)
+    rc = lib().emo_oracle_topo(n, _ptr(row_ptr), _ptr(col), _ptr(order))
+    if rc:
+        raise OracleError(f"emo_oracle_topo rc={rc}")
+    return order[:n]
+
+
+def forward(n, row_ptr, col, dur, order=None):
+    """One policy given its durations: returns (T, ES, C)."""
+    row_ptr = _c(row_ptr, np.int64)
+    col = _c(col, np.int32)
+    dur = _c(dur, np.int64)
+    order = topo_order(n, row_ptr, col) if order is None else _c(order, np.int32)
+    ES = np.empty(max(n, 1), dtype=np.int64)
+    C = np.empty(max(n, 1), dtype=np.int64)
+    T = lib().emo_oracle_forward(n, _ptr(row_ptr), _ptr(col), _ptr(order), _ptr(dur), _ptr(ES), _ptr(C))
+    return int(T), ES[:n], C[:n]
+
+
+def backward(n, row_ptr, col, dur, T, order=None):
+    row_ptr = _c(row_ptr, np.int64)
+    col = _c(col, np.int32)
+    dur = _c(dur, np.int64)
+    order = topo_order(n, row_ptr, col) if order is None else _c(order, np.int32)
+    LS = np.empty(max(n, 1), dtype=np.int64)
+    rc = lib().emo_oracle_backward(n, _ptr(row_ptr), _ptr(col), _ptr(order), _ptr(dur), int(T), _ptr(LS))
+    if rc:
+        raise OracleError(f"emo_oracle_backward rc={rc}")
+    return LS[:n]
+
+
+def energy_sum(e) -> float:
+    e = _c(e, np.float64)
+    return float(lib().emo_oracle_energy(e.shape[0], _ptr(e)))
+
+
+def batch(g, lvl, B=None, b0=0, b1=None, want_slack=False, want_arrays=False, group_of=None,
+          threads: int = 1):
+    """Evaluate policies b0..b1 of the uint8 level matrix lvl[rows][ldb] on graph g (any object with
+    n, row_ptr, col, L, lat, energy).  Returns a dict of numpy arrays: makespan, energy and, when
+    asked, slack_sum / n_critical and ES / LS / slack as [n][b1-b0].
+
+    threads > 1 only splits the policy range over Python threads; every thread runs the same plain
+    single-policy C routine on its own columns."""
+    lvl = np.ascontiguousarray(lvl, dtype=np.uint8)
+    if lvl.ndim == 1:
+        lvl = lvl.reshape(-1, 1)
+    ldb = lvl.shape[1]
+    B = int(B if B is not None else ldb)
+    b1 = int(B if b1 is None else b1)
+    nb = b1 - b0
+    row_ptr = _c(g.row_ptr, np.int64)
+    col = _c(g.col, np.int32)
+    lat = _c(g.lat, np.int64)
+    en = _c(g.energy, np.float64)
+    go = None if group_of is None else _c(group_of, np.int32)
+    out = {"makespan": np.zeros(B, dtype=np.int64), "energy": np.zeros(B, dtype=np.float64)}
+    if want_slack or want_arrays:
+        out["slack_sum"] = np.zeros(B, dtype=np.int64)
+        out["n_critical"] = np.zeros(B, dtype=np.int32)
+    if want_arrays:
+        for k in ("ES", "LS", "slack"):
+            out[k] = np.zeros((g.n, max(nb, 1)), dtype=np.int64)
+
+    def run(lo, hi):
+        rc = lib().emo_oracle_batch(
+            g.n, _ptr(row_ptr), _ptr(col), g.L, _ptr(lat), _ptr(en), _ptr(go), _ptr(lvl), ldb, lo, hi,
+            _ptr(out["makespan"]), _ptr(out["energy"]),
+            _ptr(out.get("ES")), _ptr(out.get("LS")), _ptr(out.get("slack")), max(nb, 1), b0,
+            _ptr(out.get("slack_sum")), _ptr(out.get("n_critical")))
+        if rc:
+            raise OracleError(f"emo_oracle_batch rc={rc}")
+
+    threads = max(1, min(int(threads), max(nb, 1)))
+    if threads == 1 or nb <= 1:
+        run(b0, b1)
+    else:
+        cuts = np.linspace(b0, b1, threads + 1).astype(np.int64)
+        with ThreadPoolExecutor(threads) as ex:
+            list(ex.map(lambda i: run(int(cuts[i]), int(cuts[i + 1])), range(threads)))
+    out["makespan"] = out["makespan"][b0:b1]
+    out["energy"] = out["energy"][b0:b1]
+    if "slack_sum" in out:
+        out["slack_sum"] = out["slack_sum"][b0:b1]
+        out["n_critical"] = out["n_critical"][b0:b1]
+    return out
+
+
+def target_from_delta(T0: int, delta_ppm: int) -> int:
+    return int(lib().emo_oracle_target(int(T0), int(delta_ppm)))
+
+
+def select(makespan, energy, target: int) -> int:
+    makespan = _c(makespan, np.int64)
+    energy = _c(energy, np.float64)
+    return int(lib().emo_oracle_select(makespan.shape[0], _ptr(makespan), _ptr(energy), int(target)))

@@ -1,0 +1,244 @@
+/*
+ * CPU oracle for the what-if timing / energy evaluation over an execution DAG.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the plain, slow, one-policy-at-a-time restatement of
+ * what the method computes; the CUDA library is checked against it.  It shares no code, header,
+ * table or helper with the CUDA path and must never be linked into or called from it.  Only the
+ * tests, the smoke check and the bench's CPU-baseline leg may call it.
+ *
+ * What each routine follows:
+ *   durations / energies of a policy ........ Eq. 3 (frequency-indexed t_v, e_v; Alg. 1 "dur <- T_f[v], e <- E_f[v]")
+ *   forward pass ............................. Eq. 1 (C_v = t_v + max over predecessors of C_k), Alg. 1 main loop
+ *   makespan ................................. Eq. 2 (T_DAG = max over all v of C_v), Alg. 1 "T <- max comp[v]"
+ *   energy ................................... Eq. 2 without E_idle (sum over v of e_v), Alg. 1 "E_a <- E_a + e"
+ *   backward pass / slack .................... critical-path-method total float; the paper only
+ *                                              describes slack in words (Sec. 1, "time windows where
+ *                                              kernels are not on the critical path"), so the textbook
+ *                                              recurrence is used: LF_v = min over successors of LS_u
+ *                                              (T for sinks), LS_v = LF_v - t_v, slack_v = LS_v - ES_v
+ *   target ................................... Sec. 4.6: T_0 is the makespan at maximum frequency and
+ *                                              the budget is a fraction of it (2 %, 5 % in Sec. 5)
+ *   selection ................................ Eq. 4 over a finite candidate set, with the feasibility
+ *                                              and strict-improvement test of Alg. 2 (first best kept)
+ *
+ * Readings where the paper is silent: a node without predecessors starts at 0; edges carry no lag;
+ * the maximum in Eq. 2 runs over all nodes; energies are summed in node order with Neumaier
+ * compensation in fp64; times are int64 nanoseconds.
+ *
+ * Graph format: predecessor CSR (row_ptr[n+1], col[m]).  The oracle derives its own topological
+ * order (Kahn) and its own successor lists; it never relies on the caller's numbering.
+ *
+ * Parity pins: every routine here is pinned by tests/test_oracle_pins.py (brute-force path
+ * enumeration, closed forms, reversal duality, invariants, a hand-worked example).  Nothing in
+ * this file is "parity unpinned".
+ */
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#include <math.h>
+
+#define ORACLE_OK 0
+#define ORACLE_E_CYCLE (-1)
+#define ORACLE_E_RANGE (-2)
+#define ORACLE_E_ARG (-3)
+#define ORACLE_E_NOMEM (-4)
+
+/* Kahn's algorithm on the predecessor CSR.  order[i] = i-th node of a topological order. */
+int emo_oracle_topo(int32_t n, const int64_t *row_ptr, const int32_t *col, int32_t *order)
+{
+    if (n < 0) return ORACLE_E_ARG;
+    if (n == 0) return ORACLE_OK;
+    int64_t m = row_ptr[n];
+    int32_t *outdeg = calloc((size_t)n, sizeof *outdeg);
+    int64_t *sp = calloc((size_t)n + 1, sizeof *sp);
+    int32_t *succ = malloc(sizeof *succ * (size_t)(m > 0 ? m : 1));
+    int32_t *indeg = malloc(sizeof *indeg * (size_t)n);
+    if (!outdeg || !sp || !succ || !indeg) { free(outdeg); free(sp); free(succ); free(indeg); return ORACLE_E_NOMEM; }
+    for (int32_t v = 0; v < n; ++v) {
+        indeg[v] = (int32_t)(row_ptr[v + 1] - row_ptr[v]);
+        for (int64_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e) {
+            if (col[e] < 0 || col[e] >= n) { free(outdeg); free(sp); free(succ); free(indeg); return ORACLE_E_RANGE; }
+            outdeg[col[e]]++;
+        }
+    }
+    for (int32_t v = 0; v < n; ++v) sp[v + 1] = sp[v] + outdeg[v];
+    memset(outdeg, 0, sizeof *outdeg * (size_t)n);
+    for (int32_t v = 0; v < n; ++v)
+        for (int64_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e) {
+            int32_t k = col[e];
+            succ[sp[k] + outdeg[k]++] = v;
+        }
+    int32_t head = 0, tail = 0;
+    for (int32_t v = 0; v < n; ++v) if (indeg[v] == 0) order[tail++] = v;
+    while (head < tail) {
+        int32_t v = order[head++];
+        for (int64_t e = sp[v]; e < sp[v + 1]; ++e) {
+            int32_t u = succ[e];
+            if (--indeg[u] == 0) order[tail++] = u;
+        }
+    }
+    free(outdeg); free(sp); free(succ); free(indeg);
+    return tail == n ? ORACLE_OK : ORACLE_E_CYCLE;
+}
+
+/* Eq. 3: the duration and energy a policy gives each node.  Node v reads the level of policy row
+ * group_of[v] (v itself when group_of is NULL); a negative group means the node ignores the
+ * policy and uses table column 0.  lvl points at the first row of one policy column, rows are
+ * ld bytes apart. */
+int emo_oracle_durations(int32_t n, int32_t L, const int64_t *lat, const double *energy,
+                         const int32_t *group_of, const uint8_t *lvl, int64_t ld,
+                         int64_t *dur, double *e)
+{
+    for (int32_t v = 0; v < n; ++v) {
+        int32_t r = group_of ? group_of[v] : v;
+        int32_t l = 0;
+        if (r >= 0) {
+            l = lvl[(int64_t)r * ld];
+            if (l >= L) return ORACLE_E_RANGE;
+        }
+        dur[v] = lat[(int64_t)v * L + l];
+        if (e) e[v] = energy[(int64_t)v * L + l];
+    }
+    return ORACLE_OK;
+}
+
+/* Eq. 1 in topological order.  ES_v = max(0, max_k C_k), C_v = ES_v + dur_v.  Returns the
+ * makespan of Eq. 2, the maximum of C_v over ALL nodes. */
+int64_t emo_oracle_forward(int32_t n, const int64_t *row_ptr, const int32_t *col,
+                           const int32_t *order, const int64_t *dur, int64_t *ES, int64_t *C)
+{
+    int64_t T = 0;
+    for (int32_t i = 0; i < n; ++i) {
+        int32_t v = order[i];
+        int64_t start = 0;
+        for (int64_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e) {
+            int64_t ck = C[col[e]];
+            if (ck > start) start = ck;
+        }
+        ES[v] = start;
+        C[v] = start + dur[v];
+        if (C[v] > T) T = C[v];
+    }
+    return T;
+}
+
+/* Backward pass, written independently of the forward one: explicit successor lists, nodes in
+ * reverse topological order.  LF_v = T for a node without successors, else min over successors
+ * of LS_u;  LS_v = LF_v - dur_v. */
+int emo_oracle_backward(int32_t n, const int64_t *row_ptr, const int32_t *col,
+                        const int32_t *order, const int64_t *dur, int64_t T, int64_t *LS)
+{
+    int64_t m = n > 0 ? row_ptr[n] : 0;
+    int64_t *sp = calloc((size_t)n + 2, sizeof *sp);
+    int32_t *succ = malloc(sizeof *succ * (size_t)(m > 0 ? m : 1));
+    int64_t *fill = calloc((size_t)n + 1, sizeof *fill);
+    if (!sp || !succ || !fill) { free(sp); free(succ); free(fill); return ORACLE_E_NOMEM; }
+    for (int64_t e = 0; e < m; ++e) sp[col[e] + 1]++;
+    for (int32_t v = 0; v < n; ++v) sp[v + 1] += sp[v];
+    for (int32_t v = 0; v < n; ++v)
+        for (int64_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e) {
+            int32_t k = col[e];
+            succ[sp[k] + fill[k]++] = v;
+        }
+    for (int32_t i = n - 1; i >= 0; --i) {
+        int32_t v = order[i];
+        int64_t lf;
+        if (sp[v + 1] == sp[v]) {
+            lf = T;
+        } else {
+            lf = LS[succ[sp[v]]];
+            for (int64_t e = sp[v] + 1; e < sp[v + 1]; ++e) {
+                int64_t x = LS[succ[e]];
+                if (x < lf) lf = x;
+            }
+        }
+        LS[v] = lf - dur[v];
+    }
+    free(sp); free(succ); free(fill);
+    return ORACLE_OK;
+}
+
+/* Sum of the node energies in node order, Neumaier-compensated, fp64. */
+double emo_oracle_energy(int32_t n, const double *e)
+{
+    double sum = 0.0, comp = 0.0;   /* built without -ffast-math: no reassociation */
+    for (int32_t v = 0; v < n; ++v) {
+        double x = e[v];
+        double t = sum + x;
+        if (fabs(sum) >= fabs(x)) comp += (sum - t) + x;
+        else comp += (x - t) + sum;
+        sum = t;
+    }
+    return sum + comp;
+}
+
+/* Policies b0 <= b < b1 of a level matrix lvl[rows][ldb], one at a time.
+ * Outputs (each may be NULL): makespan[B], energy_out[B] indexed by b; ES/LS/slack laid out
+ * [n][ldo] with column b - ocol0 (so a caller can ask for a slab of columns); slack_sum[B],
+ * n_critical[B] (nodes with slack 0). */
+int emo_oracle_batch(int32_t n, const int64_t *row_ptr, const int32_t *col, int32_t L,
+                     const int64_t *lat, const double *energy, const int32_t *group_of,
+                     const uint8_t *lvl, int64_t ldb, int64_t b0, int64_t b1,
+                     int64_t *makespan, double *energy_out,
+                     int64_t *ES_out, int64_t *LS_out, int64_t *slack_out, int64_t ldo, int64_t ocol0,
+                     int64_t *slack_sum, int32_t *n_critical)
+{
+    if (n < 0 || L < 1 || b0 < 0 || b1 < b0) return ORACLE_E_ARG;
+    size_t nn = (size_t)(n > 0 ? n : 1);
+    int32_t *order = malloc(sizeof *order * nn);
+    int64_t *dur = malloc(sizeof *dur * nn), *ES = malloc(sizeof *ES * nn);
+    int64_t *C = malloc(sizeof *C * nn), *LS = malloc(sizeof *LS * nn);
+    double *e = malloc(sizeof *e * nn);
+    int rc = ORACLE_OK;
+    if (!order || !dur || !ES || !C || !LS || !e) { rc = ORACLE_E_NOMEM; goto done; }
+    rc = emo_oracle_topo(n, row_ptr, col, order);
+    if (rc) goto done;
+    int need_back = ES_out || LS_out || slack_out || slack_sum || n_critical;
+    for (int64_t b = b0; b < b1; ++b) {
+        rc = emo_oracle_durations(n, L, lat, energy, group_of, lvl + b, ldb, dur, e);
+        if (rc) goto done;
+        int64_t T = emo_oracle_forward(n, row_ptr, col, order, dur, ES, C);
+        if (makespan) makespan[b] = T;
+        if (energy_out) energy_out[b] = emo_oracle_energy(n, e);
+        if (need_back) {
+            rc = emo_oracle_backward(n, row_ptr, col, order, dur, T, LS);
+            if (rc) goto done;
+            int64_t ssum = 0;
+            int32_t ncrit = 0;
+            for (int32_t v = 0; v < n; ++v) {
+                int64_t s = LS[v] - ES[v];
+                ssum += s;
+                ncrit += (s == 0);
+                int64_t o = (int64_t)v * ldo + (b - ocol0);
+                if (ES_out) ES_out[o] = ES[v];
+                if (LS_out) LS_out[o] = LS[v];
+                if (slack_out) slack_out[o] = s;
+            }
+            if (slack_sum) slack_sum[b] = ssum;
+            if (n_critical) n_critical[b] = ncrit;
+        }
+    }
+done:
+    free(order); free(dur); free(ES); free(C); free(LS); free(e);
+    return rc;
+}
+
+/* T_set = T_0 + floor(T_0 * delta_ppm / 10^6): the latency budget relative to the
+ * maximum-frequency makespan (Sec. 4.6; budgets of 2 % and 5 % in Sec. 5). */
+int64_t emo_oracle_target(int64_t T0, int64_t delta_ppm)
+{
+    __int128 x = (__int128)T0 * (__int128)delta_ppm;
+    return T0 + (int64_t)(x / 1000000);
+}
+
+/* Eq. 4 over a finite batch: the feasible policy (T <= target) of least energy; a later policy
+ * replaces the incumbent only if strictly better (Alg. 2), so ties go to the lowest index.
+ * Returns -1 when no policy is feasible. */
+int64_t emo_oracle_select(int64_t B, const int64_t *makespan, const double *energy, int64_t target)
+{
+    int64_t best = -1;
+    for (int64_t b = 0; b < B; ++b) {
+        if (makespan[b] <= target && (best < 0 || energy[b] < energy[best])) best = b;
+    }
+    return best;
+}
