@@ -1,0 +1,215 @@
+/*
+ * emo.h - C ABI of the batched what-if timing and energy evaluator for kernel dependency graphs.
+ *
+ * The library evaluates many candidate frequency-level policies at once on one execution graph:
+ * earliest start times by a max-plus forward pass (Eq. 1) giving the makespan (Eq. 2), latest
+ * start times by a backward pass giving per-node slack, total energy from frequency-indexed
+ * per-node tables (Eq. 2, Eq. 3), and the least-energy policy within a latency budget (Eq. 4).
+ * All of it runs in CUDA kernels for sm_100a; there is no CPU fallback.
+ *
+ * Conventions
+ *   - Every function returns an int: EMO_OK (0) or a negative EMO_E_* code.  Nothing throws or
+ *     aborts across this boundary.  Output parameters are written only on success.
+ *   - "host" / "device" on a pointer says where the memory lives.  Device pointers are borrowed
+ *     until the work queued on `stream` has completed; the library never frees caller memory.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls that take a
+ *     stream are asynchronous: they queue kernels and return.
+ *   - A graph handle is immutable after emo_graph_load and may be shared by concurrent calls that
+ *     use distinct workspaces and streams.
+ *   - Notation: n nodes, m edges, L frequency levels (level L-1 = maximum frequency, the
+ *     default), B policies.  A policy assigns a level to every policy row; node v reads row
+ *     group_of[v] (row v when no grouping was given).  Times are int64 nanoseconds, energies
+ *     fp64 joules.
+ *   - Level matrix layout: lvl[r * ldb + b] is the level policy b gives row r (uint8, row-major
+ *     over rows, policies contiguous).  Per-node outputs use the same shape: X[v * ldo + b].
+ */
+#ifndef EMO_H_
+#define EMO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define EMO_OK 0
+#define EMO_E_INVALID_ARG (-1)     /* NULL where a pointer is required, negative size, bad ld */
+#define EMO_E_NOT_TOPOLOGICAL (-2) /* an edge does not go from a lower to a higher node number */
+#define EMO_E_RANGE (-3)           /* value outside the supported range (level >= L, lat >= 2^32, ...) */
+#define EMO_E_OVERFLOW (-4)        /* the slowest-level makespan does not stay below 2^62 ns */
+#define EMO_E_NONFINITE (-5)       /* NaN or infinity in the energy table */
+#define EMO_E_OOM (-6)             /* host or device allocation failed, or workspace too small */
+#define EMO_E_CUDA (-7)            /* a CUDA runtime call failed (no device, launch error, ...) */
+#define EMO_E_TIMEOUT (-8)         /* a bounded device-side wait ran out; results are invalid */
+#define EMO_E_UNSUPPORTED (-9)     /* the graph needs more on-chip exchange slots than exist */
+
+/* flags of emo_graph_load */
+#define EMO_F_HOST_ONLY 0x1u       /* build the handle without touching a device (inspection) */
+#define EMO_F_LANES(c) (((uint32_t)(c) & 0xFFu) << 8)      /* force c cooperating warps per policy group */
+#define EMO_F_LOOKAHEAD(d) (((uint32_t)(d) & 0xFFu) << 16) /* scheduling look-ahead in steps */
+/* flags of the evaluation calls */
+#define EMO_F_VALIDATE 0x1u        /* check every level < L first; EMO_E_RANGE goes to *status */
+#define EMO_F_NO_STAGING 0x2u      /* use the plain-load kernels instead of the staged ones */
+
+typedef struct emo_graph emo_graph;
+
+typedef struct emo_info {
+    int32_t n;          /* nodes */
+    int64_t m;          /* edges as given (duplicates included) */
+    int32_t L;          /* frequency levels */
+    int32_t rows;       /* policy rows (max group + 1, or n) */
+    int32_t depth;      /* number of hop-count levels */
+    int32_t max_span;   /* largest v - pred(v) in the caller's numbering */
+    int64_t T_worst;    /* makespan with every node at its slowest level */
+    int64_t T_best;     /* makespan with every node at its fastest level */
+    int32_t lanes;      /* warps that cooperate on one group of 32 policies */
+    int32_t steps_fwd, slots_fwd, aux_fwd;   /* forward program: steps, exchange slots, helper ops */
+    int32_t steps_bwd, slots_bwd, aux_bwd;   /* backward program */
+} emo_info;
+
+/* Human-readable text for a status code (static storage). */
+const char *emo_strerror(int code);
+
+/*
+ * emo_graph_load - take an execution graph (Sec. 4.3: nodes are execution primitives, an edge
+ * (i, j) means i must finish before j starts) with its frequency-indexed tables (Eq. 3) and
+ * prepare it for evaluation.
+ *   n, row_ptr[n+1], col[m]   host. Predecessor CSR: predecessors of v are col[row_ptr[v] ..
+ *                             row_ptr[v+1]).  Nodes must be numbered topologically (every
+ *                             predecessor < v); level-ordered numbering is the usual case.
+ *                             Duplicate edges and isolated nodes are allowed.
+ *   level_ptr[n_levels+1]     host, optional (NULL): node ranges of the caller's levels; when given
+ *                             it is checked (every predecessor in a strictly lower level).
+ *   L                         1..255 levels.
+ *   lat[n][L]                 host, int64 ns, 0 <= lat < 2^32.
+ *   energy[n][L]              host, fp64, finite.
+ *   group_of[n]               host, optional: policy row of each node; -1 = the node ignores the
+ *                             policy and uses table column 0.
+ *   flags                     EMO_F_* of emo_graph_load.
+ *   out                       receives the handle.
+ * Everything is copied; the caller may free its arrays on return.  The device copies belong to
+ * the handle until emo_graph_free.  Not asynchronous: it synchronises the device copies it makes.
+ * Errors: INVALID_ARG, NOT_TOPOLOGICAL, RANGE, OVERFLOW, NONFINITE, OOM, CUDA, UNSUPPORTED.
+ */
+int emo_graph_load(int32_t n, const int64_t *row_ptr, const int32_t *col,
+                   const int32_t *level_ptr, int32_t n_levels, int32_t L,
+                   const int64_t *lat, const double *energy, const int32_t *group_of,
+                   uint32_t flags, emo_graph **out);
+
+/* Release a handle and its device memory.  NULL is allowed. */
+int emo_graph_free(emo_graph *g);
+
+/* Sizes and derived facts of a loaded graph. */
+int emo_graph_info(const emo_graph *g, emo_info *info);
+
+/*
+ * emo_workspace_bytes - device scratch a call on B policies needs.  need_slack = 0 gives the size
+ * for emo_eval_policies, emo_baseline and emo_select; 1 the size emo_slack_batch needs when the
+ * caller passes no ES array (the earliest start times are then kept in the workspace between the
+ * two passes); 2 the size emo_slack_batch_host needs.  The caller allocates; no call allocates
+ * device memory per invocation.
+ */
+int emo_workspace_bytes(const emo_graph *g, int64_t B, int need_slack, size_t *out);
+
+/*
+ * emo_eval_policies - Alg. 1 without the idle-energy loop, for B policies at once:
+ * makespan[b] = max_v C_v (Eq. 1, Eq. 2) and energy[b] = sum_v e_v (Eq. 2) under policy b.
+ *   lvl          device uint8 [rows][ldb], ldb >= B.
+ *   makespan     device int64 [B];  energy  device fp64 [B].
+ *   ws, ws_bytes device scratch of at least emo_workspace_bytes(g, B, 0).
+ *   status       device int32, optional: set to a negative code if a kernel detected an error
+ *                (left untouched otherwise; the caller zeroes it).
+ * B == 0 returns EMO_OK and writes nothing.  Asynchronous on `stream`.
+ */
+int emo_eval_policies(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t ldb,
+                      int64_t *makespan, double *energy, void *ws, size_t ws_bytes,
+                      int32_t *status, uint32_t flags, void *stream);
+
+/*
+ * emo_slack_batch - forward and backward pass for B policies: earliest start ES, latest start LS
+ * (critical-path backward pass: LF_v = min over successors of LS_u, the makespan for nodes
+ * without successors; LS_v = LF_v - t_v) and slack = LS - ES per node and policy.
+ *   ES, LS, slack   device int64 [n][ldo], each optional (NULL); ldo >= B.
+ *   makespan, energy device [B] (required).
+ *   slack_sum       device int64 [B], optional: sum of slack over nodes.
+ *   n_critical      device int32 [B], optional: number of nodes with slack 0.
+ *   ws              at least emo_workspace_bytes(g, B, ES == NULL).
+ * Asynchronous on `stream`.
+ */
+int emo_slack_batch(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t ldb,
+                    int64_t *ES, int64_t *LS, int64_t *slack, int64_t ldo,
+                    int64_t *makespan, double *energy, int64_t *slack_sum, int32_t *n_critical,
+                    void *ws, size_t ws_bytes, int32_t *status, uint32_t flags, void *stream);
+
+/*
+ * emo_slack - one policy: lvl_one is device uint8 [rows]; ES, LS, slack are device int64 [n]
+ * (each optional); makespan device int64 [1], energy device fp64 [1] (optional).
+ */
+int emo_slack(const emo_graph *g, const uint8_t *lvl_one, int64_t *ES, int64_t *LS, int64_t *slack,
+              int64_t *makespan, double *energy, void *ws, size_t ws_bytes, int32_t *status,
+              void *stream);
+
+/*
+ * emo_baseline - T_0 and E_0 of the default policy, every row at level L-1 (Alg. 2 line 1-2:
+ * P_0 = default frequency everywhere; Sec. 4.6: T_0 is the latency at maximum frequency).
+ * T0 device int64 [1], E0 device fp64 [1].
+ */
+int emo_baseline(const emo_graph *g, int64_t *T0, double *E0, void *ws, size_t ws_bytes,
+                 int32_t *status, void *stream);
+
+/* T_set = T0 + floor(T0 * delta_ppm / 10^6), exact in 128-bit.  Pure host function. */
+int64_t emo_target_from_delta(int64_t T0, int64_t delta_ppm);
+
+/*
+ * emo_select - Eq. 4 over the batch: the index of the least-energy policy among those with
+ * makespan[b] <= target; equal energies go to the lowest index (the strict-improvement test of
+ * Alg. 2 keeps the incumbent).  out_index receives -1 when no policy is feasible (still EMO_OK).
+ *   makespan, energy  device [B];  out_index device int64 [1];  out_T device int64 [1] and
+ *   out_E device fp64 [1] (optional) receive the selected policy's values.
+ *   target_dev        optional device int64 [1]: when not NULL the target is read from it on the
+ *                     device (so a budget computed from emo_baseline needs no host round trip)
+ *                     as target_dev[0] + floor(target_dev[0] * delta_ppm / 10^6) and `target` is
+ *                     ignored; when NULL, `target` is used and delta_ppm ignored.
+ */
+int emo_select(int64_t B, const int64_t *makespan, const double *energy, int64_t target,
+               const int64_t *target_dev, int64_t delta_ppm,
+               int64_t *out_index, int64_t *out_T, double *out_E,
+               void *ws, size_t ws_bytes, void *stream);
+
+/*
+ * emo_transpose_policies - layout helper: src device uint8 [B][lds] (one policy per row) to
+ * dst device uint8 [rows][ldb].
+ */
+int emo_transpose_policies(int64_t B, int64_t rows, const uint8_t *src, int64_t lds,
+                           uint8_t *dst, int64_t ldb, void *stream);
+
+/*
+ * emo_slack_batch_host - the same computation as emo_slack_batch followed by emo_baseline and
+ * emo_select, driven from host memory: lvl_host is host uint8 [rows][ldb] (pinned memory gives
+ * the best copy rate); makespan_host, energy_host, slack_sum_host, n_critical_host are host
+ * arrays [B] (the last two optional); sel_host receives {index, T, E-bits, T0} as 4 int64.
+ * slack_dev (device int64 [n][ldo], optional) stays on the device.  dev_lvl is a device buffer
+ * of rows*ldb bytes and ws a device workspace of emo_workspace_bytes(g, B, 2).
+ * The call copies the levels in, runs the passes, copies the per-policy results out and waits
+ * for the stream.
+ */
+int emo_slack_batch_host(const emo_graph *g, int64_t B, const uint8_t *lvl_host, int64_t ldb,
+                         uint8_t *dev_lvl, int64_t *slack_dev, int64_t ldo, int64_t delta_ppm,
+                         int64_t *makespan_host, double *energy_host, int64_t *slack_sum_host,
+                         int32_t *n_critical_host, int64_t *sel_host,
+                         void *ws, size_t ws_bytes, uint32_t flags, void *stream);
+
+/*
+ * Inspection of the compiled evaluation program (host memory owned by the handle; valid until
+ * emo_graph_free).  dir 0 = forward, 1 = backward.  entries is [steps][lanes][4] uint32,
+ * lat is uint32 [steps*lanes][Lp], Lp = row stride (a power of two >= L).  Used by host-side
+ * tests of the scheduler; not needed to evaluate anything.
+ */
+int emo_graph_program(const emo_graph *g, int dir, int32_t *lanes, int32_t *steps, int32_t *slots,
+                      int32_t *Lp, const uint32_t **entries, const uint32_t **lat);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EMO_H_ */

@@ -1,0 +1,357 @@
+// Step-program compiler: list scheduling of the (forward or reversed) DAG onto `lanes` warps,
+// register/slot assignment for the values that flow along edges, and the schedule-ordered copies
+// of the duration and energy tables (Eq. 3) the kernels stream through.
+#include "emo_compile.h"
+
+#include <algorithm>
+#include <climits>
+#include <queue>
+
+#include "../../include/emo.h"
+
+namespace emo {
+
+namespace {
+
+struct Op {
+    int32_t node;                 // caller's node id, -1 for a helper op that only takes a maximum
+    std::vector<int32_t> preds;   // op indices whose values this op needs
+};
+
+// A node with more operands than one entry can name is split: helper ops take the maximum of up
+// to kMaxSlotPreds operands each (duration 0, no output), and the node reads the helpers.
+void add_with_helpers(std::vector<Op> &ops, int32_t node, std::vector<int32_t> preds, int &n_aux)
+{
+    std::sort(preds.begin(), preds.end());
+    preds.erase(std::unique(preds.begin(), preds.end()), preds.end());
+    while ((int)preds.size() > kMaxSlotPreds) {
+        Op h;
+        h.node = -1;
+        h.preds.assign(preds.begin(), preds.begin() + kMaxSlotPreds);
+        preds.erase(preds.begin(), preds.begin() + kMaxSlotPreds);
+        preds.push_back((int32_t)ops.size());
+        ops.push_back(std::move(h));
+        ++n_aux;
+    }
+    Op o;
+    o.node = node;
+    o.preds = std::move(preds);
+    ops.push_back(std::move(o));
+}
+
+}  // namespace
+
+int pick_lanes(int64_t n_ops, int depth)
+{
+    if (depth <= 0) return 1;
+    // a little spare capacity (10 %) lets the list scheduler catch up after a narrow stretch
+    int64_t c = (n_ops * 11 + (int64_t)depth * 10 - 1) / ((int64_t)depth * 10);
+    if (c < 1) c = 1;
+    if (c > kMaxLanes) c = kMaxLanes;
+    return (int)c;
+}
+
+int compile_program(const HostGraph &g, const int64_t *lat, const double *energy, bool backward,
+                    int lanes, int lookahead, Program &out, std::string &err)
+{
+    const int32_t n = g.n;
+    const int L = g.L;
+    int Lp = 1;
+    while (Lp < L) Lp <<= 1;
+    out = Program();
+    out.Lp = Lp;
+
+    // ---- ops in a topological order of the direction being compiled --------------------------
+    std::vector<Op> ops;
+    ops.reserve((size_t)n + 16);
+    std::vector<int32_t> op_of_node((size_t)std::max(n, 1), -1);
+    int n_aux = 0;
+    if (!backward) {
+        for (int32_t v = 0; v < n; ++v) {
+            std::vector<int32_t> p;
+            for (int64_t e = g.row_ptr[v]; e < g.row_ptr[v + 1]; ++e) p.push_back(op_of_node[g.col[e]]);
+            add_with_helpers(ops, v, std::move(p), n_aux);
+            op_of_node[v] = (int32_t)ops.size() - 1;
+        }
+    } else {
+        std::vector<int64_t> sp((size_t)n + 1, 0);
+        for (int64_t e = 0; e < g.m; ++e) sp[g.col[e] + 1]++;
+        for (int32_t v = 0; v < n; ++v) sp[v + 1] += sp[v];
+        std::vector<int32_t> succ((size_t)std::max<int64_t>(g.m, 1));
+        std::vector<int64_t> fill(sp.begin(), sp.end() - 1);
+        for (int32_t v = 0; v < n; ++v)
+            for (int64_t e = g.row_ptr[v]; e < g.row_ptr[v + 1]; ++e) succ[fill[g.col[e]]++] = v;
+        for (int32_t v = n - 1; v >= 0; --v) {
+            std::vector<int32_t> p;
+            for (int64_t e = sp[v]; e < sp[v + 1]; ++e) p.push_back(op_of_node[succ[e]]);
+            add_with_helpers(ops, v, std::move(p), n_aux);
+            op_of_node[v] = (int32_t)ops.size() - 1;
+        }
+    }
+    const int32_t N = (int32_t)ops.size();
+    out.aux = n_aux;
+
+    // consumers of each op
+    std::vector<int64_t> cp((size_t)N + 1, 0);
+    for (int32_t i = 0; i < N; ++i)
+        for (int32_t p : ops[i].preds) cp[p + 1]++;
+    for (int32_t i = 0; i < N; ++i) cp[i + 1] += cp[i];
+    std::vector<int32_t> cons((size_t)std::max<int64_t>(cp[N], 1));
+    {
+        std::vector<int64_t> f(cp.begin(), cp.end() - 1);
+        for (int32_t i = 0; i < N; ++i)
+            for (int32_t p : ops[i].preds) cons[f[p]++] = i;
+    }
+
+    // hop levels: earliest step (asap) and the number of hops to the end (rem; alap = D - rem)
+    std::vector<int32_t> asap((size_t)N, 0), rem((size_t)N, 1), tgt((size_t)N, 0);
+    int32_t D = 0;
+    for (int32_t i = 0; i < N; ++i) {
+        int32_t a = 0;
+        for (int32_t p : ops[i].preds) a = std::max(a, asap[p] + 1);
+        asap[i] = a;
+        D = std::max(D, a + 1);
+    }
+    for (int32_t i = N - 1; i >= 0; --i) {
+        int32_t r = 1;
+        for (int64_t e = cp[i]; e < cp[i + 1]; ++e) r = std::max(r, rem[cons[e]] + 1);
+        rem[i] = r;
+    }
+    // Target steps.  A value occupies an exchange slot from the step that produces it to the step
+    // of its last consumer, so the targets are moved, within the precedence constraints, to
+    // shorten the summed lifetimes: starting from the earliest steps, a backward sweep moves an op
+    // later (next to its earliest consumer) when that shortens its own value's life by more than
+    // it stretches its operands' lives, and a forward sweep moves an op earlier under the mirrored
+    // test.  This puts a chain that has hop slack (a launch chain running ahead of the kernels, or
+    // short streams beside a long launch chain) next to the ops it exchanges values with.
+    // Two starting points are refined, all ops at their earliest and all at their latest steps,
+    // and the one with the smaller summed lifetime is kept.
+    auto last_cons_excl = [&](int32_t p, int32_t skip) {
+        int32_t m = -1;
+        for (int64_t e = cp[p]; e < cp[p + 1]; ++e)
+            if (cons[e] != skip) m = std::max(m, tgt[cons[e]]);
+        return m;
+    };
+    auto sweep_later = [&]() {
+        for (int32_t i = N - 1; i >= 0; --i) {
+            if (cp[i + 1] == cp[i]) continue;
+            int32_t hi = INT32_MAX;
+            for (int64_t e = cp[i]; e < cp[i + 1]; ++e) hi = std::min(hi, tgt[cons[e]] - 1);
+            if (hi <= tgt[i]) continue;
+            int64_t gain = hi - tgt[i], cost = 0;
+            for (int32_t p : ops[i].preds) {
+                if (cp[p + 1] - cp[p] == 1) continue;   // its only consumer: it follows later in this sweep
+                int32_t other = last_cons_excl(p, i);
+                cost += std::max(other, hi) - std::max(other, tgt[i]);
+            }
+            if (gain > cost) tgt[i] = hi;
+        }
+    };
+    auto sweep_earlier = [&]() {
+        for (int32_t i = 0; i < N; ++i) {
+            if (ops[i].preds.empty()) continue;
+            int32_t lo = 0;
+            for (int32_t p : ops[i].preds) lo = std::max(lo, tgt[p] + 1);
+            if (lo >= tgt[i]) continue;
+            bool held = false;   // a consumer with other operands keeps this op's value alive
+            for (int64_t e = cp[i]; e < cp[i + 1]; ++e) held |= ops[cons[e]].preds.size() > 1;
+            int64_t cost = held ? tgt[i] - lo : 0, gain = 0;
+            for (int32_t p : ops[i].preds) {
+                int32_t other = last_cons_excl(p, i);
+                gain += std::max(other, tgt[i]) - std::max(other, lo);
+            }
+            if (gain > cost) tgt[i] = lo;
+        }
+    };
+    auto total_life = [&]() {
+        int64_t sum = 0;
+        for (int32_t i = 0; i < N; ++i) {
+            int32_t m = last_cons_excl(i, -1);
+            if (m >= 0) sum += m - tgt[i];
+        }
+        return sum;
+    };
+    tgt = asap;
+    for (int round = 0; round < 2; ++round) { sweep_later(); sweep_earlier(); }
+    const int64_t life_early = total_life();
+    std::vector<int32_t> tgt_early = tgt;
+    for (int32_t i = 0; i < N; ++i) tgt[i] = D - rem[i];
+    for (int round = 0; round < 2; ++round) { sweep_earlier(); sweep_later(); }
+    if (life_early <= total_life()) tgt.swap(tgt_early);
+    if (lanes <= 0) lanes = pick_lanes(N, D);
+    if (lanes > kMaxLanes) lanes = kMaxLanes;
+    if (lookahead <= 0) lookahead = 8;
+    out.lanes = lanes;
+
+    // ---- list scheduling ----------------------------------------------------------------------
+    // Priority: smallest target step first (ties: the more critical op).  An op is not started more
+    // than `lookahead` steps before its target step, which keeps a cheap chain from running far
+    // ahead of the ops that consume its values.
+    std::vector<int32_t> step_of((size_t)N, -1), warp_of((size_t)N, -1), prev_on_warp((size_t)N, -1);
+    std::vector<int32_t> left((size_t)N);
+    std::vector<int32_t> unsched_cons((size_t)N);
+    using Key = std::pair<int64_t, int32_t>;   // (target step, alap | op)
+    std::priority_queue<Key, std::vector<Key>, std::greater<Key>> ready;
+    auto prio = [&](int32_t i) { return ((int64_t)tgt[i] << 32) | (uint32_t)(D - rem[i]); };
+    for (int32_t i = 0; i < N; ++i) {
+        left[i] = (int32_t)ops[i].preds.size();
+        unsched_cons[i] = (int32_t)(cp[i + 1] - cp[i]);
+        if (left[i] == 0) ready.push({prio(i), i});
+    }
+    std::vector<int32_t> last((size_t)lanes, -1);
+    std::vector<std::vector<int32_t>> sched;   // per step: op per warp (-1 idle)
+    std::vector<int32_t> chosen, next_ready;
+    int32_t done = 0;
+    int32_t t = 0;
+    while (done < N) {
+        chosen.clear();
+        while (!ready.empty() && (int)chosen.size() < lanes) {
+            Key k = ready.top();
+            // an op that is not due yet waits, unless the step would otherwise be empty
+            if ((k.first >> 32) > t + lookahead && !chosen.empty()) break;
+            ready.pop();
+            chosen.push_back(k.second);
+        }
+        std::vector<int32_t> row((size_t)lanes, -1);
+        std::vector<char> placed(chosen.size(), 0);
+        // first the ops whose operand sits in a free warp's register
+        for (size_t j = 0; j < chosen.size(); ++j) {
+            int32_t i = chosen[j];
+            for (int32_t p : ops[i].preds) {
+                int w = warp_of[p];
+                if (w >= 0 && last[w] == p && row[w] < 0) {
+                    row[w] = i;
+                    placed[j] = 1;
+                    break;
+                }
+            }
+        }
+        // then the rest: prefer a warp whose register value nobody is waiting for
+        for (size_t j = 0; j < chosen.size(); ++j) {
+            if (placed[j]) continue;
+            int best = -1;
+            for (int w = 0; w < lanes; ++w) {
+                if (row[w] >= 0) continue;
+                bool dead = last[w] < 0 || unsched_cons[last[w]] == 0;
+                if (dead) { best = w; break; }
+                if (best < 0) best = w;
+            }
+            row[best] = chosen[j];
+        }
+        next_ready.clear();
+        for (int w = 0; w < lanes; ++w) {
+            int32_t i = row[w];
+            if (i < 0) continue;
+            step_of[i] = t;
+            warp_of[i] = w;
+            prev_on_warp[i] = last[w];
+            ++done;
+        }
+        for (int w = 0; w < lanes; ++w) {
+            int32_t i = row[w];
+            if (i < 0) continue;
+            last[w] = i;
+            for (int32_t p : ops[i].preds) unsched_cons[p]--;
+            for (int64_t e = cp[i]; e < cp[i + 1]; ++e)
+                if (--left[cons[e]] == 0) next_ready.push_back(cons[e]);
+        }
+        for (int32_t i : next_ready) ready.push({prio(i), i});
+        sched.push_back(std::move(row));
+        ++t;
+        if (chosen.empty() && ready.empty() && done < N) {
+            err = "scheduler stalled (graph is not acyclic?)";
+            return EMO_E_NOT_TOPOLOGICAL;
+        }
+    }
+    const int32_t S = t;
+    out.steps = S;
+
+    // ---- slots ---------------------------------------------------------------------------------
+    // An operand is read from the warp's register when the producing op was the previous op of the
+    // same warp; every other operand is read from the producer's slot.  A slot lives from the
+    // producer's step to the last step that reads it and is reused from the following step on.
+    std::vector<int32_t> last_use((size_t)N, -1);
+    for (int32_t i = 0; i < N; ++i)
+        for (int32_t p : ops[i].preds)
+            if (!(warp_of[p] == warp_of[i] && prev_on_warp[i] == p)) last_use[p] = std::max(last_use[p], step_of[i]);
+    std::vector<int32_t> slot_of((size_t)N, -1);
+    {
+        std::priority_queue<int32_t, std::vector<int32_t>, std::greater<int32_t>> free_ids;
+        std::priority_queue<Key, std::vector<Key>, std::greater<Key>> busy;   // (last use step, slot)
+        int32_t next_id = 0;
+        for (int32_t s = 0; s < S; ++s) {
+            while (!busy.empty() && busy.top().first < s) {
+                free_ids.push(busy.top().second);
+                busy.pop();
+            }
+            for (int w = 0; w < lanes; ++w) {
+                int32_t i = sched[s][w];
+                if (i < 0 || last_use[i] < 0) continue;
+                int32_t id;
+                if (!free_ids.empty()) {
+                    id = free_ids.top();
+                    free_ids.pop();
+                } else {
+                    id = next_id++;
+                }
+                slot_of[i] = id;
+                busy.push({last_use[i], id});
+            }
+        }
+        out.slots = next_id;
+        if (next_id > kMaxSlots) {
+            err = "graph needs " + std::to_string(next_id) + " live exchange values per policy; at most " +
+                  std::to_string(kMaxSlots) + " are supported";
+            return EMO_E_UNSUPPORTED;
+        }
+    }
+
+    // ---- entries and schedule-ordered tables -------------------------------------------------
+    const size_t Q = (size_t)S * lanes;
+    out.entries.assign(Q * 4, 0);
+    out.lat.assign(Q * Lp, 0);
+    if (!backward) out.energy.assign(Q * Lp, 0.0);
+    for (int32_t s = 0; s < S; ++s) {
+        for (int w = 0; w < lanes; ++w) {
+            int32_t i = sched[s][w];
+            size_t q = (size_t)s * lanes + w;
+            uint32_t *en = &out.entries[q * 4];
+            en[0] = kNone;
+            en[1] = kNone;
+            if (i < 0) continue;
+            const Op &o = ops[i];
+            uint32_t flags = kValid;
+            uint32_t operands = 0;
+            int np = 0;
+            for (int32_t p : o.preds) {
+                if (warp_of[p] == w && prev_on_warp[i] == p) {
+                    flags |= kRegPred;
+                } else {
+                    if (np < 4) operands |= (uint32_t)slot_of[p] << (8 * np);
+                    else flags |= (uint32_t)slot_of[p] << (16 + 8 * (np - 4));
+                    ++np;
+                }
+            }
+            flags |= (uint32_t)np << kNPredShift;
+            if (slot_of[i] >= 0) flags |= kWriteSlot | ((uint32_t)slot_of[i] << kOutShift);
+            if (o.node < 0) {
+                flags |= kAux;
+            } else {
+                int32_t v = o.node;
+                en[1] = (uint32_t)v;
+                if (g.group[v] >= 0) en[0] = (uint32_t)g.group[v];
+                if (cp[i + 1] == cp[i]) flags |= kTerminal;
+                for (int l = 0; l < Lp; ++l) {
+                    int ll = l < L ? l : L - 1;
+                    out.lat[q * Lp + l] = (uint32_t)lat[(size_t)v * L + ll];
+                    if (!backward) out.energy[q * Lp + l] = energy[(size_t)v * L + ll];
+                }
+            }
+            en[2] = flags;
+            en[3] = operands;
+        }
+    }
+    return EMO_OK;
+}
+
+}  // namespace emo

@@ -1,0 +1,245 @@
+// CUDA kernels of the evaluator (sm_100a).  Included only by emo_lib.cu.
+#pragma once
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "emo_compile.h"
+
+struct PassParams {
+    const uint4 *prog;        // [steps][lanes] program entries
+    const uint32_t *lat;      // [steps*lanes][Lp]
+    const double *en;         // [steps*lanes][Lp] (forward only)
+    int steps, lanes, Lp, Lmask, slots, groups;
+    int64_t B;
+    const uint8_t *lvl;       // [rows][ldb]
+    int64_t ldb;
+    int64_t *ES;              // forward: written when not NULL; backward: read
+    int64_t ldes;
+    int64_t *LS, *slack;      // backward outputs, optional
+    int64_t ldo;
+    int64_t *makespan;        // forward: written; backward: read
+    double *energy;
+    int64_t *slack_sum;
+    int32_t *n_critical;
+    int32_t *status;
+};
+
+// T0 + floor(T0 * ppm / 10^6) without a 128-bit product: with T0 = q*10^6 + r the quotient is
+// q*ppm + floor(r*ppm / 10^6), and r*ppm stays far below 2^63.
+__host__ __device__ inline int64_t emo_budget(int64_t T0, int64_t ppm)
+{
+    const int64_t M = 1000000;
+    int64_t q = T0 / M, r = T0 % M;
+    return T0 + q * ppm + (r * ppm) / M;
+}
+
+__device__ __forceinline__ void emo_group_barrier(int id, int nthreads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+// ------------------------------------------------------------------------------------------------
+// Pass kernel, plain loads.  One warp = 32 policies of one schedule lane; `lanes` warps form a group
+// and meet at a named barrier after every step.  Forward (BWD = false): Eq. 1 with the value
+// C_v kept in h; makespan over terminal nodes (equal to the maximum over all nodes because
+// durations are >= 0), energy accumulated per warp in step order and combined in lane order.
+// Backward: the same recurrence on the reversed graph gives Q_v = t_v + max over successors of Q_u,
+// so LS_v = T - Q_v and slack_v = LS_v - ES_v.
+// ------------------------------------------------------------------------------------------------
+template <bool BWD>
+__global__ void __launch_bounds__(1024) emo_pass_plain(PassParams p)
+{
+    extern __shared__ __align__(16) unsigned char emo_smem[];
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const int group = warp / p.lanes;
+    const int chain = warp - group * p.lanes;
+    const int64_t b = ((int64_t)blockIdx.x * p.groups + group) * 32 + lane;
+    const bool active = b < p.B;
+    long long *slots = reinterpret_cast<long long *>(emo_smem) + (size_t)group * p.slots * 32 + lane;
+    unsigned char *part_base = emo_smem + (size_t)p.groups * p.slots * 256;
+
+    long long h = 0;
+    double eacc = 0.0;
+    long long tmax = 0, ssum = 0;
+    int ncrit = 0;
+    const long long T = (BWD && active) ? p.makespan[b] : 0;
+    const uint4 *pe = p.prog + chain;
+    uint4 e = make_uint4(emo::kNone, emo::kNone, 0u, 0u);
+    if (p.steps > 0) e = __ldg(pe);
+    for (int t = 0; t < p.steps; ++t) {
+        uint4 nxt = make_uint4(emo::kNone, emo::kNone, 0u, 0u);
+        if (t + 1 < p.steps) nxt = __ldg(pe + (size_t)(t + 1) * p.lanes);
+        if (e.z & emo::kValid) {
+            unsigned lv = 0;
+            if (e.x != emo::kNone && active) lv = p.lvl[(size_t)e.x * p.ldb + b];
+            lv &= (unsigned)p.Lmask;
+            const size_t q = ((size_t)t * p.lanes + chain) * p.Lp + lv;
+            const long long dur = (long long)__ldg(p.lat + q);
+            long long start = (e.z & emo::kRegPred) ? h : 0;
+            const int np = (e.z >> emo::kNPredShift) & 7;
+            unsigned long long ops = (unsigned long long)e.w | ((unsigned long long)(e.z >> 16) << 32);
+            for (int k = 0; k < np; ++k) {
+                long long x = slots[(unsigned)(ops & 255u) * 32];
+                ops >>= 8;
+                start = x > start ? x : start;
+            }
+            h = start + dur;
+            if (!BWD) {
+                eacc += __ldg(p.en + q);
+                if (e.z & emo::kTerminal) tmax = h > tmax ? h : tmax;
+                if (p.ES && e.y != emo::kNone && active) p.ES[(size_t)e.y * p.ldes + b] = start;
+            } else if (e.y != emo::kNone && active) {
+                const long long ls = T - h;
+                const long long es = p.ES[(size_t)e.y * p.ldes + b];
+                const long long sl = ls - es;
+                if (p.LS) p.LS[(size_t)e.y * p.ldo + b] = ls;
+                if (p.slack) p.slack[(size_t)e.y * p.ldo + b] = sl;
+                ssum += sl;
+                ncrit += (sl == 0);
+            }
+            if (e.z & emo::kWriteSlot) slots[((e.z >> emo::kOutShift) & 255u) * 32] = h;
+        }
+        if (p.lanes > 1) emo_group_barrier(group + 1, p.lanes * 32);
+        e = nxt;
+    }
+
+    // combine the warps of a group in lane order (fixed order: run-to-run identical energy)
+    double *pd = reinterpret_cast<double *>(part_base) + ((size_t)(group * p.lanes + chain) * 32 + lane) * 2;
+    if (!BWD) {
+        pd[0] = eacc;
+        reinterpret_cast<long long *>(pd)[1] = tmax;
+    } else {
+        reinterpret_cast<long long *>(pd)[0] = ssum;
+        reinterpret_cast<long long *>(pd)[1] = (long long)ncrit;
+    }
+    __syncthreads();
+    if (chain == 0 && active) {
+        const double *g0 = reinterpret_cast<const double *>(part_base) + ((size_t)(group * p.lanes) * 32 + lane) * 2;
+        if (!BWD) {
+            double es = 0.0;
+            long long tm = 0;
+            for (int k = 0; k < p.lanes; ++k) {
+                es += g0[(size_t)k * 64];
+                long long x = reinterpret_cast<const long long *>(g0)[(size_t)k * 64 + 1];
+                tm = x > tm ? x : tm;
+            }
+            p.makespan[b] = tm;
+            p.energy[b] = es;
+        } else {
+            long long ss = 0, nc = 0;
+            for (int k = 0; k < p.lanes; ++k) {
+                ss += reinterpret_cast<const long long *>(g0)[(size_t)k * 64];
+                nc += reinterpret_cast<const long long *>(g0)[(size_t)k * 64 + 1];
+            }
+            if (p.slack_sum) p.slack_sum[b] = ss;
+            if (p.n_critical) p.n_critical[b] = (int32_t)nc;
+        }
+    }
+}
+
+// Every level must be < L; the first offender sets *status to EMO_E_RANGE (-3).
+__global__ void emo_validate_levels(const uint8_t *lvl, int64_t ldb, int64_t rows, int64_t B, int L, int32_t *status)
+{
+    const int64_t total = rows * B;
+    bool bad = false;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = i / B, b = i - r * B;
+        bad |= lvl[r * ldb + b] >= L;
+    }
+    if (__any_sync(0xFFFFFFFFu, bad) && (threadIdx.x & 31) == 0) atomicMin(status, -3);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Constrained arg-min (Eq. 4 over a finite batch): least energy among makespan <= target, equal
+// energies to the lower index.  Stage 1 leaves one candidate per block, stage 2 finishes.
+// ------------------------------------------------------------------------------------------------
+struct SelectPartial {
+    double e;
+    long long idx;
+};
+constexpr int kSelectMaxBlocks = 1024;
+
+__device__ __forceinline__ bool emo_better(double e1, long long i1, double e2, long long i2)
+{
+    // (e1, i1) beats (e2, i2); idx < 0 means "no candidate"
+    if (i1 < 0) return false;
+    if (i2 < 0) return true;
+    return e1 < e2 || (e1 == e2 && i1 < i2);
+}
+
+__device__ __forceinline__ void emo_select_reduce(double &e, long long &idx, SelectPartial *sh)
+{
+    for (int off = 16; off > 0; off >>= 1) {
+        double e2 = __shfl_down_sync(0xFFFFFFFFu, e, off);
+        long long i2 = __shfl_down_sync(0xFFFFFFFFu, idx, off);
+        if (emo_better(e2, i2, e, idx)) { e = e2; idx = i2; }
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) { sh[warp].e = e; sh[warp].idx = idx; }
+    __syncthreads();
+    if (warp == 0) {
+        const int nw = blockDim.x >> 5;
+        e = lane < nw ? sh[lane].e : 0.0;
+        idx = lane < nw ? sh[lane].idx : -1;
+        for (int off = 16; off > 0; off >>= 1) {
+            double e2 = __shfl_down_sync(0xFFFFFFFFu, e, off);
+            long long i2 = __shfl_down_sync(0xFFFFFFFFu, idx, off);
+            if (emo_better(e2, i2, e, idx)) { e = e2; idx = i2; }
+        }
+    }
+}
+
+__global__ void emo_select_stage1(int64_t B, const int64_t *makespan, const double *energy, int64_t target,
+                                  const int64_t *target_dev, int64_t delta_ppm, SelectPartial *part)
+{
+    __shared__ SelectPartial sh[32];
+    if (target_dev) target = emo_budget(target_dev[0], delta_ppm);
+    double e = 0.0;
+    long long idx = -1;
+    for (int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; b < B; b += (int64_t)gridDim.x * blockDim.x) {
+        if (makespan[b] <= target) {
+            const double x = energy[b];
+            if (emo_better(x, b, e, idx)) { e = x; idx = b; }
+        }
+    }
+    emo_select_reduce(e, idx, sh);
+    if (threadIdx.x == 0) { part[blockIdx.x].e = e; part[blockIdx.x].idx = idx; }
+}
+
+__global__ void emo_select_stage2(int nparts, const SelectPartial *part, const int64_t *makespan,
+                                  int64_t *out_index, int64_t *out_T, double *out_E)
+{
+    __shared__ SelectPartial sh[32];
+    double e = 0.0;
+    long long idx = -1;
+    for (int i = threadIdx.x; i < nparts; i += blockDim.x) {
+        if (emo_better(part[i].e, part[i].idx, e, idx)) { e = part[i].e; idx = part[i].idx; }
+    }
+    emo_select_reduce(e, idx, sh);
+    if (threadIdx.x == 0) {
+        *out_index = idx;
+        if (out_T) *out_T = idx >= 0 ? makespan[idx] : 0;
+        if (out_E) *out_E = idx >= 0 ? e : 0.0;
+    }
+}
+
+// src [B][lds] -> dst [rows][ldb], 32x32 byte tiles through shared memory.
+__global__ void emo_transpose_u8(int64_t B, int64_t rows, const uint8_t *src, int64_t lds, uint8_t *dst, int64_t ldb)
+{
+    __shared__ uint8_t tile[32][33];
+    const int64_t r0 = (int64_t)blockIdx.x * 32;
+    for (int64_t b0 = (int64_t)blockIdx.y * 32; b0 < B; b0 += (int64_t)gridDim.y * 32) {
+        for (int j = threadIdx.y; j < 32; j += blockDim.y) {
+            const int64_t b = b0 + j, r = r0 + threadIdx.x;
+            if (b < B && r < rows) tile[j][threadIdx.x] = src[b * lds + r];
+        }
+        __syncthreads();
+        for (int j = threadIdx.y; j < 32; j += blockDim.y) {
+            const int64_t r = r0 + j, b = b0 + threadIdx.x;
+            if (r < rows && b < B) dst[r * ldb + b] = tile[threadIdx.x][j];
+        }
+        __syncthreads();
+    }
+}

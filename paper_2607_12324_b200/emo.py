@@ -1,0 +1,242 @@
+"""Thin ctypes binding over the C-ABI library (include/emo.h): argument marshalling only.
+
+Function names and argument order follow the header.  Device buffers are torch tensors (or raw
+integer addresses); torch is used for device memory and streams, never for the computation.
+Loading fails loudly when the CUDA library has not been built: there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libemo_b200.so")
+
+EMO_OK = 0
+EMO_E_INVALID_ARG, EMO_E_NOT_TOPOLOGICAL, EMO_E_RANGE, EMO_E_OVERFLOW = -1, -2, -3, -4
+EMO_E_NONFINITE, EMO_E_OOM, EMO_E_CUDA, EMO_E_TIMEOUT, EMO_E_UNSUPPORTED = -5, -6, -7, -8, -9
+EMO_F_HOST_ONLY = 0x1
+EMO_F_VALIDATE = 0x1
+EMO_F_NO_STAGING = 0x2
+
+EXPORTS = [
+    "emo_strerror", "emo_graph_load", "emo_graph_free", "emo_graph_info", "emo_workspace_bytes",
+    "emo_eval_policies", "emo_slack_batch", "emo_slack", "emo_baseline", "emo_target_from_delta",
+    "emo_select", "emo_transpose_policies", "emo_slack_batch_host", "emo_graph_program",
+]
+
+
+def EMO_F_LANES(c: int) -> int:
+    return (c & 0xFF) << 8
+
+
+def EMO_F_LOOKAHEAD(d: int) -> int:
+    return (d & 0xFF) << 16
+
+
+class EmoError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {strerror(code)} ({code})")
+
+
+class emo_info(ctypes.Structure):
+    _fields_ = [("n", ctypes.c_int32), ("m", ctypes.c_int64), ("L", ctypes.c_int32), ("rows", ctypes.c_int32),
+                ("depth", ctypes.c_int32), ("max_span", ctypes.c_int32), ("T_worst", ctypes.c_int64),
+                ("T_best", ctypes.c_int64), ("lanes", ctypes.c_int32),
+                ("steps_fwd", ctypes.c_int32), ("slots_fwd", ctypes.c_int32), ("aux_fwd", ctypes.c_int32),
+                ("steps_bwd", ctypes.c_int32), ("slots_bwd", ctypes.c_int32), ("aux_bwd", ctypes.c_int32)]
+
+
+_lib = None
+
+
+def lib():
+    """The loaded shared library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2607_12324_b200.build` "
+                               "(there is no CPU fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        p, i32, i64, u32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_uint32, ctypes.c_size_t
+        L.emo_strerror.argtypes = [ctypes.c_int]
+        L.emo_strerror.restype = ctypes.c_char_p
+        L.emo_graph_load.argtypes = [i32, p, p, p, i32, i32, p, p, p, u32, ctypes.POINTER(p)]
+        L.emo_graph_free.argtypes = [p]
+        L.emo_graph_info.argtypes = [p, ctypes.POINTER(emo_info)]
+        L.emo_workspace_bytes.argtypes = [p, i64, ctypes.c_int, ctypes.POINTER(sz)]
+        L.emo_eval_policies.argtypes = [p, i64, p, i64, p, p, p, sz, p, u32, p]
+        L.emo_slack_batch.argtypes = [p, i64, p, i64, p, p, p, i64, p, p, p, p, p, sz, p, u32, p]
+        L.emo_slack.argtypes = [p, p, p, p, p, p, p, p, sz, p, p]
+        L.emo_baseline.argtypes = [p, p, p, p, sz, p, p]
+        L.emo_target_from_delta.argtypes = [i64, i64]
+        L.emo_target_from_delta.restype = i64
+        L.emo_select.argtypes = [i64, p, p, i64, p, i64, p, p, p, p, sz, p]
+        L.emo_transpose_policies.argtypes = [i64, i64, p, i64, p, i64, p]
+        L.emo_slack_batch_host.argtypes = [p, i64, p, i64, p, p, i64, i64, p, p, p, p, p, p, sz, u32, p]
+        L.emo_graph_program.argtypes = [p, ctypes.c_int, ctypes.POINTER(i32), ctypes.POINTER(i32),
+                                        ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(p),
+                                        ctypes.POINTER(p)]
+        for name in EXPORTS:
+            if name not in ("emo_strerror", "emo_target_from_delta"):
+                getattr(L, name).restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return lib().emo_strerror(int(code)).decode()
+
+
+def _addr(x) -> Optional[int]:
+    """Address of a torch tensor, numpy array, int, or None."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if isinstance(x, np.ndarray):
+        return x.ctypes.data
+    return int(x.data_ptr())
+
+
+def _check(rc: int, where: str):
+    if rc != EMO_OK:
+        raise EmoError(rc, where)
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return int(torch.cuda.current_stream().cuda_stream) or None
+    if isinstance(stream, int):
+        return stream or None
+    return int(stream.cuda_stream) or None
+
+
+class Graph:
+    """Owner of an emo_graph handle."""
+
+    def __init__(self, handle: int):
+        self.handle = handle
+
+    def free(self):
+        if self.handle:
+            lib().emo_graph_free(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
+
+    @property
+    def info(self) -> emo_info:
+        return emo_graph_info(self)
+
+
+def emo_graph_load(n, row_ptr, col, level_ptr, L, lat, energy, group_of=None, flags: int = 0) -> Graph:
+    row_ptr = np.ascontiguousarray(row_ptr, dtype=np.int64)
+    col = np.ascontiguousarray(col, dtype=np.int32)
+    lat = np.ascontiguousarray(lat, dtype=np.int64)
+    energy = np.ascontiguousarray(energy, dtype=np.float64)
+    lp = None if level_ptr is None else np.ascontiguousarray(level_ptr, dtype=np.int32)
+    go = None if group_of is None else np.ascontiguousarray(group_of, dtype=np.int32)
+    out = ctypes.c_void_p()
+    rc = lib().emo_graph_load(int(n), _addr(row_ptr), _addr(col), _addr(lp), 0 if lp is None else len(lp) - 1,
+                              int(L), _addr(lat), _addr(energy), _addr(go), int(flags), ctypes.byref(out))
+    _check(rc, "emo_graph_load")
+    return Graph(out.value)
+
+
+def load_workload(g, flags: int = 0, group_of=None, with_levels: bool = True) -> Graph:
+    """emo_graph_load on a workloads.Graph."""
+    return emo_graph_load(g.n, g.row_ptr, g.col, g.level_ptr if with_levels and len(g.level_ptr) > 2 else None,
+                          g.L, g.lat, g.energy, group_of, flags)
+
+
+def emo_graph_info(g: Graph) -> emo_info:
+    info = emo_info()
+    _check(lib().emo_graph_info(g.handle, ctypes.byref(info)), "emo_graph_info")
+    return info
+
+
+def emo_workspace_bytes(g: Graph, B: int, need_slack: int = 0) -> int:
+    out = ctypes.c_size_t()
+    _check(lib().emo_workspace_bytes(g.handle, int(B), int(need_slack), ctypes.byref(out)), "emo_workspace_bytes")
+    return int(out.value)
+
+
+def _nbytes(ws) -> int:
+    return 0 if ws is None else int(ws.numel() * ws.element_size())
+
+
+def emo_eval_policies(g: Graph, B, lvl, ldb, makespan, energy, ws=None, status=None, flags=0, stream=None):
+    _check(lib().emo_eval_policies(g.handle, int(B), _addr(lvl), int(ldb), _addr(makespan), _addr(energy),
+                                   _addr(ws), _nbytes(ws), _addr(status), int(flags), _stream(stream)),
+           "emo_eval_policies")
+
+
+def emo_slack_batch(g: Graph, B, lvl, ldb, ES, LS, slack, ldo, makespan, energy, slack_sum=None,
+                    n_critical=None, ws=None, status=None, flags=0, stream=None):
+    _check(lib().emo_slack_batch(g.handle, int(B), _addr(lvl), int(ldb), _addr(ES), _addr(LS), _addr(slack),
+                                 int(ldo), _addr(makespan), _addr(energy), _addr(slack_sum), _addr(n_critical),
+                                 _addr(ws), _nbytes(ws), _addr(status), int(flags), _stream(stream)),
+           "emo_slack_batch")
+
+
+def emo_slack(g: Graph, lvl_one, ES, LS, slack, makespan, energy=None, ws=None, status=None, stream=None):
+    _check(lib().emo_slack(g.handle, _addr(lvl_one), _addr(ES), _addr(LS), _addr(slack), _addr(makespan),
+                           _addr(energy), _addr(ws), _nbytes(ws), _addr(status), _stream(stream)), "emo_slack")
+
+
+def emo_baseline(g: Graph, T0, E0, ws, status=None, stream=None):
+    _check(lib().emo_baseline(g.handle, _addr(T0), _addr(E0), _addr(ws), _nbytes(ws), _addr(status),
+                              _stream(stream)), "emo_baseline")
+
+
+def emo_target_from_delta(T0: int, delta_ppm: int) -> int:
+    return int(lib().emo_target_from_delta(int(T0), int(delta_ppm)))
+
+
+def emo_select(B, makespan, energy, target, out_index, out_T=None, out_E=None, ws=None, target_dev=None,
+               delta_ppm: int = 0, stream=None):
+    _check(lib().emo_select(int(B), _addr(makespan), _addr(energy), int(target), _addr(target_dev),
+                            int(delta_ppm), _addr(out_index), _addr(out_T), _addr(out_E), _addr(ws),
+                            _nbytes(ws), _stream(stream)), "emo_select")
+
+
+def emo_transpose_policies(B, rows, src, lds, dst, ldb, stream=None):
+    _check(lib().emo_transpose_policies(int(B), int(rows), _addr(src), int(lds), _addr(dst), int(ldb),
+                                        _stream(stream)), "emo_transpose_policies")
+
+
+def emo_slack_batch_host(g: Graph, B, lvl_host, ldb, dev_lvl, slack_dev, ldo, delta_ppm, makespan_host,
+                         energy_host, slack_sum_host, n_critical_host, sel_host, ws, flags=0, stream=None):
+    _check(lib().emo_slack_batch_host(g.handle, int(B), _addr(lvl_host), int(ldb), _addr(dev_lvl),
+                                      _addr(slack_dev), int(ldo), int(delta_ppm), _addr(makespan_host),
+                                      _addr(energy_host), _addr(slack_sum_host), _addr(n_critical_host),
+                                      _addr(sel_host), _addr(ws), _nbytes(ws), int(flags), _stream(stream)),
+           "emo_slack_batch_host")
+
+
+def emo_graph_program(g: Graph, direction: int):
+    """(lanes, steps, slots, Lp, entries[steps][lanes][4] uint32, lat[steps*lanes][Lp] uint32) as
+    numpy copies of the compiled program (host-side inspection)."""
+    lanes, steps, slots, Lp = (ctypes.c_int32() for _ in range(4))
+    pe, pl = ctypes.c_void_p(), ctypes.c_void_p()
+    _check(lib().emo_graph_program(g.handle, int(direction), ctypes.byref(lanes), ctypes.byref(steps),
+                                   ctypes.byref(slots), ctypes.byref(Lp), ctypes.byref(pe), ctypes.byref(pl)),
+           "emo_graph_program")
+    q = steps.value * lanes.value
+    if q == 0:
+        return lanes.value, 0, slots.value, Lp.value, np.zeros((0, max(lanes.value, 1), 4), np.uint32), \
+            np.zeros((0, Lp.value), np.uint32)
+    ent = np.ctypeslib.as_array(ctypes.cast(pe, ctypes.POINTER(ctypes.c_uint32)), shape=(q * 4,)).copy()
+    lat = np.ctypeslib.as_array(ctypes.cast(pl, ctypes.POINTER(ctypes.c_uint32)), shape=(q * Lp.value,)).copy()
+    return lanes.value, steps.value, slots.value, Lp.value, ent.reshape(steps.value, lanes.value, 4), \
+        lat.reshape(q, Lp.value)
