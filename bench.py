@@ -1,0 +1,317 @@
+"""Benchmark of the batched what-if evaluation hot path on the largest workload configuration.
+
+One step = the whole hot path over one batch: forward + backward pass for all policies with the
+per-node slack matrix materialised (emo_slack_batch), the all-max-frequency baseline (emo_baseline)
+and the constrained arg-min (emo_select), on the cfg4-llm graph (200 000 kernels + 50 000 CPU
+nodes, ~470 k edges, 32 levels, 16 384 policies) with seeded synthetic inputs.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+Prints ONE JSON line (rank 0).  With N > 1 (torchrun) every rank runs a replica of the same
+workload on its own GPU; the path has no exchange between GPUs.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "policy_edge_relaxations_per_s"
+UNIT = "relaxations/s"
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.gpu)], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_sample(g, lv_cols, threads, want_slack=True):
+    """Times the CPU oracle as it stands on the given policy columns; returns seconds."""
+    import oracle
+    t0 = time.perf_counter()
+    oracle.batch(g, lv_cols, want_slack=want_slack, threads=threads)
+    return time.perf_counter() - t0
+
+
+def run_reference(args, rank, world):
+    """The reference arm: the CPU oracle on the host cores, a bounded sample per step."""
+    if rank != 0:
+        return
+    import numpy as np
+    from paper_2607_12324_b200 import workloads as W
+    g = W.make_graph(args.workload)
+    B = g.meta["B"]
+    threads = os.cpu_count() or 1
+    per_step = max(threads, 2 * threads)
+    total = per_step * (args.steps + args.warmup)
+    cols = np.linspace(0, B - 1, total).astype(np.int64)
+    lv = np.empty((g.n, total), dtype=np.uint8)
+    for j0 in range(0, total, 64):
+        js = cols[j0:j0 + 64]
+        for k, c in enumerate(js):
+            lv[:, j0 + k] = W.policy_levels(g.meta["policy_seed"], g.n, g.L, B, g.meta["policy_mode"], g.meta["q_max"],
+                                            cols=(int(c), int(c) + 1)).numpy()[:, 0]
+    for w in range(args.warmup):
+        oracle_sample(g, np.ascontiguousarray(lv[:, w * per_step:(w + 1) * per_step]), threads)
+    t = 0.0
+    for s in range(args.steps):
+        a = (args.warmup + s) * per_step
+        t += oracle_sample(g, np.ascontiguousarray(lv[:, a:a + per_step]), threads)
+    value = per_step * args.steps * g.m * 2 / t
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+            "config": {"workload": args.workload, "n": g.n, "m": g.m, "L": g.L, "policies": B,
+                       "passes": "forward+backward"},
+            "policies_per_s": per_step * args.steps / t,
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                             "sample": f"{per_step} of {B} policies per step, forward+backward with slack sums"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg4-llm")
+    ap.add_argument("--policies", type=int, default=0, help="override the number of policies (profiling a small case)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--flags", type=int, default=0, help="extra EMO_F_* load flags (lanes / look-ahead)")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+
+    import numpy as np
+    import torch
+    from paper_2607_12324_b200 import build, emo, workloads as W
+
+    if rank == 0:
+        build.build()
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist.barrier()
+
+    g = W.make_graph(args.workload)
+    B = args.policies or g.meta["B"]
+    ppm = (g.meta["delta_ppm"] or [50_000])[-1]
+    lv = W.policies_for(g, B=B, device="cuda")
+    ldb = lv.stride(0)
+    h = emo.load_workload(g, flags=args.flags)
+    info = h.info
+    n, m = g.n, g.m
+    slack = torch.empty((n, B), dtype=torch.int64, device="cuda")
+    T = torch.zeros(B, dtype=torch.int64, device="cuda")
+    E = torch.zeros(B, dtype=torch.float64, device="cuda")
+    ss = torch.zeros(B, dtype=torch.int64, device="cuda")
+    nc = torch.zeros(B, dtype=torch.int32, device="cuda")
+    T0 = torch.zeros(1, dtype=torch.int64, device="cuda")
+    E0 = torch.zeros(1, dtype=torch.float64, device="cuda")
+    sel = torch.zeros(2, dtype=torch.int64, device="cuda")
+    selE = torch.zeros(1, dtype=torch.float64, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ws = torch.empty(emo.emo_workspace_bytes(h, B, 2), dtype=torch.uint8, device="cuda")
+
+    def step(events=None):
+        if events is not None:
+            emo.emo_set_pass_events(*events)
+        emo.emo_slack_batch(h, B, lv, ldb, None, None, slack, B, T, E, ss, nc, ws, status)
+        if events is not None:
+            emo.emo_set_pass_events(None, None, None, None)
+        emo.emo_baseline(h, T0, E0, ws, status)
+        emo.emo_select(B, T, E, 0, sel[0:1], sel[1:2], selE, ws, target_dev=T0, delta_ppm=ppm)
+
+    launches_per_step = 5          # forward pass, backward pass, baseline forward pass, 2 selection kernels
+    for _ in range(max(args.warmup, 0)):
+        step()
+    torch.cuda.synchronize()
+
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    for e4 in evs:
+        for e in e4:
+            e.record()                      # creates the handles before the timed region
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for s in range(args.steps):
+        step(evs[s])
+    stop.record()
+    torch.cuda.synchronize()
+    total_ms = start.elapsed_time(stop)
+    fwd_ms = [e4[0].elapsed_time(e4[1]) for e4 in evs]
+    bwd_ms = [e4[2].elapsed_time(e4[3]) for e4 in evs]
+    clocks = sampler.stop() if rank == 0 else None
+    if dist is not None:
+        tt = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+        dist.barrier()
+    assert int(status.item()) == 0, f"device status {int(status.item())}"
+    ms_per_step = total_ms / args.steps
+    passes = 2
+    value = world * B * m * passes / (ms_per_step * 1e-3)
+
+    # roofline of the dominant kernel (the backward pass: reads the levels, writes the slack matrix)
+    peak, peak_kind = measured_peaks()
+    bwd = sum(bwd_ms) / len(bwd_ms)        # average launch duration over the timed region
+    fwd = sum(fwd_ms) / len(fwd_ms)
+    dom_is_bwd = bwd >= fwd
+    alg_bwd = n * B * 9 + B * 12            # 1 B level in + 8 B slack out per node x policy, per-policy sums out
+    alg_fwd = n * B * 1 + B * 16            # 1 B level in per node x policy, makespan + energy out
+    dom_ms, dom_bytes = (bwd, alg_bwd) if dom_is_bwd else (fwd, alg_fwd)
+    achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "backward pass" if dom_is_bwd else "forward pass", "achieved": achieved,
+                "peak": peak, "peak_source": peak_kind, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                "kernel_ms": dom_ms, "fwd_ms": fwd, "bwd_ms": bwd}
+    step_bytes = n * B * 9 + B * 28
+    roofline_step = {"bound": "hbm", "algorithmic_bytes": step_bytes, "achieved": step_bytes / (ms_per_step * 1e-3) / 1e9,
+                     "peak": peak, "unit": "GB/s", "frac": step_bytes / (ms_per_step * 1e-3) / 1e9 / peak}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "int64", "data": "synthetic",
+            "config": {"workload": args.workload, "n": n, "m": m, "L": g.L, "policies": B, "passes": "forward+backward",
+                       "slack_materialised": True, "delta_ppm": ppm, "lanes": info.lanes, "steps_fwd": info.steps_fwd,
+                       "slots_fwd": info.slots_fwd, "slots_bwd": info.slots_bwd,
+                       "l2": "inputs larger than L2 (levels %.1f GB, slack %.1f GB per step)" % (n * ldb / 1e9, n * B * 8 / 1e9),
+                       "parallelism": "replicas" if world > 1 else "single"},
+            "policies_per_s": world * B / (ms_per_step * 1e-3),
+            "gpu_launches": launches_per_step * args.steps,
+            "roofline": roofline, "roofline_step": roofline_step, "clocks": clocks,
+            "selected": {"index": int(sel[0].item()), "T": int(sel[1].item()), "E": float(selE.item()),
+                         "T0": int(T0.item()), "E0": float(E0.item())}}
+
+    # end to end through the host-buffer entry point: levels from pinned host memory every step,
+    # per-policy results and the selection back to the host; the slack matrix stays on the device
+    if not args.no_e2e:
+        lv_host = torch.empty((g.n, ldb), dtype=torch.uint8).pin_memory()
+        lv_host.copy_(lv)
+        hT = torch.zeros(B, dtype=torch.int64).pin_memory()
+        hE = torch.zeros(B, dtype=torch.float64).pin_memory()
+        hss = torch.zeros(B, dtype=torch.int64).pin_memory()
+        hnc = torch.zeros(B, dtype=torch.int32).pin_memory()
+        hsel = torch.zeros(4, dtype=torch.int64)
+        dev_lvl = torch.empty_like(lv)
+        emo.emo_slack_batch_host(h, B, lv_host, ldb, dev_lvl, slack, B, ppm, hT, hE, hss, hnc, hsel, ws)
+        torch.cuda.synchronize()
+        k = max(1, min(args.steps, 5))
+        if dist is not None:
+            dist.barrier()
+        t0 = time.perf_counter()
+        for _ in range(k):
+            emo.emo_slack_batch_host(h, B, lv_host, ldb, dev_lvl, slack, B, ppm, hT, hE, hss, hnc, hsel, ws)
+        torch.cuda.synchronize()
+        e2e_s = (time.perf_counter() - t0) / k
+        if dist is not None:
+            tt = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            e2e_s = float(tt.item())
+        assert int(hsel[0]) == int(sel[0].item())
+        line["e2e"] = {"value": world * B * m * passes / e2e_s, "unit": UNIT, "ms_per_step": e2e_s * 1e3,
+                       "h2d_bytes_per_step": int(g.n * ldb), "d2h_bytes_per_step": int(B * 28 + 80),
+                       "note": "slack matrix stays on the device"}
+        del lv_host
+
+    if rank == 0 and not args.no_cpu:
+        threads = os.cpu_count() or 1
+        cnt = max(threads, 16)
+        cols = np.linspace(0, B - 1, cnt).astype(np.int64)
+        sub = lv[:, cols].contiguous().cpu().numpy()
+        t1 = oracle_sample(g, sub[:, :threads].copy(), threads)
+        cnt2 = int(min(B, max(threads, (12.0 / max(t1, 1e-3)) * threads)))
+        cols = np.linspace(0, B - 1, cnt2).astype(np.int64)
+        sub = lv[:, torch.as_tensor(cols, device="cuda")].contiguous().cpu().numpy()
+        t2 = oracle_sample(g, sub, threads)
+        line["cpu_baseline"] = {"value": cnt2 * m * passes / t2, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                "sample": f"{cnt2} of {B} policies, forward+backward with slack sums, {t2:.1f} s",
+                                "policies_per_s": cnt2 / t2}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    h.free()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -201,6 +201,14 @@ int emo_slack_batch_host(const emo_graph *g, int64_t B, const uint8_t *lvl_host,
                          void *ws, size_t ws_bytes, uint32_t flags, void *stream);
 
 /*
+ * emo_set_pass_events - measurement hook (no counterpart in the method): four cudaEvent_t handles
+ * (as void*, any may be NULL) that later emo_slack_batch / emo_eval_policies / emo_baseline calls
+ * record on their stream immediately before and after the forward pass kernel and before and after
+ * the backward pass kernel.  Pass four NULLs to switch it off.  Process-wide, not thread-safe.
+ */
+int emo_set_pass_events(void *fwd_start, void *fwd_stop, void *bwd_start, void *bwd_stop);
+
+/*
  * Inspection of the compiled evaluation program (host memory owned by the handle; valid until
  * emo_graph_free).  dir 0 = forward, 1 = backward.  entries is [steps][lanes][4] uint32,
  * lat is uint32 [steps*lanes][Lp], Lp = row stride (a power of two >= L).  Used by host-side

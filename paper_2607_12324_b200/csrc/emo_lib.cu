@@ -34,6 +34,9 @@ namespace {
 
 constexpr size_t kSmallWs = 65536;   // head of the workspace: selection partials and scalars
 
+// Optional timing hook: events recorded around the forward and the backward pass kernel.
+cudaEvent_t g_pass_events[4] = {nullptr, nullptr, nullptr, nullptr};
+
 size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 #define EMO_CUDA(call)                                  \
@@ -142,6 +145,8 @@ int launch_pass(const emo_graph *g, bool backward, int64_t B, const uint8_t *lvl
     a.slack_sum = slack_sum;
     a.n_critical = n_critical;
     a.status = status;
+    cudaEvent_t ev0 = g_pass_events[backward ? 2 : 0], ev1 = g_pass_events[backward ? 3 : 1];
+    if (ev0) EMO_CUDA(cudaEventRecord(ev0, st));
     if (backward) {
         if (s.smem > 48 * 1024) EMO_CUDA(cudaFuncSetAttribute(emo_pass_plain<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s.smem));
         emo_pass_plain<true><<<s.grid, s.threads, s.smem, st>>>(a);
@@ -150,6 +155,7 @@ int launch_pass(const emo_graph *g, bool backward, int64_t B, const uint8_t *lvl
         emo_pass_plain<false><<<s.grid, s.threads, s.smem, st>>>(a);
     }
     EMO_CUDA(cudaGetLastError());
+    if (ev1) EMO_CUDA(cudaEventRecord(ev1, st));
     return EMO_OK;
 }
 
@@ -183,6 +189,15 @@ const char *emo_strerror(int code)
         case EMO_E_UNSUPPORTED: return "graph needs more exchange slots than supported";
         default: return "unknown status";
     }
+}
+
+int emo_set_pass_events(void *fwd_start, void *fwd_stop, void *bwd_start, void *bwd_stop)
+{
+    g_pass_events[0] = (cudaEvent_t)fwd_start;
+    g_pass_events[1] = (cudaEvent_t)fwd_stop;
+    g_pass_events[2] = (cudaEvent_t)bwd_start;
+    g_pass_events[3] = (cudaEvent_t)bwd_stop;
+    return EMO_OK;
 }
 
 int emo_graph_load(int32_t n, const int64_t *row_ptr, const int32_t *col, const int32_t *level_ptr,

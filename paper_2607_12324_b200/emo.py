@@ -26,6 +26,7 @@ EXPORTS = [
     "emo_strerror", "emo_graph_load", "emo_graph_free", "emo_graph_info", "emo_workspace_bytes",
     "emo_eval_policies", "emo_slack_batch", "emo_slack", "emo_baseline", "emo_target_from_delta",
     "emo_select", "emo_transpose_policies", "emo_slack_batch_host", "emo_graph_program",
+    "emo_set_pass_events",
 ]
 
 
@@ -81,6 +82,7 @@ def lib():
         L.emo_graph_program.argtypes = [p, ctypes.c_int, ctypes.POINTER(i32), ctypes.POINTER(i32),
                                         ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(p),
                                         ctypes.POINTER(p)]
+        L.emo_set_pass_events.argtypes = [p, p, p, p]
         for name in EXPORTS:
             if name not in ("emo_strerror", "emo_target_from_delta"):
                 getattr(L, name).restype = ctypes.c_int
@@ -222,6 +224,17 @@ def emo_slack_batch_host(g: Graph, B, lvl_host, ldb, dev_lvl, slack_dev, ldo, de
                                       _addr(energy_host), _addr(slack_sum_host), _addr(n_critical_host),
                                       _addr(sel_host), _addr(ws), _nbytes(ws), int(flags), _stream(stream)),
            "emo_slack_batch_host")
+
+
+def emo_set_pass_events(fwd_start=None, fwd_stop=None, bwd_start=None, bwd_stop=None):
+    """Events are torch.cuda.Event objects created with enable_timing=True (or None)."""
+    def h(ev):
+        if ev is None:
+            return None
+        if not ev.cuda_event:          # torch creates the handle lazily, on the first record
+            ev.record()
+        return int(ev.cuda_event)
+    _check(lib().emo_set_pass_events(h(fwd_start), h(fwd_stop), h(bwd_start), h(bwd_stop)), "emo_set_pass_events")
 
 
 def emo_graph_program(g: Graph, direction: int):

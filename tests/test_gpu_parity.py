@@ -1,0 +1,360 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same seeded
+inputs.  Integer results (ES, LS, slack, makespan, slack sums, critical counts, selected index) must
+be bit-exact; energies within 1e-9 relative."""
+from __future__ import annotations
+
+import json
+import os
+
+import numpy as np
+import pytest
+
+from paper_2607_12324_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+E_RTOL = 1e-9
+
+
+@pytest.fixture(scope="module")
+def torch_cuda():
+    import torch
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    torch.cuda.set_device(0)
+    return torch
+
+
+@pytest.fixture(scope="module")
+def emo(torch_cuda):
+    from paper_2607_12324_b200 import build, emo as E
+    build.build()
+    return E
+
+
+@pytest.fixture(scope="module")
+def golden():
+    with open(os.path.join(HERE, "golden", "config_golden.json")) as f:
+        return json.load(f)
+
+
+def gpu_slack_batch(torch, emo, h, lv_dev, B, n, want=("ES", "LS", "slack"), flags=0, ldo=None):
+    dev = lv_dev.device
+    ldo = int(ldo or max(B, 1))
+    out = {k: (torch.full((n, ldo), -7, dtype=torch.int64, device=dev) if k in want else None)
+           for k in ("ES", "LS", "slack")}
+    T = torch.full((max(B, 1),), -1, dtype=torch.int64, device=dev)
+    E = torch.full((max(B, 1),), -1.0, dtype=torch.float64, device=dev)
+    ss = torch.full((max(B, 1),), -1, dtype=torch.int64, device=dev)
+    nc = torch.full((max(B, 1),), -1, dtype=torch.int32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    ws = torch.empty(emo.emo_workspace_bytes(h, B, 1), dtype=torch.uint8, device=dev)
+    emo.emo_slack_batch(h, B, lv_dev, lv_dev.stride(0), out["ES"], out["LS"], out["slack"], ldo, T, E, ss, nc,
+                        ws, status, flags)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    res = {k: v.cpu().numpy() for k, v in out.items() if v is not None}
+    res.update(makespan=T.cpu().numpy()[:B], energy=E.cpu().numpy()[:B], slack_sum=ss.cpu().numpy()[:B],
+               n_critical=nc.cpu().numpy()[:B])
+    return res
+
+
+def gpu_eval(torch, emo, h, lv_dev, B, flags=0):
+    dev = lv_dev.device
+    T = torch.full((max(B, 1),), -1, dtype=torch.int64, device=dev)
+    E = torch.full((max(B, 1),), -1.0, dtype=torch.float64, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    ws = torch.empty(emo.emo_workspace_bytes(h, B, 0), dtype=torch.uint8, device=dev)
+    emo.emo_eval_policies(h, B, lv_dev, lv_dev.stride(0), T, E, ws, status, flags)
+    torch.cuda.synchronize()
+    return T.cpu().numpy()[:B], E.cpu().numpy()[:B], int(status.item())
+
+
+def gpu_select(torch, emo, T, E, target=0, target_dev=None, delta_ppm=0):
+    dev = "cuda"
+    Td = torch.as_tensor(T, dtype=torch.int64, device=dev)
+    Ed = torch.as_tensor(E, dtype=torch.float64, device=dev)
+    out = torch.full((3,), -5, dtype=torch.int64, device=dev)
+    oe = torch.zeros(1, dtype=torch.float64, device=dev)
+    ws = torch.empty(65536, dtype=torch.uint8, device=dev)
+    emo.emo_select(len(T), Td, Ed, target, out[0:1], out[1:2], oe, ws, target_dev, delta_ppm)
+    torch.cuda.synchronize()
+    return int(out[0].item()), int(out[1].item()), float(oe.item())
+
+
+def assert_matches(r_gpu, r_or, B, arrays=True):
+    assert np.array_equal(r_gpu["makespan"], r_or["makespan"])
+    np.testing.assert_allclose(r_gpu["energy"], r_or["energy"], rtol=E_RTOL, atol=0)
+    assert np.array_equal(r_gpu["slack_sum"], r_or["slack_sum"])
+    assert np.array_equal(r_gpu["n_critical"], r_or["n_critical"])
+    if arrays:
+        for k in ("ES", "LS", "slack"):
+            if k in r_gpu:
+                assert np.array_equal(r_gpu[k][:, :B], r_or[k]), k
+
+
+# ------------------------------------------------------------------------------------------------
+def test_tiny_graphs_all_outputs(torch_cuda, emo, oracle_mod):
+    """Hand-made and random tiny DAGs (ties, zero durations, duplicate edges, isolated nodes,
+    non-monotone rows), every policy, all outputs, several lane counts and a ragged ld."""
+    from tests.test_oracle_pins import TINY, all_policies
+    torch = torch_cuda
+    for gi in range(0, len(TINY), 2):
+        g = TINY[gi]
+        lv = all_policies(g.n, g.L)
+        B = lv.shape[1]
+        r_or = oracle_mod.batch(g, lv, want_arrays=True)
+        ldb = B + 5
+        lvp = np.full((g.n, ldb), 0xFF, dtype=np.uint8)
+        lvp[:, :B] = lv
+        lv_dev = torch.as_tensor(lvp, device="cuda")
+        for lanes in (0, 1, 2):
+            h = emo.load_workload(g, emo.EMO_F_LANES(lanes))
+            r = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, ldo=B + 3)
+            assert_matches(r, r_or, B)
+            for k in ("ES", "LS", "slack"):
+                assert (r[k][:, B:] == -7).all(), "padding columns of the outputs were written"
+            T, E, st = gpu_eval(torch, emo, h, lv_dev, B, emo.EMO_F_VALIDATE)
+            assert st == 0 and np.array_equal(T, r_or["makespan"])
+            np.testing.assert_allclose(E, r_or["energy"], rtol=E_RTOL)
+            h.free()
+
+
+def test_hand_worked_example_on_gpu(torch_cuda, emo):
+    torch = torch_cuda
+    with open(os.path.join(HERE, "golden", "hand_worked_dag.json")) as f:
+        gold = json.load(f)
+    n = len(gold["nodes"])
+    g = W.tiny_graph(n, gold["edges_pred_succ"], gold["lat"], gold["energy"])
+    lv = np.array([p["levels"] for p in gold["policies"]], dtype=np.uint8).T.copy()
+    h = emo.load_workload(g)
+    r = gpu_slack_batch(torch, emo, h, torch.as_tensor(lv, device="cuda"), 2, n)
+    for b, p in enumerate(gold["policies"]):
+        assert r["makespan"][b] == p["T"] and r["energy"][b] == p["E"]
+        assert r["ES"][:, b].tolist() == p["ES"] and r["LS"][:, b].tolist() == p["LS"]
+        assert r["slack"][:, b].tolist() == p["slack"]
+    for s in gold["selection"]:
+        assert emo.emo_target_from_delta(gold["policies"][0]["T"], s["delta_ppm"]) == s["target"]
+        assert gpu_select(torch, emo, r["makespan"], r["energy"], s["target"])[0] == s["index"]
+    h.free()
+
+
+@pytest.mark.parametrize("name,scale,B", [("cfg0-tiny", 1.0, 64), ("cfg1-train", 0.25, 333), ("cfg2-packed", 0.5, 1000),
+                                            ("cfg3-8dev", 0.03, 200), ("cfg4-llm", 0.02, 257)])
+def test_config_graphs_all_outputs(torch_cuda, emo, oracle_mod, name, scale, B):
+    """Scaled configuration graphs: several policy tiles and a ragged tail, all per-node outputs."""
+    torch = torch_cuda
+    g = W.make_graph(name, scale)
+    lv_dev = W.policies_for(g, B=B, device="cuda")
+    lv = lv_dev.cpu().numpy()
+    r_or = oracle_mod.batch(g, lv, B=B, want_arrays=True, threads=os.cpu_count() or 1)
+    h = emo.load_workload(g)
+    r = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n)
+    assert_matches(r, r_or, B)
+    # slack only (ES kept in the workspace), same result
+    r2 = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, want=("slack",))
+    assert np.array_equal(r2["slack"][:, :B], r_or["slack"])
+    # single-policy call
+    b = B // 2
+    one = lv_dev[:, b].contiguous()
+    ES, LS, SL = (torch.zeros(g.n, dtype=torch.int64, device="cuda") for _ in range(3))
+    T1 = torch.zeros(1, dtype=torch.int64, device="cuda")
+    E1 = torch.zeros(1, dtype=torch.float64, device="cuda")
+    ws = torch.empty(emo.emo_workspace_bytes(h, 1, 1), dtype=torch.uint8, device="cuda")
+    emo.emo_slack(h, one, ES, LS, SL, T1, E1, ws)
+    torch.cuda.synchronize()
+    assert int(T1.item()) == r_or["makespan"][b]
+    assert np.array_equal(ES.cpu().numpy(), r_or["ES"][:, b])
+    assert np.array_equal(LS.cpu().numpy(), r_or["LS"][:, b])
+    assert np.array_equal(SL.cpu().numpy(), r_or["slack"][:, b])
+    h.free()
+
+
+@pytest.mark.parametrize("name", ["cfg0-tiny", "cfg1-train", "cfg2-packed", "cfg3-8dev"])
+def test_full_configs_against_oracle_and_golden(torch_cuda, emo, oracle_mod, golden, name):
+    """Full-size configurations 0-3: every policy's makespan, energy, slack sum and critical count
+    against the oracle run here, per-node arrays on a sample of policies, baseline and selection
+    against the oracle and against the stored oracle results."""
+    torch = torch_cuda
+    g = W.make_graph(name)
+    B = g.meta["B"]
+    gold = golden[name]
+    assert (g.n, g.m, B) == (gold["n"], gold["m"], gold["B"])
+    lv_dev = W.policies_for(g, device="cuda")
+    h = emo.load_workload(g)
+    want = ("slack",)
+    r = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, want=want)
+    lv = lv_dev.cpu().numpy()
+    r_or = oracle_mod.batch(g, lv, B=B, want_slack=True, threads=os.cpu_count() or 1)
+    assert_matches(r, r_or, B, arrays=False)
+    cols = sorted(set(np.linspace(0, B - 1, 12).astype(int).tolist()))
+    sub = np.ascontiguousarray(lv[:, cols])
+    r_sub = oracle_mod.batch(g, sub, want_arrays=True)
+    assert np.array_equal(r["slack"][:, cols], r_sub["slack"])
+    # stored oracle values
+    assert [int(r["makespan"][i]) for i in gold["sample_idx"]] == gold["sample_makespan"]
+    np.testing.assert_allclose([r["energy"][i] for i in gold["sample_idx"]], gold["sample_energy"], rtol=E_RTOL)
+    # baseline (all rows at level L-1) and selection
+    T0 = torch.zeros(1, dtype=torch.int64, device="cuda")
+    E0 = torch.zeros(1, dtype=torch.float64, device="cuda")
+    ws = torch.empty(emo.emo_workspace_bytes(h, B, 0), dtype=torch.uint8, device="cuda")
+    emo.emo_baseline(h, T0, E0, ws)
+    torch.cuda.synchronize()
+    assert int(T0.item()) == gold["T0"]
+    assert float(E0.item()) == pytest.approx(gold["E0"], rel=E_RTOL)
+    for s in gold["select"]:
+        tgt = emo.emo_target_from_delta(int(T0.item()), s["delta_ppm"])
+        assert tgt == s["target"] == oracle_mod.target_from_delta(gold["T0"], s["delta_ppm"])
+        want_idx = oracle_mod.select(r_or["makespan"], r_or["energy"], tgt)
+        assert want_idx == s["index"]
+        assert s["margin_rel"] is None or s["margin_rel"] > 2e-9, "selection is ambiguous at the energy tolerance"
+        idx, Tsel, Esel = gpu_select(torch, emo, r["makespan"], r["energy"], tgt)
+        assert idx == want_idx and Tsel == s["T"]
+        assert Esel == pytest.approx(s["E"], rel=E_RTOL)
+        idx2, _, _ = gpu_select(torch, emo, r["makespan"], r["energy"], 0, target_dev=T0, delta_ppm=s["delta_ppm"])
+        assert idx2 == want_idx
+    h.free()
+
+
+def test_cfg4_full_size_sampled(torch_cuda, emo, oracle_mod, golden):
+    """The largest configuration at full size, in the launch configuration the bench times: all
+    16 384 policies on the GPU with slack materialised; the oracle checks sampled policies node by
+    node, and the stored oracle results check every policy's makespan / slack sum / critical
+    count (digests) and the selection."""
+    torch = torch_cuda
+    import hashlib
+    name = "cfg4-llm"
+    gold = golden.get(name)
+    g = W.make_graph(name)
+    B = g.meta["B"]
+    lv_dev = W.policies_for(g, device="cuda")
+    h = emo.load_workload(g)
+    r = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, want=())
+    cols = sorted(set(np.linspace(0, B - 1, 16).astype(int).tolist() + [1, 2, B // 2 - 1, B // 2]))
+    sub = lv_dev[:, cols].contiguous().cpu().numpy()
+    r_sub = oracle_mod.batch(g, sub, want_arrays=True, threads=os.cpu_count() or 1)
+    assert np.array_equal(r["makespan"][cols], r_sub["makespan"])
+    np.testing.assert_allclose(r["energy"][cols], r_sub["energy"], rtol=E_RTOL)
+    assert np.array_equal(r["slack_sum"][cols], r_sub["slack_sum"])
+    assert np.array_equal(r["n_critical"][cols], r_sub["n_critical"])
+    # per-node slack of the sampled policies: run them as their own small batch with arrays
+    sub_dev = torch.as_tensor(sub, device="cuda")
+    r2 = gpu_slack_batch(torch, emo, h, sub_dev, len(cols), g.n)
+    assert_matches(r2, r_sub, len(cols))
+    if gold is not None:
+        assert (g.n, g.m, B) == (gold["n"], gold["m"], gold["B"])
+        assert hashlib.sha256(np.ascontiguousarray(r["makespan"]).tobytes()).hexdigest() == gold["makespan_sha256"]
+        assert hashlib.sha256(np.ascontiguousarray(r["slack_sum"]).tobytes()).hexdigest() == gold["slack_sum_sha256"]
+        assert hashlib.sha256(np.ascontiguousarray(r["n_critical"]).tobytes()).hexdigest() == gold["n_critical_sha256"]
+        np.testing.assert_allclose([r["energy"][i] for i in gold["sample_idx"]], gold["sample_energy"], rtol=E_RTOL)
+        for s in gold["select"]:
+            assert s["margin_rel"] > 2e-9
+            idx, Tsel, Esel = gpu_select(torch, emo, r["makespan"], r["energy"], s["target"])
+            assert idx == s["index"] and Tsel == s["T"]
+            assert Esel == pytest.approx(s["E"], rel=E_RTOL)
+    h.free()
+
+
+def test_selection_cases(torch_cuda, emo, oracle_mod):
+    torch = torch_cuda
+    T = np.array([100, 105, 103, 103, 99, 110], dtype=np.int64)
+    E = np.array([9.0, 5.0, 7.0, 7.0, 9.5, 1.0])
+    for tgt in (98, 99, 100, 102, 103, 104, 105, 109, 110, 1000):
+        assert gpu_select(torch, emo, T, E, tgt)[0] == oracle_mod.select(T, E, tgt)
+    assert gpu_select(torch, emo, T, E, 98)[0] == -1
+    assert gpu_select(torch, emo, T[:1], E[:1], 100)[0] == 0
+    e2 = np.array([1.0, np.nextafter(1.0, 0.0), 1.0])
+    assert gpu_select(torch, emo, np.ones(3, dtype=np.int64), e2, 1)[0] == 1
+    rs = np.random.RandomState(0)
+    for B in (1, 31, 32, 33, 1000, 4097, 70001):
+        T = rs.randint(50, 150, B).astype(np.int64)
+        E = np.round(rs.rand(B) * 20) / 4.0          # many exact ties
+        for tgt in (49, 60, 100, 149):
+            idx, Ts, Es = gpu_select(torch, emo, T, E, tgt)
+            want = oracle_mod.select(T, E, tgt)
+            assert idx == want
+            if want >= 0:
+                assert Ts == T[want] and Es == E[want]
+
+
+def test_batch_edge_cases(torch_cuda, emo, oracle_mod):
+    """B = 0, B = 1, a level out of range with validation on, a graph without nodes, transpose."""
+    torch = torch_cuda
+    g = W.make_graph("cfg0-tiny")
+    h = emo.load_workload(g)
+    lv_dev = W.policies_for(g, B=40, device="cuda")
+    T = torch.full((4,), -1, dtype=torch.int64, device="cuda")
+    E = torch.full((4,), -1.0, dtype=torch.float64, device="cuda")
+    emo.emo_eval_policies(h, 0, lv_dev, lv_dev.stride(0), T, E, None, None, 0)
+    torch.cuda.synchronize()
+    assert (T == -1).all()
+    Tg, Eg, st = gpu_eval(torch, emo, h, lv_dev, 1)
+    r = oracle_mod.batch(g, lv_dev.cpu().numpy(), B=1)
+    assert Tg[0] == r["makespan"][0] and st == 0
+    # padding columns hold 0xFF: asking for them with validation reports EMO_E_RANGE
+    Tg, Eg, st = gpu_eval(torch, emo, h, lv_dev, 44, emo.EMO_F_VALIDATE)
+    assert st == emo.EMO_E_RANGE
+    Tg, Eg, st = gpu_eval(torch, emo, h, lv_dev, 40, emo.EMO_F_VALIDATE)
+    assert st == 0
+    with pytest.raises(emo.EmoError):
+        emo.emo_eval_policies(h, 50, lv_dev, 40, T, E, None, None, 0)          # ldb < B
+    # transpose helper
+    src = torch.randint(0, g.L, (37, g.n), dtype=torch.uint8, device="cuda")
+    dst = torch.zeros((g.n, 48), dtype=torch.uint8, device="cuda")
+    emo.emo_transpose_policies(37, g.n, src, g.n, dst, 48)
+    torch.cuda.synchronize()
+    assert torch.equal(dst[:, :37], src.t())
+    h.free()
+    h0 = emo.emo_graph_load(0, np.zeros(1, np.int64), np.zeros(0, np.int32), None, 3, np.zeros((0, 3), np.int64),
+                            np.zeros((0, 3)))
+    lv0 = torch.zeros((1, 16), dtype=torch.uint8, device="cuda")
+    Tg, Eg, st = gpu_eval(torch, emo, h0, lv0, 5)
+    assert (Tg == 0).all() and (Eg == 0).all()
+    h0.free()
+
+
+def test_group_of_on_gpu(torch_cuda, emo, oracle_mod):
+    torch = torch_cuda
+    g = W.make_graph("cfg1-train", 0.1)
+    group = (np.arange(g.n) // 4).astype(np.int32)
+    group[g.kind == W.KIND_CPU] = -1
+    rows = int(group.max()) + 1
+    B = 70
+    lv = np.random.RandomState(3).randint(0, g.L, (rows, B)).astype(np.uint8)
+    r_or = oracle_mod.batch(g, lv, want_arrays=True, group_of=group)
+    h = emo.load_workload(g, group_of=group)
+    r = gpu_slack_batch(torch, emo, h, torch.as_tensor(lv, device="cuda"), B, g.n)
+    assert_matches(r, r_or, B)
+    h.free()
+
+
+def test_host_buffer_call(torch_cuda, emo, oracle_mod):
+    """emo_slack_batch_host: levels from pinned host memory, per-policy results back to the host."""
+    torch = torch_cuda
+    g = W.make_graph("cfg1-train", 0.2)
+    B, ppm = 500, 30_000
+    lv = W.policies_for(g, B=B, device="cpu").pin_memory()
+    ldb = lv.stride(0)
+    h = emo.load_workload(g)
+    dev_lvl = torch.empty((g.n, ldb), dtype=torch.uint8, device="cuda")
+    slack = torch.zeros((g.n, B), dtype=torch.int64, device="cuda")
+    T = torch.zeros(B, dtype=torch.int64).pin_memory()
+    E = torch.zeros(B, dtype=torch.float64).pin_memory()
+    ss = torch.zeros(B, dtype=torch.int64).pin_memory()
+    nc = torch.zeros(B, dtype=torch.int32).pin_memory()
+    sel = torch.zeros(4, dtype=torch.int64)
+    ws = torch.empty(emo.emo_workspace_bytes(h, B, 2), dtype=torch.uint8, device="cuda")
+    for _ in range(2):
+        emo.emo_slack_batch_host(h, B, lv, ldb, dev_lvl, slack, B, ppm, T, E, ss, nc, sel, ws)
+    r_or = oracle_mod.batch(g, lv.numpy(), B=B, want_arrays=True)
+    assert np.array_equal(T.numpy(), r_or["makespan"])
+    np.testing.assert_allclose(E.numpy(), r_or["energy"], rtol=E_RTOL)
+    assert np.array_equal(ss.numpy(), r_or["slack_sum"]) and np.array_equal(nc.numpy(), r_or["n_critical"])
+    assert np.array_equal(slack.cpu().numpy(), r_or["slack"])
+    allmax = np.full((g.n, 1), g.L - 1, dtype=np.uint8)
+    T0 = int(oracle_mod.batch(g, allmax)["makespan"][0])
+    assert int(sel[3]) == T0
+    want = oracle_mod.select(r_or["makespan"], r_or["energy"], oracle_mod.target_from_delta(T0, ppm))
+    assert int(sel[0]) == want and int(sel[1]) == r_or["makespan"][want]
+    assert np.array([int(sel[2])], dtype=np.int64).view(np.float64)[0] == pytest.approx(r_or["energy"][want], rel=E_RTOL)
+    h.free()
