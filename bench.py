@@ -142,6 +142,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg4-llm")
     ap.add_argument("--policies", type=int, default=0, help="override the number of policies (profiling a small case)")
+    ap.add_argument("--scale", type=float, default=1.0, help="shrink the graph (profiling a small case)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--flags", type=int, default=0, help="extra EMO_F_* load flags (lanes / look-ahead)")
@@ -167,7 +168,7 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
         dist.barrier()
 
-    g = W.make_graph(args.workload)
+    g = W.make_graph(args.workload, args.scale)
     B = args.policies or g.meta["B"]
     ppm = (g.meta["delta_ppm"] or [50_000])[-1]
     lv = W.policies_for(g, B=B, device="cuda")
@@ -251,7 +252,7 @@ def main():
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "int64", "data": "synthetic",
-            "config": {"workload": args.workload, "n": n, "m": m, "L": g.L, "policies": B, "passes": "forward+backward",
+            "config": {"workload": args.workload if args.scale == 1.0 else f"{args.workload} x{args.scale}", "n": n, "m": m, "L": g.L, "policies": B, "passes": "forward+backward",
                        "slack_materialised": True, "delta_ppm": ppm, "lanes": info.lanes, "steps_fwd": info.steps_fwd,
                        "slots_fwd": info.slots_fwd, "slots_bwd": info.slots_bwd,
                        "l2": "inputs larger than L2 (levels %.1f GB, slack %.1f GB per step)" % (n * ldb / 1e9, n * B * 8 / 1e9),

@@ -56,7 +56,7 @@ int compile_program(const HostGraph &g, const int64_t *lat, const double *energy
 {
     const int32_t n = g.n;
     const int L = g.L;
-    int Lp = 1;
+    int Lp = 4;   // at least 4 so that a table row is a multiple of 16 bytes (bulk-copy granularity)
     while (Lp < L) Lp <<= 1;
     out = Program();
     out.Lp = Lp;

@@ -50,7 +50,7 @@ __device__ __forceinline__ void emo_group_barrier(int id, int nthreads)
 template <bool BWD>
 __global__ void __launch_bounds__(1024) emo_pass_plain(PassParams p)
 {
-    extern __shared__ __align__(16) unsigned char emo_smem[];
+    extern __shared__ __align__(128) unsigned char emo_smem[];
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     const int group = warp / p.lanes;

@@ -11,6 +11,7 @@
 #include "../../include/emo.h"
 #include "emo_compile.h"
 #include "emo_kernels.cuh"
+#include "emo_pass_staged.cuh"
 
 using namespace emo;
 
@@ -38,6 +39,9 @@ constexpr size_t kSmallWs = 65536;   // head of the workspace: selection partial
 cudaEvent_t g_pass_events[4] = {nullptr, nullptr, nullptr, nullptr};
 
 size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// workspace area for one policy's levels laid out [rows][16] (row pitch a bulk copy accepts)
+size_t lvl_area(const emo_graph *g);
 
 #define EMO_CUDA(call)                                  \
     do {                                                \
@@ -88,6 +92,8 @@ __int128 host_longest(const HostGraph &h, F dur)
     return T;
 }
 
+size_t lvl_area(const emo_graph *g) { return round_up((size_t)std::max(g->h.rows, 1) * 16, 256); }
+
 struct LaunchShape {
     int groups, grid, threads;
     size_t smem;
@@ -112,16 +118,61 @@ int shape_for(const emo_graph *g, const Program &p, int64_t B, LaunchShape &s)
     return EMO_OK;
 }
 
+// Shape of the staged kernel: groups per block as above (one more warp produces), then as many
+// steps per stage as fit beside the slots.  Returns false when the staged kernel cannot be used.
+bool staged_shape(const emo_graph *g, const Program &p, bool backward, int64_t B, LaunchShape &s, StagedParams &sp)
+{
+    if (p.steps == 0 || !g->smem_optin) return false;
+    int64_t n_groups = (B + 31) / 32;
+    int gmax = std::min(31 / p.lanes, 15);
+    if (gmax < 1) return false;
+    int64_t want = (n_groups + g->sm_count - 1) / g->sm_count;
+    int G = (int)std::max<int64_t>(1, std::min<int64_t>(gmax, want));
+    const size_t budget = g->smem_optin;
+    for (; G >= 1; --G) {
+        const size_t P = 32 * (size_t)G;
+        const size_t fixed = (size_t)G * p.slots * 256 + (size_t)G * p.lanes * 512 + 256;
+        const size_t per_step = (size_t)p.lanes * (16 + (size_t)p.Lp * 4 + (backward ? 0 : (size_t)p.Lp * 8) + P + (backward ? P * 8 : 0));
+        if (fixed + kStages * per_step > budget) continue;
+        int sc = (int)std::min<size_t>(16, (budget - fixed) / (kStages * per_step));
+        sc = std::min(sc, std::max(1, p.steps));
+        const size_t ne = (size_t)sc * p.lanes;
+        sp.sc = sc;
+        sp.ptile = (int)P;
+        sp.off_lat = (unsigned)(ne * 16);
+        sp.off_en = sp.off_lat + (unsigned)(ne * p.Lp * 4);
+        sp.off_lvl = sp.off_en + (backward ? 0u : (unsigned)(ne * p.Lp * 8));
+        sp.off_es = sp.off_lvl + (unsigned)(ne * P);
+        sp.stage_bytes = (unsigned)round_up(sp.off_es + (backward ? ne * P * 8 : 0), 128);
+        sp.off_part = (unsigned)((size_t)G * p.slots * 256);
+        sp.off_bar = sp.off_part + (unsigned)((size_t)G * p.lanes * 512);
+        sp.off_stage0 = (unsigned)round_up(sp.off_bar + 256, 128);
+        s.groups = G;
+        s.grid = (int)((n_groups + G - 1) / G);
+        s.threads = (G * p.lanes + 1) * 32;
+        s.smem = sp.off_stage0 + (size_t)kStages * sp.stage_bytes;
+        if (s.smem > budget) continue;
+        return true;
+    }
+    return false;
+}
+
 int launch_pass(const emo_graph *g, bool backward, int64_t B, const uint8_t *lvl, int64_t ldb,
                 int64_t *ES, int64_t ldes, int64_t *LS, int64_t *slack, int64_t ldo,
                 int64_t *makespan, double *energy, int64_t *slack_sum, int32_t *n_critical,
-                int32_t *status, cudaStream_t st)
+                int32_t *status, cudaStream_t st, uint32_t flags = 0)
 {
     const Program &p = backward ? g->bwd : g->fwd;
     const DevProgram &d = backward ? g->dbwd : g->dfwd;
     LaunchShape s;
-    int rc = shape_for(g, p, B, s);
-    if (rc) return rc;
+    StagedParams sp;
+    bool staged = !(flags & EMO_F_NO_STAGING) && ldb % 16 == 0 && ((uintptr_t)lvl % 16) == 0 &&
+                  (!backward || (ldes % 2 == 0 && ((uintptr_t)ES % 16) == 0)) &&
+                  staged_shape(g, p, backward, B, s, sp);
+    if (!staged) {
+        int rc = shape_for(g, p, B, s);
+        if (rc) return rc;
+    }
     PassParams a;
     a.prog = d.entries;
     a.lat = d.lat;
@@ -147,7 +198,16 @@ int launch_pass(const emo_graph *g, bool backward, int64_t B, const uint8_t *lvl
     a.status = status;
     cudaEvent_t ev0 = g_pass_events[backward ? 2 : 0], ev1 = g_pass_events[backward ? 3 : 1];
     if (ev0) EMO_CUDA(cudaEventRecord(ev0, st));
-    if (backward) {
+    if (staged) {
+        sp.p = a;
+        if (backward) {
+            EMO_CUDA(cudaFuncSetAttribute(emo_pass_staged<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s.smem));
+            emo_pass_staged<true><<<s.grid, s.threads, s.smem, st>>>(sp);
+        } else {
+            EMO_CUDA(cudaFuncSetAttribute(emo_pass_staged<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s.smem));
+            emo_pass_staged<false><<<s.grid, s.threads, s.smem, st>>>(sp);
+        }
+    } else if (backward) {
         if (s.smem > 48 * 1024) EMO_CUDA(cudaFuncSetAttribute(emo_pass_plain<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s.smem));
         emo_pass_plain<true><<<s.grid, s.threads, s.smem, st>>>(a);
     } else {
@@ -356,7 +416,7 @@ int emo_graph_program(const emo_graph *g, int dir, int32_t *lanes, int32_t *step
 int emo_workspace_bytes(const emo_graph *g, int64_t B, int need_slack, size_t *out)
 {
     if (!g || !out || B < 0) return EMO_E_INVALID_ARG;
-    size_t bytes = kSmallWs + round_up((size_t)std::max(g->h.rows, 1), 256);
+    size_t bytes = kSmallWs + lvl_area(g);
     if (need_slack) bytes += (size_t)g->h.n * round_up((size_t)B, 16) * sizeof(int64_t);
     if (need_slack == 2) bytes += 4 * round_up((size_t)B * 8, 256) + 256;
     *out = bytes;
@@ -379,7 +439,7 @@ int emo_eval_policies(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t
         if (rc) return rc;
     }
     return launch_pass(g, false, B, lvl, ldb, nullptr, 0, nullptr, nullptr, 0, makespan, energy, nullptr,
-                       nullptr, status, st);
+                       nullptr, status, st, flags);
 }
 
 int emo_slack_batch(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t ldb, int64_t *ES,
@@ -399,7 +459,7 @@ int emo_slack_batch(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t l
         size_t need = 0;
         emo_workspace_bytes(g, B, 1, &need);
         if (!ws || ws_bytes < need) return EMO_E_OOM;
-        es = (int64_t *)((char *)ws + kSmallWs + round_up((size_t)std::max(g->h.rows, 1), 256));
+        es = (int64_t *)((char *)ws + kSmallWs + lvl_area(g));
         ldes = (int64_t)round_up((size_t)B, 16);
     }
     if (flags & EMO_F_VALIDATE) {
@@ -407,10 +467,10 @@ int emo_slack_batch(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t l
         if (rc) return rc;
     }
     int rc = launch_pass(g, false, B, lvl, ldb, es, ldes, nullptr, nullptr, 0, makespan, energy, nullptr,
-                         nullptr, status, st);
+                         nullptr, status, st, flags);
     if (rc) return rc;
     return launch_pass(g, true, B, lvl, ldb, es, ldes, LS, slack, ldo, makespan, energy, slack_sum,
-                       n_critical, status, st);
+                       n_critical, status, st, flags);
 }
 
 int emo_slack(const emo_graph *g, const uint8_t *lvl_one, int64_t *ES, int64_t *LS, int64_t *slack,
@@ -435,8 +495,8 @@ int emo_baseline(const emo_graph *g, int64_t *T0, double *E0, void *ws, size_t w
     if (!ws || ws_bytes < need) return EMO_E_OOM;
     cudaStream_t st = (cudaStream_t)stream;
     uint8_t *lv = (uint8_t *)ws + kSmallWs;
-    EMO_CUDA(cudaMemsetAsync(lv, g->h.L - 1, (size_t)std::max(g->h.rows, 1), st));
-    return launch_pass(g, false, 1, lv, 1, nullptr, 0, nullptr, nullptr, 0, T0, E0, nullptr, nullptr, status, st);
+    EMO_CUDA(cudaMemsetAsync(lv, g->h.L - 1, (size_t)std::max(g->h.rows, 1) * 16, st));
+    return launch_pass(g, false, 1, lv, 16, nullptr, 0, nullptr, nullptr, 0, T0, E0, nullptr, nullptr, status, st);
 }
 
 int64_t emo_target_from_delta(int64_t T0, int64_t delta_ppm)

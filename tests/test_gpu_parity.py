@@ -151,9 +151,15 @@ def test_config_graphs_all_outputs(torch_cuda, emo, oracle_mod, name, scale, B):
     h = emo.load_workload(g)
     r = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n)
     assert_matches(r, r_or, B)
-    # slack only (ES kept in the workspace), same result
+    # slack only (ES kept in the workspace), same result; then the plain-load kernels
     r2 = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, want=("slack",))
     assert np.array_equal(r2["slack"][:, :B], r_or["slack"])
+    r3 = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, flags=emo.EMO_F_NO_STAGING)
+    assert_matches(r3, r_or, B)
+    # an output pitch that is odd (no bulk copies of the ES rows possible) and one that is even
+    for ldo in (B + 1, B + 2):
+        r4 = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, ldo=ldo)
+        assert_matches(r4, r_or, B)
     # single-policy call
     b = B // 2
     one = lv_dev[:, b].contiguous()
