@@ -144,6 +144,7 @@ def main():
     ap.add_argument("--policies", type=int, default=0, help="override the number of policies (profiling a small case)")
     ap.add_argument("--scale", type=float, default=1.0, help="shrink the graph (profiling a small case)")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--sums", action="store_true", help="also produce per-policy slack sums and critical counts")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--flags", type=int, default=0, help="extra EMO_F_* load flags (lanes / look-ahead)")
     args = ap.parse_args()
@@ -191,13 +192,13 @@ def main():
     def step(events=None):
         if events is not None:
             emo.emo_set_pass_events(*events)
-        emo.emo_slack_batch(h, B, lv, ldb, None, None, slack, B, T, E, ss, nc, ws, status)
+        emo.emo_slack_batch(h, B, lv, ldb, None, None, slack, B, T, E, sums[0], sums[1], ws, status, T0=T0, E0=E0)
         if events is not None:
             emo.emo_set_pass_events(None, None, None, None)
-        emo.emo_baseline(h, T0, E0, ws, status)
         emo.emo_select(B, T, E, 0, sel[0:1], sel[1:2], selE, ws, target_dev=T0, delta_ppm=ppm)
 
-    launches_per_step = 5          # forward pass, backward pass, baseline forward pass, 2 selection kernels
+    sums = (ss, nc) if args.sums else (None, None)
+    launches_per_step = 4          # forward pass (with the baseline column), backward pass, 2 selection kernels
     for _ in range(max(args.warmup, 0)):
         step()
     torch.cuda.synchronize()
@@ -253,7 +254,7 @@ def main():
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "int64", "data": "synthetic",
             "config": {"workload": args.workload if args.scale == 1.0 else f"{args.workload} x{args.scale}", "n": n, "m": m, "L": g.L, "policies": B, "passes": "forward+backward",
-                       "slack_materialised": True, "delta_ppm": ppm, "lanes": info.lanes, "steps_fwd": info.steps_fwd,
+                       "slack_materialised": True, "slack_sums": bool(args.sums), "delta_ppm": ppm, "lanes": info.lanes, "steps_fwd": info.steps_fwd,
                        "slots_fwd": info.slots_fwd, "slots_bwd": info.slots_bwd,
                        "l2": "inputs larger than L2 (levels %.1f GB, slack %.1f GB per step)" % (n * ldb / 1e9, n * B * 8 / 1e9),
                        "parallelism": "replicas" if world > 1 else "single"},
@@ -274,14 +275,15 @@ def main():
         hnc = torch.zeros(B, dtype=torch.int32).pin_memory()
         hsel = torch.zeros(4, dtype=torch.int64)
         dev_lvl = torch.empty_like(lv)
-        emo.emo_slack_batch_host(h, B, lv_host, ldb, dev_lvl, slack, B, ppm, hT, hE, hss, hnc, hsel, ws)
+        hsums = (hss, hnc) if args.sums else (None, None)
+        emo.emo_slack_batch_host(h, B, lv_host, ldb, dev_lvl, slack, B, ppm, hT, hE, hsums[0], hsums[1], hsel, ws)
         torch.cuda.synchronize()
         k = max(1, min(args.steps, 5))
         if dist is not None:
             dist.barrier()
         t0 = time.perf_counter()
         for _ in range(k):
-            emo.emo_slack_batch_host(h, B, lv_host, ldb, dev_lvl, slack, B, ppm, hT, hE, hss, hnc, hsel, ws)
+            emo.emo_slack_batch_host(h, B, lv_host, ldb, dev_lvl, slack, B, ppm, hT, hE, hsums[0], hsums[1], hsel, ws)
         torch.cuda.synchronize()
         e2e_s = (time.perf_counter() - t0) / k
         if dist is not None:
@@ -290,7 +292,7 @@ def main():
             e2e_s = float(tt.item())
         assert int(hsel[0]) == int(sel[0].item())
         line["e2e"] = {"value": world * B * m * passes / e2e_s, "unit": UNIT, "ms_per_step": e2e_s * 1e3,
-                       "h2d_bytes_per_step": int(g.n * ldb), "d2h_bytes_per_step": int(B * 28 + 80),
+                       "h2d_bytes_per_step": int(g.n * ldb), "d2h_bytes_per_step": int(B * (28 if args.sums else 16) + 80),
                        "note": "slack matrix stays on the device"}
         del lv_host
 

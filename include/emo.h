@@ -118,13 +118,16 @@ int emo_workspace_bytes(const emo_graph *g, int64_t B, int need_slack, size_t *o
  *   lvl          device uint8 [rows][ldb], ldb >= B.
  *   makespan     device int64 [B];  energy  device fp64 [B].
  *   ws, ws_bytes device scratch of at least emo_workspace_bytes(g, B, 0).
+ *   T0, E0       device int64 [1] / fp64 [1], optional: when given, the default policy P_0 (every
+ *                row at level L-1, Alg. 2 line 1) is evaluated in the same launch as one more
+ *                column and its makespan and energy are written here.
  *   status       device int32, optional: set to a negative code if a kernel detected an error
  *                (left untouched otherwise; the caller zeroes it).
- * B == 0 returns EMO_OK and writes nothing.  Asynchronous on `stream`.
+ * B == 0 writes nothing but T0 / E0.  Asynchronous on `stream`.
  */
 int emo_eval_policies(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t ldb,
-                      int64_t *makespan, double *energy, void *ws, size_t ws_bytes,
-                      int32_t *status, uint32_t flags, void *stream);
+                      int64_t *makespan, double *energy, int64_t *T0, double *E0,
+                      void *ws, size_t ws_bytes, int32_t *status, uint32_t flags, void *stream);
 
 /*
  * emo_slack_batch - forward and backward pass for B policies: earliest start ES, latest start LS
@@ -134,12 +137,14 @@ int emo_eval_policies(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t
  *   makespan, energy device [B] (required).
  *   slack_sum       device int64 [B], optional: sum of slack over nodes.
  *   n_critical      device int32 [B], optional: number of nodes with slack 0.
+ *   T0, E0          optional, as in emo_eval_policies.
  *   ws              at least emo_workspace_bytes(g, B, ES == NULL).
  * Asynchronous on `stream`.
  */
 int emo_slack_batch(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t ldb,
                     int64_t *ES, int64_t *LS, int64_t *slack, int64_t ldo,
                     int64_t *makespan, double *energy, int64_t *slack_sum, int32_t *n_critical,
+                    int64_t *T0, double *E0,
                     void *ws, size_t ws_bytes, int32_t *status, uint32_t flags, void *stream);
 
 /*
@@ -210,12 +215,13 @@ int emo_set_pass_events(void *fwd_start, void *fwd_stop, void *bwd_start, void *
 
 /*
  * Inspection of the compiled evaluation program (host memory owned by the handle; valid until
- * emo_graph_free).  dir 0 = forward, 1 = backward.  entries is [steps][lanes][4] uint32,
- * lat is uint32 [steps*lanes][Lp], Lp = row stride (a power of two >= L).  Used by host-side
- * tests of the scheduler; not needed to evaluate anything.
+ * emo_graph_free).  dir 0 = forward, 1 = backward.  entries is [steps][lanes][8] uint32, rows is
+ * uint32 [steps*lanes] (policy row read by the entry, 0xFFFFFFFF = none), lat is uint32
+ * [steps*lanes][Lp], Lp = row stride (a power of two >= max(L, 4)).  Used by host-side tests of
+ * the scheduler; not needed to evaluate anything.
  */
 int emo_graph_program(const emo_graph *g, int dir, int32_t *lanes, int32_t *steps, int32_t *slots,
-                      int32_t *Lp, const uint32_t **entries, const uint32_t **lat);
+                      int32_t *Lp, const uint32_t **entries, const uint32_t **rows, const uint32_t **lat);
 
 #ifdef __cplusplus
 }

@@ -52,7 +52,8 @@ int pick_lanes(int64_t n_ops, int depth)
 }
 
 int compile_program(const HostGraph &g, const int64_t *lat, const double *energy, bool backward,
-                    int lanes, int lookahead, Program &out, std::string &err)
+                    int lanes, int lookahead, const std::vector<uint32_t> *row_in_other, Program &out,
+                    std::string &err)
 {
     const int32_t n = g.n;
     const int L = g.L;
@@ -269,18 +270,24 @@ int compile_program(const HostGraph &g, const int64_t *lat, const double *energy
     // ---- slots ---------------------------------------------------------------------------------
     // An operand is read from the warp's register when the producing op was the previous op of the
     // same warp; every other operand is read from the producer's slot.  A slot lives from the
-    // producer's step to the last step that reads it and is reused from the following step on.
+    // producer's step to the last step that reads it.  The warps of a group only meet at a barrier
+    // every kSyncSteps steps and otherwise run at their own pace, so a slot is reused no earlier
+    // than the first step of the block after its last read: the barrier between the two blocks
+    // orders the last read before the next write.  Readers find out that a value has been written
+    // from a per-slot phase counter; the entry carries the phase parity of every value it touches.
     std::vector<int32_t> last_use((size_t)N, -1);
     for (int32_t i = 0; i < N; ++i)
         for (int32_t p : ops[i].preds)
             if (!(warp_of[p] == warp_of[i] && prev_on_warp[i] == p)) last_use[p] = std::max(last_use[p], step_of[i]);
     std::vector<int32_t> slot_of((size_t)N, -1);
+    std::vector<uint8_t> parity_of((size_t)N, 0);
     {
+        std::vector<uint8_t> phase;   // number of values written to a slot so far, mod 2
         std::priority_queue<int32_t, std::vector<int32_t>, std::greater<int32_t>> free_ids;
         std::priority_queue<Key, std::vector<Key>, std::greater<Key>> busy;   // (last use step, slot)
         int32_t next_id = 0;
         for (int32_t s = 0; s < S; ++s) {
-            while (!busy.empty() && busy.top().first < s) {
+            while (!busy.empty() && busy.top().first / kSyncSteps < s / kSyncSteps) {
                 free_ids.push(busy.top().second);
                 busy.pop();
             }
@@ -293,8 +300,11 @@ int compile_program(const HostGraph &g, const int64_t *lat, const double *energy
                     free_ids.pop();
                 } else {
                     id = next_id++;
+                    phase.push_back(0);
                 }
                 slot_of[i] = id;
+                parity_of[i] = phase[id];
+                phase[id] ^= 1;
                 busy.push({last_use[i], id});
             }
         }
@@ -308,38 +318,55 @@ int compile_program(const HostGraph &g, const int64_t *lat, const double *energy
 
     // ---- entries and schedule-ordered tables -------------------------------------------------
     const size_t Q = (size_t)S * lanes;
-    out.entries.assign(Q * 4, 0);
+    out.entries.assign(Q * kEntryWords, 0);
+    out.rows.assign(Q, kNone);
+    out.pos_of_node.assign((size_t)std::max(n, 1), kNone);
     out.lat.assign(Q * Lp, 0);
     if (!backward) out.energy.assign(Q * Lp, 0.0);
     for (int32_t s = 0; s < S; ++s) {
         for (int w = 0; w < lanes; ++w) {
             int32_t i = sched[s][w];
             size_t q = (size_t)s * lanes + w;
-            uint32_t *en = &out.entries[q * 4];
+            uint32_t *en = &out.entries[q * kEntryWords];
             en[0] = kNone;
-            en[1] = kNone;
+            en[4] = kNone;
+            out.rows[q] = kNone;
             if (i < 0) continue;
             const Op &o = ops[i];
             uint32_t flags = kValid;
-            uint32_t operands = 0;
+            uint32_t operands = 0, operands_hi = 0;
             int np = 0;
             for (int32_t p : o.preds) {
                 if (warp_of[p] == w && prev_on_warp[i] == p) {
                     flags |= kRegPred;
                 } else {
                     if (np < 4) operands |= (uint32_t)slot_of[p] << (8 * np);
-                    else flags |= (uint32_t)slot_of[p] << (16 + 8 * (np - 4));
+                    else operands_hi |= (uint32_t)slot_of[p] << (8 * (np - 4));
+                    flags |= (uint32_t)parity_of[p] << (kOperandParityShift + np);
                     ++np;
                 }
             }
             flags |= (uint32_t)np << kNPredShift;
-            if (slot_of[i] >= 0) flags |= kWriteSlot | ((uint32_t)slot_of[i] << kOutShift);
+            if (slot_of[i] >= 0)
+                flags |= kWriteSlot | ((uint32_t)slot_of[i] << kOutShift) | ((uint32_t)parity_of[i] << kOutParityShift);
             if (o.node < 0) {
                 flags |= kAux;
             } else {
                 int32_t v = o.node;
-                en[1] = (uint32_t)v;
-                if (g.group[v] >= 0) en[0] = (uint32_t)g.group[v];
+                // word 0: the row this entry addresses in the kernel's main per-node array - the
+                // node's position in the other direction's program when that is known (the forward
+                // pass leaves ES where the backward pass will stream it from), else the node id
+                en[0] = row_in_other ? (*row_in_other)[v] : (uint32_t)v;
+                en[4] = (uint32_t)v;
+                out.pos_of_node[v] = (uint32_t)q;
+                // a node whose duration and energy do not depend on the level needs no level
+                bool constant = true;
+                for (int l = 1; l < L && constant; ++l)
+                    constant = lat[(size_t)v * L + l] == lat[(size_t)v * L] && energy[(size_t)v * L + l] == energy[(size_t)v * L];
+                if (g.group[v] >= 0 && !constant) {
+                    out.rows[q] = (uint32_t)g.group[v];
+                    flags |= (uint32_t)(Lp - 1) << kMaskShift;
+                }
                 if (cp[i + 1] == cp[i]) flags |= kTerminal;
                 for (int l = 0; l < Lp; ++l) {
                     int ll = l < L ? l : L - 1;
@@ -347,8 +374,9 @@ int compile_program(const HostGraph &g, const int64_t *lat, const double *energy
                     if (!backward) out.energy[q * Lp + l] = energy[(size_t)v * L + ll];
                 }
             }
-            en[2] = flags;
-            en[3] = operands;
+            en[1] = flags;
+            en[2] = operands;
+            en[3] = operands_hi;
         }
     }
     return EMO_OK;

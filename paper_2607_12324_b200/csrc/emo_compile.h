@@ -20,14 +20,24 @@ constexpr int kMaxSlotPreds = 6;      // slot operands one entry can name
 constexpr int kMaxSlots = 250;        // exchange slots per policy group (8-bit ids)
 constexpr int kMaxLanes = 32;
 
-// entry word 2
+// Program entry (32 bytes, 8 words): word 0 = row the entry addresses in the kernel's main per-node
+// array (kNone for helper ops and idle entries); word 1 = flags; word 2 = operand slots 0..3,
+// word 3 = operand slots 4..5 (8 bits each); word 4 = node id in the caller's numbering (kNone for
+// helper ops and idle entries); words 5..7 unused.
+constexpr int kEntryWords = 8;
 constexpr uint32_t kValid = 1u, kRegPred = 2u, kWriteSlot = 4u, kTerminal = 8u, kAux = 0x80u;
 constexpr int kNPredShift = 4;        // bits 4..6: number of slot operands
-constexpr int kOutShift = 8;          // bits 8..15: slot written; bits 16..31: operand slots 4 and 5
+constexpr int kMaskShift = 8;         // bits 8..15: mask applied to the level byte (0 = node ignores the policy)
+constexpr int kOutShift = 16;         // bits 16..23: slot written
+constexpr int kOutParityShift = 24;   // bit 24: phase parity of the value written
+constexpr int kOperandParityShift = 25;   // bits 25..30: phase parity of each operand's value
+constexpr int kSyncSteps = 8;         // the warps of a group meet at a barrier every kSyncSteps steps
 
 struct Program {
     int lanes = 0, steps = 0, slots = 0, aux = 0, Lp = 0;
-    std::vector<uint32_t> entries;    // [steps][lanes][4]: {policy row, node id, flags|out slot|operands 4-5, operand slots 0-3}
+    std::vector<uint32_t> entries;    // [steps][lanes][kEntryWords], see above
+    std::vector<uint32_t> pos_of_node;   // [n] index (step*lanes + lane) of the entry that handles node v
+    std::vector<uint32_t> rows;       // [steps][lanes] policy row whose level the entry reads (kNone: none)
     std::vector<uint32_t> lat;        // [steps*lanes][Lp] durations of the scheduled node per level
     std::vector<double> energy;       // [steps*lanes][Lp], forward program only
 };
@@ -42,8 +52,10 @@ struct HostGraph {
 
 // Builds the forward (backward = false) or backward program.  lanes <= 0 picks a value from the
 // graph's shape.  Returns 0 or an EMO_E_* code and a message in err.
+// row_in_other (optional, [n]): what to put into word 0 of a node's entry instead of its id.
 int compile_program(const HostGraph &g, const int64_t *lat, const double *energy, bool backward,
-                    int lanes, int lookahead, Program &out, std::string &err);
+                    int lanes, int lookahead, const std::vector<uint32_t> *row_in_other, Program &out,
+                    std::string &err);
 
 int pick_lanes(int64_t n_ops, int depth);
 

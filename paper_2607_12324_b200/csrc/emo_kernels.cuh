@@ -6,22 +6,43 @@
 
 #include "emo_compile.h"
 
+// One pass (forward or backward) over the step program.
+//
+// Device layout of a program: an array of fixed-size records, one per (step, lane) in schedule
+// order.  A record is the 32-byte entry, the node's duration row (Lp x uint32) and, in the forward
+// program, its energy row (Lp x fp64).  `rows` holds, per record, the policy row whose level the
+// entry reads (kNone: none).
+//
+// Earliest start times travel from the forward to the backward pass in one of two layouts: `ES`,
+// [n][ldes] in the caller's numbering (also the caller-visible ES output), or `spill`, laid out
+// [policy tile][row of the backward program][spill_ptile] so that the backward pass streams the
+// rows of a run of steps with one contiguous copy.
+//
+// Columns: policies 0..B-1 come from the level matrix; when want_base is set, column B is a
+// virtual policy with every row at level L-1 (the default, maximum-frequency policy P_0 of Alg. 2),
+// whose makespan and energy go to base_T / base_E.
 struct PassParams {
-    const uint4 *prog;        // [steps][lanes] program entries
-    const uint32_t *lat;      // [steps*lanes][Lp]
-    const double *en;         // [steps*lanes][Lp] (forward only)
-    int steps, lanes, Lp, Lmask, slots, groups;
+    const unsigned char *rec;  // records
+    const uint32_t *rows;      // [steps*lanes]
+    int rec_bytes;             // 32 + Lp*4 (+ Lp*8 forward)
+    int steps, lanes, Lp, L, slots, groups;
+    int want_base;
     int64_t B;
     const uint8_t *lvl;       // [rows][ldb]
     int64_t ldb;
-    int64_t *ES;              // forward: written when not NULL; backward: read
+    int64_t *ES;              // forward: written when not NULL; backward (plain kernel): read
     int64_t ldes;
+    int64_t *spill;           // staged kernels: forward writes, backward reads
+    int64_t spill_rows;       // rows of the backward program (steps * lanes)
+    int spill_ptile;          // policies per tile of the spill
     int64_t *LS, *slack;      // backward outputs, optional
     int64_t ldo;
     int64_t *makespan;        // forward: written; backward: read
     double *energy;
     int64_t *slack_sum;
     int32_t *n_critical;
+    int64_t *base_T;
+    double *base_E;
     int32_t *status;
 };
 
@@ -40,12 +61,13 @@ __device__ __forceinline__ void emo_group_barrier(int id, int nthreads)
 }
 
 // ------------------------------------------------------------------------------------------------
-// Pass kernel, plain loads.  One warp = 32 policies of one schedule lane; `lanes` warps form a group
-// and meet at a named barrier after every step.  Forward (BWD = false): Eq. 1 with the value
-// C_v kept in h; makespan over terminal nodes (equal to the maximum over all nodes because
-// durations are >= 0), energy accumulated per warp in step order and combined in lane order.
-// Backward: the same recurrence on the reversed graph gives Q_v = t_v + max over successors of Q_u,
-// so LS_v = T - Q_v and slack_v = LS_v - ES_v.
+// Pass kernel, plain loads (used when the caller's pitches or pointers rule out bulk copies).
+// One warp = 32 policies of one schedule lane; `lanes` warps form a group and meet at a named
+// barrier after every step.  Forward (BWD = false): Eq. 1 with the value C_v kept in h; makespan
+// over terminal nodes (equal to the maximum over all nodes because durations are >= 0), energy
+// accumulated per warp in step order and combined in lane order.  Backward: the same recurrence on
+// the reversed graph gives Q_v = t_v + max over successors of Q_u, so LS_v = T - Q_v and
+// slack_v = LS_v - ES_v.
 // ------------------------------------------------------------------------------------------------
 template <bool BWD>
 __global__ void __launch_bounds__(1024) emo_pass_plain(PassParams p)
@@ -57,6 +79,7 @@ __global__ void __launch_bounds__(1024) emo_pass_plain(PassParams p)
     const int chain = warp - group * p.lanes;
     const int64_t b = ((int64_t)blockIdx.x * p.groups + group) * 32 + lane;
     const bool active = b < p.B;
+    const bool is_base = !BWD && p.want_base && b == p.B;
     long long *slots = reinterpret_cast<long long *>(emo_smem) + (size_t)group * p.slots * 32 + lane;
     unsigned char *part_base = emo_smem + (size_t)p.groups * p.slots * 256;
 
@@ -65,21 +88,21 @@ __global__ void __launch_bounds__(1024) emo_pass_plain(PassParams p)
     long long tmax = 0, ssum = 0;
     int ncrit = 0;
     const long long T = (BWD && active) ? p.makespan[b] : 0;
-    const uint4 *pe = p.prog + chain;
-    uint4 e = make_uint4(emo::kNone, emo::kNone, 0u, 0u);
-    if (p.steps > 0) e = __ldg(pe);
     for (int t = 0; t < p.steps; ++t) {
-        uint4 nxt = make_uint4(emo::kNone, emo::kNone, 0u, 0u);
-        if (t + 1 < p.steps) nxt = __ldg(pe + (size_t)(t + 1) * p.lanes);
-        if (e.z & emo::kValid) {
+        const size_t q = (size_t)t * p.lanes + chain;
+        const unsigned char *r = p.rec + q * p.rec_bytes;
+        uint4 e = __ldg(reinterpret_cast<const uint4 *>(r));
+        e.x = __ldg(reinterpret_cast<const unsigned *>(r + 16));      // the plain kernel addresses by node id
+        if (e.y & emo::kValid) {
             unsigned lv = 0;
-            if (e.x != emo::kNone && active) lv = p.lvl[(size_t)e.x * p.ldb + b];
-            lv &= (unsigned)p.Lmask;
-            const size_t q = ((size_t)t * p.lanes + chain) * p.Lp + lv;
-            const long long dur = (long long)__ldg(p.lat + q);
-            long long start = (e.z & emo::kRegPred) ? h : 0;
-            const int np = (e.z >> emo::kNPredShift) & 7;
-            unsigned long long ops = (unsigned long long)e.w | ((unsigned long long)(e.z >> 16) << 32);
+            const uint32_t row = __ldg(p.rows + q);
+            if (row != emo::kNone && active) lv = p.lvl[(size_t)row * p.ldb + b];
+            if (is_base) lv = (unsigned)(p.L - 1);
+            lv &= (e.y >> emo::kMaskShift) & 255u;
+            const long long dur = (long long)__ldg(reinterpret_cast<const uint32_t *>(r + 32) + lv);
+            long long start = (e.y & emo::kRegPred) ? h : 0;
+            const int np = (e.y >> emo::kNPredShift) & 7;
+            unsigned long long ops = (unsigned long long)e.z | ((unsigned long long)e.w << 32);
             for (int k = 0; k < np; ++k) {
                 long long x = slots[(unsigned)(ops & 255u) * 32];
                 ops >>= 8;
@@ -87,22 +110,21 @@ __global__ void __launch_bounds__(1024) emo_pass_plain(PassParams p)
             }
             h = start + dur;
             if (!BWD) {
-                eacc += __ldg(p.en + q);
-                if (e.z & emo::kTerminal) tmax = h > tmax ? h : tmax;
-                if (p.ES && e.y != emo::kNone && active) p.ES[(size_t)e.y * p.ldes + b] = start;
-            } else if (e.y != emo::kNone && active) {
+                eacc += __ldg(reinterpret_cast<const double *>(r + 32 + p.Lp * 4) + lv);
+                if (e.y & emo::kTerminal) tmax = h > tmax ? h : tmax;
+                if (p.ES && e.x != emo::kNone && active) p.ES[(size_t)e.x * p.ldes + b] = start;
+            } else if (e.x != emo::kNone && active) {
                 const long long ls = T - h;
-                const long long es = p.ES[(size_t)e.y * p.ldes + b];
+                const long long es = p.ES[(size_t)e.x * p.ldes + b];
                 const long long sl = ls - es;
-                if (p.LS) p.LS[(size_t)e.y * p.ldo + b] = ls;
-                if (p.slack) p.slack[(size_t)e.y * p.ldo + b] = sl;
+                if (p.LS) p.LS[(size_t)e.x * p.ldo + b] = ls;
+                if (p.slack) p.slack[(size_t)e.x * p.ldo + b] = sl;
                 ssum += sl;
                 ncrit += (sl == 0);
             }
-            if (e.z & emo::kWriteSlot) slots[((e.z >> emo::kOutShift) & 255u) * 32] = h;
+            if (e.y & emo::kWriteSlot) slots[((e.y >> emo::kOutShift) & 255u) * 32] = h;
         }
         if (p.lanes > 1) emo_group_barrier(group + 1, p.lanes * 32);
-        e = nxt;
     }
 
     // combine the warps of a group in lane order (fixed order: run-to-run identical energy)
@@ -115,7 +137,7 @@ __global__ void __launch_bounds__(1024) emo_pass_plain(PassParams p)
         reinterpret_cast<long long *>(pd)[1] = (long long)ncrit;
     }
     __syncthreads();
-    if (chain == 0 && active) {
+    if (chain == 0 && (active || is_base)) {
         const double *g0 = reinterpret_cast<const double *>(part_base) + ((size_t)(group * p.lanes) * 32 + lane) * 2;
         if (!BWD) {
             double es = 0.0;
@@ -125,8 +147,13 @@ __global__ void __launch_bounds__(1024) emo_pass_plain(PassParams p)
                 long long x = reinterpret_cast<const long long *>(g0)[(size_t)k * 64 + 1];
                 tm = x > tm ? x : tm;
             }
-            p.makespan[b] = tm;
-            p.energy[b] = es;
+            if (is_base) {
+                if (p.base_T) *p.base_T = tm;
+                if (p.base_E) *p.base_E = es;
+            } else {
+                p.makespan[b] = tm;
+                p.energy[b] = es;
+            }
         } else {
             long long ss = 0, nc = 0;
             for (int k = 0; k < p.lanes; ++k) {

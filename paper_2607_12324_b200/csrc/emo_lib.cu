@@ -16,9 +16,9 @@
 using namespace emo;
 
 struct DevProgram {
-    uint4 *entries = nullptr;
-    uint32_t *lat = nullptr;
-    double *energy = nullptr;
+    unsigned char *rec = nullptr;   // records: entry, duration row, (forward) energy row
+    uint32_t *rows = nullptr;
+    int rec_bytes = 0;
 };
 
 struct emo_graph {
@@ -61,19 +61,25 @@ int upload(T **dst, const void *src, size_t bytes)
 
 int upload_program(const Program &p, DevProgram &d)
 {
-    int rc = upload(&d.entries, p.entries.data(), p.entries.size() * sizeof(uint32_t));
+    const size_t Q = (size_t)p.steps * p.lanes;
+    const bool fwd = !p.energy.empty();
+    d.rec_bytes = 32 + p.Lp * 4 + (fwd ? p.Lp * 8 : 0);
+    std::vector<unsigned char> rec(Q * d.rec_bytes);
+    for (size_t q = 0; q < Q; ++q) {
+        unsigned char *r = rec.data() + q * d.rec_bytes;
+        std::memcpy(r, &p.entries[q * kEntryWords], 32);
+        std::memcpy(r + 32, &p.lat[q * p.Lp], (size_t)p.Lp * 4);
+        if (fwd) std::memcpy(r + 32 + p.Lp * 4, &p.energy[q * p.Lp], (size_t)p.Lp * 8);
+    }
+    int rc = upload(&d.rec, rec.data(), rec.size());
     if (rc) return rc;
-    rc = upload(&d.lat, p.lat.data(), p.lat.size() * sizeof(uint32_t));
-    if (rc) return rc;
-    if (!p.energy.empty()) rc = upload(&d.energy, p.energy.data(), p.energy.size() * sizeof(double));
-    return rc;
+    return upload(&d.rows, p.rows.data(), p.rows.size() * sizeof(uint32_t));
 }
 
 void free_program(DevProgram &d)
 {
-    if (d.entries) cudaFree(d.entries);
-    if (d.lat) cudaFree(d.lat);
-    if (d.energy) cudaFree(d.energy);
+    if (d.rec) cudaFree(d.rec);
+    if (d.rows) cudaFree(d.rows);
     d = DevProgram();
 }
 
@@ -94,6 +100,20 @@ __int128 host_longest(const HostGraph &h, F dur)
 
 size_t lvl_area(const emo_graph *g) { return round_up((size_t)std::max(g->h.rows, 1) * 16, 256); }
 
+// lanes from the graph's shape: nodes per hop level plus a little spare capacity
+int pick_lanes_for(const HostGraph &h)
+{
+    std::vector<int32_t> hop((size_t)std::max(h.n, 1), 0);
+    int32_t depth = 0;
+    for (int32_t v = 0; v < h.n; ++v) {
+        int32_t a = 0;
+        for (int64_t e = h.row_ptr[v]; e < h.row_ptr[v + 1]; ++e) a = std::max(a, hop[h.col[e]] + 1);
+        hop[v] = a;
+        depth = std::max(depth, a + 1);
+    }
+    return pick_lanes(h.n, depth);
+}
+
 struct LaunchShape {
     int groups, grid, threads;
     size_t smem;
@@ -101,9 +121,9 @@ struct LaunchShape {
 
 // Policy groups (32 policies each) per block: enough to give every SM one block, bounded by the
 // block size, the named barriers (ids 1..15) and shared memory.
-int shape_for(const emo_graph *g, const Program &p, int64_t B, LaunchShape &s)
+int shape_for(const emo_graph *g, const Program &p, int64_t NB, LaunchShape &s)
 {
-    int64_t n_groups = (B + 31) / 32;
+    int64_t n_groups = (NB + 31) / 32;
     int gmax = std::min(32 / p.lanes, 15);
     if (gmax < 1) return EMO_E_UNSUPPORTED;
     size_t per_group = (size_t)p.slots * 256 + (size_t)p.lanes * 32 * 16;
@@ -118,76 +138,112 @@ int shape_for(const emo_graph *g, const Program &p, int64_t B, LaunchShape &s)
     return EMO_OK;
 }
 
-// Shape of the staged kernel: groups per block as above (one more warp produces), then as many
-// steps per stage as fit beside the slots.  Returns false when the staged kernel cannot be used.
-bool staged_shape(const emo_graph *g, const Program &p, bool backward, int64_t B, LaunchShape &s, StagedParams &sp)
+// Shape of the staged kernel: groups of 64 policies (two per thread), one more warp produces, then
+// as many steps per stage as fit beside the slots.  Returns false when it cannot be used.
+bool staged_shape(const emo_graph *g, const Program &p, int rec_bytes, bool backward, int64_t NB, LaunchShape &s,
+                  StagedParams &sp)
 {
     if (p.steps == 0 || !g->smem_optin) return false;
-    int64_t n_groups = (B + 31) / 32;
+    int64_t n_groups = (NB + 63) / 64;
     int gmax = std::min(31 / p.lanes, 15);
     if (gmax < 1) return false;
     int64_t want = (n_groups + g->sm_count - 1) / g->sm_count;
     int G = (int)std::max<int64_t>(1, std::min<int64_t>(gmax, want));
     const size_t budget = g->smem_optin;
+    static const int kTry[5][2] = {{16, 4}, {16, 3}, {8, 4}, {8, 3}, {8, 2}};   // {steps per stage, stages}
     for (; G >= 1; --G) {
-        const size_t P = 32 * (size_t)G;
-        const size_t fixed = (size_t)G * p.slots * 256 + (size_t)G * p.lanes * 512 + 256;
-        const size_t per_step = (size_t)p.lanes * (16 + (size_t)p.Lp * 4 + (backward ? 0 : (size_t)p.Lp * 8) + P + (backward ? P * 8 : 0));
-        if (fixed + kStages * per_step > budget) continue;
-        int sc = (int)std::min<size_t>(16, (budget - fixed) / (kStages * per_step));
-        sc = std::min(sc, std::max(1, p.steps));
-        const size_t ne = (size_t)sc * p.lanes;
-        sp.sc = sc;
-        sp.ptile = (int)P;
-        sp.off_lat = (unsigned)(ne * 16);
-        sp.off_en = sp.off_lat + (unsigned)(ne * p.Lp * 4);
-        sp.off_lvl = sp.off_en + (backward ? 0u : (unsigned)(ne * p.Lp * 8));
-        sp.off_es = sp.off_lvl + (unsigned)(ne * P);
-        sp.stage_bytes = (unsigned)round_up(sp.off_es + (backward ? ne * P * 8 : 0), 128);
-        sp.off_part = (unsigned)((size_t)G * p.slots * 256);
-        sp.off_bar = sp.off_part + (unsigned)((size_t)G * p.lanes * 512);
-        sp.off_stage0 = (unsigned)round_up(sp.off_bar + 256, 128);
-        s.groups = G;
-        s.grid = (int)((n_groups + G - 1) / G);
-        s.threads = (G * p.lanes + 1) * 32;
-        s.smem = sp.off_stage0 + (size_t)kStages * sp.stage_bytes;
-        if (s.smem > budget) continue;
-        return true;
+        const size_t P = 64 * (size_t)G;
+        const size_t fixed = (size_t)G * p.slots * kSlotStride + (size_t)G * p.lanes * 1024 + 256 + 128;
+        const size_t per_step = (size_t)p.lanes * ((size_t)rec_bytes + P + (backward ? P * 8 : 0));
+        for (int t = 0; t < 5; ++t) {
+            const int sc = kTry[t][0], stages = kTry[t][1];
+            const size_t ne = (size_t)sc * p.lanes;
+            const size_t stage_bytes = round_up(ne * ((size_t)rec_bytes + P + (backward ? P * 8 : 0)), 128);
+            if (fixed + stages * stage_bytes > budget) continue;
+            (void)per_step;
+            sp.sc = sc;
+            sp.stages = stages;
+            sp.ptile = (int)P;
+            sp.off_lvl = (unsigned)(ne * rec_bytes);
+            sp.off_es = sp.off_lvl + (unsigned)(ne * P);
+            sp.stage_bytes = (unsigned)stage_bytes;
+            sp.off_part = (unsigned)round_up((size_t)G * p.slots * kSlotStride, 16);
+            sp.off_bar = sp.off_part + (unsigned)((size_t)G * p.lanes * 1024);
+            sp.off_stage0 = (unsigned)round_up(sp.off_bar + 256, 128);
+            s.groups = G;
+            s.grid = (int)((n_groups + G - 1) / G);
+            s.threads = (G * p.lanes + 1) * 32;
+            s.smem = sp.off_stage0 + (size_t)stages * sp.stage_bytes;
+            if (s.smem > budget) continue;
+            return true;
+        }
     }
     return false;
 }
 
-int launch_pass(const emo_graph *g, bool backward, int64_t B, const uint8_t *lvl, int64_t ldb,
-                int64_t *ES, int64_t ldes, int64_t *LS, int64_t *slack, int64_t ldo,
+// How the two passes of one call will run: both staged (earliest starts travel through the tiled
+// spill) or both with the plain kernels (through an [n][ldes] array).
+struct PassPlan {
+    bool staged = false;
+    LaunchShape sf, sb;       // forward / backward launch shapes
+    StagedParams pf, pb;
+    size_t spill_bytes = 0;   // tiled spill: [tiles][rows of the backward program][backward tile]
+};
+
+bool aligned16(const void *q) { return ((uintptr_t)q % 16) == 0; }
+
+// Decides the plan for B policies (+ the virtual baseline column in the forward pass).
+int make_plan(const emo_graph *g, int64_t B, bool want_base, bool need_bwd, const uint8_t *lvl, int64_t ldb,
+              int64_t ldes_plain, int64_t ldo, uint32_t flags, PassPlan &pl)
+{
+    const int64_t big = (int64_t)1 << 28;
+    const int64_t NBf = B + (want_base ? 1 : 0);
+    pl.staged = !(flags & EMO_F_NO_STAGING) && ldb % 16 == 0 && aligned16(lvl) && ldb < big && ldes_plain < big && ldo < big &&
+                staged_shape(g, g->fwd, g->dfwd.rec_bytes, false, NBf, pl.sf, pl.pf) &&
+                (!need_bwd || staged_shape(g, g->bwd, g->dbwd.rec_bytes, true, B, pl.sb, pl.pb));
+    if (!pl.staged) {
+        int rc = shape_for(g, g->fwd, NBf, pl.sf);
+        if (rc == EMO_OK && need_bwd) rc = shape_for(g, g->bwd, B, pl.sb);
+        return rc;
+    }
+    if (need_bwd) {
+        const size_t tiles = ((size_t)B + pl.pb.ptile - 1) / pl.pb.ptile;
+        pl.spill_bytes = tiles * (size_t)g->bwd.steps * g->bwd.lanes * pl.pb.ptile * sizeof(int64_t);
+    }
+    return EMO_OK;
+}
+
+// One pass under a plan.  Forward: B policies from lvl plus, when base_T/base_E are given, the
+// virtual all-max column.
+int launch_pass(const emo_graph *g, const PassPlan &pl, bool backward, int64_t B, const uint8_t *lvl, int64_t ldb,
+                int64_t *ES, int64_t ldes, int64_t *spill, int64_t *LS, int64_t *slack, int64_t ldo,
                 int64_t *makespan, double *energy, int64_t *slack_sum, int32_t *n_critical,
-                int32_t *status, cudaStream_t st, uint32_t flags = 0)
+                int64_t *base_T, double *base_E, int32_t *status, cudaStream_t st)
 {
     const Program &p = backward ? g->bwd : g->fwd;
     const DevProgram &d = backward ? g->dbwd : g->dfwd;
-    LaunchShape s;
-    StagedParams sp;
-    bool staged = !(flags & EMO_F_NO_STAGING) && ldb % 16 == 0 && ((uintptr_t)lvl % 16) == 0 &&
-                  (!backward || (ldes % 2 == 0 && ((uintptr_t)ES % 16) == 0)) &&
-                  staged_shape(g, p, backward, B, s, sp);
-    if (!staged) {
-        int rc = shape_for(g, p, B, s);
-        if (rc) return rc;
-    }
+    const int want_base = (!backward && (base_T || base_E)) ? 1 : 0;
+    if (B + want_base == 0) return EMO_OK;
+    const LaunchShape &s = backward ? pl.sb : pl.sf;
     PassParams a;
-    a.prog = d.entries;
-    a.lat = d.lat;
-    a.en = d.energy;
+    a.rec = d.rec;
+    a.rows = d.rows;
+    a.rec_bytes = d.rec_bytes;
     a.steps = p.steps;
     a.lanes = p.lanes;
     a.Lp = p.Lp;
-    a.Lmask = p.Lp - 1;
+    a.L = g->h.L;
     a.slots = p.slots;
     a.groups = s.groups;
+    a.want_base = want_base;
     a.B = B;
     a.lvl = lvl;
     a.ldb = ldb;
     a.ES = ES;
     a.ldes = ldes;
+    a.spill = spill;
+    a.spill_rows = (int64_t)g->bwd.steps * g->bwd.lanes;
+    a.spill_ptile = pl.staged ? pl.pb.ptile : 64;
     a.LS = LS;
     a.slack = slack;
     a.ldo = ldo;
@@ -195,18 +251,22 @@ int launch_pass(const emo_graph *g, bool backward, int64_t B, const uint8_t *lvl
     a.energy = energy;
     a.slack_sum = slack_sum;
     a.n_critical = n_critical;
+    a.base_T = base_T;
+    a.base_E = base_E;
     a.status = status;
     cudaEvent_t ev0 = g_pass_events[backward ? 2 : 0], ev1 = g_pass_events[backward ? 3 : 1];
     if (ev0) EMO_CUDA(cudaEventRecord(ev0, st));
-    if (staged) {
+    if (pl.staged) {
+        StagedParams sp = backward ? pl.pb : pl.pf;
         sp.p = a;
-        if (backward) {
-            EMO_CUDA(cudaFuncSetAttribute(emo_pass_staged<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s.smem));
-            emo_pass_staged<true><<<s.grid, s.threads, s.smem, st>>>(sp);
-        } else {
-            EMO_CUDA(cudaFuncSetAttribute(emo_pass_staged<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s.smem));
-            emo_pass_staged<false><<<s.grid, s.threads, s.smem, st>>>(sp);
-        }
+        sp.vec_es = (ES && ldes % 2 == 0 && aligned16(ES)) ? 1 : 0;
+        sp.vec_out = (ldo % 2 == 0 && aligned16(LS) && aligned16(slack)) ? 1 : 0;
+        sp.want_sums = (slack_sum || n_critical) ? 1 : 0;
+        // two register budgets: blocks of at most 512 threads may use 128 registers per thread
+        void (*kern)(StagedParams) = backward ? (s.threads <= 512 ? emo_pass_pair<true, 512> : emo_pass_pair<true, 1024>)
+                                              : (s.threads <= 512 ? emo_pass_pair<false, 512> : emo_pass_pair<false, 1024>);
+        EMO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s.smem));
+        kern<<<s.grid, s.threads, s.smem, st>>>(sp);
     } else if (backward) {
         if (s.smem > 48 * 1024) EMO_CUDA(cudaFuncSetAttribute(emo_pass_plain<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s.smem));
         emo_pass_plain<true><<<s.grid, s.threads, s.smem, st>>>(a);
@@ -334,8 +394,11 @@ int emo_graph_load(int32_t n, const int64_t *row_ptr, const int32_t *col, const 
         int lanes = (int)((flags >> 8) & 0xFF);
         int look = (int)((flags >> 16) & 0xFF);
         std::string err;
-        int rc = compile_program(h, lat, energy, false, lanes, look, g->fwd, err);
-        if (rc == EMO_OK) rc = compile_program(h, lat, energy, true, g->fwd.lanes, look, g->bwd, err);
+        // backward first: the forward entries name the row of the backward program that will read
+        // the node's earliest start
+        if (lanes <= 0) lanes = pick_lanes_for(h);
+        int rc = compile_program(h, lat, energy, true, lanes, look, nullptr, g->bwd, err);
+        if (rc == EMO_OK) rc = compile_program(h, lat, energy, false, g->bwd.lanes, look, &g->bwd.pos_of_node, g->fwd, err);
         if (rc != EMO_OK) { delete g; return rc; }
         std::vector<int32_t> hop((size_t)std::max(n, 1), 0);
         int32_t depth = 0;
@@ -400,7 +463,7 @@ int emo_graph_info(const emo_graph *g, emo_info *info)
 }
 
 int emo_graph_program(const emo_graph *g, int dir, int32_t *lanes, int32_t *steps, int32_t *slots,
-                      int32_t *Lp, const uint32_t **entries, const uint32_t **lat)
+                      int32_t *Lp, const uint32_t **entries, const uint32_t **rows, const uint32_t **lat)
 {
     if (!g || (dir != 0 && dir != 1)) return EMO_E_INVALID_ARG;
     const Program &p = dir ? g->bwd : g->fwd;
@@ -409,79 +472,121 @@ int emo_graph_program(const emo_graph *g, int dir, int32_t *lanes, int32_t *step
     if (slots) *slots = p.slots;
     if (Lp) *Lp = p.Lp;
     if (entries) *entries = p.entries.data();
+    if (rows) *rows = p.rows.data();
     if (lat) *lat = p.lat.data();
     return EMO_OK;
 }
+
+}  // extern "C"
+
+namespace {
+
+// Spill area behind the head of the workspace: large enough for either layout.
+size_t spill_need(const emo_graph *g, int64_t B)
+{
+    size_t plain = (size_t)g->h.n * round_up((size_t)B, 16) * sizeof(int64_t);
+    size_t tiled = 0;
+    if (!g->host_only && B > 0) {
+        LaunchShape s;
+        StagedParams sp;
+        if (staged_shape(g, g->bwd, g->dbwd.rec_bytes, true, B, s, sp)) {
+            const size_t tiles = ((size_t)B + sp.ptile - 1) / sp.ptile;
+            tiled = tiles * (size_t)g->bwd.steps * g->bwd.lanes * sp.ptile * sizeof(int64_t);
+        }
+    }
+    return round_up(std::max(plain, tiled), 256);
+}
+
+}  // namespace
+
+extern "C" {
 
 int emo_workspace_bytes(const emo_graph *g, int64_t B, int need_slack, size_t *out)
 {
     if (!g || !out || B < 0) return EMO_E_INVALID_ARG;
     size_t bytes = kSmallWs + lvl_area(g);
-    if (need_slack) bytes += (size_t)g->h.n * round_up((size_t)B, 16) * sizeof(int64_t);
+    if (need_slack) bytes += spill_need(g, B);
     if (need_slack == 2) bytes += 4 * round_up((size_t)B * 8, 256) + 256;
     *out = bytes;
     return EMO_OK;
 }
 
 int emo_eval_policies(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t ldb, int64_t *makespan,
-                      double *energy, void *ws, size_t ws_bytes, int32_t *status, uint32_t flags,
-                      void *stream)
+                      double *energy, int64_t *T0, double *E0, void *ws, size_t ws_bytes, int32_t *status,
+                      uint32_t flags, void *stream)
 {
     if (!g || B < 0) return EMO_E_INVALID_ARG;
     if (g->host_only) return EMO_E_CUDA;
-    if (B == 0) return EMO_OK;
-    if (!lvl || !makespan || !energy || ldb < B) return EMO_E_INVALID_ARG;
+    if (B == 0 && !T0 && !E0) return EMO_OK;
+    if (B > 0 && (!lvl || !makespan || !energy || ldb < B)) return EMO_E_INVALID_ARG;
     (void)ws;
     (void)ws_bytes;
     cudaStream_t st = (cudaStream_t)stream;
-    if (flags & EMO_F_VALIDATE) {
+    if ((flags & EMO_F_VALIDATE) && B > 0) {
         int rc = launch_validate(g, B, lvl, ldb, status, st);
         if (rc) return rc;
     }
-    return launch_pass(g, false, B, lvl, ldb, nullptr, 0, nullptr, nullptr, 0, makespan, energy, nullptr,
-                       nullptr, status, st, flags);
+    if (B == 0) { lvl = nullptr; ldb = 0; }
+    PassPlan pl;
+    int rc = make_plan(g, B, T0 || E0, false, lvl, ldb, 0, 0, flags, pl);
+    if (rc) return rc;
+    return launch_pass(g, pl, false, B, lvl, ldb, nullptr, 0, nullptr, nullptr, nullptr, 0, makespan, energy, nullptr,
+                       nullptr, T0, E0, status, st);
 }
 
 int emo_slack_batch(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t ldb, int64_t *ES,
                     int64_t *LS, int64_t *slack, int64_t ldo, int64_t *makespan, double *energy,
-                    int64_t *slack_sum, int32_t *n_critical, void *ws, size_t ws_bytes, int32_t *status,
-                    uint32_t flags, void *stream)
+                    int64_t *slack_sum, int32_t *n_critical, int64_t *T0, double *E0, void *ws, size_t ws_bytes,
+                    int32_t *status, uint32_t flags, void *stream)
 {
     if (!g || B < 0) return EMO_E_INVALID_ARG;
     if (g->host_only) return EMO_E_CUDA;
-    if (B == 0) return EMO_OK;
+    if (B == 0) return emo_eval_policies(g, 0, nullptr, 0, nullptr, nullptr, T0, E0, ws, ws_bytes, status, flags, stream);
     if (!lvl || !makespan || !energy || ldb < B) return EMO_E_INVALID_ARG;
     if ((ES || LS || slack) && ldo < B) return EMO_E_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
-    int64_t *es = ES;
-    int64_t ldes = ldo;
-    if (!es) {
-        size_t need = 0;
-        emo_workspace_bytes(g, B, 1, &need);
-        if (!ws || ws_bytes < need) return EMO_E_OOM;
-        es = (int64_t *)((char *)ws + kSmallWs + lvl_area(g));
-        ldes = (int64_t)round_up((size_t)B, 16);
-    }
     if (flags & EMO_F_VALIDATE) {
         int rc = launch_validate(g, B, lvl, ldb, status, st);
         if (rc) return rc;
     }
-    int rc = launch_pass(g, false, B, lvl, ldb, es, ldes, nullptr, nullptr, 0, makespan, energy, nullptr,
-                         nullptr, status, st, flags);
+    const int64_t ld_ws = (int64_t)round_up((size_t)B, 16);
+    PassPlan pl;
+    int rc = make_plan(g, B, T0 || E0, true, lvl, ldb, ES ? ldo : ld_ws, ldo, flags, pl);
     if (rc) return rc;
-    return launch_pass(g, true, B, lvl, ldb, es, ldes, LS, slack, ldo, makespan, energy, slack_sum,
-                       n_critical, status, st, flags);
+    int64_t *area = (int64_t *)((char *)ws + kSmallWs + lvl_area(g));
+    int64_t *spill = nullptr, *es = ES;
+    int64_t ldes = ldo;
+    if (pl.staged) {
+        if (!ws || ws_bytes < kSmallWs + lvl_area(g) + pl.spill_bytes) return EMO_E_OOM;
+        spill = area;
+    } else if (!es) {
+        if (!ws || ws_bytes < kSmallWs + lvl_area(g) + (size_t)g->h.n * ld_ws * sizeof(int64_t)) return EMO_E_OOM;
+        es = area;
+        ldes = ld_ws;
+    }
+    rc = launch_pass(g, pl, false, B, lvl, ldb, es, ldes, spill, nullptr, nullptr, 0, makespan, energy, nullptr,
+                     nullptr, T0, E0, status, st);
+    if (rc) return rc;
+    return launch_pass(g, pl, true, B, lvl, ldb, es, ldes, spill, LS, slack, ldo, makespan, energy, slack_sum,
+                       n_critical, nullptr, nullptr, status, st);
 }
 
 int emo_slack(const emo_graph *g, const uint8_t *lvl_one, int64_t *ES, int64_t *LS, int64_t *slack,
               int64_t *makespan, double *energy, void *ws, size_t ws_bytes, int32_t *status, void *stream)
 {
-    if (!g || !makespan) return EMO_E_INVALID_ARG;
+    if (!g || !makespan || !lvl_one) return EMO_E_INVALID_ARG;
+    if (g->host_only) return EMO_E_CUDA;
     size_t need = 0;
     emo_workspace_bytes(g, 1, 1, &need);
     if (!ws || ws_bytes < need) return EMO_E_OOM;
+    cudaStream_t st = (cudaStream_t)stream;
+    // re-pitch the level vector to [rows][16] so that the staged kernels can be used; the
+    // per-node outputs are written at pitch 1 directly
+    uint8_t *lv = (uint8_t *)ws + kSmallWs;
+    const size_t rows = (size_t)std::max(g->h.rows, 1);
+    EMO_CUDA(cudaMemcpy2DAsync(lv, 16, lvl_one, 1, 1, rows, cudaMemcpyDeviceToDevice, st));
     double *e = energy ? energy : (double *)((char *)ws + 1024);
-    return emo_slack_batch(g, 1, lvl_one, 1, ES, LS, slack, 1, makespan, e, nullptr, nullptr, ws, ws_bytes,
+    return emo_slack_batch(g, 1, lv, 16, ES, LS, slack, 1, makespan, e, nullptr, nullptr, nullptr, nullptr, ws, ws_bytes,
                            status, 0, stream);
 }
 
@@ -489,14 +594,7 @@ int emo_baseline(const emo_graph *g, int64_t *T0, double *E0, void *ws, size_t w
                  void *stream)
 {
     if (!g || !T0 || !E0) return EMO_E_INVALID_ARG;
-    if (g->host_only) return EMO_E_CUDA;
-    size_t need = 0;
-    emo_workspace_bytes(g, 1, 0, &need);
-    if (!ws || ws_bytes < need) return EMO_E_OOM;
-    cudaStream_t st = (cudaStream_t)stream;
-    uint8_t *lv = (uint8_t *)ws + kSmallWs;
-    EMO_CUDA(cudaMemsetAsync(lv, g->h.L - 1, (size_t)std::max(g->h.rows, 1) * 16, st));
-    return launch_pass(g, false, 1, lv, 16, nullptr, 0, nullptr, nullptr, 0, T0, E0, nullptr, nullptr, status, st);
+    return emo_eval_policies(g, 0, nullptr, 0, nullptr, nullptr, T0, E0, ws, ws_bytes, status, 0, stream);
 }
 
 int64_t emo_target_from_delta(int64_t T0, int64_t delta_ppm)
@@ -558,10 +656,9 @@ int emo_slack_batch_host(const emo_graph *g, int64_t B, const uint8_t *lvl_host,
     int32_t *d_status = (int32_t *)(d_sel + 8);
     EMO_CUDA(cudaMemsetAsync(d_sel, 0, 128, st));
     EMO_CUDA(cudaMemcpyAsync(dev_lvl, lvl_host, (size_t)g->h.rows * (size_t)ldb, cudaMemcpyHostToDevice, st));
-    int rc = emo_slack_batch(g, B, dev_lvl, ldb, nullptr, nullptr, slack_dev, ldo, d_T, d_E, d_ss, d_nc, ws,
-                             need, d_status, flags, st);
-    if (rc) return rc;
-    rc = emo_baseline(g, d_sel + 3, (double *)(d_sel + 4), ws, need, d_status, st);
+    int rc = emo_slack_batch(g, B, dev_lvl, ldb, nullptr, nullptr, slack_dev, ldo, d_T, d_E,
+                             slack_sum_host ? d_ss : nullptr, n_critical_host ? d_nc : nullptr, d_sel + 3,
+                             (double *)(d_sel + 4), ws, need, d_status, flags, st);
     if (rc) return rc;
     rc = emo_select(B, d_T, d_E, 0, d_sel + 3, delta_ppm, d_sel, d_sel + 1, (double *)(d_sel + 2), ws, need, st);
     if (rc) return rc;

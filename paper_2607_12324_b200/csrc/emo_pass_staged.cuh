@@ -1,9 +1,22 @@
-// Staged pass kernel (sm_100a): the same step interpreter as emo_pass_plain, but everything a step
-// reads - program entries, the schedule-ordered duration and energy tables, the level rows of the
-// block's policy tile and (backward) the earliest-start rows - is brought into shared memory by one
-// producer warp with bulk asynchronous copies (TMA, cp.async.bulk) through a ring of stages guarded
-// by full/empty mbarriers.  Each table chunk and each level row is fetched once per block and used
-// by every policy of the block.  Included only by emo_lib.cu.
+// Staged pass kernel (sm_100a): the step interpreter with everything a step reads brought into
+// shared memory by one producer warp with bulk asynchronous copies (TMA, cp.async.bulk) through a
+// ring of stages guarded by full/empty mbarriers: the program records (entry + duration row +
+// energy row) of a run of steps in one bulk copy, (backward) the earliest-start rows of those steps
+// in a second bulk copy, and the level rows of the block's policy tile, which lie scattered in the
+// caller's matrix, as 16-byte cp.async pieces issued by all lanes of the producer warp (a bulk copy
+// per 128-byte row costs far more than it moves).  Each record and each level row is fetched once
+// per block and used by every policy of the block.
+//
+// A consumer thread carries TWO adjacent policies, so a warp covers 64 policies of one schedule
+// lane: the entry decode and the address arithmetic are paid once per pair, the level pair is one
+// 16-bit load, an exchange slot holds both values and moves with one 128-bit access, and the
+// per-node outputs leave as 128-bit stores.
+//
+// The warps of a group do not run in lockstep.  Each walks its own column of the step program and
+// waits only for the values it reads: every exchange slot has an mbarrier whose phase completes
+// when the slot's next value has been written, and the entry names the phase parity to wait for.
+// The group meets at a named barrier every kSyncSteps steps, which bounds the drift between its
+// warps; the host compiler reuses a slot only across such a barrier.  Included only by emo_lib.cu.
 #pragma once
 #include <cuda_runtime.h>
 
@@ -12,15 +25,19 @@
 #include "emo_compile.h"
 #include "emo_kernels.cuh"
 
-constexpr int kStages = 3;
+constexpr int kMaxStages = 4;
+constexpr unsigned kSlotStride = 528;   // 8-byte mbarrier, 8 bytes unused, 32 lanes x 16 bytes
 constexpr long long kWaitCycles = 4000000000LL;   // about two seconds: a wait that long has failed
 
 struct StagedParams {
     PassParams p;
-    int sc;                    // steps per stage
-    int ptile;                 // policies per block = 32 * groups
+    int sc;                    // steps per stage (a multiple of kSyncSteps)
+    int stages;                // ring depth
+    int ptile;                 // policies per block = 64 * groups
+    int vec_es, vec_out;       // 128-bit global accesses allowed for ES / for LS and slack
+    int want_sums;             // backward: accumulate slack sums and critical counts
     unsigned stage_bytes;      // bytes of one stage
-    unsigned off_lat, off_en, off_lvl, off_es;   // offsets inside a stage
+    unsigned off_lvl, off_es;  // offsets inside a stage (records start at 0)
     unsigned off_part, off_bar, off_stage0;      // offsets inside dynamic shared memory
 };
 
@@ -69,53 +86,166 @@ __device__ __forceinline__ void emo_bulk_g2s(unsigned dst, const void *src, unsi
                  : "memory");
 }
 
+// 16-byte asynchronous copy global -> shared, and the arrival that reports a thread's copies done
+__device__ __forceinline__ void emo_cp_async16(unsigned dst, const void *src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void emo_cp_async_arrive(unsigned bar)
+{
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// shared-memory accesses by 32-bit address
+__device__ __forceinline__ uint4 emo_lds128(unsigned a)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ unsigned emo_lds_u16(unsigned a)
+{
+    unsigned short v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ unsigned emo_lds_u32(unsigned a)
+{
+    unsigned v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ double emo_lds_f64(unsigned a)
+{
+    double v;
+    asm volatile("ld.shared.f64 %0, [%1];" : "=d"(v) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ void emo_lds_pair(unsigned a, long long &x0, long long &x1)
+{
+    asm volatile("ld.shared.v2.s64 {%0, %1}, [%2];" : "=l"(x0), "=l"(x1) : "r"(a));
+}
+__device__ __forceinline__ void emo_sts_pair(unsigned a, long long x0, long long x1)
+{
+    asm volatile("st.shared.v2.s64 [%0], {%1, %2};" ::"r"(a), "l"(x0), "l"(x1) : "memory");
+}
+__device__ __forceinline__ void emo_stg_pair(long long *p, long long x0, long long x1)
+{
+    asm volatile("st.global.v2.s64 [%0], {%1, %2};" ::"l"(p), "l"(x0), "l"(x1) : "memory");
+}
+__device__ __forceinline__ long long emo_max64(long long a, long long b) { return a > b ? a : b; }
+// h + d with d an unsigned 32-bit duration: one wide multiply-add
+__device__ __forceinline__ long long emo_add_dur(long long h, unsigned d)
+{
+    long long r;
+    asm("mad.wide.u32 %0, %1, 1, %2;" : "=l"(r) : "r"(d), "l"(h));
+    return r;
+}
+
+// What a step needs from its stage, independent of the recurrence.
+struct EmoFetched {
+    uint4 e;
+    unsigned node;
+    unsigned d0, d1;
+    double g0, g1;
+    long long es0, es1;
+};
 template <bool BWD>
-__global__ void __launch_bounds__(1024) emo_pass_staged(StagedParams sp)
+__device__ __forceinline__ void emo_fetch(EmoFetched &x, unsigned rec_a, unsigned lvl_a, unsigned es_a, unsigned en_off,
+                                          bool want_node)
+{
+    x.e = emo_lds128(rec_a);
+    if (want_node) x.node = emo_lds_u32(rec_a + 16u);
+    const unsigned lv2 = emo_lds_u16(lvl_a);
+    const unsigned m = (x.e.y >> emo::kMaskShift) & 255u;
+    const unsigned l0 = lv2 & m, l1 = (lv2 >> 8) & m;
+    x.d0 = emo_lds_u32(rec_a + 32u + l0 * 4u);
+    x.d1 = emo_lds_u32(rec_a + 32u + l1 * 4u);
+    if (!BWD) {
+        x.g0 = emo_lds_f64(rec_a + en_off + l0 * 8u);
+        x.g1 = emo_lds_f64(rec_a + en_off + l1 * 8u);
+    } else {
+        emo_lds_pair(es_a, x.es0, x.es1);
+    }
+}
+// base + row * pitch (bytes) as one wide multiply-add
+__device__ __forceinline__ long long *emo_row_ptr(long long *base, unsigned row, unsigned pitch_bytes)
+{
+    unsigned long long r;
+    asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(r) : "r"(row), "r"(pitch_bytes), "l"(reinterpret_cast<unsigned long long>(base)));
+    return reinterpret_cast<long long *>(r);
+}
+// Wait until the slot's value with the given phase parity has been written.  Bounded; also gives
+// up as soon as another warp of the group has raised the abort flag.
+__device__ __forceinline__ bool emo_slot_wait(unsigned bar, unsigned parity, volatile int *abort_flag)
+{
+    if (emo_mbar_try(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!emo_mbar_try(bar, parity)) {
+        if (*abort_flag || clock64() - t0 > kWaitCycles) return false;
+    }
+    return true;
+}
+
+template <bool BWD, int MAXT>
+__global__ void __launch_bounds__(MAXT, 1) emo_pass_pair(StagedParams sp)
 {
     extern __shared__ __align__(128) unsigned char emo_smem[];
     const PassParams &p = sp.p;
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
-    const int n_cons = p.groups * p.lanes;              // consumer warps; warp n_cons is the producer
+    const int lanes = p.lanes, groups = p.groups, steps = p.steps, nstages = sp.stages, sc = sp.sc;
+    const int n_cons = groups * lanes;                  // consumer warps; warp n_cons is the producer
     const bool producer = warp == n_cons;
-    const int group = producer ? 0 : warp / p.lanes;
-    const int chain = warp - group * p.lanes;
-    const int64_t b0 = (int64_t)blockIdx.x * sp.ptile;
-    const int64_t b = b0 + group * 32 + lane;
-    const bool active = !producer && b < p.B;
+    const int group = producer ? 0 : warp / lanes;
+    const int chain = warp - group * lanes;
+    const int ptile = sp.ptile;
+    const int64_t b0 = (int64_t)blockIdx.x * ptile;
+    const int col = group * 64 + 2 * lane;
+    const int64_t b = b0 + col;
+    const bool act0 = !producer && b < p.B, act1 = !producer && b + 1 < p.B;
+    // column of the virtual all-max policy inside this block's tile (fwd only), or -1
+    const int base_col = (!BWD && p.want_base && p.B >= b0 && p.B < b0 + ptile) ? (int)(p.B - b0) : -1;
     unsigned char *part_base = emo_smem + sp.off_part;
-    const unsigned bar0 = emo_smem_addr(emo_smem + sp.off_bar);        // full[k] at bar0 + 8k, empty[k] after
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(emo_smem + sp.off_bar + 16 * kStages);
-    unsigned char *stage0 = emo_smem + sp.off_stage0;
+    const unsigned smem0 = emo_smem_addr(emo_smem);
+    const unsigned bar0 = smem0 + sp.off_bar;           // full[k] at bar0 + 8k, empty[k] after them
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(emo_smem + sp.off_bar + 16 * kMaxStages);
+    const unsigned stage0 = smem0 + sp.off_stage0;
+    const unsigned stage_bytes = sp.stage_bytes;
 
+    for (int i = threadIdx.x; i < groups * p.slots; i += blockDim.x) emo_mbar_init(smem0 + (unsigned)i * kSlotStride, 1);
     if (threadIdx.x == 0) {
-        for (int k = 0; k < kStages; ++k) {
-            emo_mbar_init(bar0 + 8 * k, 1);
-            emo_mbar_init(bar0 + 8 * (kStages + k), n_cons);
+        for (int k = 0; k < nstages; ++k) {
+            emo_mbar_init(bar0 + 8 * k, 33);      // one expect-tx arrival + the 32 lanes' cp.async arrivals
+            emo_mbar_init(bar0 + 8 * (kMaxStages + k), n_cons);
         }
-        for (int k = 0; k <= p.groups; ++k) abort_flag[k] = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        for (int k = 0; k <= groups; ++k) abort_flag[k] = 0;
     }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncthreads();
 
-    const int n_chunks = (p.steps + sp.sc - 1) / sp.sc;
-    long long h = 0;
-    double eacc = 0.0;
-    long long tmax = 0, ssum = 0;
-    int ncrit = 0;
+    const int n_chunks = (steps + sc - 1) / sc;
+    long long h0 = 0, h1 = 0;
+    double ea0 = 0.0, ea1 = 0.0;
+    long long acc0 = 0, acc1 = 0;      // forward: running makespan; backward: slack sums
+    int nc0 = 0, nc1 = 0;
 
     if (producer) {
         // ---------------------------------------------------------------------------- producer
-        const unsigned lvl_bytes = (unsigned)min((int64_t)sp.ptile, p.ldb - b0);
-        const unsigned es_bytes = BWD ? (unsigned)min((int64_t)sp.ptile, p.ldes - b0) * 8u : 0u;
+        const int64_t lvl_left = p.ldb - b0;
+        const unsigned lvl_bytes = lvl_left > 0 ? (unsigned)min((int64_t)ptile, lvl_left) : 0u;
+        const int pieces = (int)(lvl_bytes >> 4);
+        const unsigned rec_bytes = (unsigned)p.rec_bytes;
+        // this block's tile of the spill: [spill_rows][ptile] (the backward kernel's own tile width)
+        const long long *spill_tile = BWD ? reinterpret_cast<const long long *>(p.spill) + (size_t)blockIdx.x * p.spill_rows * ptile : nullptr;
         int issued = 0;
         bool gave_up = false;
         for (int c = 0; c < n_chunks; ++c) {
-            const int s = c % kStages;
-            if (c >= kStages) {
-                if (!emo_mbar_wait(bar0 + 8 * (kStages + s), ((c / kStages) - 1) & 1)) {
+            const int s = c % nstages;
+            if (c >= nstages) {
+                if (!emo_mbar_wait(bar0 + 8 * (kMaxStages + s), ((c / nstages) - 1) & 1)) {
                     if (lane == 0) {
-                        abort_flag[p.groups] = 1;
+                        abort_flag[groups] = 1;
                         if (p.status) atomicMin(p.status, -8);
                     }
                     gave_up = true;
@@ -123,137 +253,239 @@ __global__ void __launch_bounds__(1024) emo_pass_staged(StagedParams sp)
                 }
             }
             issued = c + 1;
-            const int step0 = c * sp.sc;
-            const int ne = min(sp.sc, p.steps - step0) * p.lanes;
-            const size_t q0 = (size_t)step0 * p.lanes;
-            unsigned bytes = 0;
-            for (int i = lane; i < ne; i += 32) {
-                const uint4 e = __ldg(p.prog + q0 + i);
-                if (e.z & emo::kValid) {
-                    if (e.x != emo::kNone) bytes += lvl_bytes;
-                    if (BWD && e.y != emo::kNone) bytes += es_bytes;
-                }
-            }
-            for (int off = 16; off > 0; off >>= 1) bytes += __shfl_xor_sync(0xFFFFFFFFu, bytes, off);
-            unsigned char *st = stage0 + (size_t)s * sp.stage_bytes;
-            const unsigned sta = emo_smem_addr(st);
+            const int step0 = c * sc;
+            const int ne = min(sc, steps - step0) * lanes;
+            const size_t q0 = (size_t)step0 * lanes;
+            const unsigned sta = stage0 + (unsigned)s * stage_bytes;
             const unsigned full = bar0 + 8 * s;
             if (lane == 0) {
-                const unsigned fixed = (unsigned)ne * 16u + (unsigned)ne * p.Lp * 4u + (BWD ? 0u : (unsigned)ne * p.Lp * 8u);
-                emo_mbar_expect_tx(full, bytes + fixed);
-                emo_bulk_g2s(sta, p.prog + q0, (unsigned)ne * 16u, full);
-                emo_bulk_g2s(sta + sp.off_lat, p.lat + q0 * p.Lp, (unsigned)ne * p.Lp * 4u, full);
-                if (!BWD) emo_bulk_g2s(sta + sp.off_en, p.en + q0 * p.Lp, (unsigned)ne * p.Lp * 8u, full);
+                const unsigned rb = (unsigned)ne * rec_bytes, eb = BWD ? (unsigned)ne * ptile * 8u : 0u;
+                emo_mbar_expect_tx(full, rb + eb);
+                emo_bulk_g2s(sta, p.rec + q0 * rec_bytes, rb, full);
+                if (BWD) emo_bulk_g2s(sta + sp.off_es, spill_tile + q0 * ptile, eb, full);
             }
-            __syncwarp();
-            for (int i = lane; i < ne; i += 32) {
-                const uint4 e = __ldg(p.prog + q0 + i);
-                if (e.z & emo::kValid) {
-                    if (e.x != emo::kNone)
-                        emo_bulk_g2s(sta + sp.off_lvl + (unsigned)i * sp.ptile, p.lvl + (size_t)e.x * p.ldb + b0, lvl_bytes, full);
-                    if (BWD && e.y != emo::kNone)
-                        emo_bulk_g2s(sta + sp.off_es + (unsigned)i * sp.ptile * 8u, p.ES + (size_t)e.y * p.ldes + b0, es_bytes, full);
+            // level rows: entry i, 16-byte piece pc
+            if (pieces) {
+                int i = lane / pieces, pc = lane - i * pieces;
+                const int di = 32 / pieces, dpc = 32 - di * pieces;
+                while (i < ne) {
+                    const unsigned row = __ldg(p.rows + q0 + i);
+                    if (row != emo::kNone)
+                        emo_cp_async16(sta + sp.off_lvl + (unsigned)i * ptile + (unsigned)pc * 16u,
+                                       p.lvl + (size_t)row * p.ldb + b0 + pc * 16);
+                    i += di;
+                    pc += dpc;
+                    if (pc >= pieces) { pc -= pieces; ++i; }
                 }
             }
+            emo_cp_async_arrive(full);
         }
         if (gave_up) {
             // do not leave the block while copies into its shared memory may still be in flight
-            for (int c = max(0, issued - kStages); c < issued; ++c) (void)emo_mbar_wait(bar0 + 8 * (c % kStages), (c / kStages) & 1);
+            for (int c = max(0, issued - nstages); c < issued; ++c) (void)emo_mbar_wait(bar0 + 8 * (c % nstages), (c / nstages) & 1);
         }
     } else {
         // --------------------------------------------------------------------------- consumers
-        long long *slots = reinterpret_cast<long long *>(emo_smem) + (size_t)group * p.slots * 32 + lane;
-        const long long T = (BWD && active) ? p.makespan[b] : 0;
-        const int col = group * 32 + lane;
-        bool failed = false;
-        for (int c = 0; c < n_chunks && !failed; ++c) {
-            const int s = c % kStages;
-            const bool ok = emo_mbar_wait(bar0 + 8 * s, (c / kStages) & 1);
+        const unsigned slotbar_base = smem0 + (unsigned)group * p.slots * kSlotStride;
+        const unsigned lane16 = 16u + (unsigned)lane * 16u;
+        const long long T0 = (BWD && act0) ? p.makespan[b] : 0, T1 = (BWD && act1) ? p.makespan[b + 1] : 0;
+        const unsigned d_rec = (unsigned)lanes * p.rec_bytes, d_lvl = (unsigned)lanes * ptile;
+        const unsigned en_off = 32u + (unsigned)p.Lp * 4u;
+        const unsigned ldes8 = (unsigned)p.ldes * 8u, ldo8 = (unsigned)p.ldo * 8u;     // pitches below 2^28 elements
+        long long *const es_lane = (!BWD && p.ES) ? reinterpret_cast<long long *>(p.ES) + b : nullptr;
+        // forward: this thread's column pair inside the spill tile it belongs to
+        long long *const spill_lane = (!BWD && p.spill)
+            ? reinterpret_cast<long long *>(p.spill) + (size_t)(b / p.spill_ptile) * p.spill_rows * p.spill_ptile + (b % p.spill_ptile)
+            : nullptr;
+        const unsigned spill8 = (unsigned)p.spill_ptile * 8u;
+        long long *const ls_lane = p.LS ? reinterpret_cast<long long *>(p.LS) + b : nullptr;
+        long long *const sl_lane = p.slack ? reinterpret_cast<long long *>(p.slack) + b : nullptr;
+        const bool store_es = es_lane != nullptr && act0, store_spill = spill_lane != nullptr && act0;
+        const bool vec_es = sp.vec_es && act1, vec_out = sp.vec_out && act1;
+        const bool want_sums = sp.want_sums != 0;
+        const int gthreads = lanes * 32;
+        volatile int *my_abort = abort_flag + group;
+        bool dead = false;
+
+        // one node for both policies of this thread
+        auto process = [&](const EmoFetched &f) {
+            const uint4 e = f.e;
+            if (!(e.y & emo::kValid) || dead) return;
+            if (!BWD) {
+                ea0 += f.g0;
+                ea1 += f.g1;
+            }
+            if (!(e.y & emo::kRegPred)) { h0 = 0; h1 = 0; }
+            const unsigned np = (e.y >> emo::kNPredShift) & 7u;
+            if (np) {
+                unsigned ops = e.z, par = e.y >> emo::kOperandParityShift;
+                for (unsigned k = 0; k < np; ++k) {
+                    if (k == 4) ops = e.w;
+                    const unsigned bar = slotbar_base + (ops & 255u) * kSlotStride;
+                    if (!emo_slot_wait(bar, par & 1u, my_abort)) {
+                        *my_abort = 1;
+                        dead = true;
+                        return;
+                    }
+                    long long x0, x1;
+                    emo_lds_pair(bar + lane16, x0, x1);
+                    ops >>= 8;
+                    par >>= 1;
+                    h0 = emo_max64(h0, x0);
+                    h1 = emo_max64(h1, x1);
+                }
+            }
+            // here h is the node's start (forward: ES_v; backward: the longest tail behind v)
+            if (!BWD && e.x != emo::kNone) {
+                if (store_spill) {
+                    long long *dst = emo_row_ptr(spill_lane, e.x, spill8);     // 16-byte aligned by construction
+                    if (act1) {
+                        emo_stg_pair(dst, h0, h1);
+                    } else {
+                        dst[0] = h0;
+                    }
+                }
+                if (store_es) {
+                    long long *dst = emo_row_ptr(es_lane, f.node, ldes8);
+                    if (vec_es) {
+                        emo_stg_pair(dst, h0, h1);
+                    } else {
+                        dst[0] = h0;
+                        if (act1) dst[1] = h1;
+                    }
+                }
+            }
+            h0 = emo_add_dur(h0, f.d0);
+            h1 = emo_add_dur(h1, f.d1);
+            if (e.y & emo::kWriteSlot) {
+                const unsigned bar = slotbar_base + ((e.y >> emo::kOutShift) & 255u) * kSlotStride;
+                emo_sts_pair(bar + lane16, h0, h1);
+                __syncwarp();
+                if (lane == 0) emo_mbar_arrive(bar);
+            }
+            if (!BWD) {
+                if (e.y & emo::kTerminal) {
+                    acc0 = emo_max64(acc0, h0);
+                    acc1 = emo_max64(acc1, h1);
+                }
+            } else if (e.x != emo::kNone && act0) {
+                const long long ls0 = T0 - h0, ls1 = T1 - h1;
+                const long long s0 = ls0 - f.es0, s1 = ls1 - f.es1;
+                if (ls_lane) {
+                    long long *dst = emo_row_ptr(ls_lane, e.x, ldo8);
+                    if (vec_out) {
+                        emo_stg_pair(dst, ls0, ls1);
+                    } else {
+                        dst[0] = ls0;
+                        if (act1) dst[1] = ls1;
+                    }
+                }
+                if (sl_lane) {
+                    long long *dst = emo_row_ptr(sl_lane, e.x, ldo8);
+                    if (vec_out) {
+                        emo_stg_pair(dst, s0, s1);
+                    } else {
+                        dst[0] = s0;
+                        if (act1) dst[1] = s1;
+                    }
+                }
+                if (want_sums) {
+                    acc0 += s0;
+                    acc1 += s1;
+                    nc0 += (s0 == 0);
+                    nc1 += (s1 == 0);
+                }
+            }
+        };
+
+        for (int c = 0; c < n_chunks; ++c) {
+            const int s = c % nstages;
+            const bool ok = emo_mbar_wait(bar0 + 8 * s, (c / nstages) & 1);
             // the warps of a group must take the same decision: one flag, read after a barrier
-            if (!ok || (chain == 0 && abort_flag[p.groups])) abort_flag[group] = 1;
-            if (p.lanes > 1) emo_group_barrier(group + 1, p.lanes * 32);
-            if (abort_flag[group]) {
+            if (!ok || dead || (chain == 0 && abort_flag[groups])) *my_abort = 1;
+            const unsigned sta = stage0 + (unsigned)s * stage_bytes;
+            const int ns = min(sc, steps - c * sc);
+            if (base_col >= 0 && chain == 0 && (base_col >> 6) == group) {
+                // the virtual all-max column: overwrite its byte in every level row of this stage
+                const unsigned char top = (unsigned char)(p.L - 1);
+                for (int i = lane; i < ns * lanes; i += 32)
+                    emo_smem[sp.off_stage0 + (size_t)s * stage_bytes + sp.off_lvl + (size_t)i * ptile + (size_t)base_col] = top;
+                __syncwarp();
+            }
+            if (lanes > 1) emo_group_barrier(group + 1, gthreads);
+            if (*my_abort) {
                 if (lane == 0 && p.status) atomicMin(p.status, -8);
-                failed = true;
                 break;
             }
-            const unsigned char *st = stage0 + (size_t)s * sp.stage_bytes;
-            const uint4 *s_ent = reinterpret_cast<const uint4 *>(st);
-            const uint32_t *s_lat = reinterpret_cast<const uint32_t *>(st + sp.off_lat);
-            const double *s_en = reinterpret_cast<const double *>(st + sp.off_en);
-            const unsigned char *s_lvl = st + sp.off_lvl;
-            const long long *s_es = reinterpret_cast<const long long *>(st + sp.off_es);
-            const int ns = min(sp.sc, p.steps - c * sp.sc);
-            for (int j = 0; j < ns; ++j) {
-                const int i = j * p.lanes + chain;
-                const uint4 e = s_ent[i];
-                if (e.z & emo::kValid) {
-                    unsigned lv = 0;
-                    if (e.x != emo::kNone) lv = s_lvl[i * sp.ptile + col];
-                    lv &= (unsigned)p.Lmask;
-                    const long long dur = (long long)s_lat[i * p.Lp + lv];
-                    long long start = (e.z & emo::kRegPred) ? h : 0;
-                    const int np = (e.z >> emo::kNPredShift) & 7;
-                    unsigned long long ops = (unsigned long long)e.w | ((unsigned long long)(e.z >> 16) << 32);
-                    for (int k = 0; k < np; ++k) {
-                        long long x = slots[(unsigned)(ops & 255u) * 32];
-                        ops >>= 8;
-                        start = x > start ? x : start;
-                    }
-                    h = start + dur;
-                    if (!BWD) {
-                        eacc += s_en[i * p.Lp + lv];
-                        if (e.z & emo::kTerminal) tmax = h > tmax ? h : tmax;
-                        if (p.ES && e.y != emo::kNone && active) p.ES[(size_t)e.y * p.ldes + b] = start;
-                    } else if (e.y != emo::kNone && active) {
-                        const long long ls = T - h;
-                        const long long es = s_es[i * sp.ptile + col];
-                        const long long sl = ls - es;
-                        if (p.LS) p.LS[(size_t)e.y * p.ldo + b] = ls;
-                        if (p.slack) p.slack[(size_t)e.y * p.ldo + b] = sl;
-                        ssum += sl;
-                        ncrit += (sl == 0);
-                    }
-                    if (e.z & emo::kWriteSlot) slots[((e.z >> emo::kOutShift) & 255u) * 32] = h;
+            unsigned rec_a = sta + (unsigned)chain * p.rec_bytes;
+            unsigned lvl_a = sta + sp.off_lvl + (unsigned)chain * ptile + col;
+            unsigned es_a = sta + sp.off_es + ((unsigned)chain * ptile + col) * 8u;
+            // Everything a step reads from the stage (entry, level pair, durations, energies, ES pair)
+            // is independent of the recurrence, so it is fetched one step ahead.
+            EmoFetched fa, fb;
+            emo_fetch<BWD>(fa, rec_a, lvl_a, es_a, en_off, store_es);
+            for (int j = 0; j < ns; j += 2) {
+                if (j && (j % emo::kSyncSteps) == 0 && lanes > 1) emo_group_barrier(group + 1, gthreads);
+                rec_a += d_rec;
+                lvl_a += d_lvl;
+                es_a += d_lvl * 8u;
+                if (j + 1 < ns) emo_fetch<BWD>(fb, rec_a, lvl_a, es_a, en_off, store_es);
+                process(fa);
+                if (j + 1 < ns) {
+                    rec_a += d_rec;
+                    lvl_a += d_lvl;
+                    es_a += d_lvl * 8u;
+                    if (j + 2 < ns) emo_fetch<BWD>(fa, rec_a, lvl_a, es_a, en_off, store_es);
+                    process(fb);
                 }
-                if (p.lanes > 1) emo_group_barrier(group + 1, p.lanes * 32);
             }
-            if (lane == 0) emo_mbar_arrive(bar0 + 8 * (kStages + s));
+            __syncwarp();
+            if (lane == 0) emo_mbar_arrive(bar0 + 8 * (kMaxStages + s));
         }
     }
 
     // combine the warps of a group in lane order (fixed order: run-to-run identical energy)
+    // per (group, chain, lane): {energy0 | sum0, energy1 | sum1, makespan0 | count0, makespan1 | count1}
     if (!producer) {
-        double *pd = reinterpret_cast<double *>(part_base) + ((size_t)(group * p.lanes + chain) * 32 + lane) * 2;
+        long long *pd = reinterpret_cast<long long *>(part_base) + ((size_t)(group * lanes + chain) * 32 + lane) * 4;
         if (!BWD) {
-            pd[0] = eacc;
-            reinterpret_cast<long long *>(pd)[1] = tmax;
+            pd[0] = __double_as_longlong(ea0);
+            pd[1] = __double_as_longlong(ea1);
+            pd[2] = acc0;
+            pd[3] = acc1;
         } else {
-            reinterpret_cast<long long *>(pd)[0] = ssum;
-            reinterpret_cast<long long *>(pd)[1] = (long long)ncrit;
+            pd[0] = acc0;
+            pd[1] = acc1;
+            pd[2] = nc0;
+            pd[3] = nc1;
         }
     }
     __syncthreads();
-    if (!producer && chain == 0 && active) {
-        const double *g0 = reinterpret_cast<const double *>(part_base) + ((size_t)(group * p.lanes) * 32 + lane) * 2;
+    if (!producer && chain == 0) {
+        const long long *g0 = reinterpret_cast<const long long *>(part_base) + ((size_t)(group * lanes) * 32 + lane) * 4;
         if (!BWD) {
-            double es = 0.0;
-            long long tm = 0;
-            for (int k = 0; k < p.lanes; ++k) {
-                es += g0[(size_t)k * 64];
-                long long x = reinterpret_cast<const long long *>(g0)[(size_t)k * 64 + 1];
-                tm = x > tm ? x : tm;
+            double e0 = 0.0, e1 = 0.0;
+            long long t0 = 0, t1 = 0;
+            for (int k = 0; k < lanes; ++k) {
+                e0 += __longlong_as_double(g0[(size_t)k * 128]);
+                e1 += __longlong_as_double(g0[(size_t)k * 128 + 1]);
+                t0 = emo_max64(t0, g0[(size_t)k * 128 + 2]);
+                t1 = emo_max64(t1, g0[(size_t)k * 128 + 3]);
             }
-            p.makespan[b] = tm;
-            p.energy[b] = es;
-        } else {
-            long long ss = 0, nc = 0;
-            for (int k = 0; k < p.lanes; ++k) {
-                ss += reinterpret_cast<const long long *>(g0)[(size_t)k * 64];
-                nc += reinterpret_cast<const long long *>(g0)[(size_t)k * 64 + 1];
+            if (act0) { p.makespan[b] = t0; p.energy[b] = e0; }
+            if (act1) { p.makespan[b + 1] = t1; p.energy[b + 1] = e1; }
+            if (base_col == col) { if (p.base_T) *p.base_T = t0; if (p.base_E) *p.base_E = e0; }
+            if (base_col == col + 1) { if (p.base_T) *p.base_T = t1; if (p.base_E) *p.base_E = e1; }
+        } else if (sp.want_sums) {
+            long long s0 = 0, s1 = 0, c0 = 0, c1 = 0;
+            for (int k = 0; k < lanes; ++k) {
+                s0 += g0[(size_t)k * 128];
+                s1 += g0[(size_t)k * 128 + 1];
+                c0 += g0[(size_t)k * 128 + 2];
+                c1 += g0[(size_t)k * 128 + 3];
             }
-            if (p.slack_sum) p.slack_sum[b] = ss;
-            if (p.n_critical) p.n_critical[b] = (int32_t)nc;
+            if (act0) { if (p.slack_sum) p.slack_sum[b] = s0; if (p.n_critical) p.n_critical[b] = (int32_t)c0; }
+            if (act1) { if (p.slack_sum) p.slack_sum[b + 1] = s1; if (p.n_critical) p.n_critical[b + 1] = (int32_t)c1; }
         }
     }
 }

@@ -70,8 +70,8 @@ def lib():
         L.emo_graph_free.argtypes = [p]
         L.emo_graph_info.argtypes = [p, ctypes.POINTER(emo_info)]
         L.emo_workspace_bytes.argtypes = [p, i64, ctypes.c_int, ctypes.POINTER(sz)]
-        L.emo_eval_policies.argtypes = [p, i64, p, i64, p, p, p, sz, p, u32, p]
-        L.emo_slack_batch.argtypes = [p, i64, p, i64, p, p, p, i64, p, p, p, p, p, sz, p, u32, p]
+        L.emo_eval_policies.argtypes = [p, i64, p, i64, p, p, p, p, p, sz, p, u32, p]
+        L.emo_slack_batch.argtypes = [p, i64, p, i64, p, p, p, i64, p, p, p, p, p, p, p, sz, p, u32, p]
         L.emo_slack.argtypes = [p, p, p, p, p, p, p, p, sz, p, p]
         L.emo_baseline.argtypes = [p, p, p, p, sz, p, p]
         L.emo_target_from_delta.argtypes = [i64, i64]
@@ -81,7 +81,7 @@ def lib():
         L.emo_slack_batch_host.argtypes = [p, i64, p, i64, p, p, i64, i64, p, p, p, p, p, p, sz, u32, p]
         L.emo_graph_program.argtypes = [p, ctypes.c_int, ctypes.POINTER(i32), ctypes.POINTER(i32),
                                         ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(p),
-                                        ctypes.POINTER(p)]
+                                        ctypes.POINTER(p), ctypes.POINTER(p)]
         L.emo_set_pass_events.argtypes = [p, p, p, p]
         for name in EXPORTS:
             if name not in ("emo_strerror", "emo_target_from_delta"):
@@ -177,17 +177,20 @@ def _nbytes(ws) -> int:
     return 0 if ws is None else int(ws.numel() * ws.element_size())
 
 
-def emo_eval_policies(g: Graph, B, lvl, ldb, makespan, energy, ws=None, status=None, flags=0, stream=None):
+def emo_eval_policies(g: Graph, B, lvl, ldb, makespan, energy, ws=None, status=None, flags=0, stream=None,
+                      T0=None, E0=None):
     _check(lib().emo_eval_policies(g.handle, int(B), _addr(lvl), int(ldb), _addr(makespan), _addr(energy),
-                                   _addr(ws), _nbytes(ws), _addr(status), int(flags), _stream(stream)),
+                                   _addr(T0), _addr(E0), _addr(ws), _nbytes(ws), _addr(status), int(flags),
+                                   _stream(stream)),
            "emo_eval_policies")
 
 
 def emo_slack_batch(g: Graph, B, lvl, ldb, ES, LS, slack, ldo, makespan, energy, slack_sum=None,
-                    n_critical=None, ws=None, status=None, flags=0, stream=None):
+                    n_critical=None, ws=None, status=None, flags=0, stream=None, T0=None, E0=None):
     _check(lib().emo_slack_batch(g.handle, int(B), _addr(lvl), int(ldb), _addr(ES), _addr(LS), _addr(slack),
                                  int(ldo), _addr(makespan), _addr(energy), _addr(slack_sum), _addr(n_critical),
-                                 _addr(ws), _nbytes(ws), _addr(status), int(flags), _stream(stream)),
+                                 _addr(T0), _addr(E0), _addr(ws), _nbytes(ws), _addr(status), int(flags),
+                                 _stream(stream)),
            "emo_slack_batch")
 
 
@@ -238,18 +241,20 @@ def emo_set_pass_events(fwd_start=None, fwd_stop=None, bwd_start=None, bwd_stop=
 
 
 def emo_graph_program(g: Graph, direction: int):
-    """(lanes, steps, slots, Lp, entries[steps][lanes][4] uint32, lat[steps*lanes][Lp] uint32) as
-    numpy copies of the compiled program (host-side inspection)."""
+    """(lanes, steps, slots, Lp, entries[steps][lanes][8], rows[steps][lanes], lat[steps*lanes][Lp]), all
+    uint32 numpy copies of the compiled program (host-side inspection)."""
     lanes, steps, slots, Lp = (ctypes.c_int32() for _ in range(4))
-    pe, pl = ctypes.c_void_p(), ctypes.c_void_p()
+    pe, pr, pl = ctypes.c_void_p(), ctypes.c_void_p(), ctypes.c_void_p()
     _check(lib().emo_graph_program(g.handle, int(direction), ctypes.byref(lanes), ctypes.byref(steps),
-                                   ctypes.byref(slots), ctypes.byref(Lp), ctypes.byref(pe), ctypes.byref(pl)),
-           "emo_graph_program")
+                                   ctypes.byref(slots), ctypes.byref(Lp), ctypes.byref(pe), ctypes.byref(pr),
+                                   ctypes.byref(pl)), "emo_graph_program")
     q = steps.value * lanes.value
     if q == 0:
-        return lanes.value, 0, slots.value, Lp.value, np.zeros((0, max(lanes.value, 1), 4), np.uint32), \
-            np.zeros((0, Lp.value), np.uint32)
-    ent = np.ctypeslib.as_array(ctypes.cast(pe, ctypes.POINTER(ctypes.c_uint32)), shape=(q * 4,)).copy()
-    lat = np.ctypeslib.as_array(ctypes.cast(pl, ctypes.POINTER(ctypes.c_uint32)), shape=(q * Lp.value,)).copy()
-    return lanes.value, steps.value, slots.value, Lp.value, ent.reshape(steps.value, lanes.value, 4), \
-        lat.reshape(q, Lp.value)
+        return lanes.value, 0, slots.value, Lp.value, np.zeros((0, max(lanes.value, 1), 8), np.uint32), \
+            np.zeros((0, max(lanes.value, 1)), np.uint32), np.zeros((0, Lp.value), np.uint32)
+    u32p = ctypes.POINTER(ctypes.c_uint32)
+    ent = np.ctypeslib.as_array(ctypes.cast(pe, u32p), shape=(q * 8,)).copy()
+    rows = np.ctypeslib.as_array(ctypes.cast(pr, u32p), shape=(q,)).copy()
+    lat = np.ctypeslib.as_array(ctypes.cast(pl, u32p), shape=(q * Lp.value,)).copy()
+    return lanes.value, steps.value, slots.value, Lp.value, ent.reshape(steps.value, lanes.value, 8), \
+        rows.reshape(steps.value, lanes.value), lat.reshape(q, Lp.value)

@@ -38,7 +38,8 @@ def golden():
         return json.load(f)
 
 
-def gpu_slack_batch(torch, emo, h, lv_dev, B, n, want=("ES", "LS", "slack"), flags=0, ldo=None):
+def gpu_slack_batch(torch, emo, h, lv_dev, B, n, want=("ES", "LS", "slack"), flags=0, ldo=None, sums=True,
+                    base=False):
     dev = lv_dev.device
     ldo = int(ldo or max(B, 1))
     out = {k: (torch.full((n, ldo), -7, dtype=torch.int64, device=dev) if k in want else None)
@@ -49,11 +50,15 @@ def gpu_slack_batch(torch, emo, h, lv_dev, B, n, want=("ES", "LS", "slack"), fla
     nc = torch.full((max(B, 1),), -1, dtype=torch.int32, device=dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     ws = torch.empty(emo.emo_workspace_bytes(h, B, 1), dtype=torch.uint8, device=dev)
-    emo.emo_slack_batch(h, B, lv_dev, lv_dev.stride(0), out["ES"], out["LS"], out["slack"], ldo, T, E, ss, nc,
-                        ws, status, flags)
+    T0 = torch.full((1,), -1, dtype=torch.int64, device=dev) if base else None
+    E0 = torch.full((1,), -1.0, dtype=torch.float64, device=dev) if base else None
+    emo.emo_slack_batch(h, B, lv_dev, lv_dev.stride(0), out["ES"], out["LS"], out["slack"], ldo, T, E,
+                        ss if sums else None, nc if sums else None, ws, status, flags, T0=T0, E0=E0)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     res = {k: v.cpu().numpy() for k, v in out.items() if v is not None}
+    if base:
+        res["T0"], res["E0"] = int(T0.item()), float(E0.item())
     res.update(makespan=T.cpu().numpy()[:B], energy=E.cpu().numpy()[:B], slack_sum=ss.cpu().numpy()[:B],
                n_critical=nc.cpu().numpy()[:B])
     return res
@@ -154,8 +159,16 @@ def test_config_graphs_all_outputs(torch_cuda, emo, oracle_mod, name, scale, B):
     # slack only (ES kept in the workspace), same result; then the plain-load kernels
     r2 = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, want=("slack",))
     assert np.array_equal(r2["slack"][:, :B], r_or["slack"])
-    r3 = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, flags=emo.EMO_F_NO_STAGING)
-    assert_matches(r3, r_or, B)
+    base = oracle_mod.batch(g, np.full((g.n, 1), g.L - 1, dtype=np.uint8))
+    for fl in (emo.EMO_F_NO_STAGING, 0):
+        r3 = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, flags=fl, base=True)
+        assert_matches(r3, r_or, B)
+        assert r3["T0"] == base["makespan"][0]
+        assert r3["E0"] == pytest.approx(base["energy"][0], rel=E_RTOL)
+    # without the per-policy sums (the configuration the bench times)
+    r5 = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, want=("slack",), sums=False, base=True)
+    assert np.array_equal(r5["slack"][:, :B], r_or["slack"]) and r5["T0"] == base["makespan"][0]
+    assert (r5["slack_sum"] == -1).all()
     # an output pitch that is odd (no bulk copies of the ES rows possible) and one that is even
     for ldo in (B + 1, B + 2):
         r4 = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, ldo=ldo)
@@ -235,7 +248,7 @@ def test_cfg4_full_size_sampled(torch_cuda, emo, oracle_mod, golden):
     B = g.meta["B"]
     lv_dev = W.policies_for(g, device="cuda")
     h = emo.load_workload(g)
-    r = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, want=())
+    r = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, want=(), base=True)
     cols = sorted(set(np.linspace(0, B - 1, 16).astype(int).tolist() + [1, 2, B // 2 - 1, B // 2]))
     sub = lv_dev[:, cols].contiguous().cpu().numpy()
     r_sub = oracle_mod.batch(g, sub, want_arrays=True, threads=os.cpu_count() or 1)
@@ -247,7 +260,25 @@ def test_cfg4_full_size_sampled(torch_cuda, emo, oracle_mod, golden):
     sub_dev = torch.as_tensor(sub, device="cuda")
     r2 = gpu_slack_batch(torch, emo, h, sub_dev, len(cols), g.n)
     assert_matches(r2, r_sub, len(cols))
+    # the bench's configuration: slack materialised, no per-policy sums, baseline in the same launch
+    slack = torch.empty((g.n, B), dtype=torch.int64, device="cuda")
+    T = torch.zeros(B, dtype=torch.int64, device="cuda")
+    E = torch.zeros(B, dtype=torch.float64, device="cuda")
+    T0 = torch.zeros(1, dtype=torch.int64, device="cuda")
+    E0 = torch.zeros(1, dtype=torch.float64, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ws = torch.empty(emo.emo_workspace_bytes(h, B, 1), dtype=torch.uint8, device="cuda")
+    emo.emo_slack_batch(h, B, lv_dev, lv_dev.stride(0), None, None, slack, B, T, E, None, None, ws, status, T0=T0, E0=E0)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert np.array_equal(T.cpu().numpy(), r["makespan"])
+    assert np.array_equal(slack[:, torch.as_tensor(cols, device="cuda")].cpu().numpy(), r_sub["slack"])
+    assert np.array_equal(slack.sum(dim=0).cpu().numpy(), r["slack_sum"])
+    assert np.array_equal((slack == 0).sum(dim=0).cpu().numpy(), r["n_critical"])
+    assert int(T0.item()) == r["T0"]
+    del slack, ws
     if gold is not None:
+        assert r["T0"] == gold["T0"] and r["E0"] == pytest.approx(gold["E0"], rel=E_RTOL)
         assert (g.n, g.m, B) == (gold["n"], gold["m"], gold["B"])
         assert hashlib.sha256(np.ascontiguousarray(r["makespan"]).tobytes()).hexdigest() == gold["makespan_sha256"]
         assert hashlib.sha256(np.ascontiguousarray(r["slack_sum"]).tobytes()).hexdigest() == gold["slack_sum_sha256"]

@@ -50,15 +50,23 @@ def check_programs(emo, oracle_mod, g, lv, flags=0, group_of=None):
     info = h.info
     assert info.n == g.n and info.m == g.m and info.L == g.L
     r = oracle_mod.batch(g, lv, want_arrays=True, group_of=group_of)
-    lanes, steps, slots, Lp, ent, lat = emo.emo_graph_program(h, 0)
-    f = PE.run(ent, lat, Lp, g.L, slots, lv, g.n, False)
+    lanes, steps, slots, Lp, ent, rows, lat = emo.emo_graph_program(h, 0)
+    f = PE.run(ent, rows, lat, Lp, g.L, slots, lv, g.n, False)
     assert (f["seen"] == 1).all()
     assert np.array_equal(f["T"], r["makespan"])
     assert np.array_equal(f["ES"], r["ES"])
-    lanes_b, steps_b, slots_b, Lp_b, ent_b, lat_b = emo.emo_graph_program(h, 1)
+    lanes_b, steps_b, slots_b, Lp_b, ent_b, rows_b, lat_b = emo.emo_graph_program(h, 1)
     assert lanes_b == lanes
-    b = PE.run(ent_b, lat_b, Lp_b, g.L, slots_b, lv, g.n, True, ES_in=f["ES"], T_in=f["T"])
+    b = PE.run(ent_b, rows_b, lat_b, Lp_b, g.L, slots_b, lv, g.n, True, ES_in=f["ES"], T_in=f["T"])
     assert (b["seen"] == 1).all()
+    # forward entries address the row of the backward program that handles the same node
+    pos_b = {}
+    for t in range(steps_b):
+        for w in range(lanes_b):
+            if int(ent_b[t, w, 1]) & 1 and int(ent_b[t, w, 4]) != 0xFFFFFFFF:
+                pos_b[int(ent_b[t, w, 4])] = t * lanes_b + w
+    assert all(pos_b[node] == row for node, row in f["main_rows"])
+    assert all(node == row for node, row in b["main_rows"])
     assert np.array_equal(b["LS"], r["LS"])
     assert np.array_equal(b["slack"], r["slack"])
     h.free()
