@@ -67,12 +67,49 @@ int compile_program(const HostGraph &g, const int64_t *lat, const double *energy
     ops.reserve((size_t)n + 16);
     std::vector<int32_t> op_of_node((size_t)std::max(n, 1), -1);
     int n_aux = 0;
+    // Bounds of every node's value over all policies (forward: completion time C_v; backward: the
+    // longest tail Q_v), from the smallest and the largest entry of its duration row.  An operand
+    // whose upper bound does not exceed the lower bound of another operand of the same node can
+    // never decide that node's maximum (Eq. 1), under any policy, so the edge is dropped before
+    // scheduling: typically the launch edge of a kernel whose stream predecessor always finishes
+    // long after the launch chain has issued it.  Results are unchanged; slots, waits and maximum
+    // operations for such edges disappear.
+    std::vector<int64_t> lbv((size_t)std::max(n, 1), 0), ubv((size_t)std::max(n, 1), 0);
+    int64_t n_pruned = 0;
+    auto dur_bounds = [&](int32_t v, int64_t &lo, int64_t &hi) {
+        lo = hi = lat[(size_t)v * L];
+        if (g.group[v] < 0) return;
+        for (int l = 1; l < L; ++l) {
+            lo = std::min(lo, lat[(size_t)v * L + l]);
+            hi = std::max(hi, lat[(size_t)v * L + l]);
+        }
+    };
+    auto add_node = [&](int32_t v, std::vector<int32_t> &pn) {
+        std::sort(pn.begin(), pn.end());
+        pn.erase(std::unique(pn.begin(), pn.end()), pn.end());
+        int64_t lo_start = 0, hi_start = 0;
+        int32_t best = -1;
+        for (int32_t k : pn) {
+            hi_start = std::max(hi_start, ubv[k]);
+            if (best < 0 || lbv[k] > lbv[best]) best = k;
+        }
+        if (best >= 0) lo_start = lbv[best];
+        std::vector<int32_t> p;
+        for (int32_t k : pn) {
+            if (k != best && ubv[k] <= lbv[best]) { ++n_pruned; continue; }
+            p.push_back(op_of_node[k]);
+        }
+        int64_t dlo, dhi;
+        dur_bounds(v, dlo, dhi);
+        lbv[v] = lo_start + dlo;
+        ubv[v] = hi_start + dhi;
+        add_with_helpers(ops, v, std::move(p), n_aux);
+        op_of_node[v] = (int32_t)ops.size() - 1;
+    };
     if (!backward) {
         for (int32_t v = 0; v < n; ++v) {
-            std::vector<int32_t> p;
-            for (int64_t e = g.row_ptr[v]; e < g.row_ptr[v + 1]; ++e) p.push_back(op_of_node[g.col[e]]);
-            add_with_helpers(ops, v, std::move(p), n_aux);
-            op_of_node[v] = (int32_t)ops.size() - 1;
+            std::vector<int32_t> pn(g.col.begin() + g.row_ptr[v], g.col.begin() + g.row_ptr[v + 1]);
+            add_node(v, pn);
         }
     } else {
         std::vector<int64_t> sp((size_t)n + 1, 0);
@@ -83,12 +120,11 @@ int compile_program(const HostGraph &g, const int64_t *lat, const double *energy
         for (int32_t v = 0; v < n; ++v)
             for (int64_t e = g.row_ptr[v]; e < g.row_ptr[v + 1]; ++e) succ[fill[g.col[e]]++] = v;
         for (int32_t v = n - 1; v >= 0; --v) {
-            std::vector<int32_t> p;
-            for (int64_t e = sp[v]; e < sp[v + 1]; ++e) p.push_back(op_of_node[succ[e]]);
-            add_with_helpers(ops, v, std::move(p), n_aux);
-            op_of_node[v] = (int32_t)ops.size() - 1;
+            std::vector<int32_t> pn(succ.begin() + sp[v], succ.begin() + sp[v + 1]);
+            add_node(v, pn);
         }
     }
+    out.pruned = n_pruned;
     const int32_t N = (int32_t)ops.size();
     out.aux = n_aux;
 

@@ -35,6 +35,7 @@ constexpr int kSyncSteps = 8;         // the warps of a group meet at a barrier 
 
 struct Program {
     int lanes = 0, steps = 0, slots = 0, aux = 0, Lp = 0;
+    int64_t pruned = 0;               // edges dropped because they can never decide a maximum
     std::vector<uint32_t> entries;    // [steps][lanes][kEntryWords], see above
     std::vector<uint32_t> pos_of_node;   // [n] index (step*lanes + lane) of the entry that handles node v
     std::vector<uint32_t> rows;       // [steps][lanes] policy row whose level the entry reads (kNone: none)

@@ -158,6 +158,7 @@ bool staged_shape(const emo_graph *g, const Program &p, int rec_bytes, bool back
         for (int t = 0; t < 5; ++t) {
             const int sc = kTry[t][0], stages = kTry[t][1];
             const size_t ne = (size_t)sc * p.lanes;
+            if (ne > 32 * (size_t)kRowRegs) continue;
             const size_t stage_bytes = round_up(ne * ((size_t)rec_bytes + P + (backward ? P * 8 : 0)), 128);
             if (fixed + stages * stage_bytes > budget) continue;
             (void)per_step;

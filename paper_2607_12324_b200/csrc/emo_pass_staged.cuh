@@ -26,8 +26,10 @@
 #include "emo_kernels.cuh"
 
 constexpr int kMaxStages = 4;
+constexpr int kRowRegs = 8;             // a stage holds at most 32 * kRowRegs records
 constexpr unsigned kSlotStride = 528;   // 8-byte mbarrier, 8 bytes unused, 32 lanes x 16 bytes
 constexpr long long kWaitCycles = 4000000000LL;   // about two seconds: a wait that long has failed
+constexpr unsigned kSpinPolls = 1u << 14;          // polls between two looks at the clock
 
 struct StagedParams {
     PassParams p;
@@ -68,14 +70,19 @@ __device__ __forceinline__ bool emo_mbar_try(unsigned bar, unsigned parity)
     return ok != 0;
 }
 // Bounded wait: gives up after kWaitCycles and reports false (the caller raises EMO_E_TIMEOUT).
+__device__ __noinline__ bool emo_mbar_wait_slow(unsigned bar, unsigned parity)
+{
+    const long long t0 = clock64();
+    for (;;) {
+        for (unsigned i = 0; i < (1u << 14); ++i)
+            if (emo_mbar_try(bar, parity)) return true;
+        if (clock64() - t0 > kWaitCycles) return false;
+    }
+}
 __device__ __forceinline__ bool emo_mbar_wait(unsigned bar, unsigned parity)
 {
     if (emo_mbar_try(bar, parity)) return true;
-    const long long t0 = clock64();
-    while (!emo_mbar_try(bar, parity)) {
-        if (clock64() - t0 > kWaitCycles) return false;
-    }
-    return true;
+    return emo_mbar_wait_slow(bar, parity);
 }
 // 1-D bulk copy global -> shared, completion counted in bytes on an mbarrier.
 // dst, src 16-byte aligned, bytes a multiple of 16.
@@ -177,14 +184,20 @@ __device__ __forceinline__ long long *emo_row_ptr(long long *base, unsigned row,
 }
 // Wait until the slot's value with the given phase parity has been written.  Bounded; also gives
 // up as soon as another warp of the group has raised the abort flag.
+__device__ __noinline__ bool emo_slot_wait_slow(unsigned bar, unsigned parity, volatile int *abort_flag)
+{
+    // the clock is read rarely: reading it on every poll would keep the special-register path busy
+    const long long t0 = clock64();
+    for (;;) {
+        for (unsigned i = 0; i < kSpinPolls; ++i)
+            if (emo_mbar_try(bar, parity)) return true;
+        if (*abort_flag || clock64() - t0 > kWaitCycles) return false;
+    }
+}
 __device__ __forceinline__ bool emo_slot_wait(unsigned bar, unsigned parity, volatile int *abort_flag)
 {
     if (emo_mbar_try(bar, parity)) return true;
-    const long long t0 = clock64();
-    while (!emo_mbar_try(bar, parity)) {
-        if (*abort_flag || clock64() - t0 > kWaitCycles) return false;
-    }
-    return true;
+    return emo_slot_wait_slow(bar, parity, abort_flag);
 }
 
 template <bool BWD, int MAXT>
@@ -240,8 +253,23 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_pair(StagedParams sp)
         const long long *spill_tile = BWD ? reinterpret_cast<const long long *>(p.spill) + (size_t)blockIdx.x * p.spill_rows * ptile : nullptr;
         int issued = 0;
         bool gave_up = false;
+        // The level-row indices of a chunk are loaded one chunk ahead, 32 per register, so that no
+        // copy waits on a dependent global load: entry i's row sits in lane i % 32 of rr[i / 32].
+        unsigned rr[kRowRegs], rr_next[kRowRegs];
+        auto load_rows = [&](int c, unsigned *dst) {
+            const int step0 = c * sc;
+            const int ne = (c < n_chunks) ? min(sc, steps - step0) * lanes : 0;
+            const size_t q0 = (size_t)step0 * lanes;
+#pragma unroll
+            for (int k = 0; k < kRowRegs; ++k) {
+                const int i = 32 * k + lane;
+                dst[k] = (i < ne) ? __ldg(p.rows + q0 + i) : emo::kNone;
+            }
+        };
+        load_rows(0, rr);
         for (int c = 0; c < n_chunks; ++c) {
             const int s = c % nstages;
+            load_rows(c + 1, rr_next);
             if (c >= nstages) {
                 if (!emo_mbar_wait(bar0 + 8 * (kMaxStages + s), ((c / nstages) - 1) & 1)) {
                     if (lane == 0) {
@@ -264,21 +292,29 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_pair(StagedParams sp)
                 emo_bulk_g2s(sta, p.rec + q0 * rec_bytes, rb, full);
                 if (BWD) emo_bulk_g2s(sta + sp.off_es, spill_tile + q0 * ptile, eb, full);
             }
-            // level rows: entry i, 16-byte piece pc
+            // level rows: 32 entries x `pieces` 16-byte pieces per register of row indices
             if (pieces) {
-                int i = lane / pieces, pc = lane - i * pieces;
                 const int di = 32 / pieces, dpc = 32 - di * pieces;
-                while (i < ne) {
-                    const unsigned row = __ldg(p.rows + q0 + i);
-                    if (row != emo::kNone)
-                        emo_cp_async16(sta + sp.off_lvl + (unsigned)i * ptile + (unsigned)pc * 16u,
-                                       p.lvl + (size_t)row * p.ldb + b0 + pc * 16);
-                    i += di;
-                    pc += dpc;
-                    if (pc >= pieces) { pc -= pieces; ++i; }
+#pragma unroll
+                for (int k = 0; k < kRowRegs; ++k) {
+                    if (32 * k < ne) {
+                        int e = lane / pieces, pc = lane - e * pieces;
+                        for (int it = 0; it < pieces; ++it) {
+                            const unsigned row = __shfl_sync(0xFFFFFFFFu, rr[k], e & 31);
+                            const int i = 32 * k + e;
+                            if (e < 32 && i < ne && row != emo::kNone)
+                                emo_cp_async16(sta + sp.off_lvl + (unsigned)i * ptile + (unsigned)pc * 16u,
+                                               p.lvl + (size_t)row * p.ldb + b0 + pc * 16);
+                            e += di;
+                            pc += dpc;
+                            if (pc >= pieces) { pc -= pieces; ++e; }
+                        }
+                    }
                 }
             }
             emo_cp_async_arrive(full);
+#pragma unroll
+            for (int k = 0; k < kRowRegs; ++k) rr[k] = rr_next[k];
         }
         if (gave_up) {
             // do not leave the block while copies into its shared memory may still be in flight
