@@ -183,6 +183,27 @@ int emo_select(int64_t B, const int64_t *makespan, const double *energy, int64_t
                void *ws, size_t ws_bytes, void *stream);
 
 /*
+ * emo_select_static - emo_select for callers that must not allocate.  (The paper has no counterpart;
+ * this is a packaging variant of the selection above.)  Some callers cannot call cudaMalloc or any
+ * allocating routine: code running inside a latency-critical control loop that must not take the
+ * driver's allocation lock, a plug-in that was handed a stream but owns no memory pool, or a process
+ * whose device memory is fully pre-partitioned.  For them the scratch that emo_select takes as `ws`
+ * (one candidate per thread block) lives in a 16 KiB array inside the library, held by every GPU
+ * that loads the library until the process exits.
+ *   Arguments as emo_select, without ws.  B must not exceed EMO_SELECT_STATIC_MAX_B
+ *   (else EMO_E_RANGE); inputs and outputs are still the caller's device arrays.
+ *   The first call on a device looks up the array's device address (with that device current);
+ *   make that first call before any stream capture.  The call itself allocates nothing.
+ *   All calls on a device share the one array: calls whose kernels may overlap on the GPU (two
+ *   streams, two threads) race and give wrong results; serialise them.  The array keeps the last
+ *   call's candidates; every call overwrites what it later reads, so no clearing is needed.
+ */
+#define EMO_SELECT_STATIC_MAX_B 1048576
+int emo_select_static(int64_t B, const int64_t *makespan, const double *energy, int64_t target,
+                      const int64_t *target_dev, int64_t delta_ppm,
+                      int64_t *out_index, int64_t *out_T, double *out_E, void *stream);
+
+/*
  * emo_transpose_policies - layout helper: src device uint8 [B][lds] (one policy per row) to
  * dst device uint8 [rows][ldb].
  */

@@ -620,6 +620,43 @@ int emo_select(int64_t B, const int64_t *makespan, const double *energy, int64_t
     return EMO_OK;
 }
 
+// ---- selection without any allocation --------------------------------------------------------
+// Scratch for emo_select_static: the stage-1 candidates (one per block) live in this file-scope
+// device array instead of a caller workspace.  Every GPU that loads the library holds these 16 KiB
+// until the process exits.  In host code the array's name is only a stand-in; the device address
+// comes from cudaGetSymbolAddress, looked up once per device.
+static __device__ __align__(256) unsigned char emo_select_static_scratch[kSelectMaxBlocks * sizeof(SelectPartial)];
+static void *g_select_static_ptr[64] = {nullptr};
+
+int emo_select_static(int64_t B, const int64_t *makespan, const double *energy, int64_t target,
+                      const int64_t *target_dev, int64_t delta_ppm, int64_t *out_index, int64_t *out_T,
+                      double *out_E, void *stream)
+{
+    if (B < 0 || !out_index) return EMO_E_INVALID_ARG;
+    if (B > EMO_SELECT_STATIC_MAX_B) return EMO_E_RANGE;
+    if (B > 0 && (!makespan || !energy)) return EMO_E_INVALID_ARG;
+    int dev = 0;
+    EMO_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return EMO_E_UNSUPPORTED;
+    if (!g_select_static_ptr[dev]) {
+        // first call on this device (it is the current one): resolve the array's device address
+        void *ptr = nullptr;
+        EMO_CUDA(cudaGetSymbolAddress(&ptr, emo_select_static_scratch));
+        if (!ptr) return EMO_E_CUDA;
+        g_select_static_ptr[dev] = ptr;
+    }
+    SelectPartial *part = (SelectPartial *)g_select_static_ptr[dev];
+    cudaStream_t st = (cudaStream_t)stream;
+    int blocks = (int)std::max<int64_t>(1, std::min<int64_t>((B + 1023) / 1024, kSelectMaxBlocks));
+    // stage 1 overwrites the first `blocks` candidates and stage 2 reads exactly those, so nothing
+    // left behind by an earlier call is ever read and nothing needs clearing
+    emo_select_stage1<<<blocks, 256, 0, st>>>(B, makespan, energy, target, target_dev, delta_ppm, part);
+    EMO_CUDA(cudaGetLastError());
+    emo_select_stage2<<<1, 256, 0, st>>>(blocks, part, makespan, out_index, out_T, out_E);
+    EMO_CUDA(cudaGetLastError());
+    return EMO_OK;
+}
+
 int emo_transpose_policies(int64_t B, int64_t rows, const uint8_t *src, int64_t lds, uint8_t *dst,
                            int64_t ldb, void *stream)
 {

@@ -26,7 +26,7 @@ EXPORTS = [
     "emo_strerror", "emo_graph_load", "emo_graph_free", "emo_graph_info", "emo_workspace_bytes",
     "emo_eval_policies", "emo_slack_batch", "emo_slack", "emo_baseline", "emo_target_from_delta",
     "emo_select", "emo_transpose_policies", "emo_slack_batch_host", "emo_graph_program",
-    "emo_set_pass_events",
+    "emo_set_pass_events", "emo_select_static",
 ]
 
 
@@ -83,6 +83,7 @@ def lib():
                                         ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(p),
                                         ctypes.POINTER(p), ctypes.POINTER(p)]
         L.emo_set_pass_events.argtypes = [p, p, p, p]
+        L.emo_select_static.argtypes = [i64, p, p, i64, p, i64, p, p, p, p]
         for name in EXPORTS:
             if name not in ("emo_strerror", "emo_target_from_delta"):
                 getattr(L, name).restype = ctypes.c_int
@@ -213,6 +214,19 @@ def emo_select(B, makespan, energy, target, out_index, out_T=None, out_E=None, w
     _check(lib().emo_select(int(B), _addr(makespan), _addr(energy), int(target), _addr(target_dev),
                             int(delta_ppm), _addr(out_index), _addr(out_T), _addr(out_E), _addr(ws),
                             _nbytes(ws), _stream(stream)), "emo_select")
+
+
+EMO_SELECT_STATIC_MAX_B = 1048576
+
+
+def emo_select_static(B, makespan, energy, target, out_index, out_T=None, out_E=None, target_dev=None,
+                      delta_ppm: int = 0, stream=None):
+    """emo_select without a workspace: the per-block candidates live in a fixed array inside the
+    library, for callers that may not allocate device memory.  At most EMO_SELECT_STATIC_MAX_B
+    policies; calls on one device must not overlap."""
+    _check(lib().emo_select_static(int(B), _addr(makespan), _addr(energy), int(target), _addr(target_dev),
+                                   int(delta_ppm), _addr(out_index), _addr(out_T), _addr(out_E), _stream(stream)),
+           "emo_select_static")
 
 
 def emo_transpose_policies(B, rows, src, lds, dst, ldb, stream=None):
