@@ -145,7 +145,7 @@ bool staged_shape(const emo_graph *g, const Program &p, int rec_bytes, bool back
 {
     if (p.steps == 0 || !g->smem_optin) return false;
     int64_t n_groups = (NB + 63) / 64;
-    int gmax = std::min(31 / p.lanes, 15);
+    int gmax = std::min((32 - kProducerWarps) / p.lanes, 15);
     if (gmax < 1) return false;
     int64_t want = (n_groups + g->sm_count - 1) / g->sm_count;
     int G = (int)std::max<int64_t>(1, std::min<int64_t>(gmax, want));
@@ -173,7 +173,7 @@ bool staged_shape(const emo_graph *g, const Program &p, int rec_bytes, bool back
             sp.off_stage0 = (unsigned)round_up(sp.off_bar + 256, 128);
             s.groups = G;
             s.grid = (int)((n_groups + G - 1) / G);
-            s.threads = (G * p.lanes + 1) * 32;
+            s.threads = (G * p.lanes + kProducerWarps) * 32;
             s.smem = sp.off_stage0 + (size_t)stages * sp.stage_bytes;
             if (s.smem > budget) continue;
             return true;
@@ -264,8 +264,10 @@ int launch_pass(const emo_graph *g, const PassPlan &pl, bool backward, int64_t B
         sp.vec_out = (ldo % 2 == 0 && aligned16(LS) && aligned16(slack)) ? 1 : 0;
         sp.want_sums = (slack_sum || n_critical) ? 1 : 0;
         // two register budgets: blocks of at most 512 threads may use 128 registers per thread
-        void (*kern)(StagedParams) = backward ? (s.threads <= 512 ? emo_pass_pair<true, 512> : emo_pass_pair<true, 1024>)
-                                              : (s.threads <= 512 ? emo_pass_pair<false, 512> : emo_pass_pair<false, 1024>);
+        void (*kern)(StagedParams);
+        if (s.threads <= 512) kern = backward ? emo_pass_pair<true, 512> : emo_pass_pair<false, 512>;
+        else if (s.threads <= 768) kern = backward ? emo_pass_pair<true, 768> : emo_pass_pair<false, 768>;
+        else kern = backward ? emo_pass_pair<true, 1024> : emo_pass_pair<false, 1024>;
         EMO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s.smem));
         kern<<<s.grid, s.threads, s.smem, st>>>(sp);
     } else if (backward) {

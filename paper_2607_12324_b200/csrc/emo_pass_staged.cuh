@@ -27,6 +27,7 @@
 
 constexpr int kMaxStages = 4;
 constexpr int kRowRegs = 8;             // a stage holds at most 32 * kRowRegs records
+constexpr int kProducerWarps = 2;       // warps that issue the copies (they share the level-row pieces)
 constexpr unsigned kSlotStride = 528;   // 8-byte mbarrier, 8 bytes unused, 32 lanes x 16 bytes
 constexpr long long kWaitCycles = 4000000000LL;   // about two seconds: a wait that long has failed
 constexpr unsigned kSpinPolls = 1u << 14;          // polls between two looks at the clock
@@ -149,30 +150,36 @@ __device__ __forceinline__ long long emo_add_dur(long long h, unsigned d)
     return r;
 }
 
-// What a step needs from its stage, independent of the recurrence.
+// What a step needs from its stage, independent of the recurrence.  It is fetched in two phases,
+// each one step of the warp ahead of its use, so that no load is waited for: phase 1 reads the entry
+// and the level pair, phase 2 (one step later) looks the durations / energies up with those levels.
 struct EmoFetched {
     uint4 e;
-    unsigned node;
+    unsigned node, lv2;
+    unsigned rec_a;
     unsigned d0, d1;
     double g0, g1;
     long long es0, es1;
 };
 template <bool BWD>
-__device__ __forceinline__ void emo_fetch(EmoFetched &x, unsigned rec_a, unsigned lvl_a, unsigned es_a, unsigned en_off,
-                                          bool want_node)
+__device__ __forceinline__ void emo_fetch1(EmoFetched &x, unsigned rec_a, unsigned lvl_a, unsigned es_a, bool want_node)
 {
     x.e = emo_lds128(rec_a);
+    x.lv2 = emo_lds_u16(lvl_a);
+    x.rec_a = rec_a;
     if (want_node) x.node = emo_lds_u32(rec_a + 16u);
-    const unsigned lv2 = emo_lds_u16(lvl_a);
+    if (BWD) emo_lds_pair(es_a, x.es0, x.es1);
+}
+template <bool BWD>
+__device__ __forceinline__ void emo_fetch2(EmoFetched &x, unsigned en_off)
+{
     const unsigned m = (x.e.y >> emo::kMaskShift) & 255u;
-    const unsigned l0 = lv2 & m, l1 = (lv2 >> 8) & m;
-    x.d0 = emo_lds_u32(rec_a + 32u + l0 * 4u);
-    x.d1 = emo_lds_u32(rec_a + 32u + l1 * 4u);
+    const unsigned l0 = x.lv2 & m, l1 = (x.lv2 >> 8) & m;
+    x.d0 = emo_lds_u32(x.rec_a + 32u + l0 * 4u);
+    x.d1 = emo_lds_u32(x.rec_a + 32u + l1 * 4u);
     if (!BWD) {
-        x.g0 = emo_lds_f64(rec_a + en_off + l0 * 8u);
-        x.g1 = emo_lds_f64(rec_a + en_off + l1 * 8u);
-    } else {
-        emo_lds_pair(es_a, x.es0, x.es1);
+        x.g0 = emo_lds_f64(x.rec_a + en_off + l0 * 8u);
+        x.g1 = emo_lds_f64(x.rec_a + en_off + l1 * 8u);
     }
 }
 // base + row * pitch (bytes) as one wide multiply-add
@@ -208,8 +215,9 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_pair(StagedParams sp)
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     const int lanes = p.lanes, groups = p.groups, steps = p.steps, nstages = sp.stages, sc = sp.sc;
-    const int n_cons = groups * lanes;                  // consumer warps; warp n_cons is the producer
-    const bool producer = warp == n_cons;
+    const int n_cons = groups * lanes;                  // consumer warps; the warps after them produce
+    const bool producer = warp >= n_cons;
+    const int pw = warp - n_cons;                       // producer warp index
     const int group = producer ? 0 : warp / lanes;
     const int chain = warp - group * lanes;
     const int ptile = sp.ptile;
@@ -229,7 +237,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_pair(StagedParams sp)
     for (int i = threadIdx.x; i < groups * p.slots; i += blockDim.x) emo_mbar_init(smem0 + (unsigned)i * kSlotStride, 1);
     if (threadIdx.x == 0) {
         for (int k = 0; k < nstages; ++k) {
-            emo_mbar_init(bar0 + 8 * k, 33);      // one expect-tx arrival + the 32 lanes' cp.async arrivals
+            emo_mbar_init(bar0 + 8 * k, 1 + 32 * kProducerWarps);   // one expect-tx arrival + every producer lane's cp.async arrival
             emo_mbar_init(bar0 + 8 * (kMaxStages + k), n_cons);
         }
         for (int k = 0; k <= groups; ++k) abort_flag[k] = 0;
@@ -248,6 +256,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_pair(StagedParams sp)
         const int64_t lvl_left = p.ldb - b0;
         const unsigned lvl_bytes = lvl_left > 0 ? (unsigned)min((int64_t)ptile, lvl_left) : 0u;
         const int pieces = (int)(lvl_bytes >> 4);
+        const unsigned inv_pieces = pieces > 1 ? (unsigned)((0x100000000ULL + pieces - 1) / pieces) : 0u;
         const unsigned rec_bytes = (unsigned)p.rec_bytes;
         // this block's tile of the spill: [spill_rows][ptile] (the backward kernel's own tile width)
         const long long *spill_tile = BWD ? reinterpret_cast<const long long *>(p.spill) + (size_t)blockIdx.x * p.spill_rows * ptile : nullptr;
@@ -280,34 +289,34 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_pair(StagedParams sp)
                     break;
                 }
             }
+            if (abort_flag[groups]) { gave_up = true; break; }      // the other producer warp gave up
             issued = c + 1;
             const int step0 = c * sc;
             const int ne = min(sc, steps - step0) * lanes;
             const size_t q0 = (size_t)step0 * lanes;
             const unsigned sta = stage0 + (unsigned)s * stage_bytes;
             const unsigned full = bar0 + 8 * s;
-            if (lane == 0) {
+            if (lane == 0 && pw == 0) {
                 const unsigned rb = (unsigned)ne * rec_bytes, eb = BWD ? (unsigned)ne * ptile * 8u : 0u;
                 emo_mbar_expect_tx(full, rb + eb);
                 emo_bulk_g2s(sta, p.rec + q0 * rec_bytes, rb, full);
                 if (BWD) emo_bulk_g2s(sta + sp.off_es, spill_tile + q0 * ptile, eb, full);
             }
-            // level rows: 32 entries x `pieces` 16-byte pieces per register of row indices
+            // level rows: 32 entries x `pieces` 16-byte pieces per register of row indices; the
+            // producer warps take alternate iterations
             if (pieces) {
-                const int di = 32 / pieces, dpc = 32 - di * pieces;
 #pragma unroll
                 for (int k = 0; k < kRowRegs; ++k) {
                     if (32 * k < ne) {
-                        int e = lane / pieces, pc = lane - e * pieces;
-                        for (int it = 0; it < pieces; ++it) {
+                        for (int it = pw; it < pieces; it += kProducerWarps) {
+                            const unsigned t = (unsigned)lane + 32u * (unsigned)it;
+                            const unsigned e = pieces > 1 ? __umulhi(t, inv_pieces) : t;   // t / pieces (t < 2^16)
+                            const unsigned pc = t - e * (unsigned)pieces;
                             const unsigned row = __shfl_sync(0xFFFFFFFFu, rr[k], e & 31);
-                            const int i = 32 * k + e;
-                            if (e < 32 && i < ne && row != emo::kNone)
-                                emo_cp_async16(sta + sp.off_lvl + (unsigned)i * ptile + (unsigned)pc * 16u,
+                            const int i = 32 * k + (int)e;
+                            if (i < ne && row != emo::kNone)
+                                emo_cp_async16(sta + sp.off_lvl + (unsigned)i * ptile + pc * 16u,
                                                p.lvl + (size_t)row * p.ldb + b0 + pc * 16);
-                            e += di;
-                            pc += dpc;
-                            if (pc >= pieces) { pc -= pieces; ++e; }
                         }
                     }
                 }
@@ -354,21 +363,40 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_pair(StagedParams sp)
             if (!(e.y & emo::kRegPred)) { h0 = 0; h1 = 0; }
             const unsigned np = (e.y >> emo::kNPredShift) & 7u;
             if (np) {
-                unsigned ops = e.z, par = e.y >> emo::kOperandParityShift;
-                for (unsigned k = 0; k < np; ++k) {
-                    if (k == 4) ops = e.w;
-                    const unsigned bar = slotbar_base + (ops & 255u) * kSlotStride;
-                    if (!emo_slot_wait(bar, par & 1u, my_abort)) {
-                        *my_abort = 1;
-                        dead = true;
-                        return;
+                // all operands at once: poll every slot's barrier, then load every value, then take
+                // the maxima - the loads overlap instead of queuing behind one another
+                unsigned bars[emo::kMaxSlotPreds];
+                bool ready = true;
+#pragma unroll
+                for (int k = 0; k < emo::kMaxSlotPreds; ++k) {
+                    if (k < (int)np) {
+                        const unsigned id = ((k < 4 ? e.z : e.w) >> (8 * (k & 3))) & 255u;
+                        bars[k] = slotbar_base + id * kSlotStride;
+                        ready &= emo_mbar_try(bars[k], (e.y >> (emo::kOperandParityShift + k)) & 1u);
                     }
-                    long long x0, x1;
-                    emo_lds_pair(bar + lane16, x0, x1);
-                    ops >>= 8;
-                    par >>= 1;
-                    h0 = emo_max64(h0, x0);
-                    h1 = emo_max64(h1, x1);
+                }
+                if (!ready) {
+#pragma unroll
+                    for (int k = 0; k < emo::kMaxSlotPreds; ++k) {
+                        if (k < (int)np && !dead) {
+                            if (!emo_slot_wait(bars[k], (e.y >> (emo::kOperandParityShift + k)) & 1u, my_abort)) {
+                                *my_abort = 1;
+                                dead = true;
+                            }
+                        }
+                    }
+                    if (dead) return;
+                }
+                long long x0[emo::kMaxSlotPreds], x1[emo::kMaxSlotPreds];
+#pragma unroll
+                for (int k = 0; k < emo::kMaxSlotPreds; ++k)
+                    if (k < (int)np) emo_lds_pair(bars[k] + lane16, x0[k], x1[k]);
+#pragma unroll
+                for (int k = 0; k < emo::kMaxSlotPreds; ++k) {
+                    if (k < (int)np) {
+                        h0 = emo_max64(h0, x0[k]);
+                        h1 = emo_max64(h1, x1[k]);
+                    }
                 }
             }
             // here h is the node's start (forward: ES_v; backward: the longest tail behind v)
@@ -456,24 +484,26 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_pair(StagedParams sp)
             unsigned rec_a = sta + (unsigned)chain * p.rec_bytes;
             unsigned lvl_a = sta + sp.off_lvl + (unsigned)chain * ptile + col;
             unsigned es_a = sta + sp.off_es + ((unsigned)chain * ptile + col) * 8u;
-            // Everything a step reads from the stage (entry, level pair, durations, energies, ES pair)
-            // is independent of the recurrence, so it is fetched one step ahead.
-            EmoFetched fa, fb;
-            emo_fetch<BWD>(fa, rec_a, lvl_a, es_a, en_off, store_es);
-            for (int j = 0; j < ns; j += 2) {
+            // three records in flight per warp: `cur` is processed, `nxt` has its levels and gets its
+            // durations looked up, `pre` is being read from the stage
+            const unsigned d_es = d_lvl * 8u;
+            EmoFetched cur, nxt, pre;
+            emo_fetch1<BWD>(cur, rec_a, lvl_a, es_a, store_es);
+            if (ns > 1) emo_fetch1<BWD>(nxt, rec_a + d_rec, lvl_a + d_lvl, es_a + d_es, store_es);
+            emo_fetch2<BWD>(cur, en_off);
+            rec_a += 2 * d_rec;
+            lvl_a += 2 * d_lvl;
+            es_a += 2 * d_es;
+            for (int j = 0; j < ns; ++j) {
                 if (j && (j % emo::kSyncSteps) == 0 && lanes > 1) emo_group_barrier(group + 1, gthreads);
+                if (j + 2 < ns) emo_fetch1<BWD>(pre, rec_a, lvl_a, es_a, store_es);
+                if (j + 1 < ns) emo_fetch2<BWD>(nxt, en_off);
+                process(cur);
+                cur = nxt;
+                nxt = pre;
                 rec_a += d_rec;
                 lvl_a += d_lvl;
-                es_a += d_lvl * 8u;
-                if (j + 1 < ns) emo_fetch<BWD>(fb, rec_a, lvl_a, es_a, en_off, store_es);
-                process(fa);
-                if (j + 1 < ns) {
-                    rec_a += d_rec;
-                    lvl_a += d_lvl;
-                    es_a += d_lvl * 8u;
-                    if (j + 2 < ns) emo_fetch<BWD>(fa, rec_a, lvl_a, es_a, en_off, store_es);
-                    process(fb);
-                }
+                es_a += d_es;
             }
             __syncwarp();
             if (lane == 0) emo_mbar_arrive(bar0 + 8 * (kMaxStages + s));
