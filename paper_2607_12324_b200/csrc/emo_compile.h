@@ -31,7 +31,7 @@ constexpr int kMaskShift = 8;         // bits 8..15: mask applied to the level b
 constexpr int kOutShift = 16;         // bits 16..23: slot written
 constexpr int kOutParityShift = 24;   // bit 24: phase parity of the value written
 constexpr int kOperandParityShift = 25;   // bits 25..30: phase parity of each operand's value
-constexpr int kSyncSteps = 4;         // the warps of a group meet at a barrier every kSyncSteps steps
+constexpr int kSyncSteps = 8;         // the warps of a group meet at a barrier every kSyncSteps steps
 
 struct Program {
     int lanes = 0, steps = 0, slots = 0, aux = 0, Lp = 0;

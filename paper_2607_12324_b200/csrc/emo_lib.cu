@@ -138,51 +138,42 @@ int shape_for(const emo_graph *g, const Program &p, int64_t NB, LaunchShape &s)
     return EMO_OK;
 }
 
-// Shape of the staged kernel: groups of 64 policies (two per thread) served by `lanes` chain warps
-// each, plus lookup warps, (backward) output warps and the producer warps; then as many steps per
-// stage and stages as fit beside the slots.  Returns false when it cannot be used.
+// Shape of the staged kernel: groups of 64 policies (two per thread), one more warp produces, then
+// as many steps per stage as fit beside the slots.  Returns false when it cannot be used.
 bool staged_shape(const emo_graph *g, const Program &p, int rec_bytes, bool backward, int64_t NB, LaunchShape &s,
                   StagedParams &sp)
 {
     if (p.steps == 0 || !g->smem_optin) return false;
     int64_t n_groups = (NB + 63) / 64;
+    int gmax = std::min((32 - kProducerWarps) / p.lanes, 15);
+    if (gmax < 1) return false;
     int64_t want = (n_groups + g->sm_count - 1) / g->sm_count;
+    int G = (int)std::max<int64_t>(1, std::min<int64_t>(gmax, want));
     const size_t budget = g->smem_optin;
-    static const int kTry[9][2] = {{16, 4}, {16, 3}, {8, 4}, {8, 3}, {4, 4}, {8, 2}, {4, 3}, {16, 2}, {4, 2}};   // {steps per stage, stages}
-    for (int G = (int)std::max<int64_t>(1, std::min<int64_t>(15, want)); G >= 1; --G) {
-        // lookup (and output) lanes: two per policy pair while the block stays small, else one
-        const int n_look = (G <= 4) ? 2 * G : G;
-        const int nparts = (G <= 4) ? 2 : 1;
-        const int n_out = backward ? n_look : 0;
-        const int warps = G * p.lanes + n_look + n_out + kProducerWarps;
-        if (warps > 32) continue;
+    static const int kTry[5][2] = {{16, 4}, {16, 3}, {8, 4}, {8, 3}, {8, 2}};   // {steps per stage, stages}
+    for (; G >= 1; --G) {
         const size_t P = 64 * (size_t)G;
-        const size_t part_bytes = (size_t)G * p.lanes * 32 * 16 + (size_t)n_look * 32 * 16 + (size_t)n_out * 32 * 32;
-        const size_t fixed = round_up((size_t)G * p.slots * kSlotStride, 16) + part_bytes + 256 + 128;
-        const size_t per_entry = (size_t)rec_bytes + P + P * 4 + (backward ? P * 8 : 0);
-        for (int t = 0; t < 9; ++t) {
+        const size_t fixed = (size_t)G * p.slots * kSlotStride + (size_t)G * p.lanes * 1024 + 256 + 128;
+        const size_t per_step = (size_t)p.lanes * ((size_t)rec_bytes + P + (backward ? P * 8 : 0));
+        for (int t = 0; t < 5; ++t) {
             const int sc = kTry[t][0], stages = kTry[t][1];
-            if (sc % kSyncSteps != 0) continue;
             const size_t ne = (size_t)sc * p.lanes;
             if (ne > 32 * (size_t)kRowRegs) continue;
-            const size_t stage_bytes = round_up(ne * per_entry, 128);
+            const size_t stage_bytes = round_up(ne * ((size_t)rec_bytes + P + (backward ? P * 8 : 0)), 128);
             if (fixed + stages * stage_bytes > budget) continue;
+            (void)per_step;
             sp.sc = sc;
             sp.stages = stages;
             sp.ptile = (int)P;
-            sp.n_lookup = n_look;
-            sp.n_output = n_out;
-            sp.nparts = nparts;
             sp.off_lvl = (unsigned)(ne * rec_bytes);
-            sp.off_d = sp.off_lvl + (unsigned)(ne * P);
-            sp.off_q = sp.off_d + (unsigned)(ne * P * 4);
+            sp.off_es = sp.off_lvl + (unsigned)(ne * P);
             sp.stage_bytes = (unsigned)stage_bytes;
             sp.off_part = (unsigned)round_up((size_t)G * p.slots * kSlotStride, 16);
-            sp.off_bar = sp.off_part + (unsigned)part_bytes;
+            sp.off_bar = sp.off_part + (unsigned)((size_t)G * p.lanes * 1024);
             sp.off_stage0 = (unsigned)round_up(sp.off_bar + 256, 128);
             s.groups = G;
             s.grid = (int)((n_groups + G - 1) / G);
-            s.threads = warps * 32;
+            s.threads = (G * p.lanes + kProducerWarps) * 32;
             s.smem = sp.off_stage0 + (size_t)stages * sp.stage_bytes;
             if (s.smem > budget) continue;
             return true;
@@ -273,11 +264,17 @@ int launch_pass(const emo_graph *g, const PassPlan &pl, bool backward, int64_t B
         sp.vec_out = (ldo % 2 == 0 && aligned16(LS) && aligned16(slack)) ? 1 : 0;
         sp.want_sums = (slack_sum || n_critical) ? 1 : 0;
         // two register budgets: blocks of at most 512 threads may use 128 registers per thread
+        // lean instantiation when the call asks for nothing beyond the spill (forward) or the slack
+        // matrix with 16-byte aligned rows (backward); register budget by block size
+        const bool extra = backward ? (LS != nullptr || sp.want_sums || !sp.vec_out) : (ES != nullptr);
         void (*kern)(StagedParams);
-        if (s.threads <= 512) kern = backward ? emo_pass_pair<true, 512> : emo_pass_pair<false, 512>;
-        else if (s.threads <= 640) kern = backward ? emo_pass_pair<true, 640> : emo_pass_pair<false, 640>;
-        else if (s.threads <= 768) kern = backward ? emo_pass_pair<true, 768> : emo_pass_pair<false, 768>;
-        else kern = backward ? emo_pass_pair<true, 1024> : emo_pass_pair<false, 1024>;
+#define EMO_PICK(MAXT)                                                                                         \
+    kern = backward ? (extra ? emo_pass_pair<true, true, MAXT> : emo_pass_pair<true, false, MAXT>)                 \
+                    : (extra ? emo_pass_pair<false, true, MAXT> : emo_pass_pair<false, false, MAXT>)
+        if (s.threads <= 512) EMO_PICK(512);
+        else if (s.threads <= 768) EMO_PICK(768);
+        else EMO_PICK(1024);
+#undef EMO_PICK
         EMO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s.smem));
         kern<<<s.grid, s.threads, s.smem, st>>>(sp);
     } else if (backward) {

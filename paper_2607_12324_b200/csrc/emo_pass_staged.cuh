@@ -7,25 +7,16 @@
 // per 128-byte row costs far more than it moves).  Each record and each level row is fetched once
 // per block and used by every policy of the block.
 //
-// A thread carries TWO adjacent policies, so a warp covers 64 policies: the level pair is one
+// A consumer thread carries TWO adjacent policies, so a warp covers 64 policies of one schedule
+// lane: the entry decode and the address arithmetic are paid once per pair, the level pair is one
 // 16-bit load, an exchange slot holds both values and moves with one 128-bit access, and the
 // per-node outputs leave as 128-bit stores.
 //
-// The block is warp-specialised, because the recurrence is a long serial chain per policy and a
-// single warp issues dependent instructions slowly.  Only what is serial stays on the chain warps:
-//   producer warps  copy a stage in;
-//   lookup warps    turn every level of the stage into a duration (and add up the energies): this
-//                   work has no order, so any number of warps can share it;
-//   chain warps     one per schedule lane and group of 64 policies, run the max-plus recurrence
-//                   over their column of the step program, reading durations that are already there;
-//   output warps    (backward pass) turn the chain warps' values into LS and slack and store them.
-// A stage passes through full -> ready -> (done ->) empty mbarriers.
-//
-// The chain warps of a group do not run in lockstep.  Each waits only for the values it reads:
-// every exchange slot has an mbarrier whose phase completes when the slot's next value has been
-// written, and the entry names the phase parity to wait for.  The group meets at a named barrier
-// every kSyncSteps steps, which bounds the drift between its warps; the host compiler reuses a slot
-// only across such a barrier.  Included only by emo_lib.cu.
+// The warps of a group do not run in lockstep.  Each walks its own column of the step program and
+// waits only for the values it reads: every exchange slot has an mbarrier whose phase completes
+// when the slot's next value has been written, and the entry names the phase parity to wait for.
+// The group meets at a named barrier every kSyncSteps steps, which bounds the drift between its
+// warps; the host compiler reuses a slot only across such a barrier.  Included only by emo_lib.cu.
 #pragma once
 #include <cuda_runtime.h>
 
@@ -36,7 +27,7 @@
 
 constexpr int kMaxStages = 4;
 constexpr int kRowRegs = 8;             // a stage holds at most 32 * kRowRegs records
-constexpr int kProducerWarps = 2;       // warps that issue the copies (they share the level-row pieces)
+constexpr int kProducerWarps = 1;       // warps that issue the copies (they share the level-row pieces)
 constexpr unsigned kSlotStride = 528;   // 8-byte mbarrier, 8 bytes unused, 32 lanes x 16 bytes
 constexpr long long kWaitCycles = 4000000000LL;   // about two seconds: a wait that long has failed
 constexpr unsigned kSpinPolls = 1u << 14;          // polls between two looks at the clock
@@ -46,12 +37,10 @@ struct StagedParams {
     int sc;                    // steps per stage (a multiple of kSyncSteps)
     int stages;                // ring depth
     int ptile;                 // policies per block = 64 * groups
-    int n_lookup, n_output;    // lookup warps; output warps (backward only)
-    int nparts;                // lookup/output lanes per policy pair (they split the entries of a stage)
     int vec_es, vec_out;       // 128-bit global accesses allowed for ES / for LS and slack
     int want_sums;             // backward: accumulate slack sums and critical counts
     unsigned stage_bytes;      // bytes of one stage
-    unsigned off_lvl, off_d, off_q;   // offsets inside a stage: level rows, durations, chain values (records at 0)
+    unsigned off_lvl, off_es;  // offsets inside a stage (records start at 0)
     unsigned off_part, off_bar, off_stage0;      // offsets inside dynamic shared memory
 };
 
@@ -81,21 +70,20 @@ __device__ __forceinline__ bool emo_mbar_try(unsigned bar, unsigned parity)
         : "memory");
     return ok != 0;
 }
-__device__ __noinline__ bool emo_mbar_wait_slow(unsigned bar, unsigned parity, volatile int *abort_flag)
+// Bounded wait: gives up after kWaitCycles and reports false (the caller raises EMO_E_TIMEOUT).
+__device__ __noinline__ bool emo_mbar_wait_slow(unsigned bar, unsigned parity)
 {
-    // the clock is read rarely: reading it on every poll would keep the special-register path busy
     const long long t0 = clock64();
     for (;;) {
-        for (unsigned i = 0; i < kSpinPolls; ++i)
+        for (unsigned i = 0; i < (1u << 14); ++i)
             if (emo_mbar_try(bar, parity)) return true;
-        if (*abort_flag || clock64() - t0 > kWaitCycles) return false;
+        if (clock64() - t0 > kWaitCycles) return false;
     }
 }
-// Bounded wait; also gives up as soon as another warp of the block has raised the abort flag.
-__device__ __forceinline__ bool emo_mbar_wait(unsigned bar, unsigned parity, volatile int *abort_flag)
+__device__ __forceinline__ bool emo_mbar_wait(unsigned bar, unsigned parity)
 {
     if (emo_mbar_try(bar, parity)) return true;
-    return emo_mbar_wait_slow(bar, parity, abort_flag);
+    return emo_mbar_wait_slow(bar, parity);
 }
 // 1-D bulk copy global -> shared, completion counted in bytes on an mbarrier.
 // dst, src 16-byte aligned, bytes a multiple of 16.
@@ -162,6 +150,32 @@ __device__ __forceinline__ long long emo_add_dur(long long h, unsigned d)
     return r;
 }
 
+// What a step needs from its stage, independent of the recurrence; fetched one step ahead of its use.
+struct EmoFetched {
+    uint4 e;
+    unsigned node;
+    unsigned d0, d1;
+    double g0, g1;
+    long long es0, es1;
+};
+template <bool BWD>
+__device__ __forceinline__ void emo_fetch(EmoFetched &x, unsigned rec_a, unsigned lvl_a, unsigned es_a, unsigned en_off,
+                                          bool want_node)
+{
+    x.e = emo_lds128(rec_a);
+    if (want_node) x.node = emo_lds_u32(rec_a + 16u);
+    const unsigned lv2 = emo_lds_u16(lvl_a);
+    const unsigned m = (x.e.y >> emo::kMaskShift) & 255u;
+    const unsigned l0 = lv2 & m, l1 = (lv2 >> 8) & m;
+    x.d0 = emo_lds_u32(rec_a + 32u + l0 * 4u);
+    x.d1 = emo_lds_u32(rec_a + 32u + l1 * 4u);
+    if (!BWD) {
+        x.g0 = emo_lds_f64(rec_a + en_off + l0 * 8u);
+        x.g1 = emo_lds_f64(rec_a + en_off + l1 * 8u);
+    } else {
+        emo_lds_pair(es_a, x.es0, x.es1);
+    }
+}
 // base + row * pitch (bytes) as one wide multiply-add
 __device__ __forceinline__ long long *emo_row_ptr(long long *base, unsigned row, unsigned pitch_bytes)
 {
@@ -169,33 +183,28 @@ __device__ __forceinline__ long long *emo_row_ptr(long long *base, unsigned row,
     asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(r) : "r"(row), "r"(pitch_bytes), "l"(reinterpret_cast<unsigned long long>(base)));
     return reinterpret_cast<long long *>(r);
 }
-__device__ __forceinline__ void emo_lds_u32x2(unsigned a, unsigned &x0, unsigned &x1)
+// Wait until the slot's value with the given phase parity has been written.  Bounded; also gives
+// up as soon as another warp of the group has raised the abort flag.
+__device__ __noinline__ bool emo_slot_wait_slow(unsigned bar, unsigned parity, volatile int *abort_flag)
 {
-    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(x0), "=r"(x1) : "r"(a));
+    // the clock is read rarely: reading it on every poll would keep the special-register path busy
+    const long long t0 = clock64();
+    for (;;) {
+        for (unsigned i = 0; i < kSpinPolls; ++i)
+            if (emo_mbar_try(bar, parity)) return true;
+        if (*abort_flag || clock64() - t0 > kWaitCycles) return false;
+    }
 }
-__device__ __forceinline__ void emo_sts_u32x2(unsigned a, unsigned x0, unsigned x1)
+__device__ __forceinline__ bool emo_slot_wait(unsigned bar, unsigned parity, volatile int *abort_flag)
 {
-    asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"(a), "r"(x0), "r"(x1) : "memory");
-}
-__device__ __forceinline__ void emo_ldg_pair(const long long *p, long long &x0, long long &x1)
-{
-    asm volatile("ld.global.v2.s64 {%0, %1}, [%2];" : "=l"(x0), "=l"(x1) : "l"(p));
-}
-
-// What a chain warp reads per step: the entry and the duration pair (and the node id when the
-// caller wants ES in its own numbering).  Fetched one step ahead.
-struct EmoFetched {
-    uint4 e;
-    unsigned node, d0, d1;
-};
-__device__ __forceinline__ void emo_fetch(EmoFetched &x, unsigned rec_a, unsigned d_a, bool want_node)
-{
-    x.e = emo_lds128(rec_a);
-    emo_lds_u32x2(d_a, x.d0, x.d1);
-    if (want_node) x.node = emo_lds_u32(rec_a + 16u);
+    if (emo_mbar_try(bar, parity)) return true;
+    return emo_slot_wait_slow(bar, parity, abort_flag);
 }
 
-template <bool BWD, int MAXT>
+// EXTRA = false is the lean instantiation for the common call (forward: ES only into the spill;
+// backward: slack only, 16-byte aligned rows, no per-policy sums): the hot loop stays small, which
+// matters because all warps of the block share the instruction cache.
+template <bool BWD, bool EXTRA, int MAXT>
 __global__ void __launch_bounds__(MAXT, 1) emo_pass_pair(StagedParams sp)
 {
     extern __shared__ __align__(128) unsigned char emo_smem[];
@@ -203,32 +212,30 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_pair(StagedParams sp)
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     const int lanes = p.lanes, groups = p.groups, steps = p.steps, nstages = sp.stages, sc = sp.sc;
-    const int n_cons = groups * lanes;                  // chain warps
-    const int w_lookup = n_cons, w_output = w_lookup + sp.n_lookup, w_prod = w_output + (BWD ? sp.n_output : 0);
-    const int role = warp < w_lookup ? 0 : warp < w_output ? 1 : warp < w_prod ? 2 : 3;   // chain, lookup, output, producer
-    const int ptile = sp.ptile, pairs = ptile >> 1;
+    const int n_cons = groups * lanes;                  // consumer warps; the warps after them produce
+    const bool producer = warp >= n_cons;
+    const int pw = warp - n_cons;                       // producer warp index
+    const int group = producer ? 0 : warp / lanes;
+    const int chain = warp - group * lanes;
+    const int ptile = sp.ptile;
     const int64_t b0 = (int64_t)blockIdx.x * ptile;
+    const int col = group * 64 + 2 * lane;
+    const int64_t b = b0 + col;
+    const bool act0 = !producer && b < p.B, act1 = !producer && b + 1 < p.B;
+    // column of the virtual all-max policy inside this block's tile (fwd only), or -1
+    const int base_col = (!BWD && p.want_base && p.B >= b0 && p.B < b0 + ptile) ? (int)(p.B - b0) : -1;
+    unsigned char *part_base = emo_smem + sp.off_part;
     const unsigned smem0 = emo_smem_addr(emo_smem);
-    // barriers: full[k], ready[k], done[k], empty[k] (kMaxStages each), then the abort flags
-    const unsigned bar_full = smem0 + sp.off_bar, bar_ready = bar_full + 8 * kMaxStages,
-                   bar_done = bar_ready + 8 * kMaxStages, bar_empty = bar_done + 8 * kMaxStages;
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(emo_smem + sp.off_bar + 32 * kMaxStages);
-    volatile int *abort_all = abort_flag + groups;      // one per group, then one for the whole block
+    const unsigned bar0 = smem0 + sp.off_bar;           // full[k] at bar0 + 8k, empty[k] after them
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(emo_smem + sp.off_bar + 16 * kMaxStages);
     const unsigned stage0 = smem0 + sp.off_stage0;
     const unsigned stage_bytes = sp.stage_bytes;
-    const unsigned rec_bytes = (unsigned)p.rec_bytes;
-    // partial results: chain warps {acc0, acc1} per thread, then lookup lanes {e0, e1}, then output lanes {s0, s1, c0, c1}
-    long long *part_chain = reinterpret_cast<long long *>(emo_smem + sp.off_part);
-    long long *part_look = part_chain + (size_t)n_cons * 32 * 2;
-    long long *part_out = part_look + (size_t)sp.n_lookup * 32 * 2;
 
     for (int i = threadIdx.x; i < groups * p.slots; i += blockDim.x) emo_mbar_init(smem0 + (unsigned)i * kSlotStride, 1);
     if (threadIdx.x == 0) {
         for (int k = 0; k < nstages; ++k) {
-            emo_mbar_init(bar_full + 8 * k, 1 + 32 * kProducerWarps);   // one expect-tx arrival + every producer lane's cp.async arrival
-            emo_mbar_init(bar_ready + 8 * k, sp.n_lookup);
-            emo_mbar_init(bar_done + 8 * k, n_cons);
-            emo_mbar_init(bar_empty + 8 * k, BWD ? sp.n_output : n_cons);
+            emo_mbar_init(bar0 + 8 * k, 1 + 32 * kProducerWarps);   // one expect-tx arrival + every producer lane's cp.async arrival
+            emo_mbar_init(bar0 + 8 * (kMaxStages + k), n_cons);
         }
         for (int k = 0; k <= groups; ++k) abort_flag[k] = 0;
     }
@@ -236,16 +243,20 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_pair(StagedParams sp)
     __syncthreads();
 
     const int n_chunks = (steps + sc - 1) / sc;
-    // column of the virtual all-max policy inside this block's tile (forward only), or -1
-    const int base_col = (!BWD && p.want_base && p.B >= b0 && p.B < b0 + ptile) ? (int)(p.B - b0) : -1;
+    long long h0 = 0, h1 = 0;
+    double ea0 = 0.0, ea1 = 0.0;
+    long long acc0 = 0, acc1 = 0;      // forward: running makespan; backward: slack sums
+    int nc0 = 0, nc1 = 0;
 
-    if (role == 3) {
-        // ---------------------------------------------------------------------------- producers
-        const int pw = warp - w_prod;
+    if (producer) {
+        // ---------------------------------------------------------------------------- producer
         const int64_t lvl_left = p.ldb - b0;
         const unsigned lvl_bytes = lvl_left > 0 ? (unsigned)min((int64_t)ptile, lvl_left) : 0u;
         const int pieces = (int)(lvl_bytes >> 4);
         const unsigned inv_pieces = pieces > 1 ? (unsigned)((0x100000000ULL + pieces - 1) / pieces) : 0u;
+        const unsigned rec_bytes = (unsigned)p.rec_bytes;
+        // this block's tile of the spill: [spill_rows][ptile] (the backward kernel's own tile width)
+        const long long *spill_tile = BWD ? reinterpret_cast<const long long *>(p.spill) + (size_t)blockIdx.x * p.spill_rows * ptile : nullptr;
         int issued = 0;
         bool gave_up = false;
         // The level-row indices of a chunk are loaded one chunk ahead, 32 per register, so that no
@@ -265,24 +276,28 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_pair(StagedParams sp)
         for (int c = 0; c < n_chunks; ++c) {
             const int s = c % nstages;
             load_rows(c + 1, rr_next);
-            if (c >= nstages && !emo_mbar_wait(bar_empty + 8 * s, ((c / nstages) - 1) & 1, abort_all)) {
-                if (lane == 0) {
-                    *abort_all = 1;
-                    if (p.status) atomicMin(p.status, -8);
+            if (c >= nstages) {
+                if (!emo_mbar_wait(bar0 + 8 * (kMaxStages + s), ((c / nstages) - 1) & 1)) {
+                    if (lane == 0) {
+                        abort_flag[groups] = 1;
+                        if (p.status) atomicMin(p.status, -8);
+                    }
+                    gave_up = true;
+                    break;
                 }
-                gave_up = true;
-                break;
             }
+            if (abort_flag[groups]) { gave_up = true; break; }      // the other producer warp gave up
             issued = c + 1;
             const int step0 = c * sc;
             const int ne = min(sc, steps - step0) * lanes;
             const size_t q0 = (size_t)step0 * lanes;
             const unsigned sta = stage0 + (unsigned)s * stage_bytes;
-            const unsigned full = bar_full + 8 * s;
+            const unsigned full = bar0 + 8 * s;
             if (lane == 0 && pw == 0) {
-                const unsigned rb = (unsigned)ne * rec_bytes;
-                emo_mbar_expect_tx(full, rb);
+                const unsigned rb = (unsigned)ne * rec_bytes, eb = BWD ? (unsigned)ne * ptile * 8u : 0u;
+                emo_mbar_expect_tx(full, rb + eb);
                 emo_bulk_g2s(sta, p.rec + q0 * rec_bytes, rb, full);
+                if (BWD) emo_bulk_g2s(sta + sp.off_es, spill_tile + q0 * ptile, eb, full);
             }
             // level rows: 32 entries x `pieces` 16-byte pieces per register of row indices; the
             // producer warps take alternate iterations
@@ -309,168 +324,61 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_pair(StagedParams sp)
         }
         if (gave_up) {
             // do not leave the block while copies into its shared memory may still be in flight
-            for (int c = max(0, issued - nstages); c < issued; ++c) {
-                const unsigned bar = bar_full + 8 * (c % nstages);
-                const long long t0 = clock64();
-                while (!emo_mbar_try(bar, (c / nstages) & 1) && clock64() - t0 < kWaitCycles) {}
-            }
+            for (int c = max(0, issued - nstages); c < issued; ++c) (void)emo_mbar_wait(bar0 + 8 * (c % nstages), (c / nstages) & 1);
         }
-    } else if (role == 1) {
-        // ------------------------------------------------------------------------- lookup warps
-        // lane = (policy pair, part); the parts of a pair split the entries of a stage between them
-        const int lt = (warp - w_lookup) * 32 + lane;
-        const int pair = lt % pairs, part = lt / pairs;
-        const unsigned en_off = 32u + (unsigned)p.Lp * 4u;
-        const unsigned top = (unsigned)(p.L - 1);
-        const bool isb0 = base_col == 2 * pair, isb1 = base_col == 2 * pair + 1;
-        double ea0 = 0.0, ea1 = 0.0;
-        for (int c = 0; c < n_chunks; ++c) {
-            const int s = c % nstages;
-            if (!emo_mbar_wait(bar_full + 8 * s, (c / nstages) & 1, abort_all)) {
-                if (lane == 0) {
-                    *abort_all = 1;
-                    if (p.status) atomicMin(p.status, -8);
-                }
-                break;
-            }
-            const unsigned sta = stage0 + (unsigned)s * stage_bytes;
-            const int ne = min(sc, steps - c * sc) * lanes;
-            for (int i = part; i < ne; i += sp.nparts) {
-                const unsigned rec_a = sta + (unsigned)i * rec_bytes;
-                const unsigned m = (emo_lds_u32(rec_a + 4u) >> emo::kMaskShift) & 255u;
-                unsigned lv2 = emo_lds_u16(sta + sp.off_lvl + (unsigned)i * ptile + 2u * (unsigned)pair);
-                unsigned l0 = lv2 & 255u, l1 = lv2 >> 8;
-                if (isb0) l0 = top;
-                if (isb1) l1 = top;
-                l0 &= m;
-                l1 &= m;
-                const unsigned d0 = emo_lds_u32(rec_a + 32u + l0 * 4u), d1 = emo_lds_u32(rec_a + 32u + l1 * 4u);
-                emo_sts_u32x2(sta + sp.off_d + ((unsigned)i * ptile + 2u * (unsigned)pair) * 4u, d0, d1);
-                if (!BWD) {
-                    ea0 += emo_lds_f64(rec_a + en_off + l0 * 8u);
-                    ea1 += emo_lds_f64(rec_a + en_off + l1 * 8u);
-                }
-            }
-            __syncwarp();
-            if (lane == 0) emo_mbar_arrive(bar_ready + 8 * s);
-        }
-        if (!BWD) {
-            part_look[(size_t)lt * 2] = __double_as_longlong(ea0);
-            part_look[(size_t)lt * 2 + 1] = __double_as_longlong(ea1);
-        }
-    } else if (role == 2) {
-        // ------------------------------------------------------------------------- output warps
-        // (backward pass) LS_v = T - Q_v, slack_v = LS_v - ES_v for every node of the stage
-        const int ot = (warp - w_output) * 32 + lane;
-        const int pair = ot % pairs, part = ot / pairs;
-        const int64_t b = b0 + 2 * pair;
-        const bool act0 = b < p.B, act1 = b + 1 < p.B;
-        const long long T0 = act0 ? p.makespan[b] : 0, T1 = act1 ? p.makespan[b + 1] : 0;
-        const unsigned ldo8 = (unsigned)p.ldo * 8u;
-        long long *const ls_lane = p.LS ? reinterpret_cast<long long *>(p.LS) + b : nullptr;
-        long long *const sl_lane = p.slack ? reinterpret_cast<long long *>(p.slack) + b : nullptr;
-        const bool vec_out = sp.vec_out && act1;
-        const long long *spill_lane = reinterpret_cast<const long long *>(p.spill) + (size_t)blockIdx.x * p.spill_rows * ptile + 2 * pair;
-        long long sum0 = 0, sum1 = 0;
-        int cnt0 = 0, cnt1 = 0;
-        constexpr int kBatch = 4;
-        for (int c = 0; c < n_chunks; ++c) {
-            const int s = c % nstages;
-            if (!emo_mbar_wait(bar_done + 8 * s, (c / nstages) & 1, abort_all)) {
-                if (lane == 0) {
-                    *abort_all = 1;
-                    if (p.status) atomicMin(p.status, -8);
-                }
-                break;
-            }
-            const unsigned sta = stage0 + (unsigned)s * stage_bytes;
-            const int ne = min(sc, steps - c * sc) * lanes;
-            const size_t q0 = (size_t)c * sc * lanes;
-            for (int i0 = part; i0 < ne; i0 += sp.nparts * kBatch) {
-                unsigned node[kBatch];
-                long long es0[kBatch], es1[kBatch];
-#pragma unroll
-                for (int k = 0; k < kBatch; ++k) {
-                    const int i = i0 + k * sp.nparts;
-                    node[k] = emo::kNone;
-                    if (i < ne) {
-                        node[k] = emo_lds_u32(sta + (unsigned)i * rec_bytes);
-                        if (node[k] != emo::kNone && act0) emo_ldg_pair(spill_lane + (q0 + i) * ptile, es0[k], es1[k]);
-                    }
-                }
-#pragma unroll
-                for (int k = 0; k < kBatch; ++k) {
-                    const int i = i0 + k * sp.nparts;
-                    if (node[k] != emo::kNone && act0) {
-                        long long q0v, q1v;
-                        emo_lds_pair(sta + sp.off_q + ((unsigned)i * ptile + 2u * (unsigned)pair) * 8u, q0v, q1v);
-                        const long long ls0 = T0 - q0v, ls1 = T1 - q1v;
-                        const long long s0 = ls0 - es0[k], s1 = ls1 - es1[k];
-                        if (ls_lane) {
-                            long long *dst = emo_row_ptr(ls_lane, node[k], ldo8);
-                            if (vec_out) {
-                                emo_stg_pair(dst, ls0, ls1);
-                            } else {
-                                dst[0] = ls0;
-                                if (act1) dst[1] = ls1;
-                            }
-                        }
-                        if (sl_lane) {
-                            long long *dst = emo_row_ptr(sl_lane, node[k], ldo8);
-                            if (vec_out) {
-                                emo_stg_pair(dst, s0, s1);
-                            } else {
-                                dst[0] = s0;
-                                if (act1) dst[1] = s1;
-                            }
-                        }
-                        if (sp.want_sums) {
-                            sum0 += s0;
-                            sum1 += s1;
-                            cnt0 += (s0 == 0);
-                            cnt1 += (s1 == 0);
-                        }
-                    }
-                }
-            }
-            __syncwarp();
-            if (lane == 0) emo_mbar_arrive(bar_empty + 8 * s);
-        }
-        part_out[(size_t)ot * 4] = sum0;
-        part_out[(size_t)ot * 4 + 1] = sum1;
-        part_out[(size_t)ot * 4 + 2] = cnt0;
-        part_out[(size_t)ot * 4 + 3] = cnt1;
     } else {
-        // --------------------------------------------------------------------------- chain warps
-        const int group = warp / lanes, chain = warp - group * lanes;
-        const int col = group * 64 + 2 * lane;
-        const int64_t b = b0 + col;
-        const bool act0 = b < p.B, act1 = b + 1 < p.B;
+        // --------------------------------------------------------------------------- consumers
         const unsigned slotbar_base = smem0 + (unsigned)group * p.slots * kSlotStride;
         const unsigned lane16 = 16u + (unsigned)lane * 16u;
-        const unsigned d_rec = (unsigned)lanes * rec_bytes, d_d = (unsigned)lanes * ptile * 4u, d_q = (unsigned)lanes * ptile * 8u;
-        const unsigned ldes8 = (unsigned)p.ldes * 8u;     // pitches below 2^28 elements
+        const long long T0 = (BWD && act0) ? p.makespan[b] : 0, T1 = (BWD && act1) ? p.makespan[b + 1] : 0;
+        const unsigned d_rec = (unsigned)lanes * p.rec_bytes, d_lvl = (unsigned)lanes * ptile;
+        const unsigned en_off = 32u + (unsigned)p.Lp * 4u;
+        const unsigned ldes8 = (unsigned)p.ldes * 8u, ldo8 = (unsigned)p.ldo * 8u;     // pitches below 2^28 elements
         long long *const es_lane = (!BWD && p.ES) ? reinterpret_cast<long long *>(p.ES) + b : nullptr;
         // forward: this thread's column pair inside the spill tile it belongs to
         long long *const spill_lane = (!BWD && p.spill)
             ? reinterpret_cast<long long *>(p.spill) + (size_t)(b / p.spill_ptile) * p.spill_rows * p.spill_ptile + (b % p.spill_ptile)
             : nullptr;
         const unsigned spill8 = (unsigned)p.spill_ptile * 8u;
-        const bool store_es = es_lane != nullptr && act0, store_spill = spill_lane != nullptr && act0;
-        const bool vec_es = sp.vec_es && act1;
+        long long *const ls_lane = p.LS ? reinterpret_cast<long long *>(p.LS) + b : nullptr;
+        long long *const sl_lane = p.slack ? reinterpret_cast<long long *>(p.slack) + b : nullptr;
+        const bool store_es = EXTRA && es_lane != nullptr && act0, store_spill = spill_lane != nullptr && act0;
+        const bool vec_es = sp.vec_es && act1, vec_out = (!EXTRA || sp.vec_out) && act1;
+        const bool want_sums = EXTRA && sp.want_sums != 0;
         const int gthreads = lanes * 32;
         volatile int *my_abort = abort_flag + group;
         bool dead = false;
-        long long h0 = 0, h1 = 0, acc0 = 0, acc1 = 0;      // acc: running makespan (forward)
-        unsigned q_a = 0;
 
         // one node for both policies of this thread
         auto process = [&](const EmoFetched &f) {
             const uint4 e = f.e;
             if (!(e.y & emo::kValid) || dead) return;
+            if (!BWD) {
+                ea0 += f.g0;
+                ea1 += f.g1;
+            }
             if (!(e.y & emo::kRegPred)) { h0 = 0; h1 = 0; }
             const unsigned np = (e.y >> emo::kNPredShift) & 7u;
-            if (np) {
+            if (np && !BWD) {
+                // forward programs have few slot operands: a plain loop keeps the code small
+                unsigned ops = e.z, par = e.y >> emo::kOperandParityShift;
+                for (unsigned k = 0; k < np; ++k) {
+                    if (k == 4) ops = e.w;
+                    const unsigned bar = slotbar_base + (ops & 255u) * kSlotStride;
+                    if (!emo_slot_wait(bar, par & 1u, my_abort)) {
+                        *my_abort = 1;
+                        dead = true;
+                        return;
+                    }
+                    long long x0, x1;
+                    emo_lds_pair(bar + lane16, x0, x1);
+                    ops >>= 8;
+                    par >>= 1;
+                    h0 = emo_max64(h0, x0);
+                    h1 = emo_max64(h1, x1);
+                }
+            }
+            if (np && BWD) {
                 // all operands at once: poll every slot's barrier, then load every value, then take
                 // the maxima - the loads overlap instead of queuing behind one another
                 unsigned bars[emo::kMaxSlotPreds];
@@ -487,7 +395,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_pair(StagedParams sp)
 #pragma unroll
                     for (int k = 0; k < emo::kMaxSlotPreds; ++k) {
                         if (k < (int)np && !dead) {
-                            if (!emo_mbar_wait(bars[k], (e.y >> (emo::kOperandParityShift + k)) & 1u, my_abort)) {
+                            if (!emo_slot_wait(bars[k], (e.y >> (emo::kOperandParityShift + k)) & 1u, my_abort)) {
                                 *my_abort = 1;
                                 dead = true;
                             }
@@ -517,7 +425,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_pair(StagedParams sp)
                         dst[0] = h0;
                     }
                 }
-                if (store_es) {
+                if (EXTRA && store_es) {
                     long long *dst = emo_row_ptr(es_lane, f.node, ldes8);
                     if (vec_es) {
                         emo_stg_pair(dst, h0, h1);
@@ -540,83 +448,119 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_pair(StagedParams sp)
                     acc0 = emo_max64(acc0, h0);
                     acc1 = emo_max64(acc1, h1);
                 }
-            } else if (e.x != emo::kNone) {
-                emo_sts_pair(q_a, h0, h1);          // Q_v for the output warps
+            } else if (e.x != emo::kNone && act0) {
+                const long long ls0 = T0 - h0, ls1 = T1 - h1;
+                const long long s0 = ls0 - f.es0, s1 = ls1 - f.es1;
+                if (EXTRA && ls_lane) {
+                    long long *dst = emo_row_ptr(ls_lane, e.x, ldo8);
+                    if (vec_out) {
+                        emo_stg_pair(dst, ls0, ls1);
+                    } else {
+                        dst[0] = ls0;
+                        if (act1) dst[1] = ls1;
+                    }
+                }
+                if (sl_lane) {
+                    long long *dst = emo_row_ptr(sl_lane, e.x, ldo8);
+                    if (vec_out) {
+                        emo_stg_pair(dst, s0, s1);
+                    } else {
+                        dst[0] = s0;
+                        if (act1) dst[1] = s1;
+                    }
+                }
+                if (want_sums) {
+                    acc0 += s0;
+                    acc1 += s1;
+                    nc0 += (s0 == 0);
+                    nc1 += (s1 == 0);
+                }
             }
         };
 
         for (int c = 0; c < n_chunks; ++c) {
             const int s = c % nstages;
-            const bool ok = emo_mbar_wait(bar_ready + 8 * s, (c / nstages) & 1, abort_all);
+            const bool ok = emo_mbar_wait(bar0 + 8 * s, (c / nstages) & 1);
             // the warps of a group must take the same decision: one flag, read after a barrier
-            if (!ok || dead || (chain == 0 && *abort_all)) *my_abort = 1;
-            if (lanes > 1) emo_group_barrier(group + 1, gthreads);
-            if (*my_abort) {
-                if (lane == 0) {
-                    *abort_all = 1;
-                    if (p.status) atomicMin(p.status, -8);
-                }
-                break;
-            }
+            if (!ok || dead || (chain == 0 && abort_flag[groups])) *my_abort = 1;
             const unsigned sta = stage0 + (unsigned)s * stage_bytes;
             const int ns = min(sc, steps - c * sc);
-            unsigned rec_a = sta + (unsigned)chain * rec_bytes;
-            unsigned d_a = sta + sp.off_d + ((unsigned)chain * ptile + col) * 4u;
-            q_a = sta + sp.off_q + ((unsigned)chain * ptile + col) * 8u;
+            if (base_col >= 0 && chain == 0 && (base_col >> 6) == group) {
+                // the virtual all-max column: overwrite its byte in every level row of this stage
+                const unsigned char top = (unsigned char)(p.L - 1);
+                for (int i = lane; i < ns * lanes; i += 32)
+                    emo_smem[sp.off_stage0 + (size_t)s * stage_bytes + sp.off_lvl + (size_t)i * ptile + (size_t)base_col] = top;
+                __syncwarp();
+            }
+            if (lanes > 1) emo_group_barrier(group + 1, gthreads);
+            if (*my_abort) {
+                if (lane == 0 && p.status) atomicMin(p.status, -8);
+                break;
+            }
+            unsigned rec_a = sta + (unsigned)chain * p.rec_bytes;
+            unsigned lvl_a = sta + sp.off_lvl + (unsigned)chain * ptile + col;
+            unsigned es_a = sta + sp.off_es + ((unsigned)chain * ptile + col) * 8u;
+            // everything a step reads from the stage is fetched one step ahead (one copy of the step
+            // body: a small hot loop matters more than the few register moves)
+            const unsigned d_es = d_lvl * 8u;
             EmoFetched cur, nxt;
-            emo_fetch(cur, rec_a, d_a, store_es);
+            emo_fetch<BWD>(cur, rec_a, lvl_a, es_a, en_off, store_es);
             for (int j = 0; j < ns; ++j) {
                 if (j && (j % emo::kSyncSteps) == 0 && lanes > 1) emo_group_barrier(group + 1, gthreads);
                 rec_a += d_rec;
-                d_a += d_d;
-                if (j + 1 < ns) emo_fetch(nxt, rec_a, d_a, store_es);
+                lvl_a += d_lvl;
+                es_a += d_es;
+                if (j + 1 < ns) emo_fetch<BWD>(nxt, rec_a, lvl_a, es_a, en_off, store_es);
                 process(cur);
-                if (BWD) q_a += d_q;
                 cur = nxt;
             }
             __syncwarp();
-            if (lane == 0) emo_mbar_arrive((BWD ? bar_done : bar_empty) + 8 * s);
+            if (lane == 0) emo_mbar_arrive(bar0 + 8 * (kMaxStages + s));
         }
-        part_chain[((size_t)warp * 32 + lane) * 2] = acc0;
-        part_chain[((size_t)warp * 32 + lane) * 2 + 1] = acc1;
     }
 
-    // combine per policy in a fixed order (run-to-run identical energies)
+    // combine the warps of a group in lane order (fixed order: run-to-run identical energy)
+    // per (group, chain, lane): {energy0 | sum0, energy1 | sum1, makespan0 | count0, makespan1 | count1}
+    if (!producer) {
+        long long *pd = reinterpret_cast<long long *>(part_base) + ((size_t)(group * lanes + chain) * 32 + lane) * 4;
+        if (!BWD) {
+            pd[0] = __double_as_longlong(ea0);
+            pd[1] = __double_as_longlong(ea1);
+            pd[2] = acc0;
+            pd[3] = acc1;
+        } else {
+            pd[0] = acc0;
+            pd[1] = acc1;
+            pd[2] = nc0;
+            pd[3] = nc1;
+        }
+    }
     __syncthreads();
-    if (role == 0) {
-        const int group = warp / lanes, chain = warp - group * lanes;
-        if (chain == 0) {
-            const int pair_g = group * 32 + lane;            // this thread's pair within the block
-            const int64_t b = b0 + 2 * pair_g;
-            const bool act0 = b < p.B, act1 = b + 1 < p.B;
-            const int col = 2 * pair_g;
-            if (!BWD) {
-                double e0 = 0.0, e1 = 0.0;
-                long long t0 = 0, t1 = 0;
-                for (int k = 0; k < lanes; ++k) {
-                    t0 = emo_max64(t0, part_chain[((size_t)(group * lanes + k) * 32 + lane) * 2]);
-                    t1 = emo_max64(t1, part_chain[((size_t)(group * lanes + k) * 32 + lane) * 2 + 1]);
-                }
-                for (int k = 0; k < sp.nparts; ++k) {
-                    e0 += __longlong_as_double(part_look[((size_t)k * pairs + pair_g) * 2]);
-                    e1 += __longlong_as_double(part_look[((size_t)k * pairs + pair_g) * 2 + 1]);
-                }
-                if (act0) { p.makespan[b] = t0; p.energy[b] = e0; }
-                if (act1) { p.makespan[b + 1] = t1; p.energy[b + 1] = e1; }
-                if (base_col == col) { if (p.base_T) *p.base_T = t0; if (p.base_E) *p.base_E = e0; }
-                if (base_col == col + 1) { if (p.base_T) *p.base_T = t1; if (p.base_E) *p.base_E = e1; }
-            } else if (sp.want_sums) {
-                long long s0 = 0, s1 = 0, c0 = 0, c1 = 0;
-                for (int k = 0; k < sp.nparts; ++k) {
-                    const long long *q = part_out + ((size_t)k * pairs + pair_g) * 4;
-                    s0 += q[0];
-                    s1 += q[1];
-                    c0 += q[2];
-                    c1 += q[3];
-                }
-                if (act0) { if (p.slack_sum) p.slack_sum[b] = s0; if (p.n_critical) p.n_critical[b] = (int32_t)c0; }
-                if (act1) { if (p.slack_sum) p.slack_sum[b + 1] = s1; if (p.n_critical) p.n_critical[b + 1] = (int32_t)c1; }
+    if (!producer && chain == 0) {
+        const long long *g0 = reinterpret_cast<const long long *>(part_base) + ((size_t)(group * lanes) * 32 + lane) * 4;
+        if (!BWD) {
+            double e0 = 0.0, e1 = 0.0;
+            long long t0 = 0, t1 = 0;
+            for (int k = 0; k < lanes; ++k) {
+                e0 += __longlong_as_double(g0[(size_t)k * 128]);
+                e1 += __longlong_as_double(g0[(size_t)k * 128 + 1]);
+                t0 = emo_max64(t0, g0[(size_t)k * 128 + 2]);
+                t1 = emo_max64(t1, g0[(size_t)k * 128 + 3]);
             }
+            if (act0) { p.makespan[b] = t0; p.energy[b] = e0; }
+            if (act1) { p.makespan[b + 1] = t1; p.energy[b + 1] = e1; }
+            if (base_col == col) { if (p.base_T) *p.base_T = t0; if (p.base_E) *p.base_E = e0; }
+            if (base_col == col + 1) { if (p.base_T) *p.base_T = t1; if (p.base_E) *p.base_E = e1; }
+        } else if (sp.want_sums) {
+            long long s0 = 0, s1 = 0, c0 = 0, c1 = 0;
+            for (int k = 0; k < lanes; ++k) {
+                s0 += g0[(size_t)k * 128];
+                s1 += g0[(size_t)k * 128 + 1];
+                c0 += g0[(size_t)k * 128 + 2];
+                c1 += g0[(size_t)k * 128 + 3];
+            }
+            if (act0) { if (p.slack_sum) p.slack_sum[b] = s0; if (p.n_critical) p.n_critical[b] = (int32_t)c0; }
+            if (act1) { if (p.slack_sum) p.slack_sum[b + 1] = s1; if (p.n_critical) p.n_critical[b + 1] = (int32_t)c1; }
         }
     }
 }

@@ -8,7 +8,7 @@ import numpy as np
 
 NONE = 0xFFFFFFFF
 VALID, REGPRED, WRITE, TERMINAL, AUX = 1, 2, 4, 8, 0x80
-SYNC_STEPS = 4      # the warps of a group meet at a barrier every SYNC_STEPS steps
+SYNC_STEPS = 8      # the warps of a group meet at a barrier every SYNC_STEPS steps
 
 
 def run(entries, rows, lat, Lp, L, slots, lvl, n, backward, ES_in=None, T_in=None):
