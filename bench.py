@@ -28,6 +28,17 @@ METRIC = "policy_edge_relaxations_per_s"
 UNIT = "relaxations/s"
 
 
+def measured_traffic(kernel: str):
+    """DRAM bytes per node x policy of a pass kernel, from the committed ncu summary
+    (profiles/dram_traffic.json, taken on a scaled-down case; traffic is proportional to n x B)."""
+    p = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if not os.path.exists(p):
+        return None
+    with open(p) as f:
+        d = json.load(f)
+    return d.get(kernel, {}).get("dram_bytes_per_node_policy")
+
+
 def measured_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -243,8 +254,10 @@ def main():
     alg_fwd = n * B * 1 + B * 16            # 1 B level in per node x policy, makespan + energy out
     dom_ms, dom_bytes = (bwd, alg_bwd) if dom_is_bwd else (fwd, alg_fwd)
     achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
+    per_unit = measured_traffic("backward" if dom_is_bwd else "forward")
+    traffic = None if per_unit is None else per_unit * n * B          # bytes per launch, scaled from the capture
     roofline = {"bound": "hbm", "kernel": "backward pass" if dom_is_bwd else "forward pass", "achieved": achieved,
-                "peak": peak, "peak_source": peak_kind, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                "peak": peak, "peak_source": peak_kind, "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
                 "kernel_ms": dom_ms, "fwd_ms": fwd, "bwd_ms": bwd}
     step_bytes = n * B * 9 + B * 28
     roofline_step = {"bound": "hbm", "algorithmic_bytes": step_bytes, "achieved": step_bytes / (ms_per_step * 1e-3) / 1e9,
