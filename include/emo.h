@@ -63,9 +63,10 @@ typedef struct emo_info {
     int32_t max_span;   /* largest v - pred(v) in the caller's numbering */
     int64_t T_worst;    /* makespan with every node at its slowest level */
     int64_t T_best;     /* makespan with every node at its fastest level */
-    int32_t lanes;      /* warps that cooperate on one group of 32 policies */
+    int32_t lanes;      /* warps that cooperate on one group of policies, forward program */
     int32_t steps_fwd, slots_fwd, aux_fwd;   /* forward program: steps, exchange slots, helper ops */
     int32_t steps_bwd, slots_bwd, aux_bwd;   /* backward program */
+    int32_t lanes_bwd;  /* cooperating warps of the backward program */
 } emo_info;
 
 /* Human-readable text for a status code (static storage). */

@@ -20,23 +20,39 @@ struct Op {
 
 // A node with more operands than one entry can name is split: helper ops take the maximum of up
 // to kMaxSlotPreds operands each (duration 0, no output), and the node reads the helpers.
-void add_with_helpers(std::vector<Op> &ops, int32_t node, std::vector<int32_t> preds, int &n_aux)
+// A node with more operands than kMaxOperands is split: helper ops take the maximum of a few
+// operands each (duration 0, no output) and the node reads the helpers.  The operands that are
+// ready earliest (smallest hop level) go into helpers, the latest one stays with the node, so the
+// helpers can run on other warps ahead of time and the node's own warp - typically a serial chain
+// such as the launch chain in the backward direction, whose every node waits for four kernels -
+// is left with a short step.
+void add_with_helpers(std::vector<Op> &ops, std::vector<int32_t> &hop, int32_t node, std::vector<int32_t> preds, int &n_aux)
 {
     std::sort(preds.begin(), preds.end());
     preds.erase(std::unique(preds.begin(), preds.end()), preds.end());
-    while ((int)preds.size() > kMaxSlotPreds) {
+    auto by_hop = [&](int32_t a, int32_t b) { return hop[a] != hop[b] ? hop[a] < hop[b] : a < b; };
+    std::sort(preds.begin(), preds.end(), by_hop);
+    while ((int)preds.size() > kMaxOperands) {
+        const int take = std::min<int>(kMaxOperands, (int)preds.size() - kMaxOperands + 1);
         Op h;
         h.node = -1;
-        h.preds.assign(preds.begin(), preds.begin() + kMaxSlotPreds);
-        preds.erase(preds.begin(), preds.begin() + kMaxSlotPreds);
-        preds.push_back((int32_t)ops.size());
+        h.preds.assign(preds.begin(), preds.begin() + take);
+        int32_t lvl = 0;
+        for (int32_t q : h.preds) lvl = std::max(lvl, hop[q] + 1);
+        preds.erase(preds.begin(), preds.begin() + take);
+        const int32_t id = (int32_t)ops.size();
         ops.push_back(std::move(h));
+        hop.push_back(lvl);
+        preds.insert(std::upper_bound(preds.begin(), preds.end(), id, by_hop), id);
         ++n_aux;
     }
+    int32_t lvl = 0;
+    for (int32_t q : preds) lvl = std::max(lvl, hop[q] + 1);
     Op o;
     o.node = node;
     o.preds = std::move(preds);
     ops.push_back(std::move(o));
+    hop.push_back(lvl);
 }
 
 }  // namespace
@@ -66,6 +82,8 @@ int compile_program(const HostGraph &g, const int64_t *lat, const double *energy
     std::vector<Op> ops;
     ops.reserve((size_t)n + 16);
     std::vector<int32_t> op_of_node((size_t)std::max(n, 1), -1);
+    std::vector<int32_t> op_hop;      // hop level of every op built so far
+    op_hop.reserve((size_t)n + 16);
     int n_aux = 0;
     // Bounds of every node's value over all policies (forward: completion time C_v; backward: the
     // longest tail Q_v), from the smallest and the largest entry of its duration row.  An operand
@@ -103,7 +121,7 @@ int compile_program(const HostGraph &g, const int64_t *lat, const double *energy
         dur_bounds(v, dlo, dhi);
         lbv[v] = lo_start + dlo;
         ubv[v] = hi_start + dhi;
-        add_with_helpers(ops, v, std::move(p), n_aux);
+        add_with_helpers(ops, op_hop, v, std::move(p), n_aux);
         op_of_node[v] = (int32_t)ops.size() - 1;
     };
     if (!backward) {
@@ -413,6 +431,28 @@ int compile_program(const HostGraph &g, const int64_t *lat, const double *energy
             en[1] = flags;
             en[2] = operands;
             en[3] = operands_hi;
+        }
+    }
+    // Runs of simple entries.  An entry is simple when its only operand is the warp's register and
+    // it neither writes a slot nor ends a path: the kernels handle a run of them in a tight loop
+    // without decoding flags.  Every simple entry carries the length of the run that starts at it
+    // (in the bits that name slots, unused here); a run stays inside one block of kSyncSteps steps
+    // and its entries agree on whether they read a level.
+    for (int w = 0; w < lanes; ++w) {
+        uint32_t next_run = 0, next_mask = 0;
+        for (int32_t s = S - 1; s >= 0; --s) {
+            uint32_t &fl = out.entries[((size_t)s * lanes + w) * kEntryWords + 1];
+            const bool simple = (fl & kValid) && (fl & kRegPred) && !(fl & (kWriteSlot | kTerminal | kAux)) &&
+                                ((fl >> kNPredShift) & 7u) == 0;
+            uint32_t run = 0;
+            const uint32_t mask = (fl >> kMaskShift) & 255u;
+            if (simple) {
+                run = 1;
+                if ((s + 1) % kSyncSteps != 0 && next_run > 0 && next_mask == mask) run = next_run + 1;
+                fl |= kSimple | (run << kRunShift);
+            }
+            next_run = run;
+            next_mask = mask;
         }
     }
     return EMO_OK;

@@ -17,6 +17,7 @@ namespace emo {
 
 constexpr uint32_t kNone = 0xFFFFFFFFu;
 constexpr int kMaxSlotPreds = 6;      // slot operands one entry can name
+constexpr int kMaxOperands = 6;       // operands per op; a node with more gets helper ops (3 was measured slower)
 constexpr int kMaxSlots = 250;        // exchange slots per policy group (8-bit ids)
 constexpr int kMaxLanes = 32;
 
@@ -31,6 +32,8 @@ constexpr int kMaskShift = 8;         // bits 8..15: mask applied to the level b
 constexpr int kOutShift = 16;         // bits 16..23: slot written
 constexpr int kOutParityShift = 24;   // bit 24: phase parity of the value written
 constexpr int kOperandParityShift = 25;   // bits 25..30: phase parity of each operand's value
+constexpr uint32_t kSimple = 0x80000000u;   // bit 31: simple entry (register operand only, no slot written, not terminal)
+constexpr int kRunShift = 16;         // simple entries: bits 16..19 = length of the run of simple entries starting here
 constexpr int kSyncSteps = 8;         // the warps of a group meet at a barrier every kSyncSteps steps
 
 struct Program {

@@ -100,20 +100,6 @@ __int128 host_longest(const HostGraph &h, F dur)
 
 size_t lvl_area(const emo_graph *g) { return round_up((size_t)std::max(g->h.rows, 1) * 16, 256); }
 
-// lanes from the graph's shape: nodes per hop level plus a little spare capacity
-int pick_lanes_for(const HostGraph &h)
-{
-    std::vector<int32_t> hop((size_t)std::max(h.n, 1), 0);
-    int32_t depth = 0;
-    for (int32_t v = 0; v < h.n; ++v) {
-        int32_t a = 0;
-        for (int64_t e = h.row_ptr[v]; e < h.row_ptr[v + 1]; ++e) a = std::max(a, hop[h.col[e]] + 1);
-        hop[v] = a;
-        depth = std::max(depth, a + 1);
-    }
-    return pick_lanes(h.n, depth);
-}
-
 struct LaunchShape {
     int groups, grid, threads;
     size_t smem;
@@ -406,9 +392,9 @@ int emo_graph_load(int32_t n, const int64_t *row_ptr, const int32_t *col, const 
         std::string err;
         // backward first: the forward entries name the row of the backward program that will read
         // the node's earliest start
-        if (lanes <= 0) lanes = pick_lanes_for(h);
+        // (each direction picks its own number of lanes from its ops and depth unless one is forced)
         int rc = compile_program(h, lat, energy, true, lanes, look, nullptr, g->bwd, err);
-        if (rc == EMO_OK) rc = compile_program(h, lat, energy, false, g->bwd.lanes, look, &g->bwd.pos_of_node, g->fwd, err);
+        if (rc == EMO_OK) rc = compile_program(h, lat, energy, false, lanes, look, &g->bwd.pos_of_node, g->fwd, err);
         if (rc != EMO_OK) { delete g; return rc; }
         std::vector<int32_t> hop((size_t)std::max(n, 1), 0);
         int32_t depth = 0;
@@ -463,6 +449,7 @@ int emo_graph_info(const emo_graph *g, emo_info *info)
     info->T_worst = g->h.T_worst;
     info->T_best = g->h.T_best;
     info->lanes = g->fwd.lanes;
+    info->lanes_bwd = g->bwd.lanes;
     info->steps_fwd = g->fwd.steps;
     info->slots_fwd = g->fwd.slots;
     info->aux_fwd = g->fwd.aux;

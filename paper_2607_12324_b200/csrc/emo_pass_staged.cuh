@@ -505,14 +505,62 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_pair(StagedParams sp)
             const unsigned d_es = d_lvl * 8u;
             EmoFetched cur, nxt;
             emo_fetch<BWD>(cur, rec_a, lvl_a, es_a, en_off, store_es);
-            for (int j = 0; j < ns; ++j) {
+            int j = 0;
+            while (j < ns) {
                 if (j && (j % emo::kSyncSteps) == 0 && lanes > 1) emo_group_barrier(group + 1, gthreads);
+                if (!EXTRA && !BWD && (cur.e.y & emo::kSimple) && !dead) {
+                    // a run of simple nodes: h += duration, nothing else to decide
+                    const int run = (int)((cur.e.y >> emo::kRunShift) & 15u);
+                    const unsigned m = (cur.e.y >> emo::kMaskShift) & 255u;
+                    for (int k = 0; k < run; ++k) {
+                        const unsigned row = emo_lds_u32(rec_a);
+                        const unsigned lv2 = emo_lds_u16(lvl_a);
+                        const unsigned l0 = lv2 & m, l1 = (lv2 >> 8) & m;
+                        const unsigned d0 = emo_lds_u32(rec_a + 32u + l0 * 4u), d1 = emo_lds_u32(rec_a + 32u + l1 * 4u);
+                        if (!BWD) {
+                            const double g0 = emo_lds_f64(rec_a + en_off + l0 * 8u), g1 = emo_lds_f64(rec_a + en_off + l1 * 8u);
+                            if (store_spill) {
+                                long long *dst = emo_row_ptr(spill_lane, row, spill8);
+                                if (act1) {
+                                    emo_stg_pair(dst, h0, h1);
+                                } else {
+                                    dst[0] = h0;
+                                }
+                            }
+                            ea0 += g0;
+                            ea1 += g1;
+                            h0 = emo_add_dur(h0, d0);
+                            h1 = emo_add_dur(h1, d1);
+                        } else {
+                            long long es0, es1;
+                            emo_lds_pair(es_a, es0, es1);
+                            h0 = emo_add_dur(h0, d0);
+                            h1 = emo_add_dur(h1, d1);
+                            if (act0 && sl_lane) {
+                                long long *dst = emo_row_ptr(sl_lane, row, ldo8);
+                                const long long s0 = T0 - h0 - es0, s1 = T1 - h1 - es1;
+                                if (act1) {
+                                    emo_stg_pair(dst, s0, s1);
+                                } else {
+                                    dst[0] = s0;
+                                }
+                            }
+                        }
+                        rec_a += d_rec;
+                        lvl_a += d_lvl;
+                        es_a += d_es;
+                    }
+                    j += run;
+                    if (j < ns) emo_fetch<BWD>(cur, rec_a, lvl_a, es_a, en_off, store_es);
+                    continue;
+                }
                 rec_a += d_rec;
                 lvl_a += d_lvl;
                 es_a += d_es;
                 if (j + 1 < ns) emo_fetch<BWD>(nxt, rec_a, lvl_a, es_a, en_off, store_es);
                 process(cur);
                 cur = nxt;
+                ++j;
             }
             __syncwarp();
             if (lane == 0) emo_mbar_arrive(bar0 + 8 * (kMaxStages + s));

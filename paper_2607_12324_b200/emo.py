@@ -49,7 +49,8 @@ class emo_info(ctypes.Structure):
                 ("depth", ctypes.c_int32), ("max_span", ctypes.c_int32), ("T_worst", ctypes.c_int64),
                 ("T_best", ctypes.c_int64), ("lanes", ctypes.c_int32),
                 ("steps_fwd", ctypes.c_int32), ("slots_fwd", ctypes.c_int32), ("aux_fwd", ctypes.c_int32),
-                ("steps_bwd", ctypes.c_int32), ("slots_bwd", ctypes.c_int32), ("aux_bwd", ctypes.c_int32)]
+                ("steps_bwd", ctypes.c_int32), ("slots_bwd", ctypes.c_int32), ("aux_bwd", ctypes.c_int32),
+                ("lanes_bwd", ctypes.c_int32)]
 
 
 _lib = None

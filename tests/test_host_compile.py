@@ -56,7 +56,6 @@ def check_programs(emo, oracle_mod, g, lv, flags=0, group_of=None):
     assert np.array_equal(f["T"], r["makespan"])
     assert np.array_equal(f["ES"], r["ES"])
     lanes_b, steps_b, slots_b, Lp_b, ent_b, rows_b, lat_b = emo.emo_graph_program(h, 1)
-    assert lanes_b == lanes
     b = PE.run(ent_b, rows_b, lat_b, Lp_b, g.L, slots_b, lv, g.n, True, ES_in=f["ES"], T_in=f["T"])
     assert (b["seen"] == 1).all()
     # forward entries address the row of the backward program that handles the same node
@@ -67,6 +66,22 @@ def check_programs(emo, oracle_mod, g, lv, flags=0, group_of=None):
                 pos_b[int(ent_b[t, w, 4])] = t * lanes_b + w
     assert all(pos_b[node] == row for node, row in f["main_rows"])
     assert all(node == row for node, row in b["main_rows"])
+    # runs of simple entries: the stored length counts the simple entries that follow in the same
+    # column, never crosses a block of SYNC_STEPS steps and keeps one level mask
+    for ent_x in (ent, ent_b):
+        fl = ent_x[:, :, 1].astype(np.int64)
+        S_, W_ = fl.shape
+        for w in range(W_):
+            for t in range(S_):
+                f = int(fl[t, w])
+                simple = (f & 1) and (f & 2) and not (f & (4 | 8 | 0x80)) and ((f >> 4) & 7) == 0
+                assert bool(f >> 31) == bool(simple)
+                if simple:
+                    run = (f >> 16) & 15
+                    assert 1 <= run <= PE.SYNC_STEPS - (t % PE.SYNC_STEPS)
+                    for k in range(1, run):
+                        g2 = int(fl[t + k, w])
+                        assert (g2 >> 31) and ((g2 >> 16) & 15) == run - k and ((g2 >> 8) & 255) == ((f >> 8) & 255)
     assert np.array_equal(b["LS"], r["LS"])
     assert np.array_equal(b["slack"], r["slack"])
     h.free()
