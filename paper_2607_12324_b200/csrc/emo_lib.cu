@@ -11,6 +11,7 @@
 #include "../../include/emo.h"
 #include "emo_compile.h"
 #include "emo_kernels.cuh"
+#include "emo_pass_ilp.cuh"
 #include "emo_pass_staged.cuh"
 
 using namespace emo;
@@ -21,10 +22,21 @@ struct DevProgram {
     int rec_bytes = 0;
 };
 
+// The same program in the layout of emo_pass_ilp (see that file), padded to whole stages.
+struct DevProgramIlp {
+    unsigned char *ent = nullptr;   // [Qp][16]
+    unsigned char *node = nullptr;  // [Qp][4]
+    unsigned char *tab = nullptr;   // [Qp][tab_entry]
+    uint32_t *rows = nullptr;       // [Qp]
+    int steps_pad = 0;
+    unsigned tab_entry = 0;
+};
+
 struct emo_graph {
     HostGraph h;
     Program fwd, bwd;
     DevProgram dfwd, dbwd;
+    DevProgramIlp ifwd, ibwd;       // only for programs of at most kIlpMaxLanes lanes
     bool host_only = false;
     int device = 0;
     int sm_count = 148;
@@ -74,6 +86,61 @@ int upload_program(const Program &p, DevProgram &d)
     int rc = upload(&d.rec, rec.data(), rec.size());
     if (rc) return rc;
     return upload(&d.rows, p.rows.data(), p.rows.size() * sizeof(uint32_t));
+}
+
+int upload_program_ilp(const Program &p, DevProgramIlp &d)
+{
+    const bool fwd = !p.energy.empty();
+    const size_t Q = (size_t)p.steps * p.lanes;
+    d.steps_pad = (p.steps + kIlpStepPad - 1) / kIlpStepPad * kIlpStepPad;
+    const size_t Qp = (size_t)d.steps_pad * p.lanes;
+    d.tab_entry = (unsigned)p.Lp * (fwd ? 16u : 4u);
+    std::vector<uint32_t> ent(Qp * 4), node(Qp, kNone), rows(Qp, kNone);
+    std::vector<unsigned char> tab(Qp * d.tab_entry, 0);
+    for (size_t q = 0; q < Qp; ++q) {
+        uint32_t *w = &ent[q * 4];
+        w[0] = kNone;
+        w[1] = kIlpNoSlot;
+        w[2] = 0xFFFFFFFFu;      // idle: the lane keeps its value
+        w[3] = 0;
+        if (q >= Q) continue;
+        const uint32_t *en = &p.entries[q * kEntryWords];
+        const uint32_t fl = en[1];
+        if (!(fl & kValid)) continue;
+        uint32_t op[6];
+        for (int i = 0; i < 6; ++i) op[i] = ((i < 4 ? en[2] : en[3]) >> (8 * (i & 3))) & 255u;
+        const uint32_t np = (fl >> kNPredShift) & 7u;
+        const uint32_t out = (fl & kWriteSlot) ? ((fl >> kOutShift) & 255u) : kIlpNoSlot;
+        w[0] = en[0];
+        w[1] = out | (np << kIlpNpShift) | ((fl & kTerminal) ? kIlpTerminal : 0u) | (op[0] << kIlpOp0Shift) | (op[1] << (kIlpOp0Shift + 8));
+        w[2] = (fl & kRegPred) ? 0xFFFFFFFFu : 0u;
+        w[3] = op[2] | (op[3] << 8) | (op[4] << 16) | (op[5] << 24);
+        node[q] = en[4];
+        rows[q] = p.rows[q];
+        // a node that ignores the policy (level mask 0) gets its level-0 value at every index:
+        // the kernel indexes the row with whatever byte it finds
+        const bool uses_level = ((fl >> kMaskShift) & 255u) != 0;
+        for (int l = 0; l < p.Lp; ++l) {
+            const size_t src = q * p.Lp + (uses_level ? l : 0);
+            unsigned char *t = tab.data() + q * d.tab_entry + (size_t)l * (fwd ? 16 : 4);
+            std::memcpy(t, &p.lat[src], 4);
+            if (fwd) std::memcpy(t + 8, &p.energy[src], 8);
+        }
+    }
+    int rc = upload(&d.ent, ent.data(), ent.size() * 4);
+    if (rc == EMO_OK) rc = upload(&d.node, node.data(), node.size() * 4);
+    if (rc == EMO_OK) rc = upload(&d.tab, tab.data(), tab.size());
+    if (rc == EMO_OK) rc = upload(&d.rows, rows.data(), rows.size() * 4);
+    return rc;
+}
+
+void free_program_ilp(DevProgramIlp &d)
+{
+    if (d.ent) cudaFree(d.ent);
+    if (d.node) cudaFree(d.node);
+    if (d.tab) cudaFree(d.tab);
+    if (d.rows) cudaFree(d.rows);
+    d = DevProgramIlp();
 }
 
 void free_program(DevProgram &d)
@@ -168,14 +235,66 @@ bool staged_shape(const emo_graph *g, const Program &p, int rec_bytes, bool back
     return false;
 }
 
+// Shape of the kernel that keeps the schedule lanes inside one thread: consumer warps of 32 policies,
+// one more warp produces; private exchange slots first, then the stage ring.  Stages of few steps
+// are tried too: the backward pass stages 8 bytes of earliest start per policy and entry, and many
+// short stages keep more copies in flight than two long ones.  Returns false when it cannot be used.
+bool ilp_shape(const emo_graph *g, const Program &p, bool backward, int64_t NB, LaunchShape &s, StagedParams &sp)
+{
+    if (p.steps == 0 || !g->smem_optin || !g->ifwd.ent || !g->ibwd.ent) return false;
+    const size_t rec_bytes = 16 + 4 + (size_t)p.Lp * (backward ? 4 : 16);     // entry, node id, table row
+    const int64_t n_warps = (NB + 31) / 32;
+    const int64_t want = (n_warps + g->sm_count - 1) / g->sm_count;
+    int G = (int)std::max<int64_t>(1, std::min<int64_t>(kIlpMaxWarps, want));
+    const size_t budget = g->smem_optin;
+    static const int kTry[10][2] = {{16, 4}, {16, 3}, {8, 4}, {8, 3}, {4, 6}, {4, 5}, {4, 4}, {8, 2}, {4, 3}, {4, 2}};
+    for (; G >= 1; --G) {
+        const size_t P = 32 * (size_t)G;
+        const size_t slot_bytes = round_up((size_t)p.slots * P * 8, 128);
+        for (int t = 0; t < 10; ++t) {
+            const int sc = kTry[t][0], stages = kTry[t][1];
+            const size_t ne = (size_t)sc * p.lanes;
+            if (ne > 32 * (size_t)kRowRegs || stages > kMaxStages) continue;
+            const size_t stage_bytes = round_up(ne * ((size_t)rec_bytes + P + (backward ? P * 8 : 0)), 128);
+            // behind the last stage: room for the look-ahead of its last step, which reads one step
+            // past the stage in every area (the widest is the earliest-start area)
+            const size_t pad = round_up((size_t)p.lanes * std::max<size_t>(P * 8, rec_bytes), 128);
+            const size_t total = slot_bytes + 256 + stages * stage_bytes + pad;
+            if (total > budget) continue;
+            sp.sc = sc;
+            sp.stages = stages;
+            sp.ptile = (int)P;
+            sp.off_lvl = (unsigned)(ne * rec_bytes);
+            sp.off_es = sp.off_lvl + (unsigned)(ne * P);
+            sp.stage_bytes = (unsigned)stage_bytes;
+            sp.off_part = 0;
+            sp.off_bar = (unsigned)slot_bytes;
+            sp.off_stage0 = (unsigned)(slot_bytes + 256);
+            s.groups = G;
+            s.grid = (int)((n_warps + G - 1) / G);
+            s.threads = (G + 1) * 32;
+            s.smem = total;
+            return true;
+        }
+    }
+    return false;
+}
+
 // How the two passes of one call will run: both staged (earliest starts travel through the tiled
 // spill) or both with the plain kernels (through an [n][ldes] array).
 struct PassPlan {
     bool staged = false;
+    bool ilp = false;         // staged, with the schedule lanes inside one thread
     LaunchShape sf, sb;       // forward / backward launch shapes
     StagedParams pf, pb;
     size_t spill_bytes = 0;   // tiled spill: [tiles][rows of the backward program][backward tile]
 };
+
+// rows of one tile of the spill: the entries of the backward program (padded for the in-thread kernel)
+size_t spill_rows_of(const emo_graph *g, bool ilp)
+{
+    return (size_t)(ilp ? g->ibwd.steps_pad : g->bwd.steps) * g->bwd.lanes;
+}
 
 bool aligned16(const void *q) { return ((uintptr_t)q % 16) == 0; }
 
@@ -185,9 +304,11 @@ int make_plan(const emo_graph *g, int64_t B, bool want_base, bool need_bwd, cons
 {
     const int64_t big = (int64_t)1 << 28;
     const int64_t NBf = B + (want_base ? 1 : 0);
-    pl.staged = !(flags & EMO_F_NO_STAGING) && ldb % 16 == 0 && aligned16(lvl) && ldb < big && ldes_plain < big && ldo < big &&
-                staged_shape(g, g->fwd, g->dfwd.rec_bytes, false, NBf, pl.sf, pl.pf) &&
-                (!need_bwd || staged_shape(g, g->bwd, g->dbwd.rec_bytes, true, B, pl.sb, pl.pb));
+    const bool can_stage = !(flags & EMO_F_NO_STAGING) && ldb % 16 == 0 && aligned16(lvl) && ldb < big && ldes_plain < big && ldo < big;
+    pl.ilp = can_stage && !(flags & EMO_F_PAIR_KERNEL) && ilp_shape(g, g->fwd, false, NBf, pl.sf, pl.pf) &&
+             (!need_bwd || ilp_shape(g, g->bwd, true, B, pl.sb, pl.pb));
+    pl.staged = pl.ilp || (can_stage && staged_shape(g, g->fwd, g->dfwd.rec_bytes, false, NBf, pl.sf, pl.pf) &&
+                           (!need_bwd || staged_shape(g, g->bwd, g->dbwd.rec_bytes, true, B, pl.sb, pl.pb)));
     if (!pl.staged) {
         int rc = shape_for(g, g->fwd, NBf, pl.sf);
         if (rc == EMO_OK && need_bwd) rc = shape_for(g, g->bwd, B, pl.sb);
@@ -195,7 +316,7 @@ int make_plan(const emo_graph *g, int64_t B, bool want_base, bool need_bwd, cons
     }
     if (need_bwd) {
         const size_t tiles = ((size_t)B + pl.pb.ptile - 1) / pl.pb.ptile;
-        pl.spill_bytes = tiles * (size_t)g->bwd.steps * g->bwd.lanes * pl.pb.ptile * sizeof(int64_t);
+        pl.spill_bytes = tiles * spill_rows_of(g, pl.ilp) * pl.pb.ptile * sizeof(int64_t);
     }
     return EMO_OK;
 }
@@ -229,7 +350,7 @@ int launch_pass(const emo_graph *g, const PassPlan &pl, bool backward, int64_t B
     a.ES = ES;
     a.ldes = ldes;
     a.spill = spill;
-    a.spill_rows = (int64_t)g->bwd.steps * g->bwd.lanes;
+    a.spill_rows = (int64_t)spill_rows_of(g, pl.ilp);
     a.spill_ptile = pl.staged ? pl.pb.ptile : 64;
     a.LS = LS;
     a.slack = slack;
@@ -253,7 +374,61 @@ int launch_pass(const emo_graph *g, const PassPlan &pl, bool backward, int64_t B
         // lean instantiation when the call asks for nothing beyond the spill (forward) or the slack
         // matrix with 16-byte aligned rows (backward); register budget by block size
         const bool extra = backward ? (LS != nullptr || sp.want_sums || !sp.vec_out) : (ES != nullptr);
-        void (*kern)(StagedParams);
+        void (*kern)(StagedParams) = nullptr;
+        if (pl.ilp) {
+            const DevProgramIlp &di = backward ? g->ibwd : g->ifwd;
+            IlpParams ip;
+            const unsigned ne = (unsigned)sp.sc * (unsigned)p.lanes;
+            sp.p.steps = di.steps_pad;
+            sp.p.rows = di.rows;
+            ip.tab_entry = di.tab_entry;
+            ip.st.off_node = ne * 16u;
+            ip.st.off_tab = ip.st.off_node + ne * 4u;
+            int nb = 0;
+            auto bulk = [&](const void *src, unsigned per_entry, unsigned off, unsigned long long per_block) {
+                sp.bsrc[nb] = (const unsigned char *)src;
+                sp.bentry[nb] = per_entry;
+                sp.boff[nb] = off;
+                sp.bblock[nb] = per_block;
+                ++nb;
+            };
+            bulk(di.ent, 16, 0, 0);
+            if (!backward && ES) bulk(di.node, 4, ip.st.off_node, 0);
+            bulk(di.tab, di.tab_entry, ip.st.off_tab, 0);
+            if (backward) bulk(spill, (unsigned)sp.ptile * 8u, sp.off_es, (unsigned long long)a.spill_rows * sp.ptile * 8ull);
+            sp.nbulk = nb;
+            void (*kern_ilp)(IlpParams) = nullptr;
+#define EMO_PICK_W(W_)                                                                                         \
+    case W_:                                                                                                   \
+        kern_ilp = backward ? (extra ? emo_pass_ilp<true, true, W_> : emo_pass_ilp<true, false, W_>)               \
+                            : (extra ? emo_pass_ilp<false, true, W_> : emo_pass_ilp<false, false, W_>);            \
+        break
+            const bool extra_ilp = backward ? (LS != nullptr || sp.want_sums) : (ES != nullptr);
+            const bool extra = extra_ilp;
+            switch (p.lanes) {
+                EMO_PICK_W(1);
+                EMO_PICK_W(2);
+                EMO_PICK_W(3);
+                EMO_PICK_W(4);
+                EMO_PICK_W(5);
+                EMO_PICK_W(6);
+                EMO_PICK_W(7);
+                EMO_PICK_W(8);
+                default: return EMO_E_UNSUPPORTED;
+            }
+#undef EMO_PICK_W
+            ip.sp = sp;
+            EMO_CUDA(cudaFuncSetAttribute(kern_ilp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s.smem));
+            kern_ilp<<<s.grid, s.threads, s.smem, st>>>(ip);
+        } else {
+            sp.nbulk = 0;
+            sp.bsrc[sp.nbulk] = d.rec; sp.bentry[sp.nbulk] = (unsigned)d.rec_bytes; sp.boff[sp.nbulk] = 0; sp.bblock[sp.nbulk] = 0;
+            ++sp.nbulk;
+            if (backward) {
+                sp.bsrc[sp.nbulk] = (const unsigned char *)spill; sp.bentry[sp.nbulk] = (unsigned)sp.ptile * 8u; sp.boff[sp.nbulk] = sp.off_es;
+                sp.bblock[sp.nbulk] = (unsigned long long)a.spill_rows * sp.ptile * 8ull;
+                ++sp.nbulk;
+            }
 #define EMO_PICK(MAXT)                                                                                         \
     kern = backward ? (extra ? emo_pass_pair<true, true, MAXT> : emo_pass_pair<true, false, MAXT>)                 \
                     : (extra ? emo_pass_pair<false, true, MAXT> : emo_pass_pair<false, false, MAXT>)
@@ -263,6 +438,7 @@ int launch_pass(const emo_graph *g, const PassPlan &pl, bool backward, int64_t B
 #undef EMO_PICK
         EMO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s.smem));
         kern<<<s.grid, s.threads, s.smem, st>>>(sp);
+        }
     } else if (backward) {
         if (s.smem > 48 * 1024) EMO_CUDA(cudaFuncSetAttribute(emo_pass_plain<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s.smem));
         emo_pass_plain<true><<<s.grid, s.threads, s.smem, st>>>(a);
@@ -420,6 +596,10 @@ int emo_graph_load(int32_t n, const int64_t *row_ptr, const int32_t *col, const 
         g->smem_optin = prop.sharedMemPerBlockOptin;
         int rc = upload_program(g->fwd, g->dfwd);
         if (rc == EMO_OK) rc = upload_program(g->bwd, g->dbwd);
+        if (rc == EMO_OK && g->fwd.lanes <= kIlpMaxLanes && g->bwd.lanes <= kIlpMaxLanes) {
+            rc = upload_program_ilp(g->fwd, g->ifwd);
+            if (rc == EMO_OK) rc = upload_program_ilp(g->bwd, g->ibwd);
+        }
         if (rc != EMO_OK) { emo_graph_free(g); return rc; }
     }
     *out = g;
@@ -432,6 +612,8 @@ int emo_graph_free(emo_graph *g)
     if (!g->host_only) {
         free_program(g->dfwd);
         free_program(g->dbwd);
+        free_program_ilp(g->ifwd);
+        free_program_ilp(g->ibwd);
     }
     delete g;
     return EMO_OK;
@@ -486,9 +668,13 @@ size_t spill_need(const emo_graph *g, int64_t B)
     if (!g->host_only && B > 0) {
         LaunchShape s;
         StagedParams sp;
-        if (staged_shape(g, g->bwd, g->dbwd.rec_bytes, true, B, s, sp)) {
+        // either staged kernel may run (the call's flags decide): room for the wider tiling
+        for (int which = 0; which < 2; ++which) {
+            const bool ok = which ? staged_shape(g, g->bwd, g->dbwd.rec_bytes, true, B, s, sp)
+                                  : ilp_shape(g, g->bwd, true, B, s, sp);
+            if (!ok) continue;
             const size_t tiles = ((size_t)B + sp.ptile - 1) / sp.ptile;
-            tiled = tiles * (size_t)g->bwd.steps * g->bwd.lanes * sp.ptile * sizeof(int64_t);
+            tiled = std::max(tiled, tiles * spill_rows_of(g, which == 0) * sp.ptile * sizeof(int64_t));
         }
     }
     return round_up(std::max(plain, tiled), 256);

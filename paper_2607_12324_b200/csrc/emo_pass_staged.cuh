@@ -25,7 +25,8 @@
 #include "emo_compile.h"
 #include "emo_kernels.cuh"
 
-constexpr int kMaxStages = 4;
+constexpr int kMaxStages = 8;
+constexpr int kMaxBulk = 5;              // bulk copies per stage
 constexpr int kRowRegs = 8;             // a stage holds at most 32 * kRowRegs records
 constexpr int kProducerWarps = 1;       // warps that issue the copies (they share the level-row pieces)
 constexpr unsigned kSlotStride = 528;   // 8-byte mbarrier, 8 bytes unused, 32 lanes x 16 bytes
@@ -42,6 +43,13 @@ struct StagedParams {
     unsigned stage_bytes;      // bytes of one stage
     unsigned off_lvl, off_es;  // offsets inside a stage (records start at 0)
     unsigned off_part, off_bar, off_stage0;      // offsets inside dynamic shared memory
+    // the bulk copies that fill a stage besides the level rows: per copy its global source, the
+    // bytes one program entry takes in it, the offset of its area inside a stage and the distance
+    // between the sources of consecutive blocks (0: all blocks read the same array)
+    int nbulk;
+    const unsigned char *bsrc[kMaxBulk];
+    unsigned bentry[kMaxBulk], boff[kMaxBulk];
+    unsigned long long bblock[kMaxBulk];
 };
 
 __device__ __forceinline__ unsigned emo_smem_addr(const void *p)
@@ -201,6 +209,95 @@ __device__ __forceinline__ bool emo_slot_wait(unsigned bar, unsigned parity, vol
     return emo_slot_wait_slow(bar, parity, abort_flag);
 }
 
+// The producer warp: for every chunk of steps, the bulk copies the launch lists (program records,
+// backward: the earliest-start rows) and the level rows of the block's policy tile as 16-byte pieces; then
+// the arrivals that complete the stage's full barrier.  Waits for a free stage are bounded: on
+// failure the warp raises *abort_all and EMO_E_TIMEOUT and returns once its copies have landed.
+__device__ __forceinline__ void emo_produce(const StagedParams &sp, unsigned stage0, unsigned bar0, volatile int *abort_all,
+                                            int lane, int pw)
+{
+    const PassParams &p = sp.p;
+    const int steps = p.steps, nstages = sp.stages, sc = sp.sc, lanes = p.lanes, ptile = sp.ptile;
+    const int n_chunks = (steps + sc - 1) / sc;
+    const unsigned stage_bytes = sp.stage_bytes;
+    const int64_t b0 = (int64_t)blockIdx.x * ptile;
+    const int64_t lvl_left = p.ldb - b0;
+    const unsigned lvl_bytes = lvl_left > 0 ? (unsigned)min((int64_t)ptile, lvl_left) : 0u;
+    const int pieces = (int)(lvl_bytes >> 4);
+    const unsigned inv_pieces = pieces > 1 ? (unsigned)((0x100000000ULL + pieces - 1) / pieces) : 0u;
+    int issued = 0;
+    bool gave_up = false;
+    // The level-row indices of a chunk are loaded one chunk ahead, 32 per register, so that no
+    // copy waits on a dependent global load: entry i's row sits in lane i % 32 of rr[i / 32].
+    unsigned rr[kRowRegs], rr_next[kRowRegs];
+    auto load_rows = [&](int c, unsigned *dst) {
+        const int step0 = c * sc;
+        const int ne = (c < n_chunks) ? min(sc, steps - step0) * lanes : 0;
+        const size_t q0 = (size_t)step0 * lanes;
+#pragma unroll
+        for (int k = 0; k < kRowRegs; ++k) {
+            const int i = 32 * k + lane;
+            dst[k] = (i < ne) ? __ldg(p.rows + q0 + i) : emo::kNone;
+        }
+    };
+    load_rows(0, rr);
+    for (int c = 0; c < n_chunks; ++c) {
+        const int s = c % nstages;
+        load_rows(c + 1, rr_next);
+        if (c >= nstages) {
+            if (!emo_mbar_wait(bar0 + 8 * (kMaxStages + s), ((c / nstages) - 1) & 1)) {
+                if (lane == 0) {
+                    *abort_all = 1;
+                    if (p.status) atomicMin(p.status, -8);
+                }
+                gave_up = true;
+                break;
+            }
+        }
+        if (*abort_all) { gave_up = true; break; }      // the other producer warp gave up
+        issued = c + 1;
+        const int step0 = c * sc;
+        const int ne = min(sc, steps - step0) * lanes;
+        const size_t q0 = (size_t)step0 * lanes;
+        const unsigned sta = stage0 + (unsigned)s * stage_bytes;
+        const unsigned full = bar0 + 8 * s;
+        if (lane == 0 && pw == 0) {
+            unsigned total = 0;
+            for (int i = 0; i < sp.nbulk; ++i) total += (unsigned)ne * sp.bentry[i];
+            emo_mbar_expect_tx(full, total);
+            for (int i = 0; i < sp.nbulk; ++i)
+                emo_bulk_g2s(sta + sp.boff[i], sp.bsrc[i] + blockIdx.x * sp.bblock[i] + q0 * sp.bentry[i],
+                             (unsigned)ne * sp.bentry[i], full);
+        }
+        // level rows: 32 entries x `pieces` 16-byte pieces per register of row indices; the
+        // producer warps take alternate iterations
+        if (pieces) {
+#pragma unroll
+            for (int k = 0; k < kRowRegs; ++k) {
+                if (32 * k < ne) {
+                    for (int it = pw; it < pieces; it += kProducerWarps) {
+                        const unsigned t = (unsigned)lane + 32u * (unsigned)it;
+                        const unsigned e = pieces > 1 ? __umulhi(t, inv_pieces) : t;   // t / pieces (t < 2^16)
+                        const unsigned pc = t - e * (unsigned)pieces;
+                        const unsigned row = __shfl_sync(0xFFFFFFFFu, rr[k], e & 31);
+                        const int i = 32 * k + (int)e;
+                        if (i < ne && row != emo::kNone)
+                            emo_cp_async16(sta + sp.off_lvl + (unsigned)i * ptile + pc * 16u,
+                                           p.lvl + (size_t)row * p.ldb + b0 + pc * 16);
+                    }
+                }
+            }
+        }
+        emo_cp_async_arrive(full);
+#pragma unroll
+        for (int k = 0; k < kRowRegs; ++k) rr[k] = rr_next[k];
+    }
+    if (gave_up) {
+        // do not leave the block while copies into its shared memory may still be in flight
+        for (int c = max(0, issued - nstages); c < issued; ++c) (void)emo_mbar_wait(bar0 + 8 * (c % nstages), (c / nstages) & 1);
+    }
+}
+
 // EXTRA = false is the lean instantiation for the common call (forward: ES only into the spill;
 // backward: slack only, 16-byte aligned rows, no per-policy sums): the hot loop stays small, which
 // matters because all warps of the block share the instruction cache.
@@ -249,83 +346,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_pair(StagedParams sp)
     int nc0 = 0, nc1 = 0;
 
     if (producer) {
-        // ---------------------------------------------------------------------------- producer
-        const int64_t lvl_left = p.ldb - b0;
-        const unsigned lvl_bytes = lvl_left > 0 ? (unsigned)min((int64_t)ptile, lvl_left) : 0u;
-        const int pieces = (int)(lvl_bytes >> 4);
-        const unsigned inv_pieces = pieces > 1 ? (unsigned)((0x100000000ULL + pieces - 1) / pieces) : 0u;
-        const unsigned rec_bytes = (unsigned)p.rec_bytes;
-        // this block's tile of the spill: [spill_rows][ptile] (the backward kernel's own tile width)
-        const long long *spill_tile = BWD ? reinterpret_cast<const long long *>(p.spill) + (size_t)blockIdx.x * p.spill_rows * ptile : nullptr;
-        int issued = 0;
-        bool gave_up = false;
-        // The level-row indices of a chunk are loaded one chunk ahead, 32 per register, so that no
-        // copy waits on a dependent global load: entry i's row sits in lane i % 32 of rr[i / 32].
-        unsigned rr[kRowRegs], rr_next[kRowRegs];
-        auto load_rows = [&](int c, unsigned *dst) {
-            const int step0 = c * sc;
-            const int ne = (c < n_chunks) ? min(sc, steps - step0) * lanes : 0;
-            const size_t q0 = (size_t)step0 * lanes;
-#pragma unroll
-            for (int k = 0; k < kRowRegs; ++k) {
-                const int i = 32 * k + lane;
-                dst[k] = (i < ne) ? __ldg(p.rows + q0 + i) : emo::kNone;
-            }
-        };
-        load_rows(0, rr);
-        for (int c = 0; c < n_chunks; ++c) {
-            const int s = c % nstages;
-            load_rows(c + 1, rr_next);
-            if (c >= nstages) {
-                if (!emo_mbar_wait(bar0 + 8 * (kMaxStages + s), ((c / nstages) - 1) & 1)) {
-                    if (lane == 0) {
-                        abort_flag[groups] = 1;
-                        if (p.status) atomicMin(p.status, -8);
-                    }
-                    gave_up = true;
-                    break;
-                }
-            }
-            if (abort_flag[groups]) { gave_up = true; break; }      // the other producer warp gave up
-            issued = c + 1;
-            const int step0 = c * sc;
-            const int ne = min(sc, steps - step0) * lanes;
-            const size_t q0 = (size_t)step0 * lanes;
-            const unsigned sta = stage0 + (unsigned)s * stage_bytes;
-            const unsigned full = bar0 + 8 * s;
-            if (lane == 0 && pw == 0) {
-                const unsigned rb = (unsigned)ne * rec_bytes, eb = BWD ? (unsigned)ne * ptile * 8u : 0u;
-                emo_mbar_expect_tx(full, rb + eb);
-                emo_bulk_g2s(sta, p.rec + q0 * rec_bytes, rb, full);
-                if (BWD) emo_bulk_g2s(sta + sp.off_es, spill_tile + q0 * ptile, eb, full);
-            }
-            // level rows: 32 entries x `pieces` 16-byte pieces per register of row indices; the
-            // producer warps take alternate iterations
-            if (pieces) {
-#pragma unroll
-                for (int k = 0; k < kRowRegs; ++k) {
-                    if (32 * k < ne) {
-                        for (int it = pw; it < pieces; it += kProducerWarps) {
-                            const unsigned t = (unsigned)lane + 32u * (unsigned)it;
-                            const unsigned e = pieces > 1 ? __umulhi(t, inv_pieces) : t;   // t / pieces (t < 2^16)
-                            const unsigned pc = t - e * (unsigned)pieces;
-                            const unsigned row = __shfl_sync(0xFFFFFFFFu, rr[k], e & 31);
-                            const int i = 32 * k + (int)e;
-                            if (i < ne && row != emo::kNone)
-                                emo_cp_async16(sta + sp.off_lvl + (unsigned)i * ptile + pc * 16u,
-                                               p.lvl + (size_t)row * p.ldb + b0 + pc * 16);
-                        }
-                    }
-                }
-            }
-            emo_cp_async_arrive(full);
-#pragma unroll
-            for (int k = 0; k < kRowRegs; ++k) rr[k] = rr_next[k];
-        }
-        if (gave_up) {
-            // do not leave the block while copies into its shared memory may still be in flight
-            for (int c = max(0, issued - nstages); c < issued; ++c) (void)emo_mbar_wait(bar0 + 8 * (c % nstages), (c / nstages) & 1);
-        }
+        emo_produce(sp, stage0, bar0, abort_flag + groups, lane, pw);
     } else {
         // --------------------------------------------------------------------------- consumers
         const unsigned slotbar_base = smem0 + (unsigned)group * p.slots * kSlotStride;

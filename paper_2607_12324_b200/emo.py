@@ -21,6 +21,7 @@ EMO_E_NONFINITE, EMO_E_OOM, EMO_E_CUDA, EMO_E_TIMEOUT, EMO_E_UNSUPPORTED = -5, -
 EMO_F_HOST_ONLY = 0x1
 EMO_F_VALIDATE = 0x1
 EMO_F_NO_STAGING = 0x2
+EMO_F_PAIR_KERNEL = 0x4
 
 EXPORTS = [
     "emo_strerror", "emo_graph_load", "emo_graph_free", "emo_graph_info", "emo_workspace_bytes",
