@@ -158,6 +158,7 @@ def main():
     ap.add_argument("--sums", action="store_true", help="also produce per-policy slack sums and critical counts")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--flags", type=int, default=0, help="extra EMO_F_* load flags (lanes / look-ahead)")
+    ap.add_argument("--call-flags", type=int, default=0, help="EMO_F_* flags of the pass calls (kernel choice)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -203,7 +204,8 @@ def main():
     def step(events=None):
         if events is not None:
             emo.emo_set_pass_events(*events)
-        emo.emo_slack_batch(h, B, lv, ldb, None, None, slack, B, T, E, sums[0], sums[1], ws, status, T0=T0, E0=E0)
+        emo.emo_slack_batch(h, B, lv, ldb, None, None, slack, B, T, E, sums[0], sums[1], ws, status, T0=T0, E0=E0,
+                            flags=args.call_flags)
         if events is not None:
             emo.emo_set_pass_events(None, None, None, None)
         emo.emo_select(B, T, E, 0, sel[0:1], sel[1:2], selE, ws, target_dev=T0, delta_ppm=ppm)

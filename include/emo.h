@@ -51,7 +51,7 @@ extern "C" {
 /* flags of the evaluation calls */
 #define EMO_F_VALIDATE 0x1u        /* check every level < L first; EMO_E_RANGE goes to *status */
 #define EMO_F_NO_STAGING 0x2u      /* use the plain-load kernels instead of the staged ones */
-#define EMO_F_PAIR_KERNEL 0x4u     /* staged kernels: one warp per schedule lane even where one thread could carry all lanes */
+#define EMO_F_PAIR_KERNEL 0x4u     /* staged pass kernel with two policies per thread */
 
 typedef struct emo_graph emo_graph;
 

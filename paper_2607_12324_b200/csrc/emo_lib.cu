@@ -11,7 +11,7 @@
 #include "../../include/emo.h"
 #include "emo_compile.h"
 #include "emo_kernels.cuh"
-#include "emo_pass_ilp.cuh"
+#include "emo_pass_lane.cuh"
 #include "emo_pass_staged.cuh"
 
 using namespace emo;
@@ -22,10 +22,9 @@ struct DevProgram {
     int rec_bytes = 0;
 };
 
-// The same program in the layout of emo_pass_ilp (see that file), padded to whole stages.
-struct DevProgramIlp {
-    unsigned char *ent = nullptr;   // [Qp][16]
-    unsigned char *node = nullptr;  // [Qp][4]
+// The same program in the layout of emo_pass_lane (see emo_lane_layout.cuh), padded to whole stages.
+struct DevProgramLane {
+    unsigned char *ent = nullptr;   // [Qp][32]
     unsigned char *tab = nullptr;   // [Qp][tab_entry]
     uint32_t *rows = nullptr;       // [Qp]
     int steps_pad = 0;
@@ -36,7 +35,7 @@ struct emo_graph {
     HostGraph h;
     Program fwd, bwd;
     DevProgram dfwd, dbwd;
-    DevProgramIlp ifwd, ibwd;       // only for programs of at most kIlpMaxLanes lanes
+    DevProgramLane lfwd, lbwd;       // only for programs of at most kLaneMaxLanes lanes
     bool host_only = false;
     int device = 0;
     int sm_count = 148;
@@ -88,34 +87,36 @@ int upload_program(const Program &p, DevProgram &d)
     return upload(&d.rows, p.rows.data(), p.rows.size() * sizeof(uint32_t));
 }
 
-int upload_program_ilp(const Program &p, DevProgramIlp &d)
+int upload_program_lane(const Program &p, DevProgramLane &d)
 {
     const bool fwd = !p.energy.empty();
     const size_t Q = (size_t)p.steps * p.lanes;
-    d.steps_pad = (p.steps + kIlpStepPad - 1) / kIlpStepPad * kIlpStepPad;
+    d.steps_pad = (p.steps + kLaneStepPad - 1) / kLaneStepPad * kLaneStepPad;
     const size_t Qp = (size_t)d.steps_pad * p.lanes;
     d.tab_entry = (unsigned)p.Lp * (fwd ? 16u : 4u);
-    std::vector<uint32_t> ent(Qp * 4), node(Qp, kNone), rows(Qp, kNone);
+    std::vector<uint32_t> ent(Qp * 8, 0), rows(Qp, kNone);
     std::vector<unsigned char> tab(Qp * d.tab_entry, 0);
     for (size_t q = 0; q < Qp; ++q) {
-        uint32_t *w = &ent[q * 4];
+        uint32_t *w = &ent[q * 8];
         w[0] = kNone;
-        w[1] = kIlpNoSlot;
+        w[1] = kLaneNoSlot | kLaneIdle;
         w[2] = 0xFFFFFFFFu;      // idle: the lane keeps its value
-        w[3] = 0;
+        w[5] = kNone;
         if (q >= Q) continue;
         const uint32_t *en = &p.entries[q * kEntryWords];
         const uint32_t fl = en[1];
         if (!(fl & kValid)) continue;
-        uint32_t op[6];
-        for (int i = 0; i < 6; ++i) op[i] = ((i < 4 ? en[2] : en[3]) >> (8 * (i & 3))) & 255u;
         const uint32_t np = (fl >> kNPredShift) & 7u;
-        const uint32_t out = (fl & kWriteSlot) ? ((fl >> kOutShift) & 255u) : kIlpNoSlot;
+        const uint32_t out = (fl & kWriteSlot) ? ((fl >> kOutShift) & 255u) : kLaneNoSlot;
+        const uint32_t outpar = (fl & kWriteSlot) ? ((fl >> kOutParityShift) & 1u) : 0u;
+        const uint32_t oppar = (fl >> kOperandParityShift) & 63u;
         w[0] = en[0];
-        w[1] = out | (np << kIlpNpShift) | ((fl & kTerminal) ? kIlpTerminal : 0u) | (op[0] << kIlpOp0Shift) | (op[1] << (kIlpOp0Shift + 8));
+        w[1] = out | (np << kLaneNpShift) | ((fl & kTerminal) ? kLaneTerminal : 0u) | (outpar << kLaneOutParShift) | (oppar << kLaneOpParShift);
+        if (fwd && (fl & kSimple)) w[1] |= ((fl >> kRunShift) & 15u) << kLaneRunShift;
         w[2] = (fl & kRegPred) ? 0xFFFFFFFFu : 0u;
-        w[3] = op[2] | (op[3] << 8) | (op[4] << 16) | (op[5] << 24);
-        node[q] = en[4];
+        w[3] = en[2];
+        w[4] = en[3];
+        w[5] = en[4];
         rows[q] = p.rows[q];
         // a node that ignores the policy (level mask 0) gets its level-0 value at every index:
         // the kernel indexes the row with whatever byte it finds
@@ -128,19 +129,17 @@ int upload_program_ilp(const Program &p, DevProgramIlp &d)
         }
     }
     int rc = upload(&d.ent, ent.data(), ent.size() * 4);
-    if (rc == EMO_OK) rc = upload(&d.node, node.data(), node.size() * 4);
     if (rc == EMO_OK) rc = upload(&d.tab, tab.data(), tab.size());
     if (rc == EMO_OK) rc = upload(&d.rows, rows.data(), rows.size() * 4);
     return rc;
 }
 
-void free_program_ilp(DevProgramIlp &d)
+void free_program_lane(DevProgramLane &d)
 {
     if (d.ent) cudaFree(d.ent);
-    if (d.node) cudaFree(d.node);
     if (d.tab) cudaFree(d.tab);
     if (d.rows) cudaFree(d.rows);
-    d = DevProgramIlp();
+    d = DevProgramLane();
 }
 
 void free_program(DevProgram &d)
@@ -235,31 +234,32 @@ bool staged_shape(const emo_graph *g, const Program &p, int rec_bytes, bool back
     return false;
 }
 
-// Shape of the kernel that keeps the schedule lanes inside one thread: consumer warps of 32 policies,
-// one more warp produces; private exchange slots first, then the stage ring.  Stages of few steps
-// are tried too: the backward pass stages 8 bytes of earliest start per policy and entry, and many
-// short stages keep more copies in flight than two long ones.  Returns false when it cannot be used.
-bool ilp_shape(const emo_graph *g, const Program &p, bool backward, int64_t NB, LaunchShape &s, StagedParams &sp)
+// Shape of the kernel with one warp per schedule lane and one policy per thread: groups of 32
+// policies, one more warp produces; slot area, partial results, barriers, then the stage ring.
+bool lane_shape(const emo_graph *g, const Program &p, bool backward, int64_t NB, LaunchShape &s, StagedParams &sp)
 {
-    if (p.steps == 0 || !g->smem_optin || !g->ifwd.ent || !g->ibwd.ent) return false;
-    const size_t rec_bytes = 16 + 4 + (size_t)p.Lp * (backward ? 4 : 16);     // entry, node id, table row
-    const int64_t n_warps = (NB + 31) / 32;
-    const int64_t want = (n_warps + g->sm_count - 1) / g->sm_count;
-    int G = (int)std::max<int64_t>(1, std::min<int64_t>(kIlpMaxWarps, want));
+    if (p.steps == 0 || !g->smem_optin || !g->lfwd.ent || !g->lbwd.ent) return false;
+    const size_t rec_bytes = 32 + (size_t)p.Lp * (backward ? 4 : 16);     // entry and table row
+    const int64_t n_groups = (NB + 31) / 32;
+    const int gmax = std::min(31 / p.lanes, 15);
+    if (gmax < 1) return false;
+    const int64_t want = (n_groups + g->sm_count - 1) / g->sm_count;
+    int G = (int)std::max<int64_t>(1, std::min<int64_t>(gmax, want));
     const size_t budget = g->smem_optin;
     static const int kTry[10][2] = {{16, 4}, {16, 3}, {8, 4}, {8, 3}, {4, 6}, {4, 5}, {4, 4}, {8, 2}, {4, 3}, {4, 2}};
     for (; G >= 1; --G) {
         const size_t P = 32 * (size_t)G;
-        const size_t slot_bytes = round_up((size_t)p.slots * P * 8, 128);
+        const size_t slot_bytes = round_up((size_t)G * p.slots * kLaneSlotStride, 16);
+        const size_t part_bytes = (size_t)G * p.lanes * 32 * 16;
+        const size_t head = round_up(slot_bytes + part_bytes + 256, 128);
         for (int t = 0; t < 10; ++t) {
             const int sc = kTry[t][0], stages = kTry[t][1];
             const size_t ne = (size_t)sc * p.lanes;
             if (ne > 32 * (size_t)kRowRegs || stages > kMaxStages) continue;
-            const size_t stage_bytes = round_up(ne * ((size_t)rec_bytes + P + (backward ? P * 8 : 0)), 128);
-            // behind the last stage: room for the look-ahead of its last step, which reads one step
-            // past the stage in every area (the widest is the earliest-start area)
+            const size_t stage_bytes = round_up(ne * (rec_bytes + P + (backward ? P * 8 : 0)), 128);
+            // behind the last stage: room for the look-ahead of its last step
             const size_t pad = round_up((size_t)p.lanes * std::max<size_t>(P * 8, rec_bytes), 128);
-            const size_t total = slot_bytes + 256 + stages * stage_bytes + pad;
+            const size_t total = head + stages * stage_bytes + pad;
             if (total > budget) continue;
             sp.sc = sc;
             sp.stages = stages;
@@ -267,12 +267,12 @@ bool ilp_shape(const emo_graph *g, const Program &p, bool backward, int64_t NB, 
             sp.off_lvl = (unsigned)(ne * rec_bytes);
             sp.off_es = sp.off_lvl + (unsigned)(ne * P);
             sp.stage_bytes = (unsigned)stage_bytes;
-            sp.off_part = 0;
-            sp.off_bar = (unsigned)slot_bytes;
-            sp.off_stage0 = (unsigned)(slot_bytes + 256);
+            sp.off_part = (unsigned)slot_bytes;
+            sp.off_bar = (unsigned)(slot_bytes + part_bytes);
+            sp.off_stage0 = (unsigned)head;
             s.groups = G;
-            s.grid = (int)((n_warps + G - 1) / G);
-            s.threads = (G + 1) * 32;
+            s.grid = (int)((n_groups + G - 1) / G);
+            s.threads = (G * p.lanes + 1) * 32;
             s.smem = total;
             return true;
         }
@@ -284,16 +284,16 @@ bool ilp_shape(const emo_graph *g, const Program &p, bool backward, int64_t NB, 
 // spill) or both with the plain kernels (through an [n][ldes] array).
 struct PassPlan {
     bool staged = false;
-    bool ilp = false;         // staged, with the schedule lanes inside one thread
+    bool lane = false;        // staged, one policy per thread (program in the padded layout)
     LaunchShape sf, sb;       // forward / backward launch shapes
     StagedParams pf, pb;
     size_t spill_bytes = 0;   // tiled spill: [tiles][rows of the backward program][backward tile]
 };
 
 // rows of one tile of the spill: the entries of the backward program (padded for the in-thread kernel)
-size_t spill_rows_of(const emo_graph *g, bool ilp)
+size_t spill_rows_of(const emo_graph *g, bool lane)
 {
-    return (size_t)(ilp ? g->ibwd.steps_pad : g->bwd.steps) * g->bwd.lanes;
+    return (size_t)(lane ? g->lbwd.steps_pad : g->bwd.steps) * g->bwd.lanes;
 }
 
 bool aligned16(const void *q) { return ((uintptr_t)q % 16) == 0; }
@@ -305,9 +305,9 @@ int make_plan(const emo_graph *g, int64_t B, bool want_base, bool need_bwd, cons
     const int64_t big = (int64_t)1 << 28;
     const int64_t NBf = B + (want_base ? 1 : 0);
     const bool can_stage = !(flags & EMO_F_NO_STAGING) && ldb % 16 == 0 && aligned16(lvl) && ldb < big && ldes_plain < big && ldo < big;
-    pl.ilp = can_stage && !(flags & EMO_F_PAIR_KERNEL) && ilp_shape(g, g->fwd, false, NBf, pl.sf, pl.pf) &&
-             (!need_bwd || ilp_shape(g, g->bwd, true, B, pl.sb, pl.pb));
-    pl.staged = pl.ilp || (can_stage && staged_shape(g, g->fwd, g->dfwd.rec_bytes, false, NBf, pl.sf, pl.pf) &&
+    if (can_stage && !(flags & EMO_F_PAIR_KERNEL))
+        pl.lane = lane_shape(g, g->fwd, false, NBf, pl.sf, pl.pf) && (!need_bwd || lane_shape(g, g->bwd, true, B, pl.sb, pl.pb));
+    pl.staged = pl.lane || (can_stage && staged_shape(g, g->fwd, g->dfwd.rec_bytes, false, NBf, pl.sf, pl.pf) &&
                            (!need_bwd || staged_shape(g, g->bwd, g->dbwd.rec_bytes, true, B, pl.sb, pl.pb)));
     if (!pl.staged) {
         int rc = shape_for(g, g->fwd, NBf, pl.sf);
@@ -316,7 +316,7 @@ int make_plan(const emo_graph *g, int64_t B, bool want_base, bool need_bwd, cons
     }
     if (need_bwd) {
         const size_t tiles = ((size_t)B + pl.pb.ptile - 1) / pl.pb.ptile;
-        pl.spill_bytes = tiles * spill_rows_of(g, pl.ilp) * pl.pb.ptile * sizeof(int64_t);
+        pl.spill_bytes = tiles * spill_rows_of(g, pl.lane) * pl.pb.ptile * sizeof(int64_t);
     }
     return EMO_OK;
 }
@@ -350,7 +350,7 @@ int launch_pass(const emo_graph *g, const PassPlan &pl, bool backward, int64_t B
     a.ES = ES;
     a.ldes = ldes;
     a.spill = spill;
-    a.spill_rows = (int64_t)spill_rows_of(g, pl.ilp);
+    a.spill_rows = (int64_t)spill_rows_of(g, pl.lane);
     a.spill_ptile = pl.staged ? pl.pb.ptile : 64;
     a.LS = LS;
     a.slack = slack;
@@ -375,15 +375,14 @@ int launch_pass(const emo_graph *g, const PassPlan &pl, bool backward, int64_t B
         // matrix with 16-byte aligned rows (backward); register budget by block size
         const bool extra = backward ? (LS != nullptr || sp.want_sums || !sp.vec_out) : (ES != nullptr);
         void (*kern)(StagedParams) = nullptr;
-        if (pl.ilp) {
-            const DevProgramIlp &di = backward ? g->ibwd : g->ifwd;
-            IlpParams ip;
+        if (pl.lane) {
+            const DevProgramLane &di = backward ? g->lbwd : g->lfwd;
+            LaneParams ip;
             const unsigned ne = (unsigned)sp.sc * (unsigned)p.lanes;
             sp.p.steps = di.steps_pad;
             sp.p.rows = di.rows;
             ip.tab_entry = di.tab_entry;
-            ip.st.off_node = ne * 16u;
-            ip.st.off_tab = ip.st.off_node + ne * 4u;
+            ip.st.off_tab = ne * 32u;
             int nb = 0;
             auto bulk = [&](const void *src, unsigned per_entry, unsigned off, unsigned long long per_block) {
                 sp.bsrc[nb] = (const unsigned char *)src;
@@ -392,34 +391,22 @@ int launch_pass(const emo_graph *g, const PassPlan &pl, bool backward, int64_t B
                 sp.bblock[nb] = per_block;
                 ++nb;
             };
-            bulk(di.ent, 16, 0, 0);
-            if (!backward && ES) bulk(di.node, 4, ip.st.off_node, 0);
+            bulk(di.ent, 32, 0, 0);
             bulk(di.tab, di.tab_entry, ip.st.off_tab, 0);
             if (backward) bulk(spill, (unsigned)sp.ptile * 8u, sp.off_es, (unsigned long long)a.spill_rows * sp.ptile * 8ull);
             sp.nbulk = nb;
-            void (*kern_ilp)(IlpParams) = nullptr;
-#define EMO_PICK_W(W_)                                                                                         \
-    case W_:                                                                                                   \
-        kern_ilp = backward ? (extra ? emo_pass_ilp<true, true, W_> : emo_pass_ilp<true, false, W_>)               \
-                            : (extra ? emo_pass_ilp<false, true, W_> : emo_pass_ilp<false, false, W_>);            \
-        break
-            const bool extra_ilp = backward ? (LS != nullptr || sp.want_sums) : (ES != nullptr);
-            const bool extra = extra_ilp;
-            switch (p.lanes) {
-                EMO_PICK_W(1);
-                EMO_PICK_W(2);
-                EMO_PICK_W(3);
-                EMO_PICK_W(4);
-                EMO_PICK_W(5);
-                EMO_PICK_W(6);
-                EMO_PICK_W(7);
-                EMO_PICK_W(8);
-                default: return EMO_E_UNSUPPORTED;
-            }
-#undef EMO_PICK_W
+            void (*kern_lane)(LaneParams) = nullptr;
+            const bool extra_l = backward ? (LS != nullptr || sp.want_sums) : (ES != nullptr);
+#define EMO_PICK_L(MAXT)                                                                                        \
+    kern_lane = backward ? (extra_l ? emo_pass_lane<true, true, MAXT> : emo_pass_lane<true, false, MAXT>)           \
+                        : (extra_l ? emo_pass_lane<false, true, MAXT> : emo_pass_lane<false, false, MAXT>)
+            if (s.threads <= 512) EMO_PICK_L(512);
+            else if (s.threads <= 768) EMO_PICK_L(768);
+            else EMO_PICK_L(1024);
+#undef EMO_PICK_L
             ip.sp = sp;
-            EMO_CUDA(cudaFuncSetAttribute(kern_ilp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s.smem));
-            kern_ilp<<<s.grid, s.threads, s.smem, st>>>(ip);
+            EMO_CUDA(cudaFuncSetAttribute(kern_lane, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s.smem));
+            kern_lane<<<s.grid, s.threads, s.smem, st>>>(ip);
         } else {
             sp.nbulk = 0;
             sp.bsrc[sp.nbulk] = d.rec; sp.bentry[sp.nbulk] = (unsigned)d.rec_bytes; sp.boff[sp.nbulk] = 0; sp.bblock[sp.nbulk] = 0;
@@ -596,9 +583,9 @@ int emo_graph_load(int32_t n, const int64_t *row_ptr, const int32_t *col, const 
         g->smem_optin = prop.sharedMemPerBlockOptin;
         int rc = upload_program(g->fwd, g->dfwd);
         if (rc == EMO_OK) rc = upload_program(g->bwd, g->dbwd);
-        if (rc == EMO_OK && g->fwd.lanes <= kIlpMaxLanes && g->bwd.lanes <= kIlpMaxLanes) {
-            rc = upload_program_ilp(g->fwd, g->ifwd);
-            if (rc == EMO_OK) rc = upload_program_ilp(g->bwd, g->ibwd);
+        if (rc == EMO_OK && g->fwd.lanes < 32 && g->bwd.lanes < 32) {
+            rc = upload_program_lane(g->fwd, g->lfwd);
+            if (rc == EMO_OK) rc = upload_program_lane(g->bwd, g->lbwd);
         }
         if (rc != EMO_OK) { emo_graph_free(g); return rc; }
     }
@@ -612,8 +599,8 @@ int emo_graph_free(emo_graph *g)
     if (!g->host_only) {
         free_program(g->dfwd);
         free_program(g->dbwd);
-        free_program_ilp(g->ifwd);
-        free_program_ilp(g->ibwd);
+        free_program_lane(g->lfwd);
+        free_program_lane(g->lbwd);
     }
     delete g;
     return EMO_OK;
@@ -670,8 +657,7 @@ size_t spill_need(const emo_graph *g, int64_t B)
         StagedParams sp;
         // either staged kernel may run (the call's flags decide): room for the wider tiling
         for (int which = 0; which < 2; ++which) {
-            const bool ok = which ? staged_shape(g, g->bwd, g->dbwd.rec_bytes, true, B, s, sp)
-                                  : ilp_shape(g, g->bwd, true, B, s, sp);
+            const bool ok = which ? staged_shape(g, g->bwd, g->dbwd.rec_bytes, true, B, s, sp) : lane_shape(g, g->bwd, true, B, s, sp);
             if (!ok) continue;
             const size_t tiles = ((size_t)B + sp.ptile - 1) / sp.ptile;
             tiled = std::max(tiled, tiles * spill_rows_of(g, which == 0) * sp.ptile * sizeof(int64_t));

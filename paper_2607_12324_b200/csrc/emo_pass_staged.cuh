@@ -68,6 +68,11 @@ __device__ __forceinline__ void emo_mbar_arrive(unsigned bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+__device__ __forceinline__ void emo_mbar_arrive_if(unsigned bar, bool cond)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %1, 0;\n\t@p mbarrier.arrive.shared::cta.b64 _, [%0];\n\t}" ::"r"(bar), "r"((unsigned)cond)
+                 : "memory");
+}
 __device__ __forceinline__ bool emo_mbar_try(unsigned bar, unsigned parity)
 {
     unsigned ok;
@@ -191,6 +196,16 @@ __device__ __forceinline__ long long *emo_row_ptr(long long *base, unsigned row,
     asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(r) : "r"(row), "r"(pitch_bytes), "l"(reinterpret_cast<unsigned long long>(base)));
     return reinterpret_cast<long long *>(r);
 }
+__device__ __forceinline__ bool emo_mbar_test(unsigned bar, unsigned parity)
+{
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 // Wait until the slot's value with the given phase parity has been written.  Bounded; also gives
 // up as soon as another warp of the group has raised the abort flag.
 __device__ __noinline__ bool emo_slot_wait_slow(unsigned bar, unsigned parity, volatile int *abort_flag)
@@ -199,7 +214,7 @@ __device__ __noinline__ bool emo_slot_wait_slow(unsigned bar, unsigned parity, v
     const long long t0 = clock64();
     for (;;) {
         for (unsigned i = 0; i < kSpinPolls; ++i)
-            if (emo_mbar_try(bar, parity)) return true;
+            if (emo_mbar_test(bar, parity)) return true;
         if (*abort_flag || clock64() - t0 > kWaitCycles) return false;
     }
 }
