@@ -9,8 +9,9 @@
 //                        (bits 20..23, forward; see emo_compile.h); word 2 = mask applied to the lane's running value (0 =
 //                        start from 0, ~0 = continue from the lane's last node); word 3 = operand
 //                        slots 0..3; word 4 = operand slots 4..5; word 5 = node id
-//   table  [Q][Lp]       forward: {duration, 0, energy} in 16 bytes per level; backward: duration
-//                        in 4 bytes.  Rows of nodes that ignore the policy hold one value Lp times.
+//   table  [Q][Lp]       forward: {duration, high word of the energy, low word} in 12 bytes per
+//                        level; backward: duration in 4 bytes.  Rows of nodes that ignore the policy
+//                        hold one value Lp times.
 // Q = padded steps x lanes; the padding steps are idle entries, so every stage holds whole steps.
 // Included only by emo_lib.cu.
 #pragma once

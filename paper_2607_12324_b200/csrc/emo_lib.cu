@@ -93,7 +93,7 @@ int upload_program_lane(const Program &p, DevProgramLane &d)
     const size_t Q = (size_t)p.steps * p.lanes;
     d.steps_pad = (p.steps + kLaneStepPad - 1) / kLaneStepPad * kLaneStepPad;
     const size_t Qp = (size_t)d.steps_pad * p.lanes;
-    d.tab_entry = (unsigned)p.Lp * (fwd ? 16u : 4u);
+    d.tab_entry = (unsigned)p.Lp * (fwd ? 12u : 4u);
     std::vector<uint32_t> ent(Qp * 8, 0), rows(Qp, kNone);
     std::vector<unsigned char> tab(Qp * d.tab_entry, 0);
     for (size_t q = 0; q < Qp; ++q) {
@@ -123,9 +123,15 @@ int upload_program_lane(const Program &p, DevProgramLane &d)
         const bool uses_level = ((fl >> kMaskShift) & 255u) != 0;
         for (int l = 0; l < p.Lp; ++l) {
             const size_t src = q * p.Lp + (uses_level ? l : 0);
-            unsigned char *t = tab.data() + q * d.tab_entry + (size_t)l * (fwd ? 16 : 4);
+            unsigned char *t = tab.data() + q * d.tab_entry + (size_t)l * (fwd ? 12 : 4);
             std::memcpy(t, &p.lat[src], 4);
-            if (fwd) std::memcpy(t + 8, &p.energy[src], 8);
+            if (fwd) {
+                uint64_t bits;
+                std::memcpy(&bits, &p.energy[src], 8);
+                const uint32_t hi = (uint32_t)(bits >> 32), lo = (uint32_t)bits;
+                std::memcpy(t + 4, &hi, 4);
+                std::memcpy(t + 8, &lo, 4);
+            }
         }
     }
     int rc = upload(&d.ent, ent.data(), ent.size() * 4);
@@ -239,7 +245,7 @@ bool staged_shape(const emo_graph *g, const Program &p, int rec_bytes, bool back
 bool lane_shape(const emo_graph *g, const Program &p, bool backward, int64_t NB, LaunchShape &s, StagedParams &sp)
 {
     if (p.steps == 0 || !g->smem_optin || !g->lfwd.ent || !g->lbwd.ent) return false;
-    const size_t rec_bytes = 32 + (size_t)p.Lp * (backward ? 4 : 16);     // entry and table row
+    const size_t rec_bytes = 32 + (size_t)p.Lp * (backward ? 4 : 12);     // entry and table row
     const int64_t n_groups = (NB + 31) / 32;
     const int gmax = std::min(31 / p.lanes, 15);
     if (gmax < 1) return false;

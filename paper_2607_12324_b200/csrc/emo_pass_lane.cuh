@@ -103,9 +103,12 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_lane(LaneParams ip)
             const unsigned l = emo_lds_u8(lvl_a) & lmask;
             if (BWD) x.es = emo_lds_s64(es_a);
             if (!BWD) {
-                const uint4 t = emo_lds128(tab_a + l * 16u);
-                x.d = t.x;
-                x.g = __hiloint2double((int)t.w, (int)t.z);
+                // three words per level, 12 bytes apart: with a stride of three words the 32 levels
+                // of a row fall into 32 different banks, so each of these loads is one wavefront
+                // whatever levels the lanes hold (one 16-byte load per lane cost about ten)
+                const unsigned ta = tab_a + l * 12u;
+                x.d = emo_lds_u32(ta);
+                x.g = __hiloint2double((int)emo_lds_u32(ta + 4u), (int)emo_lds_u32(ta + 8u));
             } else {
                 x.d = emo_lds_u32(tab_a + l * 4u);
             }
@@ -240,7 +243,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_lane(LaneParams ip)
             };
             // a simple node (forward): the lane's own value is its start, nothing is exchanged
             auto simple = [&](const EmoLaneFetched &f) {
-                emo_stg_row_if(spill_lane, f.e.x, spill8, h, spill_ok);
+                if (spill_lane) *emo_row_ptr(spill_lane, f.e.x, spill8) = h;
                 if (EXTRA && es_lane) *emo_row_ptr(es_lane, emo_lds_u32(ent_a - d_ent + 20u), ldes8) = h;
                 ea += f.g;
                 h = emo_add_dur(h, f.d);
@@ -257,12 +260,13 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_lane(LaneParams ip)
                         step(x1, x0);
                     }
                 } else {
-                    // forward: most entries are simple and come in runs (the entry that starts a run
-                    // says how long it is; a run ends with its block of kSyncSteps steps)
+                    // forward: most entries are simple (the lane's own value is the node's start,
+                    // nothing is exchanged) and come in runs; the entry that starts a run says how
+                    // long it is (a run ends with its block of kSyncSteps steps, and here with the
+                    // stage: the rest of it starts the next stage)
                     int j = 0;
 #pragma unroll 1
                     while (j < n) {
-                        // (a stage may end before the run does: the rest of it starts the next stage)
                         int run = dead ? 0 : min((int)((x0.e.y >> kLaneRunShift) & 15u), n - j);
                         if (run) {
                             j += run;
