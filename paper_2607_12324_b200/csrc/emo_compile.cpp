@@ -269,16 +269,28 @@ int compile_program(const HostGraph &g, const int64_t *lat, const double *energy
         }
         std::vector<int32_t> row((size_t)lanes, -1);
         std::vector<char> placed(chosen.size(), 0);
-        // first the ops whose operand sits in a free warp's register
+        // first the ops whose operand sits in a free warp's register.  Where several operands do,
+        // the op follows the one with the fewest readers: a value with one reader that travels in a
+        // register is never written to a slot, and a serial chain (the launch chain, whose nodes
+        // each have one chain successor but also read several kernels) stays on one warp instead
+        // of hopping from warp to warp with a slot hand-over on its critical path every step.
         for (size_t j = 0; j < chosen.size(); ++j) {
             int32_t i = chosen[j];
+            int best_w = -1;
+            int64_t best_fan = 0;
             for (int32_t p : ops[i].preds) {
                 int w = warp_of[p];
                 if (w >= 0 && last[w] == p && row[w] < 0) {
-                    row[w] = i;
-                    placed[j] = 1;
-                    break;
+                    const int64_t fan = cp[p + 1] - cp[p];
+                    if (best_w < 0 || fan < best_fan) {
+                        best_w = w;
+                        best_fan = fan;
+                    }
                 }
+            }
+            if (best_w >= 0) {
+                row[best_w] = i;
+                placed[j] = 1;
             }
         }
         // then the rest: prefer a warp whose register value nobody is waiting for
@@ -453,6 +465,24 @@ int compile_program(const HostGraph &g, const int64_t *lat, const double *energy
             }
             next_run = run;
             next_mask = mask;
+        }
+    }
+    // Runs of plain entries for the one-policy-per-thread kernel (word 5).  An entry is plain when its
+    // only operand is the warp's register and it handles a real node; forward it also writes no
+    // slot and ends no path, backward it may write one (there nearly every node hands its value to
+    // the node that launched it).  Word 5 of a plain entry is the length of the run that starts at
+    // it, inside one block of kSyncSteps steps; 0 for every other entry.
+    for (int w = 0; w < lanes; ++w) {
+        uint32_t next_run = 0;
+        for (int32_t s = S - 1; s >= 0; --s) {
+            uint32_t *en = &out.entries[((size_t)s * lanes + w) * kEntryWords];
+            const uint32_t fl = en[1];
+            bool plain = (fl & kValid) && (fl & kRegPred) && !(fl & kAux) && ((fl >> kNPredShift) & 7u) == 0;
+            if (plain && !backward && (fl & (kWriteSlot | kTerminal))) plain = false;
+            uint32_t run = 0;
+            if (plain) run = ((s + 1) % kSyncSteps != 0) ? next_run + 1 : 1;
+            en[5] = run;
+            next_run = run;
         }
     }
     return EMO_OK;

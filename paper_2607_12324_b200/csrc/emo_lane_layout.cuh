@@ -5,8 +5,8 @@
 //                        spill; backward: node id) or kNone; word 1 = out slot (bits 0..7, 255 =
 //                        none) | number of slot operands (bits 8..10) | terminal (bit 11) | phase
 //                        parity of the value written (bit 12) and of each operand (bits 13..18) |
-//                        idle (bit 19) | length of the run of simple entries that starts here
-//                        (bits 20..23, forward; see emo_compile.h); word 2 = mask applied to the lane's running value (0 =
+//                        idle (bit 19) | length of the run of plain entries that starts here
+//                        (bits 20..23; see emo_compile.cpp); word 2 = mask applied to the lane's running value (0 =
 //                        start from 0, ~0 = continue from the lane's last node); word 3 = operand
 //                        slots 0..3; word 4 = operand slots 4..5; word 5 = node id
 //   table  [Q][Lp]       forward: {duration, high word of the energy, low word} in 12 bytes per
@@ -17,7 +17,7 @@
 #pragma once
 #include "emo_pass_staged.cuh"
 
-constexpr int kLaneStepPad = 16;                 // programs are padded to a multiple of this many steps
+constexpr int kLaneStepPad = 32;                 // programs are padded to a multiple of this many steps (the longest stage)
 constexpr unsigned kLaneNoSlot = 255u;
 constexpr unsigned kLaneNpShift = 8, kLaneTerminal = 0x800u, kLaneOutParShift = 12, kLaneOpParShift = 13, kLaneIdle = 1u << 19, kLaneRunShift = 20;
 

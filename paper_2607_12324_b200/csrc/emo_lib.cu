@@ -112,7 +112,7 @@ int upload_program_lane(const Program &p, DevProgramLane &d)
         const uint32_t oppar = (fl >> kOperandParityShift) & 63u;
         w[0] = en[0];
         w[1] = out | (np << kLaneNpShift) | ((fl & kTerminal) ? kLaneTerminal : 0u) | (outpar << kLaneOutParShift) | (oppar << kLaneOpParShift);
-        if (fwd && (fl & kSimple)) w[1] |= ((fl >> kRunShift) & 15u) << kLaneRunShift;
+        w[1] |= (en[5] & 15u) << kLaneRunShift;
         w[2] = (fl & kRegPred) ? 0xFFFFFFFFu : 0u;
         w[3] = en[2];
         w[4] = en[3];
@@ -252,7 +252,10 @@ bool lane_shape(const emo_graph *g, const Program &p, bool backward, int64_t NB,
     const int64_t want = (n_groups + g->sm_count - 1) / g->sm_count;
     int G = (int)std::max<int64_t>(1, std::min<int64_t>(gmax, want));
     const size_t budget = g->smem_optin;
-    static const int kTry[10][2] = {{16, 4}, {16, 3}, {8, 4}, {8, 3}, {4, 6}, {4, 5}, {4, 4}, {8, 2}, {4, 3}, {4, 2}};
+    // {steps per stage, stages}: long stages first - a stage boundary costs every warp about a
+    // microsecond (measured: 8, 16, 32 steps per stage gave 15.1, 12.3, 11.4 ms on the same forward
+    // pass), while two stages hide the refill as well as four
+    static const int kTry[10][2] = {{32, 2}, {16, 3}, {16, 2}, {8, 3}, {8, 2}, {4, 6}, {4, 5}, {4, 4}, {4, 3}, {4, 2}};
     for (; G >= 1; --G) {
         const size_t P = 32 * (size_t)G;
         const size_t slot_bytes = round_up((size_t)G * p.slots * kLaneSlotStride, 16);
@@ -261,7 +264,7 @@ bool lane_shape(const emo_graph *g, const Program &p, bool backward, int64_t NB,
         for (int t = 0; t < 10; ++t) {
             const int sc = kTry[t][0], stages = kTry[t][1];
             const size_t ne = (size_t)sc * p.lanes;
-            if (ne > 32 * (size_t)kRowRegs || stages > kMaxStages) continue;
+            if (ne > 32 * (size_t)kRowRegs || stages > kMaxStages || kLaneStepPad % sc != 0) continue;
             const size_t stage_bytes = round_up(ne * (rec_bytes + P + (backward ? P * 8 : 0)), 128);
             // behind the last stage: room for the look-ahead of its last step
             const size_t pad = round_up((size_t)p.lanes * std::max<size_t>(P * 8, rec_bytes), 128);

@@ -113,10 +113,41 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_lane(LaneParams ip)
                 x.d = emo_lds_u32(tab_a + l * 4u);
             }
         };
+        // a plain node: the lane's own value is its start and no slot is read (forward: none
+        // is written either)
+        auto simple = [&](const EmoLaneFetched &f) {
+            if (!BWD) {
+                if (spill_lane) *emo_row_ptr(spill_lane, f.e.x, spill8) = h;
+                if (EXTRA && es_lane) *emo_row_ptr(es_lane, emo_lds_u32(ent_a - d_ent + 20u), ldes8) = h;
+                ea += f.g;
+                h = emo_add_dur(h, f.d);
+            } else {
+                h = emo_add_dur(h, f.d);
+                const unsigned out = f.e.y & 255u;
+                const unsigned bar = slotbar_base + out * kLaneSlotStride;
+                emo_sts_s64_if(bar + lane8, h, out, kLaneNoSlot);
+                __syncwarp();
+                emo_mbar_arrive_if(bar, out != kLaneNoSlot && lane == 0);
+                const long long ls = T0 - h, sl = ls - f.es;
+                if (sl_lane) *emo_row_ptr(sl_lane, f.e.x, ldo8) = sl;
+                if (EXTRA) {
+                    if (ls_lane) *emo_row_ptr(ls_lane, f.e.x, ldo8) = ls;
+                    if (want_sums) {
+                        acc += sl;
+                        nc += (sl == 0);
+                    }
+                }
+            }
+        };
         // one node; ent is the address of its entry (for the rarely needed words 4 and 5)
         auto process = [&](const EmoLaneFetched &f, unsigned ent) {
             const unsigned fl = f.e.y;
             if ((fl & kLaneIdle) || dead) return;
+            if (BWD && (fl & (15u << kLaneRunShift))) {
+                // backward: most nodes are plain - skip every other test
+                simple(f);
+                return;
+            }
             long long v = h & (long long)(int)f.e.z;
             if (fl & (7u << kLaneNpShift)) {
                 const unsigned np = (fl >> kLaneNpShift) & 7u;
@@ -201,7 +232,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_lane(LaneParams ip)
 
         for (int c = 0; c < n_chunks; ++c) {
             const int s = c % nstages;
-            const bool ok = emo_mbar_wait(bar0 + 8 * s, (c / nstages) & 1);
+            const bool ok = emo_mbar_test(bar0 + 8 * s, (c / nstages) & 1) || emo_mbar_wait(bar0 + 8 * s, (c / nstages) & 1);
             // a warp that gave up (or heard that the producer did) stops working but keeps walking
             // until the group's next meeting, where all its warps read one flag and leave together
             if (!ok || dead || (chain == 0 && abort_flag[groups])) {
@@ -241,13 +272,6 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_lane(LaneParams ip)
                 fetch(nxt);
                 process(cur, ent);
             };
-            // a simple node (forward): the lane's own value is its start, nothing is exchanged
-            auto simple = [&](const EmoLaneFetched &f) {
-                if (spill_lane) *emo_row_ptr(spill_lane, f.e.x, spill8) = h;
-                if (EXTRA && es_lane) *emo_row_ptr(es_lane, emo_lds_u32(ent_a - d_ent + 20u), ldes8) = h;
-                ea += f.g;
-                h = emo_add_dur(h, f.d);
-            };
             EmoLaneFetched x0, x1;
             fetch(x0);
             for (int j0 = 0; j0 < sc; j0 += emo::kSyncSteps) {
@@ -260,10 +284,9 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_lane(LaneParams ip)
                         step(x1, x0);
                     }
                 } else {
-                    // forward: most entries are simple (the lane's own value is the node's start,
-                    // nothing is exchanged) and come in runs; the entry that starts a run says how
-                    // long it is (a run ends with its block of kSyncSteps steps, and here with the
-                    // stage: the rest of it starts the next stage)
+                    // most entries are plain (the lane's own value is the node's start) and come in
+                    // runs; the entry that starts a run says how long it is (a run ends with its block
+                    // of kSyncSteps steps, and here with the stage: the rest of it starts the next stage)
                     int j = 0;
 #pragma unroll 1
                     while (j < n) {

@@ -82,6 +82,24 @@ def check_programs(emo, oracle_mod, g, lv, flags=0, group_of=None):
                     for k in range(1, run):
                         g2 = int(fl[t + k, w])
                         assert (g2 >> 31) and ((g2 >> 16) & 15) == run - k and ((g2 >> 8) & 255) == ((f >> 8) & 255)
+    # runs of plain entries (word 5): register operand only, a real node; the forward program also
+    # excludes entries that write a slot or end a path
+    for ent_x, bwd_x in ((ent, False), (ent_b, True)):
+        fl = ent_x[:, :, 1].astype(np.int64)
+        runs = ent_x[:, :, 5].astype(np.int64)
+        S_, W_ = fl.shape
+        for w in range(W_):
+            nxt = 0
+            for t in range(S_ - 1, -1, -1):
+                f = int(fl[t, w])
+                plain = (f & 1) and (f & 2) and not (f & 0x80) and ((f >> 4) & 7) == 0
+                if plain and not bwd_x and (f & (4 | 8)):
+                    plain = False
+                want = 0
+                if plain:
+                    want = nxt + 1 if (t + 1) % PE.SYNC_STEPS != 0 else 1
+                assert int(runs[t, w]) == want
+                nxt = want
     assert np.array_equal(b["LS"], r["LS"])
     assert np.array_equal(b["slack"], r["slack"])
     h.free()
