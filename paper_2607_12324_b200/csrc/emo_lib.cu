@@ -247,7 +247,7 @@ bool lane_shape(const emo_graph *g, const Program &p, bool backward, int64_t NB,
     if (p.steps == 0 || !g->smem_optin || !g->lfwd.ent || !g->lbwd.ent) return false;
     const size_t rec_bytes = 32 + (size_t)p.Lp * (backward ? 4 : 12);     // entry and table row
     const int64_t n_groups = (NB + 31) / 32;
-    const int gmax = std::min(31 / p.lanes, 15);
+    const int gmax = std::min((32 - kProducerWarps) / p.lanes, 15);
     if (gmax < 1) return false;
     const int64_t want = (n_groups + g->sm_count - 1) / g->sm_count;
     int G = (int)std::max<int64_t>(1, std::min<int64_t>(gmax, want));
@@ -281,7 +281,7 @@ bool lane_shape(const emo_graph *g, const Program &p, bool backward, int64_t NB,
             sp.off_stage0 = (unsigned)head;
             s.groups = G;
             s.grid = (int)((n_groups + G - 1) / G);
-            s.threads = (G * p.lanes + 1) * 32;
+            s.threads = (G * p.lanes + kProducerWarps) * 32;
             s.smem = total;
             return true;
         }
@@ -592,7 +592,7 @@ int emo_graph_load(int32_t n, const int64_t *row_ptr, const int32_t *col, const 
         g->smem_optin = prop.sharedMemPerBlockOptin;
         int rc = upload_program(g->fwd, g->dfwd);
         if (rc == EMO_OK) rc = upload_program(g->bwd, g->dbwd);
-        if (rc == EMO_OK && g->fwd.lanes < 32 && g->bwd.lanes < 32) {
+        if (rc == EMO_OK && g->fwd.lanes <= 32 - kProducerWarps && g->bwd.lanes <= 32 - kProducerWarps) {
             rc = upload_program_lane(g->fwd, g->lfwd);
             if (rc == EMO_OK) rc = upload_program_lane(g->bwd, g->lbwd);
         }

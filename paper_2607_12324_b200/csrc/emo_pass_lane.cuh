@@ -1,7 +1,7 @@
 // Staged pass kernel, one warp per schedule lane and ONE policy per thread (sm_100a).
 //
 // A group of 32 policies is carried by `lanes` warps, one per schedule lane; a block holds several
-// groups and one producer warp that fills the ring of stages (emo_produce).  Compared with two
+// groups and the producer warps that fill the ring of stages (emo_produce).  Compared with two
 // policies per thread this doubles the number of resident warps, which is what the path is short
 // of: every warp is a serial chain of dependent steps, and only other warps can fill the issue slots
 // it leaves.  The per-entry work is kept small by a program layout made for it (see
@@ -39,7 +39,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_lane(LaneParams ip)
     const int warp = threadIdx.x >> 5;
     const int lanes = p.lanes, groups = p.groups, nstages = sp.stages, sc = sp.sc;
     const int steps = p.steps;                          // padded: a multiple of sc
-    const int n_cons = groups * lanes;                  // consumer warps; the warp after them produces
+    const int n_cons = groups * lanes;                  // consumer warps; the warps after them produce
     const bool producer = warp >= n_cons;
     const int group = producer ? 0 : warp / lanes;
     const int chain = warp - group * lanes;
@@ -60,7 +60,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_lane(LaneParams ip)
     for (int i = threadIdx.x; i < groups * p.slots; i += blockDim.x) emo_mbar_init(smem0 + (unsigned)i * kLaneSlotStride, 1);
     if (threadIdx.x == 0) {
         for (int k = 0; k < nstages; ++k) {
-            emo_mbar_init(bar0 + 8 * k, 1 + 32);       // expect-tx arrival + the producer lanes' cp.async arrivals
+            emo_mbar_init(bar0 + 8 * k, 1 + 32 * kProducerWarps);   // expect-tx arrival + every producer lane's cp.async arrival
             emo_mbar_init(bar0 + 8 * (kMaxStages + k), n_cons);
         }
         for (int k = 0; k <= groups; ++k) abort_flag[k] = 0;
@@ -74,7 +74,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_lane(LaneParams ip)
     int nc = 0;               // backward: critical nodes
 
     if (producer) {
-        emo_produce(sp, stage0, bar0, abort_flag + groups, lane, 0);
+        emo_produce(sp, stage0, bar0, abort_flag + groups, lane, warp - n_cons);
     } else {
         const int n_chunks = steps / sc;
         const unsigned slotbar_base = smem0 + (unsigned)group * p.slots * kLaneSlotStride;

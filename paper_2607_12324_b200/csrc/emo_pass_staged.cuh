@@ -28,7 +28,7 @@
 constexpr int kMaxStages = 8;
 constexpr int kMaxBulk = 5;              // bulk copies per stage
 constexpr int kRowRegs = 8;             // a stage holds at most 32 * kRowRegs records
-constexpr int kProducerWarps = 1;       // warps that issue the copies (they share the level-row pieces)
+constexpr int kProducerWarps = 2;       // warps that issue the copies (they share the level-row pieces)
 constexpr unsigned kSlotStride = 528;   // 8-byte mbarrier, 8 bytes unused, 32 lanes x 16 bytes
 constexpr long long kWaitCycles = 4000000000LL;   // about two seconds: a wait that long has failed
 constexpr unsigned kSpinPolls = 1u << 14;          // polls between two looks at the clock
