@@ -51,7 +51,8 @@ extern "C" {
 /* flags of the evaluation calls */
 #define EMO_F_VALIDATE 0x1u        /* check every level < L first; EMO_E_RANGE goes to *status */
 #define EMO_F_NO_STAGING 0x2u      /* use the plain-load kernels instead of the staged ones */
-#define EMO_F_PAIR_KERNEL 0x4u     /* staged pass kernel with two policies per thread */
+#define EMO_F_PAIR_KERNEL 0x4u     /* staged pass kernel with two policies per thread (default only for very large batches) */
+#define EMO_F_LANE_KERNEL 0x8u     /* staged pass kernel with one policy per thread (the default otherwise) */
 
 typedef struct emo_graph emo_graph;
 

@@ -88,8 +88,10 @@ __device__ __noinline__ bool emo_mbar_wait_slow(unsigned bar, unsigned parity)
 {
     const long long t0 = clock64();
     for (;;) {
-        for (unsigned i = 0; i < (1u << 14); ++i)
+        for (unsigned i = 0; i < (1u << 12); ++i) {
             if (emo_mbar_try(bar, parity)) return true;
+            __nanosleep(100);      // a waiting warp must not take issue slots from the warps that work
+        }
         if (clock64() - t0 > kWaitCycles) return false;
     }
 }
@@ -213,8 +215,10 @@ __device__ __noinline__ bool emo_slot_wait_slow(unsigned bar, unsigned parity, v
     // the clock is read rarely: reading it on every poll would keep the special-register path busy
     const long long t0 = clock64();
     for (;;) {
-        for (unsigned i = 0; i < kSpinPolls; ++i)
-            if (emo_mbar_test(bar, parity)) return true;
+        for (unsigned i = 0; i < (1u << 12); ++i) {
+            if (emo_mbar_try(bar, parity)) return true;
+            __nanosleep(40);       // a waiting warp must not take issue slots from the warps that work
+        }
         if (*abort_flag || clock64() - t0 > kWaitCycles) return false;
     }
 }

@@ -22,6 +22,7 @@ EMO_F_HOST_ONLY = 0x1
 EMO_F_VALIDATE = 0x1
 EMO_F_NO_STAGING = 0x2
 EMO_F_PAIR_KERNEL = 0x4
+EMO_F_LANE_KERNEL = 0x8
 
 EXPORTS = [
     "emo_strerror", "emo_graph_load", "emo_graph_free", "emo_graph_info", "emo_workspace_bytes",

@@ -115,10 +115,11 @@ def test_tiny_graphs_all_outputs(torch_cuda, emo, oracle_mod):
         lv_dev = torch.as_tensor(lvp, device="cuda")
         for lanes in (0, 1, 2):
             h = emo.load_workload(g, emo.EMO_F_LANES(lanes))
-            r = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, ldo=B + 3)
-            assert_matches(r, r_or, B)
-            for k in ("ES", "LS", "slack"):
-                assert (r[k][:, B:] == -7).all(), "padding columns of the outputs were written"
+            for fl in (0, emo.EMO_F_PAIR_KERNEL, emo.EMO_F_LANE_KERNEL):
+                r = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, ldo=B + 3, flags=fl)
+                assert_matches(r, r_or, B)
+                for k in ("ES", "LS", "slack"):
+                    assert (r[k][:, B:] == -7).all(), "padding columns of the outputs were written"
             T, E, st = gpu_eval(torch, emo, h, lv_dev, B, emo.EMO_F_VALIDATE)
             assert st == 0 and np.array_equal(T, r_or["makespan"])
             np.testing.assert_allclose(E, r_or["energy"], rtol=E_RTOL)
@@ -160,7 +161,8 @@ def test_config_graphs_all_outputs(torch_cuda, emo, oracle_mod, name, scale, B):
     r2 = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, want=("slack",))
     assert np.array_equal(r2["slack"][:, :B], r_or["slack"])
     base = oracle_mod.batch(g, np.full((g.n, 1), g.L - 1, dtype=np.uint8))
-    for fl in (emo.EMO_F_NO_STAGING, 0):
+    # every pass kernel: plain loads, two policies per thread, one policy per thread
+    for fl in (emo.EMO_F_NO_STAGING, emo.EMO_F_PAIR_KERNEL, emo.EMO_F_LANE_KERNEL):
         r3 = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, flags=fl, base=True)
         assert_matches(r3, r_or, B)
         assert r3["T0"] == base["makespan"][0]
@@ -169,10 +171,11 @@ def test_config_graphs_all_outputs(torch_cuda, emo, oracle_mod, name, scale, B):
     r5 = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, want=("slack",), sums=False, base=True)
     assert np.array_equal(r5["slack"][:, :B], r_or["slack"]) and r5["T0"] == base["makespan"][0]
     assert (r5["slack_sum"] == -1).all()
-    # an output pitch that is odd (no bulk copies of the ES rows possible) and one that is even
+    # an output pitch that is odd (no 16-byte stores of policy pairs possible) and one that is even
     for ldo in (B + 1, B + 2):
-        r4 = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, ldo=ldo)
-        assert_matches(r4, r_or, B)
+        for fl in (emo.EMO_F_PAIR_KERNEL, emo.EMO_F_LANE_KERNEL):
+            r4 = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, ldo=ldo, flags=fl)
+            assert_matches(r4, r_or, B)
     # single-policy call
     b = B // 2
     one = lv_dev[:, b].contiguous()
