@@ -152,7 +152,23 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_lane(LaneParams ip)
             if (fl & (7u << kLaneNpShift)) {
                 const unsigned np = (fl >> kLaneNpShift) & 7u;
                 unsigned ops = f.e.w, par = fl >> kLaneOpParShift;
-                if (BWD && np > 1) {
+                if (BWD && np == 4) {
+                    // four operands (backward: a launch node waits for the four kernels it launched),
+                    // straight-line: poll the four barriers, load the four values, take the maxima
+                    const unsigned b0 = slotbar_base + (ops & 255u) * kLaneSlotStride, b1 = slotbar_base + ((ops >> 8) & 255u) * kLaneSlotStride,
+                                   b2 = slotbar_base + ((ops >> 16) & 255u) * kLaneSlotStride, b3 = slotbar_base + (ops >> 24) * kLaneSlotStride;
+                    if (!emo_mbar_test4(b0, b1, b2, b3, par)) {
+                        if (!emo_slot_wait(b0, par & 1u, my_abort) || !emo_slot_wait(b1, (par >> 1) & 1u, my_abort) ||
+                            !emo_slot_wait(b2, (par >> 2) & 1u, my_abort) || !emo_slot_wait(b3, (par >> 3) & 1u, my_abort)) {
+                            *my_abort = 1;
+                            dead = true;
+                            return;
+                        }
+                    }
+                    const long long x0 = emo_lds_s64(b0 + lane8), x1 = emo_lds_s64(b1 + lane8), x2 = emo_lds_s64(b2 + lane8),
+                                    x3 = emo_lds_s64(b3 + lane8);
+                    v = emo_max64(emo_max64(v, x0), emo_max64(emo_max64(x1, x2), x3));
+                } else if (BWD && np > 1) {
                     // several operands (backward: a launch node waits for every kernel it launched):
                     // poll every slot's barrier, then load every value, then take the maxima - the
                     // latencies overlap instead of queuing behind one another

@@ -208,6 +208,25 @@ __device__ __forceinline__ bool emo_mbar_test(unsigned bar, unsigned parity)
         : "memory");
     return ok != 0;
 }
+// four barriers at once: true when every one of them has completed the phase with its parity
+__device__ __forceinline__ bool emo_mbar_test4(unsigned b0, unsigned b1, unsigned b2, unsigned b3, unsigned par)
+{
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p0, p1, p2, p3;\n\t.reg .u32 q0, q1, q2, q3;\n\t"
+        "and.b32 q0, %5, 1;\n\tshr.u32 q1, %5, 1;\n\tand.b32 q1, q1, 1;\n\t"
+        "shr.u32 q2, %5, 2;\n\tand.b32 q2, q2, 1;\n\tshr.u32 q3, %5, 3;\n\tand.b32 q3, q3, 1;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p0, [%1], q0;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p1, [%2], q1;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p2, [%3], q2;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p3, [%4], q3;\n\t"
+        "and.pred p0, p0, p1;\n\tand.pred p2, p2, p3;\n\tand.pred p0, p0, p2;\n\t"
+        "selp.u32 %0, 1, 0, p0;\n\t}"
+        : "=r"(ok)
+        : "r"(b0), "r"(b1), "r"(b2), "r"(b3), "r"(par)
+        : "memory");
+    return ok != 0;
+}
 // Wait until the slot's value with the given phase parity has been written.  Bounded; also gives
 // up as soon as another warp of the group has raised the abort flag.
 __device__ __noinline__ bool emo_slot_wait_slow(unsigned bar, unsigned parity, volatile int *abort_flag)
