@@ -69,6 +69,7 @@ typedef struct emo_info {
     int32_t steps_fwd, slots_fwd, aux_fwd;   /* forward program: steps, exchange slots, helper ops */
     int32_t steps_bwd, slots_bwd, aux_bwd;   /* backward program */
     int32_t lanes_bwd;  /* cooperating warps of the backward program */
+    int32_t sync_fwd, sync_bwd;   /* steps between two barriers of a group's warps (8, 16 or 32) */
 } emo_info;
 
 /* Human-readable text for a status code (static storage). */

@@ -68,15 +68,17 @@ int pick_lanes(int64_t n_ops, int depth)
 }
 
 int compile_program(const HostGraph &g, const int64_t *lat, const double *energy, bool backward,
-                    int lanes, int lookahead, const std::vector<uint32_t> *row_in_other, Program &out,
-                    std::string &err)
+                    int lanes, int lookahead, int sync_steps, const std::vector<uint32_t> *row_in_other,
+                    Program &out, std::string &err)
 {
+    if (sync_steps != 8 && sync_steps != 16 && sync_steps != 32) sync_steps = kSyncSteps;
     const int32_t n = g.n;
     const int L = g.L;
     int Lp = 4;   // at least 4 so that a table row is a multiple of 16 bytes (bulk-copy granularity)
     while (Lp < L) Lp <<= 1;
     out = Program();
     out.Lp = Lp;
+    out.sync = sync_steps;
 
     // ---- ops in a topological order of the direction being compiled --------------------------
     std::vector<Op> ops;
@@ -337,7 +339,7 @@ int compile_program(const HostGraph &g, const int64_t *lat, const double *energy
     // An operand is read from the warp's register when the producing op was the previous op of the
     // same warp; every other operand is read from the producer's slot.  A slot lives from the
     // producer's step to the last step that reads it.  The warps of a group only meet at a barrier
-    // every kSyncSteps steps and otherwise run at their own pace, so a slot is reused no earlier
+    // every sync_steps steps and otherwise run at their own pace, so a slot is reused no earlier
     // than the first step of the block after its last read: the barrier between the two blocks
     // orders the last read before the next write.  Readers find out that a value has been written
     // from a per-slot phase counter; the entry carries the phase parity of every value it touches.
@@ -353,7 +355,7 @@ int compile_program(const HostGraph &g, const int64_t *lat, const double *energy
         std::priority_queue<Key, std::vector<Key>, std::greater<Key>> busy;   // (last use step, slot)
         int32_t next_id = 0;
         for (int32_t s = 0; s < S; ++s) {
-            while (!busy.empty() && busy.top().first / kSyncSteps < s / kSyncSteps) {
+            while (!busy.empty() && busy.top().first / sync_steps < s / sync_steps) {
                 free_ids.push(busy.top().second);
                 busy.pop();
             }
@@ -448,7 +450,7 @@ int compile_program(const HostGraph &g, const int64_t *lat, const double *energy
     // Runs of simple entries.  An entry is simple when its only operand is the warp's register and
     // it neither writes a slot nor ends a path: the kernels handle a run of them in a tight loop
     // without decoding flags.  Every simple entry carries the length of the run that starts at it
-    // (in the bits that name slots, unused here); a run stays inside one block of kSyncSteps steps
+    // (in the bits that name slots, unused here); a run stays inside one block of sync_steps steps (and names at most 15 entries)
     // and its entries agree on whether they read a level.
     for (int w = 0; w < lanes; ++w) {
         uint32_t next_run = 0, next_mask = 0;
@@ -460,7 +462,7 @@ int compile_program(const HostGraph &g, const int64_t *lat, const double *energy
             const uint32_t mask = (fl >> kMaskShift) & 255u;
             if (simple) {
                 run = 1;
-                if ((s + 1) % kSyncSteps != 0 && next_run > 0 && next_mask == mask) run = next_run + 1;
+                if ((s + 1) % sync_steps != 0 && next_run > 0 && next_mask == mask) run = std::min<uint32_t>(next_run + 1, 15u);
                 fl |= kSimple | (run << kRunShift);
             }
             next_run = run;
@@ -471,7 +473,7 @@ int compile_program(const HostGraph &g, const int64_t *lat, const double *energy
     // only operand is the warp's register and it handles a real node; forward it also writes no
     // slot and ends no path, backward it may write one (there nearly every node hands its value to
     // the node that launched it).  Word 5 of a plain entry is the length of the run that starts at
-    // it, inside one block of kSyncSteps steps; 0 for every other entry.
+    // it, inside one block of sync_steps steps and 15 at most; 0 for every other entry.
     for (int w = 0; w < lanes; ++w) {
         uint32_t next_run = 0;
         for (int32_t s = S - 1; s >= 0; --s) {
@@ -480,7 +482,7 @@ int compile_program(const HostGraph &g, const int64_t *lat, const double *energy
             bool plain = (fl & kValid) && (fl & kRegPred) && !(fl & kAux) && ((fl >> kNPredShift) & 7u) == 0;
             if (plain && !backward && (fl & (kWriteSlot | kTerminal))) plain = false;
             uint32_t run = 0;
-            if (plain) run = ((s + 1) % kSyncSteps != 0) ? next_run + 1 : 1;
+            if (plain) run = ((s + 1) % sync_steps != 0) ? std::min<uint32_t>(next_run + 1, 15u) : 1;
             en[5] = run;
             next_run = run;
         }

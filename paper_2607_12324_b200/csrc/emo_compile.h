@@ -35,10 +35,11 @@ constexpr int kOutParityShift = 24;   // bit 24: phase parity of the value writt
 constexpr int kOperandParityShift = 25;   // bits 25..30: phase parity of each operand's value
 constexpr uint32_t kSimple = 0x80000000u;   // bit 31: simple entry (register operand only, no slot written, not terminal)
 constexpr int kRunShift = 16;         // simple entries: bits 16..19 = length of the run of simple entries starting here
-constexpr int kSyncSteps = 8;         // the warps of a group meet at a barrier every kSyncSteps steps
+constexpr int kSyncSteps = 8;         // default distance (in steps) between two barriers of a group's warps
 
 struct Program {
     int lanes = 0, steps = 0, slots = 0, aux = 0, Lp = 0;
+    int sync = kSyncSteps;            // the warps of a group meet at a barrier every `sync` steps (a power of two)
     int64_t pruned = 0;               // edges dropped because they can never decide a maximum
     std::vector<uint32_t> entries;    // [steps][lanes][kEntryWords], see above
     std::vector<uint32_t> pos_of_node;   // [n] index (step*lanes + lane) of the entry that handles node v
@@ -58,9 +59,11 @@ struct HostGraph {
 // Builds the forward (backward = false) or backward program.  lanes <= 0 picks a value from the
 // graph's shape.  Returns 0 or an EMO_E_* code and a message in err.
 // row_in_other (optional, [n]): what to put into word 0 of a node's entry instead of its id.
+// sync_steps (8, 16 or 32): distance between the barriers at which the warps of a group meet; a slot is
+// reused only across such a barrier, so a larger distance costs slots and saves barriers.
 int compile_program(const HostGraph &g, const int64_t *lat, const double *energy, bool backward,
-                    int lanes, int lookahead, const std::vector<uint32_t> *row_in_other, Program &out,
-                    std::string &err);
+                    int lanes, int lookahead, int sync_steps, const std::vector<uint32_t> *row_in_other,
+                    Program &out, std::string &err);
 
 int pick_lanes(int64_t n_ops, int depth);
 

@@ -26,6 +26,7 @@ struct PassParams {
     const uint32_t *rows;      // [steps*lanes]
     int rec_bytes;             // 32 + Lp*4 (+ Lp*8 forward)
     int steps, lanes, Lp, L, slots, groups;
+    int sync;                  // staged kernels: the warps of a group meet every `sync` steps
     int want_base;
     int64_t B;
     const uint8_t *lvl;       // [rows][ldb]

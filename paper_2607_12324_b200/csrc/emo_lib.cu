@@ -44,6 +44,7 @@ struct emo_graph {
 
 namespace {
 
+constexpr int kManySlots = 48;       // above this, a program is compiled with the short barrier distance
 constexpr size_t kSmallWs = 65536;   // head of the workspace: selection partials and scalars
 
 // Optional timing hook: events recorded around the forward and the backward pass kernel.
@@ -357,6 +358,7 @@ int launch_pass(const emo_graph *g, const PassPlan &pl, bool backward, int64_t B
     a.Lp = p.Lp;
     a.L = g->h.L;
     a.slots = p.slots;
+    a.sync = p.sync;
     a.groups = s.groups;
     a.want_base = want_base;
     a.B = B;
@@ -571,8 +573,22 @@ int emo_graph_load(int32_t n, const int64_t *row_ptr, const int32_t *col, const 
         // backward first: the forward entries name the row of the backward program that will read
         // the node's earliest start
         // (each direction picks its own number of lanes from its ops and depth unless one is forced)
-        int rc = compile_program(h, lat, energy, true, lanes, look, nullptr, g->bwd, err);
-        if (rc == EMO_OK) rc = compile_program(h, lat, energy, false, lanes, look, &g->bwd.pos_of_node, g->fwd, err);
+        // The distance between the group barriers: 16 steps where that costs few slots (a barrier
+        // makes every warp of a group wait for the slowest), else 8 (slots take shared memory from
+        // the stages).  Measured on the 250 000-node workload: forward 18 -> 25 slots and 11.2 -> 10.3 ms
+        // with 16, backward 82 -> 120 slots and 20.4 -> 24.5 ms.
+        auto compile_dir = [&](bool backward, const std::vector<uint32_t> *row_in_other, Program &out) {
+            int rc = compile_program(h, lat, energy, backward, lanes, look, 16, row_in_other, out, err);
+            if (rc == EMO_E_UNSUPPORTED || (rc == EMO_OK && out.slots > kManySlots)) {
+                Program tight;
+                const int rc8 = compile_program(h, lat, energy, backward, lanes, look, 8, row_in_other, tight, err);
+                if (rc8 == EMO_OK) out = std::move(tight);
+                rc = rc8;
+            }
+            return rc;
+        };
+        int rc = compile_dir(true, nullptr, g->bwd);
+        if (rc == EMO_OK) rc = compile_dir(false, &g->bwd.pos_of_node, g->fwd);
         if (rc != EMO_OK) { delete g; return rc; }
         std::vector<int32_t> hop((size_t)std::max(n, 1), 0);
         int32_t depth = 0;
@@ -634,6 +650,8 @@ int emo_graph_info(const emo_graph *g, emo_info *info)
     info->T_best = g->h.T_best;
     info->lanes = g->fwd.lanes;
     info->lanes_bwd = g->bwd.lanes;
+    info->sync_fwd = g->fwd.sync;
+    info->sync_bwd = g->bwd.sync;
     info->steps_fwd = g->fwd.steps;
     info->slots_fwd = g->fwd.slots;
     info->aux_fwd = g->fwd.aux;

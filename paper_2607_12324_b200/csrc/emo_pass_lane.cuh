@@ -11,7 +11,7 @@
 // The warps of a group do not run in lockstep.  Each walks its own column of the step program and
 // waits only for the values it reads: every exchange slot (32 x 8 bytes) has an mbarrier whose phase
 // completes when the slot's next value has been written, and the entry names the phase parity to
-// wait for.  The group meets at a named barrier every kSyncSteps steps, which bounds the drift
+// wait for.  The group meets at a named barrier every `sync` steps, which bounds the drift
 // between its warps; the host compiler reuses a slot only across such a barrier.
 // (Tried and measured slower on the backward pass: carrying the parity in bit 63 of the value and
 // polling the word itself instead of an mbarrier.)
@@ -37,7 +37,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_lane(LaneParams ip)
     const PassParams &p = sp.p;
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
-    const int lanes = p.lanes, groups = p.groups, nstages = sp.stages, sc = sp.sc;
+    const int lanes = p.lanes, groups = p.groups, nstages = sp.stages, sc = sp.sc, sync = p.sync;
     const int steps = p.steps;                          // padded: a multiple of sc
     const int n_cons = groups * lanes;                  // consumer warps; the warps after them produce
     const bool producer = warp >= n_cons;
@@ -263,8 +263,8 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_lane(LaneParams ip)
                     emo_smem[sp.off_stage0 + (size_t)s * stage_bytes + sp.off_lvl + (size_t)i * ptile + (size_t)base_col] = top;
                 __syncwarp();
             }
-            // the group meets where a block of kSyncSteps steps begins (stages may be shorter than that)
-            const bool meet = lanes > 1 && ((c * sc) % emo::kSyncSteps == 0 || base_col >= 0);
+            // the group meets where a block of `sync` steps begins (stages may be shorter than that)
+            const bool meet = lanes > 1 && ((c * sc) % sync == 0 || base_col >= 0);
             if (meet) emo_group_barrier(group + 1, gthreads);
             if ((meet || lanes == 1) && *my_abort) {
                 if (lane == 0 && p.status) atomicMin(p.status, -8);
@@ -290,9 +290,9 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_lane(LaneParams ip)
             };
             EmoLaneFetched x0, x1;
             fetch(x0);
-            for (int j0 = 0; j0 < sc; j0 += emo::kSyncSteps) {
+            for (int j0 = 0; j0 < sc; j0 += sync) {
                 if (j0 && lanes > 1) emo_group_barrier(group + 1, gthreads);
-                const int n = min(emo::kSyncSteps, sc - j0);      // even
+                const int n = min(sync, sc - j0);      // even
                 if (BWD) {
 #pragma unroll 1
                     for (int j = 0; j < n; j += 2) {
@@ -302,7 +302,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_lane(LaneParams ip)
                 } else {
                     // most entries are plain (the lane's own value is the node's start) and come in
                     // runs; the entry that starts a run says how long it is (a run ends with its block
-                    // of kSyncSteps steps, and here with the stage: the rest of it starts the next stage)
+                    // of `sync` steps, and here with the stage: the rest of it starts the next stage)
                     int j = 0;
 #pragma unroll 1
                     while (j < n) {

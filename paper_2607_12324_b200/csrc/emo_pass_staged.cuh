@@ -15,7 +15,7 @@
 // The warps of a group do not run in lockstep.  Each walks its own column of the step program and
 // waits only for the values it reads: every exchange slot has an mbarrier whose phase completes
 // when the slot's next value has been written, and the entry names the phase parity to wait for.
-// The group meets at a named barrier every kSyncSteps steps, which bounds the drift between its
+// The group meets at a named barrier every `sync` steps, which bounds the drift between its
 // warps; the host compiler reuses a slot only across such a barrier.  Included only by emo_lib.cu.
 #pragma once
 #include <cuda_runtime.h>
@@ -35,7 +35,7 @@ constexpr unsigned kSpinPolls = 1u << 14;          // polls between two looks at
 
 struct StagedParams {
     PassParams p;
-    int sc;                    // steps per stage (a multiple of kSyncSteps)
+    int sc;                    // steps per stage (a power of two, like the distance between group barriers)
     int stages;                // ring depth
     int ptile;                 // policies per block = 64 * groups
     int vec_es, vec_out;       // 128-bit global accesses allowed for ES / for LS and slack
@@ -566,10 +566,11 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_pair(StagedParams sp)
             emo_fetch<BWD>(cur, rec_a, lvl_a, es_a, en_off, store_es);
             int j = 0;
             while (j < ns) {
-                if (j && (j % emo::kSyncSteps) == 0 && lanes > 1) emo_group_barrier(group + 1, gthreads);
+                if (j && (j % p.sync) == 0 && lanes > 1) emo_group_barrier(group + 1, gthreads);
                 if (!EXTRA && !BWD && (cur.e.y & emo::kSimple) && !dead) {
                     // a run of simple nodes: h += duration, nothing else to decide
-                    const int run = (int)((cur.e.y >> emo::kRunShift) & 15u);
+                    // (a stage may end before the run does: the rest of it starts the next stage)
+                    const int run = min((int)((cur.e.y >> emo::kRunShift) & 15u), ns - j);
                     const unsigned m = (cur.e.y >> emo::kMaskShift) & 255u;
                     for (int k = 0; k < run; ++k) {
                         const unsigned row = emo_lds_u32(rec_a);

@@ -52,7 +52,7 @@ class emo_info(ctypes.Structure):
                 ("T_best", ctypes.c_int64), ("lanes", ctypes.c_int32),
                 ("steps_fwd", ctypes.c_int32), ("slots_fwd", ctypes.c_int32), ("aux_fwd", ctypes.c_int32),
                 ("steps_bwd", ctypes.c_int32), ("slots_bwd", ctypes.c_int32), ("aux_bwd", ctypes.c_int32),
-                ("lanes_bwd", ctypes.c_int32)]
+                ("lanes_bwd", ctypes.c_int32), ("sync_fwd", ctypes.c_int32), ("sync_bwd", ctypes.c_int32)]
 
 
 _lib = None

@@ -8,10 +8,10 @@ import numpy as np
 
 NONE = 0xFFFFFFFF
 VALID, REGPRED, WRITE, TERMINAL, AUX = 1, 2, 4, 8, 0x80
-SYNC_STEPS = 8      # the warps of a group meet at a barrier every SYNC_STEPS steps
+SYNC_STEPS = 8      # default distance between two barriers of a group's warps (a program names its own)
 
 
-def run(entries, rows, lat, Lp, L, slots, lvl, n, backward, ES_in=None, T_in=None):
+def run(entries, rows, lat, Lp, L, slots, lvl, n, backward, ES_in=None, T_in=None, sync=SYNC_STEPS):
     """entries [steps][lanes][8], lat [steps*lanes][Lp], lvl uint8 [rows][B].
     Forward: returns dict(T[B], ES[n][B], seen[n]).  Backward: dict(LS, slack)."""
     steps, lanes, _ = entries.shape
@@ -78,7 +78,7 @@ def run(entries, rows, lat, Lp, L, slots, lvl, n, backward, ES_in=None, T_in=Non
             if s is not None:
                 assert s not in read_ids, f"step {t}: slot {s} read and written in the same step"
                 # between barriers the warps drift: the last read must lie in an earlier block
-                assert last_read[s] < 0 or last_read[s] // SYNC_STEPS < t // SYNC_STEPS, \
+                assert last_read[s] < 0 or last_read[s] // sync < t // sync, \
                     f"step {t}: slot {s} rewritten in the block of its last read"
                 assert ((int(entries[t, w, 1]) >> 24) & 1) == n_written[s] % 2, f"step {t} lane {w}: write parity"
                 n_written[s] += 1

@@ -51,12 +51,13 @@ def check_programs(emo, oracle_mod, g, lv, flags=0, group_of=None):
     assert info.n == g.n and info.m == g.m and info.L == g.L
     r = oracle_mod.batch(g, lv, want_arrays=True, group_of=group_of)
     lanes, steps, slots, Lp, ent, rows, lat = emo.emo_graph_program(h, 0)
-    f = PE.run(ent, rows, lat, Lp, g.L, slots, lv, g.n, False)
+    assert info.sync_fwd in (8, 16, 32) and info.sync_bwd in (8, 16, 32)
+    f = PE.run(ent, rows, lat, Lp, g.L, slots, lv, g.n, False, sync=info.sync_fwd)
     assert (f["seen"] == 1).all()
     assert np.array_equal(f["T"], r["makespan"])
     assert np.array_equal(f["ES"], r["ES"])
     lanes_b, steps_b, slots_b, Lp_b, ent_b, rows_b, lat_b = emo.emo_graph_program(h, 1)
-    b = PE.run(ent_b, rows_b, lat_b, Lp_b, g.L, slots_b, lv, g.n, True, ES_in=f["ES"], T_in=f["T"])
+    b = PE.run(ent_b, rows_b, lat_b, Lp_b, g.L, slots_b, lv, g.n, True, ES_in=f["ES"], T_in=f["T"], sync=info.sync_bwd)
     assert (b["seen"] == 1).all()
     # forward entries address the row of the backward program that handles the same node
     pos_b = {}
@@ -67,8 +68,8 @@ def check_programs(emo, oracle_mod, g, lv, flags=0, group_of=None):
     assert all(pos_b[node] == row for node, row in f["main_rows"])
     assert all(node == row for node, row in b["main_rows"])
     # runs of simple entries: the stored length counts the simple entries that follow in the same
-    # column, never crosses a block of SYNC_STEPS steps and keeps one level mask
-    for ent_x in (ent, ent_b):
+    # column (15 at most), never crosses a block of the program's barrier distance and keeps one level mask
+    for ent_x, sync_x in ((ent, info.sync_fwd), (ent_b, info.sync_bwd)):
         fl = ent_x[:, :, 1].astype(np.int64)
         S_, W_ = fl.shape
         for w in range(W_):
@@ -78,13 +79,13 @@ def check_programs(emo, oracle_mod, g, lv, flags=0, group_of=None):
                 assert bool(f >> 31) == bool(simple)
                 if simple:
                     run = (f >> 16) & 15
-                    assert 1 <= run <= PE.SYNC_STEPS - (t % PE.SYNC_STEPS)
+                    assert 1 <= run <= min(15, sync_x - (t % sync_x))
                     for k in range(1, run):
                         g2 = int(fl[t + k, w])
-                        assert (g2 >> 31) and ((g2 >> 16) & 15) == run - k and ((g2 >> 8) & 255) == ((f >> 8) & 255)
+                        assert (g2 >> 31) and ((g2 >> 16) & 15) >= run - k and ((g2 >> 8) & 255) == ((f >> 8) & 255)
     # runs of plain entries (word 5): register operand only, a real node; the forward program also
     # excludes entries that write a slot or end a path
-    for ent_x, bwd_x in ((ent, False), (ent_b, True)):
+    for ent_x, bwd_x, sync_x in ((ent, False, info.sync_fwd), (ent_b, True, info.sync_bwd)):
         fl = ent_x[:, :, 1].astype(np.int64)
         runs = ent_x[:, :, 5].astype(np.int64)
         S_, W_ = fl.shape
@@ -97,7 +98,7 @@ def check_programs(emo, oracle_mod, g, lv, flags=0, group_of=None):
                     plain = False
                 want = 0
                 if plain:
-                    want = nxt + 1 if (t + 1) % PE.SYNC_STEPS != 0 else 1
+                    want = min(nxt + 1, 15) if (t + 1) % sync_x != 0 else 1
                 assert int(runs[t, w]) == want
                 nxt = want
     assert np.array_equal(b["LS"], r["LS"])
