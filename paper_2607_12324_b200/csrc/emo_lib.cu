@@ -573,17 +573,20 @@ int emo_graph_load(int32_t n, const int64_t *row_ptr, const int32_t *col, const 
         // backward first: the forward entries name the row of the backward program that will read
         // the node's earliest start
         // (each direction picks its own number of lanes from its ops and depth unless one is forced)
-        // The distance between the group barriers: 16 steps where that costs few slots (a barrier
-        // makes every warp of a group wait for the slowest), else 8 (slots take shared memory from
-        // the stages).  Measured on the 250 000-node workload: forward 18 -> 25 slots and 11.2 -> 10.3 ms
-        // with 16, backward 82 -> 120 slots and 20.4 -> 24.5 ms.
+        // The distance between the group barriers: the longest of 32, 16, 8 steps that costs few slots
+        // (a barrier makes every warp of a group wait for the slowest; slots take shared memory from
+        // the stages).  Measured on the 250 000-node workload: forward 18 / 26 / 37 slots and
+        // 11.2 / 10.5 / 10.0 ms with 8 / 16 / 32, backward 82 slots and 20.4 ms with 8, 24.5 ms with 16.
         auto compile_dir = [&](bool backward, const std::vector<uint32_t> *row_in_other, Program &out) {
-            int rc = compile_program(h, lat, energy, backward, lanes, look, 16, row_in_other, out, err);
-            if (rc == EMO_E_UNSUPPORTED || (rc == EMO_OK && out.slots > kManySlots)) {
-                Program tight;
-                const int rc8 = compile_program(h, lat, energy, backward, lanes, look, 8, row_in_other, tight, err);
-                if (rc8 == EMO_OK) out = std::move(tight);
-                rc = rc8;
+            int rc = EMO_E_UNSUPPORTED;
+            for (int sync = 32; sync >= 8; sync /= 2) {
+                Program cand;
+                rc = compile_program(h, lat, energy, backward, lanes, look, sync, row_in_other, cand, err);
+                if (rc != EMO_OK && rc != EMO_E_UNSUPPORTED) return rc;
+                if (rc == EMO_OK && (cand.slots <= kManySlots || sync == 8)) {
+                    out = std::move(cand);
+                    return EMO_OK;
+                }
             }
             return rc;
         };
