@@ -313,11 +313,13 @@ def main():
 
     if rank == 0 and not args.no_cpu:
         threads = os.cpu_count() or 1
-        cnt = max(threads, 16)
+        # a probe of a few policies per thread sizes the sample for about 15 s of CPU work
+        cnt = min(B, 8 * threads)
         cols = np.linspace(0, B - 1, cnt).astype(np.int64)
-        sub = lv[:, cols].contiguous().cpu().numpy()
-        t1 = oracle_sample(g, sub[:, :threads].copy(), threads)
-        cnt2 = int(min(B, max(threads, (12.0 / max(t1, 1e-3)) * threads)))
+        sub = lv[:, torch.as_tensor(cols, device="cuda")].contiguous().cpu().numpy()
+        oracle_sample(g, sub[:, :threads].copy(), threads)           # start the threads, touch the tables
+        t1 = oracle_sample(g, sub, threads)
+        cnt2 = int(min(B, max(threads, (15.0 / max(t1, 1e-3)) * cnt)))
         cols = np.linspace(0, B - 1, cnt2).astype(np.int64)
         sub = lv[:, torch.as_tensor(cols, device="cuda")].contiguous().cpu().numpy()
         t2 = oracle_sample(g, sub, threads)

@@ -472,7 +472,9 @@ int compile_program(const HostGraph &g, const int64_t *lat, const double *energy
     // Runs of plain entries for the one-policy-per-thread kernel (word 5).  An entry is plain when its
     // only operand is the warp's register and it handles a real node; forward it also writes no
     // slot and ends no path, backward it may write one (there nearly every node hands its value to
-    // the node that launched it).  Word 5 of a plain entry is the length of the run that starts at
+    // the node that launched it).  Forward, an idle entry counts as plain too (nothing is stored for
+    // it and its duration and energy are 0), so idle steps do not cut a run.
+    // Word 5 of a plain entry is the length of the run that starts at
     // it, inside one block of sync_steps steps and 15 at most; 0 for every other entry.
     for (int w = 0; w < lanes; ++w) {
         uint32_t next_run = 0;
@@ -481,6 +483,7 @@ int compile_program(const HostGraph &g, const int64_t *lat, const double *energy
             const uint32_t fl = en[1];
             bool plain = (fl & kValid) && (fl & kRegPred) && !(fl & kAux) && ((fl >> kNPredShift) & 7u) == 0;
             if (plain && !backward && (fl & (kWriteSlot | kTerminal))) plain = false;
+            if (!backward && !(fl & kValid)) plain = true;
             uint32_t run = 0;
             if (plain) run = ((s + 1) % sync_steps != 0) ? std::min<uint32_t>(next_run + 1, 15u) : 1;
             en[5] = run;

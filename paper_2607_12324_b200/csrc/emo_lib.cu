@@ -106,7 +106,10 @@ int upload_program_lane(const Program &p, DevProgramLane &d)
         if (q >= Q) continue;
         const uint32_t *en = &p.entries[q * kEntryWords];
         const uint32_t fl = en[1];
-        if (!(fl & kValid)) continue;
+        if (!(fl & kValid)) {
+            w[1] |= (en[5] & 15u) << kLaneRunShift;      // forward: an idle entry may sit inside a run
+            continue;
+        }
         const uint32_t np = (fl >> kNPredShift) & 7u;
         const uint32_t out = (fl & kWriteSlot) ? ((fl >> kOutShift) & 255u) : kLaneNoSlot;
         const uint32_t outpar = (fl & kWriteSlot) ? ((fl >> kOutParityShift) & 1u) : 0u;

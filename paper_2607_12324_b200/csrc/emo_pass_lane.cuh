@@ -117,8 +117,9 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_lane(LaneParams ip)
         // is written either)
         auto simple = [&](const EmoLaneFetched &f) {
             if (!BWD) {
-                if (spill_lane) *emo_row_ptr(spill_lane, f.e.x, spill8) = h;
-                if (EXTRA && es_lane) *emo_row_ptr(es_lane, emo_lds_u32(ent_a - d_ent + 20u), ldes8) = h;
+                // (an idle entry inside a run: row kNone, nothing stored, duration and energy 0)
+                emo_stg_row_if(spill_lane, f.e.x, spill8, h, spill_ok);
+                if (EXTRA && es_lane && f.e.x != emo::kNone) *emo_row_ptr(es_lane, emo_lds_u32(ent_a - d_ent + 20u), ldes8) = h;
                 ea += f.g;
                 h = emo_add_dur(h, f.d);
             } else {

@@ -96,6 +96,8 @@ def check_programs(emo, oracle_mod, g, lv, flags=0, group_of=None):
                 plain = (f & 1) and (f & 2) and not (f & 0x80) and ((f >> 4) & 7) == 0
                 if plain and not bwd_x and (f & (4 | 8)):
                     plain = False
+                if not bwd_x and not (f & 1):
+                    plain = True          # forward: idle entries do not cut a run
                 want = 0
                 if plain:
                     want = min(nxt + 1, 15) if (t + 1) % sync_x != 0 else 1
