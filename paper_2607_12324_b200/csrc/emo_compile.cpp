@@ -404,10 +404,12 @@ int compile_program(const HostGraph &g, const int64_t *lat, const double *energy
             uint32_t flags = kValid;
             uint32_t operands = 0, operands_hi = 0;
             int np = 0;
+            bool settled = true;      // every slot operand was written before the group's last barrier
             for (int32_t p : o.preds) {
                 if (warp_of[p] == w && prev_on_warp[i] == p) {
                     flags |= kRegPred;
                 } else {
+                    settled = settled && step_of[p] / sync_steps < s / sync_steps;
                     if (np < 4) operands |= (uint32_t)slot_of[p] << (8 * np);
                     else operands_hi |= (uint32_t)slot_of[p] << (8 * (np - 4));
                     flags |= (uint32_t)parity_of[p] << (kOperandParityShift + np);
@@ -445,6 +447,9 @@ int compile_program(const HostGraph &g, const int64_t *lat, const double *energy
             en[1] = flags;
             en[2] = operands;
             en[3] = operands_hi;
+            // word 6: 1 when the entry has slot operands and all of them are settled - the barrier the
+            // group passed since has ordered the writes before this read, so no slot needs polling
+            en[6] = (np > 0 && settled) ? 1u : 0u;
         }
     }
     // Runs of simple entries.  An entry is simple when its only operand is the warp's register and

@@ -25,7 +25,8 @@ constexpr int kMaxLanes = 32;
 // array (kNone for helper ops and idle entries); word 1 = flags; word 2 = operand slots 0..3,
 // word 3 = operand slots 4..5 (8 bits each); word 4 = node id in the caller's numbering (kNone for
 // helper ops and idle entries); word 5 = length of the run of plain entries that starts here (see
-// emo_compile.cpp; 0 = not plain); words 6..7 unused.
+// emo_compile.cpp; 0 = not plain); word 6 = 1 when every slot operand was written before the last
+// barrier of the group (no need to poll); word 7 unused.
 constexpr int kEntryWords = 8;
 constexpr uint32_t kValid = 1u, kRegPred = 2u, kWriteSlot = 4u, kTerminal = 8u, kAux = 0x80u;
 constexpr int kNPredShift = 4;        // bits 4..6: number of slot operands

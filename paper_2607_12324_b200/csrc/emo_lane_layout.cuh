@@ -6,7 +6,8 @@
 //                        none) | number of slot operands (bits 8..10) | terminal (bit 11) | phase
 //                        parity of the value written (bit 12) and of each operand (bits 13..18) |
 //                        idle (bit 19) | length of the run of plain entries that starts here
-//                        (bits 20..23; see emo_compile.cpp); word 2 = mask applied to the lane's running value (0 =
+//                        (bits 20..23; see emo_compile.cpp) | every slot operand was written before
+//                        the group's last barrier, none needs polling (bit 24); word 2 = mask applied to the lane's running value (0 =
 //                        start from 0, ~0 = continue from the lane's last node); word 3 = operand
 //                        slots 0..3; word 4 = operand slots 4..5; word 5 = node id
 //   table  [Q][Lp]       forward: {duration, high word of the energy, low word} in 12 bytes per
@@ -19,7 +20,7 @@
 
 constexpr int kLaneStepPad = 32;                 // programs are padded to a multiple of this many steps (the longest stage)
 constexpr unsigned kLaneNoSlot = 255u;
-constexpr unsigned kLaneNpShift = 8, kLaneTerminal = 0x800u, kLaneOutParShift = 12, kLaneOpParShift = 13, kLaneIdle = 1u << 19, kLaneRunShift = 20;
+constexpr unsigned kLaneNpShift = 8, kLaneTerminal = 0x800u, kLaneOutParShift = 12, kLaneOpParShift = 13, kLaneIdle = 1u << 19, kLaneRunShift = 20, kLaneSettled = 1u << 24;
 
 // offsets of the areas of one stage (records first, then what emo_produce addresses)
 struct LaneStage {

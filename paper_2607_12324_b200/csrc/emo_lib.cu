@@ -117,6 +117,7 @@ int upload_program_lane(const Program &p, DevProgramLane &d)
         w[0] = en[0];
         w[1] = out | (np << kLaneNpShift) | ((fl & kTerminal) ? kLaneTerminal : 0u) | (outpar << kLaneOutParShift) | (oppar << kLaneOpParShift);
         w[1] |= (en[5] & 15u) << kLaneRunShift;
+        if (en[6] & 1u) w[1] |= kLaneSettled;
         w[2] = (fl & kRegPred) ? 0xFFFFFFFFu : 0u;
         w[3] = en[2];
         w[4] = en[3];

@@ -158,7 +158,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_lane(LaneParams ip)
                     // straight-line: poll the four barriers, load the four values, take the maxima
                     const unsigned b0 = slotbar_base + (ops & 255u) * kLaneSlotStride, b1 = slotbar_base + ((ops >> 8) & 255u) * kLaneSlotStride,
                                    b2 = slotbar_base + ((ops >> 16) & 255u) * kLaneSlotStride, b3 = slotbar_base + (ops >> 24) * kLaneSlotStride;
-                    if (!emo_mbar_test4(b0, b1, b2, b3, par)) {
+                    if (!(fl & kLaneSettled) && !emo_mbar_test4(b0, b1, b2, b3, par)) {
                         if (!emo_slot_wait(b0, par & 1u, my_abort) || !emo_slot_wait(b1, (par >> 1) & 1u, my_abort) ||
                             !emo_slot_wait(b2, (par >> 2) & 1u, my_abort) || !emo_slot_wait(b3, (par >> 3) & 1u, my_abort)) {
                             *my_abort = 1;
@@ -204,7 +204,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_lane(LaneParams ip)
                     for (unsigned k = 0; k < np; ++k) {
                         if (k == 4) ops = emo_lds_u32(ent + 16u);
                         const unsigned bar = slotbar_base + (ops & 255u) * kLaneSlotStride;
-                        if (!emo_mbar_test(bar, par & 1u) && !emo_slot_wait(bar, par & 1u, my_abort)) {
+                        if (!(fl & kLaneSettled) && !emo_mbar_test(bar, par & 1u) && !emo_slot_wait(bar, par & 1u, my_abort)) {
                             *my_abort = 1;
                             dead = true;
                             return;
@@ -223,8 +223,9 @@ __global__ void __launch_bounds__(MAXT, 1) emo_pass_lane(LaneParams ip)
                 ea += f.g;
             }
             v = emo_add_dur(v, f.d);
-            {
-                // slot write without a branch: store under a predicate, then lane 0 reports the value
+            if (!BWD || (fl & 255u) != kLaneNoSlot) {
+                // slot write: store under a predicate, then lane 0 reports the value (backward: a
+                // launch node writes nothing and skips this)
                 const unsigned out = fl & 255u;
                 const unsigned bar = slotbar_base + out * kLaneSlotStride;
                 emo_sts_s64_if(bar + lane8, v, out, kLaneNoSlot);

@@ -22,6 +22,7 @@ def run(entries, rows, lat, Lp, L, slots, lvl, n, backward, ES_in=None, T_in=Non
     slot_valid = np.zeros(max(slots, 1), dtype=bool)
     n_written = np.zeros(max(slots, 1), dtype=np.int64)      # values written to a slot so far
     last_read = np.full(max(slots, 1), -1, dtype=np.int64)
+    write_step = np.full(max(slots, 1), -1, dtype=np.int64)
     seen = np.zeros(n, dtype=np.int64)
     out = {}
     if not backward:
@@ -50,14 +51,18 @@ def run(entries, rows, lat, Lp, L, slots, lvl, n, backward, ES_in=None, T_in=Non
             dur = lat[q][lv.astype(np.int64) & mask].astype(np.int64)
             start = h[w].copy() if flags & REGPRED else np.zeros(B, dtype=np.int64)
             ops |= ops_hi << 32
+            settled = ((flags >> 4) & 7) > 0
             for k in range((flags >> 4) & 7):
                 s = (ops >> (8 * k)) & 255
+                settled = settled and write_step[s] // sync < t // sync
                 assert slot_valid[s], f"step {t} lane {w} reads slot {s} before any write"
                 # the parity in the entry names the value that is in the slot now
                 assert ((flags >> (25 + k)) & 1) == (n_written[s] - 1) % 2, f"step {t} lane {w}: operand parity"
                 last_read[s] = t
                 read_ids.add(s)
                 start = np.maximum(start, slot[s])
+            # word 6: every slot operand was written before the group's last barrier
+            assert (int(entries[t, w][6]) & 1) == int(settled), f"step {t} lane {w}: settled flag"
             val = start + dur
             if node != NONE:
                 seen[node] += 1
@@ -84,6 +89,7 @@ def run(entries, rows, lat, Lp, L, slots, lvl, n, backward, ES_in=None, T_in=Non
                 n_written[s] += 1
                 slot[s] = val
                 slot_valid[s] = True
+                write_step[s] = t
     out["seen"] = seen
     out["main_rows"] = main_rows
     if not backward:
