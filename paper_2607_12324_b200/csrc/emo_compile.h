@@ -5,9 +5,10 @@
 // predecessors (Eq. 1: C_v = t_v + max over predecessors of C_k), adds the node's duration and keeps
 // the result in a register.  A value another warp (or a later, non-adjacent step of the same warp)
 // needs is also written to a numbered exchange slot in shared memory.  All predecessors of a node
-// are handled in strictly earlier steps and the warps of a group meet at a barrier after every
-// step, so a slot is always written before it is read.  The backward pass (latest start times) runs
-// the same machinery on the reversed graph.
+// are handled in strictly earlier steps.  The plain kernel runs the warps of a group in lockstep (a
+// barrier after every step); the staged kernels let them drift: a reader polls the barrier of the
+// slot it reads, the group meets only every `sync` steps, and a slot is reused only across such a
+// meeting.  The backward pass (latest start times) runs the same machinery on the reversed graph.
 #pragma once
 #include <cstdint>
 #include <string>

@@ -1,13 +1,16 @@
-// Staged pass kernel (sm_100a): the step interpreter with everything a step reads brought into
-// shared memory by one producer warp with bulk asynchronous copies (TMA, cp.async.bulk) through a
+// What the staged pass kernels share (PTX helpers, stage parameters, the producer emo_produce) and the
+// staged pass kernel with two policies per thread, emo_pass_pair (sm_100a).
+//
+// A staged kernel is the step interpreter with everything a step reads brought into shared memory
+// by producer warps with bulk asynchronous copies (TMA, cp.async.bulk) through a
 // ring of stages guarded by full/empty mbarriers: the program records (entry + duration row +
 // energy row) of a run of steps in one bulk copy, (backward) the earliest-start rows of those steps
 // in a second bulk copy, and the level rows of the block's policy tile, which lie scattered in the
-// caller's matrix, as 16-byte cp.async pieces issued by all lanes of the producer warp (a bulk copy
+// caller's matrix, as 16-byte cp.async pieces issued by all lanes of the producer warps (a bulk copy
 // per 128-byte row costs far more than it moves).  Each record and each level row is fetched once
 // per block and used by every policy of the block.
 //
-// A consumer thread carries TWO adjacent policies, so a warp covers 64 policies of one schedule
+// In emo_pass_pair a consumer thread carries TWO adjacent policies, so a warp covers 64 policies of one schedule
 // lane: the entry decode and the address arithmetic are paid once per pair, the level pair is one
 // 16-bit load, an exchange slot holds both values and moves with one 128-bit access, and the
 // per-node outputs leave as 128-bit stores.
