@@ -298,7 +298,7 @@ bool lane_shape(const emo_graph *g, const Program &p, bool backward, int64_t NB,
 // spill) or both with the plain kernels (through an [n][ldes] array).
 struct PassPlan {
     bool staged = false;
-    bool lane = false;        // staged, one policy per thread (program in the padded layout)
+    bool lane_f = false, lane_b = false;   // staged, one policy per thread (forward / backward pass)
     LaunchShape sf, sb;       // forward / backward launch shapes
     StagedParams pf, pb;
     size_t spill_bytes = 0;   // tiled spill: [tiles][rows of the backward program][backward tile]
@@ -325,10 +325,24 @@ int make_plan(const emo_graph *g, int64_t B, bool want_base, bool need_bwd, cons
     // 0.24 ms against 0.42 ms for the forward pass).
     const int64_t pair_warps = (NBf + 63) / 64 * std::max(g->fwd.lanes, g->bwd.lanes);
     const bool prefer_pair = (flags & EMO_F_PAIR_KERNEL) || (!(flags & EMO_F_LANE_KERNEL) && pair_warps >= 16 * (int64_t)g->sm_count);
-    if (can_stage && !prefer_pair)
-        pl.lane = lane_shape(g, g->fwd, false, NBf, pl.sf, pl.pf) && (!need_bwd || lane_shape(g, g->bwd, true, B, pl.sb, pl.pb));
-    pl.staged = pl.lane || (can_stage && staged_shape(g, g->fwd, g->dfwd.rec_bytes, false, NBf, pl.sf, pl.pf) &&
-                           (!need_bwd || staged_shape(g, g->bwd, g->dbwd.rec_bytes, true, B, pl.sb, pl.pb)));
+    // Each pass picks its kernel (they only share the spill, whose tiling follows the backward pass).
+    // A pass whose lane-kernel grid would need a second wave of blocks while the pair kernel's fits
+    // the SMs once takes the pair kernel (a wide forward program: 18 lanes leave room for one group
+    // of 32 policies per block; measured 2.7 ms against 4.5 ms).
+    auto pick = [&](const Program &p, int rec_bytes, bool backward, int64_t NB, LaunchShape &ls, StagedParams &sp, bool &lane) {
+        LaunchShape l1, l2;
+        StagedParams s1, s2;
+        const bool ok_lane = lane_shape(g, p, backward, NB, l1, s1);
+        const bool ok_pair = staged_shape(g, p, rec_bytes, backward, NB, l2, s2);
+        bool use_lane = ok_lane && !prefer_pair;
+        if (use_lane && ok_pair && !(flags & EMO_F_LANE_KERNEL) && !backward && l1.grid > g->sm_count && l2.grid <= g->sm_count) use_lane = false;
+        if (!use_lane && !ok_pair) use_lane = ok_lane;
+        if (use_lane) { ls = l1; sp = s1; lane = true; return true; }
+        if (ok_pair) { ls = l2; sp = s2; lane = false; return true; }
+        return false;
+    };
+    pl.staged = can_stage && pick(g->fwd, g->dfwd.rec_bytes, false, NBf, pl.sf, pl.pf, pl.lane_f) &&
+                (!need_bwd || pick(g->bwd, g->dbwd.rec_bytes, true, B, pl.sb, pl.pb, pl.lane_b));
     if (!pl.staged) {
         int rc = shape_for(g, g->fwd, NBf, pl.sf);
         if (rc == EMO_OK && need_bwd) rc = shape_for(g, g->bwd, B, pl.sb);
@@ -336,7 +350,7 @@ int make_plan(const emo_graph *g, int64_t B, bool want_base, bool need_bwd, cons
     }
     if (need_bwd) {
         const size_t tiles = ((size_t)B + pl.pb.ptile - 1) / pl.pb.ptile;
-        pl.spill_bytes = tiles * spill_rows_of(g, pl.lane) * pl.pb.ptile * sizeof(int64_t);
+        pl.spill_bytes = tiles * spill_rows_of(g, pl.lane_b) * pl.pb.ptile * sizeof(int64_t);
     }
     return EMO_OK;
 }
@@ -371,7 +385,7 @@ int launch_pass(const emo_graph *g, const PassPlan &pl, bool backward, int64_t B
     a.ES = ES;
     a.ldes = ldes;
     a.spill = spill;
-    a.spill_rows = (int64_t)spill_rows_of(g, pl.lane);
+    a.spill_rows = (int64_t)spill_rows_of(g, pl.lane_b);
     a.spill_ptile = pl.staged ? pl.pb.ptile : 64;
     a.LS = LS;
     a.slack = slack;
@@ -396,7 +410,7 @@ int launch_pass(const emo_graph *g, const PassPlan &pl, bool backward, int64_t B
         // matrix with 16-byte aligned rows (backward); register budget by block size
         const bool extra = backward ? (LS != nullptr || sp.want_sums || !sp.vec_out) : (ES != nullptr);
         void (*kern)(StagedParams) = nullptr;
-        if (pl.lane) {
+        if (backward ? pl.lane_b : pl.lane_f) {
             const DevProgramLane &di = backward ? g->lbwd : g->lfwd;
             LaneParams ip;
             const unsigned ne = (unsigned)sp.sc * (unsigned)p.lanes;
