@@ -353,6 +353,29 @@ def test_batch_edge_cases(torch_cuda, emo, oracle_mod):
     h0.free()
 
 
+def test_many_levels(torch_cuda, emo, oracle_mod):
+    """200 frequency levels (table rows of 256 entries, far wider than the 32 shared-memory banks),
+    non-monotone rows, a ragged batch; every pass kernel."""
+    torch = torch_cuda
+    L, n, B = 200, 60, 77
+    rs = np.random.RandomState(11)
+    edges = [(i, j) for i in range(n) for j in range(i + 1, min(n, i + 6)) if rs.rand() < 0.4]
+    lat = rs.randint(0, 5000, (n, L)).astype(np.int64)
+    en = rs.rand(n, L) * 3.0
+    g = W.tiny_graph(n, edges, lat, en)
+    lv = rs.randint(0, L, (n, B)).astype(np.uint8)
+    r_or = oracle_mod.batch(g, lv, want_arrays=True)
+    ldb = 96
+    lvp = np.full((n, ldb), 0xFF, dtype=np.uint8)
+    lvp[:, :B] = lv
+    lv_dev = torch.as_tensor(lvp, device="cuda")
+    h = emo.load_workload(g)
+    for fl in (emo.EMO_F_NO_STAGING, emo.EMO_F_PAIR_KERNEL, emo.EMO_F_LANE_KERNEL, 0):
+        r = gpu_slack_batch(torch, emo, h, lv_dev, B, n, flags=fl, base=True)
+        assert_matches(r, r_or, B)
+    h.free()
+
+
 def test_group_of_on_gpu(torch_cuda, emo, oracle_mod):
     torch = torch_cuda
     g = W.make_graph("cfg1-train", 0.1)
