@@ -48,6 +48,8 @@ extern "C" {
 #define EMO_F_HOST_ONLY 0x1u       /* build the handle without touching a device (inspection) */
 #define EMO_F_LANES(c) (((uint32_t)(c) & 0xFFu) << 8)      /* force c cooperating warps per policy group */
 #define EMO_F_LOOKAHEAD(d) (((uint32_t)(d) & 0xFFu) << 16) /* scheduling look-ahead in steps */
+#define EMO_F_FLOW_SYNC(s) ((((uint32_t)(s) / 8u) & 0xFu) << 4)  /* lane-stream program: steps between group barriers (8, 16, 32) */
+#define EMO_F_FLOW_STAGE(k) (((uint32_t)(k) & 0x3Fu) << 24)      /* lane-stream program: steps per stage (8, 16, 32) */
 /* flags of the evaluation calls */
 #define EMO_F_VALIDATE 0x1u        /* check every level < L first; EMO_E_RANGE goes to *status */
 #define EMO_F_NO_STAGING 0x2u      /* use the plain-load kernels instead of the staged ones */
@@ -247,6 +249,26 @@ int emo_set_pass_events(void *fwd_start, void *fwd_stop, void *bwd_start, void *
  */
 int emo_graph_program(const emo_graph *g, int dir, int32_t *lanes, int32_t *steps, int32_t *slots,
                       int32_t *Lp, const uint32_t **entries, const uint32_t **rows, const uint32_t **lat);
+
+/*
+ * Inspection of the lane-stream program that the 32-bit pass kernels walk (host memory owned by the
+ * handle; valid until emo_graph_free).  ok32 = 0 means the graph's spread of start times over all
+ * policies does not fit 32 bits (or it needs more than 30 lanes) and the 64-bit kernels serve it;
+ * the arrays are then empty.  Layouts: hdr [stages][lanes][4], rows / node / step [stages][lanes][K],
+ * tab_fwd [stages][lanes][K][Lp][3], tab_bwd [stages][lanes][K][Lp], rec_fwd [stages][lanes][K][4],
+ * rec_bwd [stages][lanes][K][8], pool_* [stages][pool_stride_*], lbes [stages][lanes][K],
+ * push_base [stages + 1].  Used by host-side tests of the compiler; not needed to evaluate anything.
+ */
+typedef struct emo_flow_view {
+    int32_t ok32, lanes, K, sync, stages, steps, Lp;
+    int32_t slots_tag_fwd, slots_set_fwd, pool_stride_fwd;
+    int32_t slots_tag_bwd, slots_set_bwd, pool_stride_bwd;
+    int64_t pushes, pruned_fwd, pruned_bwd;
+    const uint32_t *hdr, *rows, *node, *step, *tab_fwd, *tab_bwd;
+    const uint32_t *rec_fwd, *pool_fwd, *rec_bwd, *pool_bwd;
+    const int64_t *lbes, *push_base;
+} emo_flow_view;
+int emo_graph_flow(const emo_graph *g, emo_flow_view *out);
 
 #ifdef __cplusplus
 }

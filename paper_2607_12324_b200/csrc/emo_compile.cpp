@@ -67,6 +67,204 @@ int pick_lanes(int64_t n_ops, int depth)
     return (int)c;
 }
 
+// Target steps and list scheduling of ops (given by their operand lists, in a topological order)
+// onto `lanes` warps.  On return step_of / warp_of give every op's place, prev_on_warp the op the
+// same warp handled just before it (-1: none), S the number of steps.
+int schedule_ops(const std::vector<std::vector<int32_t>> &preds, int lanes, int lookahead, std::vector<int32_t> &step_of,
+                 std::vector<int32_t> &warp_of, std::vector<int32_t> &prev_on_warp, int32_t &S_out, int &lanes_out,
+                 std::string &err)
+{
+    const int32_t N = (int32_t)preds.size();
+    // consumers of each op
+    std::vector<int64_t> cp((size_t)N + 1, 0);
+    for (int32_t i = 0; i < N; ++i)
+        for (int32_t p : preds[i]) cp[p + 1]++;
+    for (int32_t i = 0; i < N; ++i) cp[i + 1] += cp[i];
+    std::vector<int32_t> cons((size_t)std::max<int64_t>(cp[N], 1));
+    {
+        std::vector<int64_t> f(cp.begin(), cp.end() - 1);
+        for (int32_t i = 0; i < N; ++i)
+            for (int32_t p : preds[i]) cons[f[p]++] = i;
+    }
+
+    // hop levels: earliest step (asap) and the number of hops to the end (rem; alap = D - rem)
+    std::vector<int32_t> asap((size_t)N, 0), rem((size_t)N, 1), tgt((size_t)N, 0);
+    int32_t D = 0;
+    for (int32_t i = 0; i < N; ++i) {
+        int32_t a = 0;
+        for (int32_t p : preds[i]) a = std::max(a, asap[p] + 1);
+        asap[i] = a;
+        D = std::max(D, a + 1);
+    }
+    for (int32_t i = N - 1; i >= 0; --i) {
+        int32_t r = 1;
+        for (int64_t e = cp[i]; e < cp[i + 1]; ++e) r = std::max(r, rem[cons[e]] + 1);
+        rem[i] = r;
+    }
+    // Target steps.  A value occupies an exchange slot from the step that produces it to the step
+    // of its last consumer, so the targets are moved, within the precedence constraints, to
+    // shorten the summed lifetimes: starting from the earliest steps, a backward sweep moves an op
+    // later (next to its earliest consumer) when that shortens its own value's life by more than
+    // it stretches its operands' lives, and a forward sweep moves an op earlier under the mirrored
+    // test.  This puts a chain that has hop slack (a launch chain running ahead of the kernels, or
+    // short streams beside a long launch chain) next to the ops it exchanges values with.
+    // Two starting points are refined, all ops at their earliest and all at their latest steps,
+    // and the one with the smaller summed lifetime is kept.
+    auto last_cons_excl = [&](int32_t p, int32_t skip) {
+        int32_t m = -1;
+        for (int64_t e = cp[p]; e < cp[p + 1]; ++e)
+            if (cons[e] != skip) m = std::max(m, tgt[cons[e]]);
+        return m;
+    };
+    auto sweep_later = [&]() {
+        for (int32_t i = N - 1; i >= 0; --i) {
+            if (cp[i + 1] == cp[i]) continue;
+            int32_t hi = INT32_MAX;
+            for (int64_t e = cp[i]; e < cp[i + 1]; ++e) hi = std::min(hi, tgt[cons[e]] - 1);
+            if (hi <= tgt[i]) continue;
+            int64_t gain = hi - tgt[i], cost = 0;
+            for (int32_t p : preds[i]) {
+                if (cp[p + 1] - cp[p] == 1) continue;   // its only consumer: it follows later in this sweep
+                int32_t other = last_cons_excl(p, i);
+                cost += std::max(other, hi) - std::max(other, tgt[i]);
+            }
+            if (gain > cost) tgt[i] = hi;
+        }
+    };
+    auto sweep_earlier = [&]() {
+        for (int32_t i = 0; i < N; ++i) {
+            if (preds[i].empty()) continue;
+            int32_t lo = 0;
+            for (int32_t p : preds[i]) lo = std::max(lo, tgt[p] + 1);
+            if (lo >= tgt[i]) continue;
+            bool held = false;   // a consumer with other operands keeps this op's value alive
+            for (int64_t e = cp[i]; e < cp[i + 1]; ++e) held |= preds[cons[e]].size() > 1;
+            int64_t cost = held ? tgt[i] - lo : 0, gain = 0;
+            for (int32_t p : preds[i]) {
+                int32_t other = last_cons_excl(p, i);
+                gain += std::max(other, tgt[i]) - std::max(other, lo);
+            }
+            if (gain > cost) tgt[i] = lo;
+        }
+    };
+    auto total_life = [&]() {
+        int64_t sum = 0;
+        for (int32_t i = 0; i < N; ++i) {
+            int32_t m = last_cons_excl(i, -1);
+            if (m >= 0) sum += m - tgt[i];
+        }
+        return sum;
+    };
+    tgt = asap;
+    for (int round = 0; round < 2; ++round) { sweep_later(); sweep_earlier(); }
+    const int64_t life_early = total_life();
+    std::vector<int32_t> tgt_early = tgt;
+    for (int32_t i = 0; i < N; ++i) tgt[i] = D - rem[i];
+    for (int round = 0; round < 2; ++round) { sweep_earlier(); sweep_later(); }
+    if (life_early <= total_life()) tgt.swap(tgt_early);
+    if (lanes <= 0) lanes = pick_lanes(N, D);
+    if (lanes > kMaxLanes) lanes = kMaxLanes;
+    if (lookahead <= 0) lookahead = 8;
+    lanes_out = lanes;
+
+    // ---- list scheduling ----------------------------------------------------------------------
+    // Priority: smallest target step first (ties: the more critical op).  An op is not started more
+    // than `lookahead` steps before its target step, which keeps a cheap chain from running far
+    // ahead of the ops that consume its values.
+    step_of.assign((size_t)N, -1);
+    warp_of.assign((size_t)N, -1);
+    prev_on_warp.assign((size_t)N, -1);
+    std::vector<int32_t> left((size_t)N);
+    std::vector<int32_t> unsched_cons((size_t)N);
+    using Key = std::pair<int64_t, int32_t>;   // (target step, alap | op)
+    std::priority_queue<Key, std::vector<Key>, std::greater<Key>> ready;
+    auto prio = [&](int32_t i) { return ((int64_t)tgt[i] << 32) | (uint32_t)(D - rem[i]); };
+    for (int32_t i = 0; i < N; ++i) {
+        left[i] = (int32_t)preds[i].size();
+        unsched_cons[i] = (int32_t)(cp[i + 1] - cp[i]);
+        if (left[i] == 0) ready.push({prio(i), i});
+    }
+    std::vector<int32_t> last((size_t)lanes, -1);
+    std::vector<std::vector<int32_t>> sched;   // per step: op per warp (-1 idle)
+    std::vector<int32_t> chosen, next_ready;
+    int32_t done = 0;
+    int32_t t = 0;
+    while (done < N) {
+        chosen.clear();
+        while (!ready.empty() && (int)chosen.size() < lanes) {
+            Key k = ready.top();
+            // an op that is not due yet waits, unless the step would otherwise be empty
+            if ((k.first >> 32) > t + lookahead && !chosen.empty()) break;
+            ready.pop();
+            chosen.push_back(k.second);
+        }
+        std::vector<int32_t> row((size_t)lanes, -1);
+        std::vector<char> placed(chosen.size(), 0);
+        // first the ops whose operand sits in a free warp's register.  Where several operands do,
+        // the op follows the one with the fewest readers: a value with one reader that travels in a
+        // register is never written to a slot, and a serial chain (the launch chain, whose nodes
+        // each have one chain successor but also read several kernels) stays on one warp instead
+        // of hopping from warp to warp with a slot hand-over on its critical path every step.
+        for (size_t j = 0; j < chosen.size(); ++j) {
+            int32_t i = chosen[j];
+            int best_w = -1;
+            int64_t best_fan = 0;
+            for (int32_t p : preds[i]) {
+                int w = warp_of[p];
+                if (w >= 0 && last[w] == p && row[w] < 0) {
+                    const int64_t fan = cp[p + 1] - cp[p];
+                    if (best_w < 0 || fan < best_fan) {
+                        best_w = w;
+                        best_fan = fan;
+                    }
+                }
+            }
+            if (best_w >= 0) {
+                row[best_w] = i;
+                placed[j] = 1;
+            }
+        }
+        // then the rest: prefer a warp whose register value nobody is waiting for
+        for (size_t j = 0; j < chosen.size(); ++j) {
+            if (placed[j]) continue;
+            int best = -1;
+            for (int w = 0; w < lanes; ++w) {
+                if (row[w] >= 0) continue;
+                bool dead = last[w] < 0 || unsched_cons[last[w]] == 0;
+                if (dead) { best = w; break; }
+                if (best < 0) best = w;
+            }
+            row[best] = chosen[j];
+        }
+        next_ready.clear();
+        for (int w = 0; w < lanes; ++w) {
+            int32_t i = row[w];
+            if (i < 0) continue;
+            step_of[i] = t;
+            warp_of[i] = w;
+            prev_on_warp[i] = last[w];
+            ++done;
+        }
+        for (int w = 0; w < lanes; ++w) {
+            int32_t i = row[w];
+            if (i < 0) continue;
+            last[w] = i;
+            for (int32_t p : preds[i]) unsched_cons[p]--;
+            for (int64_t e = cp[i]; e < cp[i + 1]; ++e)
+                if (--left[cons[e]] == 0) next_ready.push_back(cons[e]);
+        }
+        for (int32_t i : next_ready) ready.push({prio(i), i});
+        sched.push_back(std::move(row));
+        ++t;
+        if (chosen.empty() && ready.empty() && done < N) {
+            err = "scheduler stalled (graph is not acyclic?)";
+            return EMO_E_NOT_TOPOLOGICAL;
+        }
+    }
+    S_out = t;
+    return EMO_OK;
+}
+
 int compile_program(const HostGraph &g, const int64_t *lat, const double *energy, bool backward,
                     int lanes, int lookahead, int sync_steps, const std::vector<uint32_t> *row_in_other,
                     Program &out, std::string &err)
@@ -148,192 +346,23 @@ int compile_program(const HostGraph &g, const int64_t *lat, const double *energy
     const int32_t N = (int32_t)ops.size();
     out.aux = n_aux;
 
+    std::vector<std::vector<int32_t>> op_preds((size_t)N);
+    for (int32_t i = 0; i < N; ++i) op_preds[i] = ops[i].preds;
+    std::vector<int32_t> step_of, warp_of, prev_on_warp;
+    int32_t S = 0;
+    {
+        int rc = schedule_ops(op_preds, lanes, lookahead, step_of, warp_of, prev_on_warp, S, lanes, err);
+        if (rc != EMO_OK) return rc;
+    }
+    out.lanes = lanes;
+    out.steps = S;
+    std::vector<std::vector<int32_t>> sched((size_t)S, std::vector<int32_t>((size_t)lanes, -1));
+    for (int32_t i = 0; i < N; ++i) sched[step_of[i]][warp_of[i]] = i;
     // consumers of each op
     std::vector<int64_t> cp((size_t)N + 1, 0);
     for (int32_t i = 0; i < N; ++i)
         for (int32_t p : ops[i].preds) cp[p + 1]++;
     for (int32_t i = 0; i < N; ++i) cp[i + 1] += cp[i];
-    std::vector<int32_t> cons((size_t)std::max<int64_t>(cp[N], 1));
-    {
-        std::vector<int64_t> f(cp.begin(), cp.end() - 1);
-        for (int32_t i = 0; i < N; ++i)
-            for (int32_t p : ops[i].preds) cons[f[p]++] = i;
-    }
-
-    // hop levels: earliest step (asap) and the number of hops to the end (rem; alap = D - rem)
-    std::vector<int32_t> asap((size_t)N, 0), rem((size_t)N, 1), tgt((size_t)N, 0);
-    int32_t D = 0;
-    for (int32_t i = 0; i < N; ++i) {
-        int32_t a = 0;
-        for (int32_t p : ops[i].preds) a = std::max(a, asap[p] + 1);
-        asap[i] = a;
-        D = std::max(D, a + 1);
-    }
-    for (int32_t i = N - 1; i >= 0; --i) {
-        int32_t r = 1;
-        for (int64_t e = cp[i]; e < cp[i + 1]; ++e) r = std::max(r, rem[cons[e]] + 1);
-        rem[i] = r;
-    }
-    // Target steps.  A value occupies an exchange slot from the step that produces it to the step
-    // of its last consumer, so the targets are moved, within the precedence constraints, to
-    // shorten the summed lifetimes: starting from the earliest steps, a backward sweep moves an op
-    // later (next to its earliest consumer) when that shortens its own value's life by more than
-    // it stretches its operands' lives, and a forward sweep moves an op earlier under the mirrored
-    // test.  This puts a chain that has hop slack (a launch chain running ahead of the kernels, or
-    // short streams beside a long launch chain) next to the ops it exchanges values with.
-    // Two starting points are refined, all ops at their earliest and all at their latest steps,
-    // and the one with the smaller summed lifetime is kept.
-    auto last_cons_excl = [&](int32_t p, int32_t skip) {
-        int32_t m = -1;
-        for (int64_t e = cp[p]; e < cp[p + 1]; ++e)
-            if (cons[e] != skip) m = std::max(m, tgt[cons[e]]);
-        return m;
-    };
-    auto sweep_later = [&]() {
-        for (int32_t i = N - 1; i >= 0; --i) {
-            if (cp[i + 1] == cp[i]) continue;
-            int32_t hi = INT32_MAX;
-            for (int64_t e = cp[i]; e < cp[i + 1]; ++e) hi = std::min(hi, tgt[cons[e]] - 1);
-            if (hi <= tgt[i]) continue;
-            int64_t gain = hi - tgt[i], cost = 0;
-            for (int32_t p : ops[i].preds) {
-                if (cp[p + 1] - cp[p] == 1) continue;   // its only consumer: it follows later in this sweep
-                int32_t other = last_cons_excl(p, i);
-                cost += std::max(other, hi) - std::max(other, tgt[i]);
-            }
-            if (gain > cost) tgt[i] = hi;
-        }
-    };
-    auto sweep_earlier = [&]() {
-        for (int32_t i = 0; i < N; ++i) {
-            if (ops[i].preds.empty()) continue;
-            int32_t lo = 0;
-            for (int32_t p : ops[i].preds) lo = std::max(lo, tgt[p] + 1);
-            if (lo >= tgt[i]) continue;
-            bool held = false;   // a consumer with other operands keeps this op's value alive
-            for (int64_t e = cp[i]; e < cp[i + 1]; ++e) held |= ops[cons[e]].preds.size() > 1;
-            int64_t cost = held ? tgt[i] - lo : 0, gain = 0;
-            for (int32_t p : ops[i].preds) {
-                int32_t other = last_cons_excl(p, i);
-                gain += std::max(other, tgt[i]) - std::max(other, lo);
-            }
-            if (gain > cost) tgt[i] = lo;
-        }
-    };
-    auto total_life = [&]() {
-        int64_t sum = 0;
-        for (int32_t i = 0; i < N; ++i) {
-            int32_t m = last_cons_excl(i, -1);
-            if (m >= 0) sum += m - tgt[i];
-        }
-        return sum;
-    };
-    tgt = asap;
-    for (int round = 0; round < 2; ++round) { sweep_later(); sweep_earlier(); }
-    const int64_t life_early = total_life();
-    std::vector<int32_t> tgt_early = tgt;
-    for (int32_t i = 0; i < N; ++i) tgt[i] = D - rem[i];
-    for (int round = 0; round < 2; ++round) { sweep_earlier(); sweep_later(); }
-    if (life_early <= total_life()) tgt.swap(tgt_early);
-    if (lanes <= 0) lanes = pick_lanes(N, D);
-    if (lanes > kMaxLanes) lanes = kMaxLanes;
-    if (lookahead <= 0) lookahead = 8;
-    out.lanes = lanes;
-
-    // ---- list scheduling ----------------------------------------------------------------------
-    // Priority: smallest target step first (ties: the more critical op).  An op is not started more
-    // than `lookahead` steps before its target step, which keeps a cheap chain from running far
-    // ahead of the ops that consume its values.
-    std::vector<int32_t> step_of((size_t)N, -1), warp_of((size_t)N, -1), prev_on_warp((size_t)N, -1);
-    std::vector<int32_t> left((size_t)N);
-    std::vector<int32_t> unsched_cons((size_t)N);
-    using Key = std::pair<int64_t, int32_t>;   // (target step, alap | op)
-    std::priority_queue<Key, std::vector<Key>, std::greater<Key>> ready;
-    auto prio = [&](int32_t i) { return ((int64_t)tgt[i] << 32) | (uint32_t)(D - rem[i]); };
-    for (int32_t i = 0; i < N; ++i) {
-        left[i] = (int32_t)ops[i].preds.size();
-        unsched_cons[i] = (int32_t)(cp[i + 1] - cp[i]);
-        if (left[i] == 0) ready.push({prio(i), i});
-    }
-    std::vector<int32_t> last((size_t)lanes, -1);
-    std::vector<std::vector<int32_t>> sched;   // per step: op per warp (-1 idle)
-    std::vector<int32_t> chosen, next_ready;
-    int32_t done = 0;
-    int32_t t = 0;
-    while (done < N) {
-        chosen.clear();
-        while (!ready.empty() && (int)chosen.size() < lanes) {
-            Key k = ready.top();
-            // an op that is not due yet waits, unless the step would otherwise be empty
-            if ((k.first >> 32) > t + lookahead && !chosen.empty()) break;
-            ready.pop();
-            chosen.push_back(k.second);
-        }
-        std::vector<int32_t> row((size_t)lanes, -1);
-        std::vector<char> placed(chosen.size(), 0);
-        // first the ops whose operand sits in a free warp's register.  Where several operands do,
-        // the op follows the one with the fewest readers: a value with one reader that travels in a
-        // register is never written to a slot, and a serial chain (the launch chain, whose nodes
-        // each have one chain successor but also read several kernels) stays on one warp instead
-        // of hopping from warp to warp with a slot hand-over on its critical path every step.
-        for (size_t j = 0; j < chosen.size(); ++j) {
-            int32_t i = chosen[j];
-            int best_w = -1;
-            int64_t best_fan = 0;
-            for (int32_t p : ops[i].preds) {
-                int w = warp_of[p];
-                if (w >= 0 && last[w] == p && row[w] < 0) {
-                    const int64_t fan = cp[p + 1] - cp[p];
-                    if (best_w < 0 || fan < best_fan) {
-                        best_w = w;
-                        best_fan = fan;
-                    }
-                }
-            }
-            if (best_w >= 0) {
-                row[best_w] = i;
-                placed[j] = 1;
-            }
-        }
-        // then the rest: prefer a warp whose register value nobody is waiting for
-        for (size_t j = 0; j < chosen.size(); ++j) {
-            if (placed[j]) continue;
-            int best = -1;
-            for (int w = 0; w < lanes; ++w) {
-                if (row[w] >= 0) continue;
-                bool dead = last[w] < 0 || unsched_cons[last[w]] == 0;
-                if (dead) { best = w; break; }
-                if (best < 0) best = w;
-            }
-            row[best] = chosen[j];
-        }
-        next_ready.clear();
-        for (int w = 0; w < lanes; ++w) {
-            int32_t i = row[w];
-            if (i < 0) continue;
-            step_of[i] = t;
-            warp_of[i] = w;
-            prev_on_warp[i] = last[w];
-            ++done;
-        }
-        for (int w = 0; w < lanes; ++w) {
-            int32_t i = row[w];
-            if (i < 0) continue;
-            last[w] = i;
-            for (int32_t p : ops[i].preds) unsched_cons[p]--;
-            for (int64_t e = cp[i]; e < cp[i + 1]; ++e)
-                if (--left[cons[e]] == 0) next_ready.push_back(cons[e]);
-        }
-        for (int32_t i : next_ready) ready.push({prio(i), i});
-        sched.push_back(std::move(row));
-        ++t;
-        if (chosen.empty() && ready.empty() && done < N) {
-            err = "scheduler stalled (graph is not acyclic?)";
-            return EMO_E_NOT_TOPOLOGICAL;
-        }
-    }
-    const int32_t S = t;
-    out.steps = S;
 
     // ---- slots ---------------------------------------------------------------------------------
     // An operand is read from the warp's register when the producing op was the previous op of the
@@ -350,6 +379,7 @@ int compile_program(const HostGraph &g, const int64_t *lat, const double *energy
     std::vector<int32_t> slot_of((size_t)N, -1);
     std::vector<uint8_t> parity_of((size_t)N, 0);
     {
+        using Key = std::pair<int64_t, int32_t>;
         std::vector<uint8_t> phase;   // number of values written to a slot so far, mod 2
         std::priority_queue<int32_t, std::vector<int32_t>, std::greater<int32_t>> free_ids;
         std::priority_queue<Key, std::vector<Key>, std::greater<Key>> busy;   // (last use step, slot)

@@ -1,0 +1,91 @@
+// Lane-stream programs: the compiled form of an execution graph that the 32-bit pass kernels walk.
+//
+// One schedule serves both passes.  Every node is placed on one of `lanes` warps (a lane) at one
+// step; a lane's nodes, in step order, form its stream.  The forward pass (Eq. 1) walks every
+// stream from its first entry to its last, the backward pass (latest starts) walks the same streams
+// from the last entry to the first.  Streams are cut into stages of K steps (what the producer
+// warps bring into shared memory at once) and stages into periods of `sync` steps (the warps of a
+// policy group meet at a barrier where a period begins; exchange slots are reused only across such a
+// barrier).
+//
+// Times are carried as unsigned 32-bit offsets from static lower bounds.  With dmin_v / dmax_v the
+// smallest / largest entry of node v's duration row:
+//   forward   lbES_v = max over predecessors of lbC_k (0 for a source), lbC_v = lbES_v + dmin_v,
+//             eo_v = ES_v - lbES_v, co_v = C_v - lbC_v = eo_v + (t_v - dmin_v);
+//             an operand k of v contributes co_k - (lbES_v - lbC_k), floored at 0
+//   backward  Q_v = t_v + max over successors of Q_u (the longest tail from v's start), lbQin_v = max
+//             over successors of lbQ_u, lbQ_v = lbQin_v + dmin_v, qin_v = (max over successors of Q_u)
+//             - lbQin_v, qo_v = qin_v + (t_v - dmin_v)
+//   slack_v = T - Q_v - ES_v = T - (lbQ_v + lbES_v) - (qin_v + co_v)
+// The upper bounds (same recurrences with dmax) give the largest offset any policy can produce; the
+// program exists only when every such spread fits 32 bits (Flow::ok32), and they prune operands
+// that can never decide a maximum.
+//
+// The backward pass needs co_v of every node.  Along a stream it recovers it by subtraction: when
+// entry i took its start from the lane's own previous value alone (co_{i-1} = eo_i), then
+// co_{i-1} = co_i - (t_i - dmin_i).  Where that does not hold (several operands, or none) the
+// forward pass pushes the lane's previous value to a restore list and the backward pass pops it.
+#pragma once
+#include <cstdint>
+#include <string>
+#include <vector>
+
+#include "emo_compile.h"
+
+namespace emo {
+
+constexpr int kFlowMaxLanes = 30;
+constexpr int kFRecWords = 4;      // forward record: flags, out slot, out tag, pool offset
+constexpr int kBRecWords = 8;      // backward record: + A_v (2 words), node id, register delta
+constexpr int kOpWords = 3;        // operand descriptor: slot offset | kind bits, tag, delta
+constexpr int kHdrWords = 4;       // per (stage, lane): period counts, pushes, push offset, spare
+
+// forward record word 0
+constexpr uint32_t kF_RunMask = 0xFFu;      // > 0: a run of that many plain entries starts here
+constexpr uint32_t kF_HasReg = 1u << 8;     // starts from the lane's previous value
+constexpr uint32_t kF_RegDelta = 1u << 9;   // ... after a correction (first pool word)
+constexpr uint32_t kF_OutTag = 1u << 10;    // writes a tagged slot (value + tag, polled by readers)
+constexpr uint32_t kF_OutSet = 1u << 11;    // writes a settled slot (value only, read after a barrier)
+constexpr uint32_t kF_Terminal = 1u << 12;  // node without successors: candidate for the makespan
+constexpr uint32_t kF_Push = 1u << 13;      // the lane's previous value goes to the restore list
+constexpr uint32_t kF_OutAcc = 1u << 14;    // the settled slot is shared: the value is folded in with a maximum
+constexpr int kF_NopsShift = 16;            // bits 16..31: slot operands
+// backward record word 0
+constexpr uint32_t kB_HasReg = 1u, kB_RegDelta = 2u, kB_OutTag = 4u, kB_OutSet = 8u, kB_Pop = 16u, kB_OutAcc = 32u;
+constexpr int kB_NopsShift = 16;
+// operand descriptor word 0
+constexpr uint32_t kOpNoPoll = 1u << 31;    // written before the group's last barrier: no polling
+constexpr uint32_t kOpWord = 1u << 30;      // a settled slot (4 bytes per policy) instead of a tagged one (8)
+constexpr uint32_t kOpClear = 1u << 29;     // a shared slot (running maximum): the reader resets it to 0
+constexpr uint32_t kOpOffMask = (1u << 29) - 1u;
+
+struct FlowDir {
+    int slots_tag = 0, slots_set = 0;   // tagged slots (256 bytes per group) and settled slots (128 bytes)
+    int pool_stride = 4;                // words of operand pool per stage
+    int64_t pruned = 0;                 // edges that can never decide a maximum in this direction
+    std::vector<uint32_t> rec;          // [stages][lanes][K][kFRecWords | kBRecWords]
+    std::vector<uint32_t> pool;         // [stages][pool_stride]
+};
+
+struct Flow {
+    bool ok32 = false;                  // every spread fits 32 bits: the program below exists
+    int lanes = 0, K = 0, sync = 0, stages = 0, steps = 0, Lp = 0;
+    int64_t entries = 0;                // scheduled nodes
+    int64_t pushes = 0;                 // restore rows per policy, all stages (the lanes' final values follow)
+    std::vector<uint32_t> hdr;          // [stages][lanes][kHdrWords]
+    std::vector<uint32_t> rows;         // [stages][lanes][K] policy row read by the entry, kNone = none
+    std::vector<uint32_t> node;         // [stages][lanes][K] node id, kNone = unused position
+    std::vector<uint32_t> step;         // [stages][lanes][K] step of the entry (host-side inspection)
+    std::vector<uint32_t> tabF;         // [stages][lanes][K][Lp][3]: t - dmin, energy high word, low word
+    std::vector<uint32_t> tabB;         // [stages][lanes][K][Lp]: t - dmin
+    std::vector<int64_t> lbes;          // [stages][lanes][K] lbES_v (for the ES and LS outputs)
+    std::vector<int64_t> push_base;     // [stages + 1] first restore row of every stage
+    FlowDir f, b;
+};
+
+// Compiles g into a lane-stream program.  Returns EMO_OK with out.ok32 = false when the 32-bit
+// representation does not apply (spread too large, too many lanes); other codes are errors.
+int compile_flow(const HostGraph &g, const int64_t *lat, const double *energy, int lanes, int lookahead,
+                 int K, int sync, Flow &out, std::string &err);
+
+}  // namespace emo

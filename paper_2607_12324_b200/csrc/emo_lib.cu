@@ -10,6 +10,7 @@
 
 #include "../../include/emo.h"
 #include "emo_compile.h"
+#include "emo_flow.h"
 #include "emo_kernels.cuh"
 #include "emo_pass_lane.cuh"
 #include "emo_pass_staged.cuh"
@@ -34,6 +35,7 @@ struct DevProgramLane {
 struct emo_graph {
     HostGraph h;
     Program fwd, bwd;
+    Flow flow;                       // lane-stream program of the 32-bit pass kernels (flow.ok32: usable)
     DevProgram dfwd, dbwd;
     DevProgramLane lfwd, lbwd;       // only for programs of at most kLaneMaxLanes lanes
     bool host_only = false;
@@ -611,6 +613,11 @@ int emo_graph_load(int32_t n, const int64_t *row_ptr, const int32_t *col, const 
         int rc = compile_dir(true, nullptr, g->bwd);
         if (rc == EMO_OK) rc = compile_dir(false, &g->bwd.pos_of_node, g->fwd);
         if (rc != EMO_OK) { delete g; return rc; }
+        {
+            const int fk = (int)((flags >> 24) & 0x3F), fs = (int)((flags >> 4) & 0xF) * 8;
+            rc = compile_flow(h, lat, energy, lanes, look, fk, fs, g->flow, err);
+            if (rc != EMO_OK) { delete g; return rc; }
+        }
         std::vector<int32_t> hop((size_t)std::max(n, 1), 0);
         int32_t depth = 0;
         for (int32_t v = 0; v < n; ++v) {
@@ -679,6 +686,42 @@ int emo_graph_info(const emo_graph *g, emo_info *info)
     info->steps_bwd = g->bwd.steps;
     info->slots_bwd = g->bwd.slots;
     info->aux_bwd = g->bwd.aux;
+    return EMO_OK;
+}
+
+int emo_graph_flow(const emo_graph *g, emo_flow_view *v)
+{
+    if (!g || !v) return EMO_E_INVALID_ARG;
+    const Flow &f = g->flow;
+    std::memset(v, 0, sizeof *v);
+    v->ok32 = f.ok32 ? 1 : 0;
+    v->lanes = f.lanes;
+    v->K = f.K;
+    v->sync = f.sync;
+    v->stages = f.stages;
+    v->steps = f.steps;
+    v->Lp = f.Lp;
+    v->slots_tag_fwd = f.f.slots_tag;
+    v->slots_set_fwd = f.f.slots_set;
+    v->pool_stride_fwd = f.f.pool_stride;
+    v->slots_tag_bwd = f.b.slots_tag;
+    v->slots_set_bwd = f.b.slots_set;
+    v->pool_stride_bwd = f.b.pool_stride;
+    v->pushes = f.pushes;
+    v->pruned_fwd = f.f.pruned;
+    v->pruned_bwd = f.b.pruned;
+    v->hdr = f.hdr.data();
+    v->rows = f.rows.data();
+    v->node = f.node.data();
+    v->step = f.step.data();
+    v->tab_fwd = f.tabF.data();
+    v->tab_bwd = f.tabB.data();
+    v->rec_fwd = f.f.rec.data();
+    v->pool_fwd = f.f.pool.data();
+    v->rec_bwd = f.b.rec.data();
+    v->pool_bwd = f.b.pool.data();
+    v->lbes = f.lbes.data();
+    v->push_base = f.push_base.data();
     return EMO_OK;
 }
 

@@ -28,7 +28,7 @@ EXPORTS = [
     "emo_strerror", "emo_graph_load", "emo_graph_free", "emo_graph_info", "emo_workspace_bytes",
     "emo_eval_policies", "emo_slack_batch", "emo_slack", "emo_baseline", "emo_target_from_delta",
     "emo_select", "emo_transpose_policies", "emo_slack_batch_host", "emo_graph_program",
-    "emo_set_pass_events", "emo_select_static",
+    "emo_set_pass_events", "emo_select_static", "emo_graph_flow",
 ]
 
 
@@ -38,6 +38,14 @@ def EMO_F_LANES(c: int) -> int:
 
 def EMO_F_LOOKAHEAD(d: int) -> int:
     return (d & 0xFF) << 16
+
+
+def EMO_F_FLOW_SYNC(s: int) -> int:
+    return ((s // 8) & 0xF) << 4
+
+
+def EMO_F_FLOW_STAGE(k: int) -> int:
+    return (k & 0x3F) << 24
 
 
 class EmoError(RuntimeError):
@@ -53,6 +61,15 @@ class emo_info(ctypes.Structure):
                 ("steps_fwd", ctypes.c_int32), ("slots_fwd", ctypes.c_int32), ("aux_fwd", ctypes.c_int32),
                 ("steps_bwd", ctypes.c_int32), ("slots_bwd", ctypes.c_int32), ("aux_bwd", ctypes.c_int32),
                 ("lanes_bwd", ctypes.c_int32), ("sync_fwd", ctypes.c_int32), ("sync_bwd", ctypes.c_int32)]
+
+
+class emo_flow_view(ctypes.Structure):
+    _fields_ = ([(k, ctypes.c_int32) for k in ("ok32", "lanes", "K", "sync", "stages", "steps", "Lp", "slots_tag_fwd",
+                                                "slots_set_fwd", "pool_stride_fwd", "slots_tag_bwd", "slots_set_bwd",
+                                                "pool_stride_bwd")] +
+                [(k, ctypes.c_int64) for k in ("pushes", "pruned_fwd", "pruned_bwd")] +
+                [(k, ctypes.c_void_p) for k in ("hdr", "rows", "node", "step", "tab_fwd", "tab_bwd", "rec_fwd", "pool_fwd",
+                                                "rec_bwd", "pool_bwd", "lbes", "push_base")])
 
 
 _lib = None
@@ -86,6 +103,7 @@ def lib():
                                         ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(p),
                                         ctypes.POINTER(p), ctypes.POINTER(p)]
         L.emo_set_pass_events.argtypes = [p, p, p, p]
+        L.emo_graph_flow.argtypes = [p, ctypes.POINTER(emo_flow_view)]
         L.emo_select_static.argtypes = [i64, p, p, i64, p, i64, p, p, p, p]
         for name in EXPORTS:
             if name not in ("emo_strerror", "emo_target_from_delta"):
@@ -275,3 +293,32 @@ def emo_graph_program(g: Graph, direction: int):
     lat = np.ctypeslib.as_array(ctypes.cast(pl, u32p), shape=(q * Lp.value,)).copy()
     return lanes.value, steps.value, slots.value, Lp.value, ent.reshape(steps.value, lanes.value, 8), \
         rows.reshape(steps.value, lanes.value), lat.reshape(q, Lp.value)
+
+
+def emo_graph_flow(g: Graph) -> dict:
+    """The lane-stream program of the 32-bit pass kernels as numpy copies (host-side inspection)."""
+    v = emo_flow_view()
+    _check(lib().emo_graph_flow(g.handle, ctypes.byref(v)), "emo_graph_flow")
+    out = {k: getattr(v, k) for k, _ in emo_flow_view._fields_[:16]}
+    if not v.ok32:
+        return out
+    q = v.stages * v.lanes * v.K
+
+    def arr(ptr, count, ctype, dtype):
+        if count == 0:
+            return np.zeros(0, dtype)
+        return np.ctypeslib.as_array(ctypes.cast(ptr, ctypes.POINTER(ctype)), shape=(count,)).astype(dtype, copy=True)
+
+    u32, i64 = ctypes.c_uint32, ctypes.c_int64
+    out["hdr"] = arr(v.hdr, v.stages * v.lanes * 4, u32, np.uint32).reshape(v.stages, v.lanes, 4)
+    for k in ("rows", "node", "step"):
+        out[k] = arr(getattr(v, k), q, u32, np.uint32).reshape(v.stages, v.lanes, v.K)
+    out["tab_fwd"] = arr(v.tab_fwd, q * v.Lp * 3, u32, np.uint32).reshape(v.stages, v.lanes, v.K, v.Lp, 3)
+    out["tab_bwd"] = arr(v.tab_bwd, q * v.Lp, u32, np.uint32).reshape(v.stages, v.lanes, v.K, v.Lp)
+    out["rec_fwd"] = arr(v.rec_fwd, q * 4, u32, np.uint32).reshape(v.stages, v.lanes, v.K, 4)
+    out["rec_bwd"] = arr(v.rec_bwd, q * 8, u32, np.uint32).reshape(v.stages, v.lanes, v.K, 8)
+    out["pool_fwd"] = arr(v.pool_fwd, v.stages * v.pool_stride_fwd, u32, np.uint32).reshape(v.stages, v.pool_stride_fwd)
+    out["pool_bwd"] = arr(v.pool_bwd, v.stages * v.pool_stride_bwd, u32, np.uint32).reshape(v.stages, v.pool_stride_bwd)
+    out["lbes"] = arr(v.lbes, q, i64, np.int64).reshape(v.stages, v.lanes, v.K)
+    out["push_base"] = arr(v.push_base, v.stages + 1, i64, np.int64)
+    return out
