@@ -272,6 +272,8 @@ def main():
                        "slack_materialised": True, "slack_sums": bool(args.sums), "delta_ppm": ppm, "lanes": info.lanes, "steps_fwd": info.steps_fwd,
                        "slots_fwd": info.slots_fwd, "slots_bwd": info.slots_bwd,
                        "l2": "inputs larger than L2 (levels %.1f GB, slack %.1f GB per step)" % (n * ldb / 1e9, n * B * 8 / 1e9),
+                       "kernels": {2: "32-bit lane-stream", 1: "staged 64-bit", 0: "plain 64-bit"}[
+                           emo.emo_call_path(h, B, lv, ldb, B, True, args.call_flags)],
                        "parallelism": "replicas" if world > 1 else "single"},
             "policies_per_s": world * B / (ms_per_step * 1e-3),
             "gpu_launches": launches_per_step * args.steps,

@@ -55,6 +55,8 @@ extern "C" {
 #define EMO_F_NO_STAGING 0x2u      /* use the plain-load kernels instead of the staged ones */
 #define EMO_F_PAIR_KERNEL 0x4u     /* staged pass kernel with two policies per thread (default only for very large batches) */
 #define EMO_F_LANE_KERNEL 0x8u     /* staged pass kernel with one policy per thread (the default otherwise) */
+#define EMO_F_TEST_STALL 0x100u    /* test hook of the 32-bit kernels: the producer warps stop half way, so that the
+                                      consumers' bounded waits run out and EMO_E_TIMEOUT is reported */
 
 typedef struct emo_graph emo_graph;
 
@@ -241,6 +243,32 @@ int emo_slack_batch_host(const emo_graph *g, int64_t B, const uint8_t *lvl_host,
 int emo_set_pass_events(void *fwd_start, void *fwd_stop, void *bwd_start, void *bwd_stop);
 
 /*
+ * emo_call_path - which kernels emo_eval_policies (need_slack = 0) or emo_slack_batch (need_slack = 1)
+ * would run for these arguments: 2 = the 32-bit lane-stream kernels, 1 = the staged 64-bit kernels,
+ * 0 = the plain-load 64-bit kernels; negative = an EMO_E_* code.  lvl may be any pointer with the
+ * alignment of the real one.  For tests and reports; it launches nothing.
+ */
+int emo_call_path(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t ldb, int64_t ldo,
+                  int need_slack, uint32_t flags);
+
+/*
+ * emo_set_flow_counters - measurement hook (no counterpart in the method): a device array of 131072
+ * int64 that later calls of the 32-bit kernels fill with cycle counts, 4 per warp at
+ * [(pass * 512 + block) * 32 + warp] for the first 512 blocks (pass 0 forward, 1 backward): consumer
+ * warps {cycles waiting for staged data, cycles at group barriers, total}, producer warps {cycles
+ * waiting for a free buffer, cycles issuing copies, total}.  NULL switches it off.  Process-wide.
+ */
+int emo_set_flow_counters(void *dev);
+
+/*
+ * emo_set_wait_limit - bound, in SM clock cycles, of every device-side wait of the 32-bit pass kernels
+ * (a wait on a stage of staged data or on a value another warp produces).  A wait that runs out ends
+ * the kernel with EMO_E_TIMEOUT in *status instead of hanging.  Default 4 * 10^9 (about two seconds);
+ * tests use a small value.  Process-wide; applies to calls made afterwards.
+ */
+int emo_set_wait_limit(int64_t cycles);
+
+/*
  * Inspection of the compiled evaluation program (host memory owned by the handle; valid until
  * emo_graph_free).  dir 0 = forward, 1 = backward.  entries is [steps][lanes][8] uint32, rows is
  * uint32 [steps*lanes] (policy row read by the entry, 0xFFFFFFFF = none), lat is uint32
@@ -254,9 +282,10 @@ int emo_graph_program(const emo_graph *g, int dir, int32_t *lanes, int32_t *step
  * Inspection of the lane-stream program that the 32-bit pass kernels walk (host memory owned by the
  * handle; valid until emo_graph_free).  ok32 = 0 means the graph's spread of start times over all
  * policies does not fit 32 bits (or it needs more than 30 lanes) and the 64-bit kernels serve it;
- * the arrays are then empty.  Layouts: hdr [stages][lanes][4], rows / node / step [stages][lanes][K],
- * tab_fwd [stages][lanes][K][Lp][3], tab_bwd [stages][lanes][K][Lp], rec_fwd [stages][lanes][K][4],
- * rec_bwd [stages][lanes][K][8], pool_* [stages][pool_stride_*], lbes [stages][lanes][K],
+ * the arrays are then empty.  Layouts: hdr [stages][lanes][8], rows / node / step [stages][lanes][K],
+ * tab_fwd [stages][lanes][K][Lp][3], tab_bwd [stages][lanes][K][Lp], rec_fwd [stages][lanes][K][8],
+ * rec_bwd [stages][lanes][K][12], pool_* [stages][pool_stride_*], seg_* [stages][lanes][40] (bytes),
+ * lbes [stages][lanes][K],
  * push_base [stages + 1].  Used by host-side tests of the compiler; not needed to evaluate anything.
  */
 typedef struct emo_flow_view {
@@ -266,6 +295,7 @@ typedef struct emo_flow_view {
     int64_t pushes, pruned_fwd, pruned_bwd;
     const uint32_t *hdr, *rows, *node, *step, *tab_fwd, *tab_bwd;
     const uint32_t *rec_fwd, *pool_fwd, *rec_bwd, *pool_bwd;
+    const uint8_t *seg_fwd, *seg_bwd;
     const int64_t *lbes, *push_base;
 } emo_flow_view;
 int emo_graph_flow(const emo_graph *g, emo_flow_view *out);

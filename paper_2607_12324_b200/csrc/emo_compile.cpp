@@ -72,19 +72,25 @@ int pick_lanes(int64_t n_ops, int depth)
 // same warp handled just before it (-1: none), S the number of steps.
 int schedule_ops(const std::vector<std::vector<int32_t>> &preds, int lanes, int lookahead, std::vector<int32_t> &step_of,
                  std::vector<int32_t> &warp_of, std::vector<int32_t> &prev_on_warp, int32_t &S_out, int &lanes_out,
-                 std::string &err)
+                 std::string &err, const std::vector<std::vector<int32_t>> *gaps, bool hard_gaps)
 {
     const int32_t N = (int32_t)preds.size();
+    // distance in steps an op keeps from operand k of its list (1 unless the caller asks for more)
+    auto gap = [&](int32_t i, size_t k) { return gaps ? (*gaps)[i][k] : 1; };
     // consumers of each op
     std::vector<int64_t> cp((size_t)N + 1, 0);
     for (int32_t i = 0; i < N; ++i)
         for (int32_t p : preds[i]) cp[p + 1]++;
     for (int32_t i = 0; i < N; ++i) cp[i + 1] += cp[i];
-    std::vector<int32_t> cons((size_t)std::max<int64_t>(cp[N], 1));
+    std::vector<int32_t> cons((size_t)std::max<int64_t>(cp[N], 1)), cgap((size_t)std::max<int64_t>(cp[N], 1), 1);
     {
         std::vector<int64_t> f(cp.begin(), cp.end() - 1);
         for (int32_t i = 0; i < N; ++i)
-            for (int32_t p : preds[i]) cons[f[p]++] = i;
+            for (size_t k = 0; k < preds[i].size(); ++k) {
+                const int32_t p = preds[i][k];
+                cgap[f[p]] = gap(i, k);
+                cons[f[p]++] = i;
+            }
     }
 
     // hop levels: earliest step (asap) and the number of hops to the end (rem; alap = D - rem)
@@ -92,13 +98,13 @@ int schedule_ops(const std::vector<std::vector<int32_t>> &preds, int lanes, int 
     int32_t D = 0;
     for (int32_t i = 0; i < N; ++i) {
         int32_t a = 0;
-        for (int32_t p : preds[i]) a = std::max(a, asap[p] + 1);
+        for (size_t k = 0; k < preds[i].size(); ++k) a = std::max(a, asap[preds[i][k]] + gap(i, k));
         asap[i] = a;
         D = std::max(D, a + 1);
     }
     for (int32_t i = N - 1; i >= 0; --i) {
         int32_t r = 1;
-        for (int64_t e = cp[i]; e < cp[i + 1]; ++e) r = std::max(r, rem[cons[e]] + 1);
+        for (int64_t e = cp[i]; e < cp[i + 1]; ++e) r = std::max(r, rem[cons[e]] + cgap[e]);
         rem[i] = r;
     }
     // Target steps.  A value occupies an exchange slot from the step that produces it to the step
@@ -120,7 +126,7 @@ int schedule_ops(const std::vector<std::vector<int32_t>> &preds, int lanes, int 
         for (int32_t i = N - 1; i >= 0; --i) {
             if (cp[i + 1] == cp[i]) continue;
             int32_t hi = INT32_MAX;
-            for (int64_t e = cp[i]; e < cp[i + 1]; ++e) hi = std::min(hi, tgt[cons[e]] - 1);
+            for (int64_t e = cp[i]; e < cp[i + 1]; ++e) hi = std::min(hi, tgt[cons[e]] - cgap[e]);
             if (hi <= tgt[i]) continue;
             int64_t gain = hi - tgt[i], cost = 0;
             for (int32_t p : preds[i]) {
@@ -135,7 +141,7 @@ int schedule_ops(const std::vector<std::vector<int32_t>> &preds, int lanes, int 
         for (int32_t i = 0; i < N; ++i) {
             if (preds[i].empty()) continue;
             int32_t lo = 0;
-            for (int32_t p : preds[i]) lo = std::max(lo, tgt[p] + 1);
+            for (size_t k = 0; k < preds[i].size(); ++k) lo = std::max(lo, tgt[preds[i][k]] + gap(i, k));
             if (lo >= tgt[i]) continue;
             bool held = false;   // a consumer with other operands keeps this op's value alive
             for (int64_t e = cp[i]; e < cp[i + 1]; ++e) held |= preds[cons[e]].size() > 1;
@@ -187,9 +193,15 @@ int schedule_ops(const std::vector<std::vector<int32_t>> &preds, int lanes, int 
     std::vector<int32_t> last((size_t)lanes, -1);
     std::vector<std::vector<int32_t>> sched;   // per step: op per warp (-1 idle)
     std::vector<int32_t> chosen, next_ready;
+    std::priority_queue<std::pair<int32_t, int32_t>, std::vector<std::pair<int32_t, int32_t>>, std::greater<std::pair<int32_t, int32_t>>>
+        held;      // (earliest step, op): operands done, but the op keeps its distance from one of them
     int32_t done = 0;
     int32_t t = 0;
     while (done < N) {
+        while (!held.empty() && held.top().first <= t) {
+            ready.push({prio(held.top().second), held.top().second});
+            held.pop();
+        }
         chosen.clear();
         while (!ready.empty() && (int)chosen.size() < lanes) {
             Key k = ready.top();
@@ -253,10 +265,15 @@ int schedule_ops(const std::vector<std::vector<int32_t>> &preds, int lanes, int 
             for (int64_t e = cp[i]; e < cp[i + 1]; ++e)
                 if (--left[cons[e]] == 0) next_ready.push_back(cons[e]);
         }
-        for (int32_t i : next_ready) ready.push({prio(i), i});
+        for (int32_t i : next_ready) {
+            int32_t est = 0;
+            for (size_t k = 0; k < preds[i].size(); ++k) est = std::max(est, step_of[preds[i][k]] + (hard_gaps ? gap(i, k) : 1));
+            if (est <= t + 1) ready.push({prio(i), i});
+            else held.push({est, i});
+        }
         sched.push_back(std::move(row));
         ++t;
-        if (chosen.empty() && ready.empty() && done < N) {
+        if (chosen.empty() && ready.empty() && held.empty() && done < N) {
             err = "scheduler stalled (graph is not acyclic?)";
             return EMO_E_NOT_TOPOLOGICAL;
         }

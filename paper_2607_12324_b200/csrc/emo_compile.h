@@ -72,8 +72,11 @@ int pick_lanes(int64_t n_ops, int depth);
 // Target steps and list scheduling of ops, given by their operand lists in a topological order, onto
 // `lanes` warps (<= 0: chosen from the shape).  step_of / warp_of give every op's place, prev_on_warp
 // the op the same warp handled just before it (-1: none), steps the length of the schedule.
+// gaps (optional, same shape as preds): the least distance in steps between an op and that operand
+// (1 when absent).  With hard_gaps the distance is kept; without, it only shapes the target steps, so
+// that the scheduler aims for it where the lanes have room.
 int schedule_ops(const std::vector<std::vector<int32_t>> &preds, int lanes, int lookahead, std::vector<int32_t> &step_of,
                  std::vector<int32_t> &warp_of, std::vector<int32_t> &prev_on_warp, int32_t &steps, int &lanes_out,
-                 std::string &err);
+                 std::string &err, const std::vector<std::vector<int32_t>> *gaps = nullptr, bool hard_gaps = true);
 
 }  // namespace emo

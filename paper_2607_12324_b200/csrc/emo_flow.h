@@ -35,15 +35,27 @@
 namespace emo {
 
 constexpr int kFlowMaxLanes = 30;
-constexpr int kFRecWords = 4;      // forward record: flags, out slot, out tag, pool offset
-constexpr int kBRecWords = 8;      // backward record: + A_v (2 words), node id, register delta
+constexpr int kFRecWords = 8;      // forward record: flags, out slot, out tag / correction, pool offset, first operand
+                                   // (3 words), correction of the lane's previous value
+constexpr int kBRecWords = 12;     // backward record: flags, out slot, out tag / correction, pool offset, A_v (2 words),
+                                   // node id, correction of the lane's previous value, first operand (3 words), spare
 constexpr int kOpWords = 3;        // operand descriptor: slot offset | kind bits, tag, delta
-constexpr int kHdrWords = 4;       // per (stage, lane): period counts, pushes, push offset, spare
+constexpr int kHdrWords = 8;       // per (stage, lane): word 0 = forward segments (bits 0..7) | backward segments (8..15)
+                                   // | entries (16..23); word 4 pushes, word 5 first restore row inside the stage,
+                                   // word 6 first restore row of the stage; the rest spare
+constexpr int kFlowMaxStage = 32;  // most steps of a stage
+constexpr int kFlowRun = 8;        // most simple entries of one segment (their look-ups are issued together)
+constexpr int kSegBytes = 40;      // segment bytes per (stage, lane) and direction: at most K + K / sync
+// segment byte: bits 0..3 simple entries in the run, then
+constexpr uint32_t kSegRunMask = 15u;
+constexpr uint32_t kSegSpecial = 16u;   // an entry that needs its record comes first
+constexpr uint32_t kSegBarrier = 32u;   // the group meets before this segment (a period begins)
+constexpr uint32_t kSegIn = 64u;        // backward run: every entry folds in one settled single-reader slot
+constexpr uint32_t kSegOut = 128u;      // backward run: every entry writes one settled single-reader slot
 
-// forward record word 0
-constexpr uint32_t kF_RunMask = 0xFFu;      // > 0: a run of that many plain entries starts here
+// forward record word 0 (a plain entry has kF_HasReg alone)
 constexpr uint32_t kF_HasReg = 1u << 8;     // starts from the lane's previous value
-constexpr uint32_t kF_RegDelta = 1u << 9;   // ... after a correction (first pool word)
+constexpr uint32_t kF_RegDelta = 1u << 9;   // ... after a correction (record word 7)
 constexpr uint32_t kF_OutTag = 1u << 10;    // writes a tagged slot (value + tag, polled by readers)
 constexpr uint32_t kF_OutSet = 1u << 11;    // writes a settled slot (value only, read after a barrier)
 constexpr uint32_t kF_Terminal = 1u << 12;  // node without successors: candidate for the makespan
@@ -52,11 +64,15 @@ constexpr uint32_t kF_OutAcc = 1u << 14;    // the settled slot is shared: the v
 constexpr int kF_NopsShift = 16;            // bits 16..31: slot operands
 // backward record word 0
 constexpr uint32_t kB_HasReg = 1u, kB_RegDelta = 2u, kB_OutTag = 4u, kB_OutSet = 8u, kB_Pop = 16u, kB_OutAcc = 32u;
+// A simple backward entry continues from the lane's previous value (corrected by word 7), reads at
+// most one slot and writes at most one, both settled with a single reader (so the value is stored
+// already corrected and the reader resets the slot); word 3 then holds the operand's slot offset.
+constexpr uint32_t kB_Simple = 64u;
 constexpr int kB_NopsShift = 16;
 // operand descriptor word 0
 constexpr uint32_t kOpNoPoll = 1u << 31;    // written before the group's last barrier: no polling
 constexpr uint32_t kOpWord = 1u << 30;      // a settled slot (4 bytes per policy) instead of a tagged one (8)
-constexpr uint32_t kOpClear = 1u << 29;     // a shared slot (running maximum): the reader resets it to 0
+constexpr uint32_t kOpClear = 1u << 29;     // a settled slot with a single reader: the reader resets it to 0
 constexpr uint32_t kOpOffMask = (1u << 29) - 1u;
 
 struct FlowDir {
@@ -65,6 +81,7 @@ struct FlowDir {
     int64_t pruned = 0;                 // edges that can never decide a maximum in this direction
     std::vector<uint32_t> rec;          // [stages][lanes][K][kFRecWords | kBRecWords]
     std::vector<uint32_t> pool;         // [stages][pool_stride]
+    std::vector<uint8_t> seg;           // [stages][lanes][kSegBytes] segment bytes in walking order
 };
 
 struct Flow {

@@ -16,7 +16,7 @@ struct SlotUse {
     int32_t obj = -1;       // slot object holding the value (-1: the value is read from registers only)
     bool settled = false;   // every slot reader sits behind a barrier: value only, no tag
     bool pre = false;       // settled with one reader: the writer applies the reader's correction
-    bool acc = false;       // ... and shares the slot with the reader's other such operands (maximum)
+    bool acc = false;       // same as pre: the slot collects a maximum (shared with the reader's other such operands)
     uint32_t pre_delta = 0;
 };
 
@@ -24,7 +24,7 @@ struct SlotUse {
 struct SlotObj {
     int32_t first = 0, last = 0;   // periods (processing order of the direction) of the first write / last read
     bool settled = false;
-    bool acc = false;              // shared by several writers (settled slots of their own: always 0 between uses)
+    bool acc = false;              // single-reader settled values (slots of their own kind: the reader resets them to 0)
     int32_t id = -1;               // slot number within its kind
 };
 
@@ -73,7 +73,7 @@ int compile_flow(const HostGraph &g, const int64_t *lat, const double *energy, i
     while (Lp < L) Lp <<= 1;
     if (K <= 0) K = 32;
     if (sync <= 0 || sync > K) sync = K;
-    if (K % sync != 0 || K / sync > 4 || K > 255) return EMO_E_INVALID_ARG;
+    if (K > kFlowMaxStage || sync < 1 || K % sync != 0 || K / sync > 4) return EMO_E_INVALID_ARG;
     out.Lp = Lp;
     out.K = K;
     out.sync = sync;
@@ -147,7 +147,13 @@ int compile_flow(const HostGraph &g, const int64_t *lat, const double *energy, i
     // edge e (k = pc[e] -> v): live forward unless C_k can never exceed the start every policy gives v
     // through its strongest predecessor; live backward under the mirrored test on the tails
     std::vector<char> liveF((size_t)std::max<int64_t>(m, 1), 0), liveB((size_t)std::max<int64_t>(m, 1), 0);
-    std::vector<std::vector<int32_t>> preds((size_t)n);
+    // An edge that is live in one direction only keeps its two nodes a period apart in the schedule:
+    // its reader (in that direction) then finds the value settled behind a barrier instead of polling
+    // for it, and nothing waits for the reader in the other direction.  (Typical: a launch node and
+    // the kernels it launches - forward the launch never decides a kernel's start, backward the launch
+    // node collects its kernels' tails.)  Kept only if it does not stretch the schedule.
+    std::vector<std::vector<int32_t>> preds((size_t)n), gaps((size_t)n);
+    bool any_gap = false;
     for (int32_t v = 0; v < n; ++v)
         for (int64_t e = pp[v]; e < pp[v + 1]; ++e) {
             const int32_t k = pc[e];
@@ -155,12 +161,31 @@ int compile_flow(const HostGraph &g, const int64_t *lat, const double *energy, i
             liveB[e] = (v == bestB[k]) || ubQ[v] > lbQin[k];
             if (!liveF[e]) out.f.pruned++;
             if (!liveB[e]) out.b.pruned++;
-            if (liveF[e] || liveB[e]) preds[v].push_back(k);
+            if (liveF[e] || liveB[e]) {
+                preds[v].push_back(k);
+                gaps[v].push_back(liveF[e] != liveB[e] ? sync : 1);
+                any_gap = any_gap || liveF[e] != liveB[e];
+            }
         }
     std::vector<int32_t> step_of, lane_of, prev_on_lane;
     int32_t S = 0;
-    int rc = schedule_ops(preds, lanes, lookahead, step_of, lane_of, prev_on_lane, S, lanes, err);
+    const int lanes_req = lanes;
+    int rc = schedule_ops(preds, lanes_req, lookahead, step_of, lane_of, prev_on_lane, S, lanes, err, any_gap ? &gaps : nullptr, false);
     if (rc != EMO_OK) return rc;
+    if (any_gap) {
+        std::vector<int32_t> s2, l2, p2;
+        int32_t S2 = 0;
+        int lanes2 = 0;
+        rc = schedule_ops(preds, lanes_req, lookahead, s2, l2, p2, S2, lanes2, err, nullptr);
+        if (rc != EMO_OK) return rc;
+        if ((int64_t)S * 100 > (int64_t)S2 * 105 + 3200) {      // more than 5 % (and 32 steps) longer: not worth it
+            step_of.swap(s2);
+            lane_of.swap(l2);
+            prev_on_lane.swap(p2);
+            S = S2;
+            lanes = lanes2;
+        }
+    }
     if (lanes > kFlowMaxLanes) return EMO_OK;
     std::vector<int32_t> next_on_lane((size_t)n, -1);
     for (int32_t v = 0; v < n; ++v)
@@ -192,8 +217,6 @@ int compile_flow(const HostGraph &g, const int64_t *lat, const double *energy, i
         for (int32_t v : by_step) {
             const int st = step_of[v] / K, ln = lane_of[v];
             pos_of[v] = cnt[(size_t)st * lanes + ln]++;
-            const int period = (step_of[v] % K) / sync;
-            out.hdr[((size_t)st * lanes + ln) * kHdrWords] += 1u << (8 * period);
         }
     }
     auto slot_index = [&](int32_t v) { return ((size_t)(step_of[v] / K) * lanes + lane_of[v]) * K + pos_of[v]; };
@@ -251,7 +274,9 @@ int compile_flow(const HostGraph &g, const int64_t *lat, const double *energy, i
             for (int32_t v = 0; v < n; ++v) {
                 if (last[v] < 0) continue;
                 const int32_t per = backward ? bper(v) : fper(v);
-                if (use[v].pre && npre[reader[v]] >= 2) {
+                if (use[v].pre) {
+                    // single-reader settled values live in slots of their own kind, which their reader
+                    // resets: the operands of one reader share a slot that collects their maximum
                     const int32_t r = reader[v];
                     use[v].acc = true;
                     if (accobj[r] < 0) {
@@ -314,34 +339,30 @@ int compile_flow(const HostGraph &g, const int64_t *lat, const double *energy, i
             uint32_t *r = &out.f.rec[q * kFRecWords];
             std::vector<uint32_t> &pool = poolF[st];
             uint32_t fl = 0, nops = 0;
-            const uint32_t pool0 = (uint32_t)pool.size();
-            // the register operand's correction comes first in the pool
+            std::vector<uint32_t> opw;      // operand descriptors, 3 words each
             for (int64_t e = pp[v]; e < pp[v + 1]; ++e) {
                 const int32_t k = pc[e];
                 if (!liveF[e] || prev_on_lane[v] != k) continue;
                 fl |= kF_HasReg;
-                const uint32_t delta = (uint32_t)(lbES[v] - lbC[k]);
-                if (delta) {
-                    fl |= kF_RegDelta;
-                    pool.push_back(delta);
-                }
+                r[7] = (uint32_t)(lbES[v] - lbC[k]);
+                if (r[7]) fl |= kF_RegDelta;
             }
             bool acc_seen = false;
             for (int64_t e = pp[v]; e < pp[v + 1]; ++e) {
                 const int32_t k = pc[e];
                 if (!liveF[e] || prev_on_lane[v] == k) continue;
                 if (useF[k].acc) {
-                    // the members of an accumulator appear as one operand, cleared after the read
+                    // the members of a shared slot appear as one operand, reset after the read
                     if (acc_seen) continue;
                     acc_seen = true;
                 }
                 uint32_t w = slot_off(useF[k], objF, out.f);
                 if (useF[k].settled) w |= kOpWord;
                 if (fper(k) < fper(v)) w |= kOpNoPoll;
-                if (useF[k].acc) w |= kOpClear;
-                pool.push_back(w);
-                pool.push_back(tag_of(k));
-                pool.push_back(useF[k].pre ? 0u : (uint32_t)(lbES[v] - lbC[k]));
+                if (useF[k].pre) w |= kOpClear;
+                opw.push_back(w);
+                opw.push_back(tag_of(k));
+                opw.push_back(useF[k].pre ? 0u : (uint32_t)(lbES[v] - lbC[k]));
                 ++nops;
             }
             if (useF[v].obj >= 0) {
@@ -349,6 +370,12 @@ int compile_flow(const HostGraph &g, const int64_t *lat, const double *energy, i
                 if (useF[v].acc) fl |= kF_OutAcc;
                 r[1] = slot_off(useF[v], objF, out.f);
                 r[2] = useF[v].settled ? useF[v].pre_delta : tag_of(v);
+            }
+            // the first operand sits in the record, the others (and a terminal node's bound) in the pool
+            r[3] = (uint32_t)pool.size();
+            for (size_t k = 0; k < opw.size(); ++k) {
+                if (k < 3) r[4 + k] = opw[k];
+                else pool.push_back(opw[k]);
             }
             if (sp[v + 1] == sp[v]) {
                 fl |= kF_Terminal;
@@ -363,14 +390,13 @@ int compile_flow(const HostGraph &g, const int64_t *lat, const double *energy, i
             }
             if (nops > 0xFFFFu) { err = "a node has more than 65535 exchanged operands"; return EMO_E_UNSUPPORTED; }
             r[0] = fl | (nops << kF_NopsShift);
-            r[3] = pool0;
         }
         // backward record
         {
             uint32_t *r = &out.b.rec[q * kBRecWords];
             std::vector<uint32_t> &pool = poolB[st];
-            uint32_t fl = 0, nops = 0;
-            r[3] = (uint32_t)pool.size();
+            uint32_t fl = 0, nops = 0, simple_in_off = kNone;
+            std::vector<uint32_t> opw;
             bool acc_seen = false;
             for (int64_t e = sp[v]; e < sp[v + 1]; ++e) {
                 const int32_t u = sc[e];
@@ -391,10 +417,11 @@ int compile_flow(const HostGraph &g, const int64_t *lat, const double *energy, i
                 uint32_t w = slot_off(useB[u], objB, out.b);
                 if (useB[u].settled) w |= kOpWord;
                 if (bper(u) < bper(v)) w |= kOpNoPoll;
-                if (useB[u].acc) w |= kOpClear;
-                pool.push_back(w);
-                pool.push_back(tag_of(u));
-                pool.push_back(useB[u].pre ? 0u : delta);
+                if (useB[u].pre) w |= kOpClear;
+                simple_in_off = useB[u].pre ? (w & kOpOffMask) : kNone;
+                opw.push_back(w);
+                opw.push_back(tag_of(u));
+                opw.push_back(useB[u].pre ? 0u : delta);
                 ++nops;
             }
             if (useB[v].obj >= 0) {
@@ -403,43 +430,103 @@ int compile_flow(const HostGraph &g, const int64_t *lat, const double *energy, i
                 r[1] = slot_off(useB[v], objB, out.b);
                 r[2] = useB[v].settled ? useB[v].pre_delta : tag_of(v);
             }
+            r[3] = (uint32_t)pool.size();
+            for (size_t k = 0; k < opw.size(); ++k) {
+                if (k < 3) r[8 + k] = opw[k];
+                else pool.push_back(opw[k]);
+            }
             if (push_flag[v]) fl |= kB_Pop;
             if (nops > 0xFFFFu) { err = "a node has more than 65535 exchanged operands"; return EMO_E_UNSUPPORTED; }
             const int64_t A = lbQ[v] + lbES[v];
             r[0] = fl | (nops << kB_NopsShift);
+            // a simple entry (see emo_flow.h) names its one operand slot in word 3
+            {
+                const bool in_ok = nops == 0 || (nops == 1 && simple_in_off != kNone);
+                const bool out_ok = !(fl & kB_OutTag) && (!(fl & kB_OutSet) || useB[v].pre);
+                if ((fl & kB_HasReg) && in_ok && out_ok) {
+                    r[0] |= kB_Simple;
+                    if (nops == 1) r[3] = simple_in_off;
+                }
+            }
             r[4] = (uint32_t)(uint64_t)A;
             r[5] = (uint32_t)((uint64_t)A >> 32);
             r[6] = (uint32_t)v;
         }
     }
-    // runs of plain forward entries: started from the lane's previous value alone, nothing else to do.
-    // A run stays inside one period of one stage.
-    for (int st = 0; st < stages; ++st)
-        for (int ln = 0; ln < lanes; ++ln) {
-            const uint32_t h0 = out.hdr[((size_t)st * lanes + ln) * kHdrWords];
-            int base = 0;
-            for (int p = 0; p < nper; ++p) {
-                const int c = (int)((h0 >> (8 * p)) & 255u);
-                uint32_t next_run = 0;
-                for (int i = base + c - 1; i >= base; --i) {
-                    uint32_t &w = out.f.rec[(((size_t)st * lanes + ln) * K + i) * kFRecWords];
-                    const bool plain = w == kF_HasReg;
-                    const uint32_t run = plain ? std::min<uint32_t>(next_run + 1, 255u) : 0u;
-                    w |= run;
-                    next_run = run;
+    // ---- segments ------------------------------------------------------------------------------------
+    // The kernels walk a lane's entries of a stage in segments: an optional entry that needs its
+    // record (anything but a simple entry) followed by a run of up to kFlowRun simple entries, whose
+    // look-ups are issued together.  A segment stays inside one period; the first segment of a period
+    // carries the barrier flag (a lane without entries in a period gets an empty one).
+    out.f.seg.assign((size_t)stages * lanes * kSegBytes, 0);
+    out.b.seg.assign((size_t)stages * lanes * kSegBytes, 0);
+    {
+        const int nper_ = K / sync;
+        std::vector<std::vector<int32_t>> ents((size_t)stages * lanes);      // nodes per (stage, lane) by position
+        for (int32_t v : by_step) ents[(size_t)(step_of[v] / K) * lanes + lane_of[v]].push_back(v);
+        for (int st = 0; st < stages; ++st)
+            for (int ln = 0; ln < lanes; ++ln) {
+                const std::vector<int32_t> &ev = ents[(size_t)st * lanes + ln];
+                uint32_t *h = &out.hdr[((size_t)st * lanes + ln) * kHdrWords];
+                for (int dir = 0; dir < 2; ++dir) {
+                    uint8_t *sg = (dir ? out.b.seg.data() : out.f.seg.data()) + ((size_t)st * lanes + ln) * kSegBytes;
+                    int nseg = 0;
+                    for (int pi = 0; pi < nper_; ++pi) {
+                        const int p = dir ? nper_ - 1 - pi : pi;
+                        bool first = true, open = false;
+                        uint32_t kind = 0;
+                        auto start = [&](uint8_t byte) {
+                            sg[nseg++] = (uint8_t)(byte | (first ? kSegBarrier : 0));
+                            first = false;
+                        };
+                        const int ne = (int)ev.size();
+                        for (int ii = 0; ii < ne; ++ii) {
+                            const int32_t v = ev[dir ? ne - 1 - ii : ii];
+                            if ((step_of[v] % K) / sync != p) continue;
+                            const size_t q = slot_index(v);
+                            bool simple;
+                            uint32_t k2 = 0;
+                            if (!dir) {
+                                simple = out.f.rec[q * kFRecWords] == kF_HasReg;
+                            } else {
+                                const uint32_t w = out.b.rec[q * kBRecWords];
+                                simple = (w & kB_Simple) != 0;
+                                k2 = ((w >> kB_NopsShift) ? kSegIn : 0u) | ((w & kB_OutSet) ? kSegOut : 0u);
+                            }
+                            if (!simple) {
+                                start(kSegSpecial);
+                                open = true;          // a run may follow the special entry
+                                kind = 0xFFu;         // ... of whatever kind comes first
+                                continue;
+                            }
+                            uint8_t &cur = sg[nseg > 0 ? nseg - 1 : 0];
+                            if (open && (cur & kSegRunMask) < kFlowRun && (kind == 0xFFu || kind == k2)) {
+                                if (kind == 0xFFu) cur = (uint8_t)(cur | k2);
+                                cur = (uint8_t)(cur + 1);
+                            } else {
+                                start((uint8_t)(1u | k2));
+                                open = true;
+                            }
+                            kind = k2;
+                        }
+                        if (first) start(0);
+                    }
+                    if (nseg > kSegBytes) { err = "internal: too many segments"; return EMO_E_UNSUPPORTED; }
+                    h[0] |= (uint32_t)nseg << (dir ? 8 : 0);
                 }
-                base += c;
+                h[0] |= (uint32_t)ev.size() << 16;
             }
-        }
+    }
     // restore list: rows per stage and lane
     out.push_base.assign((size_t)stages + 1, 0);
     for (int st = 0; st < stages; ++st) {
         uint32_t off = 0;
         for (int ln = 0; ln < lanes; ++ln) {
             uint32_t *h = &out.hdr[((size_t)st * lanes + ln) * kHdrWords];
-            h[1] = npush[(size_t)st * lanes + ln];
-            h[2] = off;
-            off += h[1];
+            h[4] = npush[(size_t)st * lanes + ln];
+            h[5] = off;
+            h[6] = (uint32_t)out.push_base[st];
+            off += h[4];
         }
         out.push_base[st + 1] = out.push_base[st] + off;
     }

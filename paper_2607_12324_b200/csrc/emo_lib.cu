@@ -4,6 +4,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <cstdlib>
 #include <new>
 #include <string>
 #include <vector>
@@ -14,6 +15,7 @@
 #include "emo_kernels.cuh"
 #include "emo_pass_lane.cuh"
 #include "emo_pass_staged.cuh"
+#include "emo_flow.cuh"
 
 using namespace emo;
 
@@ -32,12 +34,25 @@ struct DevProgramLane {
     unsigned tab_entry = 0;
 };
 
+// The lane-stream program on the device: one blob per stage and direction (see emo_flow.cuh).
+struct DevFlow {
+    unsigned char *blobF = nullptr, *blobB = nullptr;
+    uint32_t *rows = nullptr, *push_base = nullptr;
+    unsigned blobF_bytes = 0, blobB_bytes = 0;
+    unsigned off_seg = 0;
+    unsigned f_off_rec = 0, f_off_pool = 0, f_off_tab = 0;
+    unsigned b_off_rec = 0, b_off_pool = 0, b_off_lbes = 0, b_off_tab = 0;
+    int max_push = 0;               // most restore rows of one stage
+    bool ready = false;
+};
+
 struct emo_graph {
     HostGraph h;
     Program fwd, bwd;
     Flow flow;                       // lane-stream program of the 32-bit pass kernels (flow.ok32: usable)
     DevProgram dfwd, dbwd;
     DevProgramLane lfwd, lbwd;       // only for programs of at most kLaneMaxLanes lanes
+    DevFlow dflow;
     bool host_only = false;
     int device = 0;
     int sm_count = 148;
@@ -301,8 +316,8 @@ bool lane_shape(const emo_graph *g, const Program &p, bool backward, int64_t NB,
 struct PassPlan {
     bool staged = false;
     bool lane_f = false, lane_b = false;   // staged, one policy per thread (forward / backward pass)
-    LaunchShape sf, sb;       // forward / backward launch shapes
-    StagedParams pf, pb;
+    LaunchShape sf{}, sb{};   // forward / backward launch shapes
+    StagedParams pf{}, pb{};
     size_t spill_bytes = 0;   // tiled spill: [tiles][rows of the backward program][backward tile]
 };
 
@@ -475,6 +490,234 @@ int launch_pass(const emo_graph *g, const PassPlan &pl, bool backward, int64_t B
     return EMO_OK;
 }
 
+
+// ---- lane-stream program: upload, launch shape, launches -------------------------------------------
+long long *g_flow_prof = nullptr;           // optional device array for the kernels' cycle counters (measurement hook)
+long long g_wait_cycles = 4000000000LL;    // bound of every device-side wait of the 32-bit kernels (about two seconds)
+
+int upload_flow(const Flow &f, DevFlow &d)
+{
+    if (!f.ok32 || f.stages == 0) return EMO_OK;
+    const size_t per = (size_t)f.lanes * f.K;
+    auto r16 = [](size_t x) { return (x + 15) / 16 * 16; };
+    d.off_seg = (unsigned)r16((size_t)f.lanes * kHdrWords * 4);
+    d.f_off_rec = (unsigned)r16(d.off_seg + (size_t)f.lanes * kSegBytes);
+    d.f_off_pool = (unsigned)r16(d.f_off_rec + per * kFRecWords * 4);
+    d.f_off_tab = (unsigned)r16(d.f_off_pool + (size_t)f.f.pool_stride * 4);
+    d.blobF_bytes = (unsigned)r16(d.f_off_tab + per * f.Lp * 12);
+    d.b_off_rec = d.f_off_rec;
+    d.b_off_pool = (unsigned)r16(d.b_off_rec + per * kBRecWords * 4);
+    d.b_off_lbes = (unsigned)r16(d.b_off_pool + (size_t)f.b.pool_stride * 4);
+    d.b_off_tab = (unsigned)r16(d.b_off_lbes + per * 8);
+    d.blobB_bytes = (unsigned)r16(d.b_off_tab + per * f.Lp * 4);
+    std::vector<unsigned char> bf((size_t)f.stages * d.blobF_bytes, 0), bb((size_t)f.stages * d.blobB_bytes, 0);
+    std::vector<uint32_t> pb((size_t)f.stages + 1);
+    for (int st = 0; st <= f.stages; ++st) pb[st] = (uint32_t)f.push_base[st];
+    for (int st = 0; st < f.stages; ++st) {
+        d.max_push = std::max(d.max_push, (int)(pb[st + 1] - pb[st]));
+        std::vector<uint32_t> hdr(f.hdr.begin() + (size_t)st * f.lanes * kHdrWords, f.hdr.begin() + (size_t)(st + 1) * f.lanes * kHdrWords);
+        unsigned char *F = bf.data() + (size_t)st * d.blobF_bytes, *Bk = bb.data() + (size_t)st * d.blobB_bytes;
+        std::memcpy(F, hdr.data(), hdr.size() * 4);
+        std::memcpy(Bk, hdr.data(), hdr.size() * 4);
+        std::memcpy(F + d.off_seg, &f.f.seg[(size_t)st * f.lanes * kSegBytes], (size_t)f.lanes * kSegBytes);
+        std::memcpy(Bk + d.off_seg, &f.b.seg[(size_t)st * f.lanes * kSegBytes], (size_t)f.lanes * kSegBytes);
+        std::memcpy(F + d.f_off_rec, &f.f.rec[(size_t)st * per * kFRecWords], per * kFRecWords * 4);
+        std::memcpy(F + d.f_off_pool, &f.f.pool[(size_t)st * f.f.pool_stride], (size_t)f.f.pool_stride * 4);
+        std::memcpy(F + d.f_off_tab, &f.tabF[(size_t)st * per * f.Lp * 3], per * f.Lp * 12);
+        std::memcpy(Bk + d.b_off_rec, &f.b.rec[(size_t)st * per * kBRecWords], per * kBRecWords * 4);
+        std::memcpy(Bk + d.b_off_pool, &f.b.pool[(size_t)st * f.b.pool_stride], (size_t)f.b.pool_stride * 4);
+        std::memcpy(Bk + d.b_off_lbes, &f.lbes[(size_t)st * per], per * 8);
+        std::memcpy(Bk + d.b_off_tab, &f.tabB[(size_t)st * per * f.Lp], per * f.Lp * 4);
+    }
+    int rc = upload(&d.blobF, bf.data(), bf.size());
+    if (rc == EMO_OK) rc = upload(&d.blobB, bb.data(), bb.size());
+    if (rc == EMO_OK) rc = upload(&d.rows, f.rows.data(), f.rows.size() * 4);
+    if (rc == EMO_OK) rc = upload(&d.push_base, pb.data(), pb.size() * 4);
+    d.ready = rc == EMO_OK;
+    return rc;
+}
+
+void free_flow(DevFlow &d)
+{
+    if (d.blobF) cudaFree(d.blobF);
+    if (d.blobB) cudaFree(d.blobB);
+    if (d.rows) cudaFree(d.rows);
+    if (d.push_base) cudaFree(d.push_base);
+    d = DevFlow();
+}
+
+// Launch shape of the 32-bit kernels: both passes use the same policy tile (the restore list is laid
+// out by tile), as many groups per block as cover the SMs once, two stage buffers (three when they fit).
+struct FlowPlan {
+    bool ok = false;
+    int groups = 0, grid_f = 0, grid_b = 0, threads = 0;
+    FlowParams pf, pb;
+    size_t smem_f = 0, smem_b = 0;
+    size_t restore_bytes = 0;
+};
+
+bool flow_plan(const emo_graph *g, int64_t B, bool want_base, bool need_bwd, FlowPlan &pl)
+{
+    const Flow &f = g->flow;
+    const DevFlow &d = g->dflow;
+    pl.ok = false;
+    if (!f.ok32 || !d.ready || !g->smem_optin || f.stages == 0) return false;
+    if (f.lanes * f.K > 32 * kFlowRowRegs) return false;
+    const int64_t NBf = B + (want_base ? 1 : 0);
+    const int64_t n_groups = (NBf + 31) / 32;
+    const int gmax = std::min((32 - 2) / f.lanes, 15);
+    if (gmax < 1) return false;
+    const int64_t want = (n_groups + g->sm_count - 1) / g->sm_count;
+    const size_t budget = g->smem_optin;
+    for (int G = (int)std::max<int64_t>(1, std::min<int64_t>(gmax, want)); G >= 1; --G) {
+        // four producer warps where the block has room for them (they share the level-row pieces)
+        const int nprod = G * f.lanes + 4 <= 24 ? 4 : 2;
+        const size_t P = 32 * (size_t)G;
+        const size_t lvl_bytes = (size_t)G * f.lanes * f.K * 32;
+        auto shape = [&](bool backward, FlowParams &p, size_t &smem) {
+            const FlowDir &dir = backward ? f.b : f.f;
+            const size_t slot_bytes = (size_t)dir.slots_tag * 256 + (size_t)dir.slots_set * 128;
+            const size_t blob = backward ? d.blobB_bytes : d.blobF_bytes;
+            const size_t rst = backward ? (size_t)d.max_push * P * 4 : 0;
+            const size_t stage = round_up(blob + lvl_bytes + rst, 128);
+            const size_t off_bar = round_up(G * slot_bytes, 16);
+            const size_t head = round_up(off_bar + 256, 128);
+            int nbuf = 0;
+            for (int nb = 3; nb >= 2; --nb)
+                if (head + nb * stage <= budget) { nbuf = nb; break; }
+            if (!nbuf || nbuf * stage < (size_t)G * f.lanes * 32 * 16) return false;
+            p = FlowParams();
+            p.blob = backward ? d.blobB : d.blobF;
+            p.rows = d.rows;
+            p.push_base = d.push_base;
+            p.blob_bytes = (unsigned)blob;
+            p.off_seg = d.off_seg;
+            p.off_rec = backward ? d.b_off_rec : d.f_off_rec;
+            p.off_pool = backward ? d.b_off_pool : d.f_off_pool;
+            p.off_tab = backward ? d.b_off_tab : d.f_off_tab;
+            p.off_lbes = backward ? d.b_off_lbes : 0;
+            p.tab_row = (unsigned)f.Lp * (backward ? 4u : 12u);
+            p.stages = f.stages;
+            p.lanes = f.lanes;
+            p.K = f.K;
+            p.kshift = 0;
+            while ((1 << p.kshift) < f.K) ++p.kshift;
+            p.Lp = f.Lp;
+            p.L = g->h.L;
+            p.groups = G;
+            p.ptile = (int)P;
+            p.nbuf = nbuf;
+            p.nprod = nprod;
+            p.slot_bytes = (unsigned)slot_bytes;
+            p.stage_bytes = (unsigned)stage;
+            p.off_lvl = (unsigned)blob;
+            p.off_rst = (unsigned)(blob + lvl_bytes);
+            p.off_bar = (unsigned)off_bar;
+            p.off_stage0 = (unsigned)head;
+            p.pushes = f.pushes;
+            p.restore_rows = f.pushes + f.lanes;
+            p.wait_cycles = g_wait_cycles;
+            p.stall_stage = -1;
+            p.prof = nullptr;
+            p.dbg = getenv("EMO_DBG") ? atoi(getenv("EMO_DBG")) : 0;
+            smem = head + nbuf * stage;
+            return true;
+        };
+        if (!shape(false, pl.pf, pl.smem_f)) continue;
+        if (need_bwd && !shape(true, pl.pb, pl.smem_b)) continue;
+        pl.groups = G;
+        pl.grid_f = (int)((n_groups + G - 1) / G);
+        pl.grid_b = (int)(((B + 31) / 32 + G - 1) / G);
+        pl.threads = (G * f.lanes + nprod) * 32;
+        pl.restore_bytes = need_bwd ? round_up((size_t)pl.grid_f * (size_t)(f.pushes + f.lanes) * P * 4, 256) : 0;
+        pl.ok = true;
+        return true;
+    }
+    return false;
+}
+
+// The opt-in shared-memory size is set once per kernel (not per launch: concurrent callers with
+// different batch sizes would otherwise race on the attribute).
+template <typename K>
+int flow_optin(K kern, const emo_graph *g)
+{
+    return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g->smem_optin) == cudaSuccess ? EMO_OK : EMO_E_CUDA;
+}
+
+int launch_flow_fwd(const emo_graph *g, const FlowPlan &pl, int64_t B, const uint8_t *lvl, int64_t ldb, uint32_t *restore,
+                    int64_t *makespan, double *energy, int64_t *base_T, double *base_E, int32_t *status, uint32_t flags,
+                    cudaStream_t st)
+{
+    FlowParams p = pl.pf;
+    p.want_base = (base_T || base_E) ? 1 : 0;
+    if (B + p.want_base == 0) return EMO_OK;
+    p.B = B;
+    p.lvl = lvl;
+    p.ldb = ldb;
+    p.restore = restore;
+    p.makespan = makespan;
+    p.energy = energy;
+    p.base_T = base_T;
+    p.base_E = base_E;
+    p.status = status;
+    p.prof = g_flow_prof;
+    if (flags & EMO_F_TEST_STALL) p.stall_stage = p.stages / 2;
+    cudaEvent_t ev0 = g_pass_events[0], ev1 = g_pass_events[1];
+    if (ev0) EMO_CUDA(cudaEventRecord(ev0, st));
+    void (*kern)(FlowParams) = pl.threads <= 512 ? emo_flow_fwd<512> : (pl.threads <= 768 ? emo_flow_fwd<768> : emo_flow_fwd<1024>);
+    if (flow_optin(kern, g) != EMO_OK) { (void)cudaGetLastError(); return EMO_E_CUDA; }
+    kern<<<pl.grid_f, pl.threads, pl.smem_f, st>>>(p);
+    EMO_CUDA(cudaGetLastError());
+    if (ev1) EMO_CUDA(cudaEventRecord(ev1, st));
+    return EMO_OK;
+}
+
+int launch_flow_bwd(const emo_graph *g, const FlowPlan &pl, int64_t B, const uint8_t *lvl, int64_t ldb, uint32_t *restore,
+                    int64_t *ES, int64_t *LS, int64_t *slack, int64_t ldo, int64_t *makespan, int64_t *slack_sum,
+                    int32_t *n_critical, int32_t *status, uint32_t flags, cudaStream_t st)
+{
+    if (B == 0) return EMO_OK;
+    FlowParams p = pl.pb;
+    p.B = B;
+    p.lvl = lvl;
+    p.ldb = ldb;
+    p.restore = restore;
+    p.makespan = makespan;
+    p.ES = ES;
+    p.LS = LS;
+    p.slack = slack;
+    p.ldo = ldo;
+    p.slack_sum = slack_sum;
+    p.n_critical = n_critical;
+    p.status = status;
+    p.prof = g_flow_prof ? g_flow_prof + 65536 : nullptr;
+    if (flags & EMO_F_TEST_STALL) p.stall_stage = p.stages / 2;
+    cudaEvent_t ev0 = g_pass_events[2], ev1 = g_pass_events[3];
+    if (ev0) EMO_CUDA(cudaEventRecord(ev0, st));
+    const bool extra = ES || LS || slack_sum || n_critical;
+    void (*kern)(FlowParams) = nullptr;
+#define EMO_PICK_F(MAXT) kern = extra ? emo_flow_bwd<true, MAXT> : emo_flow_bwd<false, MAXT>
+    if (pl.threads <= 512) EMO_PICK_F(512);
+    else if (pl.threads <= 768) EMO_PICK_F(768);
+    else EMO_PICK_F(1024);
+#undef EMO_PICK_F
+    if (flow_optin(kern, g) != EMO_OK) { (void)cudaGetLastError(); return EMO_E_CUDA; }
+    kern<<<pl.grid_b, pl.threads, pl.smem_b, st>>>(p);
+    EMO_CUDA(cudaGetLastError());
+    if (ev1) EMO_CUDA(cudaEventRecord(ev1, st));
+    return EMO_OK;
+}
+
+// Whether a call may take the 32-bit kernels: the program exists, the caller did not ask for another
+// kernel, and the level matrix can be fetched in 16-byte pieces.
+bool flow_allowed(const emo_graph *g, const uint8_t *lvl, int64_t ldb, int64_t ldo, uint32_t flags)
+{
+    const int64_t big = (int64_t)1 << 28;
+    if (!g->flow.ok32 || !g->dflow.ready) return false;
+    if (flags & (EMO_F_NO_STAGING | EMO_F_PAIR_KERNEL | EMO_F_LANE_KERNEL)) return false;
+    return ldb % 16 == 0 && aligned16(lvl) && ldb < big && ldo < big;
+}
+
 int launch_validate(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t ldb, int32_t *status, cudaStream_t st)
 {
     if (!status) return EMO_E_INVALID_ARG;
@@ -516,6 +759,34 @@ int emo_set_pass_events(void *fwd_start, void *fwd_stop, void *bwd_start, void *
     return EMO_OK;
 }
 
+int emo_call_path(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t ldb, int64_t ldo, int need_slack, uint32_t flags)
+{
+    if (!g || B < 0) return EMO_E_INVALID_ARG;
+    if (g->host_only) return EMO_E_CUDA;
+    if (flow_allowed(g, lvl, ldb, need_slack ? ldo : 0, flags)) {
+        FlowPlan fp;
+        if (flow_plan(g, B, true, need_slack != 0, fp)) return 2;
+    }
+    PassPlan pl;
+    const int64_t ld_ws = (int64_t)round_up((size_t)B, 16);
+    int rc = make_plan(g, B, true, need_slack != 0, lvl, ldb, ld_ws, ldo, flags, pl);
+    if (rc) return rc;
+    return pl.staged ? 1 : 0;
+}
+
+int emo_set_flow_counters(void *dev)
+{
+    g_flow_prof = (long long *)dev;
+    return EMO_OK;
+}
+
+int emo_set_wait_limit(int64_t cycles)
+{
+    if (cycles <= 0) return EMO_E_INVALID_ARG;
+    g_wait_cycles = cycles;
+    return EMO_OK;
+}
+
 int emo_graph_load(int32_t n, const int64_t *row_ptr, const int32_t *col, const int32_t *level_ptr,
                    int32_t n_levels, int32_t L, const int64_t *lat, const double *energy,
                    const int32_t *group_of, uint32_t flags, emo_graph **out)
@@ -538,15 +809,20 @@ int emo_graph_load(int32_t n, const int64_t *row_ptr, const int32_t *col, const 
             max_span = std::max(max_span, v - col[e]);
         }
     if (level_ptr) {
+        // the whole array is checked before anything is indexed with it
         if (n_levels < 0 || level_ptr[0] != 0 || level_ptr[n_levels] != n) return EMO_E_INVALID_ARG;
-        std::vector<int32_t> lev((size_t)std::max(n, 1));
-        for (int32_t l = 0; l < n_levels; ++l) {
-            if (level_ptr[l + 1] < level_ptr[l]) return EMO_E_INVALID_ARG;
-            for (int32_t v = level_ptr[l]; v < level_ptr[l + 1]; ++v) lev[v] = l;
+        for (int32_t l = 0; l < n_levels; ++l)
+            if (level_ptr[l] < 0 || level_ptr[l + 1] > n || level_ptr[l + 1] < level_ptr[l]) return EMO_E_INVALID_ARG;
+        try {
+            std::vector<int32_t> lev((size_t)std::max(n, 1));
+            for (int32_t l = 0; l < n_levels; ++l)
+                for (int32_t v = level_ptr[l]; v < level_ptr[l + 1]; ++v) lev[v] = l;
+            for (int32_t v = 0; v < n; ++v)
+                for (int64_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e)
+                    if (lev[col[e]] >= lev[v]) return EMO_E_NOT_TOPOLOGICAL;
+        } catch (const std::bad_alloc &) {
+            return EMO_E_OOM;
         }
-        for (int32_t v = 0; v < n; ++v)
-            for (int64_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e)
-                if (lev[col[e]] >= lev[v]) return EMO_E_NOT_TOPOLOGICAL;
     }
     for (int64_t i = 0; i < (int64_t)n * L; ++i) {
         if (lat[i] < 0 || lat[i] >= ((int64_t)1 << 32)) return EMO_E_RANGE;
@@ -614,7 +890,14 @@ int emo_graph_load(int32_t n, const int64_t *row_ptr, const int32_t *col, const 
         if (rc == EMO_OK) rc = compile_dir(false, &g->bwd.pos_of_node, g->fwd);
         if (rc != EMO_OK) { delete g; return rc; }
         {
-            const int fk = (int)((flags >> 24) & 0x3F), fs = (int)((flags >> 4) & 0xF) * 8;
+            // stage length: the longest of 32, 16, 8 steps whose entries the producers can index
+            // (32 * kFlowRowRegs per stage); barrier distance 16 steps unless the caller says otherwise
+            // (measured on the 250 000-node workload at 0.3 scale: 8 / 16 steps gave 8.5 / 7.7 ms for both passes)
+            int fk = (int)((flags >> 24) & 0x3F), fs = (int)((flags >> 4) & 0xF) * 8;
+            const int flanes = g->fwd.lanes > 0 ? std::max(g->fwd.lanes, g->bwd.lanes) : 1;
+            if (fk == 0) fk = flanes * 32 <= 32 * kFlowRowRegs ? 32 : (flanes * 16 <= 32 * kFlowRowRegs ? 16 : 8);
+            if (fs == 0) fs = 16;
+            if (fs > fk) fs = fk;
             rc = compile_flow(h, lat, energy, lanes, look, fk, fs, g->flow, err);
             if (rc != EMO_OK) { delete g; return rc; }
         }
@@ -640,11 +923,17 @@ int emo_graph_load(int32_t n, const int64_t *row_ptr, const int32_t *col, const 
         g->device = dev;
         g->sm_count = prop.multiProcessorCount;
         g->smem_optin = prop.sharedMemPerBlockOptin;
-        int rc = upload_program(g->fwd, g->dfwd);
+        int rc = EMO_OK;
+        try {
+        rc = upload_program(g->fwd, g->dfwd);
         if (rc == EMO_OK) rc = upload_program(g->bwd, g->dbwd);
         if (rc == EMO_OK && g->fwd.lanes <= 32 - kProducerWarps && g->bwd.lanes <= 32 - kProducerWarps) {
             rc = upload_program_lane(g->fwd, g->lfwd);
             if (rc == EMO_OK) rc = upload_program_lane(g->bwd, g->lbwd);
+        }
+        if (rc == EMO_OK) rc = upload_flow(g->flow, g->dflow);
+        } catch (const std::bad_alloc &) {
+            rc = EMO_E_OOM;
         }
         if (rc != EMO_OK) { emo_graph_free(g); return rc; }
     }
@@ -660,6 +949,7 @@ int emo_graph_free(emo_graph *g)
         free_program(g->dbwd);
         free_program_lane(g->lfwd);
         free_program_lane(g->lbwd);
+        free_flow(g->dflow);
     }
     delete g;
     return EMO_OK;
@@ -720,6 +1010,8 @@ int emo_graph_flow(const emo_graph *g, emo_flow_view *v)
     v->pool_fwd = f.f.pool.data();
     v->rec_bwd = f.b.rec.data();
     v->pool_bwd = f.b.pool.data();
+    v->seg_fwd = f.f.seg.data();
+    v->seg_bwd = f.b.seg.data();
     v->lbes = f.lbes.data();
     v->push_base = f.push_base.data();
     return EMO_OK;
@@ -771,7 +1063,13 @@ int emo_workspace_bytes(const emo_graph *g, int64_t B, int need_slack, size_t *o
 {
     if (!g || !out || B < 0) return EMO_E_INVALID_ARG;
     size_t bytes = kSmallWs + lvl_area(g);
-    if (need_slack) bytes += spill_need(g, B);
+    if (need_slack) {
+        // either family of kernels may run (the call's flags and the caller's pitches decide)
+        size_t need = spill_need(g, B);
+        FlowPlan fp;
+        if (!g->host_only && B > 0 && flow_plan(g, B, true, true, fp)) need = std::max(need, fp.restore_bytes);
+        bytes += need;
+    }
     if (need_slack == 2) bytes += 4 * round_up((size_t)B * 8, 256) + 256;
     *out = bytes;
     return EMO_OK;
@@ -793,6 +1091,11 @@ int emo_eval_policies(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t
         if (rc) return rc;
     }
     if (B == 0) { lvl = nullptr; ldb = 0; }
+    if (flow_allowed(g, lvl, ldb, 0, flags)) {
+        FlowPlan fp;
+        if (flow_plan(g, B, T0 || E0, false, fp))
+            return launch_flow_fwd(g, fp, B, lvl, ldb, nullptr, makespan, energy, T0, E0, status, flags, st);
+    }
     PassPlan pl;
     int rc = make_plan(g, B, T0 || E0, false, lvl, ldb, 0, 0, flags, pl);
     if (rc) return rc;
@@ -814,6 +1117,18 @@ int emo_slack_batch(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t l
     if (flags & EMO_F_VALIDATE) {
         int rc = launch_validate(g, B, lvl, ldb, status, st);
         if (rc) return rc;
+    }
+    if (flow_allowed(g, lvl, ldb, ldo, flags)) {
+        FlowPlan fp;
+        if (flow_plan(g, B, T0 || E0, true, fp)) {
+            const size_t head = kSmallWs + lvl_area(g);
+            if (!ws || ws_bytes < head + fp.restore_bytes) return EMO_E_OOM;
+            uint32_t *restore = (uint32_t *)((char *)ws + head);
+            int rc = launch_flow_fwd(g, fp, B, lvl, ldb, restore, makespan, energy, T0, E0, status, flags, st);
+            if (rc) return rc;
+            return launch_flow_bwd(g, fp, B, lvl, ldb, restore, ES, LS, slack, ldo, makespan, slack_sum, n_critical, status,
+                                   flags, st);
+        }
     }
     const int64_t ld_ws = (int64_t)round_up((size_t)B, 16);
     PassPlan pl;

@@ -23,12 +23,13 @@ EMO_F_VALIDATE = 0x1
 EMO_F_NO_STAGING = 0x2
 EMO_F_PAIR_KERNEL = 0x4
 EMO_F_LANE_KERNEL = 0x8
+EMO_F_TEST_STALL = 0x100
 
 EXPORTS = [
     "emo_strerror", "emo_graph_load", "emo_graph_free", "emo_graph_info", "emo_workspace_bytes",
     "emo_eval_policies", "emo_slack_batch", "emo_slack", "emo_baseline", "emo_target_from_delta",
     "emo_select", "emo_transpose_policies", "emo_slack_batch_host", "emo_graph_program",
-    "emo_set_pass_events", "emo_select_static", "emo_graph_flow",
+    "emo_set_pass_events", "emo_select_static", "emo_graph_flow", "emo_set_wait_limit", "emo_call_path", "emo_set_flow_counters",
 ]
 
 
@@ -69,7 +70,7 @@ class emo_flow_view(ctypes.Structure):
                                                 "pool_stride_bwd")] +
                 [(k, ctypes.c_int64) for k in ("pushes", "pruned_fwd", "pruned_bwd")] +
                 [(k, ctypes.c_void_p) for k in ("hdr", "rows", "node", "step", "tab_fwd", "tab_bwd", "rec_fwd", "pool_fwd",
-                                                "rec_bwd", "pool_bwd", "lbes", "push_base")])
+                                                "rec_bwd", "pool_bwd", "seg_fwd", "seg_bwd", "lbes", "push_base")])
 
 
 _lib = None
@@ -104,6 +105,9 @@ def lib():
                                         ctypes.POINTER(p), ctypes.POINTER(p)]
         L.emo_set_pass_events.argtypes = [p, p, p, p]
         L.emo_graph_flow.argtypes = [p, ctypes.POINTER(emo_flow_view)]
+        L.emo_set_wait_limit.argtypes = [i64]
+        L.emo_set_flow_counters.argtypes = [p]
+        L.emo_call_path.argtypes = [p, i64, p, i64, i64, ctypes.c_int, u32]
         L.emo_select_static.argtypes = [i64, p, p, i64, p, i64, p, p, p, p]
         for name in EXPORTS:
             if name not in ("emo_strerror", "emo_target_from_delta"):
@@ -310,15 +314,33 @@ def emo_graph_flow(g: Graph) -> dict:
         return np.ctypeslib.as_array(ctypes.cast(ptr, ctypes.POINTER(ctype)), shape=(count,)).astype(dtype, copy=True)
 
     u32, i64 = ctypes.c_uint32, ctypes.c_int64
-    out["hdr"] = arr(v.hdr, v.stages * v.lanes * 4, u32, np.uint32).reshape(v.stages, v.lanes, 4)
+    out["hdr"] = arr(v.hdr, v.stages * v.lanes * 8, u32, np.uint32).reshape(v.stages, v.lanes, 8)
     for k in ("rows", "node", "step"):
         out[k] = arr(getattr(v, k), q, u32, np.uint32).reshape(v.stages, v.lanes, v.K)
     out["tab_fwd"] = arr(v.tab_fwd, q * v.Lp * 3, u32, np.uint32).reshape(v.stages, v.lanes, v.K, v.Lp, 3)
     out["tab_bwd"] = arr(v.tab_bwd, q * v.Lp, u32, np.uint32).reshape(v.stages, v.lanes, v.K, v.Lp)
-    out["rec_fwd"] = arr(v.rec_fwd, q * 4, u32, np.uint32).reshape(v.stages, v.lanes, v.K, 4)
-    out["rec_bwd"] = arr(v.rec_bwd, q * 8, u32, np.uint32).reshape(v.stages, v.lanes, v.K, 8)
+    out["rec_fwd"] = arr(v.rec_fwd, q * 8, u32, np.uint32).reshape(v.stages, v.lanes, v.K, 8)
+    out["rec_bwd"] = arr(v.rec_bwd, q * 12, u32, np.uint32).reshape(v.stages, v.lanes, v.K, 12)
     out["pool_fwd"] = arr(v.pool_fwd, v.stages * v.pool_stride_fwd, u32, np.uint32).reshape(v.stages, v.pool_stride_fwd)
     out["pool_bwd"] = arr(v.pool_bwd, v.stages * v.pool_stride_bwd, u32, np.uint32).reshape(v.stages, v.pool_stride_bwd)
+    out["seg_fwd"] = arr(v.seg_fwd, v.stages * v.lanes * 40, ctypes.c_uint8, np.uint8).reshape(v.stages, v.lanes, 40)
+    out["seg_bwd"] = arr(v.seg_bwd, v.stages * v.lanes * 40, ctypes.c_uint8, np.uint8).reshape(v.stages, v.lanes, 40)
     out["lbes"] = arr(v.lbes, q, i64, np.int64).reshape(v.stages, v.lanes, v.K)
     out["push_base"] = arr(v.push_base, v.stages + 1, i64, np.int64)
     return out
+
+
+def emo_set_wait_limit(cycles: int):
+    _check(lib().emo_set_wait_limit(int(cycles)), "emo_set_wait_limit")
+
+
+def emo_call_path(g: Graph, B, lvl, ldb, ldo, need_slack: bool, flags: int = 0) -> int:
+    """2 = 32-bit lane-stream kernels, 1 = staged 64-bit kernels, 0 = plain-load kernels."""
+    rc = lib().emo_call_path(g.handle, int(B), _addr(lvl), int(ldb), int(ldo), int(bool(need_slack)), int(flags))
+    if rc < 0:
+        raise EmoError(rc, "emo_call_path")
+    return rc
+
+
+def emo_set_flow_counters(dev):
+    _check(lib().emo_set_flow_counters(_addr(dev)), "emo_set_flow_counters")

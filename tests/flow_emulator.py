@@ -12,6 +12,8 @@ from __future__ import annotations
 import numpy as np
 
 NONE = 0xFFFFFFFF
+SEG_SPECIAL, SEG_BARRIER, SEG_IN, SEG_OUT = 16, 32, 64, 128
+B_SIMPLE = 64
 F_HASREG, F_REGDELTA, F_OUTTAG, F_OUTSET, F_TERMINAL, F_PUSH, F_OUTACC = 1 << 8, 1 << 9, 1 << 10, 1 << 11, 1 << 12, 1 << 13, 1 << 14
 B_HASREG, B_REGDELTA, B_OUTTAG, B_OUTSET, B_POP, B_OUTACC = 1, 2, 4, 8, 16, 32
 OP_NOPOLL, OP_WORD, OP_CLEAR, OP_OFF = 1 << 31, 1 << 30, 1 << 29, (1 << 29) - 1
@@ -54,14 +56,43 @@ class _Slots:
 def _period_entries(f, st, p, reverse):
     """(step, lane, pos) of the entries of period p of stage st, in processing order."""
     out = []
-    nper = f["K"] // f["sync"]
     for ln in range(f["lanes"]):
-        h0 = int(f["hdr"][st, ln, 0])
-        cnts = [(h0 >> (8 * i)) & 255 for i in range(nper)]
-        base = sum(cnts[:p])
-        for pos in range(base, base + cnts[p]):
-            out.append((int(f["step"][st, ln, pos]), ln, pos))
+        for pos in range(f["K"]):
+            if int(f["node"][st, ln, pos]) == NONE:
+                break
+            step = int(f["step"][st, ln, pos])
+            if (step % f["K"]) // f["sync"] == p:
+                out.append((step, ln, pos))
     out.sort(reverse=reverse)
+    return out
+
+
+def segments(f, st, ln, backward):
+    """The segments of one lane of one stage as (barrier, special position or None, run positions, kind bits)."""
+    seg = f["seg_bwd" if backward else "seg_fwd"][st, ln]
+    h0 = int(f["hdr"][st, ln, 0])
+    nseg, total = (h0 >> 8) & 255 if backward else h0 & 255, (h0 >> 16) & 255
+    pos = total if backward else 0
+    out = []
+    for i in range(nseg):
+        b = int(seg[i])
+        special = None
+        if b & SEG_SPECIAL:
+            if backward:
+                pos -= 1
+                special = pos
+            else:
+                special = pos
+                pos += 1
+        r = b & 15
+        if backward:
+            run = list(range(pos - 1, pos - 1 - r, -1))
+            pos -= r
+        else:
+            run = list(range(pos, pos + r))
+            pos += r
+        out.append((bool(b & SEG_BARRIER), special, run, b & (SEG_IN | SEG_OUT)))
+    assert pos == (0 if backward else total)
     return out
 
 
@@ -92,15 +123,17 @@ def run_forward(f, lvl, L):
                 pp = int(rec[3])
                 hin = h[ln].copy()
                 v = hin.copy() if fl & F_HASREG else np.zeros(B, np.uint32)
-                if fl & F_REGDELTA:
-                    v = _floor_sub(v, pool[pp])
-                    pp += 1
-                for _ in range(fl >> 16):
-                    w, tag, delta = int(pool[pp]), int(pool[pp + 1]), int(pool[pp + 2])
-                    pp += 3
+                assert bool(fl & F_REGDELTA) == (int(rec[7]) != 0)
+                v = _floor_sub(v, rec[7])
+                for k in range(fl >> 16):
+                    if k == 0:      # the first operand sits in the record
+                        w, tag, delta = int(rec[4]), int(rec[5]), int(rec[6])
+                    else:
+                        w, tag, delta = int(pool[pp]), int(pool[pp + 1]), int(pool[pp + 2])
+                        pp += 3
                     v = np.maximum(v, _floor_sub(slots.read(w, tag, period), delta))
                 if fl & F_PUSH:
-                    restore[int(f["push_base"][st]) + int(f["hdr"][st, ln, 2]) + npushed[ln]] = hin
+                    restore[int(f["push_base"][st]) + int(f["hdr"][st, ln, 5]) + npushed[ln]] = hin
                     npushed[ln] += 1
                 else:
                     assert (fl & F_HASREG) and not (fl & F_REGDELTA) and (fl >> 16) == 0
@@ -115,7 +148,7 @@ def run_forward(f, lvl, L):
                     acc[ln] = np.maximum(acc[ln], lbc + v.astype(np.int64))
                 h[ln] = v
         for ln in range(lanes):
-            assert npushed[ln] == int(f["hdr"][st, ln, 1])
+            assert npushed[ln] == int(f["hdr"][st, ln, 4])
     for ln in range(lanes):
         restore[int(f["pushes"]) + ln] = h[ln]
     del cols
@@ -134,7 +167,7 @@ def run_backward(f, lvl, L, T, restore, n):
     slots = _Slots(B)
     T = T.astype(np.int64)
     for st in range(f["stages"] - 1, -1, -1):
-        npop = [int(f["hdr"][st, ln, 1]) for ln in range(lanes)]
+        npop = [int(f["hdr"][st, ln, 4]) for ln in range(lanes)]
         for p in range(nper - 1, -1, -1):
             period = (f["stages"] * nper - 1) - (st * nper + p)
             for _, ln, pos in _period_entries(f, st, p, True):
@@ -146,12 +179,21 @@ def run_backward(f, lvl, L, T, restore, n):
                 pool = f["pool_bwd"][st]
                 pp = int(rec[3])
                 qin = q[ln].copy() if fl & B_HASREG else np.zeros(B, np.uint32)
-                if fl & B_REGDELTA:
-                    qin = _floor_sub(qin, rec[7])
-                for _ in range(fl >> 16):
-                    w, tag, delta = int(pool[pp]), int(pool[pp + 1]), int(pool[pp + 2])
-                    pp += 3
-                    qin = np.maximum(qin, _floor_sub(slots.read(w, tag, period), delta))
+                assert bool(fl & B_REGDELTA) == (int(rec[7]) != 0)
+                qin = _floor_sub(qin, rec[7])
+                if fl & B_SIMPLE:
+                    # a simple entry: at most one operand, a settled single-reader slot named in word 3
+                    assert (fl & B_HASREG) and not (fl & B_OUTTAG) and (fl >> 16) <= 1
+                    if fl >> 16:
+                        qin = np.maximum(qin, slots.read(OP_WORD | OP_NOPOLL | OP_CLEAR | int(rec[3]), None, period))
+                else:
+                    for k in range(fl >> 16):
+                        if k == 0:
+                            w, tag, delta = int(rec[8]), int(rec[9]), int(rec[10])
+                        else:
+                            w, tag, delta = int(pool[pp]), int(pool[pp + 1]), int(pool[pp + 2])
+                            pp += 3
+                        qin = np.maximum(qin, _floor_sub(slots.read(w, tag, period), delta))
                 A = int(rec[4]) | (int(rec[5]) << 32)
                 v = int(rec[6])
                 sl = T - A - (qin.astype(np.int64) + c[ln].astype(np.int64))
@@ -165,7 +207,7 @@ def run_backward(f, lvl, L, T, restore, n):
                 SL[v], ES[v], LS[v] = sl, es, sl + es
                 if fl & B_POP:
                     npop[ln] -= 1
-                    c[ln] = restore[int(f["push_base"][st]) + int(f["hdr"][st, ln, 2]) + npop[ln]]
+                    c[ln] = restore[int(f["push_base"][st]) + int(f["hdr"][st, ln, 5]) + npop[ln]]
                 else:
                     c[ln] = eo
                 q[ln] = qn

@@ -218,6 +218,11 @@ def test_load_rejects_bad_input(emo):
     assert code(L=256) == E.EMO_E_RANGE
     assert code(level_ptr=np.array([0, 1, 2, 3], np.int32)) == 0
     assert code(level_ptr=np.array([0, 2, 3], np.int32)) == E.EMO_E_NOT_TOPOLOGICAL   # 0 and 1 share a level but 0->1
+    # a malformed level array is rejected before it is used as an index (entries out of [0, n], not monotone)
+    assert code(level_ptr=np.array([0, 1_000_000, 3], np.int32)) == E.EMO_E_INVALID_ARG
+    assert code(level_ptr=np.array([0, 2, 1, 3], np.int32)) == E.EMO_E_INVALID_ARG
+    assert code(level_ptr=np.array([0, -5, 3], np.int32)) == E.EMO_E_INVALID_ARG
+    assert code(level_ptr=np.array([1, 2, 3], np.int32)) == E.EMO_E_INVALID_ARG
     assert code(group_of=np.array([0, -2, 1], np.int32)) == E.EMO_E_INVALID_ARG
     assert code(n=-1) == E.EMO_E_INVALID_ARG
 
