@@ -56,7 +56,6 @@ struct FlowParams {
     int32_t *status;
     long long wait_cycles;               // bound of every device-side wait
     int stall_stage;                     // test hook: the producers stop before this stage (-1: off)
-    int dbg;                             // TEMPORARY timing experiments
     long long *prof;                     // optional cycle counters, 4 per warp: waits for stages, group barriers, total, spare
 };
 
@@ -133,6 +132,24 @@ __device__ __forceinline__ long long emo_tld_s64(unsigned a, unsigned tok)
     long long v;
     asm("ld.shared.s64 %0, [%1]; // %2" : "=l"(v) : "r"(a), "r"(tok));
     return v;
+}
+// the staged word when `take` is set, else `other` (no access, no branch)
+__device__ __forceinline__ unsigned emo_tld_u32_if(unsigned a, unsigned tok, unsigned take, unsigned other)
+{
+    unsigned v = other;
+    asm("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\t@p ld.shared.u32 %0, [%1]; // %3\n\t}" : "+r"(v) : "r"(a), "r"(take), "r"(tok));
+    return v;
+}
+// st.global under a predicate (no branch)
+__device__ __forceinline__ void emo_stg_s64_if(long long *base, unsigned row, unsigned pitch_bytes, long long v, unsigned ok)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .u64 a;\n\t"
+        "setp.ne.u32 p, %4, 0;\n\t"
+        "mad.wide.u32 a, %1, %2, %0;\n\t"
+        "@p st.global.s64 [a], %3;\n\t}"
+        ::"l"(base), "r"(row), "r"(pitch_bytes), "l"(v), "r"(ok)
+        : "memory");
 }
 __device__ __forceinline__ uint4 emo_tld_128(unsigned a, unsigned tok)
 {
@@ -598,6 +615,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_flow_bwd(FlowParams p)
         const unsigned ldo8 = (unsigned)p.ldo * 8u;
         const unsigned ptile4 = (unsigned)ptile * 4u;
         long long *const sl_lane = (p.slack && act) ? reinterpret_cast<long long *>(p.slack) + b : nullptr;
+        const unsigned sl_ok = sl_lane != nullptr;
         long long *const es_lane = (EXTRA && p.ES && act) ? reinterpret_cast<long long *>(p.ES) + b : nullptr;
         long long *const ls_lane = (EXTRA && p.LS && act) ? reinterpret_cast<long long *>(p.LS) + b : nullptr;
         const bool want_sums = EXTRA && (p.slack_sum || p.n_critical) && act;
@@ -625,33 +643,51 @@ __global__ void __launch_bounds__(MAXT, 1) emo_flow_bwd(FlowParams p)
                 }
             }
         };
-        // a run of R simple entries at positions rec_a .. (lowest first in memory, walked from the highest down)
-        auto run = [&](auto rc) {
+        // R simple entries of one kind at positions o .. o + R - 1 of the run (lowest first in memory, walked
+        // from the highest down).  Straight-line code without a branch (the kind is a compile-time parameter,
+        // stores and the restore pop are predicated), so that the look-ups, the record loads and the slack
+        // arithmetic of all R entries overlap and only the two running values form a chain.
+        auto run = [&](auto rc, auto inc, auto outc, unsigned o) {
             constexpr int R = decltype(rc)::value;
+            constexpr bool IN = decltype(inc)::value, OUT = decltype(outc)::value;
+            const unsigned rec_o = rec_a + 48u * o, tab_o = tab_a + o * tab_row, lvl_o = lvl_a + 32u * o, xes_o = xes_a + 8u * o;
             unsigned lv[R], d[R];
 #pragma unroll
-            for (int j = 0; j < R; ++j) lv[j] = emo_tld_u8(lvl_a + 32u * j, tok);
+            for (int j = 0; j < R; ++j) lv[j] = emo_tld_u8(lvl_o + 32u * j, tok);
 #pragma unroll
-            for (int j = 0; j < R; ++j) d[j] = emo_tld_u32(tab_a + (unsigned)j * tab_row + (lv[j] & lmask) * 4u, tok);
+            for (int j = 0; j < R; ++j) d[j] = emo_tld_u32(tab_o + (unsigned)j * tab_row + (lv[j] & lmask) * 4u, tok);
 #pragma unroll
             for (int j = R - 1; j >= 0; --j) {
-                const uint4 r0j = emo_tld_128(rec_a + 48u * j, tok);
-                const uint4 r1j = emo_tld_128(rec_a + 48u * j + 16u, tok);
+                const uint4 r0j = emo_tld_128(rec_o + 48u * j, tok);
+                const uint4 r1j = emo_tld_128(rec_o + 48u * j + 16u, tok);
                 unsigned qin = emo_floor_sub(q, r1j.w);
-                if (has_in) {
+                if (IN) {
                     const unsigned a = slot_lane + r0j.w;
                     qin = max(qin, emo_lds_u32v(a));
                     emo_sts_u32v(a, 0u);
                 }
-                finish(qin, d[j], r1j.z, r1j.x, r1j.y, xes_a + 8u * j);
-                q = qin + d[j];
-                if (has_out) emo_red_max_u32(slot_lane + r0j.y, emo_floor_sub(q, r0j.z));
-                if (r0j.x & emo::kB_Pop) {
-                    pop_a -= ptile4;
-                    c = emo_tld_u32(pop_a, tok);
+                if (EXTRA) {
+                    finish(qin, d[j], r1j.z, r1j.x, r1j.y, xes_o + 8u * j);
                 } else {
-                    c -= d[j];
+                    // slack_v = T - (lbQ_v + lbES_v) - (qin_v + co_v)
+                    const long long A = (long long)((unsigned long long)r1j.x | ((unsigned long long)r1j.y << 32));
+                    const long long sl = (T - A) - (long long)((unsigned long long)qin + (unsigned long long)c);
+                    emo_stg_s64_if(sl_lane, r1j.z, ldo8, sl, sl_ok);
                 }
+                q = qin + d[j];
+                if (OUT) emo_red_max_u32(slot_lane + r0j.y, emo_floor_sub(q, r0j.z));
+                const unsigned pops = r0j.x & emo::kB_Pop;
+                pop_a -= pops ? ptile4 : 0u;
+                c = emo_tld_u32_if(pop_a, tok, pops, c - d[j]);
+            }
+        };
+        auto run_kind = [&](auto rc, unsigned o) {
+            if (has_in) {
+                if (has_out) run(rc, std::true_type{}, std::true_type{}, o);
+                else run(rc, std::true_type{}, std::false_type{}, o);
+            } else {
+                if (has_out) run(rc, std::false_type{}, std::true_type{}, o);
+                else run(rc, std::false_type{}, std::false_type{}, o);
             }
         };
 
@@ -751,16 +787,18 @@ __global__ void __launch_bounds__(MAXT, 1) emo_flow_bwd(FlowParams p)
                 xes_a -= (unsigned)r * 8u;
                 has_in = (sg & emo::kSegIn) != 0;
                 has_out = (sg & emo::kSegOut) != 0;
-                switch (r) {
-                    case 1: run(std::integral_constant<int, 1>{}); break;
-                    case 2: run(std::integral_constant<int, 2>{}); break;
-                    case 3: run(std::integral_constant<int, 3>{}); break;
-                    case 4: run(std::integral_constant<int, 4>{}); break;
-                    case 5: run(std::integral_constant<int, 5>{}); break;
-                    case 6: run(std::integral_constant<int, 6>{}); break;
-                    case 7: run(std::integral_constant<int, 7>{}); break;
-                    case 8: run(std::integral_constant<int, 8>{}); break;
-                    default: break;
+                {
+                    // the run in pieces of 4, 2 and 1 entries, from its highest position down
+                    unsigned rem = (unsigned)r;
+                    while (rem >= 4u) {
+                        rem -= 4u;
+                        run_kind(std::integral_constant<int, 4>{}, rem);
+                    }
+                    if (rem >= 2u) {
+                        rem -= 2u;
+                        run_kind(std::integral_constant<int, 2>{}, rem);
+                    }
+                    if (rem) run_kind(std::integral_constant<int, 1>{}, 0u);
                 }
             }
             if (leave) break;

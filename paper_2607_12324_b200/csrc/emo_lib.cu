@@ -4,7 +4,6 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
-#include <cstdlib>
 #include <new>
 #include <string>
 #include <vector>
@@ -619,7 +618,6 @@ bool flow_plan(const emo_graph *g, int64_t B, bool want_base, bool need_bwd, Flo
             p.wait_cycles = g_wait_cycles;
             p.stall_stage = -1;
             p.prof = nullptr;
-            p.dbg = getenv("EMO_DBG") ? atoi(getenv("EMO_DBG")) : 0;
             smem = head + nbuf * stage;
             return true;
         };
