@@ -55,6 +55,7 @@ extern "C" {
 #define EMO_F_NO_STAGING 0x2u      /* use the plain-load kernels instead of the staged ones */
 #define EMO_F_PAIR_KERNEL 0x4u     /* staged pass kernel with two policies per thread (default only for very large batches) */
 #define EMO_F_LANE_KERNEL 0x8u     /* staged pass kernel with one policy per thread (the default otherwise) */
+#define EMO_F_FLOW_KERNEL 0x10u    /* the 32-bit lane-stream kernels (the default only for large batches: n * B >= 2^31) */
 #define EMO_F_TEST_STALL 0x100u    /* test hook of the 32-bit kernels: the producer warps stop half way, so that the
                                       consumers' bounded waits run out and EMO_E_TIMEOUT is reported */
 
@@ -119,6 +120,16 @@ int emo_graph_info(const emo_graph *g, emo_info *info);
  * device memory per invocation.
  */
 int emo_workspace_bytes(const emo_graph *g, int64_t B, int need_slack, size_t *out);
+
+/*
+ * emo_workspace_bytes_for - the same for a call that passes `flags` (EMO_F_* of the evaluation calls:
+ * they choose the kernels, and the kernels differ in what they keep between the two passes) and a
+ * level matrix that is (aligned = 1) or is not (aligned = 0) fetchable in 16-byte pieces: pointer
+ * 16-byte aligned and ldb a multiple of 16.  emo_workspace_bytes assumes no flags and an aligned
+ * matrix.  A workspace that is too small for what the call ends up running gives EMO_E_OOM.
+ */
+int emo_workspace_bytes_for(const emo_graph *g, int64_t B, int need_slack, uint32_t flags, int aligned,
+                            size_t *out);
 
 /*
  * emo_eval_policies - Alg. 1 without the idle-energy loop, for B policies at once:

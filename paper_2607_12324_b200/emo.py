@@ -23,13 +23,14 @@ EMO_F_VALIDATE = 0x1
 EMO_F_NO_STAGING = 0x2
 EMO_F_PAIR_KERNEL = 0x4
 EMO_F_LANE_KERNEL = 0x8
+EMO_F_FLOW_KERNEL = 0x10
 EMO_F_TEST_STALL = 0x100
 
 EXPORTS = [
     "emo_strerror", "emo_graph_load", "emo_graph_free", "emo_graph_info", "emo_workspace_bytes",
     "emo_eval_policies", "emo_slack_batch", "emo_slack", "emo_baseline", "emo_target_from_delta",
     "emo_select", "emo_transpose_policies", "emo_slack_batch_host", "emo_graph_program",
-    "emo_set_pass_events", "emo_select_static", "emo_graph_flow", "emo_set_wait_limit", "emo_call_path", "emo_set_flow_counters",
+    "emo_set_pass_events", "emo_select_static", "emo_graph_flow", "emo_set_wait_limit", "emo_call_path", "emo_set_flow_counters", "emo_workspace_bytes_for",
 ]
 
 
@@ -91,6 +92,7 @@ def lib():
         L.emo_graph_free.argtypes = [p]
         L.emo_graph_info.argtypes = [p, ctypes.POINTER(emo_info)]
         L.emo_workspace_bytes.argtypes = [p, i64, ctypes.c_int, ctypes.POINTER(sz)]
+        L.emo_workspace_bytes_for.argtypes = [p, i64, ctypes.c_int, u32, ctypes.c_int, ctypes.POINTER(sz)]
         L.emo_eval_policies.argtypes = [p, i64, p, i64, p, p, p, p, p, sz, p, u32, p]
         L.emo_slack_batch.argtypes = [p, i64, p, i64, p, p, p, i64, p, p, p, p, p, p, p, sz, p, u32, p]
         L.emo_slack.argtypes = [p, p, p, p, p, p, p, p, sz, p, p]
@@ -193,9 +195,11 @@ def emo_graph_info(g: Graph) -> emo_info:
     return info
 
 
-def emo_workspace_bytes(g: Graph, B: int, need_slack: int = 0) -> int:
+def emo_workspace_bytes(g: Graph, B: int, need_slack: int = 0, flags: int = 0, aligned: bool = True) -> int:
+    """Workspace a call on B policies needs; flags / aligned as in emo_workspace_bytes_for."""
     out = ctypes.c_size_t()
-    _check(lib().emo_workspace_bytes(g.handle, int(B), int(need_slack), ctypes.byref(out)), "emo_workspace_bytes")
+    _check(lib().emo_workspace_bytes_for(g.handle, int(B), int(need_slack), int(flags), int(bool(aligned)),
+                                         ctypes.byref(out)), "emo_workspace_bytes_for")
     return int(out.value)
 
 

@@ -49,7 +49,8 @@ def gpu_slack_batch(torch, emo, h, lv_dev, B, n, want=("ES", "LS", "slack"), fla
     ss = torch.full((max(B, 1),), -1, dtype=torch.int64, device=dev)
     nc = torch.full((max(B, 1),), -1, dtype=torch.int32, device=dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
-    ws = torch.empty(emo.emo_workspace_bytes(h, B, 1), dtype=torch.uint8, device=dev)
+    aligned = lv_dev.stride(0) % 16 == 0 and lv_dev.data_ptr() % 16 == 0
+    ws = torch.empty(emo.emo_workspace_bytes(h, B, 1, flags, aligned), dtype=torch.uint8, device=dev)
     T0 = torch.full((1,), -1, dtype=torch.int64, device=dev) if base else None
     E0 = torch.full((1,), -1.0, dtype=torch.float64, device=dev) if base else None
     emo.emo_slack_batch(h, B, lv_dev, lv_dev.stride(0), out["ES"], out["LS"], out["slack"], ldo, T, E,
@@ -109,17 +110,27 @@ def test_tiny_graphs_all_outputs(torch_cuda, emo, oracle_mod):
         lv = all_policies(g.n, g.L)
         B = lv.shape[1]
         r_or = oracle_mod.batch(g, lv, want_arrays=True)
-        ldb = B + 5
+        ldb = B + 5 if (B + 5) % 16 else B + 6      # a pitch that rules out 16-byte pieces
         lvp = np.full((g.n, ldb), 0xFF, dtype=np.uint8)
         lvp[:, :B] = lv
         lv_dev = torch.as_tensor(lvp, device="cuda")
+        # the same levels at a pitch of whole 16-byte pieces: what the staged kernels need
+        ldb16 = (B + 15) // 16 * 16 + 16
+        lvq = np.full((g.n, ldb16), 0xFF, dtype=np.uint8)
+        lvq[:, :B] = lv
+        lv16 = torch.as_tensor(lvq, device="cuda")
         for lanes in (0, 1, 2):
             h = emo.load_workload(g, emo.EMO_F_LANES(lanes))
-            for fl in (0, emo.EMO_F_PAIR_KERNEL, emo.EMO_F_LANE_KERNEL):
-                r = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, ldo=B + 3, flags=fl)
+            assert emo.emo_call_path(h, B, lv_dev, ldb, B + 3, True, 0) == 0, "an odd pitch takes the plain-load kernels"
+            assert emo.emo_call_path(h, B, lv16, ldb16, B + 3, True, emo.EMO_F_FLOW_KERNEL) == 2
+            for lvx, fl in ((lv_dev, 0), (lv16, emo.EMO_F_PAIR_KERNEL), (lv16, emo.EMO_F_LANE_KERNEL), (lv16, emo.EMO_F_FLOW_KERNEL)):
+                r = gpu_slack_batch(torch, emo, h, lvx, B, g.n, ldo=B + 3, flags=fl)
                 assert_matches(r, r_or, B)
                 for k in ("ES", "LS", "slack"):
                     assert (r[k][:, B:] == -7).all(), "padding columns of the outputs were written"
+            T, E, st = gpu_eval(torch, emo, h, lv16, B, emo.EMO_F_VALIDATE | emo.EMO_F_FLOW_KERNEL)
+            assert st == 0 and np.array_equal(T, r_or["makespan"])
+            np.testing.assert_allclose(E, r_or["energy"], rtol=E_RTOL)
             T, E, st = gpu_eval(torch, emo, h, lv_dev, B, emo.EMO_F_VALIDATE)
             assert st == 0 and np.array_equal(T, r_or["makespan"])
             np.testing.assert_allclose(E, r_or["energy"], rtol=E_RTOL)
@@ -161,19 +172,24 @@ def test_config_graphs_all_outputs(torch_cuda, emo, oracle_mod, name, scale, B):
     r2 = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, want=("slack",))
     assert np.array_equal(r2["slack"][:, :B], r_or["slack"])
     base = oracle_mod.batch(g, np.full((g.n, 1), g.L - 1, dtype=np.uint8))
-    # every pass kernel: plain loads, two policies per thread, one policy per thread
-    for fl in (emo.EMO_F_NO_STAGING, emo.EMO_F_PAIR_KERNEL, emo.EMO_F_LANE_KERNEL):
+    # every pass kernel: plain loads, two policies per thread, one policy per thread, 32-bit lane streams
+    assert emo.emo_call_path(h, B, lv_dev, lv_dev.stride(0), B, True, emo.EMO_F_FLOW_KERNEL) == 2
+    for fl in (emo.EMO_F_NO_STAGING, emo.EMO_F_PAIR_KERNEL, emo.EMO_F_LANE_KERNEL, emo.EMO_F_FLOW_KERNEL):
         r3 = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, flags=fl, base=True)
         assert_matches(r3, r_or, B)
         assert r3["T0"] == base["makespan"][0]
         assert r3["E0"] == pytest.approx(base["energy"][0], rel=E_RTOL)
     # without the per-policy sums (the configuration the bench times)
-    r5 = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, want=("slack",), sums=False, base=True)
-    assert np.array_equal(r5["slack"][:, :B], r_or["slack"]) and r5["T0"] == base["makespan"][0]
-    assert (r5["slack_sum"] == -1).all()
+    for fl in (0, emo.EMO_F_FLOW_KERNEL):
+        r5 = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, want=("slack",), sums=False, base=True, flags=fl)
+        assert np.array_equal(r5["slack"][:, :B], r_or["slack"]) and r5["T0"] == base["makespan"][0]
+        assert (r5["slack_sum"] == -1).all()
+    T, E, st = gpu_eval(torch, emo, h, lv_dev, B, emo.EMO_F_FLOW_KERNEL)
+    assert st == 0 and np.array_equal(T, r_or["makespan"])
+    np.testing.assert_allclose(E, r_or["energy"], rtol=E_RTOL)
     # an output pitch that is odd (no 16-byte stores of policy pairs possible) and one that is even
     for ldo in (B + 1, B + 2):
-        for fl in (emo.EMO_F_PAIR_KERNEL, emo.EMO_F_LANE_KERNEL):
+        for fl in (emo.EMO_F_PAIR_KERNEL, emo.EMO_F_LANE_KERNEL, emo.EMO_F_FLOW_KERNEL):
             r4 = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, ldo=ldo, flags=fl)
             assert_matches(r4, r_or, B)
     # single-policy call
@@ -271,10 +287,19 @@ def test_cfg4_full_size_sampled(torch_cuda, emo, oracle_mod, golden):
     E0 = torch.zeros(1, dtype=torch.float64, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     ws = torch.empty(emo.emo_workspace_bytes(h, B, 1), dtype=torch.uint8, device="cuda")
+    assert emo.emo_call_path(h, B, lv_dev, lv_dev.stride(0), B, True, 0) == 2, "the largest workload takes the 32-bit kernels"
     emo.emo_slack_batch(h, B, lv_dev, lv_dev.stride(0), None, None, slack, B, T, E, None, None, ws, status, T0=T0, E0=E0)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     assert np.array_equal(T.cpu().numpy(), r["makespan"])
+    # a contiguous slab of 256 policies, element by element: the last two policy tiles (the last one shares
+    # its launch with the block of the baseline column)
+    slab0 = B - 256
+    slab = lv_dev[:, slab0:B].contiguous().cpu().numpy()
+    r_slab = oracle_mod.batch(g, slab, want_arrays=True, threads=os.cpu_count() or 1)
+    assert np.array_equal(slack[:, slab0:B].cpu().numpy(), r_slab["slack"])
+    assert np.array_equal(T.cpu().numpy()[slab0:B], r_slab["makespan"])
+    del r_slab, slab
     assert np.array_equal(slack[:, torch.as_tensor(cols, device="cuda")].cpu().numpy(), r_sub["slack"])
     assert np.array_equal(slack.sum(dim=0).cpu().numpy(), r["slack_sum"])
     assert np.array_equal((slack == 0).sum(dim=0).cpu().numpy(), r["n_critical"])
@@ -370,7 +395,7 @@ def test_many_levels(torch_cuda, emo, oracle_mod):
     lvp[:, :B] = lv
     lv_dev = torch.as_tensor(lvp, device="cuda")
     h = emo.load_workload(g)
-    for fl in (emo.EMO_F_NO_STAGING, emo.EMO_F_PAIR_KERNEL, emo.EMO_F_LANE_KERNEL, 0):
+    for fl in (emo.EMO_F_NO_STAGING, emo.EMO_F_PAIR_KERNEL, emo.EMO_F_LANE_KERNEL, emo.EMO_F_FLOW_KERNEL, 0):
         r = gpu_slack_batch(torch, emo, h, lv_dev, B, n, flags=fl, base=True)
         assert_matches(r, r_or, B)
     h.free()
@@ -386,8 +411,11 @@ def test_group_of_on_gpu(torch_cuda, emo, oracle_mod):
     lv = np.random.RandomState(3).randint(0, g.L, (rows, B)).astype(np.uint8)
     r_or = oracle_mod.batch(g, lv, want_arrays=True, group_of=group)
     h = emo.load_workload(g, group_of=group)
-    r = gpu_slack_batch(torch, emo, h, torch.as_tensor(lv, device="cuda"), B, g.n)
-    assert_matches(r, r_or, B)
+    lvp = np.zeros((rows, 80), dtype=np.uint8)
+    lvp[:, :B] = lv
+    for fl in (0, emo.EMO_F_FLOW_KERNEL):
+        r = gpu_slack_batch(torch, emo, h, torch.as_tensor(lvp, device="cuda"), B, g.n, flags=fl)
+        assert_matches(r, r_or, B)
     h.free()
 
 
@@ -420,4 +448,106 @@ def test_host_buffer_call(torch_cuda, emo, oracle_mod):
     want = oracle_mod.select(r_or["makespan"], r_or["energy"], oracle_mod.target_from_delta(T0, ppm))
     assert int(sel[0]) == want and int(sel[1]) == r_or["makespan"][want]
     assert np.array([int(sel[2])], dtype=np.int64).view(np.float64)[0] == pytest.approx(r_or["energy"][want], rel=E_RTOL)
+    h.free()
+
+
+def test_many_groups_per_block(torch_cuda, emo, oracle_mod):
+    """A batch large enough for several policy groups per block (more than 2 x 32 x the SM count policies)
+    with a ragged last tile: ES, LS and slack of every policy, every staged kernel family."""
+    torch = torch_cuda
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    g = W.make_graph("cfg1-train", 0.05)
+    B = 2 * 32 * sms + 77
+    lv_dev = W.policies_for(g, B=B, device="cuda")
+    r_or = oracle_mod.batch(g, lv_dev.cpu().numpy(), B=B, want_arrays=True, threads=os.cpu_count() or 1)
+    h = emo.load_workload(g)
+    for fl in (emo.EMO_F_FLOW_KERNEL, emo.EMO_F_LANE_KERNEL, emo.EMO_F_PAIR_KERNEL):
+        r = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, flags=fl, base=True)
+        assert_matches(r, r_or, B)
+    h.free()
+
+
+def _spread_graph(total_spread: int, n: int = 40):
+    """A two-stream graph with cross edges whose completion times spread by about total_spread ns over
+    the policies (level 0 is fast, level 1 slow), with rows that are not monotone and zero durations."""
+    rs = np.random.RandomState(7)
+    per = total_spread // n
+    edges = [(i, i + 2) for i in range(n - 2)] + [(i, i + 1) for i in range(0, n - 1, 5)] + [(i, i + 3) for i in range(1, n - 3, 7)]
+    lat = np.zeros((n, 3), dtype=np.int64)
+    lat[:, 0] = rs.randint(0, 1000, n)
+    lat[:, 1] = lat[:, 0] + 2 * per + rs.randint(0, 1000, n)
+    lat[:, 2] = rs.randint(0, 500, n)          # faster than level 0 for some nodes: rows are not monotone
+    lat[::9] = 0
+    en = rs.rand(n, 3)
+    return W.tiny_graph(n, edges, lat, en, name="spread")
+
+
+def test_offset_guard_and_fallback(torch_cuda, emo, oracle_mod):
+    """The 32-bit kernels carry times as offsets from static bounds.  A graph whose spread of start times
+    stays below 2^32 ns runs on them (non-monotone rows and zero durations included); one whose spread is
+    larger must fall back to the 64-bit kernels; both give the oracle's results."""
+    torch = torch_cuda
+    B = 96
+    for total, want32 in ((3_000_000_000, True), (9_000_000_000, False)):
+        g = _spread_graph(total)
+        lv = np.random.RandomState(1).randint(0, 3, (g.n, B)).astype(np.uint8)
+        lv[:, 0] = 1                       # the slowest policy: the largest offsets
+        lv[:, 1] = 0
+        r_or = oracle_mod.batch(g, lv, want_arrays=True)
+        assert (int(r_or["makespan"].max()) - int(r_or["makespan"].min()) > (1 << 32)) == (not want32)
+        lv_dev = torch.as_tensor(lv, device="cuda")
+        h = emo.load_workload(g)
+        path = emo.emo_call_path(h, B, lv_dev, B, B, True, emo.EMO_F_FLOW_KERNEL)
+        assert (path == 2) == want32, "the guard decides whether the 32-bit kernels run"
+        r = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, flags=emo.EMO_F_FLOW_KERNEL, base=True)
+        assert_matches(r, r_or, B)
+        h.free()
+    # exactly at the guard: a chain whose completion times spread by 2^32 - 1 ns (fits) and by 2^32 (does not)
+    for spread, want32 in ((0xFFFFFFFF, True), (0x100000000, False)):
+        a = spread // 2
+        lat = np.array([[1, 1 + a], [1, 1 + (spread - a)]], dtype=np.int64)
+        g = W.tiny_graph(2, [(0, 1)], lat, name="edge")
+        lv = np.zeros((2, 16), dtype=np.uint8)
+        lv[:, 1] = 1
+        lv[0, 2] = 1
+        lv[1, 3] = 1
+        r_or = oracle_mod.batch(g, lv, want_arrays=True)
+        lv_dev = torch.as_tensor(lv, device="cuda")
+        h = emo.load_workload(g)
+        assert (emo.emo_call_path(h, 16, lv_dev, 16, 16, True, emo.EMO_F_FLOW_KERNEL) == 2) == want32
+        r = gpu_slack_batch(torch, emo, h, lv_dev, 16, 2, flags=emo.EMO_F_FLOW_KERNEL)
+        assert_matches(r, r_or, 16)
+        h.free()
+
+
+def test_bounded_waits_report_timeout(torch_cuda, emo, oracle_mod):
+    """Every device-side wait of the 32-bit kernels is bounded.  With the test hook the producer warps stop
+    half way (no copy is issued, nothing is read out of bounds, nothing spins for ever): the consumers' waits
+    run out after the (shortened) limit, EMO_E_TIMEOUT goes to the status word, the kernels return, and the
+    next ordinary call gives the oracle's results."""
+    torch = torch_cuda
+    g = W.make_graph("cfg1-train", 0.05)
+    B = 200
+    lv_dev = W.policies_for(g, B=B, device="cuda")
+    r_or = oracle_mod.batch(g, lv_dev.cpu().numpy(), B=B, want_arrays=True)
+    h = emo.load_workload(g)
+    emo.emo_set_wait_limit(4_000_000)          # about 2 ms
+    try:
+        slack = torch.zeros((g.n, B), dtype=torch.int64, device="cuda")
+        T = torch.zeros(B, dtype=torch.int64, device="cuda")
+        E = torch.zeros(B, dtype=torch.float64, device="cuda")
+        fl = emo.EMO_F_FLOW_KERNEL | emo.EMO_F_TEST_STALL
+        ws = torch.empty(emo.emo_workspace_bytes(h, B, 1, fl), dtype=torch.uint8, device="cuda")
+        for call in ("eval", "slack"):
+            status = torch.zeros(1, dtype=torch.int32, device="cuda")
+            if call == "eval":
+                emo.emo_eval_policies(h, B, lv_dev, lv_dev.stride(0), T, E, ws, status, fl)
+            else:
+                emo.emo_slack_batch(h, B, lv_dev, lv_dev.stride(0), None, None, slack, B, T, E, None, None, ws, status, fl)
+            torch.cuda.synchronize()
+            assert int(status.item()) == emo.EMO_E_TIMEOUT
+    finally:
+        emo.emo_set_wait_limit(4_000_000_000)
+    r = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, flags=emo.EMO_F_FLOW_KERNEL, base=True)
+    assert_matches(r, r_or, B)
     h.free()

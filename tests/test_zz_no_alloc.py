@@ -32,6 +32,7 @@ def _select_both(torch, emo, T, E, target):
 
 def test_static_selection_matches_workspace_selection():
     import torch
+    import oracle
     from paper_2607_12324_b200 import build, emo
     assert torch.cuda.is_available()
     torch.cuda.set_device(0)
@@ -45,6 +46,10 @@ def test_static_selection_matches_workspace_selection():
             ref, got = _select_both(torch, emo, T, E, target)
             assert got[0] == ref[0] and got[1] == ref[1]
             assert got[2] == ref[2]                          # same reduction, same bits
+            want = oracle.select(T, E, target)               # and directly against the CPU oracle
+            assert got[0] == want
+            if want >= 0:
+                assert got[1] == T[want] and got[2] == E[want]
     # target read on the device, as after a baseline evaluation
     T = rs.randint(1000, 2000, 5000).astype(np.int64)
     E = rs.rand(5000)
@@ -57,7 +62,7 @@ def test_static_selection_matches_workspace_selection():
     emo.emo_select(5000, Td, Ed, 0, a, None, None, ws, target_dev=T0, delta_ppm=50_000)
     emo.emo_select_static(5000, Td, Ed, 0, b, target_dev=T0, delta_ppm=50_000)
     torch.cuda.synchronize()
-    assert int(a.item()) == int(b.item()) >= 0
+    assert int(a.item()) == int(b.item()) == oracle.select(T, E, oracle.target_from_delta(1500, 50_000)) >= 0
     # beyond the stated maximum: refused, nothing launched
     with pytest.raises(emo.EmoError) as ei:
         emo.emo_select_static(emo.EMO_SELECT_STATIC_MAX_B + 1, Td, Ed, 0, b)
