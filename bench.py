@@ -100,12 +100,22 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def oracle_sample(g, lv_cols, threads, want_slack=True):
+def oracle_sample(g, lv_cols, threads, want_slack=True, keep=None):
     """Times the CPU oracle as it stands on the given policy columns; returns seconds."""
     import oracle
     t0 = time.perf_counter()
-    oracle.batch(g, lv_cols, want_slack=want_slack, threads=threads)
-    return time.perf_counter() - t0
+    r = oracle.batch(g, lv_cols, want_slack=want_slack, threads=threads)
+    dt = time.perf_counter() - t0
+    if keep is not None:
+        keep.update(r)
+    return dt
+
+
+def workload_config(name, scale, g, B, ppm):
+    """What both arms print as `config` (the same keys and values in both)."""
+    return {"workload": name if scale == 1.0 else f"{name} x{scale}", "n": int(g.n), "m": int(g.m), "L": int(g.L),
+            "policies": int(B), "passes": "forward+backward", "slack_materialised": True, "delta_ppm": int(ppm),
+            "l2": "inputs larger than L2 (levels %.1f GB, slack %.1f GB per step)" % (g.n * B / 1e9, g.n * B * 8 / 1e9)}
 
 
 def run_reference(args, rank, world):
@@ -114,8 +124,9 @@ def run_reference(args, rank, world):
         return
     import numpy as np
     from paper_2607_12324_b200 import workloads as W
-    g = W.make_graph(args.workload)
-    B = g.meta["B"]
+    g = W.make_graph(args.workload, args.scale)
+    B = args.policies or g.meta["B"]
+    ppm = (g.meta["delta_ppm"] or [50_000])[-1]
     threads = os.cpu_count() or 1
     per_step = max(threads, 2 * threads)
     total = per_step * (args.steps + args.warmup)
@@ -136,8 +147,7 @@ def run_reference(args, rank, world):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic",
-            "config": {"workload": args.workload, "n": g.n, "m": g.m, "L": g.L, "policies": B,
-                       "passes": "forward+backward"},
+            "config": workload_config(args.workload, args.scale, g, B, ppm),
             "policies_per_s": per_step * args.steps / t,
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
                              "sample": f"{per_step} of {B} policies per step, forward+backward with slack sums"},
@@ -186,8 +196,11 @@ def main():
     ppm = (g.meta["delta_ppm"] or [50_000])[-1]
     lv = W.policies_for(g, B=B, device="cuda")
     ldb = lv.stride(0)
+    t_load = time.perf_counter()
     h = emo.load_workload(g, flags=args.flags)
+    t_load = time.perf_counter() - t_load
     info = h.info
+    fl = emo.emo_graph_flow(h, arrays=False)
     n, m = g.n, g.m
     slack = torch.empty((n, B), dtype=torch.int64, device="cuda")
     T = torch.zeros(B, dtype=torch.int64, device="cuda")
@@ -199,7 +212,7 @@ def main():
     sel = torch.zeros(2, dtype=torch.int64, device="cuda")
     selE = torch.zeros(1, dtype=torch.float64, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    ws = torch.empty(emo.emo_workspace_bytes(h, B, 2), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(emo.emo_workspace_bytes(h, B, 2, args.call_flags), dtype=torch.uint8, device="cuda")
 
     def step(events=None):
         if events is not None:
@@ -265,27 +278,47 @@ def main():
     roofline_step = {"bound": "hbm", "algorithmic_bytes": step_bytes, "achieved": step_bytes / (ms_per_step * 1e-3) / 1e9,
                      "peak": peak, "unit": "GB/s", "frac": step_bytes / (ms_per_step * 1e-3) / 1e9 / peak}
 
+    # the three bounds of the step: HBM (algorithmic bytes at the measured copy rate), integer issue (one add per
+    # node and one max per edge, per pass and policy, at the measured issue rate of 32-bit adds and maxima) and
+    # the depth floor (the graph's hop levels times a dependent step of about 30 cycles; not a roofline, it
+    # explains low fractions on shallow batches)
+    scratch = torch.zeros(16, dtype=torch.int64, device="cuda")
+    ipk = emo.emo_measure_int_issue(scratch)
+    t_hbm = step_bytes / (peak * 1e9) * 1e3
+    t_issue = passes * B / 32.0 * (n / ipk["add32"] + m / ipk["max32"]) * 1e3
+    sm_mhz = (clocks or {}).get("sm_mhz") or 1965.0
+    t_depth = passes * info.depth * 30.0 / (sm_mhz * 1e6) * 1e3
+    bounds = {"t_hbm_ms": t_hbm, "t_issue_ms": t_issue, "depth_floor_ms": t_depth,
+              "binding": "hbm" if t_hbm >= t_issue else "int_issue",
+              "int_issue_peak_warp_ops_per_s": ipk,
+              "frac_of_binding": max(t_hbm, t_issue) / ms_per_step}
+    path = emo.emo_call_path(h, B, lv, ldb, B, True, args.call_flags)
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "int64", "data": "synthetic",
-            "config": {"workload": args.workload if args.scale == 1.0 else f"{args.workload} x{args.scale}", "n": n, "m": m, "L": g.L, "policies": B, "passes": "forward+backward",
-                       "slack_materialised": True, "slack_sums": bool(args.sums), "delta_ppm": ppm, "lanes": info.lanes, "steps_fwd": info.steps_fwd,
-                       "slots_fwd": info.slots_fwd, "slots_bwd": info.slots_bwd,
-                       "l2": "inputs larger than L2 (levels %.1f GB, slack %.1f GB per step)" % (n * ldb / 1e9, n * B * 8 / 1e9),
-                       "kernels": {2: "32-bit lane-stream", 1: "staged 64-bit", 0: "plain 64-bit"}[
-                           emo.emo_call_path(h, B, lv, ldb, B, True, args.call_flags)],
-                       "parallelism": "replicas" if world > 1 else "single"},
+            "config": workload_config(args.workload, args.scale, g, B, ppm),
+            "details": {"kernels": {2: "32-bit lane-stream", 1: "staged 64-bit", 0: "plain 64-bit"}[path],
+                        "slack_sums": bool(args.sums), "lanes": fl["lanes"] if path == 2 else info.lanes,
+                        "steps": fl["steps"] if path == 2 else info.steps_fwd, "stage_steps": fl["K"], "barrier_steps": fl["sync"],
+                        "restore_rows": fl["pushes"], "depth": info.depth, "graph_load_s": t_load,
+                        "workspace_gb": ws.numel() / 1e9,
+                        "parallelism": "replicas" if world > 1 else "single"},
             "policies_per_s": world * B / (ms_per_step * 1e-3),
             "gpu_launches": launches_per_step * args.steps,
-            "roofline": roofline, "roofline_step": roofline_step, "clocks": clocks,
+            "roofline": roofline, "roofline_step": roofline_step, "bounds": bounds, "clocks": clocks,
             "selected": {"index": int(sel[0].item()), "T": int(sel[1].item()), "E": float(selE.item()),
                          "T0": int(T0.item()), "E0": float(E0.item())}}
 
-    # end to end through the host-buffer entry point: levels from pinned host memory every step,
-    # per-policy results and the selection back to the host; the slack matrix stays on the device
+    # end to end through the host-buffer entry point: the levels come from pinned host memory every step, packed
+    # at ceil(log2 L) bits each (the call spreads them to bytes on the device), per-policy results and the
+    # selection go back to the host; the slack matrix stays on the device
     if not args.no_e2e:
-        lv_host = torch.empty((g.n, ldb), dtype=torch.uint8).pin_memory()
-        lv_host.copy_(lv)
+        bits = max(1, int(np.ceil(np.log2(max(g.L, 2)))))
+        ldp = ((B + 7) // 8 * bits + 15) // 16 * 16
+        dev_packed = torch.empty((g.n, ldp), dtype=torch.uint8, device="cuda")
+        emo.emo_pack_levels(bits, g.n, B, lv, ldb, dev_packed, ldp)
+        lv_host = torch.empty((g.n, ldp), dtype=torch.uint8).pin_memory()
+        lv_host.copy_(dev_packed)
         hT = torch.zeros(B, dtype=torch.int64).pin_memory()
         hE = torch.zeros(B, dtype=torch.float64).pin_memory()
         hss = torch.zeros(B, dtype=torch.int64).pin_memory()
@@ -293,14 +326,18 @@ def main():
         hsel = torch.zeros(4, dtype=torch.int64)
         dev_lvl = torch.empty_like(lv)
         hsums = (hss, hnc) if args.sums else (None, None)
-        emo.emo_slack_batch_host(h, B, lv_host, ldb, dev_lvl, slack, B, ppm, hT, hE, hsums[0], hsums[1], hsel, ws)
+
+        def e2e_step():
+            emo.emo_slack_batch_host_packed(h, B, bits, lv_host, ldp, dev_packed, dev_lvl, ldb, slack, B, ppm, hT, hE,
+                                            hsums[0], hsums[1], hsel, ws, flags=args.call_flags)
+        e2e_step()
         torch.cuda.synchronize()
         k = max(1, min(args.steps, 5))
         if dist is not None:
             dist.barrier()
         t0 = time.perf_counter()
         for _ in range(k):
-            emo.emo_slack_batch_host(h, B, lv_host, ldb, dev_lvl, slack, B, ppm, hT, hE, hsums[0], hsums[1], hsel, ws)
+            e2e_step()
         torch.cuda.synchronize()
         e2e_s = (time.perf_counter() - t0) / k
         if dist is not None:
@@ -308,10 +345,11 @@ def main():
             dist.all_reduce(tt, op=dist.ReduceOp.MAX)
             e2e_s = float(tt.item())
         assert int(hsel[0]) == int(sel[0].item())
+        assert torch.equal(hT, T.cpu()), "the host-buffer call and the device call disagree"
         line["e2e"] = {"value": world * B * m * passes / e2e_s, "unit": UNIT, "ms_per_step": e2e_s * 1e3,
-                       "h2d_bytes_per_step": int(g.n * ldb), "d2h_bytes_per_step": int(B * (28 if args.sums else 16) + 80),
-                       "note": "slack matrix stays on the device"}
-        del lv_host
+                       "h2d_bytes_per_step": int(g.n * ldp), "d2h_bytes_per_step": int(B * (28 if args.sums else 16) + 80),
+                       "note": f"levels cross the bus packed at {bits} bits each; the slack matrix stays on the device"}
+        del lv_host, dev_packed, dev_lvl
 
     if rank == 0 and not args.no_cpu:
         threads = os.cpu_count() or 1
@@ -323,11 +361,28 @@ def main():
         t1 = oracle_sample(g, sub, threads)
         cnt2 = int(min(B, max(threads, (15.0 / max(t1, 1e-3)) * cnt)))
         cols = np.linspace(0, B - 1, cnt2).astype(np.int64)
-        sub = lv[:, torch.as_tensor(cols, device="cuda")].contiguous().cpu().numpy()
-        t2 = oracle_sample(g, sub, threads)
+        cols_dev = torch.as_tensor(cols, device="cuda")
+        sub = lv[:, cols_dev].contiguous().cpu().numpy()
+        ref = {}
+        t2 = oracle_sample(g, sub, threads, keep=ref)
         line["cpu_baseline"] = {"value": cnt2 * m * passes / t2, "unit": UNIT, "cores": threads, "kind": "oracle",
                                 "sample": f"{cnt2} of {B} policies, forward+backward with slack sums, {t2:.1f} s",
                                 "policies_per_s": cnt2 / t2}
+        # the outputs of the last timed step against what the oracle just computed for the same policies:
+        # makespan and slack sums (column sums of the materialised slack matrix) exact, energy to 1e-9
+        Tg = T[cols_dev].cpu().numpy()
+        Eg = E[cols_dev].cpu().numpy()
+        bad = int((Tg != ref["makespan"]).sum()) + int((np.abs(Eg - ref["energy"]) > 1e-9 * np.abs(ref["energy"])).sum())
+        nsum = min(cnt2, 512)
+        ssg = slack[:, cols_dev[:nsum]].sum(dim=0).cpu().numpy()
+        ncg = (slack[:, cols_dev[:nsum]] == 0).sum(dim=0).cpu().numpy()
+        bad += int((ssg != ref["slack_sum"][:nsum]).sum()) + int((ncg != ref["n_critical"][:nsum]).sum())
+        import oracle
+        base = oracle.batch(g, np.full((g.n, 1), g.L - 1, dtype=np.uint8))
+        bad += int(int(T0.item()) != int(base["makespan"][0]))
+        line["checked"] = {"policies_makespan_energy": cnt2, "policies_slack_sum_and_critical_count": nsum,
+                           "baseline_makespan": True, "mismatches": bad}
+        assert bad == 0, f"{bad} outputs of the timed step differ from the oracle"
     if rank == 0:
         print(json.dumps(line), flush=True)
     h.free()

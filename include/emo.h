@@ -246,6 +246,32 @@ int emo_slack_batch_host(const emo_graph *g, int64_t B, const uint8_t *lvl_host,
                          void *ws, size_t ws_bytes, uint32_t flags, void *stream);
 
 /*
+ * Levels packed at `bits` bits each (1..8; a level needs ceil(log2 L) bits): a layout for moving
+ * policies over the bus.  In a packed row, eight consecutive levels take `bits` consecutive bytes, the
+ * first level in the lowest bits; a row of B levels takes ceil(B / 8) * bits bytes (pitch ldp).
+ * emo_pack_levels: device byte matrix lvl [rows][ldb] -> device packed [rows][ldp];
+ * emo_unpack_levels the other way (levels beyond B up to the next multiple of 8 are written too).
+ * ldb a multiple of 8, lvl 8-byte aligned.  Layout helpers: no counterpart in the method.
+ */
+int emo_pack_levels(int bits, int64_t rows, int64_t B, const uint8_t *lvl, int64_t ldb,
+                    uint8_t *packed, int64_t ldp, void *stream);
+int emo_unpack_levels(int bits, int64_t rows, int64_t B, const uint8_t *packed, int64_t ldp,
+                      uint8_t *lvl, int64_t ldb, void *stream);
+
+/*
+ * emo_slack_batch_host_packed - emo_slack_batch_host with the levels in host memory packed at `bits`
+ * bits each (see emo_pack_levels; bits = 8: plain bytes, ld_host must equal ldb and dev_packed is not
+ * used): lvl_host is host [rows][ld_host], dev_packed a device buffer of rows * ld_host bytes, dev_lvl
+ * the device byte matrix [rows][ldb] the levels are spread into before the passes run.  With 5 bits
+ * (32 levels) 0.625 bytes per level cross the bus instead of 1.  Everything else as emo_slack_batch_host.
+ */
+int emo_slack_batch_host_packed(const emo_graph *g, int64_t B, int bits, const uint8_t *lvl_host, int64_t ld_host,
+                                uint8_t *dev_packed, uint8_t *dev_lvl, int64_t ldb, int64_t *slack_dev, int64_t ldo,
+                                int64_t delta_ppm, int64_t *makespan_host, double *energy_host,
+                                int64_t *slack_sum_host, int32_t *n_critical_host, int64_t *sel_host,
+                                void *ws, size_t ws_bytes, uint32_t flags, void *stream);
+
+/*
  * emo_set_pass_events - measurement hook (no counterpart in the method): four cudaEvent_t handles
  * (as void*, any may be NULL) that later emo_slack_batch / emo_eval_policies / emo_baseline calls
  * record on their stream immediately before and after the forward pass kernel and before and after
@@ -261,6 +287,15 @@ int emo_set_pass_events(void *fwd_start, void *fwd_stop, void *bwd_start, void *
  */
 int emo_call_path(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t ldb, int64_t ldo,
                   int need_slack, uint32_t flags);
+
+/*
+ * emo_measure_int_issue - measurement helper (no counterpart in the method): the rate at which this GPU
+ * issues the integer operations of the recurrences (Eq. 1 is one add per node and one max per edge).
+ * Runs four small kernels of independent dependent-chains that fill every SM and writes warp-level
+ * operations per second to ops_per_s[4] (host): 32-bit add, 32-bit max, 64-bit add, 64-bit max.
+ * scratch_dev: device memory of at least 8 bytes.  Synchronises the stream.
+ */
+int emo_measure_int_issue(double *ops_per_s, void *scratch_dev, void *stream);
 
 /*
  * emo_set_flow_counters - measurement hook (no counterpart in the method): a device array of 131072

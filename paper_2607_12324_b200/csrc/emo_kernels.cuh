@@ -271,3 +271,80 @@ __global__ void emo_transpose_u8(int64_t B, int64_t rows, const uint8_t *src, in
         __syncthreads();
     }
 }
+
+// ------------------------------------------------------------------------------------------------
+// Integer issue rate: eight independent dependent-chains per thread of one operation (OP 0: 32-bit
+// add, 1: 32-bit max, 2: 64-bit add, 3: 64-bit max), enough warps to fill every SM.  The operations
+// are volatile so that the compiler keeps every one of them.  Gives the denominator for "integer
+// issue against peak": the forward and backward recurrences are one add per node and one max per edge.
+// ------------------------------------------------------------------------------------------------
+template <int OP>
+__global__ void __launch_bounds__(256) emo_int_chains(unsigned long long *sink, int iters, unsigned seed)
+{
+    const unsigned tid = blockIdx.x * blockDim.x + threadIdx.x;
+    if (OP < 2) {
+        unsigned a[8], b = seed | 1u;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) a[k] = tid * 8u + (unsigned)k;
+        for (int i = 0; i < iters; ++i) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    if (OP == 0) asm volatile("add.u32 %0, %0, %1;" : "+r"(a[k]) : "r"(b));
+                    else asm volatile("max.u32 %0, %0, %1;" : "+r"(a[k]) : "r"(b + (unsigned)i));
+                }
+        }
+        unsigned x = 0;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) x ^= a[k];
+        if (x == 0x12345u) sink[0] = x;      // keeps the chains alive, (almost) never true
+    } else {
+        unsigned long long a[8], b = ((unsigned long long)seed << 13) | 1ull;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) a[k] = (unsigned long long)tid * 8ull + (unsigned long long)k;
+        for (int i = 0; i < iters; ++i) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    if (OP == 2) asm volatile("add.u64 %0, %0, %1;" : "+l"(a[k]) : "l"(b));
+                    else asm volatile("max.s64 %0, %0, %1;" : "+l"(a[k]) : "l"(b + (unsigned long long)i));
+                }
+        }
+        unsigned long long x = 0;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) x ^= a[k];
+        if (x == 0x12345ull) sink[0] = x;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Levels packed at `bits` bits each (a frequency level needs ceil(log2 L) bits): eight levels of a row
+// take `bits` consecutive bytes, lowest level in the lowest bits.  One thread converts one group of
+// eight; rows of the byte matrix are 8-byte aligned.  PACK: bytes -> bits, else bits -> bytes.
+// ------------------------------------------------------------------------------------------------
+template <bool PACK>
+__global__ void emo_repack_levels(int bits, int64_t rows, int64_t groups, uint8_t *packed, int64_t ldp, uint8_t *bytes, int64_t ldb)
+{
+    const unsigned long long mask = (1ull << bits) - 1ull;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < rows * groups; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = i / groups, c = i - r * groups;
+        uint8_t *pk = packed + r * ldp + c * bits;
+        unsigned long long *by = reinterpret_cast<unsigned long long *>(bytes + r * ldb + c * 8);
+        if (PACK) {
+            const unsigned long long v = *by;
+            unsigned long long w = 0;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) w |= ((v >> (8 * k)) & mask) << (k * bits);
+            for (int k = 0; k < bits; ++k) pk[k] = (uint8_t)(w >> (8 * k));
+        } else {
+            unsigned long long w = 0;
+            for (int k = 0; k < bits; ++k) w |= (unsigned long long)pk[k] << (8 * k);
+            unsigned long long v = 0;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) v |= ((w >> (k * bits)) & mask) << (8 * k);
+            *by = v;
+        }
+    }
+}

@@ -778,6 +778,41 @@ int emo_call_path(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t ldb
     return pl.staged ? 1 : 0;
 }
 
+int emo_measure_int_issue(double *ops_per_s, void *scratch_dev, void *stream)
+{
+    if (!ops_per_s || !scratch_dev) return EMO_E_INVALID_ARG;
+    int dev = 0, sms = 0;
+    EMO_CUDA(cudaGetDevice(&dev));
+    EMO_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaEvent_t e0, e1;
+    EMO_CUDA(cudaEventCreate(&e0));
+    EMO_CUDA(cudaEventCreate(&e1));
+    const int grid = sms * 8, iters = 2048;                    // 64 warps per SM, 8 chains x 4 x iters operations per thread
+    unsigned long long *sink = (unsigned long long *)scratch_dev;
+    int rc = EMO_OK;
+    for (int op = 0; op < 4 && rc == EMO_OK; ++op) {
+        float best = 0.f;
+        for (int rep = 0; rep < 4; ++rep) {                    // the first repetition warms up
+            cudaEventRecord(e0, st);
+            if (op == 0) emo_int_chains<0><<<grid, 256, 0, st>>>(sink, iters, 12345u);
+            else if (op == 1) emo_int_chains<1><<<grid, 256, 0, st>>>(sink, iters, 12345u);
+            else if (op == 2) emo_int_chains<2><<<grid, 256, 0, st>>>(sink, iters, 12345u);
+            else emo_int_chains<3><<<grid, 256, 0, st>>>(sink, iters, 12345u);
+            cudaEventRecord(e1, st);
+            if (cudaEventSynchronize(e1) != cudaSuccess || cudaGetLastError() != cudaSuccess) { rc = EMO_E_CUDA; break; }
+            float ms = 0.f;
+            cudaEventElapsedTime(&ms, e0, e1);
+            if (rep > 0 && (best == 0.f || ms < best)) best = ms;
+        }
+        const double warp_ops = (double)grid * 8.0 /* warps per block */ * 8.0 * 4.0 * iters;
+        ops_per_s[op] = best > 0.f ? warp_ops / (best * 1e-3) : 0.0;
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    return rc;
+}
+
 int emo_set_flow_counters(void *dev)
 {
     g_flow_prof = (long long *)dev;
@@ -1263,14 +1298,41 @@ int emo_transpose_policies(int64_t B, int64_t rows, const uint8_t *src, int64_t 
     return EMO_OK;
 }
 
-int emo_slack_batch_host(const emo_graph *g, int64_t B, const uint8_t *lvl_host, int64_t ldb,
-                         uint8_t *dev_lvl, int64_t *slack_dev, int64_t ldo, int64_t delta_ppm,
-                         int64_t *makespan_host, double *energy_host, int64_t *slack_sum_host,
-                         int32_t *n_critical_host, int64_t *sel_host, void *ws, size_t ws_bytes,
-                         uint32_t flags, void *stream)
+namespace {
+int repack(bool pack, int bits, int64_t rows, int64_t B, uint8_t *packed, int64_t ldp, uint8_t *bytes, int64_t ldb, cudaStream_t st)
 {
-    if (!g || B <= 0 || !lvl_host || !dev_lvl || !makespan_host || !energy_host || !sel_host)
+    if (bits < 1 || bits > 8 || rows < 0 || B < 0) return EMO_E_INVALID_ARG;
+    if (rows == 0 || B == 0) return EMO_OK;
+    const int64_t groups = (B + 7) / 8;
+    if (!packed || !bytes || ldp < groups * bits || ldb < groups * 8 || ldb % 8 != 0 || ((uintptr_t)bytes % 8) != 0) return EMO_E_INVALID_ARG;
+    const int64_t total = rows * groups;
+    const int grid = (int)std::min<int64_t>((total + 255) / 256, 148 * 32);
+    if (pack) emo_repack_levels<true><<<grid, 256, 0, st>>>(bits, rows, groups, packed, ldp, bytes, ldb);
+    else emo_repack_levels<false><<<grid, 256, 0, st>>>(bits, rows, groups, packed, ldp, bytes, ldb);
+    EMO_CUDA(cudaGetLastError());
+    return EMO_OK;
+}
+}  // namespace
+
+int emo_pack_levels(int bits, int64_t rows, int64_t B, const uint8_t *lvl, int64_t ldb, uint8_t *packed, int64_t ldp, void *stream)
+{
+    return repack(true, bits, rows, B, packed, ldp, const_cast<uint8_t *>(lvl), ldb, (cudaStream_t)stream);
+}
+
+int emo_unpack_levels(int bits, int64_t rows, int64_t B, const uint8_t *packed, int64_t ldp, uint8_t *lvl, int64_t ldb, void *stream)
+{
+    return repack(false, bits, rows, B, const_cast<uint8_t *>(packed), ldp, lvl, ldb, (cudaStream_t)stream);
+}
+
+int emo_slack_batch_host_packed(const emo_graph *g, int64_t B, int bits, const uint8_t *lvl_host, int64_t ld_host,
+                                uint8_t *dev_packed, uint8_t *dev_lvl, int64_t ldb, int64_t *slack_dev, int64_t ldo,
+                                int64_t delta_ppm, int64_t *makespan_host, double *energy_host, int64_t *slack_sum_host,
+                                int32_t *n_critical_host, int64_t *sel_host, void *ws, size_t ws_bytes, uint32_t flags,
+                                void *stream)
+{
+    if (!g || B <= 0 || !lvl_host || !dev_lvl || !makespan_host || !energy_host || !sel_host || ldb < B)
         return EMO_E_INVALID_ARG;
+    if (bits < 1 || bits > 8 || (bits < 8 && !dev_packed)) return EMO_E_INVALID_ARG;
     if (g->host_only) return EMO_E_CUDA;
     size_t need = 0, total = 0;
     const int aligned = (ldb % 16 == 0 && aligned16(dev_lvl)) ? 1 : 0;
@@ -1288,7 +1350,15 @@ int emo_slack_batch_host(const emo_graph *g, int64_t B, const uint8_t *lvl_host,
     int64_t *d_sel = (int64_t *)(tail + 4 * per_policy);      // {index, T, E bits, T0, E0 bits}
     int32_t *d_status = (int32_t *)(d_sel + 8);
     EMO_CUDA(cudaMemsetAsync(d_sel, 0, 128, st));
-    EMO_CUDA(cudaMemcpyAsync(dev_lvl, lvl_host, (size_t)g->h.rows * (size_t)ldb, cudaMemcpyHostToDevice, st));
+    if (bits == 8) {
+        if (ld_host != ldb) return EMO_E_INVALID_ARG;
+        EMO_CUDA(cudaMemcpyAsync(dev_lvl, lvl_host, (size_t)g->h.rows * (size_t)ldb, cudaMemcpyHostToDevice, st));
+    } else {
+        // the levels cross the bus packed and are spread to bytes on the device
+        EMO_CUDA(cudaMemcpyAsync(dev_packed, lvl_host, (size_t)g->h.rows * (size_t)ld_host, cudaMemcpyHostToDevice, st));
+        int rcu = emo_unpack_levels(bits, g->h.rows, B, dev_packed, ld_host, dev_lvl, ldb, stream);
+        if (rcu) return rcu;
+    }
     int rc = emo_slack_batch(g, B, dev_lvl, ldb, nullptr, nullptr, slack_dev, ldo, d_T, d_E,
                              slack_sum_host ? d_ss : nullptr, n_critical_host ? d_nc : nullptr, d_sel + 3,
                              (double *)(d_sel + 4), ws, need, d_status, flags, st);
@@ -1309,6 +1379,16 @@ int emo_slack_batch_host(const emo_graph *g, int64_t B, const uint8_t *lvl_host,
     int32_t stc;
     std::memcpy(&stc, &tmp[8], sizeof stc);
     return stc < 0 ? stc : EMO_OK;
+}
+
+int emo_slack_batch_host(const emo_graph *g, int64_t B, const uint8_t *lvl_host, int64_t ldb,
+                         uint8_t *dev_lvl, int64_t *slack_dev, int64_t ldo, int64_t delta_ppm,
+                         int64_t *makespan_host, double *energy_host, int64_t *slack_sum_host,
+                         int32_t *n_critical_host, int64_t *sel_host, void *ws, size_t ws_bytes,
+                         uint32_t flags, void *stream)
+{
+    return emo_slack_batch_host_packed(g, B, 8, lvl_host, ldb, nullptr, dev_lvl, ldb, slack_dev, ldo, delta_ppm, makespan_host,
+                                       energy_host, slack_sum_host, n_critical_host, sel_host, ws, ws_bytes, flags, stream);
 }
 
 }  // extern "C"

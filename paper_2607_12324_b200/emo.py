@@ -30,7 +30,7 @@ EXPORTS = [
     "emo_strerror", "emo_graph_load", "emo_graph_free", "emo_graph_info", "emo_workspace_bytes",
     "emo_eval_policies", "emo_slack_batch", "emo_slack", "emo_baseline", "emo_target_from_delta",
     "emo_select", "emo_transpose_policies", "emo_slack_batch_host", "emo_graph_program",
-    "emo_set_pass_events", "emo_select_static", "emo_graph_flow", "emo_set_wait_limit", "emo_call_path", "emo_set_flow_counters", "emo_workspace_bytes_for",
+    "emo_set_pass_events", "emo_select_static", "emo_graph_flow", "emo_set_wait_limit", "emo_call_path", "emo_set_flow_counters", "emo_workspace_bytes_for", "emo_measure_int_issue", "emo_pack_levels", "emo_unpack_levels", "emo_slack_batch_host_packed",
 ]
 
 
@@ -109,6 +109,10 @@ def lib():
         L.emo_graph_flow.argtypes = [p, ctypes.POINTER(emo_flow_view)]
         L.emo_set_wait_limit.argtypes = [i64]
         L.emo_set_flow_counters.argtypes = [p]
+        L.emo_measure_int_issue.argtypes = [p, p, p]
+        L.emo_pack_levels.argtypes = [ctypes.c_int, i64, i64, p, i64, p, i64, p]
+        L.emo_unpack_levels.argtypes = [ctypes.c_int, i64, i64, p, i64, p, i64, p]
+        L.emo_slack_batch_host_packed.argtypes = [p, i64, ctypes.c_int, p, i64, p, p, i64, p, i64, i64, p, p, p, p, p, p, sz, u32, p]
         L.emo_call_path.argtypes = [p, i64, p, i64, i64, ctypes.c_int, u32]
         L.emo_select_static.argtypes = [i64, p, p, i64, p, i64, p, p, p, p]
         for name in EXPORTS:
@@ -303,12 +307,13 @@ def emo_graph_program(g: Graph, direction: int):
         rows.reshape(steps.value, lanes.value), lat.reshape(q, Lp.value)
 
 
-def emo_graph_flow(g: Graph) -> dict:
-    """The lane-stream program of the 32-bit pass kernels as numpy copies (host-side inspection)."""
+def emo_graph_flow(g: Graph, arrays: bool = True) -> dict:
+    """The lane-stream program of the 32-bit pass kernels as numpy copies (host-side inspection);
+    arrays=False gives the sizes only."""
     v = emo_flow_view()
     _check(lib().emo_graph_flow(g.handle, ctypes.byref(v)), "emo_graph_flow")
     out = {k: getattr(v, k) for k, _ in emo_flow_view._fields_[:16]}
-    if not v.ok32:
+    if not v.ok32 or not arrays:
         return out
     q = v.stages * v.lanes * v.K
 
@@ -348,3 +353,30 @@ def emo_call_path(g: Graph, B, lvl, ldb, ldo, need_slack: bool, flags: int = 0) 
 
 def emo_set_flow_counters(dev):
     _check(lib().emo_set_flow_counters(_addr(dev)), "emo_set_flow_counters")
+
+
+def emo_measure_int_issue(scratch_dev, stream=None) -> dict:
+    """Warp-level integer operations per second of this GPU: 32/64-bit add and max (see include/emo.h)."""
+    out = (ctypes.c_double * 4)()
+    _check(lib().emo_measure_int_issue(ctypes.cast(out, ctypes.c_void_p), _addr(scratch_dev), _stream(stream)),
+           "emo_measure_int_issue")
+    return {"add32": out[0], "max32": out[1], "add64": out[2], "max64": out[3]}
+
+
+def emo_pack_levels(bits, rows, B, lvl, ldb, packed, ldp, stream=None):
+    _check(lib().emo_pack_levels(int(bits), int(rows), int(B), _addr(lvl), int(ldb), _addr(packed), int(ldp), _stream(stream)),
+           "emo_pack_levels")
+
+
+def emo_unpack_levels(bits, rows, B, packed, ldp, lvl, ldb, stream=None):
+    _check(lib().emo_unpack_levels(int(bits), int(rows), int(B), _addr(packed), int(ldp), _addr(lvl), int(ldb), _stream(stream)),
+           "emo_unpack_levels")
+
+
+def emo_slack_batch_host_packed(g: Graph, B, bits, lvl_host, ld_host, dev_packed, dev_lvl, ldb, slack_dev, ldo, delta_ppm,
+                                makespan_host, energy_host, slack_sum_host, n_critical_host, sel_host, ws, flags=0, stream=None):
+    _check(lib().emo_slack_batch_host_packed(g.handle, int(B), int(bits), _addr(lvl_host), int(ld_host), _addr(dev_packed),
+                                             _addr(dev_lvl), int(ldb), _addr(slack_dev), int(ldo), int(delta_ppm),
+                                             _addr(makespan_host), _addr(energy_host), _addr(slack_sum_host),
+                                             _addr(n_critical_host), _addr(sel_host), _addr(ws), _nbytes(ws), int(flags),
+                                             _stream(stream)), "emo_slack_batch_host_packed")

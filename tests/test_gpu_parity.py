@@ -448,6 +448,27 @@ def test_host_buffer_call(torch_cuda, emo, oracle_mod):
     want = oracle_mod.select(r_or["makespan"], r_or["energy"], oracle_mod.target_from_delta(T0, ppm))
     assert int(sel[0]) == want and int(sel[1]) == r_or["makespan"][want]
     assert np.array([int(sel[2])], dtype=np.int64).view(np.float64)[0] == pytest.approx(r_or["energy"][want], rel=E_RTOL)
+    # the same call with the levels packed at 4 bits (16 levels): pack on the device, round trip, then the call
+    bits = 4
+    ldp = ((B + 7) // 8 * bits + 15) // 16 * 16
+    lv_dev = lv.cuda()
+    packed = torch.zeros((g.n, ldp), dtype=torch.uint8, device="cuda")
+    emo.emo_pack_levels(bits, g.n, B, lv_dev, ldb, packed, ldp)
+    back = torch.full_like(lv_dev, 0xEE)
+    emo.emo_unpack_levels(bits, g.n, B, packed, ldp, back, ldb)
+    torch.cuda.synchronize()
+    assert torch.equal(back[:, :B], lv_dev[:, :B])
+    pk = packed.cpu().numpy()
+    lvn = lv.numpy()
+    assert pk[3, 0] == (int(lvn[3, 0]) | (int(lvn[3, 1]) << 4)), "two 4-bit levels per byte, the first in the low bits"
+    packed_host = packed.cpu().pin_memory()
+    slack.zero_()
+    T.zero_()
+    for fl in (0, emo.EMO_F_FLOW_KERNEL):
+        ws2 = torch.empty(emo.emo_workspace_bytes(h, B, 2, fl), dtype=torch.uint8, device="cuda")
+        emo.emo_slack_batch_host_packed(h, B, bits, packed_host, ldp, packed, dev_lvl, ldb, slack, B, ppm, T, E, ss, nc, sel, ws2, flags=fl)
+        assert np.array_equal(T.numpy(), r_or["makespan"]) and int(sel[0]) == want
+        assert np.array_equal(slack.cpu().numpy(), r_or["slack"])
     h.free()
 
 
