@@ -12,9 +12,9 @@
  *   makespan ................................. Eq. 2 (T_DAG = max over all v of C_v), Alg. 1 "T <- max comp[v]"
  *   energy ................................... Eq. 2 without E_idle (sum over v of e_v), Alg. 1 "E_a <- E_a + e"
  *   backward pass / slack .................... critical-path-method total float; the paper only
- *                                              describes slack in words (Sec. 1, "time windows where
- *                                              kernels are not on the critical path"), so the textbook
- *                                              recurrence is used: LF_v = min over successors of LS_u
+ *                                              describes slack in words (Sec. 1: the time a kernel
+ *                                              can be delayed without touching the critical path), so
+ *                                              the textbook recurrence is used: LF_v = min over successors of LS_u
  *                                              (T for sinks), LS_v = LF_v - t_v, slack_v = LS_v - ES_v
  *   target ................................... Sec. 4.6: T_0 is the makespan at maximum frequency and
  *                                              the budget is a fraction of it (2 %, 5 % in Sec. 5)

@@ -233,14 +233,12 @@ bool staged_shape(const emo_graph *g, const Program &p, int rec_bytes, bool back
     for (; G >= 1; --G) {
         const size_t P = 64 * (size_t)G;
         const size_t fixed = (size_t)G * p.slots * kSlotStride + (size_t)G * p.lanes * 1024 + 256 + 128;
-        const size_t per_step = (size_t)p.lanes * ((size_t)rec_bytes + P + (backward ? P * 8 : 0));
         for (int t = 0; t < 5; ++t) {
             const int sc = kTry[t][0], stages = kTry[t][1];
             const size_t ne = (size_t)sc * p.lanes;
             if (ne > 32 * (size_t)kRowRegs) continue;
             const size_t stage_bytes = round_up(ne * ((size_t)rec_bytes + P + (backward ? P * 8 : 0)), 128);
             if (fixed + stages * stage_bytes > budget) continue;
-            (void)per_step;
             sp.sc = sc;
             sp.stages = stages;
             sp.ptile = (int)P;
@@ -320,7 +318,7 @@ struct PassPlan {
     size_t spill_bytes = 0;   // tiled spill: [tiles][rows of the backward program][backward tile]
 };
 
-// rows of one tile of the spill: the entries of the backward program (padded for the in-thread kernel)
+// rows of one tile of the spill: the entries of the backward program (padded to whole stages for the lane kernel)
 size_t spill_rows_of(const emo_graph *g, bool lane)
 {
     return (size_t)(lane ? g->lbwd.steps_pad : g->bwd.steps) * g->bwd.lanes;

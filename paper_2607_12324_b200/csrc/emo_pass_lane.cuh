@@ -5,8 +5,8 @@
 // policies per thread this doubles the number of resident warps, which is what the path is short
 // of: every warp is a serial chain of dependent steps, and only other warps can fill the issue slots
 // it leaves.  The per-entry work is kept small by a program layout made for it (see
-// emo_lane_layout.cuh: 32-byte entries with the running-value mask precomputed, one 16-byte table
-// element per level holding duration and energy together).
+// emo_lane_layout.cuh: 32-byte entries with the running-value mask precomputed, one 12-byte table
+// element per level: duration, energy high word, energy low word).
 //
 // The warps of a group do not run in lockstep.  Each walks its own column of the step program and
 // waits only for the values it reads: every exchange slot (32 x 8 bytes) has an mbarrier whose phase
