@@ -298,11 +298,13 @@ int emo_call_path(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t ldb
 int emo_measure_int_issue(double *ops_per_s, void *scratch_dev, void *stream);
 
 /*
- * emo_set_flow_counters - measurement hook (no counterpart in the method): a device array of 131072
- * int64 that later calls of the 32-bit kernels fill with cycle counts, 4 per warp at
- * [(pass * 512 + block) * 32 + warp] for the first 512 blocks (pass 0 forward, 1 backward): consumer
- * warps {cycles waiting for staged data, cycles at group barriers, total}, producer warps {cycles
- * waiting for a free buffer, cycles issuing copies, total}.  NULL switches it off.  Process-wide.
+ * emo_set_flow_counters - measurement hook (no counterpart in the method): a device array of 262144
+ * int64 that later calls of the 32-bit kernels fill with cycle counts, 8 per warp at
+ * [((pass * 512 + block) * 32 + warp) * 8] for the first 512 blocks (pass 0 forward, 1 backward): consumer
+ * warps {cycles waiting for staged data, cycles at group barriers, total, backward only: cycles in
+ * entries that need their record, cycles in runs of simple entries}, producer warps {cycles waiting
+ * for a free buffer, cycles issuing copies, total}; the other words are spare.  NULL switches it off.
+ * Process-wide.
  */
 int emo_set_flow_counters(void *dev);
 

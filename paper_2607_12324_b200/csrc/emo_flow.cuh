@@ -56,7 +56,7 @@ struct FlowParams {
     int32_t *status;
     long long wait_cycles;               // bound of every device-side wait
     int stall_stage;                     // test hook: the producers stop before this stage (-1: off)
-    long long *prof;                     // optional cycle counters, 4 per warp: waits for stages, group barriers, total, spare
+    long long *prof;                     // optional cycle counters, 8 per warp: waits for stages, group barriers, total, backward: special entries, runs
 };
 
 __device__ __forceinline__ unsigned long long emo_lds_b64v(unsigned a)
@@ -228,6 +228,56 @@ __device__ __forceinline__ void emo_flow_out(unsigned slot_base, int lane, unsig
     }
 }
 
+// The same two steps without a branch, for the entries that need their record.  Every access is
+// predicated on the descriptor's kind bits, so that an entry costs one straight run of instructions
+// whatever it reads and writes; a branch costs a lone warp some forty cycles of fetch bubble, and these
+// entries sit on the lanes' critical paths.
+// Operand: x = the slot's value (0 when the operand is absent), tg = the tag found beside it (tagged
+// slots only), a = the address read (for a later poll).
+__device__ __forceinline__ void emo_flow_operand_u(unsigned slot_lane4, unsigned lane4, unsigned w, unsigned present, unsigned &x,
+                                                   unsigned &tg, unsigned &a)
+{
+    asm volatile(
+        "{\n\t.reg .pred pp, pw, pt, pc;\n\t.reg .b32 k;\n\t.reg .b64 t;\n\t"
+        "setp.ne.u32 pp, %4, 0;\n\t"
+        "and.b32 k, %3, 0x40000000;\n\t"
+        "setp.ne.and.u32 pw, k, 0, pp;\n\t"
+        "setp.eq.and.u32 pt, k, 0, pp;\n\t"
+        "and.b32 k, %3, 0x20000000;\n\t"
+        "setp.ne.and.u32 pc, k, 0, pp;\n\t"
+        "and.b32 %2, %3, 0x1FFFFFFF;\n\t"
+        "add.u32 %2, %2, %5;\n\t"
+        "@pt add.u32 %2, %2, %6;\n\t"
+        "mov.u32 %0, 0;\n\t"
+        "mov.u32 %1, 0;\n\t"
+        "@pw ld.volatile.shared.u32 %0, [%2];\n\t"
+        "@pt ld.volatile.shared.b64 t, [%2];\n\t"
+        "@pt mov.b64 {%0, %1}, t;\n\t"
+        "@pc st.volatile.shared.u32 [%2], 0;\n\t}"
+        : "=&r"(x), "=&r"(tg), "=&r"(a)
+        : "r"(w), "r"(present), "r"(slot_lane4), "r"(lane4)
+        : "memory");
+}
+// Output: tagged (value + tag), settled (corrected value) or shared (corrected value folded in), or none.
+__device__ __forceinline__ void emo_flow_out_u(unsigned slot_lane4, unsigned lane4, unsigned v, unsigned off, unsigned aux, unsigned tagged,
+                                               unsigned settled, unsigned shared)
+{
+    asm volatile(
+        "{\n\t.reg .pred pt, ps, pa;\n\t.reg .b32 aw, at, xs;\n\t"
+        "setp.ne.u32 pt, %5, 0;\n\t"
+        "setp.ne.u32 pa, %7, 0;\n\t"
+        "setp.ne.and.u32 ps, %6, 0, !pa;\n\t"
+        "add.u32 aw, %0, %3;\n\t"
+        "add.u32 at, aw, %1;\n\t"
+        "max.u32 xs, %2, %4;\n\t"
+        "sub.u32 xs, xs, %4;\n\t"
+        "@pt st.volatile.shared.v2.u32 [at], {%2, %4};\n\t"
+        "@ps st.volatile.shared.u32 [aw], xs;\n\t"
+        "@pa red.shared.max.u32 [aw], xs;\n\t}"
+        ::"r"(slot_lane4), "r"(lane4), "r"(v), "r"(off), "r"(aux), "r"(tagged), "r"(settled), "r"(shared)
+        : "memory");
+}
+
 // The producer warps of both kernels.  Stages are issued in walking order (backward: last first).
 template <bool BWD>
 __device__ __forceinline__ void emo_flow_produce(const FlowParams &p, unsigned stage0, unsigned bar0, volatile int *abort_word,
@@ -319,7 +369,7 @@ __device__ __forceinline__ void emo_flow_produce(const FlowParams &p, unsigned s
         t_issue += clock64() - tw1;
     }
     if (p.prof && lane == 0 && blockIdx.x < 512) {
-        long long *pr = p.prof + ((size_t)blockIdx.x * 32 + (threadIdx.x >> 5)) * 4;
+        long long *pr = p.prof + ((size_t)blockIdx.x * 32 + (threadIdx.x >> 5)) * 8;
         pr[0] = t_wait;
         pr[1] = t_issue;
         pr[2] = clock64() - t_begin;
@@ -413,6 +463,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_flow_fwd(FlowParams p)
         emo_flow_produce<false>(p, stage0, bar0, abort_word, lane, warp - n_cons);
     } else {
         const unsigned slot_base = smem0 + (unsigned)group * p.slot_bytes;
+        const unsigned lane4 = (unsigned)lane * 4u, slot_lane4 = slot_base + lane4;
         const unsigned lmask = (unsigned)p.Lp - 1u, tab_row = p.tab_row;
         const int gthreads = lanes * 32;
         const long long limit = p.wait_cycles;
@@ -471,19 +522,26 @@ __global__ void __launch_bounds__(MAXT, 1) emo_flow_fwd(FlowParams p)
                 const int r = (int)(sg & emo::kSegRunMask);
                 const unsigned sp = (sg >> 4) & 1u;
                 if (sp) {
-                    // an entry that needs its record; everything it reads from the stage is requested at once
+                    // an entry that needs its record; everything it reads from the stage is requested at once, and
+                    // the common shapes (at most one operand, any output) run without a branch
                     const uint4 r0 = emo_tld_128(rec_a, tok);
                     const uint4 r1 = emo_tld_128(rec_a + 16u, tok);
                     const unsigned lb = emo_tld_u8(lvl_a, tok);
-                    const unsigned fl = emo_uniform(r0.x);
+                    const unsigned fl = r0.x;
                     const unsigned ta = tab_a + (lb & lmask) * 12u;
                     const unsigned dd = emo_tld_u32(ta, tok), ghi = emo_tld_u32(ta + 4u, tok), glo = emo_tld_u32(ta + 8u, tok);
                     const unsigned nops = fl >> emo::kF_NopsShift;
                     unsigned v = emo_floor_sub((fl & emo::kF_HasReg) ? h : 0u, r1.w);
-                    unsigned pa = pool_a + r0.w * 4u;
-                    if (nops) {
-                        const unsigned x = emo_flow_operand(slot_base, lane, r1.x, r1.y, dead, abort_word, limit);
-                        v = max(v, emo_floor_sub(x, r1.z));
+                    unsigned x0, t0, a0;
+                    emo_flow_operand_u(slot_lane4, lane4, r1.x, nops, x0, t0, a0);
+                    const bool retry0 = nops != 0u && (r1.x & (emo::kOpWord | emo::kOpNoPoll)) == 0u && t0 != r1.y;
+                    if (__any_sync(0xFFFFFFFFu, retry0 || nops > 1u || (fl & emo::kF_Terminal) != 0u)) {
+                        // the rest: a value that was not there yet, further operands, the makespan candidate
+                        if (retry0 && !emo_flow_poll(a0, r1.y, x0, abort_word, limit)) {
+                            dead = true;
+                            *abort_word = 1;
+                        }
+                        unsigned pa = pool_a + r0.w * 4u;
                         for (unsigned k = 1; k < nops; ++k) {
                             const unsigned x2 = emo_flow_operand(slot_base, lane, emo_tld_u32(pa, tok), emo_tld_u32(pa + 4u, tok), dead,
                                                                  abort_word, limit);
@@ -492,19 +550,20 @@ __global__ void __launch_bounds__(MAXT, 1) emo_flow_fwd(FlowParams p)
                         }
                         dead = __any_sync(0xFFFFFFFFu, dead);
                         if (dead) continue;      // on to the group's next barrier
+                        if (fl & emo::kF_Terminal) {
+                            const long long lbc = (long long)((unsigned long long)emo_tld_u32(pa, tok) | ((unsigned long long)emo_tld_u32(pa + 4u, tok) << 32));
+                            const unsigned vt = max(v, emo_floor_sub(x0, r1.z)) + dd;
+                            acc = emo_max64(acc, lbc + (long long)vt);
+                        }
                     }
+                    v = max(v, emo_floor_sub(x0, r1.z));
                     if ((fl & emo::kF_Push) && push) {
                         *push = h;
                         push += ptile;
                     }
                     ea += __hiloint2double((int)ghi, (int)glo);
                     v += dd;
-                    if (fl & (emo::kF_OutTag | emo::kF_OutSet))
-                        emo_flow_out(slot_base, lane, v, (fl & emo::kF_OutTag) != 0, (fl & emo::kF_OutAcc) != 0, r0.y, r0.z);
-                    if (fl & emo::kF_Terminal) {
-                        const long long lbc = (long long)((unsigned long long)emo_tld_u32(pa, tok) | ((unsigned long long)emo_tld_u32(pa + 4u, tok) << 32));
-                        acc = emo_max64(acc, lbc + (long long)v);
-                    }
+                    emo_flow_out_u(slot_lane4, lane4, v, r0.y, r0.z, fl & emo::kF_OutTag, fl & emo::kF_OutSet, fl & emo::kF_OutAcc);
                     h = v;
                     rec_a += 32u;
                     tab_a += tab_row;
@@ -533,7 +592,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_flow_fwd(FlowParams p)
             if (lane == 0) emo_mbar_arrive(bar0 + 8 * (kFlowMaxBuf + s));
         }
         if (p.prof && lane == 0 && blockIdx.x < 512) {
-            long long *pr = p.prof + ((size_t)blockIdx.x * 32 + warp) * 4;
+            long long *pr = p.prof + ((size_t)blockIdx.x * 32 + warp) * 8;
             pr[0] = t_wait;
             pr[1] = t_bar;
             pr[2] = clock64() - t_begin;
@@ -608,6 +667,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_flow_bwd(FlowParams p)
     } else {
         const unsigned slot_lane = smem0 + (unsigned)group * p.slot_bytes + (unsigned)lane * 4u;
         const unsigned slot_base = smem0 + (unsigned)group * p.slot_bytes;
+        const unsigned lane4 = (unsigned)lane * 4u, slot_lane4 = slot_lane;
         const unsigned lmask = (unsigned)p.Lp - 1u, tab_row = p.tab_row;
         const int gthreads = lanes * 32;
         const long long limit = p.wait_cycles;
@@ -625,6 +685,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_flow_bwd(FlowParams p)
         long long t_wait = 0, t_bar = 0;
         const long long t_begin = clock64();
         unsigned rec_a = 0, tab_a = 0, lvl_a = 0, xes_a = 0, pop_a = 0, tok = 0;
+        long long t_spec = 0, t_run = 0;
         bool has_in = false, has_out = false;
 
         // what every entry does once the maximum over its successors (qin) is known
@@ -650,7 +711,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_flow_bwd(FlowParams p)
         auto run = [&](auto rc, auto inc, auto outc, unsigned o) {
             constexpr int R = decltype(rc)::value;
             constexpr bool IN = decltype(inc)::value, OUT = decltype(outc)::value;
-            const unsigned rec_o = rec_a + 48u * o, tab_o = tab_a + o * tab_row, lvl_o = lvl_a + 32u * o, xes_o = xes_a + 8u * o;
+            const unsigned rec_o = rec_a + 64u * o, tab_o = tab_a + o * tab_row, lvl_o = lvl_a + 32u * o, xes_o = xes_a + 8u * o;
             unsigned lv[R], d[R];
 #pragma unroll
             for (int j = 0; j < R; ++j) lv[j] = emo_tld_u8(lvl_o + 32u * j, tok);
@@ -658,8 +719,8 @@ __global__ void __launch_bounds__(MAXT, 1) emo_flow_bwd(FlowParams p)
             for (int j = 0; j < R; ++j) d[j] = emo_tld_u32(tab_o + (unsigned)j * tab_row + (lv[j] & lmask) * 4u, tok);
 #pragma unroll
             for (int j = R - 1; j >= 0; --j) {
-                const uint4 r0j = emo_tld_128(rec_o + 48u * j, tok);
-                const uint4 r1j = emo_tld_128(rec_o + 48u * j + 16u, tok);
+                const uint4 r0j = emo_tld_128(rec_o + 64u * j, tok);
+                const uint4 r1j = emo_tld_128(rec_o + 64u * j + 16u, tok);
                 unsigned qin = emo_floor_sub(q, r1j.w);
                 if (IN) {
                     const unsigned a = slot_lane + r0j.w;
@@ -710,7 +771,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_flow_bwd(FlowParams p)
             const unsigned total = (hd0.x >> 16) & 255u;
             const unsigned seg_a = sta + p.off_seg + (unsigned)chain * emo::kSegBytes;
             // one past the lane's last entry of this stage; every segment steps down before it reads
-            rec_a = sta + p.off_rec + ((unsigned)(chain * K) + total) * 48u;
+            rec_a = sta + p.off_rec + ((unsigned)(chain * K) + total) * 64u;
             tab_a = sta + p.off_tab + ((unsigned)(chain * K) + total) * tab_row;
             lvl_a = sta + p.off_lvl + (((unsigned)((group * lanes + chain) * K) + total) << 5) + (unsigned)lane;
             xes_a = sta + p.off_lbes + ((unsigned)(chain * K) + total) * 8u;
@@ -736,52 +797,61 @@ __global__ void __launch_bounds__(MAXT, 1) emo_flow_bwd(FlowParams p)
                 }
                 tok = emo_token(tok + 1u);
                 const int r = (int)(sg & emo::kSegRunMask);
+                const long long ts0 = clock64();
                 if (sg & emo::kSegSpecial) {
-                    // an entry that needs its record: any operands, any kind of output
-                    rec_a -= 48u;
+                    // an entry that needs its record: any operands, any kind of output.  Up to two operands
+                    // and every kind of output run without a branch.
+                    rec_a -= 64u;
                     tab_a -= tab_row;
                     lvl_a -= 32u;
                     xes_a -= 8u;
                     const uint4 r0 = emo_tld_128(rec_a, tok);
                     const uint4 r1 = emo_tld_128(rec_a + 16u, tok);
                     const uint4 r2 = emo_tld_128(rec_a + 32u, tok);
+                    const uint4 r3 = emo_tld_128(rec_a + 48u, tok);
                     const unsigned lb = emo_tld_u8(lvl_a, tok);
-                    const unsigned fl = emo_uniform(r0.x);
+                    const unsigned fl = r0.x;
                     const unsigned dd = emo_tld_u32(tab_a + (lb & lmask) * 4u, tok);
                     const unsigned nops = fl >> emo::kB_NopsShift;
                     unsigned qin = emo_floor_sub((fl & emo::kB_HasReg) ? q : 0u, r1.w);
-                    if (nops) {
-                        if (fl & emo::kB_Simple) {
-                            const unsigned a = slot_lane + r0.w;
-                            qin = max(qin, emo_lds_u32v(a));
-                            emo_sts_u32v(a, 0u);
-                        } else {
-                            const unsigned x = emo_flow_operand(slot_base, lane, r2.x, r2.y, dead, abort_word, limit);
-                            qin = max(qin, emo_floor_sub(x, r2.z));
-                            unsigned pa = pool_a + r0.w * 4u;
-                            for (unsigned k = 1; k < nops; ++k) {
-                                const unsigned x2 = emo_flow_operand(slot_base, lane, emo_tld_u32(pa, tok), emo_tld_u32(pa + 4u, tok), dead,
-                                                                     abort_word, limit);
-                                qin = max(qin, emo_floor_sub(x2, emo_tld_u32(pa + 8u, tok)));
-                                pa += 12u;
-                            }
-                            dead = __any_sync(0xFFFFFFFFu, dead);
-                            if (dead) continue;      // on to the group's next barrier
+                    unsigned x0, t0, a0, x1, t1, a1;
+                    emo_flow_operand_u(slot_lane4, lane4, r2.x, nops, x0, t0, a0);
+                    emo_flow_operand_u(slot_lane4, lane4, r3.x, nops > 1u, x1, t1, a1);
+                    const bool retry0 = nops != 0u && (r2.x & (emo::kOpWord | emo::kOpNoPoll)) == 0u && t0 != r2.y;
+                    const bool retry1 = nops > 1u && (r3.x & (emo::kOpWord | emo::kOpNoPoll)) == 0u && t1 != r3.y;
+                    if (__any_sync(0xFFFFFFFFu, retry0 || retry1 || nops > 2u)) {
+                        // the rest: values that were not there yet, further operands
+                        if (retry0 && !emo_flow_poll(a0, r2.y, x0, abort_word, limit)) dead = true;
+                        if (retry1 && !emo_flow_poll(a1, r3.y, x1, abort_word, limit)) dead = true;
+                        if (dead) *abort_word = 1;      // the other waits of the block end early
+                        unsigned pa = pool_a + r0.w * 4u;
+                        for (unsigned k = 2; k < nops; ++k) {
+                            const unsigned x2 = emo_flow_operand(slot_base, lane, emo_tld_u32(pa, tok), emo_tld_u32(pa + 4u, tok), dead,
+                                                                 abort_word, limit);
+                            qin = max(qin, emo_floor_sub(x2, emo_tld_u32(pa + 8u, tok)));
+                            pa += 12u;
                         }
+                        dead = __any_sync(0xFFFFFFFFu, dead);
+                        if (dead) continue;      // on to the group's next barrier
                     }
-                    finish(qin, dd, r1.z, r1.x, r1.y, xes_a);
-                    q = qin + dd;
-                    if (fl & (emo::kB_OutTag | emo::kB_OutSet))
-                        emo_flow_out(slot_base, lane, q, (fl & emo::kB_OutTag) != 0, (fl & emo::kB_OutAcc) != 0, r0.y, r0.z);
-                    if (fl & emo::kB_Pop) {
-                        pop_a -= ptile4;
-                        c = emo_tld_u32(pop_a, tok);
+                    qin = max(qin, max(emo_floor_sub(x0, r2.z), emo_floor_sub(x1, r3.z)));
+                    if (EXTRA) {
+                        finish(qin, dd, r1.z, r1.x, r1.y, xes_a);
                     } else {
-                        c -= dd;
+                        const long long A = (long long)((unsigned long long)r1.x | ((unsigned long long)r1.y << 32));
+                        const long long sl = (T - A) - (long long)((unsigned long long)qin + (unsigned long long)c);
+                        emo_stg_s64_if(sl_lane, r1.z, ldo8, sl, sl_ok);
                     }
+                    q = qin + dd;
+                    emo_flow_out_u(slot_lane4, lane4, q, r0.y, r0.z, fl & emo::kB_OutTag, fl & emo::kB_OutSet, fl & emo::kB_OutAcc);
+                    const unsigned pops = fl & emo::kB_Pop;
+                    pop_a -= pops ? ptile4 : 0u;
+                    c = emo_tld_u32_if(pop_a, tok, pops, c - dd);
                 }
+                const long long ts1 = clock64();
+                t_spec += ts1 - ts0;
                 // the run below it, from its highest position down
-                rec_a -= (unsigned)r * 48u;
+                rec_a -= (unsigned)r * 64u;
                 tab_a -= (unsigned)r * tab_row;
                 lvl_a -= (unsigned)r * 32u;
                 xes_a -= (unsigned)r * 8u;
@@ -800,6 +870,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_flow_bwd(FlowParams p)
                     }
                     if (rem) run_kind(std::integral_constant<int, 1>{}, 0u);
                 }
+                t_run += clock64() - ts1;
             }
             if (leave) break;
             asm volatile("" ::"r"(q), "r"(c) : "memory");
@@ -807,10 +878,12 @@ __global__ void __launch_bounds__(MAXT, 1) emo_flow_bwd(FlowParams p)
             if (lane == 0) emo_mbar_arrive(bar0 + 8 * (kFlowMaxBuf + s));
         }
         if (p.prof && lane == 0 && blockIdx.x < 512) {
-            long long *pr = p.prof + ((size_t)blockIdx.x * 32 + warp) * 4;
+            long long *pr = p.prof + ((size_t)blockIdx.x * 32 + warp) * 8;
             pr[0] = t_wait;
             pr[1] = t_bar;
             pr[2] = clock64() - t_begin;
+            pr[3] = t_spec;
+            pr[4] = t_run;
         }
         if (leave && lane == 0) {
             *abort_word = 1;

@@ -37,8 +37,9 @@ namespace emo {
 constexpr int kFlowMaxLanes = 30;
 constexpr int kFRecWords = 8;      // forward record: flags, out slot, out tag / correction, pool offset, first operand
                                    // (3 words), correction of the lane's previous value
-constexpr int kBRecWords = 12;     // backward record: flags, out slot, out tag / correction, pool offset, A_v (2 words),
-                                   // node id, correction of the lane's previous value, first operand (3 words), spare
+constexpr int kBRecWords = 16;     // backward record: flags, out slot, out tag / correction, pool offset, A_v (2 words),
+                                   // node id, correction of the lane's previous value, first operand (3 words), spare,
+                                   // second operand (3 words), spare; further operands sit in the pool
 constexpr int kOpWords = 3;        // operand descriptor: slot offset | kind bits, tag, delta
 constexpr int kHdrWords = 8;       // per (stage, lane): word 0 = forward segments (bits 0..7) | backward segments (8..15)
                                    // | entries (16..23); word 4 pushes, word 5 first restore row inside the stage,

@@ -433,6 +433,7 @@ int compile_flow(const HostGraph &g, const int64_t *lat, const double *energy, i
             r[3] = (uint32_t)pool.size();
             for (size_t k = 0; k < opw.size(); ++k) {
                 if (k < 3) r[8 + k] = opw[k];
+                else if (k < 6) r[12 + (k - 3)] = opw[k];
                 else pool.push_back(opw[k]);
             }
             if (push_flag[v]) fl |= kB_Pop;

@@ -686,7 +686,7 @@ int launch_flow_bwd(const emo_graph *g, const FlowPlan &pl, int64_t B, const uin
     p.slack_sum = slack_sum;
     p.n_critical = n_critical;
     p.status = status;
-    p.prof = g_flow_prof ? g_flow_prof + 65536 : nullptr;
+    p.prof = g_flow_prof ? g_flow_prof + 131072 : nullptr;
     if (flags & EMO_F_TEST_STALL) p.stall_stage = p.stages / 2;
     cudaEvent_t ev0 = g_pass_events[2], ev1 = g_pass_events[3];
     if (ev0) EMO_CUDA(cudaEventRecord(ev0, st));

@@ -329,7 +329,7 @@ def emo_graph_flow(g: Graph, arrays: bool = True) -> dict:
     out["tab_fwd"] = arr(v.tab_fwd, q * v.Lp * 3, u32, np.uint32).reshape(v.stages, v.lanes, v.K, v.Lp, 3)
     out["tab_bwd"] = arr(v.tab_bwd, q * v.Lp, u32, np.uint32).reshape(v.stages, v.lanes, v.K, v.Lp)
     out["rec_fwd"] = arr(v.rec_fwd, q * 8, u32, np.uint32).reshape(v.stages, v.lanes, v.K, 8)
-    out["rec_bwd"] = arr(v.rec_bwd, q * 12, u32, np.uint32).reshape(v.stages, v.lanes, v.K, 12)
+    out["rec_bwd"] = arr(v.rec_bwd, q * 16, u32, np.uint32).reshape(v.stages, v.lanes, v.K, 16)
     out["pool_fwd"] = arr(v.pool_fwd, v.stages * v.pool_stride_fwd, u32, np.uint32).reshape(v.stages, v.pool_stride_fwd)
     out["pool_bwd"] = arr(v.pool_bwd, v.stages * v.pool_stride_bwd, u32, np.uint32).reshape(v.stages, v.pool_stride_bwd)
     out["seg_fwd"] = arr(v.seg_fwd, v.stages * v.lanes * 40, ctypes.c_uint8, np.uint8).reshape(v.stages, v.lanes, 40)

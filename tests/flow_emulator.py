@@ -188,8 +188,8 @@ def run_backward(f, lvl, L, T, restore, n):
                         qin = np.maximum(qin, slots.read(OP_WORD | OP_NOPOLL | OP_CLEAR | int(rec[3]), None, period))
                 else:
                     for k in range(fl >> 16):
-                        if k == 0:
-                            w, tag, delta = int(rec[8]), int(rec[9]), int(rec[10])
+                        if k < 2:      # the first two operands sit in the record
+                            w, tag, delta = int(rec[8 + 4 * k]), int(rec[9 + 4 * k]), int(rec[10 + 4 * k])
                         else:
                             w, tag, delta = int(pool[pp]), int(pool[pp + 1]), int(pool[pp + 2])
                             pp += 3
