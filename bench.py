@@ -288,11 +288,17 @@ def main():
     t_issue = passes * B / 32.0 * (n / ipk["add32"] + m / ipk["max32"]) * 1e3
     sm_mhz = (clocks or {}).get("sm_mhz") or 1965.0
     t_depth = passes * info.depth * 30.0 / (sm_mhz * 1e6) * 1e3
+    # what one warp alone pays for the kernels' steps, and the measured time per schedule step: the passes walk a
+    # dependency chain as long as the schedule, so the per-step latency times the steps is the time
+    costs = emo.emo_measure_warp_costs(scratch)
     bounds = {"t_hbm_ms": t_hbm, "t_issue_ms": t_issue, "depth_floor_ms": t_depth,
               "binding": "hbm" if t_hbm >= t_issue else "int_issue",
               "int_issue_peak_warp_ops_per_s": ipk,
-              "frac_of_binding": max(t_hbm, t_issue) / ms_per_step}
+              "frac_of_binding": max(t_hbm, t_issue) / ms_per_step,
+              "warp_costs_cycles": {k: round(v, 2) for k, v in costs.items()}}
     path = emo.emo_call_path(h, B, lv, ldb, B, True, args.call_flags)
+    if path == 2 and fl["steps"]:
+        bounds["cycles_per_schedule_step"] = {"forward": fwd * 1e-3 * sm_mhz * 1e6 / fl["steps"], "backward": bwd * 1e-3 * sm_mhz * 1e6 / fl["steps"]}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "int64", "data": "synthetic",

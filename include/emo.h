@@ -298,6 +298,18 @@ int emo_call_path(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t ldb
 int emo_measure_int_issue(double *ops_per_s, void *scratch_dev, void *stream);
 
 /*
+ * emo_measure_warp_costs - measurement helper (no counterpart in the method): what one warp alone pays, in
+ * SM cycles, for the steps the pass kernels are made of.  The recurrences (Eq. 1 and its mirror) are walked
+ * as a dependency chain of as many steps as the graph is deep, with a few warps per scheduler, so these
+ * latencies and not a pipe's throughput set the kernels' speed.  Writes cycles[8] (host): dependent 32-bit
+ * add; dependent max then subtract; dependent shared-memory load; independent adds (issue interval); a loop
+ * body of one shared load and four dependent operations with a never-taken branch on the loaded word; the
+ * same body without the branch; redux.sync then add; a named barrier of five warps.
+ * scratch_dev: device memory of at least 128 bytes.  Synchronises the stream.
+ */
+int emo_measure_warp_costs(double *cycles, void *scratch_dev, void *stream);
+
+/*
  * emo_set_flow_counters - measurement hook (no counterpart in the method): a device array of 262144
  * int64 that later calls of the 32-bit kernels fill with cycle counts, 8 per warp at
  * [((pass * 512 + block) * 32 + warp) * 8] for the first 512 blocks (pass 0 forward, 1 backward): consumer

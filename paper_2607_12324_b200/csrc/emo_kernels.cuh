@@ -273,6 +273,116 @@ __global__ void emo_transpose_u8(int64_t B, int64_t rows, const uint8_t *src, in
 }
 
 // ------------------------------------------------------------------------------------------------
+// What one warp alone pays, in cycles (clock64 around a loop, thread 0 reports): the pass kernels walk
+// a dependency chain of tens of thousands of steps with a handful of warps per scheduler, so their
+// speed is set by these latencies and not by a pipe's throughput.
+//   0 dependent 32-bit add                      1 dependent max followed by subtract (one correction)
+//   2 dependent shared-memory load              3 independent adds (issue interval)
+//   4 loop body: shared load, four dependent operations, and a never-taken branch on the loaded word
+//   5 the same body without the branch           6 redux.sync followed by an add (dependent)
+//   7 named barrier of all warps of the block (run with five warps)
+// ------------------------------------------------------------------------------------------------
+__device__ __noinline__ unsigned emo_cost_rare(unsigned a)
+{
+    for (int i = 0; i < 64; ++i) a = a * 3u + 1u;
+    return a;
+}
+__global__ void emo_warp_costs(long long *out, const unsigned *zeros, int iters, unsigned seed)
+{
+    __shared__ unsigned s[1024];
+    for (int i = threadIdx.x; i < 1024; i += blockDim.x) s[i] = ((unsigned)i + 32u) & 1023u;
+    __syncthreads();
+    const bool warp0 = threadIdx.x < 32;
+    long long t[8];
+    unsigned keep = 0;
+    if (warp0) {
+        {
+            unsigned a = seed;
+            const long long t0 = clock64();
+            for (int i = 0; i < iters; ++i)
+#pragma unroll
+                for (int j = 0; j < 32; ++j) asm volatile("add.u32 %0, %0, %1;" : "+r"(a) : "r"(seed));
+            t[0] = (clock64() - t0) / 32;
+            keep ^= a;
+        }
+        {
+            unsigned a = seed;
+            const long long t0 = clock64();
+            for (int i = 0; i < iters; ++i)
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    asm volatile("max.u32 %0, %0, %1;" : "+r"(a) : "r"(seed + (unsigned)j));
+                    asm volatile("sub.u32 %0, %0, %1;" : "+r"(a) : "r"(seed));
+                }
+            t[1] = (clock64() - t0) / 32;
+            keep ^= a;
+        }
+        {
+            unsigned q = threadIdx.x;
+            const long long t0 = clock64();
+            for (int i = 0; i < iters; ++i)
+#pragma unroll
+                for (int j = 0; j < 32; ++j) q = *(volatile unsigned *)&s[q];
+            t[2] = (clock64() - t0) / 32;
+            keep ^= q;
+        }
+        {
+            unsigned a[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) a[k] = seed + (unsigned)k;
+            const long long t0 = clock64();
+            for (int i = 0; i < iters; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) asm volatile("add.u32 %0, %0, %1;" : "+r"(a[k]) : "r"(seed));
+            t[3] = (clock64() - t0) / 32;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) keep ^= a[k];
+        }
+        for (int mode = 0; mode < 2; ++mode) {
+            unsigned a = threadIdx.x, b = seed | 1u;
+            const long long t0 = clock64();
+            for (int i = 0; i < iters; ++i)
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const unsigned f = *(volatile unsigned *)&s[(zeros[0] + (unsigned)(i + j)) & 1023u] >> 12;    // always 0
+                    a = max(a, b) - b;
+                    a += (unsigned)j;
+                    a ^= 5u;
+                    a += b;
+                    if (mode == 0 && (f & 1u)) a = emo_cost_rare(a);
+                    asm volatile("" : "+r"(a));
+                }
+            t[4 + mode] = (clock64() - t0) / 8;
+            keep ^= a;
+        }
+        {
+            unsigned a = threadIdx.x;
+            const long long t0 = clock64();
+            for (int i = 0; i < iters; ++i)
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    asm volatile("redux.sync.or.b32 %0, %0, 0xffffffff;" : "+r"(a));
+                    asm volatile("add.u32 %0, %0, 1;" : "+r"(a));
+                }
+            t[6] = (clock64() - t0) / 8;
+            keep ^= a;
+        }
+    }
+    {
+        __syncthreads();
+        const long long t0 = clock64();
+        for (int i = 0; i < iters; ++i) asm volatile("bar.sync 1, %0;" ::"r"(blockDim.x) : "memory");
+        t[7] = clock64() - t0;
+    }
+    if (threadIdx.x == 0) {
+        for (int k = 0; k < 8; ++k) out[k] = t[k];
+        if (keep == 0x12345u) out[8] = keep;      // keeps the chains alive, (almost) never true
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // Integer issue rate: eight independent dependent-chains per thread of one operation (OP 0: 32-bit
 // add, 1: 32-bit max, 2: 64-bit add, 3: 64-bit max), enough warps to fill every SM.  The operations
 // are volatile so that the compiler keeps every one of them.  Gives the denominator for "integer

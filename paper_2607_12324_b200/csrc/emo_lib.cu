@@ -811,6 +811,23 @@ int emo_measure_int_issue(double *ops_per_s, void *scratch_dev, void *stream)
     return rc;
 }
 
+int emo_measure_warp_costs(double *cycles, void *scratch_dev, void *stream)
+{
+    if (!cycles || !scratch_dev) return EMO_E_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    long long *out = (long long *)scratch_dev;                 // 9 results, then one zero word the kernel reads
+    const int iters = 512;
+    if (cudaMemsetAsync(scratch_dev, 0, 128, st) != cudaSuccess) return EMO_E_CUDA;
+    long long h[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    for (int rep = 0; rep < 2; ++rep) {                        // the first repetition warms up
+        emo_warp_costs<<<1, 160, 0, st>>>(out, (const unsigned *)(out + 12), iters, 12345u);
+        if (cudaMemcpyAsync(h, out, sizeof(h), cudaMemcpyDeviceToHost, st) != cudaSuccess) return EMO_E_CUDA;
+        if (cudaStreamSynchronize(st) != cudaSuccess || cudaGetLastError() != cudaSuccess) return EMO_E_CUDA;
+    }
+    for (int k = 0; k < 8; ++k) cycles[k] = (double)h[k] / iters;
+    return EMO_OK;
+}
+
 int emo_set_flow_counters(void *dev)
 {
     g_flow_prof = (long long *)dev;

@@ -30,7 +30,7 @@ EXPORTS = [
     "emo_strerror", "emo_graph_load", "emo_graph_free", "emo_graph_info", "emo_workspace_bytes",
     "emo_eval_policies", "emo_slack_batch", "emo_slack", "emo_baseline", "emo_target_from_delta",
     "emo_select", "emo_transpose_policies", "emo_slack_batch_host", "emo_graph_program",
-    "emo_set_pass_events", "emo_select_static", "emo_graph_flow", "emo_set_wait_limit", "emo_call_path", "emo_set_flow_counters", "emo_workspace_bytes_for", "emo_measure_int_issue", "emo_pack_levels", "emo_unpack_levels", "emo_slack_batch_host_packed",
+    "emo_set_pass_events", "emo_select_static", "emo_graph_flow", "emo_set_wait_limit", "emo_call_path", "emo_set_flow_counters", "emo_workspace_bytes_for", "emo_measure_int_issue", "emo_measure_warp_costs", "emo_pack_levels", "emo_unpack_levels", "emo_slack_batch_host_packed",
 ]
 
 
@@ -110,6 +110,7 @@ def lib():
         L.emo_set_wait_limit.argtypes = [i64]
         L.emo_set_flow_counters.argtypes = [p]
         L.emo_measure_int_issue.argtypes = [p, p, p]
+        L.emo_measure_warp_costs.argtypes = [p, p, p]
         L.emo_pack_levels.argtypes = [ctypes.c_int, i64, i64, p, i64, p, i64, p]
         L.emo_unpack_levels.argtypes = [ctypes.c_int, i64, i64, p, i64, p, i64, p]
         L.emo_slack_batch_host_packed.argtypes = [p, i64, ctypes.c_int, p, i64, p, p, i64, p, i64, i64, p, p, p, p, p, p, sz, u32, p]
@@ -361,6 +362,16 @@ def emo_measure_int_issue(scratch_dev, stream=None) -> dict:
     _check(lib().emo_measure_int_issue(ctypes.cast(out, ctypes.c_void_p), _addr(scratch_dev), _stream(stream)),
            "emo_measure_int_issue")
     return {"add32": out[0], "max32": out[1], "add64": out[2], "max64": out[3]}
+
+
+def emo_measure_warp_costs(scratch_dev, stream=None) -> dict:
+    """Cycles one warp alone pays for the steps of the pass kernels (see include/emo.h)."""
+    out = (ctypes.c_double * 8)()
+    _check(lib().emo_measure_warp_costs(ctypes.cast(out, ctypes.c_void_p), _addr(scratch_dev), _stream(stream)),
+           "emo_measure_warp_costs")
+    names = ("add_dependent", "max_sub_dependent", "shared_load_dependent", "add_independent", "body_with_untaken_branch",
+             "body_without_branch", "redux_add_dependent", "barrier_5_warps")
+    return {k: out[i] for i, k in enumerate(names)}
 
 
 def emo_pack_levels(bits, rows, B, lvl, ldb, packed, ldp, stream=None):

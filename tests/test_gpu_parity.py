@@ -572,3 +572,18 @@ def test_bounded_waits_report_timeout(torch_cuda, emo, oracle_mod):
     r = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, flags=emo.EMO_F_FLOW_KERNEL, base=True)
     assert_matches(r, r_or, B)
     h.free()
+
+
+@pytest.mark.gpu
+def test_measurement_helpers(torch_cuda, emo):
+    """The two measurement helpers run and give plausible figures (they feed the bounds bench.py prints)."""
+    torch = torch_cuda
+    scratch = torch.zeros(32, dtype=torch.int64, device="cuda")
+    ipk = emo.emo_measure_int_issue(scratch)
+    assert all(1e10 < v < 1e13 for v in ipk.values()), ipk
+    c = emo.emo_measure_warp_costs(scratch)
+    assert 1.0 <= c["add_dependent"] <= 12.0
+    assert c["add_independent"] <= c["add_dependent"]
+    assert 10.0 <= c["shared_load_dependent"] <= 80.0
+    assert c["body_without_branch"] <= c["body_with_untaken_branch"]
+    assert 5.0 <= c["barrier_5_warps"] <= 400.0
