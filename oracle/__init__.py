@@ -57,6 +57,8 @@ def lib():
         L.emo_oracle_target.restype = i64
         L.emo_oracle_select.argtypes = [i64, p, p, i64]
         L.emo_oracle_select.restype = i64
+        L.emo_oracle_intervals.argtypes = [i32, p, p, i32, p, p, p, i32, i32, p, p, i64, i64, i64, p, p, p, p, p, i64]
+        L.emo_oracle_intervals.restype = ctypes.c_int
         _lib = L
     return _lib
 
@@ -172,3 +174,29 @@ def select(makespan, energy, target: int) -> int:
     makespan = _c(makespan, np.int64)
     energy = _c(energy, np.float64)
     return int(lib().emo_oracle_select(makespan.shape[0], _ptr(makespan), _ptr(energy), int(target)))
+
+
+def intervals(g, dev_of, breaks, F, p_idle=None, b0: int = 0, b1: Optional[int] = None, want_levels: bool = False):
+    """Alg. 1 with time-interval policies.  F: uint8 [D][I][B]; breaks: int64 [I] change points (breaks[0] = 0).
+    Returns a dict with makespan, e_active, e_idle, energy (their sum) and, if asked, levels [n][b1 - b0]."""
+    F = _c(F, np.uint8)
+    D, I, B = F.shape
+    b1 = B if b1 is None else b1
+    dev_of = _c(dev_of, np.int32)
+    breaks = _c(breaks, np.int64)
+    row_ptr, col = _c(g.row_ptr, np.int64), _c(g.col, np.int32)
+    lat, energy = _c(g.lat, np.int64), _c(g.energy, np.float64)
+    pi = None if p_idle is None else _c(p_idle, np.float64)
+    T = np.zeros(B, np.int64)
+    ea = np.zeros(B, np.float64)
+    ei = np.zeros(B, np.float64)
+    lv = np.zeros((g.n, max(b1 - b0, 1)), np.uint8) if want_levels else None
+    rc = lib().emo_oracle_intervals(g.n, _ptr(row_ptr), _ptr(col), g.L, _ptr(lat), _ptr(energy), _ptr(dev_of), D, I,
+                                    _ptr(breaks), _ptr(F), B, b0, b1, _ptr(pi), _ptr(T), _ptr(ea), _ptr(ei),
+                                    _ptr(lv), lv.shape[1] if lv is not None else 0)
+    if rc:
+        raise OracleError(f"emo_oracle_intervals failed with {rc}")
+    out = {"makespan": T[b0:b1], "e_active": ea[b0:b1], "e_idle": ei[b0:b1], "energy": (ea + ei)[b0:b1]}
+    if want_levels:
+        out["levels"] = lv
+    return out

@@ -20,6 +20,8 @@
  *                                              the budget is a fraction of it (2 %, 5 % in Sec. 5)
  *   selection ................................ Eq. 4 over a finite candidate set, with the feasibility
  *                                              and strict-improvement test of Alg. 2 (first best kept)
+ *   time-interval policies and idle energy ... Alg. 1 as printed (level from the interval that holds the
+ *                                              start time, critical-predecessor tracking, E_a and E_i), Eq. 2
  *
  * Readings where the paper is silent: a node without predecessors starts at 0; edges carry no lag;
  * the maximum in Eq. 2 runs over all nodes; energies are summed in node order with Neumaier
@@ -241,4 +243,121 @@ int64_t emo_oracle_select(int64_t B, const int64_t *makespan, const double *ener
         if (makespan[b] <= target && (best < 0 || energy[b] < energy[best])) best = b;
     }
     return best;
+}
+
+/* ------------------------------------------------------------------------------------------------
+ * Alg. 1 with a time-interval policy P = {<T_i, F_i>}: the frequency of a pack is the one of the
+ * interval that holds its START time (Alg. 1: "f <- F_i where start in [T_i, T_{i+1})"; Eq. 4's
+ * side condition puts max over predecessors of C_k in the interval), plus the idle energy of Eq. 2.
+ * The steps are taken in the algorithm's order and notation: comp[], the critical predecessor
+ * pred[] updated from every finished node to its successors, start = comp[pred[v]], E_a, E_i.
+ *
+ * Inputs beyond the per-node-level routines:
+ *   dev_of[n]   device whose policy governs node v (each GPU has its own policy, Sec. 4.3);
+ *               -1 = not a pack: the policy does not touch it, dur = lat[v][0], e = energy[v][0]
+ *               (the tables hold the fixed t_v and the zero energy that Alg. 1 gives such nodes)
+ *   breaks[I]   the change points T_1 < T_2 < ... (nanoseconds), breaks[0] = 0; the last interval
+ *               has no end
+ *   F           levels, [D][I][ldb]: device d, interval i, policy b at F[(d*I + i)*ldb + b]
+ *   p_idle[L]   idle power at each level in watts (NULL: no idle energy)
+ *
+ * Readings where the paper is silent: idle_time of an interval, per device, is the interval's
+ * length inside [0, T) minus the summed overlap of that device's packs with it, not below zero
+ * (packs of several streams can overlap); the last interval ends at T; a pack that starts at or
+ * after the last change point uses the last level; E_i sums devices, then intervals, in order,
+ * compensated like E_a.
+ *
+ * Outputs (each may be NULL): makespan[b], e_active[b], e_idle[b]; level_out[v*ldo + (b - b0)] =
+ * the level the policy gave node v (0 for a node outside every policy).
+ * ------------------------------------------------------------------------------------------------ */
+int emo_oracle_intervals(int32_t n, const int64_t *row_ptr, const int32_t *col, int32_t L,
+                         const int64_t *lat, const double *energy, const int32_t *dev_of, int32_t D,
+                         int32_t I, const int64_t *breaks, const uint8_t *F, int64_t ldb,
+                         int64_t b0, int64_t b1, const double *p_idle,
+                         int64_t *makespan, double *e_active, double *e_idle,
+                         uint8_t *level_out, int64_t ldo)
+{
+    if (n < 0 || L < 1 || D < 1 || I < 1 || b0 < 0 || b1 < b0 || !breaks || breaks[0] != 0) return ORACLE_E_ARG;
+    for (int32_t i = 1; i < I; ++i)
+        if (breaks[i] <= breaks[i - 1]) return ORACLE_E_ARG;
+    size_t nn = (size_t)(n > 0 ? n : 1);
+    int64_t m = n > 0 ? row_ptr[n] : 0;
+    int32_t *order = malloc(sizeof *order * nn), *pred = malloc(sizeof *pred * nn);
+    int64_t *comp = malloc(sizeof *comp * nn), *start_of = malloc(sizeof *start_of * nn);
+    int64_t *succ_ptr = calloc(nn + 1, sizeof *succ_ptr);
+    int32_t *succ = malloc(sizeof *succ * (size_t)(m > 0 ? m : 1));
+    double *e = malloc(sizeof *e * nn), *ei = malloc(sizeof *ei * (size_t)D * (size_t)I);
+    int rc = ORACLE_OK;
+    if (!order || !pred || !comp || !start_of || !succ_ptr || !succ || !e || !ei) { rc = ORACLE_E_NOMEM; goto done; }
+    rc = emo_oracle_topo(n, row_ptr, col, order);
+    if (rc) goto done;
+    /* successor lists from the predecessor CSR */
+    for (int32_t v = 0; v < n; ++v)
+        for (int64_t k = row_ptr[v]; k < row_ptr[v + 1]; ++k) succ_ptr[col[k] + 1]++;
+    for (int32_t v = 0; v < n; ++v) succ_ptr[v + 1] += succ_ptr[v];
+    {
+        int64_t *fill = malloc(sizeof *fill * nn);
+        if (!fill) { rc = ORACLE_E_NOMEM; goto done; }
+        memcpy(fill, succ_ptr, sizeof *fill * nn);
+        for (int32_t v = 0; v < n; ++v)
+            for (int64_t k = row_ptr[v]; k < row_ptr[v + 1]; ++k) succ[fill[col[k]]++] = v;
+        free(fill);
+    }
+    for (int32_t v = 0; v < n; ++v)
+        if (dev_of[v] >= D) { rc = ORACLE_E_RANGE; goto done; }
+
+    for (int64_t b = b0; b < b1; ++b) {
+        for (int32_t v = 0; v < n; ++v) { comp[v] = 0; pred[v] = -1; }
+        for (int32_t k = 0; k < n; ++k) {
+            int32_t v = order[k];
+            int64_t start = pred[v] >= 0 ? comp[pred[v]] : 0;
+            int64_t dur;
+            int32_t f = 0;
+            if (dev_of[v] >= 0) {
+                /* f <- F_i where start in [T_i, T_{i+1}) */
+                int32_t i = 0;
+                while (i + 1 < I && breaks[i + 1] <= start) ++i;
+                f = F[((int64_t)dev_of[v] * I + i) * ldb + b];
+                if (f >= L) { rc = ORACLE_E_RANGE; goto done; }
+            }
+            dur = lat[(int64_t)v * L + f];
+            e[v] = energy[(int64_t)v * L + f];
+            start_of[v] = start;
+            comp[v] = start + dur;
+            if (level_out) level_out[(int64_t)v * ldo + (b - b0)] = (uint8_t)f;
+            for (int64_t s = succ_ptr[v]; s < succ_ptr[v + 1]; ++s) {
+                int32_t u = succ[s];
+                if (pred[u] < 0 || comp[v] > comp[pred[u]]) pred[u] = v;
+            }
+        }
+        int64_t T = 0;
+        for (int32_t v = 0; v < n; ++v)
+            if (comp[v] > T) T = comp[v];
+        /* E_i <- E_i + idle_time of [T_i, T_{i+1}) x p_idle[F_i], per device */
+        double Ei = 0.0;
+        if (p_idle) {
+            for (int32_t d = 0; d < D; ++d)
+                for (int32_t i = 0; i < I; ++i) {
+                    int64_t lo = breaks[i], hi = (i + 1 < I) ? breaks[i + 1] : T;
+                    if (hi > T) hi = T;
+                    int64_t len = hi > lo ? hi - lo : 0;
+                    int64_t busy = 0;
+                    for (int32_t v = 0; v < n; ++v) {
+                        if (dev_of[v] != d) continue;
+                        int64_t a = start_of[v] > lo ? start_of[v] : lo;
+                        int64_t z = comp[v] < hi ? comp[v] : hi;
+                        if (z > a) busy += z - a;
+                    }
+                    int64_t idle = len > busy ? len - busy : 0;
+                    ei[(size_t)d * I + i] = (double)idle * 1e-9 * p_idle[F[((int64_t)d * I + i) * ldb + b]];
+                }
+            Ei = emo_oracle_energy(D * I, ei);
+        }
+        if (makespan) makespan[b] = T;
+        if (e_active) e_active[b] = emo_oracle_energy(n, e);
+        if (e_idle) e_idle[b] = Ei;
+    }
+done:
+    free(order); free(pred); free(comp); free(start_of); free(succ_ptr); free(succ); free(e); free(ei);
+    return rc;
 }
