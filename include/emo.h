@@ -149,6 +149,36 @@ int emo_eval_policies(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t
                       void *ws, size_t ws_bytes, int32_t *status, uint32_t flags, void *stream);
 
 /*
+ * emo_eval_intervals - Alg. 1 with time-interval policies P = {<T_i, F_i>} and the idle energy of Eq. 2,
+ * for B policies at once.  The level of a node is the one of the interval that holds its START time
+ * (Alg. 1: "f <- F_i where start in [T_i, T_{i+1})"; half-open, the last interval has no end), so a node's
+ * duration depends on the recurrence of Eq. 1 itself.  Each device has its own policy (Sec. 4.3): the graph's
+ * group_of (emo_graph_load) names the device row of every pack; a node with group_of = -1 is outside every
+ * policy and uses column 0 of its tables (the fixed t_v and the zero energy Alg. 1 gives such nodes).
+ *   F            device uint8 [rows][I][ldb]: row r, interval i, policy b at F[(r*I + i)*ldb + b]; ldb >= B;
+ *                levels must be < L (a larger value is masked into the table, never read out of bounds).
+ *   I, breaks    number of intervals (1..4096) and their change points T_1 < T_2 < ..., HOST int64 [I] in
+ *                nanoseconds with breaks[0] = 0; the same for every policy of the batch.  Copied by the call.
+ *   p_idle       device fp64 [L], idle power in watts at each level, or NULL (no idle energy).
+ *   makespan     device int64 [B]: max_v C_v (Eq. 2).
+ *   energy       device fp64 [B]: sum_v e_v + E_idle (Eq. 2; E_idle = 0 without p_idle).
+ *   energy_idle  device fp64 [B], optional: E_idle alone.  Requires p_idle.
+ *   ws           device scratch of at least emo_workspace_bytes_intervals(g, B, I, p_idle != NULL).
+ * E_idle (Alg. 1, last loop) = sum over rows and intervals of idle_time x p_idle[F_i], where idle_time is the
+ * part of the interval below the makespan minus the summed overlap of the row's packs with it, not below zero
+ * (exact when the packs of a device do not overlap in time, as packs of one device timeline do not; the paper
+ * does not define idle_time further).
+ * Errors: EMO_E_INVALID_ARG (sizes, breaks not increasing from 0, energy_idle without p_idle), EMO_E_OOM
+ * (workspace too small), EMO_E_UNSUPPORTED (change points and exchange slots do not fit shared memory).
+ * Asynchronous on `stream` after the change points are copied.
+ */
+int emo_eval_intervals(const emo_graph *g, int64_t B, const uint8_t *F, int64_t ldb, int32_t I,
+                       const int64_t *breaks, const double *p_idle, int64_t *makespan, double *energy,
+                       double *energy_idle, void *ws, size_t ws_bytes, int32_t *status, uint32_t flags,
+                       void *stream);
+int emo_workspace_bytes_intervals(const emo_graph *g, int64_t B, int32_t I, int with_idle, size_t *out);
+
+/*
  * emo_slack_batch - forward and backward pass for B policies: earliest start ES, latest start LS
  * (critical-path backward pass: LF_v = min over successors of LS_u, the makespan for nodes
  * without successors; LS_v = LF_v - t_v) and slack = LS - ES per node and policy.

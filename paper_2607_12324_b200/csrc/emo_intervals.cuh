@@ -1,0 +1,137 @@
+// Time-interval policies (Alg. 1): the level of a pack is the one of the interval that holds its start
+// time, so the look-up depends on the recurrence and cannot be staged ahead of it.  Included only by
+// emo_lib.cu.
+#pragma once
+#include "emo_kernels.cuh"
+
+struct IntervalParams {
+    PassParams p;              // the forward step program, the batch size, makespan / energy outputs (lvl unused)
+    const uint8_t *F;          // [rows][I][ldb] levels
+    int64_t ldb;
+    int I;
+    const int64_t *breaks;     // device, [I] change points, breaks[0] = 0
+    double inv_mean;           // I / (breaks[I-1] + 1): first guess of the interval index
+    unsigned long long *busy;  // [rows][I][ldw] summed overlap of the row's packs with each interval (NULL: not wanted)
+    int64_t ldw;
+    unsigned slot_bytes;       // shared memory: slots and partial sums first, the change points after them
+};
+
+// Forward pass of Eq. 1 with the level of every pack taken from its start time.  One warp = 32 policies of
+// one schedule lane; `lanes` warps form a group and meet at a named barrier after every step (the layout of
+// emo_pass_plain).  Where busy is given, every pack adds its overlap with each interval it touches
+// (integer atomics: the lanes of a group work on the same policies).
+__global__ void __launch_bounds__(1024) emo_pass_intervals(IntervalParams ip)
+{
+    extern __shared__ __align__(128) unsigned char emo_smem[];
+    const PassParams &p = ip.p;
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const int group = warp / p.lanes;
+    const int chain = warp - group * p.lanes;
+    const int64_t b = ((int64_t)blockIdx.x * p.groups + group) * 32 + lane;
+    const bool active = b < p.B;
+    long long *slots = reinterpret_cast<long long *>(emo_smem) + (size_t)group * p.slots * 32 + lane;
+    unsigned char *part_base = emo_smem + (size_t)p.groups * p.slots * 256;
+    long long *brk = reinterpret_cast<long long *>(emo_smem + ip.slot_bytes);
+    const int I = ip.I;
+    for (int i = threadIdx.x; i < I; i += blockDim.x) brk[i] = ip.breaks[i];
+    __syncthreads();
+
+    long long h = 0;
+    double eacc = 0.0;
+    long long tmax = 0;
+    for (int t = 0; t < p.steps; ++t) {
+        const size_t q = (size_t)t * p.lanes + chain;
+        const unsigned char *r = p.rec + q * p.rec_bytes;
+        uint4 e = __ldg(reinterpret_cast<const uint4 *>(r));
+        if (e.y & emo::kValid) {
+            long long start = (e.y & emo::kRegPred) ? h : 0;
+            const int np = (e.y >> emo::kNPredShift) & 7;
+            unsigned long long ops = (unsigned long long)e.z | ((unsigned long long)e.w << 32);
+            for (int k = 0; k < np; ++k) {
+                long long x = slots[(unsigned)(ops & 255u) * 32];
+                ops >>= 8;
+                start = x > start ? x : start;
+            }
+            // f <- F_i where start in [T_i, T_{i+1})
+            unsigned lv = 0;
+            const uint32_t row = __ldg(p.rows + q);
+            int i = 0;
+            if (row != emo::kNone) {
+                i = (int)((double)start * ip.inv_mean);
+                i = i < 0 ? 0 : (i > I - 1 ? I - 1 : i);
+                while (i + 1 < I && brk[i + 1] <= start) ++i;
+                while (i > 0 && brk[i] > start) --i;
+                if (active) lv = ip.F[((size_t)row * I + i) * ip.ldb + b];
+            }
+            lv &= (e.y >> emo::kMaskShift) & 255u;
+            const long long dur = (long long)__ldg(reinterpret_cast<const uint32_t *>(r + 32) + lv);
+            h = start + dur;
+            eacc += __ldg(reinterpret_cast<const double *>(r + 32 + p.Lp * 4) + lv);
+            if (e.y & emo::kTerminal) tmax = h > tmax ? h : tmax;
+            if (ip.busy && row != emo::kNone && active) {
+                // the pack's overlap with every interval it touches (the last one has no end)
+                long long a = start;
+                int j = i;
+                while (a < h) {
+                    const long long hi = (j + 1 < I) ? brk[j + 1] : h;
+                    const long long z = hi < h ? hi : h;
+                    atomicAdd(ip.busy + ((size_t)row * I + j) * ip.ldw + b, (unsigned long long)(z - a));
+                    a = z;
+                    ++j;
+                }
+            }
+            if (e.y & emo::kWriteSlot) slots[((e.y >> emo::kOutShift) & 255u) * 32] = h;
+        }
+        if (p.lanes > 1) emo_group_barrier(group + 1, p.lanes * 32);
+    }
+
+    // combine the warps of a group in lane order (fixed order: run-to-run identical energy)
+    double *pd = reinterpret_cast<double *>(part_base) + ((size_t)(group * p.lanes + chain) * 32 + lane) * 2;
+    pd[0] = eacc;
+    reinterpret_cast<long long *>(pd)[1] = tmax;
+    __syncthreads();
+    if (chain == 0 && active) {
+        const double *g0 = reinterpret_cast<const double *>(part_base) + ((size_t)(group * p.lanes) * 32 + lane) * 2;
+        double es = 0.0;
+        long long tm = 0;
+        for (int k = 0; k < p.lanes; ++k) {
+            es += g0[(size_t)k * 64];
+            long long x = reinterpret_cast<const long long *>(g0)[(size_t)k * 64 + 1];
+            tm = x > tm ? x : tm;
+        }
+        p.makespan[b] = tm;
+        p.energy[b] = es;
+    }
+}
+
+// E_i of Alg. 1: for every row (device) and interval, the interval's length below the makespan minus the
+// busy time, not below zero, times the idle power of the interval's level; rows, then intervals, in order.
+// One thread per policy.  Adds the idle energy to energy[b] and, if asked, stores it alone.
+__global__ void __launch_bounds__(256) emo_idle_energy(int64_t B, int rows, int I, const int64_t *breaks, const uint8_t *F, int64_t ldb,
+                                                       const unsigned long long *busy, int64_t ldw, const double *p_idle, int L,
+                                                       const int64_t *makespan, double *energy, double *energy_idle)
+{
+    const int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    const long long T = makespan[b];
+    double sum = 0.0, comp = 0.0;      // compensated: many small terms
+    for (int r = 0; r < rows; ++r)
+        for (int i = 0; i < I; ++i) {
+            const long long lo = breaks[i];
+            long long hi = (i + 1 < I) ? breaks[i + 1] : T;
+            hi = hi < T ? hi : T;
+            const long long len = hi > lo ? hi - lo : 0;
+            const long long bz = (long long)busy[((size_t)r * I + i) * ldw + b];
+            const long long idle = len > bz ? len - bz : 0;
+            unsigned f = F[((size_t)r * I + i) * ldb + b];
+            f = f < (unsigned)L ? f : (unsigned)(L - 1);
+            const double x = (double)idle * 1e-9 * p_idle[f];
+            const double t = sum + x;
+            comp += (fabs(sum) >= fabs(x)) ? (sum - t) + x : (x - t) + sum;
+            sum = t;
+        }
+    const double ei = sum + comp;
+    if (energy_idle) energy_idle[b] = ei;
+    energy[b] += ei;
+}

@@ -15,6 +15,7 @@
 #include "emo_pass_lane.cuh"
 #include "emo_pass_staged.cuh"
 #include "emo_flow.cuh"
+#include "emo_intervals.cuh"
 
 using namespace emo;
 
@@ -1165,6 +1166,85 @@ int emo_eval_policies(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t
     if (rc) return rc;
     return launch_pass(g, pl, false, B, lvl, ldb, nullptr, 0, nullptr, nullptr, nullptr, 0, makespan, energy, nullptr,
                        nullptr, T0, E0, status, st);
+}
+
+int emo_workspace_bytes_intervals(const emo_graph *g, int64_t B, int32_t I, int with_idle, size_t *out)
+{
+    if (!g || !out || B < 0 || I < 1) return EMO_E_INVALID_ARG;
+    size_t bytes = round_up((size_t)I * 8, 256);
+    if (with_idle) bytes += (size_t)std::max(g->h.rows, 1) * (size_t)I * round_up((size_t)B, 16) * 8;
+    *out = bytes;
+    return EMO_OK;
+}
+
+int emo_eval_intervals(const emo_graph *g, int64_t B, const uint8_t *F, int64_t ldb, int32_t I, const int64_t *breaks,
+                       const double *p_idle, int64_t *makespan, double *energy, double *energy_idle, void *ws,
+                       size_t ws_bytes, int32_t *status, uint32_t flags, void *stream)
+{
+    (void)flags;
+    (void)status;
+    if (!g || B < 0 || I < 1 || I > 4096 || !breaks || breaks[0] != 0) return EMO_E_INVALID_ARG;
+    for (int32_t i = 1; i < I; ++i)
+        if (breaks[i] <= breaks[i - 1]) return EMO_E_INVALID_ARG;
+    if (g->host_only) return EMO_E_CUDA;
+    if (B == 0) return EMO_OK;
+    if (!F || !makespan || !energy || ldb < B) return EMO_E_INVALID_ARG;
+    if (energy_idle && !p_idle) return EMO_E_INVALID_ARG;
+    size_t need = 0;
+    emo_workspace_bytes_intervals(g, B, I, p_idle != nullptr, &need);
+    if (!ws || ws_bytes < need) return EMO_E_OOM;
+    cudaStream_t st = (cudaStream_t)stream;
+    const Program &p = g->fwd;
+    const DevProgram &d = g->dfwd;
+    if (p.steps == 0) return EMO_E_UNSUPPORTED;
+    LaunchShape s;
+    int rc = shape_for(g, p, B, s);
+    if (rc) return rc;
+    const size_t brk_bytes = round_up((size_t)I * 8, 16);
+    const size_t budget = g->smem_optin ? g->smem_optin : 48 * 1024;
+    if (s.smem + brk_bytes > budget) return EMO_E_UNSUPPORTED;
+    int64_t *d_breaks = (int64_t *)ws;
+    unsigned long long *busy = p_idle ? (unsigned long long *)((char *)ws + round_up((size_t)I * 8, 256)) : nullptr;
+    const int64_t ldw = (int64_t)round_up((size_t)B, 16);
+    const int rows = std::max(g->h.rows, 1);
+    EMO_CUDA(cudaMemcpyAsync(d_breaks, breaks, (size_t)I * 8, cudaMemcpyHostToDevice, st));
+    if (busy) EMO_CUDA(cudaMemsetAsync(busy, 0, (size_t)rows * (size_t)I * (size_t)ldw * 8, st));
+    IntervalParams a;
+    a.p = PassParams();
+    a.p.rec = d.rec;
+    a.p.rows = d.rows;
+    a.p.rec_bytes = d.rec_bytes;
+    a.p.steps = p.steps;
+    a.p.lanes = p.lanes;
+    a.p.Lp = p.Lp;
+    a.p.L = g->h.L;
+    a.p.slots = p.slots;
+    a.p.sync = p.sync;
+    a.p.groups = s.groups;
+    a.p.B = B;
+    a.p.makespan = makespan;
+    a.p.energy = energy;
+    a.F = F;
+    a.ldb = ldb;
+    a.I = I;
+    a.breaks = d_breaks;
+    a.inv_mean = (I > 1) ? (double)(I - 1) / (double)breaks[I - 1] : 0.0;
+    a.busy = busy;
+    a.ldw = ldw;
+    a.slot_bytes = (unsigned)s.smem;
+    const size_t smem = s.smem + brk_bytes;
+    cudaEvent_t ev0 = g_pass_events[0], ev1 = g_pass_events[1];
+    if (ev0) EMO_CUDA(cudaEventRecord(ev0, st));
+    if (smem > 48 * 1024) EMO_CUDA(cudaFuncSetAttribute(emo_pass_intervals, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    emo_pass_intervals<<<s.grid, s.threads, smem, st>>>(a);
+    EMO_CUDA(cudaGetLastError());
+    if (p_idle) {
+        emo_idle_energy<<<(unsigned)((B + 255) / 256), 256, 0, st>>>(B, rows, I, d_breaks, F, ldb, busy, ldw, p_idle, g->h.L, makespan,
+                                                                       energy, energy_idle);
+        EMO_CUDA(cudaGetLastError());
+    }
+    if (ev1) EMO_CUDA(cudaEventRecord(ev1, st));
+    return EMO_OK;
 }
 
 int emo_slack_batch(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t ldb, int64_t *ES,

@@ -30,7 +30,7 @@ EXPORTS = [
     "emo_strerror", "emo_graph_load", "emo_graph_free", "emo_graph_info", "emo_workspace_bytes",
     "emo_eval_policies", "emo_slack_batch", "emo_slack", "emo_baseline", "emo_target_from_delta",
     "emo_select", "emo_transpose_policies", "emo_slack_batch_host", "emo_graph_program",
-    "emo_set_pass_events", "emo_select_static", "emo_graph_flow", "emo_set_wait_limit", "emo_call_path", "emo_set_flow_counters", "emo_workspace_bytes_for", "emo_measure_int_issue", "emo_measure_warp_costs", "emo_pack_levels", "emo_unpack_levels", "emo_slack_batch_host_packed",
+    "emo_set_pass_events", "emo_select_static", "emo_graph_flow", "emo_set_wait_limit", "emo_call_path", "emo_set_flow_counters", "emo_workspace_bytes_for", "emo_measure_int_issue", "emo_measure_warp_costs", "emo_eval_intervals", "emo_workspace_bytes_intervals", "emo_pack_levels", "emo_unpack_levels", "emo_slack_batch_host_packed",
 ]
 
 
@@ -111,6 +111,8 @@ def lib():
         L.emo_set_flow_counters.argtypes = [p]
         L.emo_measure_int_issue.argtypes = [p, p, p]
         L.emo_measure_warp_costs.argtypes = [p, p, p]
+        L.emo_eval_intervals.argtypes = [p, i64, p, i64, i32, p, p, p, p, p, p, ctypes.c_size_t, p, u32, p]
+        L.emo_workspace_bytes_intervals.argtypes = [p, i64, i32, ctypes.c_int, p]
         L.emo_pack_levels.argtypes = [ctypes.c_int, i64, i64, p, i64, p, i64, p]
         L.emo_unpack_levels.argtypes = [ctypes.c_int, i64, i64, p, i64, p, i64, p]
         L.emo_slack_batch_host_packed.argtypes = [p, i64, ctypes.c_int, p, i64, p, p, i64, p, i64, i64, p, p, p, p, p, p, sz, u32, p]
@@ -372,6 +374,23 @@ def emo_measure_warp_costs(scratch_dev, stream=None) -> dict:
     names = ("add_dependent", "max_sub_dependent", "shared_load_dependent", "add_independent", "body_with_untaken_branch",
              "body_without_branch", "redux_add_dependent", "barrier_5_warps")
     return {k: out[i] for i, k in enumerate(names)}
+
+
+def emo_workspace_bytes_intervals(g, B, I, with_idle=True) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().emo_workspace_bytes_intervals(g.handle, int(B), int(I), int(bool(with_idle)), ctypes.byref(out)),
+           "emo_workspace_bytes_intervals")
+    return int(out.value)
+
+
+def emo_eval_intervals(g, B, F, ldb, I, breaks, p_idle, makespan, energy, energy_idle, ws, status=None, flags=0, stream=None):
+    """breaks: host int64 numpy array [I]; everything else device tensors (see include/emo.h)."""
+    brk = np.ascontiguousarray(breaks, dtype=np.int64)
+    if brk.shape != (int(I),):
+        raise ValueError("breaks must hold I change points")
+    return _check(lib().emo_eval_intervals(g.handle, int(B), _addr(F), int(ldb), int(I), brk.ctypes.data_as(ctypes.c_void_p),
+                                           _addr(p_idle), _addr(makespan), _addr(energy), _addr(energy_idle), _addr(ws),
+                                           _nbytes(ws), _addr(status), int(flags), _stream(stream)), "emo_eval_intervals")
 
 
 def emo_pack_levels(bits, rows, B, lvl, ldb, packed, ldp, stream=None):

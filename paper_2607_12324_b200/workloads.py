@@ -677,3 +677,37 @@ def policies_for(g: Graph, B: Optional[int] = None, device="cpu", ldb: Optional[
         out[r0:r1, :B] = policy_levels(g.meta["policy_seed"], g.n, g.L, B, g.meta["policy_mode"],
                                        g.meta["q_max"], rows=(r0, r1), device=device)
     return out
+
+
+# --------------------------------------------------------------------------------------
+# time-interval policies (inputs of Alg. 1 in its own form: change points and one level per interval)
+# --------------------------------------------------------------------------------------
+def device_of(g: Graph) -> np.ndarray:
+    """int32 [n]: the device timeline whose policy governs a kernel node, -1 for CPU and collective nodes
+    (their duration does not depend on the GPU frequency)."""
+    tl = np.asarray(g.meta.get("node_timeline", np.zeros(g.n, np.int64)), dtype=np.int64)
+    return np.where(g.kind == KIND_KERNEL, tl, -1).astype(np.int32)
+
+
+def interval_breaks(T_ref_ns: int, I: int) -> np.ndarray:
+    """int64 [I]: I change points on a uniform grid over [0, 1.05 * T_ref) (the paper re-assigns the frequency
+    every 20 ms; here the grid follows the workload's length)."""
+    delta = max(1, int(T_ref_ns * 1.05) // int(I))
+    return (np.arange(I, dtype=np.int64) * delta).astype(np.int64)
+
+
+def interval_policies(policy_seed: int, n_dev: int, I: int, L: int, B: int, device="cpu", ldb: Optional[int] = None):
+    """uint8 tensor [n_dev][I][ldb]: the 'mixed' recipe of policy_levels with one row per (device, interval):
+    policy 0 holds the maximum frequency everywhere, the first half lowers a few intervals, the second half is
+    uniform random.  Padding columns hold 0xFF."""
+    import torch
+    ldb = int(ldb if ldb is not None else (B + 15) // 16 * 16)
+    out = torch.full((n_dev * I, ldb), 0xFF, dtype=torch.uint8, device=device)
+    out[:, :B] = policy_levels(policy_seed + 7, n_dev * I, L, B, "mixed", 0.5, device=device)
+    return out.reshape(n_dev, I, ldb)
+
+
+def idle_power(L: int) -> np.ndarray:
+    """fp64 [L] watts: idle power at each level, rising with the frequency (synthetic: 60 W + 40 W * f / f_max)."""
+    f = 990.0 + 975.0 * np.arange(L) / max(L - 1, 1)
+    return 60.0 + 40.0 * f / 1965.0

@@ -1,0 +1,112 @@
+"""Time-interval policies on the GPU (emo_eval_intervals) against the oracle's Alg. 1: makespan bit-exact,
+active + idle energy within 1e-9 relative."""
+from __future__ import annotations
+
+import json
+import os
+
+import numpy as np
+import pytest
+
+from paper_2607_12324_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+HERE = os.path.dirname(os.path.abspath(__file__))
+
+
+@pytest.fixture(scope="module")
+def torch_cuda():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("needs a GPU")
+    return torch
+
+
+@pytest.fixture(scope="module")
+def emo():
+    from paper_2607_12324_b200 import build, emo as E
+    build.build()
+    return E
+
+
+def run_gpu(torch, emo, g, dev_of, breaks, F, p_idle, flags=0, ldb=None):
+    """F: numpy uint8 [D][I][B]."""
+    D, I, B = F.shape
+    ldb = ldb or (B + 15) // 16 * 16
+    Fd = torch.full((D, I, ldb), 0xFF, dtype=torch.uint8, device="cuda")
+    Fd[:, :, :B] = torch.from_numpy(F).cuda()
+    h = emo.load_workload(g, flags=flags, group_of=np.asarray(dev_of, np.int32))
+    T = torch.zeros(B, dtype=torch.int64, device="cuda")
+    E = torch.zeros(B, dtype=torch.float64, device="cuda")
+    Ei = torch.zeros(B, dtype=torch.float64, device="cuda") if p_idle is not None else None
+    pi = torch.from_numpy(np.asarray(p_idle, np.float64)).cuda() if p_idle is not None else None
+    ws = torch.empty(emo.emo_workspace_bytes_intervals(h, B, I, p_idle is not None), dtype=torch.uint8, device="cuda")
+    emo.emo_eval_intervals(h, B, Fd, ldb, I, np.asarray(breaks, np.int64), pi, T, E, Ei, ws)
+    torch.cuda.synchronize()
+    h.free()
+    return T.cpu().numpy(), E.cpu().numpy(), None if Ei is None else Ei.cpu().numpy()
+
+
+def check(torch, emo, oracle_mod, g, dev_of, breaks, F, p_idle, **kw):
+    T, E, Ei = run_gpu(torch, emo, g, dev_of, breaks, F, p_idle, **kw)
+    r = oracle_mod.intervals(g, dev_of, breaks, F, p_idle)
+    assert np.array_equal(T, r["makespan"])
+    assert np.allclose(E, r["energy"], rtol=1e-9, atol=0)
+    if p_idle is not None:
+        assert np.allclose(Ei, r["e_idle"], rtol=1e-9, atol=1e-30)
+
+
+def test_hand_worked_example_on_gpu(torch_cuda, emo, oracle_mod):
+    d = json.load(open(os.path.join(HERE, "golden", "hand_worked_intervals.json")))
+    g = W.tiny_graph(d["n"], d["edges"], np.asarray(d["lat"], np.int64), np.asarray(d["energy"], np.float64))
+    T, E, Ei = run_gpu(torch_cuda, emo, g, d["dev_of"], d["breaks"], np.array(d["F"], np.uint8), d["p_idle"])
+    assert T.tolist() == d["makespan"]
+    assert np.allclose(Ei, np.array(d["idle_ns_times_watts"]) * 1e-9, rtol=1e-12, atol=0)
+    assert np.allclose(E, np.array(d["e_active"]) + np.array(d["idle_ns_times_watts"]) * 1e-9, rtol=1e-12, atol=0)
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_random_dags(torch_cuda, emo, oracle_mod, seed):
+    from tests.test_oracle_intervals import _random_case
+    g, dev_of, breaks, F, p_idle = _random_case(seed, n=60, L=4, D=3, I=7, B=70)
+    check(torch_cuda, emo, oracle_mod, g, dev_of, breaks, F, p_idle)
+    check(torch_cuda, emo, oracle_mod, g, dev_of, breaks, F, None)
+    check(torch_cuda, emo, oracle_mod, g, dev_of, [0], F[:, :1, :].copy(), p_idle)          # one interval
+    check(torch_cuda, emo, oracle_mod, g, dev_of, breaks, F, p_idle, flags=emo.EMO_F_LANES(1))
+
+
+@pytest.mark.parametrize("name,scale,B,I", [("cfg0-tiny", 1.0, 64, 9), ("cfg1-train", 0.2, 200, 40), ("cfg3-8dev", 0.02, 100, 24),
+                                             ("cfg4-llm", 0.01, 96, 33)])
+def test_config_graphs(torch_cuda, emo, oracle_mod, name, scale, B, I):
+    g = W.make_graph(name, scale)
+    dev_of = W.device_of(g)
+    D = int(dev_of.max()) + 1
+    lv_max = np.full((g.n, 1), g.L - 1, np.uint8)
+    T0 = int(oracle_mod.batch(g, lv_max)["makespan"][0])
+    breaks = W.interval_breaks(T0, I)
+    F = W.interval_policies(g.meta["policy_seed"], D, I, g.L, B).numpy()[:, :, :B].copy()
+    check(torch_cuda, emo, oracle_mod, g, dev_of, breaks, F, W.idle_power(g.L))
+    # uneven change points as well
+    rs = np.random.RandomState(5)
+    br2 = np.concatenate([[0], np.sort(rs.choice(np.arange(1, int(T0 * 1.2)), size=I - 1, replace=False))]).astype(np.int64)
+    check(torch_cuda, emo, oracle_mod, g, dev_of, br2, F, W.idle_power(g.L))
+
+
+def test_argument_errors(torch_cuda, emo):
+    torch = torch_cuda
+    g = W.make_graph("cfg0-tiny", 0.2)
+    h = emo.load_workload(g, group_of=W.device_of(g))
+    B, I = 8, 3
+    F = torch.zeros((1, I, 16), dtype=torch.uint8, device="cuda")
+    T = torch.zeros(B, dtype=torch.int64, device="cuda")
+    E = torch.zeros(B, dtype=torch.float64, device="cuda")
+    ws = torch.empty(emo.emo_workspace_bytes_intervals(h, B, I, True), dtype=torch.uint8, device="cuda")
+    for bad in ([1, 2, 3], [0, 5, 5], [0, 7, 3]):
+        with pytest.raises(Exception):
+            emo.emo_eval_intervals(h, B, F, 16, I, np.array(bad, np.int64), None, T, E, None, ws)
+    with pytest.raises(Exception):      # idle output without idle power
+        emo.emo_eval_intervals(h, B, F, 16, I, np.array([0, 4, 9], np.int64), None, T, E, E, ws)
+    with pytest.raises(Exception):      # workspace too small
+        emo.emo_eval_intervals(h, B, F, 16, I, np.array([0, 4, 9], np.int64), None, T, E, None, ws[:8])
+    emo.emo_eval_intervals(h, 0, None, 0, I, np.array([0, 4, 9], np.int64), None, None, None, None, ws)      # B = 0: nothing to do
+    h.free()
