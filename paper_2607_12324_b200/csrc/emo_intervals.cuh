@@ -10,16 +10,24 @@ struct IntervalParams {
     int64_t ldb;
     int I;
     const int64_t *breaks;     // device, [I] change points, breaks[0] = 0
-    double inv_mean;           // I / (breaks[I-1] + 1): first guess of the interval index
+    float inv_mean;            // (I - 1) / breaks[I-1]: gives the first guess of the interval index
+    long long delta;           // > 0: the change points are the uniform grid i * delta
     unsigned long long *busy;  // [rows][I][ldw] summed overlap of the row's packs with each interval (NULL: not wanted)
     int64_t ldw;
-    unsigned slot_bytes;       // shared memory: slots and partial sums first, the change points after them
+    unsigned slot_bytes;       // shared memory: slots and partial sums first, the change points after them,
+    unsigned off_rec, rec_pad; // then two record buffers per warp (rec_pad bytes each),
+    unsigned off_F;            // then the block's columns of F when they fit (stage_F)
+    int stage_F, rows;
 };
 
 // Forward pass of Eq. 1 with the level of every pack taken from its start time.  One warp = 32 policies of
 // one schedule lane; `lanes` warps form a group and meet at a named barrier after every step (the layout of
-// emo_pass_plain).  Where busy is given, every pack adds its overlap with each interval it touches
-// (integer atomics: the lanes of a group work on the same policies).
+// emo_pass_plain).  The look-up chain of a step is start -> interval -> level -> duration, all of it
+// dependent, so everything it touches is brought on chip ahead of it: the change points and (when they fit)
+// the block's columns of F sit in shared memory, and every warp copies the record of its next step (entry,
+// duration row, energy row) into a buffer of its own while it works on the current one.
+// Where busy is given, every pack adds its overlap with each interval it touches (integer atomics: the lanes
+// of a group work on the same policies).
 __global__ void __launch_bounds__(1024) emo_pass_intervals(IntervalParams ip)
 {
     extern __shared__ __align__(128) unsigned char emo_smem[];
@@ -34,16 +42,49 @@ __global__ void __launch_bounds__(1024) emo_pass_intervals(IntervalParams ip)
     unsigned char *part_base = emo_smem + (size_t)p.groups * p.slots * 256;
     long long *brk = reinterpret_cast<long long *>(emo_smem + ip.slot_bytes);
     const int I = ip.I;
+    unsigned char *recbuf = emo_smem + ip.off_rec + (size_t)warp * 2 * ip.rec_pad;      // two records per warp
+    unsigned char *Fs = ip.stage_F ? emo_smem + ip.off_F : nullptr;                     // [rows * I][groups * 32]
+    const int fcols = p.groups * 32;
     for (int i = threadIdx.x; i < I; i += blockDim.x) brk[i] = ip.breaks[i];
+    if (Fs) {
+        const int64_t b0 = (int64_t)blockIdx.x * fcols;
+        const int total = ip.rows * I * fcols;
+        for (int k = threadIdx.x; k < total; k += blockDim.x) {
+            const int ri = k / fcols, c = k - ri * fcols;
+            Fs[k] = (b0 + c < p.B) ? ip.F[(size_t)ri * ip.ldb + b0 + c] : (unsigned char)0;
+        }
+    }
+    // The record of step t for this warp's lane, copied 16 bytes per thread.  The first 512 bytes travel through
+    // a register: requested when the step before begins, stored when it ends, so that step does not wait for
+    // them.  (A ring of asynchronous copies three steps ahead was slower: the step is bound by its own chain of
+    // dependent look-ups and branches, not by the copy.)
+    auto request = [&](int t) {
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (t < p.steps && lane * 16 < p.rec_bytes)
+            v = __ldg(reinterpret_cast<const uint4 *>(p.rec + ((size_t)t * p.lanes + chain) * p.rec_bytes) + lane);
+        return v;
+    };
+    auto deposit = [&](int t, const uint4 &v) {
+        if (t < p.steps) {
+            unsigned char *dst = recbuf + (size_t)(t & 1) * ip.rec_pad;
+            if (lane * 16 < p.rec_bytes) *reinterpret_cast<uint4 *>(dst + lane * 16) = v;
+            const unsigned char *r = p.rec + ((size_t)t * p.lanes + chain) * p.rec_bytes;
+            for (int o = 512 + lane * 16; o < p.rec_bytes; o += 512) *reinterpret_cast<uint4 *>(dst + o) = __ldg(reinterpret_cast<const uint4 *>(r + o));
+        }
+    };
+    deposit(0, request(0));
     __syncthreads();
 
     long long h = 0;
     double eacc = 0.0;
     long long tmax = 0;
+    uint32_t row_next = p.steps > 0 ? __ldg(p.rows + chain) : emo::kNone;
     for (int t = 0; t < p.steps; ++t) {
-        const size_t q = (size_t)t * p.lanes + chain;
-        const unsigned char *r = p.rec + q * p.rec_bytes;
-        uint4 e = __ldg(reinterpret_cast<const uint4 *>(r));
+        const unsigned char *r = recbuf + (size_t)(t & 1) * ip.rec_pad;
+        const uint32_t row = row_next;
+        if (t + 1 < p.steps) row_next = __ldg(p.rows + (size_t)(t + 1) * p.lanes + chain);
+        const uint4 nxt = request(t + 1);
+        const uint4 e = *reinterpret_cast<const uint4 *>(r);
         if (e.y & emo::kValid) {
             long long start = (e.y & emo::kRegPred) ? h : 0;
             const int np = (e.y >> emo::kNPredShift) & 7;
@@ -55,35 +96,57 @@ __global__ void __launch_bounds__(1024) emo_pass_intervals(IntervalParams ip)
             }
             // f <- F_i where start in [T_i, T_{i+1})
             unsigned lv = 0;
-            const uint32_t row = __ldg(p.rows + q);
             int i = 0;
+            long long iend = 0x7FFFFFFFFFFFFFFFLL;      // where the interval of the start time ends
             if (row != emo::kNone) {
-                i = (int)((double)start * ip.inv_mean);
+                // first guess from the mean interval length, one correction without a branch (exact on a uniform
+                // grid), then a search for whatever is left (uneven change points)
+                i = (int)((float)start * ip.inv_mean);
                 i = i < 0 ? 0 : (i > I - 1 ? I - 1 : i);
-                while (i + 1 < I && brk[i + 1] <= start) ++i;
-                while (i > 0 && brk[i] > start) --i;
-                if (active) lv = ip.F[((size_t)row * I + i) * ip.ldb + b];
+                if (ip.delta > 0) {
+                    const long long r = start - (long long)i * ip.delta;
+                    i += (r >= ip.delta && i + 1 < I) ? 1 : 0;
+                    i -= (r < 0) ? 1 : 0;
+                    if (i + 1 < I) iend = (long long)(i + 1) * ip.delta;
+                } else {
+                    const long long lo = brk[i], hi = brk[i + 1 < I ? i + 1 : i];
+                    i += (i + 1 < I && hi <= start) ? 1 : 0;
+                    i -= (lo > start) ? 1 : 0;
+                    while (i + 1 < I && brk[i + 1] <= start) ++i;
+                    while (i > 0 && brk[i] > start) --i;
+                    if (i + 1 < I) iend = brk[i + 1];
+                }
+                if (Fs) lv = Fs[((size_t)row * I + i) * fcols + group * 32 + lane];
+                else if (active) lv = ip.F[((size_t)row * I + i) * ip.ldb + b];
             }
             lv &= (e.y >> emo::kMaskShift) & 255u;
-            const long long dur = (long long)__ldg(reinterpret_cast<const uint32_t *>(r + 32) + lv);
+            const long long dur = (long long)*(reinterpret_cast<const uint32_t *>(r + 32) + lv);
             h = start + dur;
-            eacc += __ldg(reinterpret_cast<const double *>(r + 32 + p.Lp * 4) + lv);
+            eacc += *(reinterpret_cast<const double *>(r + 32 + p.Lp * 4) + lv);
             if (e.y & emo::kTerminal) tmax = h > tmax ? h : tmax;
             if (ip.busy && row != emo::kNone && active) {
-                // the pack's overlap with every interval it touches (the last one has no end)
-                long long a = start;
-                int j = i;
-                while (a < h) {
-                    const long long hi = (j + 1 < I) ? brk[j + 1] : h;
-                    const long long z = hi < h ? hi : h;
-                    atomicAdd(ip.busy + ((size_t)row * I + j) * ip.ldw + b, (unsigned long long)(z - a));
-                    a = z;
-                    ++j;
+                // the pack's overlap with every interval it touches (the last one has no end); nearly always one
+                unsigned long long *bz = ip.busy + ((size_t)row * I + i) * ip.ldw + b;
+                if (h <= iend) {
+                    if (dur) atomicAdd(bz, (unsigned long long)dur);
+                } else {
+                    long long a = start;
+                    int j = i;
+                    while (a < h) {
+                        const long long hi = (j + 1 < I) ? brk[j + 1] : h;
+                        const long long z = hi < h ? hi : h;
+                        atomicAdd(ip.busy + ((size_t)row * I + j) * ip.ldw + b, (unsigned long long)(z - a));
+                        a = z;
+                        ++j;
+                    }
                 }
             }
             if (e.y & emo::kWriteSlot) slots[((e.y >> emo::kOutShift) & 255u) * 32] = h;
         }
+        deposit(t + 1, nxt);
+        // the barrier also orders this warp's copy of the next record before its use
         if (p.lanes > 1) emo_group_barrier(group + 1, p.lanes * 32);
+        else __syncwarp();
     }
 
     // combine the warps of a group in lane order (fixed order: run-to-run identical energy)

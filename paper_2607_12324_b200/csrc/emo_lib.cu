@@ -1202,7 +1202,14 @@ int emo_eval_intervals(const emo_graph *g, int64_t B, const uint8_t *F, int64_t 
     if (rc) return rc;
     const size_t brk_bytes = round_up((size_t)I * 8, 16);
     const size_t budget = g->smem_optin ? g->smem_optin : 48 * 1024;
-    if (s.smem + brk_bytes > budget) return EMO_E_UNSUPPORTED;
+    if (d.rec_bytes % 16) return EMO_E_UNSUPPORTED;      // a warp copies a record 16 bytes per thread
+    const size_t rec_pad = round_up((size_t)d.rec_bytes, 16);
+    const size_t off_rec = round_up(s.smem + brk_bytes, 16);
+    const size_t off_F = off_rec + (size_t)(s.threads / 32) * 2 * rec_pad;
+    if (off_F > budget) return EMO_E_UNSUPPORTED;
+    const int rows_ = std::max(g->h.rows, 1);
+    const size_t f_bytes = (size_t)rows_ * (size_t)I * (size_t)s.groups * 32;
+    const bool stage_F = off_F + f_bytes <= budget;
     int64_t *d_breaks = (int64_t *)ws;
     unsigned long long *busy = p_idle ? (unsigned long long *)((char *)ws + round_up((size_t)I * 8, 256)) : nullptr;
     const int64_t ldw = (int64_t)round_up((size_t)B, 16);
@@ -1228,11 +1235,19 @@ int emo_eval_intervals(const emo_graph *g, int64_t B, const uint8_t *F, int64_t 
     a.ldb = ldb;
     a.I = I;
     a.breaks = d_breaks;
-    a.inv_mean = (I > 1) ? (double)(I - 1) / (double)breaks[I - 1] : 0.0;
+    a.inv_mean = (I > 1) ? (float)((double)(I - 1) / (double)breaks[I - 1]) : 0.0f;
+    a.delta = (I > 1) ? breaks[1] : 0;
+    for (int32_t i = 1; i < I && a.delta > 0; ++i)
+        if (breaks[i] != (int64_t)i * a.delta) a.delta = 0;
     a.busy = busy;
     a.ldw = ldw;
     a.slot_bytes = (unsigned)s.smem;
-    const size_t smem = s.smem + brk_bytes;
+    a.off_rec = (unsigned)off_rec;
+    a.rec_pad = (unsigned)rec_pad;
+    a.off_F = (unsigned)off_F;
+    a.stage_F = stage_F ? 1 : 0;
+    a.rows = rows_;
+    const size_t smem = off_F + (stage_F ? f_bytes : 0);
     cudaEvent_t ev0 = g_pass_events[0], ev1 = g_pass_events[1];
     if (ev0) EMO_CUDA(cudaEventRecord(ev0, st));
     if (smem > 48 * 1024) EMO_CUDA(cudaFuncSetAttribute(emo_pass_intervals, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
