@@ -155,6 +155,48 @@ def run_reference(args, rank, world):
     print(json.dumps(line), flush=True)
 
 
+def intervals_leg(args, g, B, m, T0_ns, check):
+    """Times emo_eval_intervals (device-resident inputs, CUDA events) and checks a few policies against the oracle."""
+    import numpy as np
+    import torch
+    from paper_2607_12324_b200 import emo, workloads as W
+    dev_of = W.device_of(g)
+    D = int(dev_of.max()) + 1
+    I = max(2, min(4096, int(T0_ns * 1.05 / 20e6) + 1))
+    breaks = W.interval_breaks(T0_ns, I)
+    F = W.interval_policies(g.meta["policy_seed"], D, I, g.L, B, device="cuda")
+    ldb = F.shape[2]
+    h = emo.load_workload(g, flags=args.flags, group_of=dev_of)
+    T = torch.zeros(B, dtype=torch.int64, device="cuda")
+    E = torch.zeros(B, dtype=torch.float64, device="cuda")
+    Ei = torch.zeros(B, dtype=torch.float64, device="cuda")
+    pi = torch.from_numpy(W.idle_power(g.L)).cuda()
+    ws = torch.empty(emo.emo_workspace_bytes_intervals(h, B, I, True), dtype=torch.uint8, device="cuda")
+    k = max(1, min(args.steps, 5))
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    for it in range(min(args.warmup, 3) + k):
+        if it == min(args.warmup, 3):
+            ev[0].record()
+        emo.emo_eval_intervals(h, B, F, ldb, I, breaks, pi, T, E, Ei, ws)
+    ev[1].record()
+    torch.cuda.synchronize()
+    ms = ev[0].elapsed_time(ev[1]) / k
+    out = {"ms_per_call": ms, "value": B * m / (ms * 1e-3), "unit": UNIT, "passes": "forward", "policies_per_s": B / (ms * 1e-3),
+           "intervals": I, "devices": D, "grid_ns": int(breaks[1]), "idle_energy": True,
+           "bound": "latency of a schedule step (the level look-up depends on the recurrence); no HBM or tensor roofline applies"}
+    if check:
+        nb = 8
+        cols = np.linspace(0, B - 1, nb).astype(np.int64)
+        Fh = F[:, :, torch.as_tensor(cols, device="cuda")].contiguous().cpu().numpy()
+        import oracle      # the CPU oracle: checks only, never on the product path
+        r = oracle.intervals(g, dev_of, breaks, Fh, W.idle_power(g.L))
+        bad = int((T.cpu().numpy()[cols] != r["makespan"]).sum()) + int((~np.isclose(E.cpu().numpy()[cols], r["energy"], rtol=1e-9, atol=0)).sum())
+        out["checked"] = {"policies": nb, "mismatches": bad}
+        assert bad == 0, "interval evaluation disagrees with the oracle"
+    h.free()
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -169,6 +211,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--flags", type=int, default=0, help="extra EMO_F_* load flags (lanes / look-ahead)")
     ap.add_argument("--call-flags", type=int, default=0, help="EMO_F_* flags of the pass calls (kernel choice)")
+    ap.add_argument("--no-intervals", action="store_true", help="skip the time-interval policy leg (Alg. 1 in its own form)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -356,6 +399,11 @@ def main():
                        "h2d_bytes_per_step": int(g.n * ldp), "d2h_bytes_per_step": int(B * (28 if args.sums else 16) + 80),
                        "note": f"levels cross the bus packed at {bits} bits each; the slack matrix stays on the device"}
         del lv_host, dev_packed, dev_lvl
+
+    # the next row of the path: Alg. 1 with time-interval policies (20 ms grid as in the paper's experiments) and
+    # idle energy, on the same graph and batch size; a separate figure, not part of `value`
+    if rank == 0 and not args.no_intervals:
+        line["intervals"] = intervals_leg(args, g, B, m, T0_ns=int(T0.item()), check=not args.no_cpu)
 
     if rank == 0 and not args.no_cpu:
         threads = os.cpu_count() or 1
