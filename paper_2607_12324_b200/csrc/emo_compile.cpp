@@ -435,6 +435,7 @@ int compile_program(const HostGraph &g, const int64_t *lat, const double *energy
     const size_t Q = (size_t)S * lanes;
     out.entries.assign(Q * kEntryWords, 0);
     out.rows.assign(Q, kNone);
+    out.groups.assign(Q, kNone);
     out.pos_of_node.assign((size_t)std::max(n, 1), kNone);
     out.lat.assign(Q * Lp, 0);
     if (!backward) out.energy.assign(Q * Lp, 0.0);
@@ -446,6 +447,7 @@ int compile_program(const HostGraph &g, const int64_t *lat, const double *energy
             en[0] = kNone;
             en[4] = kNone;
             out.rows[q] = kNone;
+            out.groups[q] = kNone;
             if (i < 0) continue;
             const Op &o = ops[i];
             uint32_t flags = kValid;
@@ -480,6 +482,7 @@ int compile_program(const HostGraph &g, const int64_t *lat, const double *energy
                 bool constant = true;
                 for (int l = 1; l < L && constant; ++l)
                     constant = lat[(size_t)v * L + l] == lat[(size_t)v * L] && energy[(size_t)v * L + l] == energy[(size_t)v * L];
+                if (g.group[v] >= 0) out.groups[q] = (uint32_t)g.group[v];
                 if (g.group[v] >= 0 && !constant) {
                     out.rows[q] = (uint32_t)g.group[v];
                     flags |= (uint32_t)(Lp - 1) << kMaskShift;

@@ -46,6 +46,8 @@ struct Program {
     std::vector<uint32_t> entries;    // [steps][lanes][kEntryWords], see above
     std::vector<uint32_t> pos_of_node;   // [n] index (step*lanes + lane) of the entry that handles node v
     std::vector<uint32_t> rows;       // [steps][lanes] policy row whose level the entry reads (kNone: none)
+    std::vector<uint32_t> groups;     // [steps][lanes] the node's group (its device, for time-interval policies) whether or not its
+                                      // tables depend on the level; kNone: outside every policy
     std::vector<uint32_t> lat;        // [steps*lanes][Lp] durations of the scheduled node per level
     std::vector<double> energy;       // [steps*lanes][Lp], forward program only
 };

@@ -15,7 +15,7 @@ struct IntervalParams {
     unsigned long long *busy;  // [rows][I][ldw] summed overlap of the row's packs with each interval (NULL: not wanted)
     int64_t ldw;
     unsigned slot_bytes;       // shared memory: slots and partial sums first, the change points after them,
-    unsigned off_rec, rec_pad; // then two record buffers per warp (rec_pad bytes each),
+    unsigned off_rec, rec_pad; // then four record buffers per warp (rec_pad bytes each: the record, then its group),
     unsigned off_F;            // then the block's columns of F when they fit (stage_F)
     int stage_F, rows;
 };
@@ -28,6 +28,7 @@ struct IntervalParams {
 // duration row, energy row) into a buffer of its own while it works on the current one.
 // Where busy is given, every pack adds its overlap with each interval it touches (integer atomics: the lanes
 // of a group work on the same policies).
+template <bool UNIFORM, bool STAGED>
 __global__ void __launch_bounds__(1024) emo_pass_intervals(IntervalParams ip)
 {
     extern __shared__ __align__(128) unsigned char emo_smem[];
@@ -42,7 +43,7 @@ __global__ void __launch_bounds__(1024) emo_pass_intervals(IntervalParams ip)
     unsigned char *part_base = emo_smem + (size_t)p.groups * p.slots * 256;
     long long *brk = reinterpret_cast<long long *>(emo_smem + ip.slot_bytes);
     const int I = ip.I;
-    unsigned char *recbuf = emo_smem + ip.off_rec + (size_t)warp * 2 * ip.rec_pad;      // two records per warp
+    unsigned char *recbuf = emo_smem + ip.off_rec + (size_t)warp * 4 * ip.rec_pad;      // four records per warp
     unsigned char *Fs = ip.stage_F ? emo_smem + ip.off_F : nullptr;                     // [rows * I][groups * 32]
     const int fcols = p.groups * 32;
     for (int i = threadIdx.x; i < I; i += blockDim.x) brk[i] = ip.breaks[i];
@@ -54,97 +55,80 @@ __global__ void __launch_bounds__(1024) emo_pass_intervals(IntervalParams ip)
             Fs[k] = (b0 + c < p.B) ? ip.F[(size_t)ri * ip.ldb + b0 + c] : (unsigned char)0;
         }
     }
-    // The record of step t for this warp's lane, copied 16 bytes per thread.  The first 512 bytes travel through
-    // a register: requested when the step before begins, stored when it ends, so that step does not wait for
-    // them.  (A ring of asynchronous copies three steps ahead was slower: the step is bound by its own chain of
-    // dependent look-ups and branches, not by the copy.)
+    // The record of step t for this warp's lane (and the group it belongs to) is copied into a ring of four
+    // buffers three steps ahead of its use with asynchronous copies, 16 bytes per thread: a step costs less
+    // than a trip to L2, so one step ahead does not hide it.
     auto request = [&](int t) {
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (t < p.steps && lane * 16 < p.rec_bytes)
-            v = __ldg(reinterpret_cast<const uint4 *>(p.rec + ((size_t)t * p.lanes + chain) * p.rec_bytes) + lane);
-        return v;
-    };
-    auto deposit = [&](int t, const uint4 &v) {
         if (t < p.steps) {
-            unsigned char *dst = recbuf + (size_t)(t & 1) * ip.rec_pad;
-            if (lane * 16 < p.rec_bytes) *reinterpret_cast<uint4 *>(dst + lane * 16) = v;
-            const unsigned char *r = p.rec + ((size_t)t * p.lanes + chain) * p.rec_bytes;
-            for (int o = 512 + lane * 16; o < p.rec_bytes; o += 512) *reinterpret_cast<uint4 *>(dst + o) = __ldg(reinterpret_cast<const uint4 *>(r + o));
+            const size_t q = (size_t)t * p.lanes + chain;
+            const unsigned char *r = p.rec + q * p.rec_bytes;
+            unsigned char *dst = recbuf + (size_t)(t & 3) * ip.rec_pad;
+            for (int o = lane * 16; o < p.rec_bytes; o += 512)
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(emo_smem_addr(dst + o)), "l"(r + o) : "memory");
+            if (lane == 0)
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(emo_smem_addr(dst + ip.rec_pad - 16)), "l"(p.rows + q) : "memory");
         }
+        asm volatile("cp.async.commit_group;" ::: "memory");
     };
-    deposit(0, request(0));
+    request(0);
+    request(1);
+    request(2);
+    asm volatile("cp.async.wait_group 2;" ::: "memory");
     __syncthreads();
 
     long long h = 0;
     double eacc = 0.0;
     long long tmax = 0;
-    uint32_t row_next = p.steps > 0 ? __ldg(p.rows + chain) : emo::kNone;
     for (int t = 0; t < p.steps; ++t) {
-        const unsigned char *r = recbuf + (size_t)(t & 1) * ip.rec_pad;
-        const uint32_t row = row_next;
-        if (t + 1 < p.steps) row_next = __ldg(p.rows + (size_t)(t + 1) * p.lanes + chain);
-        const uint4 nxt = request(t + 1);
+        const unsigned char *r = recbuf + (size_t)(t & 3) * ip.rec_pad;
+        request(t + 3);
+        const uint32_t row = *reinterpret_cast<const uint32_t *>(r + ip.rec_pad - 16);
         const uint4 e = *reinterpret_cast<const uint4 *>(r);
-        if (e.y & emo::kValid) {
+        {
+            // One straight run of instructions for every entry, idle steps included (their record is all zero: no
+            // operands, zero duration and energy, no output; only the lane's value must survive them): a branch on
+            // a freshly loaded word costs a lone warp far more than the few predicated instructions it would skip.
+            const unsigned valid = e.y & emo::kValid;
             long long start = (e.y & emo::kRegPred) ? h : 0;
             const int np = (e.y >> emo::kNPredShift) & 7;
             unsigned long long ops = (unsigned long long)e.z | ((unsigned long long)e.w << 32);
-            for (int k = 0; k < np; ++k) {
-                long long x = slots[(unsigned)(ops & 255u) * 32];
+#pragma unroll
+            for (int k = 0; k < 3; ++k) {
+                const long long x = slots[(unsigned)(ops & 255u) * 32];      // byte 0 where there is no operand: slot 0, ignored
                 ops >>= 8;
-                start = x > start ? x : start;
+                start = (k < np && x > start) ? x : start;
             }
-            // f <- F_i where start in [T_i, T_{i+1})
-            unsigned lv = 0;
-            int i = 0;
-            long long iend = 0x7FFFFFFFFFFFFFFFLL;      // where the interval of the start time ends
-            if (row != emo::kNone) {
-                // first guess from the mean interval length, one correction without a branch (exact on a uniform
-                // grid), then a search for whatever is left (uneven change points)
-                i = (int)((float)start * ip.inv_mean);
-                i = i < 0 ? 0 : (i > I - 1 ? I - 1 : i);
-                if (ip.delta > 0) {
-                    const long long r = start - (long long)i * ip.delta;
-                    i += (r >= ip.delta && i + 1 < I) ? 1 : 0;
-                    i -= (r < 0) ? 1 : 0;
-                    if (i + 1 < I) iend = (long long)(i + 1) * ip.delta;
-                } else {
-                    const long long lo = brk[i], hi = brk[i + 1 < I ? i + 1 : i];
-                    i += (i + 1 < I && hi <= start) ? 1 : 0;
-                    i -= (lo > start) ? 1 : 0;
-                    while (i + 1 < I && brk[i + 1] <= start) ++i;
-                    while (i > 0 && brk[i] > start) --i;
-                    if (i + 1 < I) iend = brk[i + 1];
+            if (np > 3) {
+                for (int k = 3; k < np; ++k) {
+                    const long long x = slots[(unsigned)(ops & 255u) * 32];
+                    ops >>= 8;
+                    start = x > start ? x : start;
                 }
-                if (Fs) lv = Fs[((size_t)row * I + i) * fcols + group * 32 + lane];
-                else if (active) lv = ip.F[((size_t)row * I + i) * ip.ldb + b];
             }
+            // f <- F_i where start in [T_i, T_{i+1}); a node outside every policy reads row 0 and masks the level away
+            const bool pack = row != emo::kNone;
+            const unsigned rowc = pack ? row : 0u;
+            long long iend;
+            const int i = emo_interval_index<UNIFORM>(start, I, ip.delta, ip.inv_mean, brk, iend);
+            unsigned lv;
+            if (STAGED) lv = Fs[((size_t)rowc * I + i) * fcols + group * 32 + lane];
+            else lv = active ? ip.F[((size_t)rowc * I + i) * ip.ldb + b] : 0u;
             lv &= (e.y >> emo::kMaskShift) & 255u;
             const long long dur = (long long)*(reinterpret_cast<const uint32_t *>(r + 32) + lv);
-            h = start + dur;
+            const long long end = start + dur;
+            h = valid ? end : h;
             eacc += *(reinterpret_cast<const double *>(r + 32 + p.Lp * 4) + lv);
-            if (e.y & emo::kTerminal) tmax = h > tmax ? h : tmax;
-            if (ip.busy && row != emo::kNone && active) {
-                // the pack's overlap with every interval it touches (the last one has no end); nearly always one
-                unsigned long long *bz = ip.busy + ((size_t)row * I + i) * ip.ldw + b;
-                if (h <= iend) {
-                    if (dur) atomicAdd(bz, (unsigned long long)dur);
-                } else {
-                    long long a = start;
-                    int j = i;
-                    while (a < h) {
-                        const long long hi = (j + 1 < I) ? brk[j + 1] : h;
-                        const long long z = hi < h ? hi : h;
-                        atomicAdd(ip.busy + ((size_t)row * I + j) * ip.ldw + b, (unsigned long long)(z - a));
-                        a = z;
-                        ++j;
-                    }
-                }
+            tmax = ((e.y & emo::kTerminal) && end > tmax) ? end : tmax;
+            if (ip.busy) {
+                // the pack's overlap with the intervals it touches: nearly always one
+                const bool on = pack && active;
+                if (on && end <= iend && dur) atomicAdd(ip.busy + ((size_t)rowc * I + i) * ip.ldw + b, (unsigned long long)dur);
+                if (on && end > iend) emo_interval_busy(ip.busy, ip.ldw, b, rowc, I, i, iend, start, end, brk);
             }
-            if (e.y & emo::kWriteSlot) slots[((e.y >> emo::kOutShift) & 255u) * 32] = h;
+            if (e.y & emo::kWriteSlot) slots[((e.y >> emo::kOutShift) & 255u) * 32] = end;
         }
-        deposit(t + 1, nxt);
-        // the barrier also orders this warp's copy of the next record before its use
+        // the copy of the next step's record has landed; the barrier makes it visible to the whole warp
+        asm volatile("cp.async.wait_group 2;" ::: "memory");
         if (p.lanes > 1) emo_group_barrier(group + 1, p.lanes * 32);
         else __syncwarp();
     }

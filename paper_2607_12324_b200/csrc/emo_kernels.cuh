@@ -56,6 +56,51 @@ __host__ __device__ inline int64_t emo_budget(int64_t T0, int64_t ppm)
     return T0 + q * ppm + (r * ppm) / M;
 }
 
+// Alg. 1: "f <- F_i where start in [T_i, T_{i+1})".  Index of the interval that holds `start` among I change
+// points brk[0] = 0 < brk[1] < ... (the last interval has no end); iend = where that interval ends.  A first
+// guess from the mean interval length, one correction without a branch (exact on a uniform grid, delta > 0),
+// then a search for whatever is left (uneven change points).
+template <bool UNIFORM>
+__device__ __forceinline__ int emo_interval_index(long long start, int I, long long delta, float inv_mean, const long long *brk,
+                                                  long long &iend)
+{
+    int i = (int)((float)start * inv_mean);
+    i = i < 0 ? 0 : (i > I - 1 ? I - 1 : i);
+    iend = 0x7FFFFFFFFFFFFFFFLL;
+    if (UNIFORM) {
+        const long long r = start - (long long)i * delta;
+        i += (r >= delta && i + 1 < I) ? 1 : 0;
+        i -= (r < 0) ? 1 : 0;
+        if (i + 1 < I) iend = (long long)(i + 1) * delta;
+    } else {
+        const long long lo = brk[i], hi = brk[i + 1 < I ? i + 1 : i];
+        i += (i + 1 < I && hi <= start) ? 1 : 0;
+        i -= (lo > start) ? 1 : 0;
+        while (i + 1 < I && brk[i + 1] <= start) ++i;
+        while (i > 0 && brk[i] > start) --i;
+        if (i + 1 < I) iend = brk[i + 1];
+    }
+    return i;
+}
+// A pack's overlap with every interval it touches, added to busy[(row * I + i) * ldw + b]; nearly always one.
+__device__ __forceinline__ void emo_interval_busy(unsigned long long *busy, int64_t ldw, int64_t b, unsigned row, int I, int i,
+                                                  long long iend, long long start, long long end, const long long *brk)
+{
+    if (end <= iend) {
+        if (end > start) atomicAdd(busy + ((size_t)row * I + i) * ldw + b, (unsigned long long)(end - start));
+    } else {
+        long long a = start;
+        int j = i;
+        while (a < end) {
+            const long long hi = (j + 1 < I) ? brk[j + 1] : end;
+            const long long z = hi < end ? hi : end;
+            atomicAdd(busy + ((size_t)row * I + j) * ldw + b, (unsigned long long)(z - a));
+            a = z;
+            ++j;
+        }
+    }
+}
+
 __device__ __forceinline__ void emo_group_barrier(int id, int nthreads)
 {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");

@@ -22,6 +22,7 @@ using namespace emo;
 struct DevProgram {
     unsigned char *rec = nullptr;   // records: entry, duration row, (forward) energy row
     uint32_t *rows = nullptr;
+    uint32_t *groups = nullptr;     // the nodes' groups (time-interval policies)
     int rec_bytes = 0;
 };
 
@@ -102,7 +103,9 @@ int upload_program(const Program &p, DevProgram &d)
     }
     int rc = upload(&d.rec, rec.data(), rec.size());
     if (rc) return rc;
-    return upload(&d.rows, p.rows.data(), p.rows.size() * sizeof(uint32_t));
+    rc = upload(&d.rows, p.rows.data(), p.rows.size() * sizeof(uint32_t));
+    if (rc) return rc;
+    return upload(&d.groups, p.groups.data(), p.groups.size() * sizeof(uint32_t));
 }
 
 int upload_program_lane(const Program &p, DevProgramLane &d)
@@ -174,6 +177,7 @@ void free_program(DevProgram &d)
 {
     if (d.rec) cudaFree(d.rec);
     if (d.rows) cudaFree(d.rows);
+    if (d.groups) cudaFree(d.groups);
     d = DevProgram();
 }
 
@@ -455,7 +459,7 @@ int launch_pass(const emo_graph *g, const PassPlan &pl, bool backward, int64_t B
             else EMO_PICK_L(1024);
 #undef EMO_PICK_L
             ip.sp = sp;
-            EMO_CUDA(cudaFuncSetAttribute(kern_lane, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s.smem));
+            EMO_CUDA(cudaFuncSetAttribute(kern_lane, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g->smem_optin));      // the same value from every call
             kern_lane<<<s.grid, s.threads, s.smem, st>>>(ip);
         } else {
             sp.nbulk = 0;
@@ -473,14 +477,14 @@ int launch_pass(const emo_graph *g, const PassPlan &pl, bool backward, int64_t B
         else if (s.threads <= 768) EMO_PICK(768);
         else EMO_PICK(1024);
 #undef EMO_PICK
-        EMO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s.smem));
+        EMO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g->smem_optin));
         kern<<<s.grid, s.threads, s.smem, st>>>(sp);
         }
     } else if (backward) {
-        if (s.smem > 48 * 1024) EMO_CUDA(cudaFuncSetAttribute(emo_pass_plain<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s.smem));
+        if (s.smem > 48 * 1024) EMO_CUDA(cudaFuncSetAttribute(emo_pass_plain<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g->smem_optin));
         emo_pass_plain<true><<<s.grid, s.threads, s.smem, st>>>(a);
     } else {
-        if (s.smem > 48 * 1024) EMO_CUDA(cudaFuncSetAttribute(emo_pass_plain<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s.smem));
+        if (s.smem > 48 * 1024) EMO_CUDA(cudaFuncSetAttribute(emo_pass_plain<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g->smem_optin));
         emo_pass_plain<false><<<s.grid, s.threads, s.smem, st>>>(a);
     }
     EMO_CUDA(cudaGetLastError());
@@ -1194,6 +1198,19 @@ int emo_eval_intervals(const emo_graph *g, int64_t B, const uint8_t *F, int64_t 
     emo_workspace_bytes_intervals(g, B, I, p_idle != nullptr, &need);
     if (!ws || ws_bytes < need) return EMO_E_OOM;
     cudaStream_t st = (cudaStream_t)stream;
+    int64_t *d_breaks = (int64_t *)ws;
+    unsigned long long *busy = p_idle ? (unsigned long long *)((char *)ws + round_up((size_t)I * 8, 256)) : nullptr;
+    const int64_t ldw = (int64_t)round_up((size_t)B, 16);
+    const int rows = std::max(g->h.rows, 1);
+    EMO_CUDA(cudaMemcpyAsync(d_breaks, breaks, (size_t)I * 8, cudaMemcpyHostToDevice, st));
+    if (busy) EMO_CUDA(cudaMemsetAsync(busy, 0, (size_t)rows * (size_t)I * (size_t)ldw * 8, st));
+    const float inv_mean = (I > 1) ? (float)((double)(I - 1) / (double)breaks[I - 1]) : 0.0f;
+    long long delta = (I > 1) ? breaks[1] : 0;
+    for (int32_t i = 1; i < I && delta > 0; ++i)
+        if (breaks[i] != (int64_t)i * delta) delta = 0;
+    cudaEvent_t ev0 = g_pass_events[0], ev1 = g_pass_events[1];
+    if (ev0) EMO_CUDA(cudaEventRecord(ev0, st));
+    {
     const Program &p = g->fwd;
     const DevProgram &d = g->dfwd;
     if (p.steps == 0) return EMO_E_UNSUPPORTED;
@@ -1203,23 +1220,17 @@ int emo_eval_intervals(const emo_graph *g, int64_t B, const uint8_t *F, int64_t 
     const size_t brk_bytes = round_up((size_t)I * 8, 16);
     const size_t budget = g->smem_optin ? g->smem_optin : 48 * 1024;
     if (d.rec_bytes % 16) return EMO_E_UNSUPPORTED;      // a warp copies a record 16 bytes per thread
-    const size_t rec_pad = round_up((size_t)d.rec_bytes, 16);
+    const size_t rec_pad = round_up((size_t)d.rec_bytes, 16) + 16;      // the record and, in the last 16 bytes, the node's group
     const size_t off_rec = round_up(s.smem + brk_bytes, 16);
-    const size_t off_F = off_rec + (size_t)(s.threads / 32) * 2 * rec_pad;
+    const size_t off_F = off_rec + (size_t)(s.threads / 32) * 4 * rec_pad;
     if (off_F > budget) return EMO_E_UNSUPPORTED;
     const int rows_ = std::max(g->h.rows, 1);
     const size_t f_bytes = (size_t)rows_ * (size_t)I * (size_t)s.groups * 32;
     const bool stage_F = off_F + f_bytes <= budget;
-    int64_t *d_breaks = (int64_t *)ws;
-    unsigned long long *busy = p_idle ? (unsigned long long *)((char *)ws + round_up((size_t)I * 8, 256)) : nullptr;
-    const int64_t ldw = (int64_t)round_up((size_t)B, 16);
-    const int rows = std::max(g->h.rows, 1);
-    EMO_CUDA(cudaMemcpyAsync(d_breaks, breaks, (size_t)I * 8, cudaMemcpyHostToDevice, st));
-    if (busy) EMO_CUDA(cudaMemsetAsync(busy, 0, (size_t)rows * (size_t)I * (size_t)ldw * 8, st));
     IntervalParams a;
     a.p = PassParams();
     a.p.rec = d.rec;
-    a.p.rows = d.rows;
+    a.p.rows = d.groups;
     a.p.rec_bytes = d.rec_bytes;
     a.p.steps = p.steps;
     a.p.lanes = p.lanes;
@@ -1235,10 +1246,8 @@ int emo_eval_intervals(const emo_graph *g, int64_t B, const uint8_t *F, int64_t 
     a.ldb = ldb;
     a.I = I;
     a.breaks = d_breaks;
-    a.inv_mean = (I > 1) ? (float)((double)(I - 1) / (double)breaks[I - 1]) : 0.0f;
-    a.delta = (I > 1) ? breaks[1] : 0;
-    for (int32_t i = 1; i < I && a.delta > 0; ++i)
-        if (breaks[i] != (int64_t)i * a.delta) a.delta = 0;
+    a.inv_mean = inv_mean;
+    a.delta = delta;
     a.busy = busy;
     a.ldw = ldw;
     a.slot_bytes = (unsigned)s.smem;
@@ -1248,11 +1257,12 @@ int emo_eval_intervals(const emo_graph *g, int64_t B, const uint8_t *F, int64_t 
     a.stage_F = stage_F ? 1 : 0;
     a.rows = rows_;
     const size_t smem = off_F + (stage_F ? f_bytes : 0);
-    cudaEvent_t ev0 = g_pass_events[0], ev1 = g_pass_events[1];
-    if (ev0) EMO_CUDA(cudaEventRecord(ev0, st));
-    if (smem > 48 * 1024) EMO_CUDA(cudaFuncSetAttribute(emo_pass_intervals, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    emo_pass_intervals<<<s.grid, s.threads, smem, st>>>(a);
+    void (*kern)(IntervalParams) = delta > 0 ? (stage_F ? emo_pass_intervals<true, true> : emo_pass_intervals<true, false>)
+                                             : (stage_F ? emo_pass_intervals<false, true> : emo_pass_intervals<false, false>);
+    if (smem > 48 * 1024) EMO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g->smem_optin));
+    kern<<<s.grid, s.threads, smem, st>>>(a);
     EMO_CUDA(cudaGetLastError());
+    }
     if (p_idle) {
         emo_idle_energy<<<(unsigned)((B + 255) / 256), 256, 0, st>>>(B, rows, I, d_breaks, F, ldb, busy, ldw, p_idle, g->h.L, makespan,
                                                                        energy, energy_idle);

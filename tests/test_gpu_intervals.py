@@ -29,7 +29,7 @@ def emo():
     return E
 
 
-def run_gpu(torch, emo, g, dev_of, breaks, F, p_idle, flags=0, ldb=None):
+def run_gpu(torch, emo, g, dev_of, breaks, F, p_idle, flags=0, ldb=None, call_flags=0):
     """F: numpy uint8 [D][I][B]."""
     D, I, B = F.shape
     ldb = ldb or (B + 15) // 16 * 16
@@ -41,15 +41,15 @@ def run_gpu(torch, emo, g, dev_of, breaks, F, p_idle, flags=0, ldb=None):
     Ei = torch.zeros(B, dtype=torch.float64, device="cuda") if p_idle is not None else None
     pi = torch.from_numpy(np.asarray(p_idle, np.float64)).cuda() if p_idle is not None else None
     ws = torch.empty(emo.emo_workspace_bytes_intervals(h, B, I, p_idle is not None), dtype=torch.uint8, device="cuda")
-    emo.emo_eval_intervals(h, B, Fd, ldb, I, np.asarray(breaks, np.int64), pi, T, E, Ei, ws)
+    emo.emo_eval_intervals(h, B, Fd, ldb, I, np.asarray(breaks, np.int64), pi, T, E, Ei, ws, flags=call_flags)
     torch.cuda.synchronize()
     h.free()
     return T.cpu().numpy(), E.cpu().numpy(), None if Ei is None else Ei.cpu().numpy()
 
 
-def check(torch, emo, oracle_mod, g, dev_of, breaks, F, p_idle, **kw):
-    T, E, Ei = run_gpu(torch, emo, g, dev_of, breaks, F, p_idle, **kw)
+def check(torch, emo, oracle_mod, g, dev_of, breaks, F, p_idle, flags=0, **kw):
     r = oracle_mod.intervals(g, dev_of, breaks, F, p_idle)
+    T, E, Ei = run_gpu(torch, emo, g, dev_of, breaks, F, p_idle, flags=flags, **kw)
     assert np.array_equal(T, r["makespan"])
     assert np.allclose(E, r["energy"], rtol=1e-9, atol=0)
     if p_idle is not None:
@@ -73,6 +73,7 @@ def test_random_dags(torch_cuda, emo, oracle_mod, seed):
     check(torch_cuda, emo, oracle_mod, g, dev_of, breaks, F, None)
     check(torch_cuda, emo, oracle_mod, g, dev_of, [0], F[:, :1, :].copy(), p_idle)          # one interval
     check(torch_cuda, emo, oracle_mod, g, dev_of, breaks, F, p_idle, flags=emo.EMO_F_LANES(1))
+    check(torch_cuda, emo, oracle_mod, g, dev_of, breaks, F, p_idle, flags=emo.EMO_F_LANES(3) | emo.EMO_F_FLOW_SYNC(8))
 
 
 @pytest.mark.parametrize("name,scale,B,I", [("cfg0-tiny", 1.0, 64, 9), ("cfg1-train", 0.2, 200, 40), ("cfg3-8dev", 0.02, 100, 24),
@@ -90,6 +91,16 @@ def test_config_graphs(torch_cuda, emo, oracle_mod, name, scale, B, I):
     rs = np.random.RandomState(5)
     br2 = np.concatenate([[0], np.sort(rs.choice(np.arange(1, int(T0 * 1.2)), size=I - 1, replace=False))]).astype(np.int64)
     check(torch_cuda, emo, oracle_mod, g, dev_of, br2, F, W.idle_power(g.L))
+
+
+def test_pack_with_constant_tables_still_counts_as_busy(torch_cuda, emo, oracle_mod):
+    """A pack whose duration and energy do not depend on the level reads no level, but it keeps its device busy."""
+    lat = [[4, 4], [10, 10], [8, 5], [4, 4], [6, 6]]
+    en = [[0.0, 0.0], [5.0, 5.0], [4.0, 6.0], [0.0, 0.0], [3.0, 3.0]]
+    g = W.tiny_graph(5, [(0, 1), (1, 2), (0, 3), (3, 4)], np.asarray(lat, np.int64), np.asarray(en, np.float64))
+    F = np.array([[[1, 0, 1, 0], [0, 0, 1, 1], [1, 0, 1, 1]]], np.uint8)
+    check(torch_cuda, emo, oracle_mod, g, [-1, 0, 0, -1, 0], [0, 10, 16], F, [2.0, 3.0])
+    check(torch_cuda, emo, oracle_mod, g, [-1, 0, 0, -1, 0], [0, 50], F[:, :2, :].copy(), [2.0, 3.0])
 
 
 def test_argument_errors(torch_cuda, emo):
