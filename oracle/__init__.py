@@ -59,6 +59,8 @@ def lib():
         L.emo_oracle_select.restype = i64
         L.emo_oracle_intervals.argtypes = [i32, p, p, i32, p, p, p, i32, i32, p, p, i64, i64, i64, p, p, p, p, p, i64]
         L.emo_oracle_intervals.restype = ctypes.c_int
+        L.emo_oracle_search_dp.argtypes = [i32, p, p, i32, p, p, p, i32, i32, p, p, i64, i64, p, p, p, p, p]
+        L.emo_oracle_search_dp.restype = ctypes.c_int
         _lib = L
     return _lib
 
@@ -200,3 +202,25 @@ def intervals(g, dev_of, breaks, F, p_idle=None, b0: int = 0, b1: Optional[int] 
     if want_levels:
         out["levels"] = lv
     return out
+
+
+def search_dp(g, dev_of, breaks, p_idle, T_max: int, bin_ns: int = 1):
+    """Alg. 2 over the intervals given by `breaks`.  Returns a dict: found, F (uint8 [I]), T, E, n_pred."""
+    dev_of = _c(dev_of, np.int32)
+    D = int(dev_of.max()) + 1 if dev_of.size and dev_of.max() >= 0 else 1
+    breaks = _c(breaks, np.int64)
+    I = int(breaks.shape[0])
+    row_ptr, col = _c(g.row_ptr, np.int64), _c(g.col, np.int32)
+    lat, energy = _c(g.lat, np.int64), _c(g.energy, np.float64)
+    pi = None if p_idle is None else _c(p_idle, np.float64)
+    F = np.zeros(I, np.uint8)
+    T = ctypes.c_int64(0)
+    E = ctypes.c_double(0.0)
+    calls = ctypes.c_int64(0)
+    found = ctypes.c_int32(0)
+    rc = lib().emo_oracle_search_dp(g.n, _ptr(row_ptr), _ptr(col), g.L, _ptr(lat), _ptr(energy), _ptr(dev_of), D, I,
+                                    _ptr(breaks), _ptr(pi), int(T_max), int(bin_ns), _ptr(F), ctypes.byref(T),
+                                    ctypes.byref(E), ctypes.byref(calls), ctypes.byref(found))
+    if rc:
+        raise OracleError(f"emo_oracle_search_dp failed with {rc}")
+    return {"found": bool(found.value), "F": F, "T": int(T.value), "E": float(E.value), "n_pred": int(calls.value)}

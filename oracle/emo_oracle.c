@@ -20,6 +20,8 @@
  *                                              the budget is a fraction of it (2 %, 5 % in Sec. 5)
  *   selection ................................ Eq. 4 over a finite candidate set, with the feasibility
  *                                              and strict-improvement test of Alg. 2 (first best kept)
+ *   policy search ............................ Alg. 2 (dynamic programming over the intervals, one prediction per
+ *                                              candidate); a heuristic, pinned only in part: see its comment
  *   time-interval policies and idle energy ... Alg. 1 as printed (level from the interval that holds the
  *                                              start time, critical-predecessor tracking, E_a and E_i), Eq. 2
  *
@@ -31,8 +33,8 @@
  * order (Kahn) and its own successor lists; it never relies on the caller's numbering.
  *
  * Parity pins: every routine here is pinned by tests/test_oracle_pins.py (brute-force path
- * enumeration, closed forms, reversal duality, invariants, a hand-worked example).  Nothing in
- * this file is "parity unpinned".
+ * enumeration, closed forms, reversal duality, invariants, a hand-worked example).  Of this file only
+ * the policy search (Alg. 2) is "parity unpinned" beyond the pins its comment lists.
  */
 #include <stdint.h>
 #include <stdlib.h>
@@ -360,4 +362,139 @@ int emo_oracle_intervals(int32_t n, const int64_t *row_ptr, const int32_t *col, 
 done:
     free(order); free(pred); free(comp); free(start_of); free(succ_ptr); free(succ); free(e); free(ei);
     return rc;
+}
+
+/* ------------------------------------------------------------------------------------------------
+ * Alg. 2: search for a near-optimal time-interval policy by dynamic programming over the intervals.
+ * dp[i] maps an end-to-end time to the least energy (and its policy) seen after the first i intervals
+ * have been decided; every state is extended by every level for interval i, each candidate is
+ * predicted by Alg. 1 (emo_oracle_intervals: active + idle energy), kept if it meets T_max and
+ * improves its time's entry strictly.  The steps are taken in the algorithm's order.
+ *
+ * Readings where the paper is silent: the DP is keyed by the discretised time floor(t / bin_ns) (Sec. 4.6
+ * discretises the constraint, "e.g., 1 ms"; bin_ns = 1 keeps exact times); the states of dp[i] are visited
+ * in ascending time and the levels in ascending order, so that with the strict test the first candidate
+ * of least energy in a bin stays; one policy governs every device (the paper drops the GPU index in
+ * Alg. 2 and replicates one GPU's policy, Sec. 6.2); the answer is the entry of dp[I] of least energy,
+ * the earliest time among equals; the default policy P_0 is the maximum level L-1 everywhere.  If even
+ * P_0 misses T_max, dp[0] is still seeded with it (Alg. 2 line 3 has no test) and the search may end
+ * with an empty dp[I]: then *found = 0.
+ *
+ * Pinned only in part (tests/test_oracle_search.py): exhaustive optimum for one interval, bounds
+ * (never worse than P_0, never better than the exhaustive optimum, always feasible), consistency of the
+ * reported (T, E) with Alg. 1 on the reported policy, L = 1, T_max = t_0.  For several intervals the DP
+ * is a heuristic (one policy per time bin survives) and has no independent definition to compare with:
+ * beyond those pins it is "parity unpinned".
+ *
+ * Outputs: F_best[I] levels of the chosen policy, T_best, E_best, n_pred = calls of Alg. 1, found.
+ * ------------------------------------------------------------------------------------------------ */
+typedef struct {
+    int64_t key;      /* floor(t / bin) */
+    int64_t t;
+    double E;
+    uint8_t *P;       /* I levels */
+} dp_state;
+
+static int dp_cmp(const void *a, const void *b)
+{
+    int64_t x = ((const dp_state *)a)->key, y = ((const dp_state *)b)->key;
+    return x < y ? -1 : (x > y ? 1 : 0);
+}
+
+int emo_oracle_search_dp(int32_t n, const int64_t *row_ptr, const int32_t *col, int32_t L,
+                         const int64_t *lat, const double *energy, const int32_t *dev_of, int32_t D,
+                         int32_t I, const int64_t *breaks, const double *p_idle,
+                         int64_t T_max, int64_t bin_ns,
+                         uint8_t *F_best, int64_t *T_best, double *E_best, int64_t *n_pred, int32_t *found)
+{
+    if (I < 1 || L < 1 || D < 1 || bin_ns < 1) return ORACLE_E_ARG;
+    int rc = ORACLE_OK;
+    size_t cap = 16, cnt = 0, ncap = 16, ncnt = 0;
+    dp_state *cur = calloc(cap, sizeof *cur), *nxt = calloc(ncap, sizeof *nxt);
+    uint8_t *Fd = malloc((size_t)D * (size_t)I);      /* one candidate: [D][I][1] */
+    uint8_t *P2 = malloc((size_t)I);
+    int64_t calls = 0;
+    if (!cur || !nxt || !Fd || !P2) { rc = ORACLE_E_NOMEM; goto done; }
+#define PRED(Pol, tt, ee)                                                                                   \
+    do {                                                                                                    \
+        for (int32_t d_ = 0; d_ < D; ++d_) memcpy(Fd + (size_t)d_ * I, (Pol), (size_t)I);                    \
+        double ea_ = 0.0, ei_ = 0.0;                                                                        \
+        rc = emo_oracle_intervals(n, row_ptr, col, L, lat, energy, dev_of, D, I, breaks, Fd, 1, 0, 1, p_idle, \
+                                  &(tt), &ea_, &ei_, NULL, 0);                                              \
+        (ee) = ea_ + ei_;                                                                                   \
+        ++calls;                                                                                            \
+    } while (0)
+    /* P_0 = default frequency in all intervals; (t_0, E_0) = Pred(P_0); dp[0][t_0] = (E_0, P_0) */
+    {
+        uint8_t *P0 = malloc((size_t)I);
+        if (!P0) { rc = ORACLE_E_NOMEM; goto done; }
+        memset(P0, L - 1, (size_t)I);
+        int64_t t0 = 0;
+        double E0 = 0.0;
+        PRED(P0, t0, E0);
+        if (rc) { free(P0); goto done; }
+        cur[0].key = t0 / bin_ns; cur[0].t = t0; cur[0].E = E0; cur[0].P = P0;
+        cnt = 1;
+    }
+    for (int32_t i = 0; i < I; ++i) {
+        qsort(cur, cnt, sizeof *cur, dp_cmp);      /* ascending time */
+        ncnt = 0;
+        for (size_t s = 0; s < cnt; ++s) {
+            for (int32_t f = 0; f < L; ++f) {
+                /* P' <- set level f in [p_i, p_{i+1}) in P;  (t', E') <- Pred(P') */
+                memcpy(P2, cur[s].P, (size_t)I);
+                P2[i] = (uint8_t)f;
+                int64_t t2 = 0;
+                double E2 = 0.0;
+                PRED(P2, t2, E2);
+                if (rc) goto done;
+                if (t2 > T_max) continue;
+                int64_t key = t2 / bin_ns;
+                size_t k = 0;
+                while (k < ncnt && nxt[k].key != key) ++k;
+                if (k == ncnt) {
+                    if (ncnt == ncap) {
+                        dp_state *g2 = realloc(nxt, 2 * ncap * sizeof *nxt);
+                        if (!g2) { rc = ORACLE_E_NOMEM; goto done; }
+                        nxt = g2;
+                        memset(nxt + ncap, 0, ncap * sizeof *nxt);
+                        ncap *= 2;
+                    }
+                    nxt[k].P = malloc((size_t)I);
+                    if (!nxt[k].P) { rc = ORACLE_E_NOMEM; goto done; }
+                    nxt[k].key = key; nxt[k].t = t2; nxt[k].E = E2;
+                    memcpy(nxt[k].P, P2, (size_t)I);
+                    ++ncnt;
+                } else if (E2 < nxt[k].E) {
+                    nxt[k].t = t2; nxt[k].E = E2;
+                    memcpy(nxt[k].P, P2, (size_t)I);
+                }
+            }
+        }
+        /* dp[i] is no longer needed */
+        for (size_t s = 0; s < cnt; ++s) { free(cur[s].P); cur[s].P = NULL; }
+        dp_state *tmp = cur; cur = nxt; nxt = tmp;
+        size_t tc = cap; cap = ncap; ncap = tc;
+        cnt = ncnt; ncnt = 0;
+    }
+    /* (E*, P*) <- min over t <= T_max of dp[N][t] */
+    qsort(cur, cnt, sizeof *cur, dp_cmp);
+    {
+        size_t best = cnt;
+        for (size_t s = 0; s < cnt; ++s)
+            if (best == cnt || cur[s].E < cur[best].E) best = s;
+        if (found) *found = best < cnt;
+        if (best < cnt) {
+            if (F_best) memcpy(F_best, cur[best].P, (size_t)I);
+            if (T_best) *T_best = cur[best].t;
+            if (E_best) *E_best = cur[best].E;
+        }
+    }
+    if (n_pred) *n_pred = calls;
+done:
+    if (cur) for (size_t s = 0; s < cap; ++s) free(cur[s].P);
+    if (nxt) for (size_t s = 0; s < ncap; ++s) free(nxt[s].P);
+    free(cur); free(nxt); free(Fd); free(P2);
+    return rc;
+#undef PRED
 }
