@@ -179,6 +179,33 @@ int emo_eval_intervals(const emo_graph *g, int64_t B, const uint8_t *F, int64_t 
 int emo_workspace_bytes_intervals(const emo_graph *g, int64_t B, int32_t I, int with_idle, size_t *out);
 
 /*
+ * emo_search_dp - Alg. 2: search for a near-optimal time-interval policy by dynamic programming over the
+ * intervals, with emo_eval_intervals (Alg. 1) as the predictor.  dp[i] maps an end-to-end time to the least
+ * energy and its policy after the first i intervals are decided; every state is extended by every level in
+ * interval i, the |dp[i]| x L candidates of a stage are predicted as one batch on the GPU (in chunks of
+ * max_batch), and a candidate replaces its time's entry only if it meets T_max and is strictly better
+ * (candidates in the order of Alg. 2: states by ascending time, levels ascending).  The answer is the entry of
+ * dp[I] of least energy (Alg. 2, last line).
+ *   I, breaks     the intervals [p_i, p_{i+1}) as change points, HOST int64 [I], breaks[0] = 0 (as in
+ *                 emo_eval_intervals); one policy governs every device row (the paper drops the GPU index here
+ *                 and replicates one GPU's policy, Sec. 6.2).
+ *   p_idle        device fp64 [L] or NULL, as in emo_eval_intervals.
+ *   T_max         the constraint in ns (emo_target_from_delta gives it from T_0 and a budget).
+ *   bin_ns        >= 1: times are keyed as floor(t / bin_ns) (Sec. 4.6 discretises the constraint, "e.g., 1 ms";
+ *                 1 keeps exact times).  The number of states per stage is at most (T_max - t_min) / bin_ns + 1.
+ *   max_batch     candidates per evaluation call (0: 16384); sizes the workspace.
+ *   F_best        HOST uint8 [I]: the chosen level of every interval; T_best, E_best HOST scalars; n_pred HOST:
+ *                 predictions made; found HOST: 0 when no candidate met T_max (the other outputs are then untouched).
+ *   ws            device scratch of at least emo_workspace_bytes_search(g, I, max_batch, p_idle != NULL).
+ * The default policy P_0 is level L-1 everywhere; dp[0] is seeded with it without a test (Alg. 2 line 3).
+ * Synchronous: the call waits for every stage's results.  Errors as emo_eval_intervals.
+ */
+int emo_search_dp(const emo_graph *g, int32_t I, const int64_t *breaks, const double *p_idle, int64_t T_max,
+                  int64_t bin_ns, int64_t max_batch, uint8_t *F_best, int64_t *T_best, double *E_best,
+                  int64_t *n_pred, int32_t *found, void *ws, size_t ws_bytes, void *stream);
+int emo_workspace_bytes_search(const emo_graph *g, int32_t I, int64_t max_batch, int with_idle, size_t *out);
+
+/*
  * emo_slack_batch - forward and backward pass for B policies: earliest start ES, latest start LS
  * (critical-path backward pass: LF_v = min over successors of LS_u, the makespan for nodes
  * without successors; LS_v = LF_v - t_v) and slack = LS - ES per node and policy.

@@ -3,6 +3,7 @@
 
 #include <cmath>
 #include <cstdio>
+#include <map>
 #include <cstring>
 #include <new>
 #include <string>
@@ -1269,6 +1270,138 @@ int emo_eval_intervals(const emo_graph *g, int64_t B, const uint8_t *F, int64_t 
         EMO_CUDA(cudaGetLastError());
     }
     if (ev1) EMO_CUDA(cudaEventRecord(ev1, st));
+    return EMO_OK;
+}
+
+// Workspace of emo_search_dp: the candidates' levels, their times and energies, and what the evaluation needs.
+static void search_layout(const emo_graph *g, int32_t I, int64_t batch, int with_idle, size_t &off_T, size_t &off_E, size_t &off_ws,
+                          size_t &total, int64_t &ldb)
+{
+    ldb = (int64_t)round_up((size_t)batch, 16);
+    const size_t f_bytes = round_up((size_t)std::max(g->h.rows, 1) * (size_t)I * (size_t)ldb, 256);
+    off_T = f_bytes;
+    off_E = off_T + round_up((size_t)batch * 8, 256);
+    off_ws = off_E + round_up((size_t)batch * 8, 256);
+    size_t iv = 0;
+    emo_workspace_bytes_intervals(g, batch, I, with_idle, &iv);
+    total = off_ws + iv;
+}
+
+int emo_workspace_bytes_search(const emo_graph *g, int32_t I, int64_t max_batch, int with_idle, size_t *out)
+{
+    if (!g || !out || I < 1 || max_batch < 0) return EMO_E_INVALID_ARG;
+    if (max_batch == 0) max_batch = 16384;
+    size_t a, b, c, total;
+    int64_t ldb;
+    search_layout(g, I, max_batch, with_idle, a, b, c, total, ldb);
+    *out = total;
+    return EMO_OK;
+}
+
+int emo_search_dp(const emo_graph *g, int32_t I, const int64_t *breaks, const double *p_idle, int64_t T_max, int64_t bin_ns,
+                  int64_t max_batch, uint8_t *F_best, int64_t *T_best, double *E_best, int64_t *n_pred, int32_t *found,
+                  void *ws, size_t ws_bytes, void *stream)
+{
+    if (!g || I < 1 || I > 4096 || !breaks || bin_ns < 1 || max_batch < 0 || !found) return EMO_E_INVALID_ARG;
+    if (g->host_only) return EMO_E_CUDA;
+    if (max_batch == 0) max_batch = 16384;
+    const int L = g->h.L, rows = std::max(g->h.rows, 1);
+    size_t off_T, off_E, off_ws, total;
+    int64_t ldb;
+    search_layout(g, I, max_batch, p_idle != nullptr, off_T, off_E, off_ws, total, ldb);
+    if (!ws || ws_bytes < total) return EMO_E_OOM;
+    cudaStream_t st = (cudaStream_t)stream;
+    uint8_t *dF = (uint8_t *)ws;
+    int64_t *dT = (int64_t *)((char *)ws + off_T);
+    double *dE = (double *)((char *)ws + off_E);
+    void *iws = (char *)ws + off_ws;
+    const size_t iws_bytes = total - off_ws;
+    struct State {
+        int64_t t;
+        double E;
+        std::vector<uint8_t> P;
+    };
+    int64_t calls = 0;
+    *found = 0;
+    try {
+        std::vector<uint8_t> hF((size_t)rows * I * ldb);
+        std::vector<int64_t> hT((size_t)max_batch);
+        std::vector<double> hE((size_t)max_batch);
+        // Pred of a chunk of candidates (policy c = cand[c], the same levels for every device row)
+        auto predict = [&](const std::vector<const uint8_t *> &cand, const std::vector<std::pair<int32_t, uint8_t>> &patch) -> int {
+            const int64_t nb = (int64_t)cand.size();
+            for (int r = 0; r < rows; ++r)
+                for (int32_t i = 0; i < I; ++i) {
+                    uint8_t *dst = &hF[((size_t)r * I + i) * ldb];
+                    for (int64_t c = 0; c < nb; ++c) dst[c] = (patch[c].first == i) ? patch[c].second : cand[c][i];
+                }
+            if (cudaMemcpyAsync(dF, hF.data(), hF.size(), cudaMemcpyHostToDevice, st) != cudaSuccess) return EMO_E_CUDA;
+            int rc = emo_eval_intervals(g, nb, dF, ldb, I, breaks, p_idle, dT, dE, nullptr, iws, iws_bytes, nullptr, 0, stream);
+            if (rc) return rc;
+            if (cudaMemcpyAsync(hT.data(), dT, (size_t)nb * 8, cudaMemcpyDeviceToHost, st) != cudaSuccess) return EMO_E_CUDA;
+            if (cudaMemcpyAsync(hE.data(), dE, (size_t)nb * 8, cudaMemcpyDeviceToHost, st) != cudaSuccess) return EMO_E_CUDA;
+            if (cudaStreamSynchronize(st) != cudaSuccess) return EMO_E_CUDA;
+            calls += nb;
+            return EMO_OK;
+        };
+        // P_0 = default level in all intervals; dp[0][t_0] = (E_0, P_0)   (Alg. 2 lines 1-3)
+        std::map<int64_t, State> cur, nxt;
+        {
+            std::vector<uint8_t> P0((size_t)I, (uint8_t)(L - 1));
+            int rc = predict({P0.data()}, {{-1, 0}});
+            if (rc) return rc;
+            cur[hT[0] / bin_ns] = State{hT[0], hE[0], P0};
+        }
+        for (int32_t i = 0; i < I; ++i) {
+            nxt.clear();
+            // candidates in the order of Alg. 2: states by ascending time, levels ascending; evaluated in chunks
+            std::vector<const uint8_t *> cand;
+            std::vector<std::pair<int32_t, uint8_t>> patch;
+            auto flush = [&]() -> int {
+                if (cand.empty()) return EMO_OK;
+                int rc = predict(cand, patch);
+                if (rc) return rc;
+                for (size_t c = 0; c < cand.size(); ++c) {
+                    if (hT[c] > T_max) continue;
+                    const int64_t key = hT[c] / bin_ns;
+                    auto it = nxt.find(key);
+                    if (it == nxt.end() || hE[c] < it->second.E) {      // strict: the first of equals stays
+                        State s2{hT[c], hE[c], std::vector<uint8_t>(cand[c], cand[c] + I)};
+                        s2.P[(size_t)i] = patch[c].second;
+                        nxt[key] = std::move(s2);
+                    }
+                }
+                cand.clear();
+                patch.clear();
+                return EMO_OK;
+            };
+            for (auto &kv : cur)
+                for (int f = 0; f < L; ++f) {
+                    cand.push_back(kv.second.P.data());
+                    patch.push_back({i, (uint8_t)f});
+                    if ((int64_t)cand.size() == max_batch) {
+                        int rc = flush();
+                        if (rc) return rc;
+                    }
+                }
+            int rc = flush();
+            if (rc) return rc;
+            cur.swap(nxt);      // dp[i] is no longer needed
+        }
+        // (E*, P*) = the entry of dp[N] of least energy, the earliest time among equals
+        const State *best = nullptr;
+        for (auto &kv : cur)
+            if (!best || kv.second.E < best->E) best = &kv.second;
+        if (best) {
+            *found = 1;
+            if (F_best) std::memcpy(F_best, best->P.data(), (size_t)I);
+            if (T_best) *T_best = best->t;
+            if (E_best) *E_best = best->E;
+        }
+    } catch (const std::bad_alloc &) {
+        return EMO_E_OOM;
+    }
+    if (n_pred) *n_pred = calls;
     return EMO_OK;
 }
 

@@ -30,7 +30,7 @@ EXPORTS = [
     "emo_strerror", "emo_graph_load", "emo_graph_free", "emo_graph_info", "emo_workspace_bytes",
     "emo_eval_policies", "emo_slack_batch", "emo_slack", "emo_baseline", "emo_target_from_delta",
     "emo_select", "emo_transpose_policies", "emo_slack_batch_host", "emo_graph_program",
-    "emo_set_pass_events", "emo_select_static", "emo_graph_flow", "emo_set_wait_limit", "emo_call_path", "emo_set_flow_counters", "emo_workspace_bytes_for", "emo_measure_int_issue", "emo_measure_warp_costs", "emo_eval_intervals", "emo_workspace_bytes_intervals", "emo_pack_levels", "emo_unpack_levels", "emo_slack_batch_host_packed",
+    "emo_set_pass_events", "emo_select_static", "emo_graph_flow", "emo_set_wait_limit", "emo_call_path", "emo_set_flow_counters", "emo_workspace_bytes_for", "emo_measure_int_issue", "emo_measure_warp_costs", "emo_eval_intervals", "emo_workspace_bytes_intervals", "emo_search_dp", "emo_workspace_bytes_search", "emo_pack_levels", "emo_unpack_levels", "emo_slack_batch_host_packed",
 ]
 
 
@@ -113,6 +113,8 @@ def lib():
         L.emo_measure_warp_costs.argtypes = [p, p, p]
         L.emo_eval_intervals.argtypes = [p, i64, p, i64, i32, p, p, p, p, p, p, ctypes.c_size_t, p, u32, p]
         L.emo_workspace_bytes_intervals.argtypes = [p, i64, i32, ctypes.c_int, p]
+        L.emo_search_dp.argtypes = [p, i32, p, p, i64, i64, i64, p, p, p, p, p, p, ctypes.c_size_t, p]
+        L.emo_workspace_bytes_search.argtypes = [p, i32, i64, ctypes.c_int, p]
         L.emo_pack_levels.argtypes = [ctypes.c_int, i64, i64, p, i64, p, i64, p]
         L.emo_unpack_levels.argtypes = [ctypes.c_int, i64, i64, p, i64, p, i64, p]
         L.emo_slack_batch_host_packed.argtypes = [p, i64, ctypes.c_int, p, i64, p, p, i64, p, i64, i64, p, p, p, p, p, p, sz, u32, p]
@@ -391,6 +393,25 @@ def emo_eval_intervals(g, B, F, ldb, I, breaks, p_idle, makespan, energy, energy
     return _check(lib().emo_eval_intervals(g.handle, int(B), _addr(F), int(ldb), int(I), brk.ctypes.data_as(ctypes.c_void_p),
                                            _addr(p_idle), _addr(makespan), _addr(energy), _addr(energy_idle), _addr(ws),
                                            _nbytes(ws), _addr(status), int(flags), _stream(stream)), "emo_eval_intervals")
+
+
+def emo_workspace_bytes_search(g, I, max_batch=0, with_idle=True) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().emo_workspace_bytes_search(g.handle, int(I), int(max_batch), int(bool(with_idle)), ctypes.byref(out)),
+           "emo_workspace_bytes_search")
+    return int(out.value)
+
+
+def emo_search_dp(g, breaks, p_idle, T_max, bin_ns, ws, max_batch=0, stream=None) -> dict:
+    """Alg. 2 on the GPU evaluator (see include/emo.h).  breaks: host int64 [I]; p_idle: device tensor or None."""
+    brk = np.ascontiguousarray(breaks, dtype=np.int64)
+    I = int(brk.shape[0])
+    F = np.zeros(I, np.uint8)
+    T, E, calls, found = ctypes.c_int64(0), ctypes.c_double(0.0), ctypes.c_int64(0), ctypes.c_int32(0)
+    _check(lib().emo_search_dp(g.handle, I, brk.ctypes.data_as(ctypes.c_void_p), _addr(p_idle), int(T_max), int(bin_ns), int(max_batch),
+                               F.ctypes.data_as(ctypes.c_void_p), ctypes.byref(T), ctypes.byref(E), ctypes.byref(calls),
+                               ctypes.byref(found), _addr(ws), _nbytes(ws), _stream(stream)), "emo_search_dp")
+    return {"found": bool(found.value), "F": F, "T": int(T.value), "E": float(E.value), "n_pred": int(calls.value)}
 
 
 def emo_pack_levels(bits, rows, B, lvl, ldb, packed, ldp, stream=None):
