@@ -193,6 +193,26 @@ def intervals_leg(args, g, B, m, T0_ns, check):
         bad = int((T.cpu().numpy()[cols] != r["makespan"]).sum()) + int((~np.isclose(E.cpu().numpy()[cols], r["energy"], rtol=1e-9, atol=0)).sum())
         out["checked"] = {"policies": nb, "mismatches": bad}
         assert bad == 0, "interval evaluation disagrees with the oracle"
+    if not args.no_search:
+        # Alg. 2 on top of it: dynamic programming over the intervals, every stage's candidates as one batch
+        T_max = T0_ns + T0_ns * int(args.search_ppm) // 1000000
+        ws2 = torch.empty(emo.emo_workspace_bytes_search(h, I, 0, True), dtype=torch.uint8, device="cuda")
+        t_start = time.perf_counter()
+        r = emo.emo_search_dp(h, breaks, pi, T_max, 1000000, ws2)
+        dt = time.perf_counter() - t_start
+        Fb = torch.from_numpy(np.repeat(r["F"][None, :, None], D, axis=0).repeat(16, axis=2).copy()).cuda()
+        emo.emo_eval_intervals(h, 1, torch.full((D, I, 16), g.L - 1, dtype=torch.uint8, device="cuda"), 16, I, breaks, pi, T, E, Ei, ws)
+        torch.cuda.synchronize()
+        E_default = float(E[0].item())
+        out["search"] = {"found": r["found"], "budget_ppm": int(args.search_ppm), "bin_ns": 1000000, "predictions": r["n_pred"], "seconds": dt,
+                         "predictions_per_s": r["n_pred"] / dt, "T_over_T0": r["T"] / T0_ns, "energy": r["E"],
+                         "energy_default": E_default, "saving": 1.0 - r["E"] / E_default}
+        if check and r["found"]:
+            import oracle      # the CPU oracle: checks only, never on the product path
+            ro = oracle.intervals(g, dev_of, breaks, Fb[:, :, :1].cpu().numpy(), W.idle_power(g.L))
+            ok = int(ro["makespan"][0]) == r["T"] and bool(np.isclose(ro["energy"][0], r["E"], rtol=1e-9, atol=0))
+            out["search"]["policy_checked_against_oracle"] = ok
+            assert ok, "the searched policy's time and energy disagree with the oracle"
     h.free()
     return out
 
@@ -212,6 +232,8 @@ def main():
     ap.add_argument("--flags", type=int, default=0, help="extra EMO_F_* load flags (lanes / look-ahead)")
     ap.add_argument("--call-flags", type=int, default=0, help="EMO_F_* flags of the pass calls (kernel choice)")
     ap.add_argument("--no-intervals", action="store_true", help="skip the time-interval policy leg (Alg. 1 in its own form)")
+    ap.add_argument("--no-search", action="store_true", help="skip the policy search (Alg. 2) inside the time-interval leg")
+    ap.add_argument("--search-ppm", type=int, default=50000, help="latency budget of the policy search, parts per million of T_0")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
