@@ -166,7 +166,7 @@ def intervals_leg(args, g, B, m, T0_ns, check):
     breaks = W.interval_breaks(T0_ns, I)
     F = W.interval_policies(g.meta["policy_seed"], D, I, g.L, B, device="cuda")
     ldb = F.shape[2]
-    h = emo.load_workload(g, flags=args.flags, group_of=dev_of)
+    h = emo.load_workload(g, flags=args.flags | emo.EMO_F_INTERVALS, group_of=dev_of)
     T = torch.zeros(B, dtype=torch.int64, device="cuda")
     E = torch.zeros(B, dtype=torch.float64, device="cuda")
     Ei = torch.zeros(B, dtype=torch.float64, device="cuda")

@@ -50,6 +50,8 @@ extern "C" {
 #define EMO_F_LOOKAHEAD(d) (((uint32_t)(d) & 0xFFu) << 16) /* scheduling look-ahead in steps */
 #define EMO_F_FLOW_SYNC(s) ((((uint32_t)(s) / 8u) & 0xFu) << 4)  /* lane-stream program: steps between group barriers (8, 16, 32) */
 #define EMO_F_FLOW_STAGE(k) (((uint32_t)(k) & 0x3Fu) << 24)      /* lane-stream program: steps per stage (8, 16, 32) */
+#define EMO_F_INTERVALS 0x2u       /* also prepare the lane-stream form of emo_eval_intervals (a second copy of the forward program on
+                                      the device); without it that call runs its step-program kernel */
 /* flags of the evaluation calls */
 #define EMO_F_VALIDATE 0x1u        /* check every level < L first; EMO_E_RANGE goes to *status */
 #define EMO_F_NO_STAGING 0x2u      /* use the plain-load kernels instead of the staged ones */
@@ -168,6 +170,9 @@ int emo_eval_policies(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t
  * part of the interval below the makespan minus the summed overlap of the row's packs with it, not below zero
  * (exact when the packs of a device do not overlap in time, as packs of one device timeline do not; the paper
  * does not define idle_time further).
+ * Kernels: a graph loaded with EMO_F_INTERVALS runs the 32-bit lane-stream kernel when the change points are a
+ * uniform grid and the columns of F fit shared memory; otherwise, or with EMO_F_NO_STAGING in flags, the
+ * step-program kernel runs.  Both give the same results.
  * Errors: EMO_E_INVALID_ARG (sizes, breaks not increasing from 0, energy_idle without p_idle), EMO_E_OOM
  * (workspace too small), EMO_E_UNSUPPORTED (change points and exchange slots do not fit shared memory).
  * Asynchronous on `stream` after the change points are copied.

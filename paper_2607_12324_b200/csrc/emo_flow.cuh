@@ -57,6 +57,18 @@ struct FlowParams {
     long long wait_cycles;               // bound of every device-side wait
     int stall_stage;                     // test hook: the producers stop before this stage (-1: off)
     long long *prof;                     // optional cycle counters, 8 per warp: waits for stages, group barriers, total, backward: special entries, runs
+    // time-interval policies (forward kernel, INTV = true): the level of a pack comes from the interval that holds its
+    // start time (uniform grid of change points, the block's columns of F in shared memory)
+    const uint8_t *F;                    // [rowsF][I][ldF] levels
+    int64_t ldF;
+    int I, rowsF;
+    long long delta;                     // the change points are i * delta
+    float inv_mean;
+    const long long *breaks;             // device [I]
+    unsigned long long *busy;            // [rowsF][I][ldw] or NULL
+    int64_t ldw;
+    unsigned off_meta;                   // inside a stage: 16 bytes per entry {lbES_v (8), group, dmin_v}
+    unsigned off_brk, off_Fs;            // inside the block's shared memory: change points, columns of F
 };
 
 __device__ __forceinline__ unsigned long long emo_lds_b64v(unsigned a)
@@ -119,6 +131,13 @@ __device__ __forceinline__ unsigned emo_tld_u8(unsigned a, unsigned tok)
 {
     unsigned v;
     asm("ld.shared.u8 %0, [%1]; // %2" : "=r"(v) : "r"(a), "r"(tok));
+    return v;
+}
+// a byte of block-lifetime shared data (written once before the walk begins)
+__device__ __forceinline__ unsigned emo_vld_u8(unsigned a)
+{
+    unsigned v;
+    asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(a));
     return v;
 }
 __device__ __forceinline__ unsigned emo_tld_u32(unsigned a, unsigned tok)
@@ -435,7 +454,65 @@ __device__ __forceinline__ void emo_flow_fwd_run(unsigned la, unsigned ta0, unsi
     ea += g[0];
 }
 
-template <int MAXT>
+// What the forward kernel carries for time-interval policies beside its parameters.
+struct FlowIntv {
+    const long long *brk;        // change points in shared memory
+    unsigned Fs;                 // the block's columns of F in shared memory (shared-window address of this thread's column): [rowsF * I][ptile]
+    int col;                     // this thread's column in the block
+    int64_t b;                   // this thread's policy
+    bool count;                  // this thread adds busy time (a live policy and a busy array)
+    unsigned key;                // busy time collected for (row, interval) = key, not yet added to memory
+    unsigned long long sum;
+};
+// The level of an entry whose start offset is eo (Alg. 1: the interval that holds the start time), then its
+// table entry.  No branch on anything loaded here: a node outside every policy reads the last row and any
+// level (its table row holds one value), the interval index is a float guess with one exact correction (uniform
+// grid), and busy time is collected in a register while the (row, interval) stays the same.
+__device__ __forceinline__ void emo_flow_intv_lookup(const FlowParams &p, FlowIntv &iv, const uint4 &meta, unsigned eo, unsigned ta0,
+                                                     unsigned lmask, unsigned tok, unsigned &dd, double &e)
+{
+    const long long start = (long long)((unsigned long long)meta.x | ((unsigned long long)meta.y << 32)) + (long long)eo;
+    const bool pack = meta.z != emo::kNone;
+    const unsigned rowc = min(meta.z, (unsigned)p.rowsF - 1u);
+    long long iend;
+    const int i = emo_interval_index<true>(start, p.I, p.delta, p.inv_mean, iv.brk, iend);
+    const unsigned key = rowc * (unsigned)p.I + (unsigned)i;
+    const unsigned lv = emo_vld_u8(iv.Fs + key * (unsigned)p.ptile);
+    const unsigned ta = ta0 + (lv & lmask) * 12u;
+    dd = emo_tld_u32(ta, tok);
+    e = __hiloint2double((int)emo_tld_u32(ta + 4u, tok), (int)emo_tld_u32(ta + 8u, tok));
+    const long long dur = (long long)meta.w + (long long)dd;
+    const bool on = pack && iv.count;
+    if (on && key != iv.key) {      // rare: the lane moved on to another interval (or device)
+        if (iv.sum) atomicAdd(p.busy + (size_t)iv.key * p.ldw + iv.b, iv.sum);
+        iv.key = key;
+        iv.sum = 0;
+    }
+    const bool single = start + dur <= iend;
+    iv.sum += (on && single) ? (unsigned long long)dur : 0ull;
+    if (on && !single) emo_interval_busy(p.busy, p.ldw, iv.b, rowc, p.I, i, iend, start, start + dur, iv.brk);      // rare
+}
+// A run of r plain entries: every start time depends on the entry before it, so the look-ups form one chain
+// and there is nothing to gain from one instantiation per length (which would only crowd the instruction
+// cache: the look-up is some sixty instructions); a loop, inlined so that the parameters and the lane's running
+// values stay in registers, with the next entry's constants requested one entry ahead.
+__device__ __forceinline__ void emo_flow_fwd_run_intv(const FlowParams &p, FlowIntv &iv, unsigned r, unsigned meta_a, unsigned ta0, unsigned tab_row,
+                                                   unsigned lmask, unsigned tok, unsigned &h, double &ea)
+{
+    uint4 meta = emo_tld_128(meta_a, tok);
+#pragma unroll 1
+    for (unsigned i = 0; i < r; ++i) {
+        const uint4 cur = meta;
+        meta = emo_tld_128(meta_a + 16u * min(i + 1u, r - 1u), tok);      // never past the run: the last entry's constants end the stage buffer
+        unsigned dd;
+        double e;
+        emo_flow_intv_lookup(p, iv, cur, h, ta0 + i * tab_row, lmask, tok, dd, e);
+        h += dd;
+        ea += e;
+    }
+}
+
+template <int MAXT, bool INTV>
 __global__ void __launch_bounds__(MAXT, 1) emo_flow_fwd(FlowParams p)
 {
     extern __shared__ __align__(128) unsigned char emo_smem[];
@@ -455,6 +532,20 @@ __global__ void __launch_bounds__(MAXT, 1) emo_flow_fwd(FlowParams p)
     volatile int *abort_word = reinterpret_cast<volatile int *>(emo_smem + p.off_bar + 16 * kFlowMaxBuf);
     const unsigned stage0 = smem0 + p.off_stage0;
     emo_flow_init(p, smem0, emo_smem, n_cons);
+    FlowIntv iv{nullptr, 0u, col, b, act && p.busy != nullptr, 0u, 0ull};
+    if (INTV) {
+        long long *brk = reinterpret_cast<long long *>(emo_smem + p.off_brk);
+        for (int i = threadIdx.x; i < p.I; i += blockDim.x) brk[i] = p.breaks[i];
+        unsigned char *Fs = emo_smem + p.off_Fs;
+        const int total = p.rowsF * p.I * ptile;
+        for (int k2 = threadIdx.x; k2 < total; k2 += blockDim.x) {
+            const int ri = k2 / ptile, c = k2 - ri * ptile;
+            Fs[k2] = (b0 + c < p.B) ? p.F[(size_t)ri * p.ldF + b0 + c] : (unsigned char)0;
+        }
+        iv.brk = brk;
+        iv.Fs = smem0 + p.off_Fs + (unsigned)col;
+        __syncthreads();
+    }
 
     unsigned h = 0;
     double ea = 0.0;
@@ -498,6 +589,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_flow_fwd(FlowParams p)
             unsigned tab_a = sta + p.off_tab + (unsigned)(chain * K) * tab_row;
             unsigned lvl_a = sta + p.off_lvl + ((unsigned)((group * lanes + chain) * K) << 5) + (unsigned)lane;
             const unsigned pool_a = sta + p.off_pool;
+            unsigned meta_a = sta + p.off_meta + (unsigned)(chain * K) * 16u;
             uint32_t *push = rst_lane ? rst_lane + ((size_t)hd1.z + hd1.y) * ptile : nullptr;
             hd0.x = emo_uniform(hd0.x);
             const int nseg = (int)(hd0.x & 255u);
@@ -526,22 +618,31 @@ __global__ void __launch_bounds__(MAXT, 1) emo_flow_fwd(FlowParams p)
                     // the common shapes (at most one operand, any output) run without a branch
                     const uint4 r0 = emo_tld_128(rec_a, tok);
                     const uint4 r1 = emo_tld_128(rec_a + 16u, tok);
-                    const unsigned lb = emo_tld_u8(lvl_a, tok);
                     const unsigned fl = r0.x;
-                    const unsigned ta = tab_a + (lb & lmask) * 12u;
-                    const unsigned dd = emo_tld_u32(ta, tok), ghi = emo_tld_u32(ta + 4u, tok), glo = emo_tld_u32(ta + 8u, tok);
+                    unsigned dd = 0;
+                    double ee = 0.0;
+                    uint4 meta = make_uint4(0, 0, 0, 0);
+                    if (INTV) {
+                        meta = emo_tld_128(meta_a, tok);
+                    } else {
+                        const unsigned lb = emo_tld_u8(lvl_a, tok);
+                        const unsigned ta = tab_a + (lb & lmask) * 12u;
+                        dd = emo_tld_u32(ta, tok);
+                        ee = __hiloint2double((int)emo_tld_u32(ta + 4u, tok), (int)emo_tld_u32(ta + 8u, tok));
+                    }
                     const unsigned nops = fl >> emo::kF_NopsShift;
                     unsigned v = emo_floor_sub((fl & emo::kF_HasReg) ? h : 0u, r1.w);
                     unsigned x0, t0, a0;
                     emo_flow_operand_u(slot_lane4, lane4, r1.x, nops, x0, t0, a0);
                     const bool retry0 = nops != 0u && (r1.x & (emo::kOpWord | emo::kOpNoPoll)) == 0u && t0 != r1.y;
+                    unsigned pa = pool_a + r0.w * 4u;
+                    bool term = false;
                     if (__any_sync(0xFFFFFFFFu, retry0 || nops > 1u || (fl & emo::kF_Terminal) != 0u)) {
-                        // the rest: a value that was not there yet, further operands, the makespan candidate
+                        // the rest: a value that was not there yet, further operands, a makespan candidate
                         if (retry0 && !emo_flow_poll(a0, r1.y, x0, abort_word, limit)) {
                             dead = true;
                             *abort_word = 1;
                         }
-                        unsigned pa = pool_a + r0.w * 4u;
                         for (unsigned k = 1; k < nops; ++k) {
                             const unsigned x2 = emo_flow_operand(slot_base, lane, emo_tld_u32(pa, tok), emo_tld_u32(pa + 4u, tok), dead,
                                                                  abort_word, limit);
@@ -550,37 +651,53 @@ __global__ void __launch_bounds__(MAXT, 1) emo_flow_fwd(FlowParams p)
                         }
                         dead = __any_sync(0xFFFFFFFFu, dead);
                         if (dead) continue;      // on to the group's next barrier
-                        if (fl & emo::kF_Terminal) {
+                        if (INTV) {
+                            term = (fl & emo::kF_Terminal) != 0u;      // its duration is not known yet
+                        } else if (fl & emo::kF_Terminal) {
+                            // a node without successors: candidate for the makespan (its bound follows the operands in the pool)
                             const long long lbc = (long long)((unsigned long long)emo_tld_u32(pa, tok) | ((unsigned long long)emo_tld_u32(pa + 4u, tok) << 32));
                             const unsigned vt = max(v, emo_floor_sub(x0, r1.z)) + dd;
                             acc = emo_max64(acc, lbc + (long long)vt);
                         }
                     }
                     v = max(v, emo_floor_sub(x0, r1.z));
+                    // time-interval policies: the level follows from the start time, which is known only now
+                    if (INTV) emo_flow_intv_lookup(p, iv, meta, v, tab_a, lmask, tok, dd, ee);
                     if ((fl & emo::kF_Push) && push) {
                         *push = h;
                         push += ptile;
                     }
-                    ea += __hiloint2double((int)ghi, (int)glo);
+                    ea += ee;
                     v += dd;
                     emo_flow_out_u(slot_lane4, lane4, v, r0.y, r0.z, fl & emo::kF_OutTag, fl & emo::kF_OutSet, fl & emo::kF_OutAcc);
+                    if (INTV && term) {
+                        // a node without successors: candidate for the makespan (its bound follows the operands in the pool)
+                        const long long lbc = (long long)((unsigned long long)emo_tld_u32(pa, tok) | ((unsigned long long)emo_tld_u32(pa + 4u, tok) << 32));
+                        acc = emo_max64(acc, lbc + (long long)v);
+                    }
                     h = v;
+                    meta_a += 16u;
                     rec_a += 32u;
                     tab_a += tab_row;
                     lvl_a += 32u;
                 }
                 // the run: every entry continues from the lane's previous value
-                switch (r) {
-                    case 1: emo_flow_fwd_run<1>(lvl_a, tab_a, tab_row, lmask, tok, h, ea); break;
-                    case 2: emo_flow_fwd_run<2>(lvl_a, tab_a, tab_row, lmask, tok, h, ea); break;
-                    case 3: emo_flow_fwd_run<3>(lvl_a, tab_a, tab_row, lmask, tok, h, ea); break;
-                    case 4: emo_flow_fwd_run<4>(lvl_a, tab_a, tab_row, lmask, tok, h, ea); break;
-                    case 5: emo_flow_fwd_run<5>(lvl_a, tab_a, tab_row, lmask, tok, h, ea); break;
-                    case 6: emo_flow_fwd_run<6>(lvl_a, tab_a, tab_row, lmask, tok, h, ea); break;
-                    case 7: emo_flow_fwd_run<7>(lvl_a, tab_a, tab_row, lmask, tok, h, ea); break;
-                    case 8: emo_flow_fwd_run<8>(lvl_a, tab_a, tab_row, lmask, tok, h, ea); break;
-                    default: break;
+                if (INTV) {
+                    if (r) emo_flow_fwd_run_intv(p, iv, (unsigned)r, meta_a, tab_a, tab_row, lmask, tok, h, ea);
+                } else {
+                    switch (r) {
+                        case 1: emo_flow_fwd_run<1>(lvl_a, tab_a, tab_row, lmask, tok, h, ea); break;
+                        case 2: emo_flow_fwd_run<2>(lvl_a, tab_a, tab_row, lmask, tok, h, ea); break;
+                        case 3: emo_flow_fwd_run<3>(lvl_a, tab_a, tab_row, lmask, tok, h, ea); break;
+                        case 4: emo_flow_fwd_run<4>(lvl_a, tab_a, tab_row, lmask, tok, h, ea); break;
+                        case 5: emo_flow_fwd_run<5>(lvl_a, tab_a, tab_row, lmask, tok, h, ea); break;
+                        case 6: emo_flow_fwd_run<6>(lvl_a, tab_a, tab_row, lmask, tok, h, ea); break;
+                        case 7: emo_flow_fwd_run<7>(lvl_a, tab_a, tab_row, lmask, tok, h, ea); break;
+                        case 8: emo_flow_fwd_run<8>(lvl_a, tab_a, tab_row, lmask, tok, h, ea); break;
+                        default: break;
+                    }
                 }
+                meta_a += (unsigned)r * 16u;
                 rec_a += (unsigned)r * 32u;
                 tab_a += (unsigned)r * tab_row;
                 lvl_a += (unsigned)r * 32u;
@@ -591,6 +708,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_flow_fwd(FlowParams p)
             __syncwarp();
             if (lane == 0) emo_mbar_arrive(bar0 + 8 * (kFlowMaxBuf + s));
         }
+        if (INTV && iv.count && iv.sum) atomicAdd(p.busy + (size_t)iv.key * p.ldw + iv.b, iv.sum);
         if (p.prof && lane == 0 && blockIdx.x < 512) {
             long long *pr = p.prof + ((size_t)blockIdx.x * 32 + warp) * 8;
             pr[0] = t_wait;

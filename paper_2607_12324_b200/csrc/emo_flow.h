@@ -97,6 +97,8 @@ struct Flow {
     std::vector<uint32_t> tabF;         // [stages][lanes][K][Lp][3]: t - dmin, energy high word, low word
     std::vector<uint32_t> tabB;         // [stages][lanes][K][Lp]: t - dmin
     std::vector<int64_t> lbes;          // [stages][lanes][K] lbES_v (for the ES and LS outputs)
+    std::vector<uint32_t> dmin;         // [stages][lanes][K] smallest entry of the node's duration row (time-interval policies)
+    std::vector<uint32_t> grp;          // [stages][lanes][K] the node's group whether or not its tables depend on the level (kNone: none)
     std::vector<int64_t> push_base;     // [stages + 1] first restore row of every stage
     FlowDir f, b;
 };

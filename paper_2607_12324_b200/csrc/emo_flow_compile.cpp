@@ -210,6 +210,8 @@ int compile_flow(const HostGraph &g, const int64_t *lat, const double *energy, i
     out.node.assign(Q, kNone);
     out.step.assign(Q, kNone);
     out.lbes.assign(Q, 0);
+    out.dmin.assign(Q, 0);
+    out.grp.assign(Q, kNone);
     out.tabF.assign(Q * Lp * 3, 0);
     out.tabB.assign(Q * Lp, 0);
     {
@@ -323,6 +325,8 @@ int compile_flow(const HostGraph &g, const int64_t *lat, const double *energy, i
         out.node[q] = (uint32_t)v;
         out.step[q] = (uint32_t)step_of[v];
         out.lbes[q] = lbES[v];
+        out.dmin[q] = (uint32_t)dmin[v];
+        if (g.group[v] >= 0) out.grp[q] = (uint32_t)g.group[v];
         if (g.group[v] >= 0 && !constant[v]) out.rows[q] = (uint32_t)g.group[v];
         for (int l = 0; l < Lp; ++l) {
             const int ll = (g.group[v] < 0 || constant[v]) ? 0 : (l < L ? l : L - 1);

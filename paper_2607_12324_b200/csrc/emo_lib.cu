@@ -39,8 +39,9 @@ struct DevProgramLane {
 // The lane-stream program on the device: one blob per stage and direction (see emo_flow.cuh).
 struct DevFlow {
     unsigned char *blobF = nullptr, *blobB = nullptr;
+    unsigned char *blobFI = nullptr;      // the forward blob followed by 16 bytes per entry {lbES_v, group, dmin_v}: time-interval policies
     uint32_t *rows = nullptr, *push_base = nullptr;
-    unsigned blobF_bytes = 0, blobB_bytes = 0;
+    unsigned blobF_bytes = 0, blobB_bytes = 0, blobFI_bytes = 0, f_off_meta = 0;
     unsigned off_seg = 0;
     unsigned f_off_rec = 0, f_off_pool = 0, f_off_tab = 0;
     unsigned b_off_rec = 0, b_off_pool = 0, b_off_lbes = 0, b_off_tab = 0;
@@ -498,7 +499,7 @@ int launch_pass(const emo_graph *g, const PassPlan &pl, bool backward, int64_t B
 long long *g_flow_prof = nullptr;           // optional device array for the kernels' cycle counters (measurement hook)
 long long g_wait_cycles = 4000000000LL;    // bound of every device-side wait of the 32-bit kernels (about two seconds)
 
-int upload_flow(const Flow &f, DevFlow &d)
+int upload_flow(const Flow &f, DevFlow &d, bool intervals)
 {
     if (!f.ok32 || f.stages == 0) return EMO_OK;
     const size_t per = (size_t)f.lanes * f.K;
@@ -534,6 +535,22 @@ int upload_flow(const Flow &f, DevFlow &d)
     }
     int rc = upload(&d.blobF, bf.data(), bf.size());
     if (rc == EMO_OK) rc = upload(&d.blobB, bb.data(), bb.size());
+    if (rc == EMO_OK && intervals) {
+        d.f_off_meta = d.blobF_bytes;
+        d.blobFI_bytes = (unsigned)r16(d.f_off_meta + per * 16);
+        std::vector<unsigned char> bi((size_t)f.stages * d.blobFI_bytes, 0);
+        for (int st = 0; st < f.stages; ++st) {
+            unsigned char *dst = bi.data() + (size_t)st * d.blobFI_bytes;
+            std::memcpy(dst, bf.data() + (size_t)st * d.blobF_bytes, d.blobF_bytes);
+            for (size_t e = 0; e < per; ++e) {
+                const size_t q = (size_t)st * per + e;
+                const int64_t lb = f.lbes[q];
+                const uint32_t w[4] = {(uint32_t)(uint64_t)lb, (uint32_t)((uint64_t)lb >> 32), f.grp[q], f.dmin[q]};
+                std::memcpy(dst + d.f_off_meta + e * 16, w, 16);
+            }
+        }
+        rc = upload(&d.blobFI, bi.data(), bi.size());
+    }
     if (rc == EMO_OK) rc = upload(&d.rows, f.rows.data(), f.rows.size() * 4);
     if (rc == EMO_OK) rc = upload(&d.push_base, pb.data(), pb.size() * 4);
     d.ready = rc == EMO_OK;
@@ -544,6 +561,7 @@ void free_flow(DevFlow &d)
 {
     if (d.blobF) cudaFree(d.blobF);
     if (d.blobB) cudaFree(d.blobB);
+    if (d.blobFI) cudaFree(d.blobFI);
     if (d.rows) cudaFree(d.rows);
     if (d.push_base) cudaFree(d.push_base);
     d = DevFlow();
@@ -559,12 +577,17 @@ struct FlowPlan {
     size_t restore_bytes = 0;
 };
 
-bool flow_plan(const emo_graph *g, int64_t B, bool want_base, bool need_bwd, FlowPlan &pl)
+// intv: the plan of the forward kernel for time-interval policies (no level rows are staged; the blob carries
+// 16 more bytes per entry; extra_fixed + G * extra_per_group bytes of the block are set aside for the change
+// points and the block's columns of F).
+bool flow_plan(const emo_graph *g, int64_t B, bool want_base, bool need_bwd, FlowPlan &pl, bool intv = false,
+               size_t extra_fixed = 0, size_t extra_per_group = 0)
 {
     const Flow &f = g->flow;
     const DevFlow &d = g->dflow;
     pl.ok = false;
     if (!f.ok32 || !d.ready || !g->smem_optin || f.stages == 0) return false;
+    if (intv && !d.blobFI) return false;
     if (f.lanes * f.K > 32 * kFlowRowRegs) return false;
     const int64_t NBf = B + (want_base ? 1 : 0);
     const int64_t n_groups = (NBf + 31) / 32;
@@ -576,21 +599,22 @@ bool flow_plan(const emo_graph *g, int64_t B, bool want_base, bool need_bwd, Flo
         // four producer warps where the block has room for them (they share the level-row pieces)
         const int nprod = G * f.lanes + 4 <= 24 ? 4 : 2;
         const size_t P = 32 * (size_t)G;
-        const size_t lvl_bytes = (size_t)G * f.lanes * f.K * 32;
+        const size_t lvl_bytes = intv ? 0 : (size_t)G * f.lanes * f.K * 32;
+        const size_t extra = intv ? round_up(extra_fixed + extra_per_group * G, 128) : 0;
         auto shape = [&](bool backward, FlowParams &p, size_t &smem) {
             const FlowDir &dir = backward ? f.b : f.f;
             const size_t slot_bytes = (size_t)dir.slots_tag * 256 + (size_t)dir.slots_set * 128;
-            const size_t blob = backward ? d.blobB_bytes : d.blobF_bytes;
+            const size_t blob = backward ? d.blobB_bytes : (intv ? d.blobFI_bytes : d.blobF_bytes);
             const size_t rst = backward ? (size_t)d.max_push * P * 4 : 0;
             const size_t stage = round_up(blob + lvl_bytes + rst, 128);
             const size_t off_bar = round_up(G * slot_bytes, 16);
-            const size_t head = round_up(off_bar + 256, 128);
+            const size_t head = round_up(off_bar + 256, 128) + extra;
             int nbuf = 0;
             for (int nb = 3; nb >= 2; --nb)
                 if (head + nb * stage <= budget) { nbuf = nb; break; }
             if (!nbuf || nbuf * stage < (size_t)G * f.lanes * 32 * 16) return false;
             p = FlowParams();
-            p.blob = backward ? d.blobB : d.blobF;
+            p.blob = backward ? d.blobB : (intv ? d.blobFI : d.blobF);
             p.rows = d.rows;
             p.push_base = d.push_base;
             p.blob_bytes = (unsigned)blob;
@@ -599,6 +623,9 @@ bool flow_plan(const emo_graph *g, int64_t B, bool want_base, bool need_bwd, Flo
             p.off_pool = backward ? d.b_off_pool : d.f_off_pool;
             p.off_tab = backward ? d.b_off_tab : d.f_off_tab;
             p.off_lbes = backward ? d.b_off_lbes : 0;
+            p.off_meta = d.f_off_meta;
+            p.off_brk = (unsigned)round_up(off_bar + 256, 128);
+            p.off_Fs = p.off_brk + (unsigned)round_up(extra_fixed, 16);
             p.tab_row = (unsigned)f.Lp * (backward ? 4u : 12u);
             p.stages = f.stages;
             p.lanes = f.lanes;
@@ -666,7 +693,7 @@ int launch_flow_fwd(const emo_graph *g, const FlowPlan &pl, int64_t B, const uin
     if (flags & EMO_F_TEST_STALL) p.stall_stage = p.stages / 2;
     cudaEvent_t ev0 = g_pass_events[0], ev1 = g_pass_events[1];
     if (ev0) EMO_CUDA(cudaEventRecord(ev0, st));
-    void (*kern)(FlowParams) = pl.threads <= 512 ? emo_flow_fwd<512> : (pl.threads <= 768 ? emo_flow_fwd<768> : emo_flow_fwd<1024>);
+    void (*kern)(FlowParams) = pl.threads <= 512 ? emo_flow_fwd<512, false> : (pl.threads <= 768 ? emo_flow_fwd<768, false> : emo_flow_fwd<1024, false>);
     if (flow_optin(kern, g) != EMO_OK) { (void)cudaGetLastError(); return EMO_E_CUDA; }
     kern<<<pl.grid_f, pl.threads, pl.smem_f, st>>>(p);
     EMO_CUDA(cudaGetLastError());
@@ -991,7 +1018,7 @@ int emo_graph_load(int32_t n, const int64_t *row_ptr, const int32_t *col, const 
             rc = upload_program_lane(g->fwd, g->lfwd);
             if (rc == EMO_OK) rc = upload_program_lane(g->bwd, g->lbwd);
         }
-        if (rc == EMO_OK) rc = upload_flow(g->flow, g->dflow);
+        if (rc == EMO_OK) rc = upload_flow(g->flow, g->dflow, (flags & EMO_F_INTERVALS) != 0);
         } catch (const std::bad_alloc &) {
             rc = EMO_E_OOM;
         }
@@ -1211,7 +1238,37 @@ int emo_eval_intervals(const emo_graph *g, int64_t B, const uint8_t *F, int64_t 
         if (breaks[i] != (int64_t)i * delta) delta = 0;
     cudaEvent_t ev0 = g_pass_events[0], ev1 = g_pass_events[1];
     if (ev0) EMO_CUDA(cudaEventRecord(ev0, st));
-    {
+    bool done = false;
+    if (!(flags & EMO_F_NO_STAGING) && g->dflow.blobFI && delta > 0) {
+        // the lane-stream forward kernel with the look-up inside the chain: uniform grids, F's columns in shared memory
+        FlowPlan fp;
+        const size_t brk_b = round_up((size_t)I * 8, 16), f_per_group = (size_t)rows * (size_t)I * 32;
+        if (flow_plan(g, B, false, false, fp, true, brk_b, f_per_group)) {
+            FlowParams q = fp.pf;
+            q.B = B;
+            q.lvl = nullptr;
+            q.ldb = 0;
+            q.restore = nullptr;
+            q.makespan = makespan;
+            q.energy = energy;
+            q.status = status;
+            q.F = F;
+            q.ldF = ldb;
+            q.I = I;
+            q.rowsF = rows;
+            q.delta = delta;
+            q.inv_mean = inv_mean;
+            q.breaks = (const long long *)d_breaks;
+            q.busy = busy;
+            q.ldw = ldw;
+            void (*kern)(FlowParams) = fp.threads <= 512 ? emo_flow_fwd<512, true> : (fp.threads <= 768 ? emo_flow_fwd<768, true> : emo_flow_fwd<1024, true>);
+            if (flow_optin(kern, g) != EMO_OK) { (void)cudaGetLastError(); return EMO_E_CUDA; }
+            kern<<<fp.grid_f, fp.threads, fp.smem_f, st>>>(q);
+            EMO_CUDA(cudaGetLastError());
+            done = true;
+        }
+    }
+    if (!done) {
     const Program &p = g->fwd;
     const DevProgram &d = g->dfwd;
     if (p.steps == 0) return EMO_E_UNSUPPORTED;

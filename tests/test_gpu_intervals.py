@@ -48,12 +48,15 @@ def run_gpu(torch, emo, g, dev_of, breaks, F, p_idle, flags=0, ldb=None, call_fl
 
 
 def check(torch, emo, oracle_mod, g, dev_of, breaks, F, p_idle, flags=0, **kw):
+    """Both forms of the evaluation: the lane-stream kernel (graph loaded with EMO_F_INTERVALS; uniform grids) and
+    the step-program kernel (without the flag, and with EMO_F_NO_STAGING on the prepared handle)."""
     r = oracle_mod.intervals(g, dev_of, breaks, F, p_idle)
-    T, E, Ei = run_gpu(torch, emo, g, dev_of, breaks, F, p_idle, flags=flags, **kw)
-    assert np.array_equal(T, r["makespan"])
-    assert np.allclose(E, r["energy"], rtol=1e-9, atol=0)
-    if p_idle is not None:
-        assert np.allclose(Ei, r["e_idle"], rtol=1e-9, atol=1e-30)
+    for load_flags, call_flags in ((emo.EMO_F_INTERVALS, 0), (0, 0), (emo.EMO_F_INTERVALS, emo.EMO_F_NO_STAGING)):
+        T, E, Ei = run_gpu(torch, emo, g, dev_of, breaks, F, p_idle, flags=flags | load_flags, call_flags=call_flags, **kw)
+        assert np.array_equal(T, r["makespan"]), (load_flags, call_flags)
+        assert np.allclose(E, r["energy"], rtol=1e-9, atol=0), (load_flags, call_flags)
+        if p_idle is not None:
+            assert np.allclose(Ei, r["e_idle"], rtol=1e-9, atol=1e-30), (load_flags, call_flags)
 
 
 def test_hand_worked_example_on_gpu(torch_cuda, emo, oracle_mod):
@@ -72,6 +75,8 @@ def test_random_dags(torch_cuda, emo, oracle_mod, seed):
     check(torch_cuda, emo, oracle_mod, g, dev_of, breaks, F, p_idle)
     check(torch_cuda, emo, oracle_mod, g, dev_of, breaks, F, None)
     check(torch_cuda, emo, oracle_mod, g, dev_of, [0], F[:, :1, :].copy(), p_idle)          # one interval
+    check(torch_cuda, emo, oracle_mod, g, dev_of, np.arange(7, dtype=np.int64) * 23, F, p_idle)      # uniform grid
+    check(torch_cuda, emo, oracle_mod, g, dev_of, np.arange(7, dtype=np.int64) * 5, F, p_idle)       # packs span several intervals
     check(torch_cuda, emo, oracle_mod, g, dev_of, breaks, F, p_idle, flags=emo.EMO_F_LANES(1))
     check(torch_cuda, emo, oracle_mod, g, dev_of, breaks, F, p_idle, flags=emo.EMO_F_LANES(3) | emo.EMO_F_FLOW_SYNC(8))
 
@@ -120,4 +125,31 @@ def test_argument_errors(torch_cuda, emo):
     with pytest.raises(Exception):      # workspace too small
         emo.emo_eval_intervals(h, B, F, 16, I, np.array([0, 4, 9], np.int64), None, T, E, None, ws[:8])
     emo.emo_eval_intervals(h, 0, None, 0, I, np.array([0, 4, 9], np.int64), None, None, None, None, ws)      # B = 0: nothing to do
+    h.free()
+
+
+def test_large_batch_sampled(torch_cuda, emo, oracle_mod):
+    """A batch that fills every block with four policy groups (the launch shape of the bench), on the lane-stream
+    form; a sample of its columns against the oracle."""
+    torch = torch_cuda
+    g = W.make_graph("cfg4-llm", 0.1)
+    dev_of = W.device_of(g)
+    B, D = 16384, 1
+    T0 = int(oracle_mod.batch(g, np.full((g.n, 1), g.L - 1, np.uint8))["makespan"][0])
+    I = int(T0 * 1.05 / 20e6) + 1
+    breaks = W.interval_breaks(T0, I)
+    F = W.interval_policies(g.meta["policy_seed"], D, I, g.L, B, device="cuda")
+    h = emo.load_workload(g, flags=emo.EMO_F_INTERVALS, group_of=dev_of)
+    T = torch.zeros(B, dtype=torch.int64, device="cuda")
+    E = torch.zeros(B, dtype=torch.float64, device="cuda")
+    Ei = torch.zeros(B, dtype=torch.float64, device="cuda")
+    pi = torch.from_numpy(W.idle_power(g.L)).cuda()
+    ws = torch.empty(emo.emo_workspace_bytes_intervals(h, B, I, True), dtype=torch.uint8, device="cuda")
+    emo.emo_eval_intervals(h, B, F, F.shape[2], I, breaks, pi, T, E, Ei, ws)
+    torch.cuda.synchronize()
+    cols = np.array([0, 1, 31, 32, 4095, 8192, 16383])
+    r = oracle_mod.intervals(g, dev_of, breaks, F[:, :, torch.as_tensor(cols, device="cuda")].cpu().numpy(), W.idle_power(g.L))
+    assert np.array_equal(T.cpu().numpy()[cols], r["makespan"])
+    assert np.allclose(E.cpu().numpy()[cols], r["energy"], rtol=1e-9, atol=0)
+    assert np.allclose(Ei.cpu().numpy()[cols], r["e_idle"], rtol=1e-9, atol=1e-30)
     h.free()
