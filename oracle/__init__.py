@@ -61,6 +61,10 @@ def lib():
         L.emo_oracle_intervals.restype = ctypes.c_int
         L.emo_oracle_search_dp.argtypes = [i32, p, p, i32, p, p, p, i32, i32, p, p, i64, i64, p, p, p, p, p]
         L.emo_oracle_search_dp.restype = ctypes.c_int
+        L.emo_oracle_crit_pred.argtypes = [i32, p, p, p, p, p]
+        L.emo_oracle_crit_pred.restype = ctypes.c_int
+        L.emo_oracle_pack_greedy.argtypes = [i32, p, p, p, p, p, p, i64, p, p]
+        L.emo_oracle_pack_greedy.restype = ctypes.c_int
         _lib = L
     return _lib
 
@@ -224,3 +228,29 @@ def search_dp(g, dev_of, breaks, p_idle, T_max: int, bin_ns: int = 1):
     if rc:
         raise OracleError(f"emo_oracle_search_dp failed with {rc}")
     return {"found": bool(found.value), "F": F, "T": int(T.value), "E": float(E.value), "n_pred": int(calls.value)}
+
+
+def crit_pred(g, dur):
+    """Eq. 5 with Alg. 1's tie rule.  dur: int64 [n].  Returns (C int64 [n], crit int32 [n])."""
+    row_ptr, col = _c(g.row_ptr, np.int64), _c(g.col, np.int32)
+    dur = _c(dur, np.int64)
+    C = np.zeros(g.n, np.int64)
+    crit = np.zeros(g.n, np.int32)
+    rc = lib().emo_oracle_crit_pred(g.n, _ptr(row_ptr), _ptr(col), _ptr(dur), _ptr(C), _ptr(crit))
+    if rc:
+        raise OracleError(f"emo_oracle_crit_pred failed with {rc}")
+    return C, crit
+
+
+def pack_greedy(g, is_kernel, stream_of, t_default, crit, delta_max: int):
+    """Dependency-aware greedy packing.  Returns (pack_of int32 [n], number of packs)."""
+    row_ptr, col = _c(g.row_ptr, np.int64), _c(g.col, np.int32)
+    isk, so = _c(is_kernel, np.uint8), _c(stream_of, np.int32)
+    td, cr = _c(t_default, np.int64), _c(crit, np.int32)
+    pack_of = np.zeros(g.n, np.int32)
+    cnt = ctypes.c_int32(0)
+    rc = lib().emo_oracle_pack_greedy(g.n, _ptr(row_ptr), _ptr(col), _ptr(isk), _ptr(so), _ptr(td), _ptr(cr), int(delta_max),
+                                      _ptr(pack_of), ctypes.byref(cnt))
+    if rc:
+        raise OracleError(f"emo_oracle_pack_greedy failed with {rc}")
+    return pack_of, int(cnt.value)

@@ -20,6 +20,8 @@
  *                                              the budget is a fraction of it (2 %, 5 % in Sec. 5)
  *   selection ................................ Eq. 4 over a finite candidate set, with the feasibility
  *                                              and strict-improvement test of Alg. 2 (first best kept)
+ *   critical predecessors, packing ........... Eq. 5 with Alg. 1's update rule; the dependency-aware greedy packing of
+ *                                              Sec. 4.4 (three rules, its listing restated)
  *   policy search ............................ Alg. 2 (dynamic programming over the intervals, one prediction per
  *                                              candidate); a heuristic, pinned only in part: see its comment
  *   time-interval policies and idle energy ... Alg. 1 as printed (level from the interval that holds the
@@ -497,4 +499,133 @@ done:
     free(cur); free(nxt); free(Fd); free(P2);
     return rc;
 #undef PRED
+}
+
+/* ------------------------------------------------------------------------------------------------
+ * Eq. 5: the critical predecessor k*_v = argmax over predecessors of C_k, tracked as Alg. 1 does it:
+ * every finished node offers itself to its successors and replaces their entry only if it finishes
+ * strictly later, so among equals the predecessor that is processed first stays.
+ *
+ * Reading: nodes are processed in index order (the caller's numbering must be topological: every
+ * predecessor has a lower index), which makes "processed first" = "lowest index".  dur[v] is the
+ * duration of v under the policy in question (the default frequency for packing).
+ * Outputs: C[v] completion times, crit[v] = k*_v or -1 for a node without predecessors.
+ * ------------------------------------------------------------------------------------------------ */
+int emo_oracle_crit_pred(int32_t n, const int64_t *row_ptr, const int32_t *col, const int64_t *dur,
+                         int64_t *C, int32_t *crit)
+{
+    if (n < 0) return ORACLE_E_ARG;
+    for (int32_t v = 0; v < n; ++v) crit[v] = -1;
+    /* successor lists */
+    int64_t m = n > 0 ? row_ptr[n] : 0;
+    int64_t *sp = calloc((size_t)n + 2, sizeof *sp);
+    int32_t *sc = malloc(sizeof *sc * (size_t)(m > 0 ? m : 1));
+    int64_t *fill = malloc(sizeof *fill * (size_t)(n > 0 ? n : 1));
+    if (!sp || !sc || !fill) { free(sp); free(sc); free(fill); return ORACLE_E_NOMEM; }
+    for (int32_t v = 0; v < n; ++v)
+        for (int64_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e) {
+            if (col[e] >= v) { free(sp); free(sc); free(fill); return ORACLE_E_CYCLE; }
+            sp[col[e] + 1]++;
+        }
+    for (int32_t v = 0; v < n; ++v) sp[v + 1] += sp[v];
+    memcpy(fill, sp, sizeof *fill * (size_t)n);
+    for (int32_t v = 0; v < n; ++v)
+        for (int64_t e = row_ptr[v]; e < row_ptr[v + 1]; ++e) sc[fill[col[e]]++] = v;
+    for (int32_t v = 0; v < n; ++v) {
+        int64_t start = crit[v] >= 0 ? C[crit[v]] : 0;
+        C[v] = start + dur[v];
+        for (int64_t s = sp[v]; s < sp[v + 1]; ++s) {
+            int32_t u = sc[s];
+            if (crit[u] < 0 || C[v] > C[crit[u]]) crit[u] = v;
+        }
+    }
+    free(sp); free(sc); free(fill);
+    return ORACLE_OK;
+}
+
+/* ------------------------------------------------------------------------------------------------
+ * Dependency-aware greedy packing (Sec. 4.4, its listing): walk the kernels of one stream in order and
+ * keep adding the next kernel v to the current pack (last member u) while
+ *   rule 1  v and its critical predecessor are in the same stream,
+ *   rule 2  every critical successor of u is in u's stream,
+ *   rule 3  the pack's duration at the default frequency plus t_v stays below delta_max (strict);
+ * otherwise the pack is closed and v starts a new one.
+ *
+ * Readings: the listing's sorted kernel list V is taken per (device, stream): a pack is a stretch of one
+ * stream (the rules speak of "the same stream", and only the first member's incoming and the last
+ * member's outgoing dependencies survive, which presupposes that the members follow each other on one
+ * stream); kernels are visited in index order; a node that is not a GPU kernel (is_kernel[v] = 0) is in
+ * no pack and in no stream, so a kernel whose critical predecessor is a launch or a collective starts a
+ * new pack; a kernel without predecessors has no critical predecessor and fails rule 1.
+ * stream_of[v] identifies the stream globally (device and stream together).
+ * Output: pack_of[v] = pack number (0, 1, ... in order of their first member) or -1; returns the count
+ * in *n_packs.
+ * ------------------------------------------------------------------------------------------------ */
+int emo_oracle_pack_greedy(int32_t n, const int64_t *row_ptr, const int32_t *col, const uint8_t *is_kernel,
+                           const int32_t *stream_of, const int64_t *t_default, const int32_t *crit,
+                           int64_t delta_max, int32_t *pack_of, int32_t *n_packs)
+{
+    if (n < 0) return ORACLE_E_ARG;
+    (void)row_ptr; (void)col;
+    int32_t max_stream = -1;
+    for (int32_t v = 0; v < n; ++v) {
+        pack_of[v] = -1;
+        if (is_kernel[v] && stream_of[v] > max_stream) max_stream = stream_of[v];
+    }
+    /* rule 2 needs, for every node, whether all its critical successors share its stream */
+    uint8_t *succ_ok = malloc((size_t)(n > 0 ? n : 1));
+    if (!succ_ok) return ORACLE_E_NOMEM;
+    for (int32_t v = 0; v < n; ++v) succ_ok[v] = 1;
+    for (int32_t v = 0; v < n; ++v) {
+        int32_t k = crit[v];
+        if (k < 0 || !is_kernel[k]) continue;
+        if (!is_kernel[v] || stream_of[v] != stream_of[k]) succ_ok[k] = 0;
+    }
+    /* pack numbers are handed out in order of the first member's index: collect (first member) per pack */
+    int32_t *first = malloc(sizeof *first * (size_t)(n > 0 ? n : 1));
+    int32_t *tmp_pack = malloc(sizeof *tmp_pack * (size_t)(n > 0 ? n : 1));
+    if (!first || !tmp_pack) { free(succ_ok); free(first); free(tmp_pack); return ORACLE_E_NOMEM; }
+    int32_t count = 0;
+    for (int32_t s = 0; s <= max_stream; ++s) {
+        int32_t u = -1;            /* last node in the current pack */
+        int64_t dur_pack = 0;
+        for (int32_t v = 0; v < n; ++v) {
+            if (!is_kernel[v] || stream_of[v] != s) continue;
+            int ok = 0;
+            if (u >= 0) {
+                int r1 = crit[v] >= 0 && is_kernel[crit[v]] && stream_of[crit[v]] == stream_of[v];
+                int r2 = succ_ok[u];
+                int r3 = dur_pack + t_default[v] < delta_max;
+                ok = r1 && r2 && r3;
+            }
+            if (ok) {
+                tmp_pack[v] = tmp_pack[u];
+                dur_pack += t_default[v];
+            } else {
+                first[count] = v;
+                tmp_pack[v] = count++;
+                dur_pack = t_default[v];
+            }
+            u = v;
+        }
+    }
+    /* renumber by first member */
+    {
+        int32_t *order = malloc(sizeof *order * (size_t)(count > 0 ? count : 1));
+        int32_t *newid = malloc(sizeof *newid * (size_t)(count > 0 ? count : 1));
+        if (!order || !newid) { free(order); free(newid); free(succ_ok); free(first); free(tmp_pack); return ORACLE_E_NOMEM; }
+        for (int32_t p = 0; p < count; ++p) order[p] = p;
+        for (int32_t i = 1; i < count; ++i) {          /* insertion sort by first member */
+            int32_t x = order[i], j = i - 1;
+            while (j >= 0 && first[order[j]] > first[x]) { order[j + 1] = order[j]; --j; }
+            order[j + 1] = x;
+        }
+        for (int32_t i = 0; i < count; ++i) newid[order[i]] = i;
+        for (int32_t v = 0; v < n; ++v)
+            if (is_kernel[v]) pack_of[v] = newid[tmp_pack[v]];
+        free(order); free(newid);
+    }
+    if (n_packs) *n_packs = count;
+    free(succ_ok); free(first); free(tmp_pack);
+    return ORACLE_OK;
 }
