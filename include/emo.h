@@ -184,6 +184,37 @@ int emo_eval_intervals(const emo_graph *g, int64_t B, const uint8_t *F, int64_t 
 int emo_workspace_bytes_intervals(const emo_graph *g, int64_t B, int32_t I, int with_idle, size_t *out);
 
 /*
+ * emo_pack_greedy - kernel packing (Sec. 4.4): the critical predecessor of every node at the default frequency
+ * (Eq. 5: k*_v = argmax over predecessors of C_k; among equals the lowest index, the one Alg. 1's update meets
+ * first) and the dependency-aware greedy packing of GPU kernels.  The kernels of every stream are walked in
+ * index order; kernel v joins the open pack of its stream (last member u) while (1) v's critical predecessor is
+ * a kernel of v's stream, (2) every node whose critical predecessor is u is a kernel of u's stream, and (3) the
+ * pack's duration at the default frequency plus t_v stays below delta_max; otherwise v opens a new pack.
+ * Host function, host arrays; nothing touches a device.
+ *   row_ptr, col   predecessor CSR in a topological numbering (every predecessor has a lower index).
+ *   is_kernel      uint8 [n]: 1 for GPU kernels (only they are packed).
+ *   stream_of      int32 [n]: global stream id (device and stream together) of every kernel, >= 0; ignored elsewhere.
+ *   t_default      int64 [n]: durations at the default frequency, ns.
+ *   delta_max      granularity bound in ns (the paper uses 5 ms).
+ *   crit_out       int32 [n], optional: the critical predecessors (-1: none).
+ *   pack_of        int32 [n]: pack number of every kernel (0, 1, ... in order of the packs' first members), -1
+ *                  for other nodes.  Usable as group_of of emo_graph_load for per-pack policies after the
+ *                  non-kernel nodes are given rows of their own (or -1).
+ *   n_packs        number of packs.
+ * Errors: EMO_E_INVALID_ARG, EMO_E_NOT_TOPOLOGICAL, EMO_E_RANGE (negative duration), EMO_E_OOM.
+ */
+int emo_pack_greedy(int32_t n, const int64_t *row_ptr, const int32_t *col, const uint8_t *is_kernel,
+                    const int32_t *stream_of, const int64_t *t_default, int64_t delta_max, int32_t *crit_out,
+                    int32_t *pack_of, int32_t *n_packs);
+/*
+ * emo_pack_tables - the packs' frequency tables: per level the sum of the members' table entries (a pack's
+ * kernels run one after the other on their stream).  pack_lat int64 [n_packs][L], pack_energy fp64 [n_packs][L];
+ * members are added in index order.  Host function.
+ */
+int emo_pack_tables(int32_t n, int32_t L, const int64_t *lat, const double *energy, const int32_t *pack_of,
+                    int32_t n_packs, int64_t *pack_lat, double *pack_energy);
+
+/*
  * emo_search_dp - Alg. 2: search for a near-optimal time-interval policy by dynamic programming over the
  * intervals, with emo_eval_intervals (Alg. 1) as the predictor.  dp[i] maps an end-to-end time to the least
  * energy and its policy after the first i intervals are decided; every state is extended by every level in

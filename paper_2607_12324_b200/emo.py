@@ -31,7 +31,7 @@ EXPORTS = [
     "emo_strerror", "emo_graph_load", "emo_graph_free", "emo_graph_info", "emo_workspace_bytes",
     "emo_eval_policies", "emo_slack_batch", "emo_slack", "emo_baseline", "emo_target_from_delta",
     "emo_select", "emo_transpose_policies", "emo_slack_batch_host", "emo_graph_program",
-    "emo_set_pass_events", "emo_select_static", "emo_graph_flow", "emo_set_wait_limit", "emo_call_path", "emo_set_flow_counters", "emo_workspace_bytes_for", "emo_measure_int_issue", "emo_measure_warp_costs", "emo_eval_intervals", "emo_workspace_bytes_intervals", "emo_search_dp", "emo_workspace_bytes_search", "emo_pack_levels", "emo_unpack_levels", "emo_slack_batch_host_packed",
+    "emo_set_pass_events", "emo_select_static", "emo_graph_flow", "emo_set_wait_limit", "emo_call_path", "emo_set_flow_counters", "emo_workspace_bytes_for", "emo_measure_int_issue", "emo_measure_warp_costs", "emo_eval_intervals", "emo_workspace_bytes_intervals", "emo_search_dp", "emo_workspace_bytes_search", "emo_pack_greedy", "emo_pack_tables", "emo_pack_levels", "emo_unpack_levels", "emo_slack_batch_host_packed",
 ]
 
 
@@ -116,6 +116,8 @@ def lib():
         L.emo_workspace_bytes_intervals.argtypes = [p, i64, i32, ctypes.c_int, p]
         L.emo_search_dp.argtypes = [p, i32, p, p, i64, i64, i64, p, p, p, p, p, p, ctypes.c_size_t, p]
         L.emo_workspace_bytes_search.argtypes = [p, i32, i64, ctypes.c_int, p]
+        L.emo_pack_greedy.argtypes = [i32, p, p, p, p, p, i64, p, p, p]
+        L.emo_pack_tables.argtypes = [i32, i32, p, p, p, i32, p, p]
         L.emo_pack_levels.argtypes = [ctypes.c_int, i64, i64, p, i64, p, i64, p]
         L.emo_unpack_levels.argtypes = [ctypes.c_int, i64, i64, p, i64, p, i64, p]
         L.emo_slack_batch_host_packed.argtypes = [p, i64, ctypes.c_int, p, i64, p, p, i64, p, i64, i64, p, p, p, p, p, p, sz, u32, p]
@@ -413,6 +415,34 @@ def emo_search_dp(g, breaks, p_idle, T_max, bin_ns, ws, max_batch=0, stream=None
                                F.ctypes.data_as(ctypes.c_void_p), ctypes.byref(T), ctypes.byref(E), ctypes.byref(calls),
                                ctypes.byref(found), _addr(ws), _nbytes(ws), _stream(stream)), "emo_search_dp")
     return {"found": bool(found.value), "F": F, "T": int(T.value), "E": float(E.value), "n_pred": int(calls.value)}
+
+
+def emo_pack_greedy(n, row_ptr, col, is_kernel, stream_of, t_default, delta_max):
+    """Host arrays in, (crit, pack_of, n_packs) out (see include/emo.h)."""
+    rp = np.ascontiguousarray(row_ptr, np.int64)
+    cl = np.ascontiguousarray(col, np.int32)
+    isk = np.ascontiguousarray(is_kernel, np.uint8)
+    so = np.ascontiguousarray(stream_of, np.int32)
+    td = np.ascontiguousarray(t_default, np.int64)
+    crit = np.zeros(int(n), np.int32)
+    pack_of = np.zeros(int(n), np.int32)
+    cnt = ctypes.c_int32(0)
+    vp = lambda a: a.ctypes.data_as(ctypes.c_void_p)
+    _check(lib().emo_pack_greedy(int(n), vp(rp), vp(cl), vp(isk), vp(so), vp(td), int(delta_max), vp(crit), vp(pack_of),
+                                 ctypes.byref(cnt)), "emo_pack_greedy")
+    return crit, pack_of, int(cnt.value)
+
+
+def emo_pack_tables(lat, energy, pack_of, n_packs):
+    lt = np.ascontiguousarray(lat, np.int64)
+    en = np.ascontiguousarray(energy, np.float64)
+    po = np.ascontiguousarray(pack_of, np.int32)
+    n, L = lt.shape
+    pl = np.zeros((int(n_packs), L), np.int64)
+    pe = np.zeros((int(n_packs), L), np.float64)
+    vp = lambda a: a.ctypes.data_as(ctypes.c_void_p)
+    _check(lib().emo_pack_tables(int(n), int(L), vp(lt), vp(en), vp(po), int(n_packs), vp(pl), vp(pe)), "emo_pack_tables")
+    return pl, pe
 
 
 def emo_pack_levels(bits, rows, B, lvl, ldb, packed, ldp, stream=None):
