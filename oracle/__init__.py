@@ -61,6 +61,10 @@ def lib():
         L.emo_oracle_intervals.restype = ctypes.c_int
         L.emo_oracle_search_dp.argtypes = [i32, p, p, i32, p, p, p, i32, i32, p, p, i64, i64, p, p, p, p, p]
         L.emo_oracle_search_dp.restype = ctypes.c_int
+        L.emo_oracle_nnls.argtypes = [i32, i32, p, p, p, p]
+        L.emo_oracle_nnls.restype = ctypes.c_int
+        L.emo_oracle_pack_model.argtypes = [i32, i32, i32, i32, p, p, p, p, p, p, p]
+        L.emo_oracle_pack_model.restype = ctypes.c_int
         L.emo_oracle_crit_pred.argtypes = [i32, p, p, p, p, p]
         L.emo_oracle_crit_pred.restype = ctypes.c_int
         L.emo_oracle_pack_greedy.argtypes = [i32, p, p, p, p, p, p, i64, p, p]
@@ -254,3 +258,28 @@ def pack_greedy(g, is_kernel, stream_of, t_default, crit, delta_max: int):
     if rc:
         raise OracleError(f"emo_oracle_pack_greedy failed with {rc}")
     return pack_of, int(cnt.value)
+
+
+def nnls(B, b):
+    """Eq. 6 for one pack: argmin ||B x - b||^2, x >= 0.  Returns (x, squared residual)."""
+    B = _c(B, np.float64)
+    b = _c(b, np.float64)
+    n, m = B.shape
+    x = np.zeros(m, np.float64)
+    r2 = ctypes.c_double(0.0)
+    rc = lib().emo_oracle_nnls(n, m, _ptr(B), _ptr(b), _ptr(x), ctypes.byref(r2))
+    if rc:
+        raise OracleError(f"emo_oracle_nnls failed with {rc}")
+    return x, float(r2.value)
+
+
+def pack_model(B, feat, Tb, Eb):
+    """Eq. 6 and Eq. 7 for every pack.  feat [packs][n], Tb / Eb [m][L].  Returns (x, T, E)."""
+    B, feat, Tb, Eb = _c(B, np.float64), _c(feat, np.float64), _c(Tb, np.float64), _c(Eb, np.float64)
+    n, m = B.shape
+    P, L = feat.shape[0], Tb.shape[1]
+    x = np.zeros((P, m)); T = np.zeros((P, L)); E = np.zeros((P, L))
+    rc = lib().emo_oracle_pack_model(P, n, m, L, _ptr(B), _ptr(feat), _ptr(Tb), _ptr(Eb), _ptr(x), _ptr(T), _ptr(E))
+    if rc:
+        raise OracleError(f"emo_oracle_pack_model failed with {rc}")
+    return x, T, E

@@ -22,6 +22,8 @@
  *                                              and strict-improvement test of Alg. 2 (first best kept)
  *   critical predecessors, packing ........... Eq. 5 with Alg. 1's update rule; the dependency-aware greedy packing of
  *                                              Sec. 4.4 (three rules, its listing restated)
+ *   pack modelling ........................... Eq. 6 (non-negative least squares, by its definition over all
+ *                                              supports) and Eq. 7 (tables as weighted sums)
  *   policy search ............................ Alg. 2 (dynamic programming over the intervals, one prediction per
  *                                              candidate); a heuristic, pinned only in part: see its comment
  *   time-interval policies and idle energy ... Alg. 1 as printed (level from the interval that holds the
@@ -627,5 +629,99 @@ int emo_oracle_pack_greedy(int32_t n, const int64_t *row_ptr, const int32_t *col
     }
     if (n_packs) *n_packs = count;
     free(succ_ok); free(first); free(tmp_pack);
+    return ORACLE_OK;
+}
+
+/* ------------------------------------------------------------------------------------------------
+ * Pack modelling (Sec. 4.5): a pack's feature vector b (n metrics at the default frequency) is
+ * written as a non-negative combination of m micro-benchmarks, x = argmin ||B x - b||^2 subject to
+ * x >= 0 (Eq. 6), and its tables follow as T_f[P] = sum_i x_i T_f[B_i], E_f[P] = sum_i x_i E_f[B_i]
+ * (Eq. 7).
+ *
+ * The minimiser has a plain definition, and that is what is written out here: every subset S of the m
+ * columns is tried, the unconstrained least-squares solution on S is computed (normal equations,
+ * Cholesky, long double), subsets whose solution has a negative entry or whose columns are dependent
+ * are skipped, and the feasible candidate of least residual wins (ties: the first subset in counting
+ * order).  The constrained optimum is among the candidates and every candidate is a feasible point, so
+ * the least residual is the optimum.  Exponential in m (m <= 16): for tests only.
+ * ------------------------------------------------------------------------------------------------ */
+int emo_oracle_nnls(int32_t n, int32_t m, const double *B /*[n][m]*/, const double *b /*[n]*/, double *x /*[m]*/, double *resid2)
+{
+    if (n < 1 || m < 1 || m > 16) return ORACLE_E_ARG;
+    long double G[16][16], c[16], bb = 0.0L;
+    for (int i = 0; i < m; ++i) {
+        c[i] = 0.0L;
+        for (int r = 0; r < n; ++r) c[i] += (long double)B[r * m + i] * b[r];
+        for (int j = 0; j < m; ++j) {
+            G[i][j] = 0.0L;
+            for (int r = 0; r < n; ++r) G[i][j] += (long double)B[r * m + i] * B[r * m + j];
+        }
+    }
+    for (int r = 0; r < n; ++r) bb += (long double)b[r] * b[r];
+    long double best = bb;              /* the empty subset: x = 0 */
+    for (int i = 0; i < m; ++i) x[i] = 0.0;
+    for (uint32_t S = 1; S < (1u << m); ++S) {
+        int idx[16], k = 0;
+        for (int i = 0; i < m; ++i)
+            if (S & (1u << i)) idx[k++] = i;
+        /* Cholesky of G_SS */
+        long double Lc[16][16], z[16], y[16];
+        int ok = 1;
+        for (int i = 0; i < k && ok; ++i)
+            for (int j = 0; j <= i; ++j) {
+                long double s = G[idx[i]][idx[j]];
+                for (int q = 0; q < j; ++q) s -= Lc[i][q] * Lc[j][q];
+                if (i == j) {
+                    if (s <= 1e-18L * G[idx[i]][idx[i]]) { ok = 0; break; }      /* dependent columns */
+                    Lc[i][i] = sqrtl(s);
+                } else {
+                    Lc[i][j] = s / Lc[j][j];
+                }
+            }
+        if (!ok) continue;
+        for (int i = 0; i < k; ++i) {
+            long double s = c[idx[i]];
+            for (int q = 0; q < i; ++q) s -= Lc[i][q] * y[q];
+            y[i] = s / Lc[i][i];
+        }
+        for (int i = k - 1; i >= 0; --i) {
+            long double s = y[i];
+            for (int q = i + 1; q < k; ++q) s -= Lc[q][i] * z[q];
+            z[i] = s / Lc[i][i];
+        }
+        int feas = 1;
+        for (int i = 0; i < k; ++i)
+            if (z[i] < 0.0L) { feas = 0; break; }
+        if (!feas) continue;
+        /* residual^2 = b.b - 2 c_S.z + z.G_SS.z = b.b - c_S.z at the least-squares solution */
+        long double r2 = bb;
+        for (int i = 0; i < k; ++i) r2 -= c[idx[i]] * z[i];
+        if (r2 < best) {
+            best = r2;
+            for (int i = 0; i < m; ++i) x[i] = 0.0;
+            for (int i = 0; i < k; ++i) x[idx[i]] = (double)z[i];
+        }
+    }
+    if (resid2) *resid2 = (double)(best > 0.0L ? best : 0.0L);
+    return ORACLE_OK;
+}
+
+/* Eq. 6 for every pack, then Eq. 7: T_out, E_out [n_packs][L] from the micro-benchmark tables Tb, Eb [m][L]. */
+int emo_oracle_pack_model(int32_t n_packs, int32_t n, int32_t m, int32_t L, const double *B, const double *feat /*[n_packs][n]*/,
+                          const double *Tb, const double *Eb, double *x /*[n_packs][m]*/, double *T_out, double *E_out)
+{
+    for (int32_t p = 0; p < n_packs; ++p) {
+        int rc = emo_oracle_nnls(n, m, B, feat + (int64_t)p * n, x + (int64_t)p * m, NULL);
+        if (rc) return rc;
+        for (int32_t l = 0; l < L; ++l) {
+            double t = 0.0, e = 0.0;
+            for (int32_t i = 0; i < m; ++i) {
+                t += x[(int64_t)p * m + i] * Tb[(int64_t)i * L + l];
+                e += x[(int64_t)p * m + i] * Eb[(int64_t)i * L + l];
+            }
+            T_out[(int64_t)p * L + l] = t;
+            E_out[(int64_t)p * L + l] = e;
+        }
+    }
     return ORACLE_OK;
 }

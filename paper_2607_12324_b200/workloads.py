@@ -711,3 +711,32 @@ def idle_power(L: int) -> np.ndarray:
     """fp64 [L] watts: idle power at each level, rising with the frequency (synthetic: 60 W + 40 W * f / f_max)."""
     f = 990.0 + 975.0 * np.arange(L) / max(L - 1, 1)
     return 60.0 + 40.0 * f / 1965.0
+
+
+# --------------------------------------------------------------------------------------
+# pack modelling inputs (Sec. 4.5; synthetic: the paper's micro-benchmark measurements are not available)
+# --------------------------------------------------------------------------------------
+def microbench_model(seed: int, n_metrics: int = 16, m: int = 12, L: int = 16):
+    """(B [n_metrics][m] metric matrix, Tb [m][L] ns, Eb [m][L] J): every micro-benchmark stresses a few metrics,
+    its time falls with the frequency, its energy follows 100 W + k f^3 as in the workload tables."""
+    u = rand_uniform(seed, 70, np.arange(n_metrics * m)).reshape(n_metrics, m)
+    hot = rand_uniform(seed, 71, np.arange(n_metrics * m)).reshape(n_metrics, m) < 0.3
+    B = 0.05 * u + np.where(hot, 1.0 + 4.0 * rand_uniform(seed, 72, np.arange(n_metrics * m)).reshape(n_metrics, m), 0.0)
+    B[np.arange(m) % n_metrics, np.arange(m)] += 3.0          # every benchmark has a metric of its own
+    f = 990.0 + 975.0 * np.arange(L) / max(L - 1, 1)
+    t_mem = 1000.0 + 9000.0 * rand_uniform(seed, 73, np.arange(m))
+    t_comp = 1000.0 + 9000.0 * rand_uniform(seed, 74, np.arange(m))
+    Tb = t_mem[:, None] + t_comp[:, None] * 1965.0 / f[None, :]
+    Eb = Tb * 1e-9 * (100.0 + 900.0 * (f[None, :] / 1965.0) ** 3)
+    return B, Tb, Eb
+
+
+def pack_features(seed: int, B: np.ndarray, n_packs: int, noise: float = 0.02):
+    """feat [n_packs][n_metrics]: sparse non-negative mixtures of the micro-benchmarks plus noise, so that the
+    constraint x >= 0 is active for some of them."""
+    n, m = B.shape
+    w = rand_uniform(seed, 75, np.arange(n_packs * m)).reshape(n_packs, m)
+    on = rand_uniform(seed, 76, np.arange(n_packs * m)).reshape(n_packs, m) < 0.3
+    x = np.where(on, 10.0 * w, 0.0)
+    z = rand_uniform(seed, 77, np.arange(n_packs * n)).reshape(n_packs, n) - 0.5
+    return x @ B.T + noise * z * (1.0 + np.abs(x @ B.T))
