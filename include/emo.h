@@ -215,6 +215,24 @@ int emo_pack_tables(int32_t n, int32_t L, const int64_t *lat, const double *ener
                     int32_t n_packs, int64_t *pack_lat, double *pack_energy);
 
 /*
+ * emo_pack_model - pack modelling (Sec. 4.5) for a batch of packs on the GPU.  Eq. 6: the weights of pack p are
+ * x_p = argmin ||B x - b_p||^2 subject to x >= 0, with B the metric matrix of the m micro-benchmarks and b_p the
+ * pack's feature vector at the default frequency; Eq. 7: its tables are T_f[P] = sum_i x_i T_f[B_i] and
+ * E_f[P] = sum_i x_i E_f[B_i].  One thread per pack (active-set method on the normal equations, fp64).
+ *   Bmat   device fp64 [n_metrics][m], m <= 16;  feat  device fp64 [n_packs][n_metrics].
+ *   Tb, Eb device fp64 [m][L]: the micro-benchmarks' latency (ns) and energy (J) at every level.
+ *   x      device fp64 [n_packs][m];  T_out, E_out  device fp64 [n_packs][L] (the caller rounds latencies to
+ *          whole ns for emo_graph_load).
+ *   status device int32, optional: EMO_E_UNSUPPORTED (-9) if a fit did not settle within its iteration bound.
+ * The minimiser is unique when B has independent columns (n_metrics >= m in practice); otherwise any minimiser
+ * may come out.  Errors: EMO_E_INVALID_ARG, EMO_E_UNSUPPORTED (tables and matrices beyond 48 KB of shared
+ * memory).  Asynchronous on `stream`.
+ */
+int emo_pack_model(int32_t n_packs, int32_t n_metrics, int32_t m, int32_t L, const double *Bmat, const double *feat,
+                   const double *Tb, const double *Eb, double *x, double *T_out, double *E_out, int32_t *status,
+                   void *stream);
+
+/*
  * emo_search_dp - Alg. 2: search for a near-optimal time-interval policy by dynamic programming over the
  * intervals, with emo_eval_intervals (Alg. 1) as the predictor.  dp[i] maps an end-to-end time to the least
  * energy and its policy after the first i intervals are decided; every state is extended by every level in

@@ -17,6 +17,7 @@
 #include "emo_pass_staged.cuh"
 #include "emo_flow.cuh"
 #include "emo_intervals.cuh"
+#include "emo_model.cuh"
 
 using namespace emo;
 
@@ -1459,6 +1460,36 @@ int emo_search_dp(const emo_graph *g, int32_t I, const int64_t *breaks, const do
         return EMO_E_OOM;
     }
     if (n_pred) *n_pred = calls;
+    return EMO_OK;
+}
+
+int emo_pack_model(int32_t n_packs, int32_t n_metrics, int32_t m, int32_t L, const double *Bmat, const double *feat,
+                   const double *Tb, const double *Eb, double *x, double *T_out, double *E_out, int32_t *status, void *stream)
+{
+    if (n_packs < 0 || n_metrics < 1 || m < 1 || m > kModelMaxM || L < 1) return EMO_E_INVALID_ARG;
+    if (n_packs == 0) return EMO_OK;
+    if (!Bmat || !feat || !Tb || !Eb || !x || !T_out || !E_out) return EMO_E_INVALID_ARG;
+    const size_t smem = ((size_t)m * m + (size_t)n_metrics * m + 2 * (size_t)m * L) * sizeof(double);
+    if (smem > 48 * 1024) return EMO_E_UNSUPPORTED;
+    ModelParams p;
+    p.n_packs = n_packs;
+    p.n = n_metrics;
+    p.m = m;
+    p.L = L;
+    p.B = Bmat;
+    p.feat = feat;
+    p.Tb = Tb;
+    p.Eb = Eb;
+    p.x = x;
+    p.T_out = T_out;
+    p.E_out = E_out;
+    p.status = status;
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaEvent_t ev0 = g_pass_events[0], ev1 = g_pass_events[1];
+    if (ev0) EMO_CUDA(cudaEventRecord(ev0, st));
+    emo_pack_model_kernel<<<(unsigned)((n_packs + 127) / 128), 128, smem, st>>>(p);
+    EMO_CUDA(cudaGetLastError());
+    if (ev1) EMO_CUDA(cudaEventRecord(ev1, st));
     return EMO_OK;
 }
 

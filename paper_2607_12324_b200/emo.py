@@ -31,7 +31,7 @@ EXPORTS = [
     "emo_strerror", "emo_graph_load", "emo_graph_free", "emo_graph_info", "emo_workspace_bytes",
     "emo_eval_policies", "emo_slack_batch", "emo_slack", "emo_baseline", "emo_target_from_delta",
     "emo_select", "emo_transpose_policies", "emo_slack_batch_host", "emo_graph_program",
-    "emo_set_pass_events", "emo_select_static", "emo_graph_flow", "emo_set_wait_limit", "emo_call_path", "emo_set_flow_counters", "emo_workspace_bytes_for", "emo_measure_int_issue", "emo_measure_warp_costs", "emo_eval_intervals", "emo_workspace_bytes_intervals", "emo_search_dp", "emo_workspace_bytes_search", "emo_pack_greedy", "emo_pack_tables", "emo_pack_levels", "emo_unpack_levels", "emo_slack_batch_host_packed",
+    "emo_set_pass_events", "emo_select_static", "emo_graph_flow", "emo_set_wait_limit", "emo_call_path", "emo_set_flow_counters", "emo_workspace_bytes_for", "emo_measure_int_issue", "emo_measure_warp_costs", "emo_eval_intervals", "emo_workspace_bytes_intervals", "emo_search_dp", "emo_workspace_bytes_search", "emo_pack_greedy", "emo_pack_tables", "emo_pack_model", "emo_pack_levels", "emo_unpack_levels", "emo_slack_batch_host_packed",
 ]
 
 
@@ -118,6 +118,7 @@ def lib():
         L.emo_workspace_bytes_search.argtypes = [p, i32, i64, ctypes.c_int, p]
         L.emo_pack_greedy.argtypes = [i32, p, p, p, p, p, i64, p, p, p]
         L.emo_pack_tables.argtypes = [i32, i32, p, p, p, i32, p, p]
+        L.emo_pack_model.argtypes = [i32, i32, i32, i32, p, p, p, p, p, p, p, p, p]
         L.emo_pack_levels.argtypes = [ctypes.c_int, i64, i64, p, i64, p, i64, p]
         L.emo_unpack_levels.argtypes = [ctypes.c_int, i64, i64, p, i64, p, i64, p]
         L.emo_slack_batch_host_packed.argtypes = [p, i64, ctypes.c_int, p, i64, p, p, i64, p, i64, i64, p, p, p, p, p, p, sz, u32, p]
@@ -443,6 +444,12 @@ def emo_pack_tables(lat, energy, pack_of, n_packs):
     vp = lambda a: a.ctypes.data_as(ctypes.c_void_p)
     _check(lib().emo_pack_tables(int(n), int(L), vp(lt), vp(en), vp(po), int(n_packs), vp(pl), vp(pe)), "emo_pack_tables")
     return pl, pe
+
+
+def emo_pack_model(n_packs, n_metrics, m, L, Bmat, feat, Tb, Eb, x, T_out, E_out, status=None, stream=None):
+    """Device tensors in and out (see include/emo.h)."""
+    return _check(lib().emo_pack_model(int(n_packs), int(n_metrics), int(m), int(L), _addr(Bmat), _addr(feat), _addr(Tb), _addr(Eb),
+                                       _addr(x), _addr(T_out), _addr(E_out), _addr(status), _stream(stream)), "emo_pack_model")
 
 
 def emo_pack_levels(bits, rows, B, lvl, ldb, packed, ldp, stream=None):
