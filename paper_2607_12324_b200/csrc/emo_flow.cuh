@@ -197,20 +197,26 @@ __device__ __forceinline__ bool emo_flow_wait(unsigned bar, unsigned parity, vol
 
 // Reads one operand: the slot word of this thread, polled for its tag when the descriptor asks.
 // Returns false when the wait ran out.
-__device__ __noinline__ bool emo_flow_poll(unsigned a, unsigned tag, unsigned &x, volatile int *abort_word, long long limit)
+__device__ __noinline__ unsigned long long emo_flow_poll_value(unsigned a, unsigned tag, volatile int *abort_word, long long limit)
 {
     const long long t0 = clock64();
     for (;;) {
         for (unsigned i = 0; i < 1024u; ++i) {
             const unsigned long long v = emo_lds_b64v(a);
-            if ((unsigned)(v >> 32) == tag) {
-                x = (unsigned)v;
-                return true;
-            }
+            if ((unsigned)(v >> 32) == tag) return (v & 0xFFFFFFFFull) | (1ull << 32);
             if (i > 16u) __nanosleep(32);
         }
-        if (*abort_word || clock64() - t0 > limit) return false;
+        if (*abort_word || clock64() - t0 > limit) return 0ull;
     }
+}
+// (The value travels in the result, not through a reference: a variable whose address is passed to a call that
+// is not inlined lives in local memory for its whole life, and these sit on the critical path of every entry
+// that reads a slot.)
+__device__ __forceinline__ bool emo_flow_poll(unsigned a, unsigned tag, unsigned &x, volatile int *abort_word, long long limit)
+{
+    const unsigned long long r = emo_flow_poll_value(a, tag, abort_word, limit);
+    if (r >> 32) x = (unsigned)r;
+    return (r >> 32) != 0ull;
 }
 __device__ __forceinline__ unsigned emo_flow_operand(unsigned slot_base, int lane, unsigned w, unsigned tag, bool &dead,
                                                      volatile int *abort_word, long long limit)
