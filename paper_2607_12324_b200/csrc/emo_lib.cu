@@ -694,7 +694,9 @@ int launch_flow_fwd(const emo_graph *g, const FlowPlan &pl, int64_t B, const uin
     if (flags & EMO_F_TEST_STALL) p.stall_stage = p.stages / 2;
     cudaEvent_t ev0 = g_pass_events[0], ev1 = g_pass_events[1];
     if (ev0) EMO_CUDA(cudaEventRecord(ev0, st));
-    void (*kern)(FlowParams) = pl.threads <= 512 ? emo_flow_fwd<512, false> : (pl.threads <= 768 ? emo_flow_fwd<768, false> : emo_flow_fwd<1024, false>);
+    void (*kern)(FlowParams) = nullptr;
+    if (p.prof) kern = pl.threads <= 512 ? emo_flow_fwd<512, false, true> : (pl.threads <= 768 ? emo_flow_fwd<768, false, true> : emo_flow_fwd<1024, false, true>);
+    else kern = pl.threads <= 512 ? emo_flow_fwd<512, false, false> : (pl.threads <= 768 ? emo_flow_fwd<768, false, false> : emo_flow_fwd<1024, false, false>);
     if (flow_optin(kern, g) != EMO_OK) { (void)cudaGetLastError(); return EMO_E_CUDA; }
     kern<<<pl.grid_f, pl.threads, pl.smem_f, st>>>(p);
     EMO_CUDA(cudaGetLastError());
@@ -726,7 +728,9 @@ int launch_flow_bwd(const emo_graph *g, const FlowPlan &pl, int64_t B, const uin
     if (ev0) EMO_CUDA(cudaEventRecord(ev0, st));
     const bool extra = ES || LS || slack_sum || n_critical;
     void (*kern)(FlowParams) = nullptr;
-#define EMO_PICK_F(MAXT) kern = extra ? emo_flow_bwd<true, MAXT> : emo_flow_bwd<false, MAXT>
+#define EMO_PICK_F(MAXT)                                                                                   \
+    kern = p.prof ? (extra ? emo_flow_bwd<true, MAXT, true> : emo_flow_bwd<false, MAXT, true>)                 \
+                  : (extra ? emo_flow_bwd<true, MAXT, false> : emo_flow_bwd<false, MAXT, false>)
     if (pl.threads <= 512) EMO_PICK_F(512);
     else if (pl.threads <= 768) EMO_PICK_F(768);
     else EMO_PICK_F(1024);
@@ -1262,7 +1266,7 @@ int emo_eval_intervals(const emo_graph *g, int64_t B, const uint8_t *F, int64_t 
             q.breaks = (const long long *)d_breaks;
             q.busy = busy;
             q.ldw = ldw;
-            void (*kern)(FlowParams) = fp.threads <= 512 ? emo_flow_fwd<512, true> : (fp.threads <= 768 ? emo_flow_fwd<768, true> : emo_flow_fwd<1024, true>);
+            void (*kern)(FlowParams) = fp.threads <= 512 ? emo_flow_fwd<512, true, false> : (fp.threads <= 768 ? emo_flow_fwd<768, true, false> : emo_flow_fwd<1024, true, false>);
             if (flow_optin(kern, g) != EMO_OK) { (void)cudaGetLastError(); return EMO_E_CUDA; }
             kern<<<fp.grid_f, fp.threads, fp.smem_f, st>>>(q);
             EMO_CUDA(cudaGetLastError());
