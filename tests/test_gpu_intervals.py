@@ -153,3 +153,35 @@ def test_large_batch_sampled(torch_cuda, emo, oracle_mod):
     assert np.allclose(E.cpu().numpy()[cols], r["energy"], rtol=1e-9, atol=0)
     assert np.allclose(Ei.cpu().numpy()[cols], r["e_idle"], rtol=1e-9, atol=1e-30)
     h.free()
+
+
+def test_cfg4_full_size_sampled(torch_cuda, emo, oracle_mod):
+    """The bench's own workload and launch configuration (cfg4-llm at full size, 16 384 policies, 20 ms grid, idle
+    energy on): a few policies one by one against the oracle, both kernels against each other on all of them."""
+    torch = torch_cuda
+    g = W.make_graph("cfg4-llm", 1.0)
+    dev_of = W.device_of(g)
+    B, D = int(g.meta["B"]), 1
+    T0 = int(oracle_mod.batch(g, np.full((g.n, 1), g.L - 1, np.uint8))["makespan"][0])
+    I = int(T0 * 1.05 / 20e6) + 1
+    breaks = W.interval_breaks(T0, I)
+    F = W.interval_policies(g.meta["policy_seed"], D, I, g.L, B, device="cuda")
+    pi = torch.from_numpy(W.idle_power(g.L)).cuda()
+    h = emo.load_workload(g, flags=emo.EMO_F_INTERVALS, group_of=dev_of)
+    ws = torch.empty(emo.emo_workspace_bytes_intervals(h, B, I, True), dtype=torch.uint8, device="cuda")
+    out = []
+    for call_flags in (0, emo.EMO_F_NO_STAGING):
+        T = torch.zeros(B, dtype=torch.int64, device="cuda")
+        E = torch.zeros(B, dtype=torch.float64, device="cuda")
+        Ei = torch.zeros(B, dtype=torch.float64, device="cuda")
+        emo.emo_eval_intervals(h, B, F, F.shape[2], I, breaks, pi, T, E, Ei, ws, flags=call_flags)
+        torch.cuda.synchronize()
+        out.append((T.cpu().numpy(), E.cpu().numpy(), Ei.cpu().numpy()))
+    assert np.array_equal(out[0][0], out[1][0])
+    assert np.allclose(out[0][1], out[1][1], rtol=1e-12, atol=0) and np.allclose(out[0][2], out[1][2], rtol=1e-9, atol=1e-30)
+    cols = np.array([0, 5, 8191, 8192, 16383])
+    r = oracle_mod.intervals(g, dev_of, breaks, F[:, :, torch.as_tensor(cols, device="cuda")].cpu().numpy(), W.idle_power(g.L))
+    assert np.array_equal(out[0][0][cols], r["makespan"])
+    assert np.allclose(out[0][1][cols], r["energy"], rtol=1e-9, atol=0)
+    assert np.allclose(out[0][2][cols], r["e_idle"], rtol=1e-9, atol=1e-30)
+    h.free()
