@@ -233,6 +233,16 @@ int emo_pack_model(int32_t n_packs, int32_t n_metrics, int32_t m, int32_t L, con
                    void *stream);
 
 /*
+ * emo_pack_classes - pack-level sampling (Sec. 4.4, last paragraph): packs whose kernels carry the same sequence
+ * of names are one class, and only the first pack of every class needs profiling.  name_id int32 [n] gives every
+ * kernel's name as a number (the caller interns the strings); class_of_pack int32 [n_packs] receives the class of
+ * every pack, classes numbered by their first pack; n_classes their count.  Exact comparison of the sequences (the
+ * paper hashes them; a hash collision would merge different packs).  Host function.
+ */
+int emo_pack_classes(int32_t n, const int32_t *pack_of, const int32_t *name_id, int32_t n_packs, int32_t *class_of_pack,
+                     int32_t *n_classes);
+
+/*
  * emo_search_dp - Alg. 2: search for a near-optimal time-interval policy by dynamic programming over the
  * intervals, with emo_eval_intervals (Alg. 1) as the predictor.  dp[i] maps an end-to-end time to the least
  * energy and its policy after the first i intervals are decided; every state is extended by every level in

@@ -2,6 +2,7 @@
 // greedy packing of GPU kernels into packs, with the packs' frequency tables.  Host code: the procedure is a
 // sequential walk over the kernels of every stream and runs once per workload, before any policy is evaluated.
 #include <algorithm>
+#include <map>
 #include <cstdint>
 #include <new>
 #include <vector>
@@ -96,6 +97,34 @@ int emo_pack_tables(int32_t n, int32_t L, const int64_t *lat, const double *ener
             pack_lat[(int64_t)p * L + l] += lat[(int64_t)v * L + l];
             pack_energy[(int64_t)p * L + l] += energy[(int64_t)v * L + l];
         }
+    }
+    return EMO_OK;
+}
+
+int emo_pack_classes(int32_t n, const int32_t *pack_of, const int32_t *name_id, int32_t n_packs, int32_t *class_of_pack,
+                     int32_t *n_classes)
+{
+    if (n < 0 || n_packs < 0 || !pack_of || !name_id || !class_of_pack) return EMO_E_INVALID_ARG;
+    try {
+        // the sequence of kernel names of every pack, members in index order
+        std::vector<std::vector<int32_t>> seq((size_t)n_packs);
+        for (int32_t v = 0; v < n; ++v) {
+            const int32_t p = pack_of[v];
+            if (p < 0) continue;
+            if (p >= n_packs) return EMO_E_RANGE;
+            seq[(size_t)p].push_back(name_id[v]);
+        }
+        // packs with the same sequence form a class; classes are numbered by their first pack
+        std::map<std::vector<int32_t>, int32_t> seen;
+        int32_t count = 0;
+        for (int32_t p = 0; p < n_packs; ++p) {
+            auto it = seen.find(seq[(size_t)p]);
+            if (it == seen.end()) it = seen.emplace(seq[(size_t)p], count++).first;
+            class_of_pack[p] = it->second;
+        }
+        if (n_classes) *n_classes = count;
+    } catch (const std::bad_alloc &) {
+        return EMO_E_OOM;
     }
     return EMO_OK;
 }

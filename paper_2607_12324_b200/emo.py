@@ -31,7 +31,7 @@ EXPORTS = [
     "emo_strerror", "emo_graph_load", "emo_graph_free", "emo_graph_info", "emo_workspace_bytes",
     "emo_eval_policies", "emo_slack_batch", "emo_slack", "emo_baseline", "emo_target_from_delta",
     "emo_select", "emo_transpose_policies", "emo_slack_batch_host", "emo_graph_program",
-    "emo_set_pass_events", "emo_select_static", "emo_graph_flow", "emo_set_wait_limit", "emo_call_path", "emo_set_flow_counters", "emo_workspace_bytes_for", "emo_measure_int_issue", "emo_measure_warp_costs", "emo_eval_intervals", "emo_workspace_bytes_intervals", "emo_search_dp", "emo_workspace_bytes_search", "emo_pack_greedy", "emo_pack_tables", "emo_pack_model", "emo_pack_levels", "emo_unpack_levels", "emo_slack_batch_host_packed",
+    "emo_set_pass_events", "emo_select_static", "emo_graph_flow", "emo_set_wait_limit", "emo_call_path", "emo_set_flow_counters", "emo_workspace_bytes_for", "emo_measure_int_issue", "emo_measure_warp_costs", "emo_eval_intervals", "emo_workspace_bytes_intervals", "emo_search_dp", "emo_workspace_bytes_search", "emo_pack_greedy", "emo_pack_tables", "emo_pack_model", "emo_pack_classes", "emo_pack_levels", "emo_unpack_levels", "emo_slack_batch_host_packed",
 ]
 
 
@@ -119,6 +119,7 @@ def lib():
         L.emo_pack_greedy.argtypes = [i32, p, p, p, p, p, i64, p, p, p]
         L.emo_pack_tables.argtypes = [i32, i32, p, p, p, i32, p, p]
         L.emo_pack_model.argtypes = [i32, i32, i32, i32, p, p, p, p, p, p, p, p, p]
+        L.emo_pack_classes.argtypes = [i32, p, p, i32, p, p]
         L.emo_pack_levels.argtypes = [ctypes.c_int, i64, i64, p, i64, p, i64, p]
         L.emo_unpack_levels.argtypes = [ctypes.c_int, i64, i64, p, i64, p, i64, p]
         L.emo_slack_batch_host_packed.argtypes = [p, i64, ctypes.c_int, p, i64, p, p, i64, p, i64, i64, p, p, p, p, p, p, sz, u32, p]
@@ -444,6 +445,16 @@ def emo_pack_tables(lat, energy, pack_of, n_packs):
     vp = lambda a: a.ctypes.data_as(ctypes.c_void_p)
     _check(lib().emo_pack_tables(int(n), int(L), vp(lt), vp(en), vp(po), int(n_packs), vp(pl), vp(pe)), "emo_pack_tables")
     return pl, pe
+
+
+def emo_pack_classes(pack_of, name_id, n_packs):
+    po = np.ascontiguousarray(pack_of, np.int32)
+    nm = np.ascontiguousarray(name_id, np.int32)
+    cls = np.zeros(int(n_packs), np.int32)
+    cnt = ctypes.c_int32(0)
+    vp = lambda a: a.ctypes.data_as(ctypes.c_void_p)
+    _check(lib().emo_pack_classes(int(po.shape[0]), vp(po), vp(nm), int(n_packs), vp(cls), ctypes.byref(cnt)), "emo_pack_classes")
+    return cls, int(cnt.value)
 
 
 def emo_pack_model(n_packs, n_metrics, m, L, Bmat, feat, Tb, Eb, x, T_out, E_out, status=None, stream=None):

@@ -740,3 +740,16 @@ def pack_features(seed: int, B: np.ndarray, n_packs: int, noise: float = 0.02):
     x = np.where(on, 10.0 * w, 0.0)
     z = rand_uniform(seed, 77, np.arange(n_packs * n)).reshape(n_packs, n) - 0.5
     return x @ B.T + noise * z * (1.0 + np.abs(x @ B.T))
+
+
+def kernel_names(g: Graph, period: int = 48) -> np.ndarray:
+    """int32 [n]: a name number for every kernel (-1 for other nodes).  The synthetic traces have no kernel names;
+    an iteration of a model launches the same kernels layer after layer, so the name is the kernel's position in its
+    stream's launch order modulo `period`, offset by the stream."""
+    st = np.asarray(g.meta["node_stream"], np.int64)
+    out = np.full(g.n, -1, np.int64)
+    key = np.asarray(g.meta.get("node_timeline", np.zeros(g.n, np.int64)), np.int64) * 64 + st
+    for s in np.unique(key[g.kind == KIND_KERNEL]):
+        idx = np.flatnonzero((g.kind == KIND_KERNEL) & (key == s))
+        out[idx] = (np.arange(idx.shape[0]) % period) + 1000 * (int(s) % 64)
+    return out.astype(np.int32)

@@ -92,3 +92,26 @@ def test_per_pack_policies_on_the_gpu(emo, oracle_mod):
     assert np.array_equal(T.cpu().numpy(), r["makespan"])
     assert np.allclose(E.cpu().numpy(), r["energy"], rtol=1e-9, atol=0)
     h.free()
+
+
+def test_pack_classes_group_equal_name_sequences(emo):
+    """Sec. 4.4: packs with the same sequence of kernel names are profiled once.  Checked against the definition
+    (a dictionary keyed by the tuple of names), on a workload whose streams repeat their kernels layer by layer."""
+    g = W.make_graph("cfg1-train", 1.0)
+    is_kernel = (g.kind == W.KIND_KERNEL).astype(np.uint8)
+    t = g.lat[:, g.L - 1].copy()
+    names = W.kernel_names(g, period=12)
+    crit, po, cnt = emo.emo_pack_greedy(g.n, g.row_ptr, g.col, is_kernel, stream_ids(g), t, 300_000)
+    cls, ncls = emo.emo_pack_classes(po, names, cnt)
+    seen, want = {}, []
+    for p in range(cnt):
+        key = tuple(names[np.flatnonzero(po == p)].tolist())
+        want.append(seen.setdefault(key, len(seen)))
+    assert cls.tolist() == want and ncls == len(seen)
+    assert 0 < ncls <= cnt
+    # permuting the names of one pack changes its class
+    names2 = names.copy()
+    mem = np.flatnonzero(po == cnt // 2)
+    names2[mem[0]] = 999_999
+    cls2, _ = emo.emo_pack_classes(po, names2, cnt)
+    assert cls2[cnt // 2] not in cls2[: cnt // 2].tolist()
