@@ -42,7 +42,8 @@ extern "C" {
 #define EMO_E_OOM (-6)             /* host or device allocation failed, or workspace too small */
 #define EMO_E_CUDA (-7)            /* a CUDA runtime call failed (no device, launch error, ...) */
 #define EMO_E_TIMEOUT (-8)         /* a bounded device-side wait ran out; results are invalid */
-#define EMO_E_UNSUPPORTED (-9)     /* the graph needs more on-chip exchange slots than exist */
+#define EMO_E_UNSUPPORTED (-9)     /* the call has no path for these arguments (for example time-interval policies on a graph
+                                      that only the generic kernels can take) */
 
 /* flags of emo_graph_load */
 #define EMO_F_HOST_ONLY 0x1u       /* build the handle without touching a device (inspection) */
@@ -52,6 +53,8 @@ extern "C" {
 #define EMO_F_FLOW_STAGE(k) (((uint32_t)(k) & 0x3Fu) << 24)      /* lane-stream program: steps per stage (8, 16, 32) */
 #define EMO_F_INTERVALS 0x2u       /* also prepare the lane-stream form of emo_eval_intervals (a second copy of the forward program on
                                       the device); without it that call runs its step-program kernel */
+#define EMO_F_GENERIC 0x4u         /* skip the schedule compilers: the generic kernels evaluate the graph (they also take every
+                                      graph whose simultaneously live values exceed the on-chip exchange slots) */
 /* flags of the evaluation calls */
 #define EMO_F_VALIDATE 0x1u        /* check every level < L first; EMO_E_RANGE goes to *status */
 #define EMO_F_NO_STAGING 0x2u      /* use the plain-load kernels instead of the staged ones */
@@ -101,7 +104,11 @@ const char *emo_strerror(int code);
  *   out                       receives the handle.
  * Everything is copied; the caller may free its arrays on return.  The device copies belong to
  * the handle until emo_graph_free.  Not asynchronous: it synchronises the device copies it makes.
- * Errors: INVALID_ARG, NOT_TOPOLOGICAL, RANGE, OVERFLOW, NONFINITE, OOM, CUDA, UNSUPPORTED.
+ * A graph whose simultaneously live exchanged values exceed what the on-chip schedules can hold still loads:
+ * the generic kernels (one thread per policy, completion times in the workspace, [n][B] int64 per pass)
+ * evaluate it, exactly but slower; emo_call_path reports 3 for such a handle, emo_eval_intervals and
+ * emo_search_dp return EMO_E_UNSUPPORTED on it.
+ * Errors: INVALID_ARG, NOT_TOPOLOGICAL, RANGE, OVERFLOW, NONFINITE, OOM, CUDA.
  */
 int emo_graph_load(int32_t n, const int64_t *row_ptr, const int32_t *col,
                    const int32_t *level_ptr, int32_t n_levels, int32_t L,
@@ -403,7 +410,8 @@ int emo_set_pass_events(void *fwd_start, void *fwd_stop, void *bwd_start, void *
 /*
  * emo_call_path - which kernels emo_eval_policies (need_slack = 0) or emo_slack_batch (need_slack = 1)
  * would run for these arguments: 2 = the 32-bit lane-stream kernels, 1 = the staged 64-bit kernels,
- * 0 = the plain-load 64-bit kernels; negative = an EMO_E_* code.  lvl may be any pointer with the
+ * 0 = the plain-load 64-bit kernels, 3 = the generic kernels (a graph beyond the on-chip schedules' limits, or
+ * loaded with EMO_F_GENERIC); negative = an EMO_E_* code.  lvl may be any pointer with the
  * alignment of the real one.  For tests and reports; it launches nothing.
  */
 int emo_call_path(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t ldb, int64_t ldo,

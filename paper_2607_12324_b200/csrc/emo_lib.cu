@@ -18,6 +18,7 @@
 #include "emo_flow.cuh"
 #include "emo_intervals.cuh"
 #include "emo_model.cuh"
+#include "emo_generic.cuh"
 
 using namespace emo;
 
@@ -58,6 +59,13 @@ struct emo_graph {
     DevProgramLane lfwd, lbwd;       // only for programs of at most kLaneMaxLanes lanes
     DevFlow dflow;
     bool host_only = false;
+    // graphs beyond the schedule compilers' limits (or loaded with EMO_F_GENERIC): evaluated by the generic kernels
+    bool generic = false;
+    int64_t *gen_row_ptr = nullptr, *gen_srow_ptr = nullptr, *gen_lat = nullptr;
+    int32_t *gen_col = nullptr, *gen_scol = nullptr, *gen_group = nullptr;
+    double *gen_energy = nullptr;
+    std::vector<int64_t> host_lat;      // kept only for the generic path's upload
+    std::vector<double> host_energy;
     int device = 0;
     int sm_count = 148;
     size_t smem_optin = 0;
@@ -785,7 +793,7 @@ const char *emo_strerror(int code)
         case EMO_E_OOM: return "out of memory or workspace too small";
         case EMO_E_CUDA: return "CUDA runtime error";
         case EMO_E_TIMEOUT: return "bounded device wait ran out";
-        case EMO_E_UNSUPPORTED: return "graph needs more exchange slots than supported";
+        case EMO_E_UNSUPPORTED: return "no path for these arguments (see the call's description)";
         default: return "unknown status";
     }
 }
@@ -803,6 +811,7 @@ int emo_call_path(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t ldb
 {
     if (!g || B < 0) return EMO_E_INVALID_ARG;
     if (g->host_only) return EMO_E_CUDA;
+    if (g->generic) return 3;
     if (flow_allowed(g, B, lvl, ldb, need_slack ? ldo : 0, flags)) {
         FlowPlan fp;
         if (flow_plan(g, B, true, need_slack != 0, fp)) return 2;
@@ -978,10 +987,19 @@ int emo_graph_load(int32_t n, const int64_t *row_ptr, const int32_t *col, const 
             }
             return rc;
         };
-        int rc = compile_dir(true, nullptr, g->bwd);
+        int rc = (flags & EMO_F_GENERIC) ? EMO_E_UNSUPPORTED : compile_dir(true, nullptr, g->bwd);
         if (rc == EMO_OK) rc = compile_dir(false, &g->bwd.pos_of_node, g->fwd);
+        if (rc == EMO_E_UNSUPPORTED) {
+            // more live exchanged values than the on-chip schedules can hold: the generic kernels take the graph
+            g->generic = true;
+            g->fwd = Program();
+            g->bwd = Program();
+            g->host_lat.assign(lat, lat + (size_t)n * L);
+            g->host_energy.assign(energy, energy + (size_t)n * L);
+            rc = EMO_OK;
+        }
         if (rc != EMO_OK) { delete g; return rc; }
-        {
+        if (!g->generic) {
             // stage length: the longest of 32, 16, 8 steps whose entries the producers can index
             // (32 * kFlowRowRegs per stage); barrier distance 16 steps unless the caller says otherwise
             // (measured on the 250 000-node workload at 0.3 scale: 8 / 16 steps gave 8.5 / 7.7 ms for both passes)
@@ -991,6 +1009,10 @@ int emo_graph_load(int32_t n, const int64_t *row_ptr, const int32_t *col, const 
             if (fs == 0) fs = 16;
             if (fs > fk) fs = fk;
             rc = compile_flow(h, lat, energy, lanes, look, fk, fs, g->flow, err);
+            if (rc == EMO_E_UNSUPPORTED) {      // the 64-bit programs exist: they serve
+                g->flow = Flow();
+                rc = EMO_OK;
+            }
             if (rc != EMO_OK) { delete g; return rc; }
         }
         std::vector<int32_t> hop((size_t)std::max(n, 1), 0);
@@ -1017,6 +1039,26 @@ int emo_graph_load(int32_t n, const int64_t *row_ptr, const int32_t *col, const 
         g->smem_optin = prop.sharedMemPerBlockOptin;
         int rc = EMO_OK;
         try {
+        if (g->generic) {
+            // successor CSR from the predecessor CSR, then everything the generic kernels read
+            const HostGraph &hh = g->h;
+            std::vector<int64_t> sp((size_t)hh.n + 1, 0);
+            std::vector<int32_t> sc((size_t)std::max<int64_t>(hh.m, 1));
+            for (int64_t e = 0; e < hh.m; ++e) sp[(size_t)hh.col[e] + 1]++;
+            for (int32_t v = 0; v < hh.n; ++v) sp[(size_t)v + 1] += sp[(size_t)v];
+            std::vector<int64_t> fill(sp.begin(), sp.end() - 1);
+            for (int32_t v = 0; v < hh.n; ++v)
+                for (int64_t e = hh.row_ptr[v]; e < hh.row_ptr[v + 1]; ++e) sc[(size_t)fill[(size_t)hh.col[e]]++] = v;
+            rc = upload(&g->gen_row_ptr, hh.row_ptr.data(), hh.row_ptr.size() * 8);
+            if (rc == EMO_OK) rc = upload(&g->gen_col, hh.col.data(), hh.col.size() * 4);
+            if (rc == EMO_OK) rc = upload(&g->gen_srow_ptr, sp.data(), sp.size() * 8);
+            if (rc == EMO_OK) rc = upload(&g->gen_scol, sc.data(), (size_t)hh.m * 4);
+            if (rc == EMO_OK) rc = upload(&g->gen_group, hh.group.data(), hh.group.size() * 4);
+            if (rc == EMO_OK) rc = upload(&g->gen_lat, g->host_lat.data(), g->host_lat.size() * 8);
+            if (rc == EMO_OK) rc = upload(&g->gen_energy, g->host_energy.data(), g->host_energy.size() * 8);
+            g->host_lat = std::vector<int64_t>();
+            g->host_energy = std::vector<double>();
+        } else {
         rc = upload_program(g->fwd, g->dfwd);
         if (rc == EMO_OK) rc = upload_program(g->bwd, g->dbwd);
         if (rc == EMO_OK && g->fwd.lanes <= 32 - kProducerWarps && g->bwd.lanes <= 32 - kProducerWarps) {
@@ -1024,6 +1066,7 @@ int emo_graph_load(int32_t n, const int64_t *row_ptr, const int32_t *col, const 
             if (rc == EMO_OK) rc = upload_program_lane(g->bwd, g->lbwd);
         }
         if (rc == EMO_OK) rc = upload_flow(g->flow, g->dflow, (flags & EMO_F_INTERVALS) != 0);
+        }
         } catch (const std::bad_alloc &) {
             rc = EMO_E_OOM;
         }
@@ -1042,6 +1085,9 @@ int emo_graph_free(emo_graph *g)
         free_program_lane(g->lfwd);
         free_program_lane(g->lbwd);
         free_flow(g->dflow);
+        void *gen[] = {g->gen_row_ptr, g->gen_col, g->gen_srow_ptr, g->gen_scol, g->gen_group, g->gen_lat, g->gen_energy};
+        for (void *q : gen)
+            if (q) cudaFree(q);
     }
     delete g;
     return EMO_OK;
@@ -1151,10 +1197,72 @@ size_t spill_need(const emo_graph *g, int64_t B)
 
 extern "C" {
 
+// The generic kernels: completion times (and, for the backward pass, tails) of every node in the workspace.
+static size_t generic_need(const emo_graph *g, int64_t B, bool need_bwd)
+{
+    const size_t ldw = round_up((size_t)B + 1, 16);
+    return (size_t)std::max(g->h.n, 1) * ldw * 8 * (need_bwd ? 2 : 1);
+}
+
+static int launch_generic(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t ldb, bool need_bwd, int64_t *ES, int64_t *LS,
+                          int64_t *slack, int64_t ldo, int64_t *makespan, double *energy, int64_t *slack_sum, int32_t *n_critical,
+                          int64_t *T0, double *E0, void *ws, size_t ws_bytes, cudaStream_t st)
+{
+    const size_t head = kSmallWs + lvl_area(g);
+    if (!ws || ws_bytes < head + generic_need(g, B, need_bwd)) return EMO_E_OOM;
+    GenericParams p;
+    p.n = g->h.n;
+    p.L = g->h.L;
+    p.row_ptr = g->gen_row_ptr;
+    p.col = g->gen_col;
+    p.srow_ptr = g->gen_srow_ptr;
+    p.scol = g->gen_scol;
+    p.group = g->gen_group;
+    p.lat = g->gen_lat;
+    p.energy = g->gen_energy;
+    p.B = B;
+    p.want_base = (T0 || E0) ? 1 : 0;
+    p.lvl = lvl;
+    p.ldb = ldb;
+    p.ldw = (int64_t)round_up((size_t)B + 1, 16);
+    p.C = (int64_t *)((char *)ws + head);
+    p.Q = p.C + (size_t)std::max(g->h.n, 1) * p.ldw;
+    p.ES = ES;
+    p.LS = LS;
+    p.slack = slack;
+    p.ldo = ldo;
+    p.makespan = makespan;
+    p.energy_out = energy;
+    p.slack_sum = slack_sum;
+    p.n_critical = n_critical;
+    p.base_T = T0;
+    p.base_E = E0;
+    const int64_t cols = B + p.want_base;
+    if (cols == 0) return EMO_OK;
+    cudaEvent_t ev0 = g_pass_events[0], ev1 = g_pass_events[1], ev2 = g_pass_events[2], ev3 = g_pass_events[3];
+    if (ev0) EMO_CUDA(cudaEventRecord(ev0, st));
+    emo_generic_fwd<<<(unsigned)((cols + 127) / 128), 128, 0, st>>>(p);
+    EMO_CUDA(cudaGetLastError());
+    if (ev1) EMO_CUDA(cudaEventRecord(ev1, st));
+    if (need_bwd && B > 0) {
+        if (ev2) EMO_CUDA(cudaEventRecord(ev2, st));
+        emo_generic_bwd<<<(unsigned)((B + 127) / 128), 128, 0, st>>>(p);
+        EMO_CUDA(cudaGetLastError());
+        if (ev3) EMO_CUDA(cudaEventRecord(ev3, st));
+    }
+    return EMO_OK;
+}
+
 int emo_workspace_bytes_for(const emo_graph *g, int64_t B, int need_slack, uint32_t flags, int aligned, size_t *out)
 {
     if (!g || !out || B < 0) return EMO_E_INVALID_ARG;
     size_t bytes = kSmallWs + lvl_area(g);
+    if (g->generic) {
+        bytes += generic_need(g, B, need_slack != 0);
+        if (need_slack == 2) bytes += 4 * round_up((size_t)B * 8, 256) + 256;
+        *out = bytes;
+        return EMO_OK;
+    }
     if (need_slack) {
         // what the call with these flags will run: the 32-bit kernels keep a restore list between the
         // passes, the 64-bit kernels the earliest starts of every node
@@ -1193,6 +1301,9 @@ int emo_eval_policies(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t
         if (rc) return rc;
     }
     if (B == 0) { lvl = nullptr; ldb = 0; }
+    if (g->generic)
+        return launch_generic(g, B, lvl, ldb, false, nullptr, nullptr, nullptr, 0, makespan, energy, nullptr, nullptr, T0, E0, ws,
+                              ws_bytes, st);
     if (flow_allowed(g, B, lvl, ldb, 0, flags)) {
         FlowPlan fp;
         if (flow_plan(g, B, T0 || E0, false, fp))
@@ -1224,6 +1335,7 @@ int emo_eval_intervals(const emo_graph *g, int64_t B, const uint8_t *F, int64_t 
     for (int32_t i = 1; i < I; ++i)
         if (breaks[i] <= breaks[i - 1]) return EMO_E_INVALID_ARG;
     if (g->host_only) return EMO_E_CUDA;
+    if (g->generic) return EMO_E_UNSUPPORTED;      // the time-interval form needs a compiled schedule
     if (B == 0) return EMO_OK;
     if (!F || !makespan || !energy || ldb < B) return EMO_E_INVALID_ARG;
     if (energy_idle && !p_idle) return EMO_E_INVALID_ARG;
@@ -1512,6 +1624,9 @@ int emo_slack_batch(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t l
         int rc = launch_validate(g, B, lvl, ldb, status, st);
         if (rc) return rc;
     }
+    if (g->generic)
+        return launch_generic(g, B, lvl, ldb, true, ES, LS, slack, ldo, makespan, energy, slack_sum, n_critical, T0, E0, ws, ws_bytes,
+                              st);
     if (flow_allowed(g, B, lvl, ldb, ldo, flags)) {
         FlowPlan fp;
         if (flow_plan(g, B, T0 || E0, true, fp)) {

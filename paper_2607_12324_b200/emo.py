@@ -24,6 +24,7 @@ EMO_F_NO_STAGING = 0x2
 EMO_F_PAIR_KERNEL = 0x4
 EMO_F_LANE_KERNEL = 0x8
 EMO_F_FLOW_KERNEL = 0x10
+EMO_F_GENERIC = 0x4        # load flag (shares its value with the call flag EMO_F_PAIR_KERNEL)
 EMO_F_INTERVALS = 0x2      # load flag (shares its value with the call flag EMO_F_NO_STAGING)
 EMO_F_TEST_STALL = 0x100
 

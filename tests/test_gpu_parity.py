@@ -587,3 +587,58 @@ def test_measurement_helpers(torch_cuda, emo):
     assert 10.0 <= c["shared_load_dependent"] <= 80.0
     assert c["body_without_branch"] <= c["body_with_untaken_branch"]
     assert 5.0 <= c["barrier_5_warps"] <= 400.0
+
+
+def _wide_graph(ns, seed=0):
+    """ns sources, each read later by three of ns sinks: every source's value stays live until the sinks run."""
+    rs = np.random.RandomState(seed)
+    edges = sorted({(int(k), ns + j) for j in range(ns) for k in rs.choice(ns, 3, replace=False)})
+    lat = rs.randint(0, 100, size=(2 * ns, 4)).astype(np.int64)
+    return W.tiny_graph(2 * ns, edges, lat, name="wide")
+
+
+def test_generic_path_takes_what_the_schedules_cannot(torch_cuda, emo, oracle_mod):
+    """A graph with more simultaneously live values than there are exchange slots loads and evaluates exactly
+    (generic kernels); the same kernels, forced on ordinary graphs, agree with the oracle on every output."""
+    torch = torch_cuda
+    cases = [(_wide_graph(400), 0, None), (W.make_graph("cfg1-train", 0.1), emo.EMO_F_GENERIC, None),
+             (W.make_graph("cfg3-8dev", 0.01), emo.EMO_F_GENERIC, None)]
+    g3 = W.make_graph("cfg0-tiny", 0.5)
+    cases.append((g3, emo.EMO_F_GENERIC, np.random.RandomState(3).randint(-1, 5, size=g3.n).astype(np.int32)))
+    for g, flags, group_of in cases:
+        B = 77
+        rows = g.n if group_of is None else 5
+        lv = np.random.RandomState(1).randint(0, g.L, size=(rows, B)).astype(np.uint8)
+        h = emo.load_workload(g, flags=flags, group_of=group_of)
+        ld = 80
+        lvd = torch.full((rows, ld), 0xFF, dtype=torch.uint8, device="cuda")
+        lvd[:, :B] = torch.from_numpy(lv).cuda()
+        assert emo.emo_call_path(h, B, lvd, ld, ld, True, 0) == 3
+        mk = lambda dt: torch.zeros((g.n, ld), dtype=dt, device="cuda")
+        ES, LS, SL = mk(torch.int64), mk(torch.int64), mk(torch.int64)
+        T = torch.zeros(B, dtype=torch.int64, device="cuda")
+        E = torch.zeros(B, dtype=torch.float64, device="cuda")
+        ss = torch.zeros(B, dtype=torch.int64, device="cuda")
+        nc = torch.zeros(B, dtype=torch.int32, device="cuda")
+        T0 = torch.zeros(1, dtype=torch.int64, device="cuda")
+        E0 = torch.zeros(1, dtype=torch.float64, device="cuda")
+        ws = torch.empty(emo.emo_workspace_bytes(h, B, 1), dtype=torch.uint8, device="cuda")
+        emo.emo_slack_batch(h, B, lvd, ld, ES, LS, SL, ld, T, E, ss, nc, ws, None, T0=T0, E0=E0)
+        torch.cuda.synchronize()
+        r = oracle_mod.batch(g, lv, want_arrays=True, group_of=group_of)
+        assert np.array_equal(T.cpu().numpy(), r["makespan"])
+        assert np.allclose(E.cpu().numpy(), r["energy"], rtol=1e-9, atol=0)
+        assert np.array_equal(ES.cpu().numpy()[:, :B], r["ES"])
+        assert np.array_equal(LS.cpu().numpy()[:, :B], r["LS"])
+        assert np.array_equal(SL.cpu().numpy()[:, :B], r["slack"])
+        assert np.array_equal(ss.cpu().numpy(), r["slack_sum"]) and np.array_equal(nc.cpu().numpy(), r["n_critical"])
+        base_lv = np.full((rows, 1), g.L - 1, np.uint8)
+        base = oracle_mod.batch(g, base_lv, group_of=group_of)
+        assert int(T0.item()) == int(base["makespan"][0]) and np.isclose(float(E0.item()), base["energy"][0], rtol=1e-9)
+        # forward only, and the single-policy call
+        T.zero_()
+        ws2 = torch.empty(emo.emo_workspace_bytes(h, B, 0), dtype=torch.uint8, device="cuda")
+        emo.emo_eval_policies(h, B, lvd, ld, T, E, ws2)
+        torch.cuda.synchronize()
+        assert np.array_equal(T.cpu().numpy(), r["makespan"])
+        h.free()

@@ -246,3 +246,19 @@ def test_eval_calls_fail_loudly_without_device(emo):
         emo.emo_eval_policies(h, 4, 16, 16, 16, 16, None, None, 0, stream=0)
     assert ei.value.code == emo.EMO_E_CUDA
     h.free()
+
+
+def test_graphs_beyond_the_slot_limit_still_load(emo):
+    """More simultaneously live values than exchange slots: the handle is built for the generic kernels
+    (no schedule, workspace for the completion times of every node) instead of failing."""
+    rs = np.random.RandomState(0)
+    ns = 400
+    edges = sorted({(int(k), ns + j) for j in range(ns) for k in rs.choice(ns, 3, replace=False)})
+    g = W.tiny_graph(2 * ns, edges, rs.randint(0, 100, size=(2 * ns, 4)).astype(np.int64))
+    h = emo.load_workload(g, flags=emo.EMO_F_HOST_ONLY)
+    info = emo.emo_graph_info(h)
+    assert info.n == 2 * ns and info.steps_fwd == 0 and info.depth == 2
+    assert emo.emo_graph_flow(h, arrays=False)["ok32"] == 0
+    assert emo.emo_workspace_bytes(h, 100, 1) >= 2 * 800 * 112 * 8
+    assert emo.emo_workspace_bytes(h, 100, 0) >= 800 * 112 * 8
+    h.free()
