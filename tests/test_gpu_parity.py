@@ -641,4 +641,14 @@ def test_generic_path_takes_what_the_schedules_cannot(torch_cuda, emo, oracle_mo
         emo.emo_eval_policies(h, B, lvd, ld, T, E, ws2)
         torch.cuda.synchronize()
         assert np.array_equal(T.cpu().numpy(), r["makespan"])
+        one = torch.from_numpy(lv[:, 5].copy()).cuda()
+        es1 = torch.zeros(g.n, dtype=torch.int64, device="cuda")
+        ls1 = torch.zeros(g.n, dtype=torch.int64, device="cuda")
+        sl1 = torch.zeros(g.n, dtype=torch.int64, device="cuda")
+        t1 = torch.zeros(1, dtype=torch.int64, device="cuda")
+        ws3 = torch.empty(emo.emo_workspace_bytes(h, 1, 1), dtype=torch.uint8, device="cuda")
+        emo.emo_slack(h, one, es1, ls1, sl1, t1, None, ws3)
+        torch.cuda.synchronize()
+        assert int(t1.item()) == int(r["makespan"][5])
+        assert np.array_equal(es1.cpu().numpy(), r["ES"][:, 5]) and np.array_equal(sl1.cpu().numpy(), r["slack"][:, 5])
         h.free()
