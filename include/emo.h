@@ -51,6 +51,7 @@ extern "C" {
 #define EMO_F_LOOKAHEAD(d) (((uint32_t)(d) & 0xFFu) << 16) /* scheduling look-ahead in steps */
 #define EMO_F_FLOW_SYNC(s) ((((uint32_t)(s) / 8u) & 0xFu) << 4)  /* lane-stream program: steps between group barriers (8, 16, 32) */
 #define EMO_F_FLOW_STAGE(k) (((uint32_t)(k) & 0x3Fu) << 24)      /* lane-stream program: steps per stage (8, 16, 32) */
+#define EMO_F_SPINE_STAGE(k) ((uint32_t)((k) == 8 ? 1u : ((k) == 32 ? 3u : 2u)) << 30)   /* spine program: steps per stage (8, 16, 32) */
 #define EMO_F_INTERVALS 0x2u       /* also prepare the lane-stream form of emo_eval_intervals (a second copy of the forward program on
                                       the device); without it that call runs its step-program kernel */
 #define EMO_F_GENERIC 0x4u         /* skip the schedule compilers: the generic kernels evaluate the graph (they also take every
@@ -61,6 +62,8 @@ extern "C" {
 #define EMO_F_PAIR_KERNEL 0x4u     /* staged pass kernel with two policies per thread (default only for very large batches) */
 #define EMO_F_LANE_KERNEL 0x8u     /* staged pass kernel with one policy per thread (the default otherwise) */
 #define EMO_F_FLOW_KERNEL 0x10u    /* the 32-bit lane-stream kernels (the default only for large batches: n * B >= 2^31) */
+#define EMO_F_SPINE_KERNEL 0x20u   /* the spine kernels (slack matrix and per-policy results only; the default on graphs of at most
+                                    * eight lanes while n * B < 2^31) */
 #define EMO_F_TEST_STALL 0x100u    /* test hook of the 32-bit kernels: the producer warps stop half way, so that the
                                       consumers' bounded waits run out and EMO_E_TIMEOUT is reported */
 
@@ -488,6 +491,13 @@ typedef struct emo_flow_view {
     const int64_t *lbes, *push_base;
 } emo_flow_view;
 int emo_graph_flow(const emo_graph *g, emo_flow_view *out);
+
+/* Sizes of the spine program (the form of the schedule that the spine kernels walk: consecutive nodes of a
+ * lane that are linked only to each other form a segment, whose members share one slack; Eq. 1 runs through
+ * one operation per segment).  out[0] = 1 if the program exists (else the rest is 0), then lanes, steps per
+ * stage, stages, segments, forward operations, backward operations, forward value slots, backward value
+ * slots, most segments of a stage, 4-byte words of sums per policy and stage, restore rows.  Host memory. */
+int emo_graph_spine(const emo_graph *g, int64_t out[12]);
 
 #ifdef __cplusplus
 }

@@ -8,8 +8,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libemo_b200.so")
-SOURCES = ["emo_lib.cu", "emo_compile.cpp", "emo_flow_compile.cpp", "emo_pack.cpp"]
-HEADERS = ["emo_kernels.cuh", "emo_pass_staged.cuh", "emo_lane_layout.cuh", "emo_pass_lane.cuh", "emo_compile.h", "emo_flow.h", "emo_flow.cuh", "emo_intervals.cuh", "emo_model.cuh", "emo_generic.cuh",
+SOURCES = ["emo_lib.cu", "emo_compile.cpp", "emo_flow_compile.cpp", "emo_spine_compile.cpp", "emo_pack.cpp"]
+HEADERS = ["emo_kernels.cuh", "emo_pass_staged.cuh", "emo_lane_layout.cuh", "emo_pass_lane.cuh", "emo_compile.h", "emo_flow.h", "emo_flow.cuh", "emo_spine.cuh", "emo_intervals.cuh", "emo_model.cuh", "emo_generic.cuh",
            os.path.join("..", "..", "include", "emo.h")]
 
 

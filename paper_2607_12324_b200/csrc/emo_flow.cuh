@@ -26,7 +26,7 @@
 #include "emo_flow.h"
 #include "emo_pass_staged.cuh"
 
-constexpr int kFlowMaxBuf = 4;
+constexpr int kFlowMaxBuf = 8;
 constexpr int kFlowRowRegs = 8;          // a stage holds at most 32 * kFlowRowRegs entries
 
 struct FlowParams {
@@ -69,6 +69,11 @@ struct FlowParams {
     int64_t ldw;
     unsigned off_meta;                   // inside a stage: 16 bytes per entry {lbES_v (8), group, dmin_v}
     unsigned off_brk, off_Fs;            // inside the block's shared memory: change points, columns of F
+    // spine kernels (emo_spine.cuh): inside a stage the operations, the segment list, the member records and the
+    // terminal nodes' bounds; inside the block's shared memory the barriers of the groups and the segments' sums
+    unsigned off_ops, off_segl, off_mem, off_tpool;
+    unsigned off_sbar, off_acc, acc_bytes;   // acc_bytes: one group's sums of one stage
+    int workers, nacc;                   // look-up / store warps per group, buffers of sums
 };
 
 __device__ __forceinline__ unsigned long long emo_lds_b64v(unsigned a)
@@ -195,6 +200,24 @@ __device__ __forceinline__ bool emo_flow_wait(unsigned bar, unsigned parity, vol
     return emo_flow_wait_slow(bar, parity, abort_word, limit);
 }
 
+// The same with short naps: for warps whose wake-up time is on the critical path of a short stage.
+__device__ __noinline__ bool emo_flow_wait_fast_slow(unsigned bar, unsigned parity, volatile int *abort_word, long long limit)
+{
+    const long long t0 = clock64();
+    for (;;) {
+        for (unsigned i = 0; i < 4096u; ++i) {
+            if (emo_mbar_try(bar, parity)) return true;
+            if (i > 32u) __nanosleep(64);
+        }
+        if (*abort_word || clock64() - t0 > limit) return false;
+    }
+}
+__device__ __forceinline__ bool emo_flow_wait_fast(unsigned bar, unsigned parity, volatile int *abort_word, long long limit)
+{
+    if (emo_mbar_test(bar, parity)) return true;
+    return emo_flow_wait_fast_slow(bar, parity, abort_word, limit);
+}
+
 // Reads one operand: the slot word of this thread, polled for its tag when the descriptor asks.
 // Returns false when the wait ran out.
 __device__ __noinline__ unsigned long long emo_flow_poll_value(unsigned a, unsigned tag, volatile int *abort_word, long long limit)
@@ -304,7 +327,7 @@ __device__ __forceinline__ void emo_flow_out_u(unsigned slot_lane4, unsigned lan
 }
 
 // The producer warps of both kernels.  Stages are issued in walking order (backward: last first).
-template <bool BWD>
+template <bool BWD, bool FAST = false>
 __device__ __forceinline__ void emo_flow_produce(const FlowParams &p, unsigned stage0, unsigned bar0, volatile int *abort_word,
                                                  int lane, int pw)
 {
@@ -346,7 +369,8 @@ __device__ __forceinline__ void emo_flow_produce(const FlowParams &p, unsigned s
         }
         const long long tw0 = clock64();
         if (c >= nbuf) {
-            if (!emo_flow_wait(bar0 + 8 * (kFlowMaxBuf + s), ((c / nbuf) - 1) & 1, abort_word, p.wait_cycles)) {
+            const unsigned eb = bar0 + 8 * (kFlowMaxBuf + s), ep = ((c / nbuf) - 1) & 1;
+            if (!(FAST ? emo_flow_wait_fast(eb, ep, abort_word, p.wait_cycles) : emo_flow_wait(eb, ep, abort_word, p.wait_cycles))) {
                 if (lane == 0) {
                     *abort_word = 1;
                     if (p.status) atomicMin(p.status, -8);

@@ -76,6 +76,47 @@ constexpr uint32_t kOpWord = 1u << 30;      // a settled slot (4 bytes per polic
 constexpr uint32_t kOpClear = 1u << 29;     // a settled slot with a single reader: the reader resets it to 0
 constexpr uint32_t kOpOffMask = (1u << 29) - 1u;
 
+
+// ---- spine programs -------------------------------------------------------------------------------
+// A second form of the same schedule for the kernels of emo_spine.cuh.  A lane's consecutive entries
+// whose only live link in both directions is the lane itself form a segment: along it completion
+// offsets are running sums, and co_v + qin_v (hence T - Q_v - ES_v relative to A_v) is one number for
+// all members.  Per stage the program lists the segments (for the warps that do the look-ups, sums,
+// stores) and, per direction, one operation per segment for the single warp that carries the
+// recurrence of a policy group (the spine): the maximum of two value slots (corrected), plus the
+// segment's sum, written to the lane's slot and to a published slot.  A node with more operands gets
+// merge operations in front.  Backward, a value that a node of a much earlier stage reads (two stages
+// or more: a launch node and its kernels) is folded by the storing warps into a slot of that reader.
+constexpr int kSpOpWordsF = 8;        // a0, d0, a1, d1, lane slot, published slot, sum offset, flags | push row << 8 | pool index << 20
+constexpr int kSpOpWordsB = 12;       // the same eight (flags | pop row << 8), then: slot to clear, lane's completion slot, spare, spare
+constexpr int kSpSegWords = 4;        // lane | first position << 8 | members << 16 | flags << 24, sum offset, A_v low, high
+constexpr int kSpMemWords = 4;        // node, fold slot, fold correction, spare
+constexpr uint32_t kSp_NoSum = 1u;    // operation flags: the segment's sum is zero / a merge operation
+constexpr uint32_t kSp_Push = 2u;     // forward: the lane's previous value goes to the restore list; backward: it is popped
+constexpr uint32_t kSp_Terminal = 4u; // forward: the segment's last node has no successor
+constexpr uint32_t kSpSeg_PreF = 1u, kSpSeg_PreB = 2u, kSpSeg_Fold = 4u;   // segment flags
+
+struct SpineDir {
+    int slots = 0;                    // value slots of a policy group (128 bytes each)
+    int max_ops = 0;
+    std::vector<uint32_t> n_ops;      // [stages]
+    std::vector<uint32_t> ops;        // [stages][max_ops][kSpOpWordsF | kSpOpWordsB]
+};
+
+struct Spine {
+    bool ok = false;
+    int max_segs = 0, max_pool = 0;
+    int acc_words = 0;                // 4-byte words per policy that the sums / results of one stage take
+    int64_t pushes = 0;
+    int64_t segments = 0;
+    std::vector<uint32_t> n_segs;     // [stages]
+    std::vector<uint32_t> seg;        // [stages][max_segs][kSpSegWords]
+    std::vector<uint32_t> mem;        // [stages][lanes * K][kSpMemWords]
+    std::vector<uint64_t> pool;       // [stages][max_pool] lbC of terminal nodes
+    std::vector<int64_t> push_base;   // [stages + 1]
+    SpineDir f, b;
+};
+
 struct FlowDir {
     int slots_tag = 0, slots_set = 0;   // tagged slots (256 bytes per group) and settled slots (128 bytes)
     int pool_stride = 4;                // words of operand pool per stage
@@ -101,11 +142,27 @@ struct Flow {
     std::vector<uint32_t> grp;          // [stages][lanes][K] the node's group whether or not its tables depend on the level (kNone: none)
     std::vector<int64_t> push_base;     // [stages + 1] first restore row of every stage
     FlowDir f, b;
+    Spine spine;                      // filled when the compiler is asked for it
 };
+
+
+// What the spine back-end takes from the compiler's analysis (all indexed as in compile_flow).
+struct SpineIn {
+    int32_t n = 0;
+    int lanes = 0, K = 0, stages = 0, L = 0;
+    const std::vector<int64_t> *pp = nullptr, *sp = nullptr;          // predecessor / successor CSR (deduplicated)
+    const std::vector<int32_t> *pc = nullptr, *sc = nullptr;
+    const std::vector<char> *liveF = nullptr, *liveB = nullptr;       // per predecessor-CSR edge
+    const std::vector<char> *constant = nullptr;                      // node's tables do not depend on the level
+    const std::vector<int64_t> *lbES = nullptr, *lbC = nullptr, *lbQin = nullptr, *lbQ = nullptr;
+    const std::vector<int32_t> *step_of = nullptr, *lane_of = nullptr, *prev_on_lane = nullptr, *next_on_lane = nullptr, *pos_of = nullptr;
+    const double *energy = nullptr;                                   // [n][L]
+};
+int build_spine(const SpineIn &in, Spine &out, std::string &err);
 
 // Compiles g into a lane-stream program.  Returns EMO_OK with out.ok32 = false when the 32-bit
 // representation does not apply (spread too large, too many lanes); other codes are errors.
 int compile_flow(const HostGraph &g, const int64_t *lat, const double *energy, int lanes, int lookahead,
-                 int K, int sync, Flow &out, std::string &err);
+                 int K, int sync, Flow &out, std::string &err, bool spine = false);
 
 }  // namespace emo

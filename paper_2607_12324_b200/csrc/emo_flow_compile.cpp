@@ -64,7 +64,7 @@ void assign_slots(std::vector<SlotObj> &objs, int &n_tag, int &n_set)   // n_set
 }  // namespace
 
 int compile_flow(const HostGraph &g, const int64_t *lat, const double *energy, int lanes, int lookahead, int K, int sync,
-                 Flow &out, std::string &err)
+                 Flow &out, std::string &err, bool spine)
 {
     out = Flow();
     const int32_t n = g.n;
@@ -163,7 +163,7 @@ int compile_flow(const HostGraph &g, const int64_t *lat, const double *energy, i
             if (!liveB[e]) out.b.pruned++;
             if (liveF[e] || liveB[e]) {
                 preds[v].push_back(k);
-                gaps[v].push_back(liveF[e] != liveB[e] ? sync : 1);
+                gaps[v].push_back(liveF[e] != liveB[e] ? (spine ? 2 * K : sync) : 1);      // spine programs fold such values two stages back
                 any_gap = any_gap || liveF[e] != liveB[e];
             }
         }
@@ -547,6 +547,33 @@ int compile_flow(const HostGraph &g, const int64_t *lat, const double *energy, i
     pack_pool(poolF, out.f);
     pack_pool(poolB, out.b);
     out.ok32 = true;
+    if (spine) {
+        SpineIn in;
+        in.n = n;
+        in.lanes = lanes;
+        in.K = K;
+        in.stages = stages;
+        in.L = L;
+        in.pp = &pp;
+        in.sp = &sp;
+        in.pc = &pc;
+        in.sc = &sc;
+        in.liveF = &liveF;
+        in.liveB = &liveB;
+        in.constant = &constant;
+        in.lbES = &lbES;
+        in.lbC = &lbC;
+        in.lbQin = &lbQin;
+        in.lbQ = &lbQ;
+        in.step_of = &step_of;
+        in.lane_of = &lane_of;
+        in.prev_on_lane = &prev_on_lane;
+        in.next_on_lane = &next_on_lane;
+        in.pos_of = &pos_of;
+        in.energy = energy;
+        rc = build_spine(in, out.spine, err);
+        if (rc != EMO_OK) return rc;
+    }
     return EMO_OK;
 }
 

@@ -16,6 +16,7 @@
 #include "emo_pass_lane.cuh"
 #include "emo_pass_staged.cuh"
 #include "emo_flow.cuh"
+#include "emo_spine.cuh"
 #include "emo_intervals.cuh"
 #include "emo_model.cuh"
 #include "emo_generic.cuh"
@@ -51,6 +52,17 @@ struct DevFlow {
     bool ready = false;
 };
 
+// The spine program on the device (emo_spine.cuh): per direction one blob per stage.
+struct DevSpine {
+    unsigned char *blobF = nullptr, *blobB = nullptr;
+    uint32_t *rows = nullptr, *push_base = nullptr;
+    unsigned blobF_bytes = 0, blobB_bytes = 0;
+    unsigned f_off_ops = 0, f_off_segl = 0, f_off_tpool = 0, f_off_tab = 0;
+    unsigned b_off_ops = 0, b_off_segl = 0, b_off_mem = 0, b_off_tab = 0;
+    int max_push = 0;
+    bool ready = false;
+};
+
 struct emo_graph {
     HostGraph h;
     Program fwd, bwd;
@@ -58,6 +70,8 @@ struct emo_graph {
     DevProgram dfwd, dbwd;
     DevProgramLane lfwd, lbwd;       // only for programs of at most kLaneMaxLanes lanes
     DevFlow dflow;
+    Flow sflow;                      // the same graph compiled with short stages and its spine program (sflow.spine.ok: usable)
+    DevSpine dspine;
     bool host_only = false;
     // graphs beyond the schedule compilers' limits (or loaded with EMO_F_GENERIC): evaluated by the generic kernels
     bool generic = false;
@@ -576,6 +590,67 @@ void free_flow(DevFlow &d)
     d = DevFlow();
 }
 
+
+int upload_spine(const Flow &f, DevSpine &d)
+{
+    const Spine &sp = f.spine;
+    if (!f.ok32 || !sp.ok || f.stages == 0) return EMO_OK;
+    const size_t per = (size_t)f.lanes * f.K;
+    auto r16 = [](size_t x) { return (x + 15) / 16 * 16; };
+    d.f_off_ops = 16;
+    d.f_off_segl = (unsigned)(d.f_off_ops + (size_t)(sp.f.max_ops + 1) * kSpOpWordsF * 4);
+    d.f_off_tpool = (unsigned)(d.f_off_segl + (size_t)sp.max_segs * kSpSegWords * 4);
+    d.f_off_tab = (unsigned)r16(d.f_off_tpool + (size_t)sp.max_pool * 8);
+    d.blobF_bytes = (unsigned)r16(d.f_off_tab + per * f.Lp * 12);
+    d.b_off_ops = 16;
+    d.b_off_segl = (unsigned)(d.b_off_ops + (size_t)(sp.b.max_ops + 1) * kSpOpWordsB * 4);
+    d.b_off_mem = (unsigned)(d.b_off_segl + (size_t)sp.max_segs * kSpSegWords * 4);
+    d.b_off_tab = (unsigned)(d.b_off_mem + per * kSpMemWords * 4);
+    d.blobB_bytes = (unsigned)r16(d.b_off_tab + per * f.Lp * 4);
+    std::vector<unsigned char> bf((size_t)f.stages * d.blobF_bytes, 0), bb((size_t)f.stages * d.blobB_bytes, 0);
+    std::vector<uint32_t> pb((size_t)f.stages + 1);
+    for (int st = 0; st <= f.stages; ++st) pb[st] = (uint32_t)sp.push_base[st];
+    for (int st = 0; st < f.stages; ++st) {
+        d.max_push = std::max(d.max_push, (int)(pb[st + 1] - pb[st]));
+        unsigned char *F = bf.data() + (size_t)st * d.blobF_bytes, *Bk = bb.data() + (size_t)st * d.blobB_bytes;
+        const uint32_t hf[4] = {sp.f.n_ops[st], sp.n_segs[st], pb[st], 0u}, hb[4] = {sp.b.n_ops[st], sp.n_segs[st], pb[st], 0u};
+        std::memcpy(F, hf, 16);
+        std::memcpy(Bk, hb, 16);
+        std::memcpy(F + d.f_off_ops, &sp.f.ops[(size_t)st * sp.f.max_ops * kSpOpWordsF], (size_t)sp.f.max_ops * kSpOpWordsF * 4);
+        std::memcpy(Bk + d.b_off_ops, &sp.b.ops[(size_t)st * sp.b.max_ops * kSpOpWordsB], (size_t)sp.b.max_ops * kSpOpWordsB * 4);
+        std::memcpy(F + d.f_off_segl, &sp.seg[(size_t)st * sp.max_segs * kSpSegWords], (size_t)sp.max_segs * kSpSegWords * 4);
+        std::memcpy(Bk + d.b_off_segl, &sp.seg[(size_t)st * sp.max_segs * kSpSegWords], (size_t)sp.max_segs * kSpSegWords * 4);
+        std::memcpy(F + d.f_off_tpool, &sp.pool[(size_t)st * sp.max_pool], (size_t)sp.max_pool * 8);
+        std::memcpy(Bk + d.b_off_mem, &sp.mem[(size_t)st * per * kSpMemWords], per * kSpMemWords * 4);
+        std::memcpy(Bk + d.b_off_tab, &f.tabB[(size_t)st * per * f.Lp], per * f.Lp * 4);
+        // forward table rows: the durations of all levels, then the energies (8-byte aligned)
+        for (size_t e = 0; e < per; ++e) {
+            const uint32_t *src = &f.tabF[((size_t)st * per + e) * f.Lp * 3];
+            unsigned char *row = F + d.f_off_tab + e * f.Lp * 12;
+            for (int l = 0; l < f.Lp; ++l) {
+                std::memcpy(row + (size_t)l * 4, &src[l * 3], 4);
+                const uint32_t lohi[2] = {src[l * 3 + 2], src[l * 3 + 1]};
+                std::memcpy(row + (size_t)f.Lp * 4 + (size_t)l * 8, lohi, 8);
+            }
+        }
+    }
+    int rc = upload(&d.blobF, bf.data(), bf.size());
+    if (rc == EMO_OK) rc = upload(&d.blobB, bb.data(), bb.size());
+    if (rc == EMO_OK) rc = upload(&d.rows, f.rows.data(), f.rows.size() * 4);
+    if (rc == EMO_OK) rc = upload(&d.push_base, pb.data(), pb.size() * 4);
+    d.ready = rc == EMO_OK;
+    return rc;
+}
+
+void free_spine(DevSpine &d)
+{
+    if (d.blobF) cudaFree(d.blobF);
+    if (d.blobB) cudaFree(d.blobB);
+    if (d.rows) cudaFree(d.rows);
+    if (d.push_base) cudaFree(d.push_base);
+    d = DevSpine();
+}
+
 // Launch shape of the 32-bit kernels: both passes use the same policy tile (the restore list is laid
 // out by tile), as many groups per block as cover the SMs once, two stage buffers (three when they fit).
 struct FlowPlan {
@@ -750,6 +825,171 @@ int launch_flow_bwd(const emo_graph *g, const FlowPlan &pl, int64_t B, const uin
     return EMO_OK;
 }
 
+// Launch shape of the spine kernels: the policy tile of flow_plan; per group one spine warp and as many worker
+// warps as the block has room for (at most 6); three buffers of sums when they fit (workers one stage ahead and
+// one behind the spine) and up to six stage buffers.
+bool spine_plan(const emo_graph *g, int64_t B, bool want_base, bool need_bwd, FlowPlan &pl)
+{
+    const Flow &f = g->sflow;
+    const Spine &sp = f.spine;
+    const DevSpine &d = g->dspine;
+    pl.ok = false;
+    if (!f.ok32 || !sp.ok || !d.ready || !g->smem_optin || f.stages == 0) return false;
+    if (f.lanes * f.K > 32 * kFlowRowRegs) return false;
+    const int64_t NBf = B + (want_base ? 1 : 0);
+    const int64_t n_groups = (NBf + 31) / 32;
+    const int64_t want = (n_groups + g->sm_count - 1) / g->sm_count;
+    const size_t budget = g->smem_optin;
+    for (int G = (int)std::max<int64_t>(1, std::min<int64_t>(7, want)); G >= 1; --G) {
+        const int nprod = G <= 4 ? 4 : 2;
+        const int W = std::min(6, (32 - nprod - G) / G);
+        if (W < 1) continue;
+        const size_t P = 32 * (size_t)G;
+        const size_t lvl_bytes = (size_t)G * f.lanes * f.K * 32;
+        const size_t acc_bytes = (size_t)sp.acc_words * 128;
+        auto shape = [&](bool backward, FlowParams &p, size_t &smem) {
+            const SpineDir &dir = backward ? sp.b : sp.f;
+            const size_t slot_bytes = (size_t)dir.slots * 128;
+            const size_t blob = backward ? d.blobB_bytes : d.blobF_bytes;
+            const size_t rst = backward ? (size_t)d.max_push * P * 4 : 0;
+            const size_t stage = round_up(blob + lvl_bytes + rst, 128);
+            const size_t off_bar = round_up(G * slot_bytes, 16);
+            const size_t off_sbar = off_bar + 192;
+            const size_t off_acc = round_up(off_sbar + (size_t)G * kFlowMaxBuf * 3 * 8, 128);
+            int nbuf = 0, nacc = 0;
+            size_t head = 0;
+            // a stage is short (about a microsecond of work): several stages must be on their way at any time
+            for (int na = 3; na >= 2 && !nbuf; --na)
+                for (int nb = std::min(6, kFlowMaxBuf); nb >= 2 && !nbuf; --nb) {
+                    head = round_up(off_acc + (size_t)na * G * acc_bytes, 128);
+                    if (head + nb * stage <= budget) {
+                        nbuf = nb;
+                        nacc = na;
+                    }
+                }
+            if (!nbuf || nbuf * stage < (size_t)G * W * 32 * 8) return false;
+            p = FlowParams();
+            p.blob = backward ? d.blobB : d.blobF;
+            p.rows = d.rows;
+            p.push_base = d.push_base;
+            p.blob_bytes = (unsigned)blob;
+            p.off_ops = backward ? d.b_off_ops : d.f_off_ops;
+            p.off_segl = backward ? d.b_off_segl : d.f_off_segl;
+            p.off_mem = d.b_off_mem;
+            p.off_tpool = d.f_off_tpool;
+            p.off_tab = backward ? d.b_off_tab : d.f_off_tab;
+            p.tab_row = (unsigned)f.Lp * (backward ? 4u : 12u);
+            p.stages = f.stages;
+            p.lanes = f.lanes;
+            p.K = f.K;
+            p.Lp = f.Lp;
+            p.L = g->h.L;
+            p.groups = G;
+            p.ptile = (int)P;
+            p.nbuf = nbuf;
+            p.nacc = nacc;
+            p.nprod = nprod;
+            p.workers = W;
+            p.slot_bytes = (unsigned)slot_bytes;
+            p.stage_bytes = (unsigned)stage;
+            p.off_lvl = (unsigned)blob;
+            p.off_rst = (unsigned)(blob + lvl_bytes);
+            p.off_bar = (unsigned)off_bar;
+            p.off_sbar = (unsigned)off_sbar;
+            p.off_acc = (unsigned)off_acc;
+            p.acc_bytes = (unsigned)acc_bytes;
+            p.off_stage0 = (unsigned)head;
+            p.pushes = sp.pushes;
+            p.restore_rows = sp.pushes + f.lanes;
+            p.wait_cycles = g_wait_cycles;
+            p.stall_stage = -1;
+            p.prof = nullptr;
+            smem = head + nbuf * stage;
+            return true;
+        };
+        if (!shape(false, pl.pf, pl.smem_f)) continue;
+        if (need_bwd && !shape(true, pl.pb, pl.smem_b)) continue;
+        pl.groups = G;
+        pl.grid_f = (int)((n_groups + G - 1) / G);
+        pl.grid_b = (int)(((B + 31) / 32 + G - 1) / G);
+        pl.threads = (G * (1 + W) + nprod) * 32;
+        pl.restore_bytes = need_bwd ? round_up((size_t)pl.grid_f * (size_t)(sp.pushes + f.lanes) * P * 4, 256) : 0;
+        pl.ok = true;
+        return true;
+    }
+    return false;
+}
+
+int launch_spine_fwd(const emo_graph *g, const FlowPlan &pl, int64_t B, const uint8_t *lvl, int64_t ldb, uint32_t *restore,
+                     int64_t *makespan, double *energy, int64_t *base_T, double *base_E, int32_t *status, uint32_t flags,
+                     cudaStream_t st)
+{
+    FlowParams p = pl.pf;
+    p.want_base = (base_T || base_E) ? 1 : 0;
+    if (B + p.want_base == 0) return EMO_OK;
+    p.B = B;
+    p.lvl = lvl;
+    p.ldb = ldb;
+    p.restore = restore;
+    p.makespan = makespan;
+    p.energy = energy;
+    p.base_T = base_T;
+    p.base_E = base_E;
+    p.status = status;
+    p.prof = g_flow_prof;
+    if (flags & EMO_F_TEST_STALL) p.stall_stage = p.stages / 2;
+    cudaEvent_t ev0 = g_pass_events[0], ev1 = g_pass_events[1];
+    if (ev0) EMO_CUDA(cudaEventRecord(ev0, st));
+    void (*kern)(FlowParams) = pl.threads <= 512 ? emo_spine_fwd<512> : emo_spine_fwd<1024>;
+    if (flow_optin(kern, g) != EMO_OK) { (void)cudaGetLastError(); return EMO_E_CUDA; }
+    kern<<<pl.grid_f, pl.threads, pl.smem_f, st>>>(p);
+    EMO_CUDA(cudaGetLastError());
+    if (ev1) EMO_CUDA(cudaEventRecord(ev1, st));
+    return EMO_OK;
+}
+
+int launch_spine_bwd(const emo_graph *g, const FlowPlan &pl, int64_t B, const uint8_t *lvl, int64_t ldb, uint32_t *restore,
+                     int64_t *slack, int64_t ldo, int64_t *makespan, int32_t *status, uint32_t flags, cudaStream_t st)
+{
+    if (B == 0) return EMO_OK;
+    FlowParams p = pl.pb;
+    p.B = B;
+    p.lvl = lvl;
+    p.ldb = ldb;
+    p.restore = restore;
+    p.makespan = makespan;
+    p.slack = slack;
+    p.ldo = ldo;
+    p.status = status;
+    if (flags & EMO_F_TEST_STALL) p.stall_stage = p.stages / 2;
+    cudaEvent_t ev0 = g_pass_events[2], ev1 = g_pass_events[3];
+    if (ev0) EMO_CUDA(cudaEventRecord(ev0, st));
+    void (*kern)(FlowParams) = pl.threads <= 512 ? emo_spine_bwd<512> : emo_spine_bwd<1024>;
+    if (flow_optin(kern, g) != EMO_OK) { (void)cudaGetLastError(); return EMO_E_CUDA; }
+    kern<<<pl.grid_b, pl.threads, pl.smem_b, st>>>(p);
+    EMO_CUDA(cudaGetLastError());
+    if (ev1) EMO_CUDA(cudaEventRecord(ev1, st));
+    return EMO_OK;
+}
+
+// Whether a call takes the spine kernels: the program exists, the call wants at most the slack matrix
+// beside the per-policy results, and either the caller asks for them (EMO_F_SPINE_KERNEL) or the graph is narrow
+// and the batch below the large-batch rule of the lane-stream kernels.
+bool spine_allowed(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t ldb, int64_t ldo, bool extra, uint32_t flags)
+{
+    const int64_t big = (int64_t)1 << 28;
+    if (!g->sflow.ok32 || !g->sflow.spine.ok || !g->dspine.ready || extra) return false;
+    if (flags & (EMO_F_NO_STAGING | EMO_F_PAIR_KERNEL | EMO_F_LANE_KERNEL | EMO_F_FLOW_KERNEL)) return false;
+    // Measured on the five workloads: on graphs of up to eight lanes with batches below the large-batch rule the spine
+    // kernels are the fastest pair (10 000 nodes x 4 096 policies: 1.1 ms against 2.3 ms for the 64-bit staged kernels
+    // and 3.1 ms for the lane-stream kernels; 1 013 nodes x 65 536 policies: 0.63 against 0.90 ms); one warp carries the
+    // recurrence of all lanes, so wide graphs (17 lanes: 21.9 against 9.0 ms) and, with four groups per block, the
+    // 250 000-node graph with 16 384 policies (the workers take the issue slots that the spine warp needs) stay with
+    // the other kernels unless the caller asks.
+    if (!(flags & EMO_F_SPINE_KERNEL) && ((int64_t)g->h.n * B >= ((int64_t)1 << 31) || g->sflow.lanes > 8)) return false;
+    return ldb % 16 == 0 && aligned16(lvl) && ldb < big && ldo < big;
+}
+
 // Whether a call takes the 32-bit lane-stream kernels: the program exists, the level matrix can be
 // fetched in 16-byte pieces, and either the caller asks for them (EMO_F_FLOW_KERNEL) or the batch is
 // large.  Measured on the five workloads: on the 250 000-node graph with 16 384 policies they are
@@ -812,6 +1052,10 @@ int emo_call_path(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t ldb
     if (!g || B < 0) return EMO_E_INVALID_ARG;
     if (g->host_only) return EMO_E_CUDA;
     if (g->generic) return 3;
+    if (spine_allowed(g, B, lvl, ldb, need_slack ? ldo : 0, need_slack == 2, flags)) {
+        FlowPlan fp;
+        if (spine_plan(g, B, true, need_slack != 0, fp)) return 4;
+    }
     if (flow_allowed(g, B, lvl, ldb, need_slack ? ldo : 0, flags)) {
         FlowPlan fp;
         if (flow_plan(g, B, true, need_slack != 0, fp)) return 2;
@@ -1014,6 +1258,22 @@ int emo_graph_load(int32_t n, const int64_t *row_ptr, const int32_t *col, const 
                 rc = EMO_OK;
             }
             if (rc != EMO_OK) { delete g; return rc; }
+            // the spine program: short stages (its sums per stage live in shared memory), 16 steps unless the caller
+            // says otherwise; only for graphs that the large-batch rule can send there
+            if (g->flow.ok32 && !(flags & EMO_F_INTERVALS)) {
+                const int code = (int)((flags >> 30) & 3u);
+                int sk = code == 1 ? 8 : (code == 3 ? 32 : 16);
+                while (sk > 8 && flanes * sk > 32 * kFlowRowRegs) sk /= 2;
+                rc = compile_flow(h, lat, energy, lanes, look, sk, sk, g->sflow, err, true);
+                if (rc == EMO_E_UNSUPPORTED) rc = EMO_OK;
+                if (rc != EMO_OK) { delete g; return rc; }
+                if (!g->sflow.spine.ok) g->sflow = Flow();
+                else {
+                    // only the spine's parts are kept
+                    g->sflow.f = FlowDir();
+                    g->sflow.b = FlowDir();
+                }
+            }
         }
         std::vector<int32_t> hop((size_t)std::max(n, 1), 0);
         int32_t depth = 0;
@@ -1066,6 +1326,7 @@ int emo_graph_load(int32_t n, const int64_t *row_ptr, const int32_t *col, const 
             if (rc == EMO_OK) rc = upload_program_lane(g->bwd, g->lbwd);
         }
         if (rc == EMO_OK) rc = upload_flow(g->flow, g->dflow, (flags & EMO_F_INTERVALS) != 0);
+        if (rc == EMO_OK) rc = upload_spine(g->sflow, g->dspine);
         }
         } catch (const std::bad_alloc &) {
             rc = EMO_E_OOM;
@@ -1085,6 +1346,7 @@ int emo_graph_free(emo_graph *g)
         free_program_lane(g->lfwd);
         free_program_lane(g->lbwd);
         free_flow(g->dflow);
+        free_spine(g->dspine);
         void *gen[] = {g->gen_row_ptr, g->gen_col, g->gen_srow_ptr, g->gen_scol, g->gen_group, g->gen_lat, g->gen_energy};
         for (void *q : gen)
             if (q) cudaFree(q);
@@ -1152,6 +1414,21 @@ int emo_graph_flow(const emo_graph *g, emo_flow_view *v)
     v->seg_bwd = f.b.seg.data();
     v->lbes = f.lbes.data();
     v->push_base = f.push_base.data();
+    return EMO_OK;
+}
+
+int emo_graph_spine(const emo_graph *g, int64_t out[12])
+{
+    if (!g || !out) return EMO_E_INVALID_ARG;
+    for (int i = 0; i < 12; ++i) out[i] = 0;
+    const Flow &f = g->sflow;
+    if (!f.ok32 || !f.spine.ok) return EMO_OK;
+    int64_t nf = 0, nb = 0;
+    for (uint32_t c : f.spine.f.n_ops) nf += c;
+    for (uint32_t c : f.spine.b.n_ops) nb += c;
+    const int64_t v[12] = {1, f.lanes, f.K, f.stages, f.spine.segments, nf, nb, f.spine.f.slots, f.spine.b.slots,
+                           f.spine.max_segs, f.spine.acc_words, f.spine.pushes};
+    for (int i = 0; i < 12; ++i) out[i] = v[i];
     return EMO_OK;
 }
 
@@ -1273,6 +1550,8 @@ int emo_workspace_bytes_for(const emo_graph *g, int64_t B, int need_slack, uint3
             need = fp.restore_bytes;
         else
             need = spill_need(g, B);
+        if (!g->host_only && B > 0 && spine_allowed(g, B, fake, aligned ? 16 : 1, 0, false, flags) && spine_plan(g, B, true, true, fp))
+            need = std::max(need, fp.restore_bytes);
         bytes += need;
     }
     if (need_slack == 2) bytes += 4 * round_up((size_t)B * 8, 256) + 256;
@@ -1304,6 +1583,11 @@ int emo_eval_policies(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t
     if (g->generic)
         return launch_generic(g, B, lvl, ldb, false, nullptr, nullptr, nullptr, 0, makespan, energy, nullptr, nullptr, T0, E0, ws,
                               ws_bytes, st);
+    if (spine_allowed(g, B, lvl, ldb, 0, false, flags)) {
+        FlowPlan fp;
+        if (spine_plan(g, B, T0 || E0, false, fp))
+            return launch_spine_fwd(g, fp, B, lvl, ldb, nullptr, makespan, energy, T0, E0, status, flags, st);
+    }
     if (flow_allowed(g, B, lvl, ldb, 0, flags)) {
         FlowPlan fp;
         if (flow_plan(g, B, T0 || E0, false, fp))
@@ -1627,6 +1911,17 @@ int emo_slack_batch(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t l
     if (g->generic)
         return launch_generic(g, B, lvl, ldb, true, ES, LS, slack, ldo, makespan, energy, slack_sum, n_critical, T0, E0, ws, ws_bytes,
                               st);
+    if (spine_allowed(g, B, lvl, ldb, ldo, ES || LS || slack_sum || n_critical, flags)) {
+        FlowPlan fp;
+        if (spine_plan(g, B, T0 || E0, true, fp)) {
+            const size_t head = kSmallWs + lvl_area(g);
+            if (!ws || ws_bytes < head + fp.restore_bytes) return EMO_E_OOM;
+            uint32_t *restore = (uint32_t *)((char *)ws + head);
+            int rc = launch_spine_fwd(g, fp, B, lvl, ldb, restore, makespan, energy, T0, E0, status, flags, st);
+            if (rc) return rc;
+            return launch_spine_bwd(g, fp, B, lvl, ldb, restore, slack, ldo, makespan, status, flags, st);
+        }
+    }
     if (flow_allowed(g, B, lvl, ldb, ldo, flags)) {
         FlowPlan fp;
         if (flow_plan(g, B, T0 || E0, true, fp)) {

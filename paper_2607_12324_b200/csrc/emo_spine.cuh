@@ -1,0 +1,417 @@
+// The spine kernels (sm_100a): emo_spine_fwd and emo_spine_bwd walk the spine program of emo_flow.h.
+// Included only by emo_lib.cu.
+//
+// A group of 32 policies (one per thread) has one spine warp and `workers` worker warps; a block holds
+// `groups` groups and the producer warps of emo_flow.cuh, which bring one stage at a time into a ring of
+// shared-memory buffers.  The recurrence of Eq. 1 runs through the spine warp alone: per segment it takes
+// the maximum of two value slots, adds the segment's sum and stores the result, all in its own program
+// order, so no value is ever waited for inside a stage.  Everything that does not depend on the
+// recurrence is done by the workers: the level and table look-ups, the sums per segment, the energy
+// (forward) and, backward, the slack of every member (one number per segment) and the tails that nodes
+// of much earlier stages read (folded into a slot of the reader with a maximum).  The workers run one
+// stage ahead of the spine with the sums and one stage behind it with the stores; mbarriers per group
+// and buffer order the three.
+//
+// Every wait is bounded (wait_cycles); a wait that runs out sets the block's abort word, which ends every
+// other wait of the block early, and EMO_E_TIMEOUT goes to *status.
+#pragma once
+#include "emo_flow.cuh"
+
+__device__ __forceinline__ bool emo_spine_wait(unsigned bar, unsigned parity, volatile int *abort_word, long long limit)
+{
+    return emo_flow_wait_fast(bar, parity, abort_word, limit);
+}
+__device__ __forceinline__ void emo_sts_u32(unsigned a, unsigned v)
+{
+    asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory");
+}
+
+// st.global of a 32-bit word under a predicate (no branch): base + row * pitch
+__device__ __forceinline__ void emo_stg_u32_if(uint32_t *base, unsigned row, unsigned pitch_bytes, unsigned v, unsigned ok)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .u64 a;\n\t"
+        "setp.ne.u32 p, %4, 0;\n\t"
+        "mad.wide.u32 a, %1, %2, %0;\n\t"
+        "@p st.global.u32 [a], %3;\n\t}"
+        ::"l"(base), "r"(row), "r"(pitch_bytes), "r"(v), "r"(ok)
+        : "memory");
+}
+#define EMO_SCLK() (p.prof ? clock64() : 0LL)
+
+// Barriers of group g and sums buffer a: workers -> spine (sums ready), spine -> workers (results ready),
+// workers -> everybody (stores done).
+__device__ __forceinline__ unsigned emo_spine_bar(const FlowParams &p, unsigned smem0, int g, int a, int which)
+{
+    return smem0 + p.off_sbar + (unsigned)(((g * kFlowMaxBuf + a) * 3 + which) * 8);
+}
+
+struct SpineRole {
+    bool producer, spine;
+    int group, widx;
+};
+__device__ __forceinline__ SpineRole emo_spine_role(const FlowParams &p, int warp)
+{
+    SpineRole r;
+    const int n_sp = p.groups, n_wk = p.groups * p.workers;
+    r.producer = warp >= n_sp + n_wk;
+    r.spine = warp < n_sp;
+    r.group = r.spine ? warp : (r.producer ? 0 : (warp - n_sp) / p.workers);
+    r.widx = r.spine || r.producer ? 0 : (warp - n_sp) - r.group * p.workers;
+    return r;
+}
+__device__ __forceinline__ void emo_spine_init(const FlowParams &p, unsigned smem0, unsigned char *smem)
+{
+    if (threadIdx.x == 0)
+        for (int g = 0; g < p.groups; ++g)
+            for (int a = 0; a < p.nacc; ++a) {
+                emo_mbar_init(emo_spine_bar(p, smem0, g, a, 0), p.workers);
+                emo_mbar_init(emo_spine_bar(p, smem0, g, a, 1), 1);
+                emo_mbar_init(emo_spine_bar(p, smem0, g, a, 2), p.workers);
+            }
+    emo_flow_init(p, smem0, smem, p.groups * (1 + p.workers));
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Forward pass (Eq. 1, Eq. 2): makespan and energy per policy, the restore list for the backward pass.
+// Stage header (first 16 bytes of the blob): operations, segments, first restore row of the stage.
+// ---------------------------------------------------------------------------------------------------
+template <int MAXT>
+__global__ void __launch_bounds__(MAXT, 1) emo_spine_fwd(FlowParams p)
+{
+    extern __shared__ __align__(128) unsigned char emo_smem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lanes = p.lanes, groups = p.groups, K = p.K, nbuf = p.nbuf, nacc = p.nacc, ptile = p.ptile, W = p.workers;
+    const SpineRole role = emo_spine_role(p, warp);
+    const int group = role.group;
+    const int64_t b0 = (int64_t)blockIdx.x * ptile;
+    const int col = group * 32 + lane;
+    const int64_t b = b0 + col;
+    const bool act = !role.producer && b < p.B;
+    const int base_col = (p.want_base && p.B >= b0 && p.B < b0 + ptile) ? (int)(p.B - b0) : -1;
+    const unsigned smem0 = emo_smem_addr(emo_smem);
+    const unsigned bar0 = smem0 + p.off_bar;
+    volatile int *abort_word = reinterpret_cast<volatile int *>(emo_smem + p.off_bar + 16 * kFlowMaxBuf);
+    const unsigned stage0 = smem0 + p.off_stage0;
+    const long long limit = p.wait_cycles;
+    emo_spine_init(p, smem0, emo_smem);
+
+    long long T = 0;
+    double ea = 0.0;
+    bool failed = false;
+    if (role.producer) {
+        emo_flow_produce<false, true>(p, stage0, bar0, abort_word, lane, warp - groups * (1 + W));
+    } else if (role.spine) {
+        const unsigned slot_lane4 = smem0 + (unsigned)group * p.slot_bytes + (unsigned)lane * 4u;
+        uint32_t *const rst_lane = p.restore ? p.restore + (size_t)blockIdx.x * p.restore_rows * ptile + col : nullptr;
+        long long t_full = 0, t_pre = 0, t_loop = 0;
+        const unsigned ptile4 = (unsigned)ptile * 4u;
+        const long long t_begin = EMO_SCLK();
+        for (int cst = 0; cst < p.stages; ++cst) {
+            const int s = cst % nbuf, a = cst % nacc;
+            const long long tw0 = EMO_SCLK();
+            const bool ok1 = emo_spine_wait(bar0 + 8 * s, (cst / nbuf) & 1, abort_word, limit);
+            const long long tw1 = EMO_SCLK();
+            if (!ok1 || !emo_spine_wait(emo_spine_bar(p, smem0, group, a, 0), (cst / nacc) & 1, abort_word, limit)) {
+                failed = true;
+                break;
+            }
+            const long long tw2 = EMO_SCLK();
+            t_full += tw1 - tw0;
+            t_pre += tw2 - tw1;
+            const unsigned sta = stage0 + (unsigned)s * p.stage_bytes;
+            const uint4 hd = emo_lds128(sta);
+            const int n_ops = (int)emo_uniform(hd.x);
+            const unsigned acc_a = smem0 + p.off_acc + (unsigned)(a * groups + group) * p.acc_bytes + (unsigned)lane * 4u;
+            unsigned op_a = sta + p.off_ops;
+            uint4 d0 = emo_lds128(op_a), d1 = emo_lds128(op_a + 16u);
+            const long long tl0 = EMO_SCLK();
+            for (int i = 0; i < n_ops; ++i) {
+                const uint4 c0 = d0, c1 = d1;
+                op_a += 32u;
+                d0 = emo_lds128(op_a);          // the next operation's words (one spare operation follows the last)
+                d1 = emo_lds128(op_a + 16u);
+                const unsigned x0 = emo_lds_u32(slot_lane4 + c0.x);
+                const unsigned x1 = emo_lds_u32(slot_lane4 + c0.z);
+                unsigned S = emo_lds_u32(acc_a + c1.z);
+                const unsigned fl = c1.w;
+                S = (fl & emo::kSp_NoSum) ? 0u : S;
+                const unsigned y = max(emo_floor_sub(x0, c0.y), emo_floor_sub(x1, c0.w)) + S;
+                // the lane's previous value (always the first operand) goes to the restore list where the backward pass cannot
+                // derive it; no branch: a taken branch costs this lone warp more than the whole operation
+                emo_stg_u32_if(rst_lane, hd.z + ((fl >> 8) & 0xFFFu), ptile4, x0, (fl & emo::kSp_Push) && rst_lane);
+                if (fl & emo::kSp_Terminal) {
+                    const unsigned pa = sta + p.off_tpool + (fl >> 20) * 8u;
+                    const long long lb = (long long)((unsigned long long)emo_lds_u32(pa) | ((unsigned long long)emo_lds_u32(pa + 4u) << 32));
+                    T = emo_max64(T, lb + (long long)(unsigned long long)y);
+                }
+                emo_sts_u32(slot_lane4 + c1.x, y);
+                emo_sts_u32(slot_lane4 + c1.y, y);
+            }
+            t_loop += EMO_SCLK() - tl0;
+            __syncwarp();
+            if (lane == 0) {
+                emo_mbar_arrive(emo_spine_bar(p, smem0, group, a, 1));
+                emo_mbar_arrive(bar0 + 8 * (kFlowMaxBuf + s));
+            }
+        }
+        if (!failed && rst_lane)
+            for (int ln = 0; ln < lanes; ++ln) rst_lane[((size_t)p.pushes + ln) * ptile] = emo_lds_u32(slot_lane4 + (unsigned)ln * 128u);
+        if (p.prof && lane == 0 && blockIdx.x < 512) {
+            long long *pr = p.prof + ((size_t)blockIdx.x * 32 + warp) * 8;
+            pr[0] = t_full;
+            pr[1] = t_pre;
+            pr[2] = EMO_SCLK() - t_begin;
+            pr[3] = t_loop;
+        }
+    } else {
+        const unsigned lmask = (unsigned)p.Lp - 1u, tab_row = p.tab_row, e_off = (unsigned)p.Lp * 4u;
+        const bool is_base = base_col == col;
+        const unsigned top = (unsigned)(p.L - 1);
+        long long t_full = 0, t_acc = 0;
+        const long long t_begin = EMO_SCLK();
+        for (int cst = 0; cst < p.stages; ++cst) {
+            const int s = cst % nbuf, a = cst % nacc;
+            const long long tw0 = EMO_SCLK();
+            const bool ok1 = emo_spine_wait(bar0 + 8 * s, (cst / nbuf) & 1, abort_word, limit);
+            const long long tw1 = EMO_SCLK();
+            if (!ok1 || (cst >= nacc && !emo_spine_wait(emo_spine_bar(p, smem0, group, a, 1), ((cst / nacc) - 1) & 1, abort_word, limit))) {
+                failed = true;
+                break;
+            }
+            t_full += tw1 - tw0;
+            t_acc += EMO_SCLK() - tw1;
+            const unsigned sta = stage0 + (unsigned)s * p.stage_bytes;
+            const int n_segs = (int)emo_uniform(emo_lds128(sta).y);
+            const unsigned acc_a = smem0 + p.off_acc + (unsigned)(a * groups + group) * p.acc_bytes + (unsigned)lane * 4u;
+            for (int i = role.widx; i < n_segs; i += W) {
+                const uint4 sd = emo_lds128(sta + p.off_segl + (unsigned)i * 16u);
+                if (!((sd.x >> 24) & emo::kSpSeg_PreF)) continue;
+                const unsigned ln = sd.x & 255u, first = (sd.x >> 8) & 255u;
+                const int cnt = (int)((sd.x >> 16) & 255u);
+                unsigned tab_a = sta + p.off_tab + (ln * (unsigned)K + first) * tab_row;
+                unsigned lvl_a = sta + p.off_lvl + ((((unsigned)(group * lanes) + ln) * (unsigned)K + first) << 5) + (unsigned)lane;
+                unsigned d = 0;
+#pragma unroll 4
+                for (int j = 0; j < cnt; ++j) {
+                    unsigned lv = emo_lds_u8(lvl_a);
+                    lv = (is_base ? top : lv) & lmask;
+                    d += emo_lds_u32(tab_a + lv * 4u);
+                    ea += emo_lds_f64(tab_a + e_off + lv * 8u);
+                    lvl_a += 32u;
+                    tab_a += tab_row;
+                }
+                emo_sts_u32(acc_a + sd.y, d);
+            }
+            __syncwarp();
+            if (lane == 0) {
+                emo_mbar_arrive(emo_spine_bar(p, smem0, group, a, 0));
+                emo_mbar_arrive(bar0 + 8 * (kFlowMaxBuf + s));
+            }
+        }
+        if (p.prof && lane == 0 && blockIdx.x < 512) {
+            long long *pr = p.prof + ((size_t)blockIdx.x * 32 + warp) * 8;
+            pr[0] = t_full;
+            pr[1] = t_acc;
+            pr[2] = EMO_SCLK() - t_begin;
+        }
+    }
+    if (failed && lane == 0) {
+        *abort_word = 1;
+        if (p.status) atomicMin(p.status, -8);
+    }
+
+    // combine the workers of a group in a fixed order (run-to-run identical energy)
+    __syncthreads();
+    double *part = reinterpret_cast<double *>(emo_smem + p.off_stage0);
+    if (!role.producer && !role.spine) part[(size_t)(group * W + role.widx) * 32 + lane] = ea;
+    __syncthreads();
+    if (role.spine && !*abort_word) {
+        double e = 0.0;
+        for (int k = 0; k < W; ++k) e += part[(size_t)(group * W + k) * 32 + lane];
+        if (act) {
+            p.makespan[b] = T;
+            p.energy[b] = e;
+        }
+        if (base_col == col) {
+            if (p.base_T) *p.base_T = T;
+            if (p.base_E) *p.base_E = e;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Backward pass: slack of every node.  Stages are walked last to first.  The spine leaves per segment
+// X = co + qin of its members (slack = T - A - X for all of them) and, where members are folded, the
+// head's tail; the workers store the slack and fold the members' tails one stage behind the spine, which
+// before a stage waits for the stores of the stage two back (folded values are read at least two stages
+// after they are written).
+// ---------------------------------------------------------------------------------------------------
+template <int MAXT>
+__global__ void __launch_bounds__(MAXT, 1) emo_spine_bwd(FlowParams p)
+{
+    extern __shared__ __align__(128) unsigned char emo_smem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lanes = p.lanes, groups = p.groups, K = p.K, nbuf = p.nbuf, nacc = p.nacc, ptile = p.ptile, W = p.workers;
+    const SpineRole role = emo_spine_role(p, warp);
+    const int group = role.group;
+    const int64_t b0 = (int64_t)blockIdx.x * ptile;
+    const int col = group * 32 + lane;
+    const int64_t b = b0 + col;
+    const bool act = !role.producer && b < p.B;
+    const unsigned smem0 = emo_smem_addr(emo_smem);
+    const unsigned bar0 = smem0 + p.off_bar;
+    volatile int *abort_word = reinterpret_cast<volatile int *>(emo_smem + p.off_bar + 16 * kFlowMaxBuf);
+    const unsigned stage0 = smem0 + p.off_stage0;
+    const long long limit = p.wait_cycles;
+    emo_spine_init(p, smem0, emo_smem);
+    const unsigned slot_lane4 = smem0 + (unsigned)group * p.slot_bytes + (unsigned)lane * 4u;
+
+    bool failed = false;
+    if (role.producer) {
+        emo_flow_produce<true, true>(p, stage0, bar0, abort_word, lane, warp - groups * (1 + W));
+    } else if (role.spine) {
+        // the lanes' last completion offsets: where the walk back begins
+        for (int ln = 0; ln < lanes; ++ln)
+            emo_sts_u32(slot_lane4 + (unsigned)(lanes + 2 + ln) * 128u,
+                        p.restore[((size_t)blockIdx.x * p.restore_rows + p.pushes + ln) * ptile + col]);
+        const unsigned col4 = (unsigned)col * 4u, ptile4 = (unsigned)ptile * 4u;
+        for (int cst = 0; cst < p.stages; ++cst) {
+            const int s = cst % nbuf, a = cst % nacc;
+            bool ok = emo_spine_wait(bar0 + 8 * s, (cst / nbuf) & 1, abort_word, limit) &&
+                      emo_spine_wait(emo_spine_bar(p, smem0, group, a, 0), (cst / nacc) & 1, abort_word, limit);
+            if (ok && cst >= 2) ok = emo_spine_wait(emo_spine_bar(p, smem0, group, (cst - 2) % nacc, 2), ((cst - 2) / nacc) & 1, abort_word, limit);
+            if (!ok) {
+                failed = true;
+                break;
+            }
+            const unsigned sta = stage0 + (unsigned)s * p.stage_bytes;
+            const uint4 hd = emo_lds128(sta);
+            const int n_ops = (int)emo_uniform(hd.x);
+            const unsigned acc_a = smem0 + p.off_acc + (unsigned)(a * groups + group) * p.acc_bytes + (unsigned)lane * 4u;
+            const unsigned rst_a = sta + p.off_rst + col4;
+            unsigned op_a = sta + p.off_ops;
+            uint4 d0 = emo_lds128(op_a), d1 = emo_lds128(op_a + 16u), d2 = emo_lds128(op_a + 32u);
+            for (int i = 0; i < n_ops; ++i) {
+                const uint4 c0 = d0, c1 = d1, c2 = d2;
+                op_a += 48u;
+                d0 = emo_lds128(op_a);
+                d1 = emo_lds128(op_a + 16u);
+                d2 = emo_lds128(op_a + 32u);
+                const unsigned x0 = emo_lds_u32(slot_lane4 + c0.x);
+                const unsigned x1 = emo_lds_u32(slot_lane4 + c0.z);
+                unsigned S = emo_lds_u32(acc_a + c1.z);
+                const unsigned c = emo_lds_u32(slot_lane4 + c2.y);
+                const unsigned fl = c1.w;
+                S = (fl & emo::kSp_NoSum) ? 0u : S;
+                const unsigned qin = max(emo_floor_sub(x0, c0.y), emo_floor_sub(x1, c0.w));
+                const unsigned qo = qin + S;
+                const unsigned cprev = emo_tld_u32_if(rst_a + ((fl >> 8) & 0xFFFu) * ptile4, 0u, fl & emo::kSp_Push, c - S);
+                emo_sts_u32(acc_a + c1.z, c + qin);
+                emo_sts_u32(acc_a + c2.z, qo);
+                emo_sts_u32(slot_lane4 + c2.x, 0u);
+                emo_sts_u32(slot_lane4 + c1.x, qo);
+                emo_sts_u32(slot_lane4 + c1.y, qo);
+                emo_sts_u32(slot_lane4 + c2.y, cprev);
+            }
+            __syncwarp();
+            if (lane == 0) {
+                emo_mbar_arrive(emo_spine_bar(p, smem0, group, a, 1));
+                emo_mbar_arrive(bar0 + 8 * (kFlowMaxBuf + s));
+            }
+        }
+    } else {
+        const unsigned lmask = (unsigned)p.Lp - 1u, tab_row = p.tab_row;
+        const long long T = act ? p.makespan[b] : 0;
+        const unsigned ldo8 = (unsigned)p.ldo * 8u;
+        long long *const sl_lane = (p.slack && act) ? reinterpret_cast<long long *>(p.slack) + b : nullptr;
+        const unsigned sl_ok = sl_lane != nullptr;
+        for (int cst = 0; cst <= p.stages && !failed; ++cst) {
+            if (cst < p.stages) {
+                // the sums of stage cst
+                const int s = cst % nbuf, a = cst % nacc;
+                if (!emo_spine_wait(bar0 + 8 * s, (cst / nbuf) & 1, abort_word, limit) ||
+                    (cst >= nacc && !emo_spine_wait(emo_spine_bar(p, smem0, group, a, 2), ((cst / nacc) - 1) & 1, abort_word, limit))) {
+                    failed = true;
+                    break;
+                }
+                const unsigned sta = stage0 + (unsigned)s * p.stage_bytes;
+                const int n_segs = (int)emo_uniform(emo_lds128(sta).y);
+                const unsigned acc_a = smem0 + p.off_acc + (unsigned)(a * groups + group) * p.acc_bytes + (unsigned)lane * 4u;
+                for (int i = role.widx; i < n_segs; i += W) {
+                    const uint4 sd = emo_lds128(sta + p.off_segl + (unsigned)i * 16u);
+                    if (!((sd.x >> 24) & emo::kSpSeg_PreB)) continue;
+                    const unsigned ln = sd.x & 255u, first = (sd.x >> 8) & 255u;
+                    const int cnt = (int)((sd.x >> 16) & 255u);
+                    unsigned tab_a = sta + p.off_tab + (ln * (unsigned)K + first) * tab_row;
+                    unsigned lvl_a = sta + p.off_lvl + ((((unsigned)(group * lanes) + ln) * (unsigned)K + first) << 5) + (unsigned)lane;
+                    unsigned d = 0;
+#pragma unroll 4
+                    for (int j = 0; j < cnt; ++j) {
+                        const unsigned lv = emo_lds_u8(lvl_a) & lmask;
+                        d += emo_lds_u32(tab_a + lv * 4u);
+                        lvl_a += 32u;
+                        tab_a += tab_row;
+                    }
+                    emo_sts_u32(acc_a + sd.y, d);
+                }
+                __syncwarp();
+                if (lane == 0) emo_mbar_arrive(emo_spine_bar(p, smem0, group, a, 0));
+            }
+            if (cst >= 1) {
+                // the stores of stage cst - 1
+                const int c1 = cst - 1, s = c1 % nbuf, a = c1 % nacc;
+                if (!emo_spine_wait(emo_spine_bar(p, smem0, group, a, 1), (c1 / nacc) & 1, abort_word, limit)) {
+                    failed = true;
+                    break;
+                }
+                const unsigned sta = stage0 + (unsigned)s * p.stage_bytes;
+                const int n_segs = (int)emo_uniform(emo_lds128(sta).y);
+                const unsigned acc_a = smem0 + p.off_acc + (unsigned)(a * groups + group) * p.acc_bytes + (unsigned)lane * 4u;
+                for (int i = role.widx; i < n_segs; i += W) {
+                    const uint4 sd = emo_lds128(sta + p.off_segl + (unsigned)i * 16u);
+                    const unsigned ln = sd.x & 255u, first = (sd.x >> 8) & 255u;
+                    const int cnt = (int)((sd.x >> 16) & 255u);
+                    const bool fold = ((sd.x >> 24) & emo::kSpSeg_Fold) != 0;
+                    const unsigned X = emo_lds_u32(acc_a + sd.y);
+                    unsigned q = fold ? emo_lds_u32(acc_a + sd.y + 128u) : 0u;
+                    // slack = T - (lbQ + lbES) - (co + qin): the same for every member
+                    const long long A = (long long)((unsigned long long)sd.z | ((unsigned long long)sd.w << 32));
+                    const long long sl = (T - A) - (long long)(unsigned long long)X;
+                    unsigned mem_a = sta + p.off_mem + (ln * (unsigned)K + first) * 16u;
+                    unsigned tab_a = sta + p.off_tab + (ln * (unsigned)K + first) * tab_row;
+                    unsigned lvl_a = sta + p.off_lvl + ((((unsigned)(group * lanes) + ln) * (unsigned)K + first) << 5) + (unsigned)lane;
+                    if (fold) {
+                        for (int j = 0; j < cnt; ++j) {
+                            const uint4 m = emo_lds128(mem_a);
+                            emo_stg_s64_if(sl_lane, m.x, ldo8, sl, sl_ok);
+                            emo_red_max_u32(slot_lane4 + m.y, emo_floor_sub(q, m.z));
+                            const unsigned lv = emo_lds_u8(lvl_a) & lmask;
+                            q -= emo_lds_u32(tab_a + lv * 4u);
+                            mem_a += 16u;
+                            lvl_a += 32u;
+                            tab_a += tab_row;
+                        }
+                    } else {
+#pragma unroll 4
+                        for (int j = 0; j < cnt; ++j) {
+                            const uint4 m = emo_lds128(mem_a);
+                            emo_stg_s64_if(sl_lane, m.x, ldo8, sl, sl_ok);
+                            mem_a += 16u;
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) {
+                    emo_mbar_arrive(emo_spine_bar(p, smem0, group, a, 2));
+                    emo_mbar_arrive(bar0 + 8 * (kFlowMaxBuf + s));
+                }
+            }
+        }
+    }
+    if (failed && lane == 0) {
+        *abort_word = 1;
+        if (p.status) atomicMin(p.status, -8);
+    }
+}
+#undef EMO_SCLK

@@ -24,6 +24,7 @@ EMO_F_NO_STAGING = 0x2
 EMO_F_PAIR_KERNEL = 0x4
 EMO_F_LANE_KERNEL = 0x8
 EMO_F_FLOW_KERNEL = 0x10
+EMO_F_SPINE_KERNEL = 0x20
 EMO_F_GENERIC = 0x4        # load flag (shares its value with the call flag EMO_F_PAIR_KERNEL)
 EMO_F_INTERVALS = 0x2      # load flag (shares its value with the call flag EMO_F_NO_STAGING)
 EMO_F_TEST_STALL = 0x100
@@ -32,7 +33,7 @@ EXPORTS = [
     "emo_strerror", "emo_graph_load", "emo_graph_free", "emo_graph_info", "emo_workspace_bytes",
     "emo_eval_policies", "emo_slack_batch", "emo_slack", "emo_baseline", "emo_target_from_delta",
     "emo_select", "emo_transpose_policies", "emo_slack_batch_host", "emo_graph_program",
-    "emo_set_pass_events", "emo_select_static", "emo_graph_flow", "emo_set_wait_limit", "emo_call_path", "emo_set_flow_counters", "emo_workspace_bytes_for", "emo_measure_int_issue", "emo_measure_warp_costs", "emo_eval_intervals", "emo_workspace_bytes_intervals", "emo_search_dp", "emo_workspace_bytes_search", "emo_pack_greedy", "emo_pack_tables", "emo_pack_model", "emo_pack_classes", "emo_pack_levels", "emo_unpack_levels", "emo_slack_batch_host_packed",
+    "emo_set_pass_events", "emo_select_static", "emo_graph_flow", "emo_graph_spine", "emo_set_wait_limit", "emo_call_path", "emo_set_flow_counters", "emo_workspace_bytes_for", "emo_measure_int_issue", "emo_measure_warp_costs", "emo_eval_intervals", "emo_workspace_bytes_intervals", "emo_search_dp", "emo_workspace_bytes_search", "emo_pack_greedy", "emo_pack_tables", "emo_pack_model", "emo_pack_classes", "emo_pack_levels", "emo_unpack_levels", "emo_slack_batch_host_packed",
 ]
 
 
@@ -46,6 +47,10 @@ def EMO_F_LOOKAHEAD(d: int) -> int:
 
 def EMO_F_FLOW_SYNC(s: int) -> int:
     return ((s // 8) & 0xF) << 4
+
+
+def EMO_F_SPINE_STAGE(k: int) -> int:
+    return (1 if k == 8 else (3 if k == 32 else 2)) << 30
 
 
 def EMO_F_FLOW_STAGE(k: int) -> int:
@@ -109,6 +114,7 @@ def lib():
                                         ctypes.POINTER(p), ctypes.POINTER(p)]
         L.emo_set_pass_events.argtypes = [p, p, p, p]
         L.emo_graph_flow.argtypes = [p, ctypes.POINTER(emo_flow_view)]
+        L.emo_graph_spine.argtypes = [p, ctypes.POINTER(ctypes.c_int64)]
         L.emo_set_wait_limit.argtypes = [i64]
         L.emo_set_flow_counters.argtypes = [p]
         L.emo_measure_int_issue.argtypes = [p, p, p]
@@ -316,6 +322,14 @@ def emo_graph_program(g: Graph, direction: int):
     lat = np.ctypeslib.as_array(ctypes.cast(pl, u32p), shape=(q * Lp.value,)).copy()
     return lanes.value, steps.value, slots.value, Lp.value, ent.reshape(steps.value, lanes.value, 8), \
         rows.reshape(steps.value, lanes.value), lat.reshape(q, Lp.value)
+
+
+def emo_graph_spine(g: Graph) -> dict:
+    """Sizes of the spine program (see emo.h)."""
+    out = (ctypes.c_int64 * 12)()
+    _check(lib().emo_graph_spine(g.handle, out), "emo_graph_spine")
+    keys = ("ok", "lanes", "K", "stages", "segments", "ops_fwd", "ops_bwd", "slots_fwd", "slots_bwd", "max_segs", "acc_words", "pushes")
+    return dict(zip(keys, [int(x) for x in out]))
 
 
 def emo_graph_flow(g: Graph, arrays: bool = True) -> dict:
