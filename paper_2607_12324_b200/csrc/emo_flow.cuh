@@ -71,8 +71,9 @@ struct FlowParams {
     unsigned off_brk, off_Fs;            // inside the block's shared memory: change points, columns of F
     // spine kernels (emo_spine.cuh): inside a stage the operations, the segment list, the member records and the
     // terminal nodes' bounds; inside the block's shared memory the barriers of the groups and the segments' sums
-    unsigned off_ops, off_segl, off_mem, off_tpool;
+    unsigned off_ops, off_mem, off_tpool, off_pos;   // off_pos: forward, one position word per lane position
     unsigned off_sbar, off_acc, acc_bytes;   // acc_bytes: one group's sums of one stage
+    unsigned off_oring, oring_bytes;     // forward: per group and buffer of sums, a copy of the front of the stage (header, bounds, operations)
     int workers, nacc;                   // look-up / store warps per group, buffers of sums
 };
 
@@ -200,15 +201,25 @@ __device__ __forceinline__ bool emo_flow_wait(unsigned bar, unsigned parity, vol
     return emo_flow_wait_slow(bar, parity, abort_word, limit);
 }
 
-// The same with short naps: for warps whose wake-up time is on the critical path of a short stage.
+// The same for warps whose wake-up time is on the critical path of a short stage: the wait is left to the hardware
+// (try_wait with a suspend-time hint: the warp sleeps inside the instruction until the phase completes or the hint runs
+// out), so a waiting warp issues next to nothing and wakes at once.
+__device__ __forceinline__ bool emo_mbar_try_hint(unsigned bar, unsigned parity, unsigned hint_ns)
+{
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(hint_ns)
+        : "memory");
+    return ok != 0;
+}
 __device__ __noinline__ bool emo_flow_wait_fast_slow(unsigned bar, unsigned parity, volatile int *abort_word, long long limit)
 {
     const long long t0 = clock64();
     for (;;) {
-        for (unsigned i = 0; i < 4096u; ++i) {
-            if (emo_mbar_try(bar, parity)) return true;
-            if (i > 32u) __nanosleep(64);
-        }
+        for (unsigned i = 0; i < 64u; ++i)
+            if (emo_mbar_try_hint(bar, parity, 20000u)) return true;
         if (*abort_word || clock64() - t0 > limit) return false;
     }
 }

@@ -90,7 +90,10 @@ constexpr uint32_t kOpOffMask = (1u << 29) - 1u;
 constexpr int kSpOpWordsF = 8;        // a0, d0, a1, d1, lane slot, published slot, sum offset, flags | push row << 8 | pool index << 20
 constexpr int kSpOpWordsB = 12;       // the same eight (flags | pop row << 8), then: slot to clear, lane's completion slot, spare, spare
 constexpr int kSpSegWords = 4;        // lane | first position << 8 | members << 16 | flags << 24, sum offset, A_v low, high
-constexpr int kSpMemWords = 4;        // node, fold slot, fold correction, spare
+constexpr int kSpMemWords = 8;        // node (kNone: unused position), fold slot, fold correction, position word, A_v low, high, spare, spare
+// position word (one per lane position of a stage): bit 0 = first member of its segment, bit 1 = last member,
+// bits 4..15 = index of the segment in the stage's list, bits 16..31 = offset of the segment's sum in 128-byte units
+constexpr uint32_t kSpPos_First = 1u, kSpPos_Last = 2u;
 constexpr uint32_t kSp_NoSum = 1u;    // operation flags: the segment's sum is zero / a merge operation
 constexpr uint32_t kSp_Push = 2u;     // forward: the lane's previous value goes to the restore list; backward: it is popped
 constexpr uint32_t kSp_Terminal = 4u; // forward: the segment's last node has no successor
@@ -112,6 +115,7 @@ struct Spine {
     std::vector<uint32_t> n_segs;     // [stages]
     std::vector<uint32_t> seg;        // [stages][max_segs][kSpSegWords]
     std::vector<uint32_t> mem;        // [stages][lanes * K][kSpMemWords]
+    std::vector<uint32_t> posw;       // [stages][lanes * K] position words
     std::vector<uint64_t> pool;       // [stages][max_pool] lbC of terminal nodes
     std::vector<int64_t> push_base;   // [stages + 1]
     SpineDir f, b;

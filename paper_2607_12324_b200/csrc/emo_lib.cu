@@ -57,8 +57,8 @@ struct DevSpine {
     unsigned char *blobF = nullptr, *blobB = nullptr;
     uint32_t *rows = nullptr, *push_base = nullptr;
     unsigned blobF_bytes = 0, blobB_bytes = 0;
-    unsigned f_off_ops = 0, f_off_segl = 0, f_off_tpool = 0, f_off_tab = 0;
-    unsigned b_off_ops = 0, b_off_segl = 0, b_off_mem = 0, b_off_tab = 0;
+    unsigned f_off_ops = 0, f_front = 0, f_off_tpool = 0, f_off_pos = 0, f_off_tab = 0;      // f_front: bytes that the spine needs
+    unsigned b_off_ops = 0, b_off_mem = 0, b_off_tab = 0;
     int max_push = 0;
     bool ready = false;
 };
@@ -597,14 +597,16 @@ int upload_spine(const Flow &f, DevSpine &d)
     if (!f.ok32 || !sp.ok || f.stages == 0) return EMO_OK;
     const size_t per = (size_t)f.lanes * f.K;
     auto r16 = [](size_t x) { return (x + 15) / 16 * 16; };
-    d.f_off_ops = 16;
-    d.f_off_segl = (unsigned)(d.f_off_ops + (size_t)(sp.f.max_ops + 1) * kSpOpWordsF * 4);
-    d.f_off_tpool = (unsigned)(d.f_off_segl + (size_t)sp.max_segs * kSpSegWords * 4);
-    d.f_off_tab = (unsigned)r16(d.f_off_tpool + (size_t)sp.max_pool * 8);
+    // forward: header, terminal bounds and operations lie together at the front (what the spine needs: a worker copies
+    // it to the group's own ring, so that the stage buffer is free again as soon as the sums are taken)
+    d.f_off_tpool = 16;
+    d.f_off_ops = (unsigned)r16(d.f_off_tpool + (size_t)sp.max_pool * 8);
+    d.f_front = (unsigned)(d.f_off_ops + (size_t)(sp.f.max_ops + 1) * kSpOpWordsF * 4);
+    d.f_off_pos = d.f_front;
+    d.f_off_tab = (unsigned)r16(d.f_off_pos + per * 4);
     d.blobF_bytes = (unsigned)r16(d.f_off_tab + per * f.Lp * 12);
     d.b_off_ops = 16;
-    d.b_off_segl = (unsigned)(d.b_off_ops + (size_t)(sp.b.max_ops + 1) * kSpOpWordsB * 4);
-    d.b_off_mem = (unsigned)(d.b_off_segl + (size_t)sp.max_segs * kSpSegWords * 4);
+    d.b_off_mem = (unsigned)(d.b_off_ops + (size_t)(sp.b.max_ops + 1) * kSpOpWordsB * 4);
     d.b_off_tab = (unsigned)(d.b_off_mem + per * kSpMemWords * 4);
     d.blobB_bytes = (unsigned)r16(d.b_off_tab + per * f.Lp * 4);
     std::vector<unsigned char> bf((size_t)f.stages * d.blobF_bytes, 0), bb((size_t)f.stages * d.blobB_bytes, 0);
@@ -618,21 +620,13 @@ int upload_spine(const Flow &f, DevSpine &d)
         std::memcpy(Bk, hb, 16);
         std::memcpy(F + d.f_off_ops, &sp.f.ops[(size_t)st * sp.f.max_ops * kSpOpWordsF], (size_t)sp.f.max_ops * kSpOpWordsF * 4);
         std::memcpy(Bk + d.b_off_ops, &sp.b.ops[(size_t)st * sp.b.max_ops * kSpOpWordsB], (size_t)sp.b.max_ops * kSpOpWordsB * 4);
-        std::memcpy(F + d.f_off_segl, &sp.seg[(size_t)st * sp.max_segs * kSpSegWords], (size_t)sp.max_segs * kSpSegWords * 4);
-        std::memcpy(Bk + d.b_off_segl, &sp.seg[(size_t)st * sp.max_segs * kSpSegWords], (size_t)sp.max_segs * kSpSegWords * 4);
         std::memcpy(F + d.f_off_tpool, &sp.pool[(size_t)st * sp.max_pool], (size_t)sp.max_pool * 8);
+        std::memcpy(F + d.f_off_pos, &sp.posw[(size_t)st * per], per * 4);
         std::memcpy(Bk + d.b_off_mem, &sp.mem[(size_t)st * per * kSpMemWords], per * kSpMemWords * 4);
         std::memcpy(Bk + d.b_off_tab, &f.tabB[(size_t)st * per * f.Lp], per * f.Lp * 4);
-        // forward table rows: the durations of all levels, then the energies (8-byte aligned)
-        for (size_t e = 0; e < per; ++e) {
-            const uint32_t *src = &f.tabF[((size_t)st * per + e) * f.Lp * 3];
-            unsigned char *row = F + d.f_off_tab + e * f.Lp * 12;
-            for (int l = 0; l < f.Lp; ++l) {
-                std::memcpy(row + (size_t)l * 4, &src[l * 3], 4);
-                const uint32_t lohi[2] = {src[l * 3 + 2], src[l * 3 + 1]};
-                std::memcpy(row + (size_t)f.Lp * 4 + (size_t)l * 8, lohi, 8);
-            }
-        }
+        // forward table rows: {duration, energy high word, low word} per level, 12 bytes apart (3 is coprime with the 32
+        // banks: the 32 policies of a warp, whatever their levels, read each of the three words without a bank conflict)
+        std::memcpy(F + d.f_off_tab, &f.tabF[(size_t)st * per * f.Lp * 3], per * f.Lp * 12);
     }
     int rc = upload(&d.blobF, bf.data(), bf.size());
     if (rc == EMO_OK) rc = upload(&d.blobB, bb.data(), bb.size());
@@ -842,7 +836,8 @@ bool spine_plan(const emo_graph *g, int64_t B, bool want_base, bool need_bwd, Fl
     const size_t budget = g->smem_optin;
     for (int G = (int)std::max<int64_t>(1, std::min<int64_t>(7, want)); G >= 1; --G) {
         const int nprod = G <= 4 ? 4 : 2;
-        const int W = std::min(6, (32 - nprod - G) / G);
+        // a worker takes whole lanes: more workers than lanes would only wait
+        const int W = std::min(f.lanes, std::min(6, (32 - nprod - G) / G));
         if (W < 1) continue;
         const size_t P = 32 * (size_t)G;
         const size_t lvl_bytes = (size_t)G * f.lanes * f.K * 32;
@@ -855,12 +850,14 @@ bool spine_plan(const emo_graph *g, int64_t B, bool want_base, bool need_bwd, Fl
             const size_t stage = round_up(blob + lvl_bytes + rst, 128);
             const size_t off_bar = round_up(G * slot_bytes, 16);
             const size_t off_sbar = off_bar + 192;
-            const size_t off_acc = round_up(off_sbar + (size_t)G * kFlowMaxBuf * 3 * 8, 128);
+            const size_t oring = backward ? 0 : d.f_front;      // forward: the spine's part of a stage, per group and buffer of sums
+            const size_t off_oring = round_up(off_sbar + (size_t)G * kFlowMaxBuf * 3 * 8, 128);
             int nbuf = 0, nacc = 0;
-            size_t head = 0;
+            size_t head = 0, off_acc = 0;
             // a stage is short (about a microsecond of work): several stages must be on their way at any time
             for (int na = 3; na >= 2 && !nbuf; --na)
                 for (int nb = std::min(6, kFlowMaxBuf); nb >= 2 && !nbuf; --nb) {
+                    off_acc = round_up(off_oring + (size_t)na * G * oring, 128);
                     head = round_up(off_acc + (size_t)na * G * acc_bytes, 128);
                     if (head + nb * stage <= budget) {
                         nbuf = nb;
@@ -874,9 +871,9 @@ bool spine_plan(const emo_graph *g, int64_t B, bool want_base, bool need_bwd, Fl
             p.push_base = d.push_base;
             p.blob_bytes = (unsigned)blob;
             p.off_ops = backward ? d.b_off_ops : d.f_off_ops;
-            p.off_segl = backward ? d.b_off_segl : d.f_off_segl;
             p.off_mem = d.b_off_mem;
             p.off_tpool = d.f_off_tpool;
+            p.off_pos = d.f_off_pos;
             p.off_tab = backward ? d.b_off_tab : d.f_off_tab;
             p.tab_row = (unsigned)f.Lp * (backward ? 4u : 12u);
             p.stages = f.stages;
@@ -897,6 +894,8 @@ bool spine_plan(const emo_graph *g, int64_t B, bool want_base, bool need_bwd, Fl
             p.off_bar = (unsigned)off_bar;
             p.off_sbar = (unsigned)off_sbar;
             p.off_acc = (unsigned)off_acc;
+            p.off_oring = (unsigned)off_oring;
+            p.oring_bytes = (unsigned)oring;
             p.acc_bytes = (unsigned)acc_bytes;
             p.off_stage0 = (unsigned)head;
             p.pushes = sp.pushes;
@@ -961,6 +960,7 @@ int launch_spine_bwd(const emo_graph *g, const FlowPlan &pl, int64_t B, const ui
     p.slack = slack;
     p.ldo = ldo;
     p.status = status;
+    p.prof = g_flow_prof ? g_flow_prof + 131072 : nullptr;
     if (flags & EMO_F_TEST_STALL) p.stall_stage = p.stages / 2;
     cudaEvent_t ev0 = g_pass_events[2], ev1 = g_pass_events[3];
     if (ev0) EMO_CUDA(cudaEventRecord(ev0, st));

@@ -5,21 +5,44 @@
 // `groups` groups and the producer warps of emo_flow.cuh, which bring one stage at a time into a ring of
 // shared-memory buffers.  The recurrence of Eq. 1 runs through the spine warp alone: per segment it takes
 // the maximum of two value slots, adds the segment's sum and stores the result, all in its own program
-// order, so no value is ever waited for inside a stage.  Everything that does not depend on the
-// recurrence is done by the workers: the level and table look-ups, the sums per segment, the energy
-// (forward) and, backward, the slack of every member (one number per segment) and the tails that nodes
-// of much earlier stages read (folded into a slot of the reader with a maximum).  The workers run one
-// stage ahead of the spine with the sums and one stage behind it with the stores; mbarriers per group
-// and buffer order the three.
+// order, so no value is ever waited for inside a stage; there is no branch in an operation (a taken branch
+// costs a lone warp more than the operation itself).  Everything that does not depend on the recurrence is
+// done by the workers, each of which walks whole lanes of the stage as streams of positions, four
+// positions at a time so that the look-ups overlap: the level and table look-ups, the running sums per
+// segment, the energy (forward) and, backward, the slack of every member (one number per segment) and the
+// tails that nodes of much earlier stages read (folded into a slot of the reader with a maximum).  The
+// workers run ahead of the spine with the sums and one stage behind it with the stores; mbarriers per group
+// and buffer of sums order the three.  Forward, a worker also copies the spine's part of the stage
+// (header, terminal bounds, operations) to a ring of the group, so that the stage buffer is free again as
+// soon as the sums are taken and the loads run several stages ahead of the spine.
 //
 // Every wait is bounded (wait_cycles); a wait that runs out sets the block's abort word, which ends every
-// other wait of the block early, and EMO_E_TIMEOUT goes to *status.
+// other wait of the block early, and EMO_E_TIMEOUT goes to *status.  The spine polls tightly (its wake-up
+// time is on the critical path), workers and producers nap between polls.
 #pragma once
 #include "emo_flow.cuh"
 
 __device__ __forceinline__ bool emo_spine_wait(unsigned bar, unsigned parity, volatile int *abort_word, long long limit)
 {
     return emo_flow_wait_fast(bar, parity, abort_word, limit);
+}
+// The workers' waits: they run ahead of the spine (sums) or behind it (stores), so a late wake-up costs nothing,
+// while every poll of the 20-odd waiting warps takes an issue slot from the spine.
+__device__ __noinline__ bool emo_worker_wait_slow(unsigned bar, unsigned parity, volatile int *abort_word, long long limit)
+{
+    const long long t0 = clock64();
+    for (;;) {
+        for (unsigned i = 0; i < 1024u; ++i) {
+            if (emo_mbar_try(bar, parity)) return true;
+            __nanosleep(250);
+        }
+        if (*abort_word || clock64() - t0 > limit) return false;
+    }
+}
+__device__ __forceinline__ bool emo_worker_wait(unsigned bar, unsigned parity, volatile int *abort_word, long long limit)
+{
+    if (emo_mbar_test(bar, parity)) return true;
+    return emo_worker_wait_slow(bar, parity, abort_word, limit);
 }
 __device__ __forceinline__ void emo_sts_u32(unsigned a, unsigned v)
 {
@@ -37,6 +60,10 @@ __device__ __forceinline__ void emo_stg_u32_if(uint32_t *base, unsigned row, uns
         ::"l"(base), "r"(row), "r"(pitch_bytes), "r"(v), "r"(ok)
         : "memory");
 }
+__device__ __forceinline__ void emo_sts_u32_if(unsigned a, unsigned v, unsigned ok)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\t@p st.shared.u32 [%0], %1;\n\t}" ::"r"(a), "r"(v), "r"(ok) : "memory");
+}
 #define EMO_SCLK() (p.prof ? clock64() : 0LL)
 
 // Barriers of group g and sums buffer a: workers -> spine (sums ready), spine -> workers (results ready),
@@ -48,8 +75,11 @@ __device__ __forceinline__ unsigned emo_spine_bar(const FlowParams &p, unsigned 
 
 struct SpineRole {
     bool producer, spine;
-    int group, widx;
+    int group, widx;      // producer: widx = its index among the producers
 };
+// Which warp does what: the spine warps first, then the workers group by group, then the producers.  (Giving the
+// spine and producer warps every fourth warp index, so that the workers sit on other schedulers, changed nothing:
+// with four groups per block the spine waits on the shared-memory pipe, which all warps of the SM share.)
 __device__ __forceinline__ SpineRole emo_spine_role(const FlowParams &p, int warp)
 {
     SpineRole r;
@@ -57,10 +87,10 @@ __device__ __forceinline__ SpineRole emo_spine_role(const FlowParams &p, int war
     r.producer = warp >= n_sp + n_wk;
     r.spine = warp < n_sp;
     r.group = r.spine ? warp : (r.producer ? 0 : (warp - n_sp) / p.workers);
-    r.widx = r.spine || r.producer ? 0 : (warp - n_sp) - r.group * p.workers;
+    r.widx = r.spine ? 0 : (r.producer ? warp - n_sp - n_wk : (warp - n_sp) - r.group * p.workers);
     return r;
 }
-__device__ __forceinline__ void emo_spine_init(const FlowParams &p, unsigned smem0, unsigned char *smem)
+__device__ __forceinline__ void emo_spine_init(const FlowParams &p, unsigned smem0, unsigned char *smem, int n_cons)
 {
     if (threadIdx.x == 0)
         for (int g = 0; g < p.groups; ++g)
@@ -69,7 +99,7 @@ __device__ __forceinline__ void emo_spine_init(const FlowParams &p, unsigned sme
                 emo_mbar_init(emo_spine_bar(p, smem0, g, a, 1), 1);
                 emo_mbar_init(emo_spine_bar(p, smem0, g, a, 2), p.workers);
             }
-    emo_flow_init(p, smem0, smem, p.groups * (1 + p.workers));
+    emo_flow_init(p, smem0, smem, n_cons);
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -94,13 +124,13 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_fwd(FlowParams p)
     volatile int *abort_word = reinterpret_cast<volatile int *>(emo_smem + p.off_bar + 16 * kFlowMaxBuf);
     const unsigned stage0 = smem0 + p.off_stage0;
     const long long limit = p.wait_cycles;
-    emo_spine_init(p, smem0, emo_smem);
+    emo_spine_init(p, smem0, emo_smem, groups * W);      // the spine reads its own copy: only the workers hold a stage buffer
 
     long long T = 0;
     double ea = 0.0;
     bool failed = false;
     if (role.producer) {
-        emo_flow_produce<false, true>(p, stage0, bar0, abort_word, lane, warp - groups * (1 + W));
+        emo_flow_produce<false>(p, stage0, bar0, abort_word, lane, role.widx);
     } else if (role.spine) {
         const unsigned slot_lane4 = smem0 + (unsigned)group * p.slot_bytes + (unsigned)lane * 4u;
         uint32_t *const rst_lane = p.restore ? p.restore + (size_t)blockIdx.x * p.restore_rows * ptile + col : nullptr;
@@ -108,18 +138,17 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_fwd(FlowParams p)
         const unsigned ptile4 = (unsigned)ptile * 4u;
         const long long t_begin = EMO_SCLK();
         for (int cst = 0; cst < p.stages; ++cst) {
-            const int s = cst % nbuf, a = cst % nacc;
+            const int a = cst % nacc;
             const long long tw0 = EMO_SCLK();
-            const bool ok1 = emo_spine_wait(bar0 + 8 * s, (cst / nbuf) & 1, abort_word, limit);
-            const long long tw1 = EMO_SCLK();
-            if (!ok1 || !emo_spine_wait(emo_spine_bar(p, smem0, group, a, 0), (cst / nacc) & 1, abort_word, limit)) {
+            const long long tw1 = tw0;
+            if (!emo_spine_wait(emo_spine_bar(p, smem0, group, a, 0), (cst / nacc) & 1, abort_word, limit)) {
                 failed = true;
                 break;
             }
             const long long tw2 = EMO_SCLK();
             t_full += tw1 - tw0;
             t_pre += tw2 - tw1;
-            const unsigned sta = stage0 + (unsigned)s * p.stage_bytes;
+            const unsigned sta = smem0 + p.off_oring + (unsigned)(a * groups + group) * p.oring_bytes;      // the group's copy
             const uint4 hd = emo_lds128(sta);
             const int n_ops = (int)emo_uniform(hd.x);
             const unsigned acc_a = smem0 + p.off_acc + (unsigned)(a * groups + group) * p.acc_bytes + (unsigned)lane * 4u;
@@ -150,10 +179,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_fwd(FlowParams p)
             }
             t_loop += EMO_SCLK() - tl0;
             __syncwarp();
-            if (lane == 0) {
-                emo_mbar_arrive(emo_spine_bar(p, smem0, group, a, 1));
-                emo_mbar_arrive(bar0 + 8 * (kFlowMaxBuf + s));
-            }
+            if (lane == 0) emo_mbar_arrive(emo_spine_bar(p, smem0, group, a, 1));
         }
         if (!failed && rst_lane)
             for (int ln = 0; ln < lanes; ++ln) rst_lane[((size_t)p.pushes + ln) * ptile] = emo_lds_u32(slot_lane4 + (unsigned)ln * 128u);
@@ -165,7 +191,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_fwd(FlowParams p)
             pr[3] = t_loop;
         }
     } else {
-        const unsigned lmask = (unsigned)p.Lp - 1u, tab_row = p.tab_row, e_off = (unsigned)p.Lp * 4u;
+        const unsigned lmask = (unsigned)p.Lp - 1u, tab_row = p.tab_row;
         const bool is_base = base_col == col;
         const unsigned top = (unsigned)(p.L - 1);
         long long t_full = 0, t_acc = 0;
@@ -173,35 +199,56 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_fwd(FlowParams p)
         for (int cst = 0; cst < p.stages; ++cst) {
             const int s = cst % nbuf, a = cst % nacc;
             const long long tw0 = EMO_SCLK();
-            const bool ok1 = emo_spine_wait(bar0 + 8 * s, (cst / nbuf) & 1, abort_word, limit);
+            const bool ok1 = emo_worker_wait(bar0 + 8 * s, (cst / nbuf) & 1, abort_word, limit);
             const long long tw1 = EMO_SCLK();
-            if (!ok1 || (cst >= nacc && !emo_spine_wait(emo_spine_bar(p, smem0, group, a, 1), ((cst / nacc) - 1) & 1, abort_word, limit))) {
+            if (!ok1 || (cst >= nacc && !emo_worker_wait(emo_spine_bar(p, smem0, group, a, 1), ((cst / nacc) - 1) & 1, abort_word, limit))) {
                 failed = true;
                 break;
             }
             t_full += tw1 - tw0;
             t_acc += EMO_SCLK() - tw1;
             const unsigned sta = stage0 + (unsigned)s * p.stage_bytes;
-            const int n_segs = (int)emo_uniform(emo_lds128(sta).y);
             const unsigned acc_a = smem0 + p.off_acc + (unsigned)(a * groups + group) * p.acc_bytes + (unsigned)lane * 4u;
-            for (int i = role.widx; i < n_segs; i += W) {
-                const uint4 sd = emo_lds128(sta + p.off_segl + (unsigned)i * 16u);
-                if (!((sd.x >> 24) & emo::kSpSeg_PreF)) continue;
-                const unsigned ln = sd.x & 255u, first = (sd.x >> 8) & 255u;
-                const int cnt = (int)((sd.x >> 16) & 255u);
-                unsigned tab_a = sta + p.off_tab + (ln * (unsigned)K + first) * tab_row;
-                unsigned lvl_a = sta + p.off_lvl + ((((unsigned)(group * lanes) + ln) * (unsigned)K + first) << 5) + (unsigned)lane;
-                unsigned d = 0;
-#pragma unroll 4
-                for (int j = 0; j < cnt; ++j) {
-                    unsigned lv = emo_lds_u8(lvl_a);
-                    lv = (is_base ? top : lv) & lmask;
-                    d += emo_lds_u32(tab_a + lv * 4u);
-                    ea += emo_lds_f64(tab_a + e_off + lv * 8u);
-                    lvl_a += 32u;
-                    tab_a += tab_row;
+            if (role.widx == 0) {
+                // the spine's part of the stage goes to the group's ring
+                const unsigned dst = smem0 + p.off_oring + (unsigned)(a * groups + group) * p.oring_bytes;
+                for (unsigned o = (unsigned)lane * 16u; o < p.oring_bytes; o += 512u) {
+                    const uint4 v = emo_lds128(sta + o);
+                    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + o), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
                 }
-                emo_sts_u32(acc_a + sd.y, d);
+            }
+            // A lane's positions of the stage are walked as one stream, four at a time (all look-ups of the four first, so
+            // that they overlap): the running sum restarts where a segment begins and is stored where one ends.  Unused
+            // positions have all-zero tables and store nothing.
+            for (int ln = role.widx; ln < lanes; ln += W) {
+                unsigned tab_a = sta + p.off_tab + (unsigned)(ln * K) * tab_row;
+                unsigned lvl_a = sta + p.off_lvl + ((unsigned)((group * lanes + ln) * K) << 5) + (unsigned)lane;
+                unsigned pos_a = sta + p.off_pos + (unsigned)(ln * K) * 4u;
+                unsigned run = 0;
+                for (int j0 = 0; j0 < K; j0 += 4) {
+                    const uint4 pw = emo_lds128(pos_a);
+                    unsigned lv[4], d[4];
+                    double e[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) lv[i] = emo_lds_u8(lvl_a + 32u * i);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        lv[i] = (is_base ? top : lv[i]) & lmask;
+                        const unsigned ta = tab_a + (unsigned)i * tab_row + lv[i] * 12u;
+                        d[i] = emo_lds_u32(ta);
+                        e[i] = __hiloint2double((int)emo_lds_u32(ta + 4u), (int)emo_lds_u32(ta + 8u));
+                    }
+                    const unsigned w4[4] = {pw.x, pw.y, pw.z, pw.w};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        run = (w4[i] & emo::kSpPos_First) ? d[i] : run + d[i];
+                        emo_sts_u32_if(acc_a + (w4[i] >> 16) * 128u, run, w4[i] & emo::kSpPos_Last);
+                        ea += e[i];
+                    }
+                    pos_a += 16u;
+                    lvl_a += 128u;
+                    tab_a += 4u * tab_row;
+                }
             }
             __syncwarp();
             if (lane == 0) {
@@ -264,27 +311,36 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_bwd(FlowParams p)
     volatile int *abort_word = reinterpret_cast<volatile int *>(emo_smem + p.off_bar + 16 * kFlowMaxBuf);
     const unsigned stage0 = smem0 + p.off_stage0;
     const long long limit = p.wait_cycles;
-    emo_spine_init(p, smem0, emo_smem);
+    emo_spine_init(p, smem0, emo_smem, groups * (1 + W));
     const unsigned slot_lane4 = smem0 + (unsigned)group * p.slot_bytes + (unsigned)lane * 4u;
 
     bool failed = false;
     if (role.producer) {
-        emo_flow_produce<true, true>(p, stage0, bar0, abort_word, lane, warp - groups * (1 + W));
+        emo_flow_produce<true>(p, stage0, bar0, abort_word, lane, role.widx);
     } else if (role.spine) {
         // the lanes' last completion offsets: where the walk back begins
         for (int ln = 0; ln < lanes; ++ln)
             emo_sts_u32(slot_lane4 + (unsigned)(lanes + 2 + ln) * 128u,
                         p.restore[((size_t)blockIdx.x * p.restore_rows + p.pushes + ln) * ptile + col]);
         const unsigned col4 = (unsigned)col * 4u, ptile4 = (unsigned)ptile * 4u;
+        long long t_full = 0, t_pre = 0, t_post = 0, t_loop = 0;
+        const long long t_begin = EMO_SCLK();
         for (int cst = 0; cst < p.stages; ++cst) {
             const int s = cst % nbuf, a = cst % nacc;
-            bool ok = emo_spine_wait(bar0 + 8 * s, (cst / nbuf) & 1, abort_word, limit) &&
-                      emo_spine_wait(emo_spine_bar(p, smem0, group, a, 0), (cst / nacc) & 1, abort_word, limit);
+            const long long tw0 = EMO_SCLK();
+            bool ok = emo_spine_wait(bar0 + 8 * s, (cst / nbuf) & 1, abort_word, limit);
+            const long long tw1 = EMO_SCLK();
+            ok = ok && emo_spine_wait(emo_spine_bar(p, smem0, group, a, 0), (cst / nacc) & 1, abort_word, limit);
+            const long long tw2 = EMO_SCLK();
             if (ok && cst >= 2) ok = emo_spine_wait(emo_spine_bar(p, smem0, group, (cst - 2) % nacc, 2), ((cst - 2) / nacc) & 1, abort_word, limit);
             if (!ok) {
                 failed = true;
                 break;
             }
+            const long long tw3 = EMO_SCLK();
+            t_full += tw1 - tw0;
+            t_pre += tw2 - tw1;
+            t_post += tw3 - tw2;
             const unsigned sta = stage0 + (unsigned)s * p.stage_bytes;
             const uint4 hd = emo_lds128(sta);
             const int n_ops = (int)emo_uniform(hd.x);
@@ -314,14 +370,25 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_bwd(FlowParams p)
                 emo_sts_u32(slot_lane4 + c1.y, qo);
                 emo_sts_u32(slot_lane4 + c2.y, cprev);
             }
+            t_loop += EMO_SCLK() - tw3;
             __syncwarp();
             if (lane == 0) {
                 emo_mbar_arrive(emo_spine_bar(p, smem0, group, a, 1));
                 emo_mbar_arrive(bar0 + 8 * (kFlowMaxBuf + s));
             }
         }
+        if (p.prof && lane == 0 && blockIdx.x < 512) {
+            long long *pr = p.prof + ((size_t)blockIdx.x * 32 + warp) * 8;
+            pr[0] = t_full;
+            pr[1] = t_pre;
+            pr[2] = EMO_SCLK() - t_begin;
+            pr[3] = t_loop;
+            pr[4] = t_post;
+        }
     } else {
         const unsigned lmask = (unsigned)p.Lp - 1u, tab_row = p.tab_row;
+        long long t_w1 = 0, t_w2 = 0, t_prew = 0, t_postw = 0;
+        const long long t_begin = EMO_SCLK();
         const long long T = act ? p.makespan[b] : 0;
         const unsigned ldo8 = (unsigned)p.ldo * 8u;
         long long *const sl_lane = (p.slack && act) ? reinterpret_cast<long long *>(p.slack) + b : nullptr;
@@ -330,75 +397,93 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_bwd(FlowParams p)
             if (cst < p.stages) {
                 // the sums of stage cst
                 const int s = cst % nbuf, a = cst % nacc;
-                if (!emo_spine_wait(bar0 + 8 * s, (cst / nbuf) & 1, abort_word, limit) ||
-                    (cst >= nacc && !emo_spine_wait(emo_spine_bar(p, smem0, group, a, 2), ((cst / nacc) - 1) & 1, abort_word, limit))) {
+                const long long tq0 = EMO_SCLK();
+                if (!emo_worker_wait(bar0 + 8 * s, (cst / nbuf) & 1, abort_word, limit) ||
+                    (cst >= nacc && !emo_worker_wait(emo_spine_bar(p, smem0, group, a, 2), ((cst / nacc) - 1) & 1, abort_word, limit))) {
                     failed = true;
                     break;
                 }
+                const long long tq1 = EMO_SCLK();
+                t_w1 += tq1 - tq0;
                 const unsigned sta = stage0 + (unsigned)s * p.stage_bytes;
-                const int n_segs = (int)emo_uniform(emo_lds128(sta).y);
                 const unsigned acc_a = smem0 + p.off_acc + (unsigned)(a * groups + group) * p.acc_bytes + (unsigned)lane * 4u;
-                for (int i = role.widx; i < n_segs; i += W) {
-                    const uint4 sd = emo_lds128(sta + p.off_segl + (unsigned)i * 16u);
-                    if (!((sd.x >> 24) & emo::kSpSeg_PreB)) continue;
-                    const unsigned ln = sd.x & 255u, first = (sd.x >> 8) & 255u;
-                    const int cnt = (int)((sd.x >> 16) & 255u);
-                    unsigned tab_a = sta + p.off_tab + (ln * (unsigned)K + first) * tab_row;
-                    unsigned lvl_a = sta + p.off_lvl + ((((unsigned)(group * lanes) + ln) * (unsigned)K + first) << 5) + (unsigned)lane;
-                    unsigned d = 0;
-#pragma unroll 4
-                    for (int j = 0; j < cnt; ++j) {
-                        const unsigned lv = emo_lds_u8(lvl_a) & lmask;
-                        d += emo_lds_u32(tab_a + lv * 4u);
-                        lvl_a += 32u;
-                        tab_a += tab_row;
+                // the sums per segment: every lane's positions as one stream, four at a time (see the forward kernel)
+                for (int ln = role.widx; ln < lanes; ln += W) {
+                    unsigned tab_a = sta + p.off_tab + (unsigned)(ln * K) * tab_row;
+                    unsigned lvl_a = sta + p.off_lvl + ((unsigned)((group * lanes + ln) * K) << 5) + (unsigned)lane;
+                    unsigned mem_a = sta + p.off_mem + (unsigned)(ln * K) * 32u + 12u;      // the position words
+                    unsigned run = 0;
+                    for (int j0 = 0; j0 < K; j0 += 4) {
+                        unsigned w4[4], lv[4], d[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            w4[i] = emo_lds_u32(mem_a + 32u * i);
+                            lv[i] = emo_lds_u8(lvl_a + 32u * i);
+                        }
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) d[i] = emo_lds_u32(tab_a + (unsigned)i * tab_row + (lv[i] & lmask) * 4u);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            run = (w4[i] & emo::kSpPos_First) ? d[i] : run + d[i];
+                            emo_sts_u32_if(acc_a + (w4[i] >> 16) * 128u, run, w4[i] & emo::kSpPos_Last);
+                        }
+                        mem_a += 128u;
+                        lvl_a += 128u;
+                        tab_a += 4u * tab_row;
                     }
-                    emo_sts_u32(acc_a + sd.y, d);
                 }
                 __syncwarp();
                 if (lane == 0) emo_mbar_arrive(emo_spine_bar(p, smem0, group, a, 0));
+                t_prew += EMO_SCLK() - tq1;
             }
             if (cst >= 1) {
                 // the stores of stage cst - 1
                 const int c1 = cst - 1, s = c1 % nbuf, a = c1 % nacc;
-                if (!emo_spine_wait(emo_spine_bar(p, smem0, group, a, 1), (c1 / nacc) & 1, abort_word, limit)) {
+                const long long tq0 = EMO_SCLK();
+                if (!emo_worker_wait(emo_spine_bar(p, smem0, group, a, 1), (c1 / nacc) & 1, abort_word, limit)) {
                     failed = true;
                     break;
                 }
+                const long long tq1 = EMO_SCLK();
+                t_w2 += tq1 - tq0;
                 const unsigned sta = stage0 + (unsigned)s * p.stage_bytes;
-                const int n_segs = (int)emo_uniform(emo_lds128(sta).y);
                 const unsigned acc_a = smem0 + p.off_acc + (unsigned)(a * groups + group) * p.acc_bytes + (unsigned)lane * 4u;
-                for (int i = role.widx; i < n_segs; i += W) {
-                    const uint4 sd = emo_lds128(sta + p.off_segl + (unsigned)i * 16u);
-                    const unsigned ln = sd.x & 255u, first = (sd.x >> 8) & 255u;
-                    const int cnt = (int)((sd.x >> 16) & 255u);
-                    const bool fold = ((sd.x >> 24) & emo::kSpSeg_Fold) != 0;
-                    const unsigned X = emo_lds_u32(acc_a + sd.y);
-                    unsigned q = fold ? emo_lds_u32(acc_a + sd.y + 128u) : 0u;
-                    // slack = T - (lbQ + lbES) - (co + qin): the same for every member
-                    const long long A = (long long)((unsigned long long)sd.z | ((unsigned long long)sd.w << 32));
-                    const long long sl = (T - A) - (long long)(unsigned long long)X;
-                    unsigned mem_a = sta + p.off_mem + (ln * (unsigned)K + first) * 16u;
-                    unsigned tab_a = sta + p.off_tab + (ln * (unsigned)K + first) * tab_row;
-                    unsigned lvl_a = sta + p.off_lvl + ((((unsigned)(group * lanes) + ln) * (unsigned)K + first) << 5) + (unsigned)lane;
-                    if (fold) {
-                        for (int j = 0; j < cnt; ++j) {
-                            const uint4 m = emo_lds128(mem_a);
-                            emo_stg_s64_if(sl_lane, m.x, ldo8, sl, sl_ok);
-                            emo_red_max_u32(slot_lane4 + m.y, emo_floor_sub(q, m.z));
-                            const unsigned lv = emo_lds_u8(lvl_a) & lmask;
-                            q -= emo_lds_u32(tab_a + lv * 4u);
-                            mem_a += 16u;
-                            lvl_a += 32u;
-                            tab_a += tab_row;
+                // Every lane's positions as one stream, four at a time.  A member's slack is T - A - X of its segment
+                // (A in its record, X where the spine left it); its tail, for the fold, is the head's tail minus the
+                // durations of the members before it.  Unused positions have no node and fold into the unread slot.
+                for (int ln = role.widx; ln < lanes; ln += W) {
+                    unsigned tab_a = sta + p.off_tab + (unsigned)(ln * K) * tab_row;
+                    unsigned lvl_a = sta + p.off_lvl + ((unsigned)((group * lanes + ln) * K) << 5) + (unsigned)lane;
+                    unsigned mem_a = sta + p.off_mem + (unsigned)(ln * K) * 32u;
+                    unsigned q = 0;
+                    for (int j0 = 0; j0 < K; j0 += 4) {
+                        uint4 m[4], n4[4];
+                        unsigned lv[4], d[4], X[4], qh[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            m[i] = emo_lds128(mem_a + 32u * i);
+                            n4[i] = emo_lds128(mem_a + 32u * i + 16u);
+                            lv[i] = emo_lds_u8(lvl_a + 32u * i);
                         }
-                    } else {
-#pragma unroll 4
-                        for (int j = 0; j < cnt; ++j) {
-                            const uint4 m = emo_lds128(mem_a);
-                            emo_stg_s64_if(sl_lane, m.x, ldo8, sl, sl_ok);
-                            mem_a += 16u;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const unsigned xa = acc_a + (m[i].w >> 16) * 128u;
+                            X[i] = emo_lds_u32(xa);
+                            qh[i] = emo_lds_u32(xa + 128u);
+                            d[i] = emo_lds_u32(tab_a + (unsigned)i * tab_row + (lv[i] & lmask) * 4u);
                         }
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const long long A = (long long)((unsigned long long)n4[i].x | ((unsigned long long)n4[i].y << 32));
+                            const long long sl = (T - A) - (long long)(unsigned long long)X[i];
+                            emo_stg_s64_if(sl_lane, m[i].x, ldo8, sl, sl_ok & (unsigned)(m[i].x != emo::kNone));
+                            q = (m[i].w & emo::kSpPos_First) ? qh[i] : q;
+                            emo_red_max_u32(slot_lane4 + m[i].y, emo_floor_sub(q, m[i].z));
+                            q -= d[i];
+                        }
+                        mem_a += 128u;
+                        lvl_a += 128u;
+                        tab_a += 4u * tab_row;
                     }
                 }
                 __syncwarp();
@@ -406,7 +491,16 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_bwd(FlowParams p)
                     emo_mbar_arrive(emo_spine_bar(p, smem0, group, a, 2));
                     emo_mbar_arrive(bar0 + 8 * (kFlowMaxBuf + s));
                 }
+                t_postw += EMO_SCLK() - tq1;
             }
+        }
+        if (p.prof && lane == 0 && blockIdx.x < 512) {
+            long long *pr = p.prof + ((size_t)blockIdx.x * 32 + warp) * 8;
+            pr[0] = t_w1;
+            pr[1] = t_w2;
+            pr[2] = EMO_SCLK() - t_begin;
+            pr[3] = t_prew;
+            pr[4] = t_postw;
         }
     }
     if (failed && lane == 0) {

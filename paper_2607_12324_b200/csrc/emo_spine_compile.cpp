@@ -150,8 +150,17 @@ int build_spine(const SpineIn &in, Spine &out, std::string &err)
     out.n_segs.assign((size_t)stages, 0);
     out.seg.assign((size_t)stages * std::max(max_segs, 1) * kSpSegWords, 0);
     out.mem.assign((size_t)stages * lanes * K * kSpMemWords, 0);
+    out.posw.assign((size_t)stages * lanes * K, 0);
     const uint32_t zero_slot = (uint32_t)lanes, dummy_slot = (uint32_t)lanes + 1u;
     auto slot_addr = [](uint32_t id) { return id * 128u; };
+    if (max_segs >= 4096 || acc_words + 2 >= 65536) return EMO_OK;      // the position word has no room: no spine program
+    // unused positions: no node, folds go to the slot nobody reads
+    for (size_t q = 0; q < (size_t)stages * lanes * K; ++q) {
+        out.mem[q * kSpMemWords + 0] = kNone;
+        out.mem[q * kSpMemWords + 1] = slot_addr(dummy_slot);
+        out.posw[q] = (uint32_t)(acc_words) << 16;      // sums of unused positions go to the scratch word
+        out.mem[q * kSpMemWords + 3] = out.posw[q];
+    }
     for (int st = 0; st < stages; ++st) {
         out.n_segs[st] = (uint32_t)stage_segs[st].size();
         for (int32_t si : stage_segs[st]) {
@@ -162,6 +171,14 @@ int build_spine(const SpineIn &in, Spine &out, std::string &err)
             w[1] = s.acc * 128u;
             w[2] = (uint32_t)(uint64_t)A;
             w[3] = (uint32_t)((uint64_t)A >> 32);
+            for (int32_t j = 0; j < s.count; ++j) {
+                const size_t q = ((size_t)st * lanes + s.lane) * K + s.first + j;
+                const uint32_t pw = (j == 0 ? kSpPos_First : 0u) | (j == s.count - 1 ? kSpPos_Last : 0u) | ((uint32_t)s.idx << 4) | (s.acc << 16);
+                out.posw[q] = pw;
+                out.mem[q * kSpMemWords + 3] = pw;
+                out.mem[q * kSpMemWords + 4] = w[2];
+                out.mem[q * kSpMemWords + 5] = w[3];
+            }
         }
     }
 
