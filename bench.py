@@ -368,7 +368,7 @@ def main():
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "int64", "data": "synthetic",
             "config": workload_config(args.workload, args.scale, g, B, ppm),
-            "details": {"kernels": {2: "32-bit lane-stream", 1: "staged 64-bit", 0: "plain 64-bit"}[path],
+            "details": {"kernels": {4: "32-bit spine", 3: "generic", 2: "32-bit lane-stream", 1: "staged 64-bit", 0: "plain 64-bit"}[path],
                         "slack_sums": bool(args.sums), "lanes": fl["lanes"] if path == 2 else info.lanes,
                         "steps": fl["steps"] if path == 2 else info.steps_fwd, "stage_steps": fl["K"], "barrier_steps": fl["sync"],
                         "restore_rows": fl["pushes"], "depth": info.depth, "graph_load_s": t_load,
@@ -380,6 +380,8 @@ def main():
             "selected": {"index": int(sel[0].item()), "T": int(sel[1].item()), "E": float(selE.item()),
                          "T0": int(T0.item()), "E0": float(E0.item())}}
 
+    if path == 4:
+        line["details"]["spine"] = emo.emo_graph_spine(h)
     # end to end through the host-buffer entry point: the levels come from pinned host memory every step, packed
     # at ceil(log2 L) bits each (the call spreads them to bytes on the device), per-policy results and the
     # selection go back to the host; the slack matrix stays on the device

@@ -201,25 +201,16 @@ __device__ __forceinline__ bool emo_flow_wait(unsigned bar, unsigned parity, vol
     return emo_flow_wait_slow(bar, parity, abort_word, limit);
 }
 
-// The same for warps whose wake-up time is on the critical path of a short stage: the wait is left to the hardware
-// (try_wait with a suspend-time hint: the warp sleeps inside the instruction until the phase completes or the hint runs
-// out), so a waiting warp issues next to nothing and wakes at once.
-__device__ __forceinline__ bool emo_mbar_try_hint(unsigned bar, unsigned parity, unsigned hint_ns)
-{
-    unsigned ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity), "r"(hint_ns)
-        : "memory");
-    return ok != 0;
-}
+// The same with one barrier read per poll (test_wait; a try_wait spins inside, several reads and naps per call): for
+// kernels whose stages are short, where the polls of the waiting warps add up.
 __device__ __noinline__ bool emo_flow_wait_fast_slow(unsigned bar, unsigned parity, volatile int *abort_word, long long limit)
 {
     const long long t0 = clock64();
     for (;;) {
-        for (unsigned i = 0; i < 64u; ++i)
-            if (emo_mbar_try_hint(bar, parity, 20000u)) return true;
+        for (unsigned i = 0; i < 1024u; ++i) {
+            __nanosleep(300);
+            if (emo_mbar_test(bar, parity)) return true;
+        }
         if (*abort_word || clock64() - t0 > limit) return false;
     }
 }

@@ -22,19 +22,32 @@
 #pragma once
 #include "emo_flow.cuh"
 
+__device__ __noinline__ bool emo_spine_wait_slow(unsigned bar, unsigned parity, volatile int *abort_word, long long limit)
+{
+    const long long t0 = clock64();
+    for (;;) {
+        for (unsigned i = 0; i < 4096u; ++i) {
+            if (emo_mbar_test(bar, parity)) return true;
+            if (i > 8u) __nanosleep(40);
+        }
+        if (*abort_word || clock64() - t0 > limit) return false;
+    }
+}
 __device__ __forceinline__ bool emo_spine_wait(unsigned bar, unsigned parity, volatile int *abort_word, long long limit)
 {
-    return emo_flow_wait_fast(bar, parity, abort_word, limit);
+    if (emo_mbar_test(bar, parity)) return true;
+    return emo_spine_wait_slow(bar, parity, abort_word, limit);
 }
 // The workers' waits: they run ahead of the spine (sums) or behind it (stores), so a late wake-up costs nothing,
 // while every poll of the 20-odd waiting warps takes an issue slot from the spine.
 __device__ __noinline__ bool emo_worker_wait_slow(unsigned bar, unsigned parity, volatile int *abort_word, long long limit)
 {
+    // test_wait, not try_wait: try_wait spins inside (several barrier reads and naps per call)
     const long long t0 = clock64();
     for (;;) {
         for (unsigned i = 0; i < 1024u; ++i) {
-            if (emo_mbar_try(bar, parity)) return true;
-            __nanosleep(250);
+            __nanosleep(200);
+            if (emo_mbar_test(bar, parity)) return true;
         }
         if (*abort_word || clock64() - t0 > limit) return false;
     }
@@ -130,7 +143,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_fwd(FlowParams p)
     double ea = 0.0;
     bool failed = false;
     if (role.producer) {
-        emo_flow_produce<false>(p, stage0, bar0, abort_word, lane, role.widx);
+        emo_flow_produce<false, true>(p, stage0, bar0, abort_word, lane, role.widx);
     } else if (role.spine) {
         const unsigned slot_lane4 = smem0 + (unsigned)group * p.slot_bytes + (unsigned)lane * 4u;
         uint32_t *const rst_lane = p.restore ? p.restore + (size_t)blockIdx.x * p.restore_rows * ptile + col : nullptr;
@@ -316,7 +329,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_bwd(FlowParams p)
 
     bool failed = false;
     if (role.producer) {
-        emo_flow_produce<true>(p, stage0, bar0, abort_word, lane, role.widx);
+        emo_flow_produce<true, true>(p, stage0, bar0, abort_word, lane, role.widx);
     } else if (role.spine) {
         // the lanes' last completion offsets: where the walk back begins
         for (int ln = 0; ln < lanes; ++ln)
