@@ -62,8 +62,7 @@ extern "C" {
 #define EMO_F_PAIR_KERNEL 0x4u     /* staged pass kernel with two policies per thread (default only for very large batches) */
 #define EMO_F_LANE_KERNEL 0x8u     /* staged pass kernel with one policy per thread (the default otherwise) */
 #define EMO_F_FLOW_KERNEL 0x10u    /* the 32-bit lane-stream kernels (the default only for large batches: n * B >= 2^31) */
-#define EMO_F_SPINE_KERNEL 0x20u   /* the spine kernels (slack matrix and per-policy results only; the default on graphs of at most
-                                    * eight lanes while n * B < 2^31) */
+#define EMO_F_SPINE_KERNEL 0x20u   /* the spine kernels (the default on graphs of at most eight lanes while n * B < 2^31) */
 #define EMO_F_TEST_STALL 0x100u    /* test hook of the 32-bit kernels: the producer warps stop half way, so that the
                                       consumers' bounded waits run out and EMO_E_TIMEOUT is reported */
 
@@ -412,7 +411,7 @@ int emo_set_pass_events(void *fwd_start, void *fwd_stop, void *bwd_start, void *
 
 /*
  * emo_call_path - which kernels emo_eval_policies (need_slack = 0) or emo_slack_batch (need_slack = 1)
- * would run for these arguments: 2 = the 32-bit lane-stream kernels, 1 = the staged 64-bit kernels,
+ * would run for these arguments: 4 = the spine kernels, 2 = the 32-bit lane-stream kernels, 1 = the staged 64-bit kernels,
  * 0 = the plain-load 64-bit kernels, 3 = the generic kernels (a graph beyond the on-chip schedules' limits, or
  * loaded with EMO_F_GENERIC); negative = an EMO_E_* code.  lvl may be any pointer with the
  * alignment of the real one.  For tests and reports; it launches nothing.
@@ -447,8 +446,11 @@ int emo_measure_warp_costs(double *cycles, void *scratch_dev, void *stream);
  * [((pass * 512 + block) * 32 + warp) * 8] for the first 512 blocks (pass 0 forward, 1 backward): consumer
  * warps {cycles waiting for staged data, cycles at group barriers, total, backward only: cycles in
  * entries that need their record, cycles in runs of simple entries}, producer warps {cycles waiting
- * for a free buffer, cycles issuing copies, total}; the other words are spare.  NULL switches it off.
- * Process-wide.
+ * for a free buffer, cycles issuing copies, total}; the other words are spare.  The spine kernels fill the same
+ * array: spine warps {waiting for staged data, waiting for the workers' sums, total, inside the operation loop,
+ * backward: waiting for the stores two stages back}, forward workers {waiting for staged data, waiting for a free
+ * buffer of sums, total}, backward workers {both of those, waiting for the spine, total, sums, stores}.
+ * NULL switches it off.  Process-wide.
  */
 int emo_set_flow_counters(void *dev);
 

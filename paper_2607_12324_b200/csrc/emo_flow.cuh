@@ -189,7 +189,7 @@ __device__ __noinline__ bool emo_flow_wait_slow(unsigned bar, unsigned parity, v
     const long long t0 = clock64();
     for (;;) {
         for (unsigned i = 0; i < 256u; ++i) {
-            if (emo_mbar_try(bar, parity)) return true;
+            if (emo_mbar_test(bar, parity)) return true;      // one barrier read per poll (a try_wait spins inside)
             __nanosleep(400);      // polling costs issue slots that the working warps need
         }
         if (*abort_word || clock64() - t0 > limit) return false;

@@ -90,7 +90,7 @@ constexpr uint32_t kOpOffMask = (1u << 29) - 1u;
 constexpr int kSpOpWordsF = 8;        // a0, d0, a1, d1, lane slot, published slot, sum offset, flags | push row << 8 | pool index << 20
 constexpr int kSpOpWordsB = 12;       // the same eight (flags | pop row << 8), then: slot to clear, lane's completion slot, spare, spare
 constexpr int kSpSegWords = 4;        // lane | first position << 8 | members << 16 | flags << 24, sum offset, A_v low, high
-constexpr int kSpMemWords = 8;        // node (kNone: unused position), fold slot, fold correction, position word, A_v low, high, spare, spare
+constexpr int kSpMemWords = 8;        // node (kNone: unused position), fold slot, fold correction, position word, A_v low, high, lbES_v low, high
 // position word (one per lane position of a stage): bit 0 = first member of its segment, bit 1 = last member,
 // bits 4..15 = index of the segment in the stage's list, bits 16..31 = offset of the segment's sum in 128-byte units
 constexpr uint32_t kSpPos_First = 1u, kSpPos_Last = 2u;
@@ -109,7 +109,7 @@ struct SpineDir {
 struct Spine {
     bool ok = false;
     int max_segs = 0, max_pool = 0;
-    int acc_words = 0;                // 4-byte words per policy that the sums / results of one stage take
+    int acc_words = 0;                // 4-byte words per policy that the sums / results of one stage take (two per segment)
     int64_t pushes = 0;
     int64_t segments = 0;
     std::vector<uint32_t> n_segs;     // [stages]

@@ -948,7 +948,8 @@ int launch_spine_fwd(const emo_graph *g, const FlowPlan &pl, int64_t B, const ui
 }
 
 int launch_spine_bwd(const emo_graph *g, const FlowPlan &pl, int64_t B, const uint8_t *lvl, int64_t ldb, uint32_t *restore,
-                     int64_t *slack, int64_t ldo, int64_t *makespan, int32_t *status, uint32_t flags, cudaStream_t st)
+                     int64_t *ES, int64_t *LS, int64_t *slack, int64_t ldo, int64_t *makespan, int64_t *slack_sum,
+                     int32_t *n_critical, int32_t *status, uint32_t flags, cudaStream_t st)
 {
     if (B == 0) return EMO_OK;
     FlowParams p = pl.pb;
@@ -957,14 +958,20 @@ int launch_spine_bwd(const emo_graph *g, const FlowPlan &pl, int64_t B, const ui
     p.ldb = ldb;
     p.restore = restore;
     p.makespan = makespan;
+    p.ES = ES;
+    p.LS = LS;
     p.slack = slack;
     p.ldo = ldo;
+    p.slack_sum = slack_sum;
+    p.n_critical = n_critical;
     p.status = status;
     p.prof = g_flow_prof ? g_flow_prof + 131072 : nullptr;
     if (flags & EMO_F_TEST_STALL) p.stall_stage = p.stages / 2;
     cudaEvent_t ev0 = g_pass_events[2], ev1 = g_pass_events[3];
     if (ev0) EMO_CUDA(cudaEventRecord(ev0, st));
-    void (*kern)(FlowParams) = pl.threads <= 512 ? emo_spine_bwd<512> : emo_spine_bwd<1024>;
+    const bool extra = ES || LS || slack_sum || n_critical;
+    void (*kern)(FlowParams) = pl.threads <= 512 ? (extra ? emo_spine_bwd<512, true> : emo_spine_bwd<512, false>)
+                                                 : (extra ? emo_spine_bwd<1024, true> : emo_spine_bwd<1024, false>);
     if (flow_optin(kern, g) != EMO_OK) { (void)cudaGetLastError(); return EMO_E_CUDA; }
     kern<<<pl.grid_b, pl.threads, pl.smem_b, st>>>(p);
     EMO_CUDA(cudaGetLastError());
@@ -972,8 +979,7 @@ int launch_spine_bwd(const emo_graph *g, const FlowPlan &pl, int64_t B, const ui
     return EMO_OK;
 }
 
-// Whether a call takes the spine kernels: the program exists, the call wants at most the slack matrix
-// beside the per-policy results, and either the caller asks for them (EMO_F_SPINE_KERNEL) or the graph is narrow
+// Whether a call takes the spine kernels: the program exists and either the caller asks for them (EMO_F_SPINE_KERNEL) or the graph is narrow
 // and the batch below the large-batch rule of the lane-stream kernels.
 bool spine_allowed(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t ldb, int64_t ldo, bool extra, uint32_t flags)
 {
@@ -1052,7 +1058,7 @@ int emo_call_path(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t ldb
     if (!g || B < 0) return EMO_E_INVALID_ARG;
     if (g->host_only) return EMO_E_CUDA;
     if (g->generic) return 3;
-    if (spine_allowed(g, B, lvl, ldb, need_slack ? ldo : 0, need_slack == 2, flags)) {
+    if (spine_allowed(g, B, lvl, ldb, need_slack ? ldo : 0, false, flags)) {
         FlowPlan fp;
         if (spine_plan(g, B, true, need_slack != 0, fp)) return 4;
     }
@@ -1911,7 +1917,7 @@ int emo_slack_batch(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t l
     if (g->generic)
         return launch_generic(g, B, lvl, ldb, true, ES, LS, slack, ldo, makespan, energy, slack_sum, n_critical, T0, E0, ws, ws_bytes,
                               st);
-    if (spine_allowed(g, B, lvl, ldb, ldo, ES || LS || slack_sum || n_critical, flags)) {
+    if (spine_allowed(g, B, lvl, ldb, ldo, false, flags)) {
         FlowPlan fp;
         if (spine_plan(g, B, T0 || E0, true, fp)) {
             const size_t head = kSmallWs + lvl_area(g);
@@ -1919,7 +1925,7 @@ int emo_slack_batch(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t l
             uint32_t *restore = (uint32_t *)((char *)ws + head);
             int rc = launch_spine_fwd(g, fp, B, lvl, ldb, restore, makespan, energy, T0, E0, status, flags, st);
             if (rc) return rc;
-            return launch_spine_bwd(g, fp, B, lvl, ldb, restore, slack, ldo, makespan, status, flags, st);
+            return launch_spine_bwd(g, fp, B, lvl, ldb, restore, ES, LS, slack, ldo, makespan, slack_sum, n_critical, status, flags, st);
         }
     }
     if (flow_allowed(g, B, lvl, ldb, ldo, flags)) {

@@ -305,9 +305,9 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_fwd(FlowParams p)
 // X = co + qin of its members (slack = T - A - X for all of them) and, where members are folded, the
 // head's tail; the workers store the slack and fold the members' tails one stage behind the spine, which
 // before a stage waits for the stores of the stage two back (folded values are read at least two stages
-// after they are written).
+// after they are written).  EXTRA: also ES, LS, the slack sums and critical counts (ES_v = lbES_v + X - tail_v).
 // ---------------------------------------------------------------------------------------------------
-template <int MAXT>
+template <int MAXT, bool EXTRA>
 __global__ void __launch_bounds__(MAXT, 1) emo_spine_bwd(FlowParams p)
 {
     extern __shared__ __align__(128) unsigned char emo_smem[];
@@ -328,6 +328,8 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_bwd(FlowParams p)
     const unsigned slot_lane4 = smem0 + (unsigned)group * p.slot_bytes + (unsigned)lane * 4u;
 
     bool failed = false;
+    long long ssum = 0;
+    int ncrit = 0;
     if (role.producer) {
         emo_flow_produce<true, true>(p, stage0, bar0, abort_word, lane, role.widx);
     } else if (role.spine) {
@@ -406,6 +408,9 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_bwd(FlowParams p)
         const unsigned ldo8 = (unsigned)p.ldo * 8u;
         long long *const sl_lane = (p.slack && act) ? reinterpret_cast<long long *>(p.slack) + b : nullptr;
         const unsigned sl_ok = sl_lane != nullptr;
+        long long *const es_lane = (EXTRA && p.ES && act) ? reinterpret_cast<long long *>(p.ES) + b : nullptr;
+        long long *const ls_lane = (EXTRA && p.LS && act) ? reinterpret_cast<long long *>(p.LS) + b : nullptr;
+        const unsigned es_ok = es_lane != nullptr, ls_ok = ls_lane != nullptr;
         for (int cst = 0; cst <= p.stages && !failed; ++cst) {
             if (cst < p.stages) {
                 // the sums of stage cst
@@ -489,8 +494,18 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_bwd(FlowParams p)
                         for (int i = 0; i < 4; ++i) {
                             const long long A = (long long)((unsigned long long)n4[i].x | ((unsigned long long)n4[i].y << 32));
                             const long long sl = (T - A) - (long long)(unsigned long long)X[i];
-                            emo_stg_s64_if(sl_lane, m[i].x, ldo8, sl, sl_ok & (unsigned)(m[i].x != emo::kNone));
+                            const unsigned real = (unsigned)(m[i].x != emo::kNone);
+                            emo_stg_s64_if(sl_lane, m[i].x, ldo8, sl, sl_ok & real);
                             q = (m[i].w & emo::kSpPos_First) ? qh[i] : q;
+                            if (EXTRA) {
+                                // ES_v = lbES_v + eo_v with eo_v = X - tail_v (X = eo + tail for every member)
+                                const long long lb = (long long)((unsigned long long)n4[i].z | ((unsigned long long)n4[i].w << 32));
+                                const long long es = lb + (long long)(unsigned long long)(X[i] - q);
+                                emo_stg_s64_if(es_lane, m[i].x, ldo8, es, es_ok & real);
+                                emo_stg_s64_if(ls_lane, m[i].x, ldo8, es + sl, ls_ok & real);
+                                ssum += real ? sl : 0;
+                                ncrit += (real && sl == 0) ? 1 : 0;
+                            }
                             emo_red_max_u32(slot_lane4 + m[i].y, emo_floor_sub(q, m[i].z));
                             q -= d[i];
                         }
@@ -519,6 +534,26 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_bwd(FlowParams p)
     if (failed && lane == 0) {
         *abort_word = 1;
         if (p.status) atomicMin(p.status, -8);
+    }
+    if (EXTRA) {
+        // per-policy sums: the workers' parts combined in worker order
+        __syncthreads();
+        long long *part = reinterpret_cast<long long *>(emo_smem + p.off_stage0);
+        if (!role.producer && !role.spine) {
+            long long *pd = part + ((size_t)(group * W + role.widx) * 32 + lane) * 2;
+            pd[0] = ssum;
+            pd[1] = (long long)ncrit;
+        }
+        __syncthreads();
+        if (role.spine && act && !*abort_word) {
+            long long s2 = 0, cnt = 0;
+            for (int k = 0; k < W; ++k) {
+                s2 += part[((size_t)(group * W + k) * 32 + lane) * 2];
+                cnt += part[((size_t)(group * W + k) * 32 + lane) * 2 + 1];
+            }
+            if (p.slack_sum) p.slack_sum[b] = s2;
+            if (p.n_critical) p.n_critical[b] = (int32_t)cnt;
+        }
     }
 }
 #undef EMO_SCLK

@@ -137,7 +137,7 @@ int build_spine(const SpineIn &in, Spine &out, std::string &err)
             Seg &s = segs[ss[i]];
             s.idx = (int32_t)i;
             s.acc = off;
-            off += (s.flags & kSpSeg_Fold) ? 2u : 1u;
+            off += 2u;      // the sum, then X; beside it the head's tail (the storing warps need both)
         }
         max_segs = std::max(max_segs, (int)ss.size());
         acc_words = std::max(acc_words, (int)off);
@@ -283,6 +283,8 @@ int build_spine(const SpineIn &in, Spine &out, std::string &err)
                         uint32_t *w = &out.mem[(((size_t)st * lanes + s.lane) * K + s.first + j) * kSpMemWords];
                         w[0] = (uint32_t)u;
                         w[1] = slot_addr(dummy_slot);
+                        w[6] = (uint32_t)(uint64_t)lbES[u];
+                        w[7] = (uint32_t)((uint64_t)lbES[u] >> 32);
                         const int32_t r = fold_reader[u];
                         if (r >= 0) {
                             if (fold_slot[r] < 0) fold_slot[r] = fpool.take();
@@ -330,11 +332,10 @@ int build_spine(const SpineIn &in, Spine &out, std::string &err)
                 if (bpub[h] && s.readersB > 0) s.pubB = pool.take();
                 uint32_t fl = (s.flags & kSpSeg_PreB) ? 0u : kSp_NoSum;
                 if (s.push >= 0) fl |= kSp_Push | ((uint32_t)s.push << 8);
-                const bool wide = (s.flags & kSpSeg_Fold) != 0;
                 const uint32_t w12[kSpOpWordsB] = {addr_of(ops[0]), ops[0].delta, addr_of(ops[1]), ops[1].delta,
                                                    slot_addr((uint32_t)s.lane), slot_addr(s.pubB >= 0 ? (uint32_t)s.pubB : dummy_slot), s.acc * 128u, fl,
                                                    clear_of(ops[0], ops[1]), slot_addr(c_slot0 + (uint32_t)s.lane),
-                                                   (wide ? s.acc + 1u : scratch_acc + 1u) * 128u, 0u};
+                                                   (s.acc + 1u) * 128u, 0u};
                 opsB[st].insert(opsB[st].end(), w12, w12 + kSpOpWordsB);
                 for (int32_t id : temps) pool.give(id);
                 for (int32_t id : done) pool.give(id);

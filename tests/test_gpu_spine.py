@@ -1,6 +1,6 @@
 """GPU parity of the spine kernels (one warp per policy group carries the recurrence of Eq. 1, the other
 warps do the look-ups, the sums per segment and the stores) against the CPU oracle, through the C ABI:
-makespan and slack bit-exact, energy within 1e-9 relative."""
+makespan, ES, LS, slack, slack sums and critical counts bit-exact, energy within 1e-9 relative."""
 from __future__ import annotations
 
 import os
@@ -9,7 +9,7 @@ import numpy as np
 import pytest
 
 from paper_2607_12324_b200 import workloads as W
-from tests.test_gpu_parity import E_RTOL, emo, gpu_eval, gpu_slack_batch, torch_cuda  # noqa: F401  (fixtures)
+from tests.test_gpu_parity import E_RTOL, assert_matches, emo, gpu_eval, gpu_slack_batch, torch_cuda  # noqa: F401  (fixtures)
 
 pytestmark = pytest.mark.gpu
 
@@ -24,6 +24,11 @@ def check(torch, emo, oracle_mod, g, h, lv_dev, B, r_or, ldo=None, flags=None):
     assert (r["slack"][:, B:] == -7).all(), "padding columns of the slack matrix were written"
     assert r["T0"] == base["makespan"][0]
     assert r["E0"] == pytest.approx(base["energy"][0], rel=E_RTOL)
+    # every per-node output and the per-policy sums
+    r2 = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, flags=fl, ldo=ldo)
+    assert_matches(r2, r_or, B)
+    for k in ("ES", "LS", "slack"):
+        assert (r2[k][:, B:] == -7).all(), "padding columns of the outputs were written"
     T, E, st = gpu_eval(torch, emo, h, lv_dev, B, fl | emo.EMO_F_VALIDATE)
     assert st == 0 and np.array_equal(T, r_or["makespan"])
     np.testing.assert_allclose(E, r_or["energy"], rtol=E_RTOL)
