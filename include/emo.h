@@ -501,6 +501,27 @@ int emo_graph_flow(const emo_graph *g, emo_flow_view *out);
  * slots, most segments of a stage, 4-byte words of sums per policy and stage, restore rows.  Host memory. */
 int emo_graph_spine(const emo_graph *g, int64_t out[12]);
 
+/* The spine program itself, as pointers into the handle's host memory (valid until emo_graph_free; for the host-side
+ * tests of the compiler, which interpret it).  Arrays: n_ops_fwd / n_ops_bwd [stages]; ops_fwd [stages][max_ops_fwd][8]
+ * = {operand slot 0, its correction, operand slot 1, its correction, the lane's slot, published slot, offset of the
+ * segment's sum, flags (1 = sum is zero, 2 = push to the restore list, 4 = terminal) | restore row in the stage << 8 |
+ * index of the terminal bound << 20}, slots and sums as byte offsets in units of 128; ops_bwd [stages][max_ops_bwd][12]
+ * = the same eight (2 = pop), then {slot to clear, slot of the lane's completion offset, offset where the head's tail
+ * goes, spare}; mem [stages][lanes * K][8] = {node (0xFFFFFFFF: unused position), fold slot, fold correction, position
+ * word (bit 0 first member, bit 1 last member of its segment, bits 16..31 offset of the segment's sum in units of 128
+ * bytes), A_v low, high, lbES_v low, high}; pos [stages][lanes * K] the position words alone; pool [stages][max_pool]
+ * lower bounds of terminal completions; push_base [stages + 1]; rows [stages][lanes][K] policy row of a position
+ * (0xFFFFFFFF: none); tab_fwd [stages][lanes][K][Lp][3] = {duration - dmin, energy high word, low word};
+ * tab_bwd [stages][lanes][K][Lp]. */
+typedef struct emo_spine_view {
+    int32_t ok, lanes, K, stages, Lp, max_ops_fwd, max_ops_bwd, max_pool, acc_words, slots_fwd, slots_bwd;
+    int64_t pushes;
+    const uint32_t *n_ops_fwd, *ops_fwd, *n_ops_bwd, *ops_bwd, *mem, *pos, *rows, *tab_fwd, *tab_bwd;
+    const uint64_t *pool;
+    const int64_t *push_base;
+} emo_spine_view;
+int emo_graph_spine_view(const emo_graph *g, emo_spine_view *out);
+
 #ifdef __cplusplus
 }
 #endif

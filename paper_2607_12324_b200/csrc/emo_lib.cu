@@ -1438,6 +1438,39 @@ int emo_graph_spine(const emo_graph *g, int64_t out[12])
     return EMO_OK;
 }
 
+int emo_graph_spine_view(const emo_graph *g, emo_spine_view *v)
+{
+    if (!g || !v) return EMO_E_INVALID_ARG;
+    std::memset(v, 0, sizeof *v);
+    const Flow &f = g->sflow;
+    const Spine &sp = f.spine;
+    if (!f.ok32 || !sp.ok) return EMO_OK;
+    v->ok = 1;
+    v->lanes = f.lanes;
+    v->K = f.K;
+    v->stages = f.stages;
+    v->Lp = f.Lp;
+    v->max_ops_fwd = sp.f.max_ops;
+    v->max_ops_bwd = sp.b.max_ops;
+    v->max_pool = sp.max_pool;
+    v->acc_words = sp.acc_words;
+    v->slots_fwd = sp.f.slots;
+    v->slots_bwd = sp.b.slots;
+    v->pushes = sp.pushes;
+    v->n_ops_fwd = sp.f.n_ops.data();
+    v->ops_fwd = sp.f.ops.data();
+    v->n_ops_bwd = sp.b.n_ops.data();
+    v->ops_bwd = sp.b.ops.data();
+    v->mem = sp.mem.data();
+    v->pos = sp.posw.data();
+    v->rows = f.rows.data();
+    v->tab_fwd = f.tabF.data();
+    v->tab_bwd = f.tabB.data();
+    v->pool = sp.pool.data();
+    v->push_base = sp.push_base.data();
+    return EMO_OK;
+}
+
 int emo_graph_program(const emo_graph *g, int dir, int32_t *lanes, int32_t *steps, int32_t *slots,
                       int32_t *Lp, const uint32_t **entries, const uint32_t **rows, const uint32_t **lat)
 {

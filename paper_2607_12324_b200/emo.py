@@ -33,7 +33,7 @@ EXPORTS = [
     "emo_strerror", "emo_graph_load", "emo_graph_free", "emo_graph_info", "emo_workspace_bytes",
     "emo_eval_policies", "emo_slack_batch", "emo_slack", "emo_baseline", "emo_target_from_delta",
     "emo_select", "emo_transpose_policies", "emo_slack_batch_host", "emo_graph_program",
-    "emo_set_pass_events", "emo_select_static", "emo_graph_flow", "emo_graph_spine", "emo_set_wait_limit", "emo_call_path", "emo_set_flow_counters", "emo_workspace_bytes_for", "emo_measure_int_issue", "emo_measure_warp_costs", "emo_eval_intervals", "emo_workspace_bytes_intervals", "emo_search_dp", "emo_workspace_bytes_search", "emo_pack_greedy", "emo_pack_tables", "emo_pack_model", "emo_pack_classes", "emo_pack_levels", "emo_unpack_levels", "emo_slack_batch_host_packed",
+    "emo_set_pass_events", "emo_select_static", "emo_graph_flow", "emo_graph_spine", "emo_graph_spine_view", "emo_set_wait_limit", "emo_call_path", "emo_set_flow_counters", "emo_workspace_bytes_for", "emo_measure_int_issue", "emo_measure_warp_costs", "emo_eval_intervals", "emo_workspace_bytes_intervals", "emo_search_dp", "emo_workspace_bytes_search", "emo_pack_greedy", "emo_pack_tables", "emo_pack_model", "emo_pack_classes", "emo_pack_levels", "emo_unpack_levels", "emo_slack_batch_host_packed",
 ]
 
 
@@ -115,6 +115,7 @@ def lib():
         L.emo_set_pass_events.argtypes = [p, p, p, p]
         L.emo_graph_flow.argtypes = [p, ctypes.POINTER(emo_flow_view)]
         L.emo_graph_spine.argtypes = [p, ctypes.POINTER(ctypes.c_int64)]
+        L.emo_graph_spine_view.argtypes = [p, ctypes.POINTER(emo_spine_view)]
         L.emo_set_wait_limit.argtypes = [i64]
         L.emo_set_flow_counters.argtypes = [p]
         L.emo_measure_int_issue.argtypes = [p, p, p]
@@ -330,6 +331,43 @@ def emo_graph_spine(g: Graph) -> dict:
     _check(lib().emo_graph_spine(g.handle, out), "emo_graph_spine")
     keys = ("ok", "lanes", "K", "stages", "segments", "ops_fwd", "ops_bwd", "slots_fwd", "slots_bwd", "max_segs", "acc_words", "pushes")
     return dict(zip(keys, [int(x) for x in out]))
+
+
+class emo_spine_view(ctypes.Structure):
+    _fields_ = ([(k, ctypes.c_int32) for k in ("ok", "lanes", "K", "stages", "Lp", "max_ops_fwd", "max_ops_bwd", "max_pool",
+                                               "acc_words", "slots_fwd", "slots_bwd")]
+                + [("pushes", ctypes.c_int64)]
+                + [(k, ctypes.c_void_p) for k in ("n_ops_fwd", "ops_fwd", "n_ops_bwd", "ops_bwd", "mem", "pos", "rows", "tab_fwd",
+                                                  "tab_bwd", "pool", "push_base")])
+
+
+def emo_graph_spine_view(g: Graph) -> dict:
+    """The spine program as numpy copies (host-side inspection; see emo.h for the layouts)."""
+    v = emo_spine_view()
+    _check(lib().emo_graph_spine_view(g.handle, ctypes.byref(v)), "emo_graph_spine_view")
+    out = {k: getattr(v, k) for k, _ in emo_spine_view._fields_[:12]}
+    if not v.ok:
+        return out
+
+    def arr(ptr, count, ctype, dtype):
+        if count == 0:
+            return np.zeros(0, dtype)
+        return np.ctypeslib.as_array(ctypes.cast(ptr, ctypes.POINTER(ctype)), shape=(count,)).astype(dtype, copy=True)
+
+    u32 = ctypes.c_uint32
+    q = v.stages * v.lanes * v.K
+    out["n_ops_fwd"] = arr(v.n_ops_fwd, v.stages, u32, np.uint32)
+    out["n_ops_bwd"] = arr(v.n_ops_bwd, v.stages, u32, np.uint32)
+    out["ops_fwd"] = arr(v.ops_fwd, v.stages * v.max_ops_fwd * 8, u32, np.uint32).reshape(v.stages, v.max_ops_fwd, 8)
+    out["ops_bwd"] = arr(v.ops_bwd, v.stages * v.max_ops_bwd * 12, u32, np.uint32).reshape(v.stages, v.max_ops_bwd, 12)
+    out["mem"] = arr(v.mem, q * 8, u32, np.uint32).reshape(v.stages, v.lanes * v.K, 8)
+    out["pos"] = arr(v.pos, q, u32, np.uint32).reshape(v.stages, v.lanes * v.K)
+    out["rows"] = arr(v.rows, q, u32, np.uint32).reshape(v.stages, v.lanes * v.K)
+    out["tab_fwd"] = arr(v.tab_fwd, q * v.Lp * 3, u32, np.uint32).reshape(v.stages, v.lanes * v.K, v.Lp, 3)
+    out["tab_bwd"] = arr(v.tab_bwd, q * v.Lp, u32, np.uint32).reshape(v.stages, v.lanes * v.K, v.Lp)
+    out["pool"] = arr(v.pool, v.stages * v.max_pool, ctypes.c_uint64, np.uint64).reshape(v.stages, v.max_pool)
+    out["push_base"] = arr(v.push_base, v.stages + 1, ctypes.c_int64, np.int64)
+    return out
 
 
 def emo_graph_flow(g: Graph, arrays: bool = True) -> dict:
