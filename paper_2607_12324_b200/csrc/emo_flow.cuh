@@ -73,6 +73,7 @@ struct FlowParams {
     // terminal nodes' bounds; inside the block's shared memory the barriers of the groups and the segments' sums
     unsigned off_ops, off_mem, off_tpool, off_pos;   // off_pos: forward, one position word per lane position
     unsigned off_sbar, off_acc, acc_bytes;   // acc_bytes: one group's sums of one stage
+    unsigned acc_all_off;                // backward with ES / LS / sums: where the heads' tails of all segments start inside them
     unsigned off_oring, oring_bytes;     // forward: per group and buffer of sums, a copy of the front of the stage (header, bounds, operations)
     int workers, nacc;                   // look-up / store warps per group, buffers of sums
 };

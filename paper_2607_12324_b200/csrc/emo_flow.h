@@ -88,7 +88,8 @@ constexpr uint32_t kOpOffMask = (1u << 29) - 1u;
 // merge operations in front.  Backward, a value that a node of a much earlier stage reads (two stages
 // or more: a launch node and its kernels) is folded by the storing warps into a slot of that reader.
 constexpr int kSpOpWordsF = 8;        // a0, d0, a1, d1, lane slot, published slot, sum offset, flags | push row << 8 | pool index << 20
-constexpr int kSpOpWordsB = 12;       // the same eight (flags | pop row << 8), then: slot to clear, lane's completion slot, spare, spare
+constexpr int kSpOpWordsB = 12;       // the same eight (flags | pop row << 8), then: slot to clear, lane's completion slot, where the head's
+                                      // tail goes (beside X if members are folded, else nowhere), where it goes when all tails are kept
 constexpr int kSpSegWords = 4;        // lane | first position << 8 | members << 16 | flags << 24, sum offset, A_v low, high
 constexpr int kSpMemWords = 8;        // node (kNone: unused position), fold slot, fold correction, position word, A_v low, high, lbES_v low, high
 // position word (one per lane position of a stage): bit 0 = first member of its segment, bit 1 = last member,
@@ -109,7 +110,8 @@ struct SpineDir {
 struct Spine {
     bool ok = false;
     int max_segs = 0, max_pool = 0;
-    int acc_words = 0;                // 4-byte words per policy that the sums / results of one stage take (two per segment)
+    int acc_words = 0;                // 4-byte words per policy that the sums / results of one stage take
+    int acc_words_all = 0;            // the same when every segment's head tail is kept (one more word per segment, behind the others)
     int64_t pushes = 0;
     int64_t segments = 0;
     std::vector<uint32_t> n_segs;     // [stages]

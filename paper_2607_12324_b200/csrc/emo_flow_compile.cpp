@@ -178,10 +178,7 @@ int compile_flow(const HostGraph &g, const int64_t *lat, const double *energy, i
         int lanes2 = 0;
         rc = schedule_ops(preds, lanes_req, lookahead, s2, l2, p2, S2, lanes2, err, nullptr);
         if (rc != EMO_OK) return rc;
-        // more than 5 % (and 32 steps) longer: not worth it.  A spine program pays per operation, not per step, and
-        // needs the distance for its folds: it accepts 25 % and four stages.
-        const bool too_long = spine ? (int64_t)S * 100 > (int64_t)S2 * 125 + 400 * (int64_t)K : (int64_t)S * 100 > (int64_t)S2 * 105 + 3200;
-        if (too_long) {
+        if ((int64_t)S * 100 > (int64_t)S2 * 105 + 3200) {      // more than 5 % (and 32 steps) longer: not worth it
             step_of.swap(s2);
             lane_of.swap(l2);
             prev_on_lane.swap(p2);

@@ -822,7 +822,7 @@ int launch_flow_bwd(const emo_graph *g, const FlowPlan &pl, int64_t B, const uin
 // Launch shape of the spine kernels: the policy tile of flow_plan; per group one spine warp and as many worker
 // warps as the block has room for (at most 6); three buffers of sums when they fit (workers one stage ahead and
 // one behind the spine) and up to six stage buffers.
-bool spine_plan(const emo_graph *g, int64_t B, bool want_base, bool need_bwd, FlowPlan &pl)
+bool spine_plan(const emo_graph *g, int64_t B, bool want_base, bool need_bwd, FlowPlan &pl, bool extra = false)
 {
     const Flow &f = g->sflow;
     const Spine &sp = f.spine;
@@ -841,10 +841,10 @@ bool spine_plan(const emo_graph *g, int64_t B, bool want_base, bool need_bwd, Fl
         if (W < 1) continue;
         const size_t P = 32 * (size_t)G;
         const size_t lvl_bytes = (size_t)G * f.lanes * f.K * 32;
-        const size_t acc_bytes = (size_t)sp.acc_words * 128;
         auto shape = [&](bool backward, FlowParams &p, size_t &smem) {
             const SpineDir &dir = backward ? sp.b : sp.f;
             const size_t slot_bytes = (size_t)dir.slots * 128;
+            const size_t acc_bytes = (size_t)((backward && extra) ? sp.acc_words_all : sp.acc_words) * 128;
             const size_t blob = backward ? d.blobB_bytes : d.blobF_bytes;
             const size_t rst = backward ? (size_t)d.max_push * P * 4 : 0;
             const size_t stage = round_up(blob + lvl_bytes + rst, 128);
@@ -897,6 +897,7 @@ bool spine_plan(const emo_graph *g, int64_t B, bool want_base, bool need_bwd, Fl
             p.off_oring = (unsigned)off_oring;
             p.oring_bytes = (unsigned)oring;
             p.acc_bytes = (unsigned)acc_bytes;
+            p.acc_all_off = (unsigned)sp.acc_words * 128u;
             p.off_stage0 = (unsigned)head;
             p.pushes = sp.pushes;
             p.restore_rows = sp.pushes + f.lanes;
@@ -1952,7 +1953,7 @@ int emo_slack_batch(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t l
                               st);
     if (spine_allowed(g, B, lvl, ldb, ldo, false, flags)) {
         FlowPlan fp;
-        if (spine_plan(g, B, T0 || E0, true, fp)) {
+        if (spine_plan(g, B, T0 || E0, true, fp, ES || LS || slack_sum || n_critical)) {
             const size_t head = kSmallWs + lvl_area(g);
             if (!ws || ws_bytes < head + fp.restore_bytes) return EMO_E_OOM;
             uint32_t *restore = (uint32_t *)((char *)ws + head);

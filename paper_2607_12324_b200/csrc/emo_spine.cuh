@@ -379,7 +379,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_bwd(FlowParams p)
                 const unsigned qo = qin + S;
                 const unsigned cprev = emo_tld_u32_if(rst_a + ((fl >> 8) & 0xFFFu) * ptile4, 0u, fl & emo::kSp_Push, c - S);
                 emo_sts_u32(acc_a + c1.z, c + qin);
-                emo_sts_u32(acc_a + c2.z, qo);
+                emo_sts_u32(acc_a + (EXTRA ? c2.w : c2.z), qo);      // EXTRA: every segment's head tail is kept, in a region of its own
                 emo_sts_u32(slot_lane4 + c2.x, 0u);
                 emo_sts_u32(slot_lane4 + c1.x, qo);
                 emo_sts_u32(slot_lane4 + c1.y, qo);
@@ -487,7 +487,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_bwd(FlowParams p)
                         for (int i = 0; i < 4; ++i) {
                             const unsigned xa = acc_a + (m[i].w >> 16) * 128u;
                             X[i] = emo_lds_u32(xa);
-                            qh[i] = emo_lds_u32(xa + 128u);
+                            qh[i] = emo_lds_u32(EXTRA ? acc_a + p.acc_all_off + ((m[i].w >> 4) & 0xFFFu) * 128u : xa + 128u);
                             d[i] = emo_lds_u32(tab_a + (unsigned)i * tab_row + (lv[i] & lmask) * 4u);
                         }
 #pragma unroll

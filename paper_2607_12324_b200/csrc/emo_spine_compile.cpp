@@ -137,13 +137,14 @@ int build_spine(const SpineIn &in, Spine &out, std::string &err)
             Seg &s = segs[ss[i]];
             s.idx = (int32_t)i;
             s.acc = off;
-            off += 2u;      // the sum, then X; beside it the head's tail (the storing warps need both)
+            off += (s.flags & kSpSeg_Fold) ? 2u : 1u;      // the sum, then X; beside it the head's tail where members are folded
         }
         max_segs = std::max(max_segs, (int)ss.size());
         acc_words = std::max(acc_words, (int)off);
     }
     out.max_segs = max_segs;
     out.acc_words = acc_words + 2;      // two scratch words behind the stage's sums (merge operations write there)
+    out.acc_words_all = out.acc_words + max_segs;      // with the heads' tails of all segments behind them (calls that want ES / LS / sums)
     const uint32_t scratch_acc = (uint32_t)acc_words;
 
     // ---- segment and member lists ---------------------------------------------------------------------
@@ -323,7 +324,7 @@ int build_spine(const SpineIn &in, Spine &out, std::string &err)
                     temps.push_back(tmp);
                     const uint32_t w12[kSpOpWordsB] = {addr_of(ops[0]), ops[0].delta, addr_of(ops[1]), ops[1].delta,
                                                        slot_addr(dummy_slot), slot_addr((uint32_t)tmp), scratch_acc * 128u, kSp_NoSum,
-                                                       clear_of(ops[0], ops[1]), slot_addr(dummy_c), (scratch_acc + 1u) * 128u, 0u};
+                                                       clear_of(ops[0], ops[1]), slot_addr(dummy_c), (scratch_acc + 1u) * 128u, (scratch_acc + 1u) * 128u};
                     opsB[st].insert(opsB[st].end(), w12, w12 + kSpOpWordsB);
                     ops.erase(ops.begin(), ops.begin() + 2);
                     ops.insert(ops.begin(), Operand{(uint32_t)tmp, 0u, false});
@@ -332,10 +333,12 @@ int build_spine(const SpineIn &in, Spine &out, std::string &err)
                 if (bpub[h] && s.readersB > 0) s.pubB = pool.take();
                 uint32_t fl = (s.flags & kSpSeg_PreB) ? 0u : kSp_NoSum;
                 if (s.push >= 0) fl |= kSp_Push | ((uint32_t)s.push << 8);
+                const bool wide = (s.flags & kSpSeg_Fold) != 0;
                 const uint32_t w12[kSpOpWordsB] = {addr_of(ops[0]), ops[0].delta, addr_of(ops[1]), ops[1].delta,
                                                    slot_addr((uint32_t)s.lane), slot_addr(s.pubB >= 0 ? (uint32_t)s.pubB : dummy_slot), s.acc * 128u, fl,
                                                    clear_of(ops[0], ops[1]), slot_addr(c_slot0 + (uint32_t)s.lane),
-                                                   (s.acc + 1u) * 128u, 0u};
+                                                   (wide ? s.acc + 1u : scratch_acc + 1u) * 128u,
+                                                   ((uint32_t)out.acc_words + (uint32_t)s.idx) * 128u};
                 opsB[st].insert(opsB[st].end(), w12, w12 + kSpOpWordsB);
                 for (int32_t id : temps) pool.give(id);
                 for (int32_t id : done) pool.give(id);

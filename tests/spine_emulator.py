@@ -81,7 +81,7 @@ def run(view: dict, lv: np.ndarray, L: int, late_stores: bool = False) -> dict:
             for pos in range(K):
                 q = ln * K + pos
                 node, fold_a, fold_d, pw, A_lo, A_hi, lb_lo, lb_hi = (int(x) for x in view["mem"][st, q])
-                X, qh = a[pw >> 16], a[(pw >> 16) + 1]
+                X, qh = a[pw >> 16], a[view["acc_words"] + ((pw >> 4) & 0xFFF)]      # the region where every head's tail is kept
                 if pw & 1:
                     qv = qh.copy()
                 if node != NONE:
@@ -95,7 +95,7 @@ def run(view: dict, lv: np.ndarray, L: int, late_stores: bool = False) -> dict:
 
     order = list(range(st_n - 1, -1, -1))
     for k, st in enumerate(order):
-        a = np.zeros((view["acc_words"], B), dtype=np.uint64)
+        a = np.zeros((view["acc_words"] + 4096, B), dtype=np.uint64)
         for ln in range(lanes):
             runsum = np.zeros(B, dtype=np.uint64)
             for pos in range(K):
@@ -108,7 +108,7 @@ def run(view: dict, lv: np.ndarray, L: int, late_stores: bool = False) -> dict:
         if late_stores and k >= 2:
             stores(order[k - 2])          # the spine waits for the stores of the stage two back, no earlier
         for i in range(int(view["n_ops_bwd"][st])):
-            a0, d0, a1, d1, o_lane, o_pub, ao, fl, a_clear, c_slot, qo_off, _ = (int(x) for x in view["ops_bwd"][st, i])
+            a0, d0, a1, d1, o_lane, o_pub, ao, fl, a_clear, c_slot, qo_narrow, qo_off = (int(x) for x in view["ops_bwd"][st, i])
             x0, x1 = slots[a0 // 128], slots[a1 // 128]
             S = np.zeros(B, dtype=np.uint64) if (fl & 1) else a[ao // 128].copy()
             c = slots[c_slot // 128].copy()
@@ -120,6 +120,7 @@ def run(view: dict, lv: np.ndarray, L: int, late_stores: bool = False) -> dict:
                 cprev = restore[rrow]
             a[ao // 128] = (c + qin) & M32
             a[qo_off // 128] = qo
+            a[qo_narrow // 128] = qo      # the place beside X (segments with folded members), else a scratch word
             slots[a_clear // 128] = 0
             slots[o_lane // 128] = qo
             slots[o_pub // 128] = qo
