@@ -1252,12 +1252,13 @@ int emo_graph_load(int32_t n, const int64_t *row_ptr, const int32_t *col, const 
         if (rc != EMO_OK) { delete g; return rc; }
         if (!g->generic) {
             // stage length: the longest of 32, 16, 8 steps whose entries the producers can index
-            // (32 * kFlowRowRegs per stage); barrier distance 16 steps unless the caller says otherwise
-            // (measured on the 250 000-node workload at 0.3 scale: 8 / 16 steps gave 8.5 / 7.7 ms for both passes)
+            // (32 * kFlowRowRegs per stage); one barrier per stage unless the caller says otherwise (measured on the
+            // 250 000-node workload with 16 384 policies: 8 / 16 / 32 steps between barriers gave 24.8 / 22.3 / 21.3 ms for
+            // both passes)
             int fk = (int)((flags >> 24) & 0x3F), fs = (int)((flags >> 4) & 0xF) * 8;
             const int flanes = g->fwd.lanes > 0 ? std::max(g->fwd.lanes, g->bwd.lanes) : 1;
             if (fk == 0) fk = flanes * 32 <= 32 * kFlowRowRegs ? 32 : (flanes * 16 <= 32 * kFlowRowRegs ? 16 : 8);
-            if (fs == 0) fs = 16;
+            if (fs == 0) fs = fk;
             if (fs > fk) fs = fk;
             rc = compile_flow(h, lat, energy, lanes, look, fk, fs, g->flow, err);
             if (rc == EMO_E_UNSUPPORTED) {      // the 64-bit programs exist: they serve
