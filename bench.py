@@ -155,6 +155,48 @@ def run_reference(args, rank, world):
     print(json.dumps(line), flush=True)
 
 
+def other_workloads_leg(sm_mhz, hbm_gbs):
+    """The smaller configurations (parity-test cases, not the headline): forward + backward pass with the slack matrix,
+    default kernels, CUDA events, median of five calls after three; each beside its depth floor and its HBM time."""
+    import numpy as np
+    import torch
+    from paper_2607_12324_b200 import emo, workloads as W
+    names = {4: "32-bit spine", 3: "generic", 2: "32-bit lane-stream", 1: "staged 64-bit", 0: "plain 64-bit"}
+    out = []
+    for name in ("cfg0-tiny", "cfg1-train", "cfg2-packed", "cfg3-8dev"):
+        g = W.make_graph(name)
+        B = g.meta["B"]
+        lv = W.policies_for(g, B=B, device="cuda")
+        h = emo.load_workload(g)
+        info = h.info
+        slack = torch.empty((g.n, B), dtype=torch.int64, device="cuda")
+        T = torch.zeros(B, dtype=torch.int64, device="cuda")
+        E = torch.zeros(B, dtype=torch.float64, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        ws = torch.empty(emo.emo_workspace_bytes(h, B, 1), dtype=torch.uint8, device="cuda")
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        for e in ev:
+            e.record()
+        fw, bw = [], []
+        for it in range(8):
+            emo.emo_set_pass_events(*ev)
+            emo.emo_slack_batch(h, B, lv, lv.stride(0), None, None, slack, B, T, E, None, None, ws, status)
+            emo.emo_set_pass_events(None, None, None, None)
+            torch.cuda.synchronize()
+            if it >= 3:
+                fw.append(ev[0].elapsed_time(ev[1]))
+                bw.append(ev[2].elapsed_time(ev[3]))
+        assert int(status.item()) == 0
+        out.append({"workload": name, "n": int(g.n), "policies": int(B),
+                    "kernels": names[emo.emo_call_path(h, B, lv, lv.stride(0), B, True, 0)],
+                    "fwd_ms": float(np.median(fw)), "bwd_ms": float(np.median(bw)),
+                    "depth_floor_ms": 2 * info.depth * 30.0 / (sm_mhz * 1e6) * 1e3,
+                    "t_hbm_ms": 9.0 * g.n * B / (hbm_gbs * 1e9) * 1e3})
+        h.free()
+        del slack, lv, ws
+    return out
+
+
 def intervals_leg(args, g, B, m, T0_ns, check):
     """Times emo_eval_intervals (device-resident inputs, CUDA events) and checks a few policies against the oracle."""
     import numpy as np
@@ -232,6 +274,7 @@ def main():
     ap.add_argument("--flags", type=int, default=0, help="extra EMO_F_* load flags (lanes / look-ahead)")
     ap.add_argument("--call-flags", type=int, default=0, help="EMO_F_* flags of the pass calls (kernel choice)")
     ap.add_argument("--no-intervals", action="store_true", help="skip the time-interval policy leg (Alg. 1 in its own form)")
+    ap.add_argument("--no-others", action="store_true", help="skip the report-only timings of the smaller configurations")
     ap.add_argument("--no-search", action="store_true", help="skip the policy search (Alg. 2) inside the time-interval leg")
     ap.add_argument("--search-ppm", type=int, default=50000, help="latency budget of the policy search, parts per million of T_0")
     args = ap.parse_args()
@@ -428,6 +471,10 @@ def main():
     # idle energy, on the same graph and batch size; a separate figure, not part of `value`
     if rank == 0 and not args.no_intervals:
         line["intervals"] = intervals_leg(args, g, B, m, T0_ns=int(T0.item()), check=not args.no_cpu)
+
+    # the other configurations: report-only figures that explain themselves (depth floor, HBM time)
+    if rank == 0 and not args.no_others and args.workload == "cfg4-llm" and args.scale == 1.0:
+        line["other_workloads"] = other_workloads_leg(sm_mhz, peak)
 
     if rank == 0 and not args.no_cpu:
         threads = os.cpu_count() or 1
