@@ -402,6 +402,25 @@ int emo_slack_batch_host_packed(const emo_graph *g, int64_t B, int bits, const u
                                 void *ws, size_t ws_bytes, uint32_t flags, void *stream);
 
 /*
+ * The same in two halves, so that the copy of the next batch runs under the kernels of the current one
+ * (two device buffers of packed levels, a copy stream of the caller's):
+ * emo_levels_prefetch enqueues the host -> device copy of packed levels (rows * ld_host bytes, bits < 8 as in
+ * emo_slack_batch_host_packed; lvl_host should be pinned) on copy_stream and records `ready` (a cudaEvent_t as
+ * void*) behind it; it returns at once.
+ * emo_slack_batch_prefetched is emo_slack_batch_host_packed without the copy: `stream` waits for `ready`, then the
+ * levels in dev_packed (pitch ld_packed) are spread to dev_lvl and everything else follows as there, including the
+ * wait for the stream at the end.  The caller must not start a prefetch into a buffer before the call that reads it
+ * has returned.
+ */
+int emo_levels_prefetch(const emo_graph *g, const uint8_t *lvl_host, int64_t ld_host, uint8_t *dev_packed, void *copy_stream,
+                        void *ready);
+int emo_slack_batch_prefetched(const emo_graph *g, int64_t B, int bits, const uint8_t *dev_packed, int64_t ld_packed, void *ready,
+                               uint8_t *dev_lvl, int64_t ldb, int64_t *slack_dev, int64_t ldo, int64_t delta_ppm,
+                               int64_t *makespan_host, double *energy_host, int64_t *slack_sum_host,
+                               int32_t *n_critical_host, int64_t *sel_host, void *ws, size_t ws_bytes, uint32_t flags,
+                               void *stream);
+
+/*
  * emo_set_pass_events - measurement hook (no counterpart in the method): four cudaEvent_t handles
  * (as void*, any may be NULL) that later emo_slack_batch / emo_eval_policies / emo_baseline calls
  * record on their stream immediately before and after the forward pass kernel and before and after

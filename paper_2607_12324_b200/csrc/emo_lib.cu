@@ -2120,24 +2120,14 @@ int emo_unpack_levels(int bits, int64_t rows, int64_t B, const uint8_t *packed, 
     return repack(false, bits, rows, B, const_cast<uint8_t *>(packed), ldp, lvl, ldb, (cudaStream_t)stream);
 }
 
-int emo_slack_batch_host_packed(const emo_graph *g, int64_t B, int bits, const uint8_t *lvl_host, int64_t ld_host,
-                                uint8_t *dev_packed, uint8_t *dev_lvl, int64_t ldb, int64_t *slack_dev, int64_t ldo,
-                                int64_t delta_ppm, int64_t *makespan_host, double *energy_host, int64_t *slack_sum_host,
-                                int32_t *n_critical_host, int64_t *sel_host, void *ws, size_t ws_bytes, uint32_t flags,
-                                void *stream)
+// The passes, the selection and the copies of the per-policy results to the host, once the levels are on the device:
+// packed in dev_packed (bits < 8: spread to dev_lvl first) or as bytes in dev_lvl (bits = 8).
+static int host_batch_tail(const emo_graph *g, int64_t B, int bits, const uint8_t *dev_packed, int64_t ld_packed, uint8_t *dev_lvl,
+                           int64_t ldb, int64_t *slack_dev, int64_t ldo, int64_t delta_ppm, int64_t *makespan_host,
+                           double *energy_host, int64_t *slack_sum_host, int32_t *n_critical_host, int64_t *sel_host, void *ws,
+                           size_t need, uint32_t flags, cudaStream_t st)
 {
-    if (!g || B <= 0 || !lvl_host || !dev_lvl || !makespan_host || !energy_host || !sel_host || ldb < B)
-        return EMO_E_INVALID_ARG;
-    if (bits < 1 || bits > 8 || (bits < 8 && !dev_packed)) return EMO_E_INVALID_ARG;
-    if (g->host_only) return EMO_E_CUDA;
-    size_t need = 0, total = 0;
-    const int aligned = (ldb % 16 == 0 && aligned16(dev_lvl)) ? 1 : 0;
-    emo_workspace_bytes_for(g, B, 1, flags, aligned, &need);
-    emo_workspace_bytes_for(g, B, 2, flags, aligned, &total);
-    // per-policy result arrays live behind the slack workspace
     size_t per_policy = round_up((size_t)B * 8, 256);
-    if (!ws || ws_bytes < total) return EMO_E_OOM;
-    cudaStream_t st = (cudaStream_t)stream;
     char *tail = (char *)ws + need;
     int64_t *d_T = (int64_t *)tail;
     double *d_E = (double *)(tail + per_policy);
@@ -2146,13 +2136,8 @@ int emo_slack_batch_host_packed(const emo_graph *g, int64_t B, int bits, const u
     int64_t *d_sel = (int64_t *)(tail + 4 * per_policy);      // {index, T, E bits, T0, E0 bits}
     int32_t *d_status = (int32_t *)(d_sel + 8);
     EMO_CUDA(cudaMemsetAsync(d_sel, 0, 128, st));
-    if (bits == 8) {
-        if (ld_host != ldb) return EMO_E_INVALID_ARG;
-        EMO_CUDA(cudaMemcpyAsync(dev_lvl, lvl_host, (size_t)g->h.rows * (size_t)ldb, cudaMemcpyHostToDevice, st));
-    } else {
-        // the levels cross the bus packed and are spread to bytes on the device
-        EMO_CUDA(cudaMemcpyAsync(dev_packed, lvl_host, (size_t)g->h.rows * (size_t)ld_host, cudaMemcpyHostToDevice, st));
-        int rcu = emo_unpack_levels(bits, g->h.rows, B, dev_packed, ld_host, dev_lvl, ldb, stream);
+    if (bits < 8) {
+        int rcu = emo_unpack_levels(bits, g->h.rows, B, dev_packed, ld_packed, dev_lvl, ldb, (void *)st);
         if (rcu) return rcu;
     }
     int rc = emo_slack_batch(g, B, dev_lvl, ldb, nullptr, nullptr, slack_dev, ldo, d_T, d_E,
@@ -2175,6 +2160,66 @@ int emo_slack_batch_host_packed(const emo_graph *g, int64_t B, int bits, const u
     int32_t stc;
     std::memcpy(&stc, &tmp[8], sizeof stc);
     return stc < 0 ? stc : EMO_OK;
+}
+
+int emo_slack_batch_host_packed(const emo_graph *g, int64_t B, int bits, const uint8_t *lvl_host, int64_t ld_host,
+                                uint8_t *dev_packed, uint8_t *dev_lvl, int64_t ldb, int64_t *slack_dev, int64_t ldo,
+                                int64_t delta_ppm, int64_t *makespan_host, double *energy_host, int64_t *slack_sum_host,
+                                int32_t *n_critical_host, int64_t *sel_host, void *ws, size_t ws_bytes, uint32_t flags,
+                                void *stream)
+{
+    if (!g || B <= 0 || !lvl_host || !dev_lvl || !makespan_host || !energy_host || !sel_host || ldb < B)
+        return EMO_E_INVALID_ARG;
+    if (bits < 1 || bits > 8 || (bits < 8 && !dev_packed)) return EMO_E_INVALID_ARG;
+    if (g->host_only) return EMO_E_CUDA;
+    size_t need = 0, total = 0;
+    const int aligned = (ldb % 16 == 0 && aligned16(dev_lvl)) ? 1 : 0;
+    emo_workspace_bytes_for(g, B, 1, flags, aligned, &need);
+    emo_workspace_bytes_for(g, B, 2, flags, aligned, &total);
+    // per-policy result arrays live behind the slack workspace
+    if (!ws || ws_bytes < total) return EMO_E_OOM;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (bits == 8) {
+        if (ld_host != ldb) return EMO_E_INVALID_ARG;
+        EMO_CUDA(cudaMemcpyAsync(dev_lvl, lvl_host, (size_t)g->h.rows * (size_t)ldb, cudaMemcpyHostToDevice, st));
+    } else {
+        // the levels cross the bus packed and are spread to bytes on the device
+        EMO_CUDA(cudaMemcpyAsync(dev_packed, lvl_host, (size_t)g->h.rows * (size_t)ld_host, cudaMemcpyHostToDevice, st));
+    }
+    return host_batch_tail(g, B, bits, dev_packed, ld_host, dev_lvl, ldb, slack_dev, ldo, delta_ppm, makespan_host, energy_host,
+                           slack_sum_host, n_critical_host, sel_host, ws, need, flags, st);
+}
+
+int emo_levels_prefetch(const emo_graph *g, const uint8_t *lvl_host, int64_t ld_host, uint8_t *dev_packed, void *copy_stream,
+                        void *ready)
+{
+    if (!g || !lvl_host || !dev_packed || !ready || ld_host <= 0) return EMO_E_INVALID_ARG;
+    if (g->host_only) return EMO_E_CUDA;
+    cudaStream_t cs = (cudaStream_t)copy_stream;
+    EMO_CUDA(cudaMemcpyAsync(dev_packed, lvl_host, (size_t)g->h.rows * (size_t)ld_host, cudaMemcpyHostToDevice, cs));
+    EMO_CUDA(cudaEventRecord((cudaEvent_t)ready, cs));
+    return EMO_OK;
+}
+
+int emo_slack_batch_prefetched(const emo_graph *g, int64_t B, int bits, const uint8_t *dev_packed, int64_t ld_packed, void *ready,
+                               uint8_t *dev_lvl, int64_t ldb, int64_t *slack_dev, int64_t ldo, int64_t delta_ppm,
+                               int64_t *makespan_host, double *energy_host, int64_t *slack_sum_host,
+                               int32_t *n_critical_host, int64_t *sel_host, void *ws, size_t ws_bytes, uint32_t flags,
+                               void *stream)
+{
+    if (!g || B <= 0 || !dev_packed || !dev_lvl || !makespan_host || !energy_host || !sel_host || ldb < B)
+        return EMO_E_INVALID_ARG;
+    if (bits < 1 || bits > 7) return EMO_E_INVALID_ARG;
+    if (g->host_only) return EMO_E_CUDA;
+    size_t need = 0, total = 0;
+    const int aligned = (ldb % 16 == 0 && aligned16(dev_lvl)) ? 1 : 0;
+    emo_workspace_bytes_for(g, B, 1, flags, aligned, &need);
+    emo_workspace_bytes_for(g, B, 2, flags, aligned, &total);
+    if (!ws || ws_bytes < total) return EMO_E_OOM;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (ready) EMO_CUDA(cudaStreamWaitEvent(st, (cudaEvent_t)ready, 0));
+    return host_batch_tail(g, B, bits, dev_packed, ld_packed, dev_lvl, ldb, slack_dev, ldo, delta_ppm, makespan_host, energy_host,
+                           slack_sum_host, n_critical_host, sel_host, ws, need, flags, st);
 }
 
 int emo_slack_batch_host(const emo_graph *g, int64_t B, const uint8_t *lvl_host, int64_t ldb,

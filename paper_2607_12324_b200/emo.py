@@ -33,7 +33,7 @@ EXPORTS = [
     "emo_strerror", "emo_graph_load", "emo_graph_free", "emo_graph_info", "emo_workspace_bytes",
     "emo_eval_policies", "emo_slack_batch", "emo_slack", "emo_baseline", "emo_target_from_delta",
     "emo_select", "emo_transpose_policies", "emo_slack_batch_host", "emo_graph_program",
-    "emo_set_pass_events", "emo_select_static", "emo_graph_flow", "emo_graph_spine", "emo_graph_spine_view", "emo_set_wait_limit", "emo_call_path", "emo_set_flow_counters", "emo_workspace_bytes_for", "emo_measure_int_issue", "emo_measure_warp_costs", "emo_eval_intervals", "emo_workspace_bytes_intervals", "emo_search_dp", "emo_workspace_bytes_search", "emo_pack_greedy", "emo_pack_tables", "emo_pack_model", "emo_pack_classes", "emo_pack_levels", "emo_unpack_levels", "emo_slack_batch_host_packed",
+    "emo_set_pass_events", "emo_select_static", "emo_graph_flow", "emo_graph_spine", "emo_graph_spine_view", "emo_set_wait_limit", "emo_call_path", "emo_set_flow_counters", "emo_workspace_bytes_for", "emo_measure_int_issue", "emo_measure_warp_costs", "emo_eval_intervals", "emo_workspace_bytes_intervals", "emo_search_dp", "emo_workspace_bytes_search", "emo_pack_greedy", "emo_pack_tables", "emo_pack_model", "emo_pack_classes", "emo_pack_levels", "emo_unpack_levels", "emo_slack_batch_host_packed", "emo_levels_prefetch", "emo_slack_batch_prefetched",
 ]
 
 
@@ -131,6 +131,8 @@ def lib():
         L.emo_pack_levels.argtypes = [ctypes.c_int, i64, i64, p, i64, p, i64, p]
         L.emo_unpack_levels.argtypes = [ctypes.c_int, i64, i64, p, i64, p, i64, p]
         L.emo_slack_batch_host_packed.argtypes = [p, i64, ctypes.c_int, p, i64, p, p, i64, p, i64, i64, p, p, p, p, p, p, sz, u32, p]
+        L.emo_levels_prefetch.argtypes = [p, p, i64, p, p, p]
+        L.emo_slack_batch_prefetched.argtypes = [p, i64, ctypes.c_int, p, i64, p, p, i64, p, i64, i64, p, p, p, p, p, p, sz, u32, p]
         L.emo_call_path.argtypes = [p, i64, p, i64, i64, ctypes.c_int, u32]
         L.emo_select_static.argtypes = [i64, p, p, i64, p, i64, p, p, p, p]
         for name in EXPORTS:
@@ -524,6 +526,29 @@ def emo_pack_levels(bits, rows, B, lvl, ldb, packed, ldp, stream=None):
 def emo_unpack_levels(bits, rows, B, packed, ldp, lvl, ldb, stream=None):
     _check(lib().emo_unpack_levels(int(bits), int(rows), int(B), _addr(packed), int(ldp), _addr(lvl), int(ldb), _stream(stream)),
            "emo_unpack_levels")
+
+
+def _event(ev) -> Optional[int]:
+    if ev is None:
+        return None
+    if not ev.cuda_event:          # torch creates the handle lazily, on the first record
+        ev.record()
+    return int(ev.cuda_event)
+
+
+def emo_levels_prefetch(g: Graph, lvl_host, ld_host, dev_packed, copy_stream, ready):
+    """Enqueues the copy of packed levels on copy_stream and records the torch event `ready` behind it."""
+    _check(lib().emo_levels_prefetch(g.handle, _addr(lvl_host), int(ld_host), _addr(dev_packed), _stream(copy_stream),
+                                     _event(ready)), "emo_levels_prefetch")
+
+
+def emo_slack_batch_prefetched(g: Graph, B, bits, dev_packed, ld_packed, ready, dev_lvl, ldb, slack_dev, ldo, delta_ppm,
+                               makespan_host, energy_host, slack_sum_host, n_critical_host, sel_host, ws, flags=0, stream=None):
+    _check(lib().emo_slack_batch_prefetched(g.handle, int(B), int(bits), _addr(dev_packed), int(ld_packed), _event(ready),
+                                            _addr(dev_lvl), int(ldb), _addr(slack_dev), int(ldo), int(delta_ppm),
+                                            _addr(makespan_host), _addr(energy_host), _addr(slack_sum_host),
+                                            _addr(n_critical_host), _addr(sel_host), _addr(ws), _nbytes(ws), int(flags),
+                                            _stream(stream)), "emo_slack_batch_prefetched")
 
 
 def emo_slack_batch_host_packed(g: Graph, B, bits, lvl_host, ld_host, dev_packed, dev_lvl, ldb, slack_dev, ldo, delta_ppm,

@@ -469,6 +469,31 @@ def test_host_buffer_call(torch_cuda, emo, oracle_mod):
         emo.emo_slack_batch_host_packed(h, B, bits, packed_host, ldp, packed, dev_lvl, ldb, slack, B, ppm, T, E, ss, nc, sel, ws2, flags=fl)
         assert np.array_equal(T.numpy(), r_or["makespan"]) and int(sel[0]) == want
         assert np.array_equal(slack.cpu().numpy(), r_or["slack"])
+    # the two-buffer form: the copy of the next batch is enqueued on a stream of its own before the current batch
+    # is evaluated; three batches (the same levels, then a second set, then the first again) through two buffers
+    lv2 = lv.clone()
+    lv2[:, :B] = (g.L - 1) - lv[:, :B]          # a second set of policies: every level mirrored
+    sets = [(lv, r_or), (lv2, oracle_mod.batch(g, lv2.numpy(), B=B, want_arrays=True))]
+    hosts = []
+    for lvx, _ in sets:
+        pkx = torch.zeros((g.n, ldp), dtype=torch.uint8, device="cuda")
+        emo.emo_pack_levels(bits, g.n, B, lvx.cuda(), ldb, pkx, ldp)
+        hosts.append(pkx.cpu().pin_memory())
+    bufs = (torch.zeros((g.n, ldp), dtype=torch.uint8, device="cuda"), torch.zeros((g.n, ldp), dtype=torch.uint8, device="cuda"))
+    copy_stream = torch.cuda.Stream()
+    ready = (torch.cuda.Event(), torch.cuda.Event())
+    order = [0, len(sets) - 1, 0]
+    emo.emo_levels_prefetch(h, hosts[order[0]], ldp, bufs[0], copy_stream, ready[0])
+    for s_, which in enumerate(order):
+        if s_ + 1 < len(order):
+            emo.emo_levels_prefetch(h, hosts[order[s_ + 1]], ldp, bufs[(s_ + 1) & 1], copy_stream, ready[(s_ + 1) & 1])
+        T.zero_()
+        slack.zero_()
+        emo.emo_slack_batch_prefetched(h, B, bits, bufs[s_ & 1], ldp, ready[s_ & 1], dev_lvl, ldb, slack, B, ppm, T, E, ss, nc, sel, ws)
+        rx = sets[which][1]
+        assert np.array_equal(T.numpy(), rx["makespan"]) and np.array_equal(ss.numpy(), rx["slack_sum"])
+        np.testing.assert_allclose(E.numpy(), rx["energy"], rtol=E_RTOL)
+        assert np.array_equal(slack.cpu().numpy(), rx["slack"])
     h.free()
 
 
