@@ -86,6 +86,18 @@ __device__ __forceinline__ unsigned emo_spine_bar(const FlowParams &p, unsigned 
     return smem0 + p.off_sbar + (unsigned)(((g * kFlowMaxBuf + a) * 3 + which) * 8);
 }
 
+// Position of a stage in a ring of n buffers and the parity of its use of the buffer, kept by steps (no division).
+struct SpineRing {
+    int idx = 0, par = 0, n = 1;
+    __device__ __forceinline__ void next()
+    {
+        if (++idx == n) {
+            idx = 0;
+            par ^= 1;
+        }
+    }
+};
+
 struct SpineRole {
     bool producer, spine;
     int group, widx;      // producer: widx = its index among the producers
@@ -149,12 +161,14 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_fwd(FlowParams p)
         uint32_t *const rst_lane = p.restore ? p.restore + (size_t)blockIdx.x * p.restore_rows * ptile + col : nullptr;
         long long t_full = 0, t_pre = 0, t_loop = 0;
         const unsigned ptile4 = (unsigned)ptile * 4u;
+        SpineRing ra;
+        ra.n = nacc;
         const long long t_begin = EMO_SCLK();
         for (int cst = 0; cst < p.stages; ++cst) {
-            const int a = cst % nacc;
+            const int a = ra.idx;
             const long long tw0 = EMO_SCLK();
             const long long tw1 = tw0;
-            if (!emo_spine_wait(emo_spine_bar(p, smem0, group, a, 0), (cst / nacc) & 1, abort_word, limit)) {
+            if (!emo_spine_wait(emo_spine_bar(p, smem0, group, a, 0), ra.par, abort_word, limit)) {
                 failed = true;
                 break;
             }
@@ -193,6 +207,7 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_fwd(FlowParams p)
             t_loop += EMO_SCLK() - tl0;
             __syncwarp();
             if (lane == 0) emo_mbar_arrive(emo_spine_bar(p, smem0, group, a, 1));
+            ra.next();
         }
         if (!failed && rst_lane)
             for (int ln = 0; ln < lanes; ++ln) rst_lane[((size_t)p.pushes + ln) * ptile] = emo_lds_u32(slot_lane4 + (unsigned)ln * 128u);
@@ -208,13 +223,16 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_fwd(FlowParams p)
         const bool is_base = base_col == col;
         const unsigned top = (unsigned)(p.L - 1);
         long long t_full = 0, t_acc = 0;
+        SpineRing rs, ra;
+        rs.n = nbuf;
+        ra.n = nacc;
         const long long t_begin = EMO_SCLK();
         for (int cst = 0; cst < p.stages; ++cst) {
-            const int s = cst % nbuf, a = cst % nacc;
+            const int s = rs.idx, a = ra.idx;
             const long long tw0 = EMO_SCLK();
-            const bool ok1 = emo_worker_wait(bar0 + 8 * s, (cst / nbuf) & 1, abort_word, limit);
+            const bool ok1 = emo_worker_wait(bar0 + 8 * s, rs.par, abort_word, limit);
             const long long tw1 = EMO_SCLK();
-            if (!ok1 || (cst >= nacc && !emo_worker_wait(emo_spine_bar(p, smem0, group, a, 1), ((cst / nacc) - 1) & 1, abort_word, limit))) {
+            if (!ok1 || (cst >= nacc && !emo_worker_wait(emo_spine_bar(p, smem0, group, a, 1), ra.par ^ 1, abort_word, limit))) {
                 failed = true;
                 break;
             }
@@ -268,6 +286,8 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_fwd(FlowParams p)
                 emo_mbar_arrive(emo_spine_bar(p, smem0, group, a, 0));
                 emo_mbar_arrive(bar0 + 8 * (kFlowMaxBuf + s));
             }
+            rs.next();
+            ra.next();
         }
         if (p.prof && lane == 0 && blockIdx.x < 512) {
             long long *pr = p.prof + ((size_t)blockIdx.x * 32 + warp) * 8;
@@ -339,15 +359,21 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_bwd(FlowParams p)
                         p.restore[((size_t)blockIdx.x * p.restore_rows + p.pushes + ln) * ptile + col]);
         const unsigned col4 = (unsigned)col * 4u, ptile4 = (unsigned)ptile * 4u;
         long long t_full = 0, t_pre = 0, t_post = 0, t_loop = 0;
+        SpineRing rs, ra, ra2;
+        rs.n = nbuf;
+        ra.n = ra2.n = nacc;
         const long long t_begin = EMO_SCLK();
         for (int cst = 0; cst < p.stages; ++cst) {
-            const int s = cst % nbuf, a = cst % nacc;
+            const int s = rs.idx, a = ra.idx;
             const long long tw0 = EMO_SCLK();
-            bool ok = emo_spine_wait(bar0 + 8 * s, (cst / nbuf) & 1, abort_word, limit);
+            bool ok = emo_spine_wait(bar0 + 8 * s, rs.par, abort_word, limit);
             const long long tw1 = EMO_SCLK();
-            ok = ok && emo_spine_wait(emo_spine_bar(p, smem0, group, a, 0), (cst / nacc) & 1, abort_word, limit);
+            ok = ok && emo_spine_wait(emo_spine_bar(p, smem0, group, a, 0), ra.par, abort_word, limit);
             const long long tw2 = EMO_SCLK();
-            if (ok && cst >= 2) ok = emo_spine_wait(emo_spine_bar(p, smem0, group, (cst - 2) % nacc, 2), ((cst - 2) / nacc) & 1, abort_word, limit);
+            if (ok && cst >= 2) {
+                ok = emo_spine_wait(emo_spine_bar(p, smem0, group, ra2.idx, 2), ra2.par, abort_word, limit);      // stage cst - 2
+                ra2.next();
+            }
             if (!ok) {
                 failed = true;
                 break;
@@ -391,6 +417,8 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_bwd(FlowParams p)
                 emo_mbar_arrive(emo_spine_bar(p, smem0, group, a, 1));
                 emo_mbar_arrive(bar0 + 8 * (kFlowMaxBuf + s));
             }
+            rs.next();
+            ra.next();
         }
         if (p.prof && lane == 0 && blockIdx.x < 512) {
             long long *pr = p.prof + ((size_t)blockIdx.x * 32 + warp) * 8;
@@ -403,6 +431,9 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_bwd(FlowParams p)
     } else {
         const unsigned lmask = (unsigned)p.Lp - 1u, tab_row = p.tab_row;
         long long t_w1 = 0, t_w2 = 0, t_prew = 0, t_postw = 0;
+        SpineRing rs, ra, rs1, ra1;
+        rs.n = rs1.n = nbuf;
+        ra.n = ra1.n = nacc;
         const long long t_begin = EMO_SCLK();
         const long long T = act ? p.makespan[b] : 0;
         const unsigned ldo8 = (unsigned)p.ldo * 8u;
@@ -414,10 +445,10 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_bwd(FlowParams p)
         for (int cst = 0; cst <= p.stages && !failed; ++cst) {
             if (cst < p.stages) {
                 // the sums of stage cst
-                const int s = cst % nbuf, a = cst % nacc;
+                const int s = rs.idx, a = ra.idx;
                 const long long tq0 = EMO_SCLK();
-                if (!emo_worker_wait(bar0 + 8 * s, (cst / nbuf) & 1, abort_word, limit) ||
-                    (cst >= nacc && !emo_worker_wait(emo_spine_bar(p, smem0, group, a, 2), ((cst / nacc) - 1) & 1, abort_word, limit))) {
+                if (!emo_worker_wait(bar0 + 8 * s, rs.par, abort_word, limit) ||
+                    (cst >= nacc && !emo_worker_wait(emo_spine_bar(p, smem0, group, a, 2), ra.par ^ 1, abort_word, limit))) {
                     failed = true;
                     break;
                 }
@@ -453,12 +484,14 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_bwd(FlowParams p)
                 __syncwarp();
                 if (lane == 0) emo_mbar_arrive(emo_spine_bar(p, smem0, group, a, 0));
                 t_prew += EMO_SCLK() - tq1;
+                rs.next();
+                ra.next();
             }
             if (cst >= 1) {
                 // the stores of stage cst - 1
-                const int c1 = cst - 1, s = c1 % nbuf, a = c1 % nacc;
+                const int s = rs1.idx, a = ra1.idx;      // stage cst - 1
                 const long long tq0 = EMO_SCLK();
-                if (!emo_worker_wait(emo_spine_bar(p, smem0, group, a, 1), (c1 / nacc) & 1, abort_word, limit)) {
+                if (!emo_worker_wait(emo_spine_bar(p, smem0, group, a, 1), ra1.par, abort_word, limit)) {
                     failed = true;
                     break;
                 }
@@ -520,6 +553,8 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_bwd(FlowParams p)
                     emo_mbar_arrive(bar0 + 8 * (kFlowMaxBuf + s));
                 }
                 t_postw += EMO_SCLK() - tq1;
+                rs1.next();
+                ra1.next();
             }
         }
         if (p.prof && lane == 0 && blockIdx.x < 512) {
