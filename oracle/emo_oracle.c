@@ -38,7 +38,8 @@
  *
  * Parity pins: every routine here is pinned by tests/test_oracle_pins.py (brute-force path
  * enumeration, closed forms, reversal duality, invariants, a hand-worked example).  Of this file only
- * the policy search (Alg. 2) is "parity unpinned" beyond the pins its comment lists.
+ * the policy search (Alg. 2) has a part that is "parity unpinned": which of two candidates of one time bin
+ * survives (its comment lists the pins, among them the exhaustive optimum where no bin is shared).
  */
 #include <stdint.h>
 #include <stdlib.h>
@@ -384,11 +385,13 @@ done:
  * P_0 misses T_max, dp[0] is still seeded with it (Alg. 2 line 3 has no test) and the search may end
  * with an empty dp[I]: then *found = 0.
  *
- * Pinned only in part (tests/test_oracle_search.py): exhaustive optimum for one interval, bounds
- * (never worse than P_0, never better than the exhaustive optimum, always feasible), consistency of the
- * reported (T, E) with Alg. 1 on the reported policy, L = 1, T_max = t_0.  For several intervals the DP
- * is a heuristic (one policy per time bin survives) and has no independent definition to compare with:
- * beyond those pins it is "parity unpinned".
+ * Pins (tests/test_oracle_search.py): the exhaustive optimum for one interval; for several intervals the
+ * exhaustive optimum (policy, time, energy, number of predictions) whenever no two policies end in one
+ * time bin, with a constraint that admits all of them and with one that cuts into the set (lower levels
+ * never faster there); bounds otherwise (never worse than P_0, never better than the exhaustive optimum,
+ * always feasible); consistency of the reported (T, E) with Alg. 1 on the reported policy; L = 1;
+ * T_max = t_0.  Where two candidates do end in one bin the DP is a heuristic (one of them survives) and
+ * has no independent definition to compare with: for that choice alone it is "parity unpinned".
  *
  * Outputs: F_best[I] levels of the chosen policy, T_best, E_best, n_pred = calls of Alg. 1, found.
  * ------------------------------------------------------------------------------------------------ */

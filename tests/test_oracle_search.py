@@ -1,6 +1,7 @@
-"""Pins of the oracle's policy search (Alg. 2).  The DP is a heuristic for several intervals, so it is pinned
-where something independent exists: the exhaustive optimum for one interval, bounds against exhaustive
-enumeration for several, feasibility, consistency with Alg. 1 on the reported policy, degenerate inputs."""
+"""Pins of the oracle's policy search (Alg. 2).  The DP is a heuristic only where two candidates end in one time
+bin (one survives), so it is pinned where something independent exists: the exhaustive optimum for one interval
+and, for several intervals, whenever no two policies share a time bin; bounds against exhaustive enumeration
+otherwise; feasibility, consistency with Alg. 1 on the reported policy, degenerate inputs."""
 from __future__ import annotations
 
 import itertools
@@ -60,6 +61,52 @@ def test_bounds_against_enumeration(oracle_mod, seed):
             col = int(np.flatnonzero((pols == s["F"][:, None]).all(axis=0))[0])
             assert s["T"] == int(r["makespan"][col]) and np.isclose(s["E"], r["energy"][col], rtol=1e-15)
             assert s["n_pred"] >= 1 + g.L and (s["n_pred"] - 1) % g.L == 0
+
+
+def _chain_case(seed, n=12, L=3, I=3):
+    """One stream of n kernels in series on one device: every node is on the critical path, so every interval's level
+    changes the end-to-end time; durations 1 000 - 2 000 with random increments (sums of different choices differ),
+    longer at lower levels; change points 5 000 apart, so every interval holds several starts under every policy."""
+    from paper_2607_12324_b200 import workloads as W
+    rs = np.random.RandomState(seed)
+    row_ptr = np.concatenate([[0], np.arange(0, n)]).astype(np.int64)      # node v > 0 has the one predecessor v - 1
+    col = np.arange(0, n - 1, dtype=np.int32)
+    level_ptr = np.arange(0, n + 1, dtype=np.int32)
+    top = rs.randint(1000, 1400, size=n)
+    lat = np.stack([top + np.cumsum(rs.randint(50, 300, size=(L, n)), axis=0)[L - 1 - l] * (l < L - 1) for l in range(L)], axis=1).astype(np.int64)
+    energy = rs.uniform(1.0, 9.0, size=(n, L))
+    g = W.Graph(n, row_ptr, col, level_ptr, L, lat, energy, np.zeros(n, np.uint8), "chain")
+    breaks = (np.arange(I) * 5000).astype(np.int64)
+    return g, np.zeros(n, np.int32), breaks, rs.uniform(10.0, 90.0, size=L)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_without_collisions_the_search_is_exhaustive(oracle_mod, seed):
+    """Several intervals: when no two policies end in the same time bin (exact keys, all L^I end-to-end times distinct)
+    and the constraint admits every policy, nothing is ever merged or dropped, so dp[I] holds every policy: the answer
+    must be the exhaustive optimum (earliest time among equal energies) and Alg. 1 runs 1 + L + L^2 + ... + L^I times.
+    With a constraint that cuts into the set the same holds among the feasible policies, because here a lower level is
+    never faster: a prefix that misses the constraint cannot be repaired by the intervals still at the top level."""
+    I, L = 3, 3
+    g, dev_of, breaks, p_idle = _chain_case(seed, L=L, I=I)
+    pols = _all_policies(I, L)
+    r = _pred_all(oracle_mod, g, dev_of, breaks, p_idle, pols)
+    assert len(np.unique(r["makespan"])) == pols.shape[1], "the construction should give every policy its own time"
+    s = oracle_mod.search_dp(g, dev_of, breaks, p_idle, int(r["makespan"].max()), 1)
+    E_opt = float(r["energy"].min())
+    cands = np.flatnonzero(r["energy"] == E_opt)
+    best = int(cands[np.argmin(r["makespan"][cands])])
+    assert s["found"] and s["E"] == E_opt and s["T"] == int(r["makespan"][best])
+    assert np.array_equal(s["F"], pols[:, best])
+    assert s["n_pred"] == sum(L ** i for i in range(I + 1))
+    # a constraint at the median time
+    T_max = int(np.median(r["makespan"]))
+    feas = r["makespan"] <= T_max
+    s = oracle_mod.search_dp(g, dev_of, breaks, p_idle, T_max, 1)
+    E_f = float(r["energy"][feas].min())
+    cands = np.flatnonzero(feas & (r["energy"] == E_f))
+    best = int(cands[np.argmin(r["makespan"][cands])])
+    assert s["found"] and s["E"] == E_f and s["T"] == int(r["makespan"][best]) and np.array_equal(s["F"], pols[:, best])
 
 
 def test_degenerate_inputs(oracle_mod):
