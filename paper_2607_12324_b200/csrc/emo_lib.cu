@@ -980,26 +980,29 @@ int launch_spine_bwd(const emo_graph *g, const FlowPlan &pl, int64_t B, const ui
     return EMO_OK;
 }
 
-// Whether a call takes the spine kernels: the program exists and either the caller asks for them (EMO_F_SPINE_KERNEL) or the graph is narrow
-// and the batch below the large-batch rule of the lane-stream kernels.
+// Whether a call takes the spine kernels: the program exists and either the caller asks for them (EMO_F_SPINE_KERNEL) or
+// the graph is narrow and the batch leaves at most three policy groups to an SM (or the graph is short).
 bool spine_allowed(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t ldb, int64_t ldo, bool extra, uint32_t flags)
 {
     const int64_t big = (int64_t)1 << 28;
     if (!g->sflow.ok32 || !g->sflow.spine.ok || !g->dspine.ready || extra) return false;
     if (flags & (EMO_F_NO_STAGING | EMO_F_PAIR_KERNEL | EMO_F_LANE_KERNEL | EMO_F_FLOW_KERNEL)) return false;
-    // Measured on the five workloads: on graphs of up to eight lanes with batches below the large-batch rule the spine
-    // kernels are the fastest pair (10 000 nodes x 4 096 policies: 1.1 ms against 2.3 ms for the 64-bit staged kernels
-    // and 3.1 ms for the lane-stream kernels; 1 013 nodes x 65 536 policies: 0.63 against 0.90 ms); one warp carries the
-    // recurrence of all lanes, so wide graphs (17 lanes: 21.9 against 9.0 ms) and, with four groups per block, the
-    // 250 000-node graph with 16 384 policies (the workers take the issue slots that the spine warp needs) stay with
+    // Measured: on graphs of up to eight lanes the spine kernels are the fastest pair while a block holds at most three
+    // policy groups (75 000 nodes, both passes, spine / lane-stream: 3.6 / 5.5 ms with one group per SM, 4.4 / 6.0 with
+    // two, 5.7 / 6.3 with three, 8.9 / 6.8 with four: the workers then take the issue slots and the shared-memory pipe
+    // that the spine warp needs) and on short graphs whatever the batch (1 013 nodes x 65 536 policies: 0.61 against
+    // 0.90 ms); one warp carries the recurrence of all lanes, so wide graphs (17 lanes: 21.9 against 9.0 ms) stay with
     // the other kernels unless the caller asks.
-    if (!(flags & EMO_F_SPINE_KERNEL) && ((int64_t)g->h.n * B >= ((int64_t)1 << 31) || g->sflow.lanes > 8)) return false;
+    if (!(flags & EMO_F_SPINE_KERNEL)) {
+        const int64_t per_sm = ((B + 1 + 31) / 32 + g->sm_count - 1) / std::max(g->sm_count, 1);
+        if (g->sflow.lanes > 8 || (per_sm > 3 && g->h.n > 8192)) return false;
+    }
     return ldb % 16 == 0 && aligned16(lvl) && ldb < big && ldo < big;
 }
 
 // Whether a call takes the 32-bit lane-stream kernels: the program exists, the level matrix can be
 // fetched in 16-byte pieces, and either the caller asks for them (EMO_F_FLOW_KERNEL) or the batch is
-// large.  Measured on the five workloads: on the 250 000-node graph with 16 384 policies they are
+// large (for the graph or for the SMs).  Measured on the five workloads: on the 250 000-node graph with 16 384 policies they are
 // the faster pair (25.8 ms against 30.1 ms for both passes) and need 1.6 GB of workspace instead of
 // 37.7 GB; on the smaller workloads, where a block holds one or two policy groups and every step is
 // latency, the 64-bit staged kernels with their one-step-ahead fetch are faster (2.3 ms against 3.7 ms on
@@ -1009,7 +1012,12 @@ bool flow_allowed(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t ldb
     const int64_t big = (int64_t)1 << 28;
     if (!g->flow.ok32 || !g->dflow.ready) return false;
     if (flags & (EMO_F_NO_STAGING | EMO_F_PAIR_KERNEL | EMO_F_LANE_KERNEL)) return false;
-    if (!(flags & EMO_F_FLOW_KERNEL) && (int64_t)g->h.n * B < ((int64_t)1 << 31)) return false;
+    if (!(flags & EMO_F_FLOW_KERNEL)) {
+        // large batches, and on narrow graphs every batch with more than three policy groups per SM (where the spine
+        // kernels stop; 75 000 nodes x 16 384 policies: 6.8 ms against 9.0 ms for the 64-bit staged kernels)
+        const int64_t per_sm = ((B + 1 + 31) / 32 + g->sm_count - 1) / std::max(g->sm_count, 1);
+        if ((int64_t)g->h.n * B < ((int64_t)1 << 31) && !(g->flow.lanes <= 8 && per_sm > 3)) return false;
+    }
     return ldb % 16 == 0 && aligned16(lvl) && ldb < big && ldo < big;
 }
 
@@ -1334,6 +1342,27 @@ int emo_graph_load(int32_t n, const int64_t *row_ptr, const int32_t *col, const 
             if (rc == EMO_OK) rc = upload_program_lane(g->bwd, g->lbwd);
         }
         if (rc == EMO_OK) rc = upload_flow(g->flow, g->dflow, (flags & EMO_F_INTERVALS) != 0);
+        // One barrier per stage needs more exchange slots than one every 16 steps (on the 250 000-node graph 20.9 KB
+        // against 13.8 KB per policy group, at 0.3 scale 29.8 KB against 17.9 KB).  Where four groups then no longer fit a
+        // block, the grid doubles and the gain turns into a loss (11.7 ms against 6.8 ms at 0.3 scale): take the shorter
+        // distance unless the caller chose one.
+        if (rc == EMO_OK && g->flow.ok32 && g->dflow.ready && !(flags & 0xF0u) && g->flow.sync > 16) {
+            FlowPlan probe;
+            const int gmax = std::min((32 - 2) / std::max(g->flow.lanes, 1), 15);
+            const bool fits = flow_plan(g, (int64_t)4 * 32 * g->sm_count - 1, true, true, probe) && probe.groups >= std::min(4, gmax);
+            if (!fits) {
+                const int fk = g->flow.K, look = (int)((flags >> 16) & 0xFF);
+                int lanes = (int)((flags >> 8) & 0xFF);
+                std::string err;
+                free_flow(g->dflow);
+                rc = compile_flow(g->h, lat, energy, lanes, look, fk, 16, g->flow, err);
+                if (rc == EMO_E_UNSUPPORTED) {
+                    g->flow = Flow();
+                    rc = EMO_OK;
+                }
+                if (rc == EMO_OK) rc = upload_flow(g->flow, g->dflow, (flags & EMO_F_INTERVALS) != 0);
+            }
+        }
         if (rc == EMO_OK) rc = upload_spine(g->sflow, g->dspine);
         }
         } catch (const std::bad_alloc &) {
