@@ -49,7 +49,8 @@ extern "C" {
 #define EMO_F_HOST_ONLY 0x1u       /* build the handle without touching a device (inspection) */
 #define EMO_F_LANES(c) (((uint32_t)(c) & 0xFFu) << 8)      /* force c cooperating warps per policy group */
 #define EMO_F_LOOKAHEAD(d) (((uint32_t)(d) & 0xFFu) << 16) /* scheduling look-ahead in steps */
-#define EMO_F_FLOW_SYNC(s) ((((uint32_t)(s) / 8u) & 0xFu) << 4)  /* lane-stream program: steps between group barriers (8, 16, 32) */
+#define EMO_F_FLOW_SYNC(s) ((((uint32_t)(s) / 8u) & 0xFu) << 4)  /* lane-stream program: steps between group barriers (8, 16, 32;
+                                                                  * default: one per stage where four policy groups then still fit a block, else 16) */
 #define EMO_F_FLOW_STAGE(k) (((uint32_t)(k) & 0x3Fu) << 24)      /* lane-stream program: steps per stage (8, 16, 32) */
 #define EMO_F_SPINE_STAGE(k) ((uint32_t)((k) == 8 ? 1u : ((k) == 32 ? 3u : 2u)) << 30)   /* spine program: steps per stage (8, 16, 32) */
 #define EMO_F_INTERVALS 0x2u       /* also prepare the lane-stream form of emo_eval_intervals (a second copy of the forward program on
@@ -61,8 +62,10 @@ extern "C" {
 #define EMO_F_NO_STAGING 0x2u      /* use the plain-load kernels instead of the staged ones */
 #define EMO_F_PAIR_KERNEL 0x4u     /* staged pass kernel with two policies per thread (default only for very large batches) */
 #define EMO_F_LANE_KERNEL 0x8u     /* staged pass kernel with one policy per thread (the default otherwise) */
-#define EMO_F_FLOW_KERNEL 0x10u    /* the 32-bit lane-stream kernels (the default only for large batches: n * B >= 2^31) */
-#define EMO_F_SPINE_KERNEL 0x20u   /* the spine kernels (the default on graphs of at most eight lanes while n * B < 2^31) */
+#define EMO_F_FLOW_KERNEL 0x10u    /* the 32-bit lane-stream kernels (the default for large batches: n * B >= 2^31, or more than three
+                                    * policy groups of 32 per SM on a graph of at most eight lanes) */
+#define EMO_F_SPINE_KERNEL 0x20u   /* the spine kernels (the default on graphs of at most eight lanes while the batch leaves at most
+                                    * three policy groups of 32 to an SM, or the graph has at most 8 192 nodes) */
 #define EMO_F_TEST_STALL 0x100u    /* test hook of the 32-bit kernels: the producer warps stop half way, so that the
                                       consumers' bounded waits run out and EMO_E_TIMEOUT is reported */
 
