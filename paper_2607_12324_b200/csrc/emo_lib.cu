@@ -7,6 +7,7 @@
 #include <cstring>
 #include <new>
 #include <string>
+#include <thread>
 #include <vector>
 
 #include "../../include/emo.h"
@@ -1268,27 +1269,42 @@ int emo_graph_load(int32_t n, const int64_t *row_ptr, const int32_t *col, const 
             if (fk == 0) fk = flanes * 32 <= 32 * kFlowRowRegs ? 32 : (flanes * 16 <= 32 * kFlowRowRegs ? 16 : 8);
             if (fs == 0) fs = fk;
             if (fs > fk) fs = fk;
-            rc = compile_flow(h, lat, energy, lanes, look, fk, fs, g->flow, err);
+            // the spine program: short stages (its sums per stage live in shared memory), 16 steps unless the caller
+            // says otherwise; compiled on a thread of its own beside the lane-stream program (they share nothing but
+            // their inputs)
+            const bool want_spine = !(flags & EMO_F_INTERVALS);
+            int rc_s = EMO_OK;
+            std::string err_s;
+            std::thread spine_thread;
+            if (want_spine) {
+                const int code = (int)((flags >> 30) & 3u);
+                int sk = code == 1 ? 8 : (code == 3 ? 32 : 16);
+                while (sk > 8 && flanes * sk > 32 * kFlowRowRegs) sk /= 2;
+                spine_thread = std::thread([&, sk]() {
+                    try {
+                        rc_s = compile_flow(h, lat, energy, lanes, look, sk, sk, g->sflow, err_s, true);
+                    } catch (const std::bad_alloc &) {
+                        rc_s = EMO_E_OOM;
+                    }
+                });
+            }
+            try {
+                rc = compile_flow(h, lat, energy, lanes, look, fk, fs, g->flow, err);
+            } catch (const std::bad_alloc &) {
+                rc = EMO_E_OOM;
+            }
+            if (spine_thread.joinable()) spine_thread.join();
             if (rc == EMO_E_UNSUPPORTED) {      // the 64-bit programs exist: they serve
                 g->flow = Flow();
                 rc = EMO_OK;
             }
+            if (rc == EMO_OK && rc_s != EMO_OK && rc_s != EMO_E_UNSUPPORTED) rc = rc_s;
             if (rc != EMO_OK) { delete g; return rc; }
-            // the spine program: short stages (its sums per stage live in shared memory), 16 steps unless the caller
-            // says otherwise; only for graphs that the large-batch rule can send there
-            if (g->flow.ok32 && !(flags & EMO_F_INTERVALS)) {
-                const int code = (int)((flags >> 30) & 3u);
-                int sk = code == 1 ? 8 : (code == 3 ? 32 : 16);
-                while (sk > 8 && flanes * sk > 32 * kFlowRowRegs) sk /= 2;
-                rc = compile_flow(h, lat, energy, lanes, look, sk, sk, g->sflow, err, true);
-                if (rc == EMO_E_UNSUPPORTED) rc = EMO_OK;
-                if (rc != EMO_OK) { delete g; return rc; }
-                if (!g->sflow.spine.ok) g->sflow = Flow();
-                else {
-                    // only the spine's parts are kept
-                    g->sflow.f = FlowDir();
-                    g->sflow.b = FlowDir();
-                }
+            if (!want_spine || rc_s != EMO_OK || !g->flow.ok32 || !g->sflow.spine.ok) g->sflow = Flow();
+            else {
+                // only the spine's parts are kept
+                g->sflow.f = FlowDir();
+                g->sflow.b = FlowDir();
             }
         }
         std::vector<int32_t> hop((size_t)std::max(n, 1), 0);
