@@ -60,3 +60,18 @@ def test_spine_program_on_config_graphs(emo, oracle_mod, name, scale, k):
         # the launch nodes' kernels are folded, not published: chains of kernels stay segments (where the graph is long
         # enough for the schedule to keep launch nodes two stages ahead of their kernels)
         assert sizes["segments"] < 0.85 * g.n
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_spine_program_on_random_dags(emo, oracle_mod, seed):
+    """Random DAGs of varying density (dense ones have nodes with many operands: merge operations; sparse ones long
+    chains: segments of several members), random policies, two lane counts and stage lengths."""
+    rs = np.random.RandomState(1000 + seed)
+    n = int(rs.randint(30, 140))
+    L = int(rs.randint(2, 7))
+    g = W.random_dag(500 + seed, n, float(rs.choice([0.02, 0.05, 0.12, 0.3])), L=L, max_dur=int(rs.choice([5, 40, 100000])))
+    lv = rs.randint(0, L, size=(g.n, 20)).astype(np.uint8)
+    lv[:, 0] = L - 1
+    lv[:, 1] = 0
+    for lanes, k in ((0, 8), (3, 16)):
+        compare(emo, oracle_mod, g, lv, emo.EMO_F_LANES(lanes) | emo.EMO_F_SPINE_STAGE(k))
