@@ -119,3 +119,27 @@ def test_bounded_waits_report_timeout(torch_cuda, emo, oracle_mod):
         emo.emo_set_wait_limit(4_000_000_000)
     check(torch, emo, oracle_mod, g, h, lv_dev, B, r_or)
     h.free()
+
+
+def test_random_dags(torch_cuda, emo, oracle_mod):
+    """Random DAGs of varying density, size and level count (merge operations, long segments, isolated nodes), every
+    output, through the kernels."""
+    torch = torch_cuda
+    done = 0
+    for seed in range(12):
+        rs = np.random.RandomState(2000 + seed)
+        n = int(rs.randint(30, 400))
+        L = int(rs.randint(2, 9))
+        g = W.random_dag(700 + seed, n, float(rs.choice([0.01, 0.03, 0.1, 0.3])), L=L, max_dur=int(rs.choice([5, 40, 100000])))
+        B = int(rs.choice([33, 96, 200]))
+        ldb = (B + 15) // 16 * 16
+        lvq = np.full((g.n, ldb), 0xFF, dtype=np.uint8)
+        lvq[:, :B] = rs.randint(0, L, size=(g.n, B))
+        lv_dev = torch.as_tensor(lvq, device="cuda")
+        r_or = oracle_mod.batch(g, lvq[:, :B].copy(), want_arrays=True)
+        h = emo.load_workload(g, emo.EMO_F_SPINE_STAGE(int(rs.choice([8, 16, 32]))))
+        if emo.emo_graph_spine(h)["ok"] == 1:      # very dense graphs go to the generic kernels: no spine program
+            check(torch, emo, oracle_mod, g, h, lv_dev, B, r_or, ldo=B + 2)
+            done += 1
+        h.free()
+    assert done >= 8
