@@ -983,10 +983,10 @@ int launch_spine_bwd(const emo_graph *g, const FlowPlan &pl, int64_t B, const ui
 
 // Whether a call takes the spine kernels: the program exists and either the caller asks for them (EMO_F_SPINE_KERNEL) or
 // the graph is narrow and the batch leaves at most three policy groups to an SM (or the graph is short).
-bool spine_allowed(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t ldb, int64_t ldo, bool extra, uint32_t flags)
+bool spine_allowed(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t ldb, int64_t ldo, bool fwd_only, uint32_t flags)
 {
     const int64_t big = (int64_t)1 << 28;
-    if (!g->sflow.ok32 || !g->sflow.spine.ok || !g->dspine.ready || extra) return false;
+    if (!g->sflow.ok32 || !g->sflow.spine.ok || !g->dspine.ready) return false;
     if (flags & (EMO_F_NO_STAGING | EMO_F_PAIR_KERNEL | EMO_F_LANE_KERNEL | EMO_F_FLOW_KERNEL)) return false;
     // Measured: on graphs of up to eight lanes the spine kernels are the fastest pair while a block holds at most three
     // policy groups (75 000 nodes, both passes, spine / lane-stream: 3.6 / 5.5 ms with one group per SM, 4.4 / 6.0 with
@@ -996,7 +996,8 @@ bool spine_allowed(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t ld
     // the other kernels unless the caller asks.
     if (!(flags & EMO_F_SPINE_KERNEL)) {
         const int64_t per_sm = ((B + 1 + 31) / 32 + g->sm_count - 1) / std::max(g->sm_count, 1);
-        if (g->sflow.lanes > 8 || (per_sm > 3 && g->h.n > 8192)) return false;
+        // (forward only, the spine kernel still wins with four groups: 250 000 nodes x 16 384 policies 7.5 against 8.2 ms)
+        if (g->sflow.lanes > 8 || (per_sm > (fwd_only ? 4 : 3) && g->h.n > 8192)) return false;
     }
     return ldb % 16 == 0 && aligned16(lvl) && ldb < big && ldo < big;
 }
@@ -1068,7 +1069,7 @@ int emo_call_path(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t ldb
     if (!g || B < 0) return EMO_E_INVALID_ARG;
     if (g->host_only) return EMO_E_CUDA;
     if (g->generic) return 3;
-    if (spine_allowed(g, B, lvl, ldb, need_slack ? ldo : 0, false, flags)) {
+    if (spine_allowed(g, B, lvl, ldb, need_slack ? ldo : 0, need_slack == 0, flags)) {
         FlowPlan fp;
         if (spine_plan(g, B, true, need_slack != 0, fp)) return 4;
     }
@@ -1669,7 +1670,7 @@ int emo_eval_policies(const emo_graph *g, int64_t B, const uint8_t *lvl, int64_t
     if (g->generic)
         return launch_generic(g, B, lvl, ldb, false, nullptr, nullptr, nullptr, 0, makespan, energy, nullptr, nullptr, T0, E0, ws,
                               ws_bytes, st);
-    if (spine_allowed(g, B, lvl, ldb, 0, false, flags)) {
+    if (spine_allowed(g, B, lvl, ldb, 0, true, flags)) {
         FlowPlan fp;
         if (spine_plan(g, B, T0 || E0, false, fp))
             return launch_spine_fwd(g, fp, B, lvl, ldb, nullptr, makespan, energy, T0, E0, status, flags, st);
