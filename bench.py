@@ -161,7 +161,7 @@ def other_workloads_leg(sm_mhz, hbm_gbs):
     import numpy as np
     import torch
     from paper_2607_12324_b200 import emo, workloads as W
-    names = {4: "32-bit spine", 3: "generic", 2: "32-bit lane-stream", 1: "staged 64-bit", 0: "plain 64-bit"}
+    names = {5: "32-bit spine forward + lane-stream backward", 4: "32-bit spine", 3: "generic", 2: "32-bit lane-stream", 1: "staged 64-bit", 0: "plain 64-bit"}
     out = []
     for name in ("cfg0-tiny", "cfg1-train", "cfg2-packed", "cfg3-8dev"):
         g = W.make_graph(name)
@@ -405,15 +405,15 @@ def main():
               "frac_of_binding": max(t_hbm, t_issue) / ms_per_step,
               "warp_costs_cycles": {k: round(v, 2) for k, v in costs.items()}}
     path = emo.emo_call_path(h, B, lv, ldb, B, True, args.call_flags)
-    if path == 2 and fl["steps"]:
+    if path in (2, 5) and fl["steps"]:
         bounds["cycles_per_schedule_step"] = {"forward": fwd * 1e-3 * sm_mhz * 1e6 / fl["steps"], "backward": bwd * 1e-3 * sm_mhz * 1e6 / fl["steps"]}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "int64", "data": "synthetic",
             "config": workload_config(args.workload, args.scale, g, B, ppm),
-            "details": {"kernels": {4: "32-bit spine", 3: "generic", 2: "32-bit lane-stream", 1: "staged 64-bit", 0: "plain 64-bit"}[path],
-                        "slack_sums": bool(args.sums), "lanes": fl["lanes"] if path == 2 else info.lanes,
-                        "steps": fl["steps"] if path == 2 else info.steps_fwd, "stage_steps": fl["K"], "barrier_steps": fl["sync"],
+            "details": {"kernels": {5: "32-bit spine forward + lane-stream backward", 4: "32-bit spine", 3: "generic", 2: "32-bit lane-stream", 1: "staged 64-bit", 0: "plain 64-bit"}[path],
+                        "slack_sums": bool(args.sums), "lanes": fl["lanes"] if path in (2, 5) else info.lanes,
+                        "steps": fl["steps"] if path in (2, 5) else info.steps_fwd, "stage_steps": fl["K"], "barrier_steps": fl["sync"],
                         "restore_rows": fl["pushes"], "depth": info.depth, "graph_load_s": t_load,
                         "workspace_gb": ws.numel() / 1e9,
                         "parallelism": "replicas" if world > 1 else "single"},
@@ -423,7 +423,7 @@ def main():
             "selected": {"index": int(sel[0].item()), "T": int(sel[1].item()), "E": float(selE.item()),
                          "T0": int(T0.item()), "E0": float(E0.item())}}
 
-    if path == 4:
+    if path in (4, 5):
         line["details"]["spine"] = emo.emo_graph_spine(h)
     # end to end through the host-buffer entry point: the levels come from pinned host memory every step, packed
     # at ceil(log2 L) bits each (the call spreads them to bytes on the device), per-policy results and the

@@ -433,7 +433,8 @@ int emo_set_pass_events(void *fwd_start, void *fwd_stop, void *bwd_start, void *
 
 /*
  * emo_call_path - which kernels emo_eval_policies (need_slack = 0) or emo_slack_batch (need_slack = 1)
- * would run for these arguments: 4 = the spine kernels, 2 = the 32-bit lane-stream kernels, 1 = the staged 64-bit kernels,
+ * would run for these arguments: 4 = the spine kernels, 5 = the forward spine kernel followed by the lane-stream backward
+ * kernel, 2 = the 32-bit lane-stream kernels, 1 = the staged 64-bit kernels,
  * 0 = the plain-load 64-bit kernels, 3 = the generic kernels (a graph beyond the on-chip schedules' limits, or
  * loaded with EMO_F_GENERIC); negative = an EMO_E_* code.  lvl may be any pointer with the
  * alignment of the real one.  For tests and reports; it launches nothing.

@@ -76,6 +76,7 @@ struct FlowParams {
     unsigned acc_all_off;                // backward with ES / LS / sums: where the heads' tails of all segments start inside them
     unsigned off_oring, oring_bytes;     // forward: per group and buffer of sums, a copy of the front of the stage (header, bounds, operations)
     int workers, nacc;                   // look-up / store warps per group, buffers of sums
+    int pair_rows;                       // forward spine kernel: number the restore rows as the paired lane-stream program does
 };
 
 __device__ __forceinline__ unsigned long long emo_lds_b64v(unsigned a)

@@ -87,7 +87,8 @@ constexpr uint32_t kOpOffMask = (1u << 29) - 1u;
 // segment's sum, written to the lane's slot and to a published slot.  A node with more operands gets
 // merge operations in front.  Backward, a value that a node of a much earlier stage reads (two stages
 // or more: a launch node and its kernels) is folded by the storing warps into a slot of that reader.
-constexpr int kSpOpWordsF = 8;        // a0, d0, a1, d1, lane slot, published slot, sum offset, flags | push row << 8 | pool index << 20
+constexpr int kSpOpWordsF = 8;        // a0, d0, a1, d1, lane slot, published slot, sum offset, flags | push row << 8 | push row in the
+                                      // paired numbering << 20 (both relative to the stage's base); terminal bounds are taken in order
 constexpr int kSpOpWordsB = 12;       // the same eight (flags | pop row << 8), then: slot to clear, lane's completion slot, where the head's
                                       // tail goes (beside X if members are folded, else nowhere), where it goes when all tails are kept
 constexpr int kSpSegWords = 4;        // lane | first position << 8 | members << 16 | flags << 24, sum offset, A_v low, high
@@ -120,6 +121,11 @@ struct Spine {
     std::vector<uint32_t> posw;       // [stages][lanes * K] position words
     std::vector<uint64_t> pool;       // [stages][max_pool] lbC of terminal nodes
     std::vector<int64_t> push_base;   // [stages + 1]
+    // the same restore rows numbered as a lane-stream program with stages of pair_K steps numbers them (per stage the
+    // lanes in order, a lane's rows by position): the forward spine kernel can then feed the lane-stream backward kernel
+    int pair_K = 0;
+    bool pair_ok = false;
+    std::vector<int64_t> pair_base;   // [stages] smallest such row of the stage's pushes
     SpineDir f, b;
 };
 
@@ -163,12 +169,13 @@ struct SpineIn {
     const std::vector<int64_t> *lbES = nullptr, *lbC = nullptr, *lbQin = nullptr, *lbQ = nullptr;
     const std::vector<int32_t> *step_of = nullptr, *lane_of = nullptr, *prev_on_lane = nullptr, *next_on_lane = nullptr, *pos_of = nullptr;
     const double *energy = nullptr;                                   // [n][L]
+    int pair_K = 0;                                                   // stage length of the lane-stream program to pair with (0: none)
 };
 int build_spine(const SpineIn &in, Spine &out, std::string &err);
 
 // Compiles g into a lane-stream program.  Returns EMO_OK with out.ok32 = false when the 32-bit
 // representation does not apply (spread too large, too many lanes); other codes are errors.
 int compile_flow(const HostGraph &g, const int64_t *lat, const double *energy, int lanes, int lookahead,
-                 int K, int sync, Flow &out, std::string &err, bool spine = false);
+                 int K, int sync, Flow &out, std::string &err, bool spine = false, int pair_K = 0);
 
 }  // namespace emo

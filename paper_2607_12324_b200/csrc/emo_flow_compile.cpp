@@ -64,7 +64,7 @@ void assign_slots(std::vector<SlotObj> &objs, int &n_tag, int &n_set)   // n_set
 }  // namespace
 
 int compile_flow(const HostGraph &g, const int64_t *lat, const double *energy, int lanes, int lookahead, int K, int sync,
-                 Flow &out, std::string &err, bool spine)
+                 Flow &out, std::string &err, bool spine, int pair_K)
 {
     out = Flow();
     const int32_t n = g.n;
@@ -571,6 +571,7 @@ int compile_flow(const HostGraph &g, const int64_t *lat, const double *energy, i
         in.next_on_lane = &next_on_lane;
         in.pos_of = &pos_of;
         in.energy = energy;
+        in.pair_K = pair_K;
         rc = build_spine(in, out.spine, err);
         if (rc != EMO_OK) return rc;
     }

@@ -181,6 +181,10 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_fwd(FlowParams p)
             const unsigned acc_a = smem0 + p.off_acc + (unsigned)(a * groups + group) * p.acc_bytes + (unsigned)lane * 4u;
             unsigned op_a = sta + p.off_ops;
             uint4 d0 = emo_lds128(op_a), d1 = emo_lds128(op_a + 16u);
+            // restore rows in the spine program's own numbering, or in that of the lane-stream program whose backward
+            // kernel will read them (pair_rows)
+            const unsigned push0 = p.pair_rows ? hd.w : hd.z, push_shift = p.pair_rows ? 20u : 8u;
+            unsigned tcount = 0;
             const long long tl0 = EMO_SCLK();
             for (int i = 0; i < n_ops; ++i) {
                 const uint4 c0 = d0, c1 = d1;
@@ -195,9 +199,9 @@ __global__ void __launch_bounds__(MAXT, 1) emo_spine_fwd(FlowParams p)
                 const unsigned y = max(emo_floor_sub(x0, c0.y), emo_floor_sub(x1, c0.w)) + S;
                 // the lane's previous value (always the first operand) goes to the restore list where the backward pass cannot
                 // derive it; no branch: a taken branch costs this lone warp more than the whole operation
-                emo_stg_u32_if(rst_lane, hd.z + ((fl >> 8) & 0xFFFu), ptile4, x0, (fl & emo::kSp_Push) && rst_lane);
+                emo_stg_u32_if(rst_lane, push0 + ((fl >> push_shift) & 0xFFFu), ptile4, x0, (fl & emo::kSp_Push) && rst_lane);
                 if (fl & emo::kSp_Terminal) {
-                    const unsigned pa = sta + p.off_tpool + (fl >> 20) * 8u;
+                    const unsigned pa = sta + p.off_tpool + (tcount++) * 8u;
                     const long long lb = (long long)((unsigned long long)emo_lds_u32(pa) | ((unsigned long long)emo_lds_u32(pa + 4u) << 32));
                     T = emo_max64(T, lb + (long long)(unsigned long long)y);
                 }

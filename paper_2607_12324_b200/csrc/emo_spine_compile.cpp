@@ -185,6 +185,30 @@ int build_spine(const SpineIn &in, Spine &out, std::string &err)
 
     // ---- forward operations -----------------------------------------------------------------------------
     // fixed slots: the lanes' values, a slot that stays zero, a slot nobody reads; published values behind them
+    // restore rows in the numbering of the lane-stream program to pair with: nodes whose start does not follow from the
+    // lane's value, per stage of pair_K steps the lanes in order, a lane's nodes by step
+    std::vector<int64_t> pair_row((size_t)n, -1);
+    out.pair_K = in.pair_K;
+    out.pair_ok = in.pair_K > 0;
+    out.pair_base.assign((size_t)stages, 0);
+    if (in.pair_K > 0) {
+        std::vector<int32_t> pushing;
+        for (int32_t v = 0; v < n; ++v)
+            if (!invertible(v)) pushing.push_back(v);
+        std::sort(pushing.begin(), pushing.end(), [&](int32_t a, int32_t b) {
+            const int sa = step_of[a] / in.pair_K, sb = step_of[b] / in.pair_K;
+            if (sa != sb) return sa < sb;
+            if (lane_of[a] != lane_of[b]) return lane_of[a] < lane_of[b];
+            return step_of[a] < step_of[b];
+        });
+        for (size_t i = 0; i < pushing.size(); ++i) pair_row[pushing[i]] = (int64_t)i;
+        std::vector<int64_t> lo((size_t)stages, -1);
+        for (int32_t v : pushing) {
+            const int st = stage_of(v);
+            if (lo[st] < 0 || pair_row[v] < lo[st]) lo[st] = pair_row[v];
+        }
+        for (int st = 0; st < stages; ++st) out.pair_base[st] = lo[st] < 0 ? 0 : lo[st];
+    }
     std::vector<std::vector<uint32_t>> opsF((size_t)stages), opsB((size_t)stages);
     std::vector<std::vector<uint64_t>> pools((size_t)stages);
     out.push_base.assign((size_t)stages + 1, 0);
@@ -237,9 +261,16 @@ int build_spine(const SpineIn &in, Spine &out, std::string &err)
                 ops.insert(ops.begin(), lane_op);
                 if (fpub[t] && s.readersF > 0) s.pubF = pool.take();
                 uint32_t fl = (s.flags & kSpSeg_PreB) ? 0u : kSp_NoSum;
-                if (!inv) fl |= kSp_Push | ((uint32_t)s.push << 8);
+                if (!inv) {
+                    fl |= kSp_Push | ((uint32_t)s.push << 8);
+                    if (in.pair_K > 0) {
+                        const int64_t rel = pair_row[h] - out.pair_base[st];
+                        if (rel < 0 || rel >= 4096) out.pair_ok = false;
+                        else fl |= (uint32_t)rel << 20;
+                    }
+                }
                 if (terminal) {
-                    fl |= kSp_Terminal | ((uint32_t)pools[st].size() << 20);
+                    fl |= kSp_Terminal;      // the kernel takes the stage's bounds in order
                     pools[st].push_back((uint64_t)lbC[t]);
                 }
                 if (s.push >= 4096 || pools[st].size() >= 4096) { err = "internal: spine stage too large"; return EMO_E_UNSUPPORTED; }

@@ -51,6 +51,7 @@ def run(view: dict, lv: np.ndarray, L: int, late_stores: bool = False) -> dict:
                 runsum = d if (pw & 1) else (runsum + d) & M32
                 if pw & 2:
                     acc[pw >> 16] = runsum
+        tcount = 0
         for i in range(int(view["n_ops_fwd"][st])):
             a0, d0, a1, d1, o_lane, o_pub, ao, fl = (int(x) for x in view["ops_fwd"][st, i])
             x0, x1 = slots[a0 // 128], slots[a1 // 128]
@@ -59,7 +60,8 @@ def run(view: dict, lv: np.ndarray, L: int, late_stores: bool = False) -> dict:
             if fl & 2:
                 restore[int(view["push_base"][st]) + ((fl >> 8) & 0xFFF)] = x0
             if fl & 4:
-                T = np.maximum(T, np.int64(view["pool"][st, fl >> 20]) + y.astype(np.int64))
+                T = np.maximum(T, np.int64(view["pool"][st, tcount]) + y.astype(np.int64))
+                tcount += 1
             slots[o_lane // 128] = y
             slots[o_pub // 128] = y
     for ln in range(lanes):

@@ -143,3 +143,30 @@ def test_random_dags(torch_cuda, emo, oracle_mod):
             done += 1
         h.free()
     assert done >= 8
+
+
+def test_forward_spine_feeds_lane_stream_backward(torch_cuda, emo, oracle_mod):
+    """Four policy groups per SM on a narrow graph: the forward spine kernel writes the restore list in the lane-stream
+    program's numbering and the lane-stream backward kernel reads it.  Same slack matrix as the lane-stream pair alone,
+    and the oracle's on sampled policies."""
+    torch = torch_cuda
+    g = W.make_graph("cfg4-llm", 0.1)
+    B = 16384
+    lv_dev = W.policies_for(g, B=B, device="cuda")
+    h = emo.load_workload(g)
+    path = emo.emo_call_path(h, B, lv_dev, lv_dev.stride(0), B, True, 0)
+    assert path in (2, 5)
+    if path != 5:
+        pytest.skip("this graph's lane-stream program does not share the spine program's schedule")
+    r_pair = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, want=("slack",), sums=False, base=True)
+    r_flow = gpu_slack_batch(torch, emo, h, lv_dev, B, g.n, want=("slack",), sums=False, base=True, flags=emo.EMO_F_FLOW_KERNEL)
+    assert np.array_equal(r_pair["makespan"], r_flow["makespan"]) and r_pair["T0"] == r_flow["T0"]
+    np.testing.assert_allclose(r_pair["energy"], r_flow["energy"], rtol=E_RTOL)
+    assert np.array_equal(r_pair["slack"], r_flow["slack"])
+    cols = np.linspace(0, B - 1, 24).astype(np.int64)
+    sub = lv_dev[:, torch.as_tensor(cols, device="cuda")].contiguous().cpu().numpy()
+    r_or = oracle_mod.batch(g, sub, want_arrays=True, threads=os.cpu_count() or 1)
+    assert np.array_equal(r_pair["makespan"][cols], r_or["makespan"])
+    np.testing.assert_allclose(r_pair["energy"][cols], r_or["energy"], rtol=E_RTOL)
+    assert np.array_equal(r_pair["slack"][:, cols], r_or["slack"])
+    h.free()
