@@ -287,7 +287,7 @@ def test_cfg4_full_size_sampled(torch_cuda, emo, oracle_mod, golden):
     E0 = torch.zeros(1, dtype=torch.float64, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     ws = torch.empty(emo.emo_workspace_bytes(h, B, 1), dtype=torch.uint8, device="cuda")
-    assert emo.emo_call_path(h, B, lv_dev, lv_dev.stride(0), B, True, 0) == 2, "the largest workload takes the 32-bit kernels"
+    assert emo.emo_call_path(h, B, lv_dev, lv_dev.stride(0), B, True, 0) in (2, 5), "the largest workload takes the 32-bit kernels"
     emo.emo_slack_batch(h, B, lv_dev, lv_dev.stride(0), None, None, slack, B, T, E, None, None, ws, status, T0=T0, E0=E0)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
